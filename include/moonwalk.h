@@ -1,0 +1,187 @@
+/*
+ * moonwalk.h -- C ABI of the B200 (sm_100a) Moonwalk gradient library.
+ *
+ * Moonwalk (mixed mode, Section 4.1 of the paper) computes the parameter gradients of a
+ * sequential network x_i = f_i(x_{i-1}; theta_i) with scalar loss J in three phases:
+ *   Phase I   forward pass that keeps only the residuals the input-cotangent path needs
+ *             (one sign bit per activation, Section "Residual Impact");
+ *   Phase II  reverse pass for the input cotangent h_0 = dJ/dx_0 only; on the way it writes
+ *             cotangent checkpoints (Section 4.1, "gradient checkpointing in Phase II") and
+ *             the fragments of non-submersive layers (Section 5.1);
+ *   Phase III forward sweep (Algorithm 1): per layer recompute x_i, carry the cotangent with
+ *             h_i = vijp(f_i, x_{i-1}, h_{i-1}) (Eq. "h_i") and form g_i = vjp(f_i, theta_i, h_i)
+ *             (Eq. "g_i").
+ *
+ * Conventions
+ *   - Layer i: z = linear_i(x_{i-1}), x_i = phi(z).  No bias.  Dense weights are row-major
+ *     [n_out][n_in], z = x W^T.  Convolutions follow Lemma 1: channel-last activations
+ *     [B][H][W][C], kernel w[kh][kw][c_in][c_out], x'[i',c'] = sum w[j,c,c'] x[s i'+j-p, c],
+ *     zero padding.  The head (MW_HEAD_LINEAR) is a dense layer on the flattened activation,
+ *     allowed only as the last layer; it needs no vijp.
+ *   - "positive" means z > 0 strictly; 0, -0.0 and NaN take the negative branch.
+ *   - Every device buffer is allocated and owned by the caller.  The library allocates no
+ *     device memory: all per-step state lives in the caller's `workspace`.
+ *   - Calls enqueue work on `stream` and return without synchronising, unless stated.
+ *     Argument errors are returned synchronously.  Device-side conditions (a bounded wait that
+ *     ran out, an inverse that did not converge) are recorded in a status word inside the
+ *     workspace and read back by mw_last_device_status().
+ *   - Nothing aborts, throws or prints.
+ */
+#ifndef MOONWALK_H_
+#define MOONWALK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mw_net mw_net; /* opaque, host side; owns no device memory */
+
+typedef enum {
+  MW_OK = 0,
+  MW_ERR_INVALID_ARG = 1,    /* null pointer, bad enum, inconsistent sizes               */
+  MW_ERR_UNSUPPORTED = 2,    /* layer / size combination this build has no kernel for   */
+  MW_ERR_WORKSPACE = 3,      /* workspace null, misaligned (256 B) or too small          */
+  MW_ERR_STATE = 4,          /* sweep called without a matching mw_input_cotangent       */
+  MW_ERR_NOT_SUBMERSIVE = 5, /* a layer's Jacobian could not be inverted to tolerance    */
+  MW_ERR_TIMEOUT = 6,        /* a bounded device-side wait expired                       */
+  MW_ERR_CUDA = 7            /* a CUDA runtime / driver call failed                      */
+} mw_status;
+
+typedef enum { MW_DENSE = 0, MW_CONV2D = 1, MW_HEAD_LINEAR = 2 } mw_kind;
+typedef enum { MW_ACT_NONE = 0, MW_ACT_LEAKY_RELU = 1, MW_ACT_RELU = 2 } mw_act;
+
+/* Storage / arithmetic:
+ *   MW_F64          x, W, targets, g0, dW double; arithmetic double (CUDA cores).
+ *   MW_F32          x, W, targets, g0, dW float; products accurate to fp32 (tensor cores with
+ *                   operands split into bf16 terms, fp32 accumulate; or CUDA-core FMA).
+ *   MW_BF16_F32ACC  x, W bf16; targets, g0, dW float; activations between layers bf16; the
+ *                   cotangent chain (h, W^-1), fragments and checkpoints fp32-accurate.    */
+typedef enum { MW_F64 = 0, MW_F32 = 1, MW_BF16_F32ACC = 2 } mw_prec;
+
+/* MW_LOSS_HALF_SSE   J = 0.5 * sum (y-t)^2 over all B*n entries; target = [B][n] floats.
+ * MW_LOSS_MSE_MEAN   J = mean (y-t)^2 over all B*n entries.
+ * MW_LOSS_XENT_MEAN  J = mean over the batch of -log softmax(y_b)[label_b]; target = int32[B]. */
+typedef enum { MW_LOSS_HALF_SSE = 0, MW_LOSS_MSE_MEAN = 1, MW_LOSS_XENT_MEAN = 2 } mw_loss;
+
+typedef enum { MW_BACKEND_AUTO = 0, MW_BACKEND_SIMT = 1, MW_BACKEND_TENSOR = 2 } mw_backend;
+
+typedef struct {
+  int32_t kind;          /* mw_kind */
+  int32_t act;           /* mw_act  */
+  double slope;          /* leaky-ReLU negative slope (ignored otherwise)                 */
+  int32_t n_in, n_out;   /* dense / head: features in and out (dense must be square)      */
+  int32_t H, W, C_in, C_out, k, stride, pad; /* conv: input H x W x C_in, kernel k x k    */
+} mw_layer_desc;
+
+typedef struct {
+  int32_t prec;            /* mw_prec */
+  int32_t loss;            /* mw_loss */
+  int32_t reseed_every;    /* K: Phase II keeps the full cotangent h_l for every l that is a
+                              multiple of K (0 < l < L) and Phase III restarts its recursion
+                              from it.  0 = never: the literal Algorithm 1.                 */
+  int32_t conv_vijp_iters; /* fixed-point updates of the stride-1 convolution vijp          */
+  int32_t backend;         /* mw_backend; AUTO = tensor cores when the sizes allow          */
+  int32_t inverse_iters;   /* Newton-Schulz steps for W^-1 (0 = default for the precision)  */
+  int32_t resident_inverse;/* 1: mw_input_cotangent computes every layer's W^-1 (and split
+                              operands) once and keeps them in the workspace; 0: the sweep
+                              builds them layer by layer in a transient slot (lean memory) */
+  int32_t reserved;
+} mw_net_opts;
+
+/* Build a host-side description.  `batch` is fixed per net.  Returns MW_ERR_UNSUPPORTED for
+ * shapes outside: dense layers square; convolutions stride 1, k = 2*pad+1, C_in = C_out;
+ * head only as the last layer; all layers of one net share `prec`. */
+mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers, int32_t batch,
+                        const mw_net_opts* opts, mw_net** out);
+void mw_net_destroy(mw_net* net);
+
+/* Bytes of workspace (256-byte aligned device memory) needed by the Moonwalk calls and by
+ * mw_backprop_reference.  `residual_bytes` (may be NULL) receives the part of each that must
+ * survive between the phases: [0] Moonwalk (sign bits + fragments + cotangent checkpoints),
+ * [1] backprop (stored activations + sign bits). */
+mw_status mw_workspace_bytes(const mw_net* net, size_t* moonwalk_bytes, size_t* backprop_bytes,
+                             size_t residual_bytes[2]);
+
+/* Phases I and II (Section 4.1): g0 = dJ/dx_0.
+ *   params       host array of n_layers DEVICE pointers to the weights (read-only).
+ *   x            device, [B][n_0] (or NHWC), storage type of `prec`.
+ *   loss_target  device, see mw_loss.
+ *   g0_out       device, [B][n_0], double (MW_F64) or float.
+ *   loss_out     device pointer to one double receiving J, or NULL.
+ * Also fills the workspace with the residual stores the sweep consumes. */
+mw_status mw_input_cotangent(mw_net* net, const void* const* params, const void* x,
+                             const void* loss_target, void* g0_out, double* loss_out,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Phase III (Algorithm 1): all parameter gradients from x and g0.
+ *   dW_out  host array of n_layers DEVICE pointers, each shaped like its weight, double
+ *           (MW_F64) or float; overwritten.  A NULL entry skips storing that layer's gradient
+ *           (gradients need not coexist, Section 4.3 last paragraph but one).
+ * Requires the workspace last written by mw_input_cotangent on the same net (MW_ERR_STATE). */
+mw_status mw_forward_sweep(mw_net* net, const void* const* params, const void* x, const void* g0,
+                           void* const* dW_out, void* workspace, size_t workspace_bytes,
+                           void* stream);
+
+/* Plain reverse mode ("Backprop", Appendix "Complexity Analysis" item 1): forward storing every
+ * layer input, backward with both vjps.  Same kernels, for the memory and runtime comparison. */
+mw_status mw_backprop_reference(mw_net* net, const void* const* params, const void* x,
+                                const void* loss_target, void* const* dW_out, double* loss_out,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Canonical copy of layer `layer`'s sign bits to HOST memory: uint32 words [rows][ceil(n/32)],
+ * rows = B (dense) or B*H*W (conv), bit (j & 31) of word (j >> 5) = (z_j > 0).  Synchronises
+ * the stream.  `rows_out`/`words_per_row_out` may be NULL. */
+mw_status mw_export_masks(const mw_net* net, const void* workspace, int32_t layer,
+                          uint32_t* host_words, size_t host_words_capacity, int32_t* rows_out,
+                          int32_t* words_per_row_out, void* stream);
+
+/* Synchronise `stream`, then return the first device-side error recorded in the workspace
+ * (MW_OK if none) and clear it.  `detail` (may be NULL) receives kernel-specific words. */
+mw_status mw_last_device_status(const mw_net* net, void* workspace, void* stream,
+                                uint32_t detail[4]);
+
+const char* mw_status_string(mw_status s);
+
+/* ---- stand-alone forms of the residual-store and elementwise kernels ------------------- */
+
+/* Sign-bit pack (Section "Residual Impact"): words[r][w] bit b = (z[r][32 w + b] > 0).
+ * z: device [rows][cols], dtype 0 = double, 1 = float, 2 = bf16; cols need not be a multiple of
+ * 32 (padding bits are zero).  words: device uint32 [rows][ceil(cols/32)]. */
+mw_status mw_pack_sign_bits(const void* z, int32_t dtype, int64_t rows, int32_t cols,
+                            uint32_t* words, void* stream);
+
+/* ReLU fragment store (Section 5.1 applied to ReLU): for every row r, the output-cotangent
+ * values at dead units (mask bit 0), in increasing column order, are written from
+ * vals[off[r]]; cnt[r] = number of dead units, off = exclusive prefix sum of cnt over rows.
+ * h: device float [rows][cols]; words: sign bits as above; cnt, off: device uint32[rows];
+ * vals: device float, capacity >= rows*cols.  total_out (device uint32, may be NULL) = sum cnt.
+ * scratch: device, >= 4*(rows+1024) bytes. */
+mw_status mw_relu_fragment_compact(const float* h, const uint32_t* words, int64_t rows,
+                                   int32_t cols, uint32_t* cnt, uint32_t* off, float* vals,
+                                   uint32_t* total_out, void* scratch, size_t scratch_bytes,
+                                   void* stream);
+
+/* Activation vijp (Eq. "h_i" restricted to phi): h_out = g_z (bit 1) or g_z / slope (bit 0) for
+ * leaky-ReLU; for ReLU (act = MW_ACT_RELU) live units take g_z and dead units pop
+ * vals[off[r] + rank], and gz_out (may be NULL) receives g_z with exact zeros at dead units. */
+mw_status mw_activation_vijp(const float* gz, const uint32_t* words, int64_t rows, int32_t cols,
+                             int32_t act, float slope, const uint32_t* off, const float* vals,
+                             float* h_out, float* gz_out, void* stream);
+
+/* Tensor-core product used by every dense step, exposed for unit parity tests:
+ *   D[M][N] (float, row-major) = A * B with A given as [M][K] (a_mn = 0) or [K][M] (a_mn = 1)
+ *   and B given as [N][K] (b_mn = 0) or [K][N] (b_mn = 1), all row-major float in device
+ *   memory.  terms = 1, 2 or 3: each operand is split into that many bf16 terms and the
+ *   1, 3 or 6 leading cross products are accumulated in fp32 (terms = 3 is fp32-accurate).
+ *   scratch: device, >= 6*(M*K + N*K) bytes + 1024.  M, N, K multiples of 64. */
+mw_status mw_gemm_split_bf16(const float* A, int32_t a_mn, const float* B, int32_t b_mn, float* D,
+                             int32_t M, int32_t N, int32_t K, int32_t terms, void* scratch,
+                             size_t scratch_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOONWALK_H_ */

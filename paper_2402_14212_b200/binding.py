@@ -1,0 +1,296 @@
+"""ctypes binding over libmoonwalk.so: argument marshalling only.
+
+Every step of the Moonwalk path runs inside the CUDA library; this module converts Python
+objects (torch tensors used purely as device buffers) into the pointers and sizes of the C ABI
+declared in include/moonwalk.h.  There is no CPU fallback: if the library is missing or a CUDA
+device is absent, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoonwalk.so")
+
+MW_OK = 0
+STATUS_NAMES = ["MW_OK", "MW_ERR_INVALID_ARG", "MW_ERR_UNSUPPORTED", "MW_ERR_WORKSPACE",
+                "MW_ERR_STATE", "MW_ERR_NOT_SUBMERSIVE", "MW_ERR_TIMEOUT", "MW_ERR_CUDA"]
+KIND = {"dense": 0, "conv2d": 1, "head": 2}
+ACT = {"none": 0, "leaky_relu": 1, "relu": 2}
+PREC = {"f64": 0, "f32": 1, "bf16_f32acc": 2}
+LOSS = {"half_sse": 0, "mse_mean": 1, "xent_mean": 2}
+BACKEND = {"auto": 0, "simt": 1, "tensor": 2}
+
+
+class MwError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        name = STATUS_NAMES[code] if 0 <= code < len(STATUS_NAMES) else str(code)
+        super().__init__(f"{where}: {name}")
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("act", C.c_int32), ("slope", C.c_double),
+                ("n_in", C.c_int32), ("n_out", C.c_int32), ("H", C.c_int32), ("W", C.c_int32),
+                ("C_in", C.c_int32), ("C_out", C.c_int32), ("k", C.c_int32),
+                ("stride", C.c_int32), ("pad", C.c_int32)]
+
+
+class NetOpts(C.Structure):
+    _fields_ = [("prec", C.c_int32), ("loss", C.c_int32), ("reseed_every", C.c_int32),
+                ("conv_vijp_iters", C.c_int32), ("backend", C.c_int32),
+                ("inverse_iters", C.c_int32), ("resident_inverse", C.c_int32),
+                ("reserved", C.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load the CUDA library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2402_14212_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+        L.mw_net_create.argtypes = [C.POINTER(LayerDesc), i32, i32, C.POINTER(NetOpts), C.POINTER(vp)]
+        L.mw_net_destroy.argtypes = [vp]
+        L.mw_net_destroy.restype = None
+        L.mw_workspace_bytes.argtypes = [vp, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
+        L.mw_input_cotangent.argtypes = [vp, C.POINTER(vp), vp, vp, vp, vp, vp, sz, vp]
+        L.mw_forward_sweep.argtypes = [vp, C.POINTER(vp), vp, vp, C.POINTER(vp), vp, sz, vp]
+        L.mw_backprop_reference.argtypes = [vp, C.POINTER(vp), vp, vp, C.POINTER(vp), vp, vp, sz, vp]
+        L.mw_export_masks.argtypes = [vp, vp, i32, vp, sz, C.POINTER(i32), C.POINTER(i32), vp]
+        L.mw_last_device_status.argtypes = [vp, vp, vp, C.POINTER(C.c_uint32)]
+        L.mw_status_string.argtypes = [i32]
+        L.mw_status_string.restype = C.c_char_p
+        L.mw_pack_sign_bits.argtypes = [vp, i32, i64, i32, vp, vp]
+        L.mw_relu_fragment_compact.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.mw_activation_vijp.argtypes = [vp, vp, i64, i32, i32, C.c_float, vp, vp, vp, vp, vp]
+        L.mw_gemm_split_bf16.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, vp, sz, vp]
+        for name in ("mw_step_host",):
+            if hasattr(L, name):
+                getattr(L, name).argtypes = [vp, C.POINTER(vp), vp, sz, vp, sz, vp, vp, vp,
+                                             C.POINTER(vp), vp, vp, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != MW_OK:
+        raise MwError(code, where)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _stream_handle(stream=None) -> int:
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _ptr_array(tensors: Sequence) -> "C.Array":
+    arr = (C.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = _ptr(t)
+    return arr
+
+
+def make_layer_descs(layers) -> "C.Array":
+    arr = (LayerDesc * len(layers))()
+    for i, l in enumerate(layers):
+        arr[i] = LayerDesc(KIND[l.kind], ACT[l.act], float(l.slope), int(l.n_in), int(l.n_out),
+                           int(l.H), int(l.W), int(l.C_in), int(l.C_out), int(l.k),
+                           int(l.stride), int(l.pad))
+    return arr
+
+
+class Net:
+    """Host-side handle of one network (mw_net).  Owns no device memory."""
+
+    def __init__(self, layers, batch: int, prec: str, loss: str, reseed_every: int = 4,
+                 conv_vijp_iters: int = 10, backend: str = "auto", inverse_iters: int = 0,
+                 resident_inverse: bool = True):
+        self.layers = list(layers)
+        self.batch = int(batch)
+        self.prec, self.loss = prec, loss
+        self._h = C.c_void_p()
+        opts = NetOpts(PREC[prec], LOSS[loss], int(reseed_every), int(conv_vijp_iters),
+                       BACKEND[backend], int(inverse_iters), int(bool(resident_inverse)), 0)
+        descs = make_layer_descs(self.layers)
+        _check(lib().mw_net_create(descs, len(self.layers), self.batch, C.byref(opts),
+                                   C.byref(self._h)), "mw_net_create")
+
+    def close(self):
+        if self._h:
+            lib().mw_net_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- sizes -------------------------------------------------------------------------
+    def workspace_bytes(self):
+        a, b = C.c_size_t(), C.c_size_t()
+        res = (C.c_size_t * 2)()
+        _check(lib().mw_workspace_bytes(self._h, C.byref(a), C.byref(b), res), "mw_workspace_bytes")
+        return int(a.value), int(b.value), (int(res[0]), int(res[1]))
+
+    def grad_dtype(self):
+        import torch
+        return torch.float64 if self.prec == "f64" else torch.float32
+
+    def storage_dtype(self):
+        import torch
+        return {"f64": torch.float64, "f32": torch.float32, "bf16_f32acc": torch.bfloat16}[self.prec]
+
+    def alloc_workspace(self, which: str = "moonwalk", device="cuda"):
+        import torch
+        a, b, _ = self.workspace_bytes()
+        n = a if which == "moonwalk" else (b if which == "backprop" else max(a, b))
+        return torch.empty(n + 256, dtype=torch.uint8, device=device)
+
+    @staticmethod
+    def _ws(workspace):
+        p = int(workspace.data_ptr())
+        ap = (p + 255) // 256 * 256
+        return ap, workspace.numel() - (ap - p)
+
+    # ---- the three calls ------------------------------------------------------------------
+    def input_cotangent(self, params, x, target, workspace, g0_out=None, loss_out=None, stream=None):
+        import torch
+        if g0_out is None:
+            g0_out = torch.empty(x.shape, dtype=self.grad_dtype(), device=x.device)
+        wp, wb = self._ws(workspace)
+        _check(lib().mw_input_cotangent(self._h, _ptr_array(params), _ptr(x), _ptr(target),
+                                        _ptr(g0_out), _ptr(loss_out), wp, wb,
+                                        _stream_handle(stream)), "mw_input_cotangent")
+        return g0_out
+
+    def forward_sweep(self, params, x, g0, workspace, dW_out=None, stream=None):
+        import torch
+        if dW_out is None:
+            dW_out = [torch.empty(p.shape, dtype=self.grad_dtype(), device=p.device) for p in params]
+        wp, wb = self._ws(workspace)
+        _check(lib().mw_forward_sweep(self._h, _ptr_array(params), _ptr(x), _ptr(g0),
+                                      _ptr_array(dW_out), wp, wb, _stream_handle(stream)),
+               "mw_forward_sweep")
+        return dW_out
+
+    def backprop_reference(self, params, x, target, workspace, dW_out=None, loss_out=None,
+                           stream=None):
+        import torch
+        if dW_out is None:
+            dW_out = [torch.empty(p.shape, dtype=self.grad_dtype(), device=p.device) for p in params]
+        wp, wb = self._ws(workspace)
+        _check(lib().mw_backprop_reference(self._h, _ptr_array(params), _ptr(x), _ptr(target),
+                                           _ptr_array(dW_out), _ptr(loss_out), wp, wb,
+                                           _stream_handle(stream)), "mw_backprop_reference")
+        return dW_out
+
+    def export_masks(self, workspace, layer: int, stream=None) -> np.ndarray:
+        l = self.layers[layer]
+        if l.kind == "conv2d":
+            rows, cols = self.batch * l.H * l.W, l.C_out
+        else:
+            rows, cols = self.batch, l.n_out
+        wpr = (cols + 31) // 32
+        out = np.zeros((rows, wpr), dtype=np.uint32)
+        wp, _ = self._ws(workspace)
+        r, w = C.c_int32(), C.c_int32()
+        _check(lib().mw_export_masks(self._h, wp, layer, out.ctypes.data, out.size, C.byref(r),
+                                     C.byref(w), _stream_handle(stream)), "mw_export_masks")
+        assert (r.value, w.value) == (rows, wpr)
+        return out
+
+    def last_device_status(self, workspace, stream=None):
+        wp, _ = self._ws(workspace)
+        detail = (C.c_uint32 * 4)()
+        code = lib().mw_last_device_status(self._h, wp, _stream_handle(stream), detail)
+        return code, list(detail)
+
+
+# ---- stand-alone kernels -----------------------------------------------------------------
+def pack_sign_bits(z, words=None, stream=None):
+    import torch
+    dt = {torch.float64: 0, torch.float32: 1, torch.bfloat16: 2}[z.dtype]
+    rows, cols = z.shape
+    if words is None:
+        words = torch.zeros((rows, (cols + 31) // 32), dtype=torch.int32, device=z.device)
+    _check(lib().mw_pack_sign_bits(_ptr(z), dt, rows, cols, _ptr(words), _stream_handle(stream)),
+           "mw_pack_sign_bits")
+    return words
+
+
+def relu_fragment_compact(h, words, stream=None):
+    import torch
+    rows, cols = h.shape
+    dev = h.device
+    cnt = torch.zeros(max(rows, 1), dtype=torch.int32, device=dev)
+    off = torch.zeros(max(rows, 1), dtype=torch.int32, device=dev)
+    vals = torch.zeros(max(rows * cols, 1), dtype=torch.float32, device=dev)
+    total = torch.zeros(1, dtype=torch.int32, device=dev)
+    scratch = torch.empty(4 * (rows + 1024), dtype=torch.uint8, device=dev)
+    _check(lib().mw_relu_fragment_compact(_ptr(h), _ptr(words), rows, cols, _ptr(cnt), _ptr(off),
+                                          _ptr(vals), _ptr(total), _ptr(scratch), scratch.numel(),
+                                          _stream_handle(stream)), "mw_relu_fragment_compact")
+    return cnt[:rows], off[:rows], vals, total
+
+
+def activation_vijp(gz, words, act: str, slope: float = 0.0, off=None, vals=None, want_gz=False,
+                    stream=None):
+    import torch
+    rows, cols = gz.shape
+    h = torch.empty_like(gz)
+    gzo = torch.empty_like(gz) if want_gz else None
+    _check(lib().mw_activation_vijp(_ptr(gz), _ptr(words), rows, cols, ACT[act], float(slope),
+                                    _ptr(off), _ptr(vals), _ptr(h), _ptr(gzo),
+                                    _stream_handle(stream)), "mw_activation_vijp")
+    return (h, gzo) if want_gz else h
+
+
+def gemm_split_bf16(A, B, a_mn: bool, b_mn: bool, terms: int, stream=None):
+    """D = op(A) op(B)^T-style product on the tensor cores (see moonwalk.h)."""
+    import torch
+    M = A.shape[1] if a_mn else A.shape[0]
+    K = A.shape[0] if a_mn else A.shape[1]
+    N = B.shape[1] if b_mn else B.shape[0]
+    D = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    scratch = torch.empty(6 * (M * K + N * K) + 4096, dtype=torch.uint8, device=A.device)
+    _check(lib().mw_gemm_split_bf16(_ptr(A), int(a_mn), _ptr(B), int(b_mn), _ptr(D), M, N, K,
+                                    int(terms), _ptr(scratch), scratch.numel(),
+                                    _stream_handle(stream)), "mw_gemm_split_bf16")
+    return D
+
+
+# ---- moving a synthetic problem onto the device -------------------------------------------
+def to_device(problem, device="cuda"):
+    """Returns (params, x, target) as torch tensors in the problem's storage types."""
+    import torch
+    st = {"f64": torch.float64, "f32": torch.float32, "bf16_f32acc": torch.bfloat16}[problem.prec]
+    gt = torch.float64 if problem.prec == "f64" else torch.float32
+    params = [torch.from_numpy(np.ascontiguousarray(p)).to(st).to(device).contiguous()
+              for p in problem.params]
+    x = torch.from_numpy(np.ascontiguousarray(problem.x)).to(st).to(device).contiguous()
+    if problem.loss == "xent_mean":
+        target = torch.from_numpy(problem.target.astype(np.int32)).to(device)
+    else:
+        target = torch.from_numpy(np.ascontiguousarray(problem.target)).to(gt).to(device).contiguous()
+    return params, x, target
+
+
+def net_for(problem, backend="auto", resident_inverse=True, inverse_iters=0) -> Net:
+    return Net(problem.layers, problem.batch, problem.prec, problem.loss,
+               reseed_every=problem.reseed_every, conv_vijp_iters=problem.conv_vijp_iters,
+               backend=backend, inverse_iters=inverse_iters, resident_inverse=resident_inverse)

@@ -1,0 +1,61 @@
+// Host-side network description and workspace layout (internal).
+#pragma once
+#include <vector>
+
+#include "mw_common.cuh"
+
+namespace mw {
+
+struct LayerInfo {
+  int64_t rows;        // B (dense, head) or B*H*W (conv): rows of the [rows][cols] view of z
+  int cols;            // n_out (dense, head) or C_out (conv)
+  int wpr;             // mask words per row
+  int64_t in_elems;    // elements of x_{l-1}
+  int64_t out_elems;   // elements of x_l
+  int64_t w_elems;     // elements of the weight
+  int inv_n;           // size of the square block that is inverted (n, or C for conv), 0 for head
+};
+
+struct Region {
+  size_t off = 0, bytes = 0;
+};
+
+struct Layout {
+  size_t total = 0;
+  size_t residual = 0;  // bytes that must survive between the phases
+  Region status, partials;
+  std::vector<Region> mask, frag_cnt, frag_off, frag_vals, reseed, stored_act;
+  Region frag_total, h_last;
+  Region act[2], cot[2], z, gz, aux0, aux1;  // aux: conv vijp iterate / h', wgrad partials
+  std::vector<Region> inv;                   // per layer (resident) or all the same slot
+  Region inv_scratch;
+  // tensor-core backend operands (bf16 term planes)
+  std::vector<Region> w_planes;              // split weights (MW_F32), per layer or one slot
+  Region xp[2], hp[2], gzp, ns_r, ns_x;      // activation / cotangent / g_z planes, NS scratch
+};
+
+}  // namespace mw
+
+struct mw_net {
+  std::vector<mw_layer_desc> layers;
+  std::vector<mw::LayerInfo> info;
+  int L = 0, B = 0;
+  mw_net_opts opts{};
+  int backend = MW_BACKEND_SIMT;
+  size_t es = 4;   // bytes of the working scalar (8 for MW_F64)
+  mw::Layout mwl, bpl;
+  // state
+  const void* ws_done = nullptr;   // workspace that holds a finished Phase I+II
+  const void* x_done = nullptr;
+  void* tc = nullptr;              // tensor-core backend private state
+};
+
+namespace mw {
+inline bool is_reseed(const mw_net* n, int l_out) {   // l_out = index of x_l / h_l, 1..L-1
+  const int K = n->opts.reseed_every;
+  return K > 0 && l_out > 0 && l_out < n->L && (l_out % K) == 0;
+}
+template <typename T>
+inline T* at(void* ws, const Region& r) { return reinterpret_cast<T*>(static_cast<char*>(ws) + r.off); }
+inline DeviceStatus* status_of(void* ws, const Layout& l) { return at<DeviceStatus>(ws, l.status); }
+}  // namespace mw

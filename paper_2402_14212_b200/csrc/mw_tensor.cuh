@@ -1,0 +1,23 @@
+// Tensor-core (tcgen05) backend: internal interface between the C-ABI layer and the pipelines.
+#pragma once
+#include "mw_common.cuh"
+#include "mw_net.cuh"
+
+namespace mw {
+
+// true when every layer of the net has a tensor-core path (dense, sizes multiples of 64,
+// MW_F32 or MW_BF16_F32ACC)
+bool tensor_supported(const mw_net* n);
+// appends the backend's transient regions to `lay` starting at byte `start`; sets lay.total
+void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start);
+void tensor_destroy(mw_net* n);
+
+mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const void* x,
+                                 const void* target, void* g0, double* loss_out, void* ws,
+                                 cudaStream_t s);
+mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void* x, const void* g0,
+                               void* const* dW, void* ws, cudaStream_t s);
+mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, const void* target,
+                          void* const* dW, double* loss_out, void* ws, cudaStream_t s);
+
+}  // namespace mw

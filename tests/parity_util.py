@@ -1,0 +1,70 @@
+"""Helpers shared by the GPU parity tests: run the CUDA path through the C ABI, run the oracle on
+the same arrays, compare."""
+import numpy as np
+
+from oracle import moonwalk_oracle as O
+from paper_2402_14212_b200 import binding as mwb
+
+
+def run_gpu(problem, backend="auto", resident_inverse=True, inverse_iters=0, backprop=True,
+            want_masks=True):
+    import torch
+    net = mwb.net_for(problem, backend=backend, resident_inverse=resident_inverse,
+                      inverse_iters=inverse_iters)
+    params, x, target = mwb.to_device(problem)
+    ws = net.alloc_workspace("both")
+    loss = torch.zeros(1, dtype=torch.float64, device="cuda")
+    g0 = net.input_cotangent(params, x, target, ws, loss_out=loss)
+    dW = net.forward_sweep(params, x, g0, ws)
+    code, detail = net.last_device_status(ws)
+    out = dict(net=net, status=code, detail=detail, loss=float(loss.item()),
+               g0=g0.double().cpu().numpy(), dW=[d.double().cpu().numpy() for d in dW])
+    if want_masks:
+        out["masks"] = [net.export_masks(ws, l) for l in range(len(problem.layers))]
+    if backprop:
+        loss2 = torch.zeros(1, dtype=torch.float64, device="cuda")
+        dWb = net.backprop_reference(params, x, target, ws, loss_out=loss2)
+        code2, _ = net.last_device_status(ws)
+        out.update(bp_status=code2, bp_loss=float(loss2.item()),
+                   bp_dW=[d.double().cpu().numpy() for d in dWb])
+    return out
+
+
+def oracle_masks_from_words(problem, words_list):
+    """GPU-exported words -> boolean masks shaped like each layer's z (for mask replay)."""
+    ms = []
+    for layer, words in zip(problem.layers, words_list):
+        if layer.kind == "conv2d":
+            ho, wo = layer.out_hw()
+            m = O.unpack_mask(words, layer.C_out).reshape(problem.batch, ho, wo, layer.C_out)
+        else:
+            m = O.unpack_mask(words, layer.n_out)
+        ms.append(m)
+    return ms
+
+
+def oracle_reference(problem, masks=None):
+    return O.backprop(problem.layers, problem.params, problem.x, problem.target, problem.loss,
+                      masks=masks)
+
+
+def mask_disagreement(problem, gpu_words, ref):
+    """Hamming distance between GPU masks and the oracle's own masks, and the largest |z| (relative
+    to the row rms) at a disagreeing element."""
+    flips, worst = 0, 0.0
+    for l, (layer, words) in enumerate(zip(problem.layers, gpu_words)):
+        if layer.act == "none":
+            continue
+        z = ref["z"][l].reshape(words.shape[0], -1)
+        mg = O.unpack_mask(words, z.shape[1])
+        mo = O.sign_mask(z)
+        d = mg != mo
+        if d.any():
+            flips += int(d.sum())
+            rms = np.sqrt((z * z).mean(axis=1, keepdims=True))
+            worst = max(worst, float((np.abs(z) / rms)[d].max()))
+    return flips, worst
+
+
+def grad_errors(gpu_dW, ref_dW):
+    return [O.normwise_error(a.reshape(b.shape), b) for a, b in zip(gpu_dW, ref_dW)]

@@ -1,0 +1,91 @@
+"""The C-ABI library loads and exports every entry point the header declares; host-side argument
+checks reject bad calls before any GPU work (runs without a GPU)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2402_14212_b200 import binding as mwb
+from paper_2402_14212_b200 import synth as S
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in os.listdir(inc):
+        if f.endswith(".h"):
+            text = open(os.path.join(inc, f)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(mw_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
+
+
+def test_library_exports_every_declared_symbol():
+    L = mwb.lib()
+    syms = declared_symbols()
+    assert len(syms) >= 12
+    for s in syms:
+        assert hasattr(L, s), f"{s} declared in include/ but not exported"
+
+
+def test_status_strings():
+    L = mwb.lib()
+    seen = {L.mw_status_string(i) for i in range(8)}
+    assert len(seen) == 8 and b"ok" in seen
+
+
+def test_net_create_rejects_bad_descriptions():
+    with pytest.raises(mwb.MwError) as e:
+        mwb.Net([S.Layer(S.DENSE, S.ACT_LEAKY, 0.1, 8, 12)], 4, S.F64, S.LOSS_MSE_MEAN)
+    assert e.value.code == 2          # non-square dense layer: unsupported
+    with pytest.raises(mwb.MwError) as e:
+        mwb.Net([S.Layer(S.HEAD, S.ACT_NONE, 0.0, 8, 3), S.Layer(S.DENSE, S.ACT_LEAKY, 0.1, 3, 3)],
+                4, S.F64, S.LOSS_MSE_MEAN)
+    assert e.value.code == 2          # head must be last
+    with pytest.raises(mwb.MwError) as e:
+        mwb.Net([S.Layer(S.DENSE, S.ACT_LEAKY, 0.1, 8, 8), S.Layer(S.DENSE, S.ACT_LEAKY, 0.1, 16, 16)],
+                4, S.F64, S.LOSS_MSE_MEAN)
+    assert e.value.code == 1          # widths do not chain
+    with pytest.raises(mwb.MwError):
+        mwb.Net([S.Layer(S.CONV2D, S.ACT_LEAKY, 0.1, H=8, W=8, C_in=4, C_out=4, k=3, stride=2, pad=1)],
+                2, S.F32, S.LOSS_MSE_MEAN)
+
+
+def test_workspace_sizes_and_residual_accounting():
+    p = S.deep_mlp(depth=8, n=128, batch=64, reseed_every=4)
+    net = mwb.net_for(p, backend="simt")
+    mw_b, bp_b, (mw_res, bp_res) = net.workspace_bytes()
+    masks = 8 * 64 * 128 // 8
+    # Moonwalk keeps sign bits + one cotangent checkpoint (l = 4); backprop keeps 7 activations
+    assert mw_res >= masks + 64 * 128 * 4 and mw_res < masks + 2 * 64 * 128 * 4 + 16384
+    assert bp_res >= masks + 7 * 64 * 128 * 4
+    assert mw_b > mw_res and bp_b > bp_res
+    p0 = S.deep_mlp(depth=8, n=128, batch=64, reseed_every=0)
+    _, _, (r0, _) = mwb.net_for(p0, backend="simt").workspace_bytes()
+    assert r0 < mw_res                 # literal Algorithm 1 keeps only the sign bits
+
+
+def test_calls_reject_null_and_small_workspace_without_touching_a_gpu():
+    p = S.tiny_mlp()
+    net = mwb.net_for(p)
+    L = mwb.lib()
+    arr = (C.c_void_p * 4)(1, 1, 1, 1)
+    # null x
+    assert L.mw_input_cotangent(net._h, arr, None, 1, 1, None, 256, 1 << 30, None) == 1
+    # null workspace / misaligned / too small
+    assert L.mw_input_cotangent(net._h, arr, 1, 1, 1, None, None, 1 << 30, None) == 3
+    assert L.mw_input_cotangent(net._h, arr, 1, 1, 1, None, 257, 1 << 30, None) == 3
+    assert L.mw_input_cotangent(net._h, arr, 1, 1, 1, None, 256, 1024, None) == 3
+    # sweep before any cotangent pass
+    assert L.mw_forward_sweep(net._h, arr, 1, 1, arr, 256, 1 << 30, None) == 4
+    # null entry in params
+    arr0 = (C.c_void_p * 4)(1, None, 1, 1)
+    assert L.mw_backprop_reference(net._h, arr0, 1, 1, arr, None, 256, 1 << 30, None) == 1
+    # stand-alone kernels: negative sizes, empty inputs
+    assert L.mw_pack_sign_bits(None, 1, -1, 4, None, None) == 1
+    assert L.mw_pack_sign_bits(None, 1, 0, 4, None, None) == 0
+    assert L.mw_pack_sign_bits(1, 7, 2, 4, 1, None) == 1
+    assert L.mw_activation_vijp(1, 1, 2, 4, 1, 0.0, None, None, 1, None, None) == 1   # slope 0
