@@ -7,4 +7,3 @@ mw_status tensor_input_cotangent(mw_net*, const void* const*, const void*, const
 mw_status tensor_forward_sweep(mw_net*, const void* const*, const void*, const void*, void* const*, void*, cudaStream_t) { return MW_ERR_UNSUPPORTED; }
 mw_status tensor_backprop(mw_net*, const void* const*, const void*, const void*, void* const*, double*, void*, cudaStream_t) { return MW_ERR_UNSUPPORTED; }
 }
-extern "C" mw_status mw_gemm_split_bf16(const float*, int32_t, const float*, int32_t, float*, int32_t, int32_t, int32_t, int32_t, void*, size_t, void*) { return MW_ERR_UNSUPPORTED; }
