@@ -1,9 +1,531 @@
+// Tensor-core pipelines of the three calls for dense nets (MW_F32 and MW_BF16_F32ACC).
+//
+// Every matrix product is one launch of the tcgen05 kernel (mw_tc_gemm.cu) with the step's
+// elementwise work fused into its epilogue:
+//   Phase I    z = x W^T          -> sign words + x_l term planes                (Section 4.1)
+//   Phase II   h_{l-1} = g_z W    -> h (fp32, where a store needs it) + next g_z term planes
+//   prep       W^-1 by Newton-Schulz, X <- X + X (I - W X), low precision first
+//   sweep      recompute (as Phase I, reading the stored sign words)             (Algorithm 1)
+//              g_z = h W^-1       -> leaky vijp fused: h_l term planes + g_z term planes (Eq. "h_i")
+//              dW = g_z^T x       -> fp32 gradient                               (Eq. "g_i")
+// ReLU layers take the stand-alone fragment kernels after a plain fp32 epilogue.
+#include "mw_tc_gemm.cuh"
 #include "mw_tensor.cuh"
+
 namespace mw {
-bool tensor_supported(const mw_net*) { return false; }
-void tensor_layout(mw_net*, bool, Layout& lay, size_t start) { lay.total = start; }
-void tensor_destroy(mw_net*) {}
-mw_status tensor_input_cotangent(mw_net*, const void* const*, const void*, const void*, void*, double*, void*, cudaStream_t) { return MW_ERR_UNSUPPORTED; }
-mw_status tensor_forward_sweep(mw_net*, const void* const*, const void*, const void*, void* const*, void*, cudaStream_t) { return MW_ERR_UNSUPPORTED; }
-mw_status tensor_backprop(mw_net*, const void* const*, const void*, const void*, void* const*, double*, void*, cudaStream_t) { return MW_ERR_UNSUPPORTED; }
+
+namespace {
+
+struct TensorState {
+  TcMapCache* cache = nullptr;
+};
+
+struct Prec {
+  int px;    // activation / weight terms (recompute, Phase I)
+  int ph;    // cotangent-chain terms (h and W^-1 in the dense vijp)
+  int pg2;   // g_z terms in Phase II
+  int pgw;   // g_z terms in the weight vjp
+  int pw;    // weight terms
+};
+
+Prec prec_of(const mw_net* n) {
+  if (n->opts.prec == MW_F32) return Prec{3, 3, 3, 3, 3};
+  return Prec{1, 2, 2, 1, 1};
 }
+
+struct NsStep { int pr, pu; };   // terms in the residual product (W, X) and the update (X, R)
+
+int ns_schedule(const mw_net* n, NsStep* out) {
+  int cnt;
+  if (n->opts.prec == MW_F32) {
+    const NsStep d[] = {{1, 1}, {2, 1}, {3, 1}, {3, 2}};
+    cnt = 4;
+    for (int i = 0; i < cnt; ++i) out[i] = d[i];
+  } else {
+    const NsStep d[] = {{1, 1}, {2, 1}, {2, 1}};
+    cnt = 3;
+    for (int i = 0; i < cnt; ++i) out[i] = d[i];
+  }
+  const int want = n->opts.inverse_iters;
+  if (want > 0) {
+    // more steps repeat the most accurate one; fewer drop the cheap leading ones last
+    if (want > 16) return -1;
+    NsStep full[16];
+    const NsStep last = out[cnt - 1];
+    if (want >= cnt) {
+      for (int i = 0; i < cnt; ++i) full[i] = out[i];
+      for (int i = cnt; i < want; ++i) full[i] = last;
+    } else {
+      for (int i = 0; i < want - 1; ++i) full[i] = out[i];
+      full[want - 1] = last;
+    }
+    for (int i = 0; i < want; ++i) out[i] = full[i];
+    cnt = want;
+  }
+  return cnt;
+}
+
+template <typename TW>
+__global__ void __launch_bounds__(1024)
+frob_scale_kernel(const TW* __restrict__ W, int64_t n2, int n, float* __restrict__ c_out) {
+  __shared__ double red[1024];
+  double a = 0.0;
+  for (int64_t i = threadIdx.x; i < n2; i += 1024) {
+    const double v = (double)to_f32(W[i]);
+    a += v * v;
+  }
+  red[threadIdx.x] = a;
+  __syncthreads();
+  for (int o = 512; o; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *c_out = red[0] > 0.0 ? (float)((double)n / red[0]) : 0.f;
+}
+
+// X0 = c W^T (fp32) through a 32x32 shared tile
+template <typename TW>
+__global__ void __launch_bounds__(256)
+x0_kernel(const TW* __restrict__ W, int n, const float* __restrict__ c, float* __restrict__ X) {
+  __shared__ float tile[32][33];
+  const int bx = blockIdx.x * 32, by = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int r = ty; r < 32; r += 8) tile[r][tx] = to_f32(W[(int64_t)(by + r) * n + bx + tx]);
+  __syncthreads();
+  const float cc = *c;
+  for (int r = ty; r < 32; r += 8) X[(int64_t)(bx + r) * n + by + tx] = cc * tile[tx][r];
+}
+
+__global__ void residual_gate_kernel(const double* __restrict__ sumsq, int n, double limit,
+                                     DeviceStatus* st, int layer) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    const double r = sqrt(*sumsq / (double)n);   // rms singular value of I - W X
+    if (!(r <= limit)) record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)layer, __float_as_uint((float)r), 3u, 0u);
+  }
+}
+
+TcOperand operand(const void* base, int rows, int cols, int planes, bool mn) {
+  TcOperand o;
+  o.base = base;
+  o.rows = rows;
+  o.cols = cols;
+  o.planes = planes;
+  o.plane_stride = (int64_t)rows * cols;
+  o.mn_major = mn;
+  return o;
+}
+
+struct Ctx {
+  mw_net* n;
+  const Layout* lay;
+  void* ws;
+  cudaStream_t s;
+  TcMapCache* cache;
+  DeviceStatus* st;
+  Prec pr;
+  int B, dim;          // batch, width
+  int64_t bn;          // B * width
+  int64_t nn;          // width^2
+  template <typename T> T* at(const Region& r) const { return mw::at<T>(ws, r); }
+};
+
+Ctx make_ctx(mw_net* n, const Layout& lay, void* ws, cudaStream_t s) {
+  Ctx c;
+  c.n = n; c.lay = &lay; c.ws = ws; c.s = s;
+  c.cache = static_cast<TensorState*>(n->tc)->cache;
+  c.st = status_of(ws, lay);
+  c.pr = prec_of(n);
+  c.B = n->B;
+  c.dim = n->layers[0].n_in;
+  c.bn = (int64_t)c.B * c.dim;
+  c.nn = (int64_t)c.dim * c.dim;
+  return c;
+}
+
+// weight operand of layer l with `terms` terms (MW_F32: split planes in the workspace, made here
+// unless resident and already made; bf16: the caller's array itself)
+mw_status weight_planes(const Ctx& c, int l, const void* W, bool make, const __nv_bfloat16** out) {
+  if (c.n->opts.prec == MW_F32) {
+    __nv_bfloat16* p = c.at<__nv_bfloat16>(c.lay->w_planes[l]);
+    if (make) MW_TRY(split_planes((const float*)W, c.nn, p, 3, c.nn, c.s));
+    *out = p;
+  } else {
+    *out = (const __nv_bfloat16*)W;
+  }
+  return MW_OK;
+}
+
+// W^-1 of layer l into the layer's inverse region as `ph` term planes (row-major X = W^-1)
+mw_status newton_schulz(const Ctx& c, int l, const void* W, const __nv_bfloat16* Wp) {
+  const Layout& lay = *c.lay;
+  const int d = c.dim;
+  float* X = c.at<float>(lay.ns_x);
+  // ns_r holds the residual planes [3][n*n] followed by two iterate plane sets [2][3][n*n]
+  __nv_bfloat16* xbase = c.at<__nv_bfloat16>(lay.ns_r) + 3 * c.nn;
+  __nv_bfloat16* Xp[2] = {xbase, xbase + 3 * c.nn};
+  __nv_bfloat16* Rp = c.at<__nv_bfloat16>(lay.ns_r);
+  double* sumsq = reinterpret_cast<double*>(c.at<char>(lay.inv_scratch));
+  float* cscale = reinterpret_cast<float*>(c.at<char>(lay.inv_scratch) + 64);
+  __nv_bfloat16* dst = c.at<__nv_bfloat16>(lay.inv[l]);
+
+  NsStep sched[16];
+  const int steps = ns_schedule(c.n, sched);
+  if (steps < 1) return MW_ERR_INVALID_ARG;
+  if (c.n->opts.prec == MW_F32) {
+    frob_scale_kernel<float><<<1, 1024, 0, c.s>>>((const float*)W, c.nn, d, cscale);
+    x0_kernel<float><<<dim3(d / 32, d / 32), 256, 0, c.s>>>((const float*)W, d, cscale, X);
+  } else {
+    frob_scale_kernel<__nv_bfloat16><<<1, 1024, 0, c.s>>>((const __nv_bfloat16*)W, c.nn, d, cscale);
+    x0_kernel<__nv_bfloat16><<<dim3(d / 32, d / 32), 256, 0, c.s>>>((const __nv_bfloat16*)W, d, cscale, X);
+  }
+  MW_TRY(launch_ok());
+  int have = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;   // terms of X currently split
+  MW_TRY(split_planes(X, c.nn, Xp[0], have, c.nn, c.s));
+  int cur = 0;
+  for (int it = 0; it < steps; ++it) {
+    const bool last = it + 1 == steps;
+    const int pw = c.pr.pw < sched[it].pr ? c.pr.pw : sched[it].pr;
+    // R = I - W X
+    MW_CUDA_OK(cudaMemsetAsync(sumsq, 0, sizeof(double), c.s));
+    TcEpilogue er;
+    er.mode = TC_EPI_RESID;
+    er.planes = Rp; er.n_planes = sched[it].pu; er.plane_stride = c.nn;
+    er.sumsq = sumsq;
+    MW_TRY(tc_gemm(c.cache, operand(Wp, d, d, pw, false), operand(Xp[cur], d, d, sched[it].pr, true),
+                   d, d, d, er, c.st, c.s));
+    if (last) {
+      // the update squares this residual: gate on it so a diverging layer is reported
+      const double limit = c.n->opts.prec == MW_F32 ? 2e-3 : 2e-2;
+      residual_gate_kernel<<<1, 32, 0, c.s>>>(sumsq, d, limit, c.st, l);
+    }
+    // X' = X + X R
+    int next_terms = c.pr.ph;
+    if (!last) next_terms = sched[it + 1].pr > sched[it + 1].pu ? sched[it + 1].pr : sched[it + 1].pu;
+    TcEpilogue eu;
+    eu.mode = TC_EPI_PLAIN;
+    eu.addend = X;
+    eu.out_f32 = last ? nullptr : X;
+    eu.planes = last ? dst : Xp[cur ^ 1];
+    eu.n_planes = next_terms;
+    eu.plane_stride = c.nn;
+    MW_TRY(tc_gemm(c.cache, operand(Xp[cur], d, d, sched[it].pu, false),
+                   operand(Rp, d, d, sched[it].pu, true), d, d, d, eu, c.st, c.s));
+    cur ^= 1;
+    have = next_terms;
+  }
+  (void)have;
+  return MW_OK;
+}
+
+mw_status prep_layer(const Ctx& c, int l, const void* W, bool make_w) {
+  const __nv_bfloat16* Wp = nullptr;
+  MW_TRY(weight_planes(c, l, W, make_w, &Wp));
+  return newton_schulz(c, l, W, Wp);
+}
+
+// x0 (caller's array) as a K-major / MN-major operand base with px terms
+mw_status input_planes(const Ctx& c, const void* x, const __nv_bfloat16** out) {
+  if (c.n->opts.prec == MW_F32) {
+    __nv_bfloat16* p = c.at<__nv_bfloat16>(c.lay->xp[0]);
+    MW_TRY(split_planes((const float*)x, c.bn, p, c.pr.px, c.bn, c.s));
+    *out = p;
+  } else {
+    *out = (const __nv_bfloat16*)x;
+  }
+  return MW_OK;
+}
+
+// forward pass shared by Phase I and backprop's forward; y (fp32 network output) lands in lay.z
+mw_status forward_pass(const Ctx& c, const void* const* params, const void* x, bool store_acts) {
+  const Layout& lay = *c.lay;
+  const int L = c.n->L, d = c.dim;
+  const __nv_bfloat16* xin = nullptr;
+  MW_TRY(input_planes(c, x, &xin));
+  const bool resident = c.n->opts.resident_inverse != 0;
+  for (int l = 0; l < L; ++l) {
+    const mw_layer_desc& ld = c.n->layers[l];
+    const __nv_bfloat16* Wp = nullptr;
+    // resident + Moonwalk: the planes were made by the prep at the top of mw_input_cotangent
+    MW_TRY(weight_planes(c, l, params[l], !(resident && !store_acts), &Wp));
+    __nv_bfloat16* xout = (store_acts && l + 1 < L) ? c.at<__nv_bfloat16>(lay.stored_act[l + 1])
+                                                   : c.at<__nv_bfloat16>(lay.xp[(l + 1) & 1]);
+    TcEpilogue e;
+    e.mode = TC_EPI_FWD;
+    e.mask = c.at<uint32_t>(lay.mask[l]);
+    e.write_mask = 1;
+    e.act = ld.act;
+    e.slope = (float)ld.slope;
+    if (l + 1 < L) {
+      e.planes = xout; e.n_planes = c.pr.px; e.plane_stride = c.bn;
+    } else {
+      e.out_f32 = c.at<float>(lay.z);
+    }
+    MW_TRY(tc_gemm(c.cache, operand(xin, c.B, d, c.pr.px, false), operand(Wp, d, d, c.pr.pw, false),
+                   c.B, d, d, e, c.st, c.s));
+    xin = xout;
+  }
+  return MW_OK;
+}
+
+// top of the reverse pass: loss, h_L (fp32 in cot[0]) and g_z of the last layer as term planes
+mw_status loss_and_top(const Ctx& c, const void* target, double* loss_out, bool fragments) {
+  const Layout& lay = *c.lay;
+  const int L = c.n->L, d = c.dim;
+  const mw_layer_desc& ld = c.n->layers[L - 1];
+  float* h = c.at<float>(lay.cot[0]);
+  MW_TRY(loss_cotangent<float>(c.at<float>(lay.z), target, c.B, d, c.n->opts.loss, h,
+                               c.at<double>(lay.partials), loss_out, c.s));
+  const uint32_t* words = c.at<uint32_t>(lay.mask[L - 1]);
+  if (fragments && ld.act == MW_ACT_RELU) {
+    MW_TRY(fragment_offsets(words, c.B, d, c.at<uint32_t>(lay.frag_cnt[L - 1]),
+                            c.at<uint32_t>(lay.frag_off[L - 1]),
+                            c.at<uint32_t>(lay.frag_total) + (L - 1), nullptr, 0, c.s));
+    MW_TRY(fragment_compact<float>(h, words, c.B, d, c.at<uint32_t>(lay.frag_off[L - 1]),
+                                   c.at<float>(lay.frag_vals[L - 1]), c.s));
+  }
+  float* g = c.at<float>(lay.cot[1]);
+  const float* src = h;
+  if (ld.act != MW_ACT_NONE) {
+    MW_TRY(scale_by_mask<float>(h, words, c.B, d, ld.act, ld.slope, g, c.s));
+    src = g;
+  }
+  return split_planes(src, c.bn, c.at<__nv_bfloat16>(lay.hp[0]), c.pr.pg2, c.bn, c.s);
+}
+
+}  // namespace
+
+bool tensor_supported(const mw_net* n) {
+  if (n->opts.prec != MW_F32 && n->opts.prec != MW_BF16_F32ACC) return false;
+  if (n->opts.loss == MW_LOSS_XENT_MEAN) return false;
+  const int d = n->layers[0].n_in;
+  for (const auto& l : n->layers) {
+    if (l.kind != MW_DENSE) return false;
+    if (l.n_in != d || d % 64 != 0) return false;
+    if (l.act == MW_ACT_LEAKY_RELU && !(l.slope != 0.0)) return false;
+  }
+  return true;
+}
+
+void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
+  struct B2 {
+    size_t cur;
+    Region take(size_t bytes) {
+      Region r; r.off = cur; r.bytes = bytes; cur = align_up(cur + bytes, 256); return r;
+    }
+  } b{start};
+  if (!n->tc) {
+    TensorState* t = new TensorState();
+    t->cache = tc_cache_create();
+    n->tc = t;
+  }
+  const Prec pr = prec_of(n);
+  const int L = n->L;
+  const size_t d = (size_t)n->layers[0].n_in;
+  const size_t bn = (size_t)n->B * d, nn = d * d;
+  const bool resident = n->opts.resident_inverse != 0;
+  lay.z = b.take(4 * bn);                                   // fp32 network output / g_z scratch
+  for (int i = 0; i < 2; ++i) lay.cot[i] = b.take(4 * bn);  // fp32 cotangent scratch
+  for (int i = 0; i < 2; ++i) lay.xp[i] = b.take(2 * (size_t)pr.px * bn);
+  const int hpl = pr.ph > pr.pg2 ? pr.ph : pr.pg2;
+  for (int i = 0; i < 2; ++i) lay.hp[i] = b.take(2 * (size_t)hpl * bn);
+  lay.gzp = b.take(2 * (size_t)(pr.pgw > pr.pg2 ? pr.pgw : pr.pg2) * bn);
+  if (n->opts.prec == MW_F32) {
+    if (resident) {
+      for (int l = 0; l < L; ++l) lay.w_planes[l] = b.take(2 * 3 * nn);
+    } else {
+      Region slot = b.take(2 * 3 * nn);
+      for (int l = 0; l < L; ++l) lay.w_planes[l] = slot;
+    }
+  }
+  if (!backprop) {
+    if (resident) {
+      for (int l = 0; l < L; ++l) lay.inv[l] = b.take(2 * (size_t)pr.ph * nn);
+    } else {
+      Region slot = b.take(2 * (size_t)pr.ph * nn);
+      for (int l = 0; l < L; ++l) lay.inv[l] = slot;
+    }
+    lay.ns_x = b.take(4 * nn);
+    lay.ns_r = b.take(2 * 9 * nn);      // R planes [3] + two iterate plane sets [2][3]
+    lay.inv_scratch = b.take(256);
+  }
+  lay.total = b.cur;
+}
+
+void tensor_destroy(mw_net* n) {
+  if (n->tc) {
+    TensorState* t = static_cast<TensorState*>(n->tc);
+    tc_cache_destroy(t->cache);
+    delete t;
+    n->tc = nullptr;
+  }
+}
+
+mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const void* x,
+                                 const void* target, void* g0, double* loss_out, void* ws,
+                                 cudaStream_t s) {
+  const Layout& lay = n->mwl;
+  Ctx c = make_ctx(n, lay, ws, s);
+  const int L = n->L, d = c.dim;
+  MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
+  const bool resident = n->opts.resident_inverse != 0;
+  if (resident)
+    for (int l = 0; l < L; ++l) MW_TRY(prep_layer(c, l, params[l], true));
+  MW_TRY(forward_pass(c, params, x, false));                 // Phase I
+  MW_TRY(loss_and_top(c, target, loss_out, true));
+  // Phase II: g_z planes ping-pong between hp[0] and hp[1]
+  int cur = 0;
+  for (int l = L - 1; l >= 0; --l) {
+    const __nv_bfloat16* Wp = nullptr;
+    MW_TRY(weight_planes(c, l, params[l], !resident, &Wp));
+    TcEpilogue e;
+    e.mode = TC_EPI_BWD;
+    float* hf = nullptr;
+    if (l == 0) {
+      hf = (float*)g0;
+    } else {
+      const mw_layer_desc& below = n->layers[l - 1];
+      if (is_reseed(n, l)) hf = c.at<float>(lay.reseed[l]);
+      else if (below.act == MW_ACT_RELU) hf = c.at<float>(lay.cot[0]);
+      e.act = below.act;
+      e.slope = (float)below.slope;
+      e.mask = c.at<uint32_t>(lay.mask[l - 1]);
+      e.planes = c.at<__nv_bfloat16>(lay.hp[cur ^ 1]);
+      e.n_planes = c.pr.pg2;
+      e.plane_stride = c.bn;
+    }
+    e.out_f32 = hf;
+    MW_TRY(tc_gemm(c.cache, operand(c.at<__nv_bfloat16>(lay.hp[cur]), c.B, d, c.pr.pg2, false),
+                   operand(Wp, d, d, c.pr.pw, true), c.B, d, d, e, c.st, s));
+    if (l > 0 && n->layers[l - 1].act == MW_ACT_RELU) {
+      const uint32_t* words = c.at<uint32_t>(lay.mask[l - 1]);
+      MW_TRY(fragment_offsets(words, c.B, d, c.at<uint32_t>(lay.frag_cnt[l - 1]),
+                              c.at<uint32_t>(lay.frag_off[l - 1]),
+                              c.at<uint32_t>(lay.frag_total) + (l - 1), nullptr, 0, s));
+      MW_TRY(fragment_compact<float>(hf, words, c.B, d, c.at<uint32_t>(lay.frag_off[l - 1]),
+                                     c.at<float>(lay.frag_vals[l - 1]), s));
+    }
+    cur ^= 1;
+  }
+  return MW_OK;
+}
+
+mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void* x, const void* g0,
+                               void* const* dW, void* ws, cudaStream_t s) {
+  const Layout& lay = n->mwl;
+  Ctx c = make_ctx(n, lay, ws, s);
+  const int L = n->L, d = c.dim;
+  const bool resident = n->opts.resident_inverse != 0;
+  const __nv_bfloat16* xin = nullptr;
+  MW_TRY(input_planes(c, x, &xin));
+  MW_TRY(split_planes((const float*)g0, c.bn, c.at<__nv_bfloat16>(lay.hp[0]), c.pr.ph, c.bn, s));
+  for (int l = 0; l < L; ++l) {
+    const mw_layer_desc& ld = n->layers[l];
+    const uint32_t* words = c.at<uint32_t>(lay.mask[l]);
+    const __nv_bfloat16* Wp = nullptr;
+    if (resident) MW_TRY(weight_planes(c, l, params[l], false, &Wp));
+    else {
+      MW_TRY(weight_planes(c, l, params[l], true, &Wp));
+      MW_TRY(newton_schulz(c, l, params[l], Wp));
+    }
+    const __nv_bfloat16* hin = c.at<__nv_bfloat16>(lay.hp[l & 1]);
+    __nv_bfloat16* hout = c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]);
+    __nv_bfloat16* xout = c.at<__nv_bfloat16>(lay.xp[(l + 1) & 1]);
+    __nv_bfloat16* gzp = c.at<__nv_bfloat16>(lay.gzp);
+    const bool more = l + 1 < L;
+    const bool reseed_next = more && is_reseed(n, l + 1);
+    // recompute x_{l+1} (not needed after the last layer)
+    if (more) {
+      TcEpilogue e;
+      e.mode = TC_EPI_FWD;
+      e.mask = const_cast<uint32_t*>(words);
+      e.write_mask = 0;
+      e.act = ld.act;
+      e.slope = (float)ld.slope;
+      e.planes = xout; e.n_planes = c.pr.px; e.plane_stride = c.bn;
+      MW_TRY(tc_gemm(c.cache, operand(xin, c.B, d, c.pr.px, false), operand(Wp, d, d, c.pr.pw, false),
+                     c.B, d, d, e, c.st, s));
+    }
+    // dense vijp g_z = h W^-1, with the activation's vijp behind it
+    const TcOperand hop = operand(hin, c.B, d, c.pr.ph, false);
+    const TcOperand iop = operand(c.at<__nv_bfloat16>(lay.inv[l]), d, d, c.pr.ph, true);
+    if (ld.act == MW_ACT_RELU) {
+      float* gzf = c.at<float>(lay.z);
+      float* hf = c.at<float>(lay.cot[1]);
+      TcEpilogue e;
+      e.mode = TC_EPI_PLAIN;
+      e.out_f32 = gzf;
+      MW_TRY(tc_gemm(c.cache, hop, iop, c.B, d, d, e, c.st, s));
+      MW_TRY(activation_vijp<float>(gzf, words, c.B, d, MW_ACT_RELU, 0.0,
+                                    c.at<uint32_t>(lay.frag_off[l]), c.at<float>(lay.frag_vals[l]),
+                                    hf, gzf, s));
+      if (more && !reseed_next) MW_TRY(split_planes(hf, c.bn, hout, c.pr.ph, c.bn, s));
+      if (dW[l]) MW_TRY(split_planes(gzf, c.bn, gzp, c.pr.pgw, c.bn, s));
+    } else {
+      TcEpilogue e;
+      e.mode = TC_EPI_VIJP;
+      e.act = ld.act;
+      e.slope = (float)ld.slope;
+      e.mask = const_cast<uint32_t*>(words);
+      if (more && !reseed_next) { e.planes2 = hout; e.n_planes2 = c.pr.ph; e.plane_stride2 = c.bn; }
+      if (dW[l]) { e.planes = gzp; e.n_planes = c.pr.pgw; e.plane_stride = c.bn; }
+      MW_TRY(tc_gemm(c.cache, hop, iop, c.B, d, d, e, c.st, s));
+    }
+    if (reseed_next)
+      MW_TRY(split_planes(c.at<float>(lay.reseed[l + 1]), c.bn, hout, c.pr.ph, c.bn, s));
+    // weight vjp dW = g_z^T x
+    if (dW[l]) {
+      TcEpilogue e;
+      e.mode = TC_EPI_PLAIN;
+      e.out_f32 = (float*)dW[l];
+      MW_TRY(tc_gemm(c.cache, operand(gzp, c.B, d, c.pr.pgw, true), operand(xin, c.B, d, c.pr.px, true),
+                     d, d, c.B, e, c.st, s));
+    }
+    xin = xout;
+  }
+  return MW_OK;
+}
+
+mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, const void* target,
+                          void* const* dW, double* loss_out, void* ws, cudaStream_t s) {
+  const Layout& lay = n->bpl;
+  Ctx c = make_ctx(n, lay, ws, s);
+  const int L = n->L, d = c.dim;
+  MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
+  MW_TRY(forward_pass(c, params, x, true));
+  MW_TRY(loss_and_top(c, target, loss_out, false));
+  const __nv_bfloat16* x0p = nullptr;
+  if (n->opts.prec == MW_F32) x0p = c.at<__nv_bfloat16>(lay.xp[0]);   // split by forward_pass
+  else x0p = (const __nv_bfloat16*)x;
+  const bool resident = n->opts.resident_inverse != 0;
+  int cur = 0;
+  for (int l = L - 1; l >= 0; --l) {
+    const __nv_bfloat16* gz = c.at<__nv_bfloat16>(lay.hp[cur]);
+    const __nv_bfloat16* xl = l == 0 ? x0p : c.at<__nv_bfloat16>(lay.stored_act[l]);
+    if (dW[l]) {
+      TcEpilogue e;
+      e.mode = TC_EPI_PLAIN;
+      e.out_f32 = (float*)dW[l];
+      MW_TRY(tc_gemm(c.cache, operand(gz, c.B, d, c.pr.pgw, true), operand(xl, c.B, d, c.pr.px, true),
+                     d, d, c.B, e, c.st, s));
+    }
+    if (l > 0) {
+      const __nv_bfloat16* Wp = nullptr;
+      MW_TRY(weight_planes(c, l, params[l], !resident, &Wp));
+      const mw_layer_desc& below = n->layers[l - 1];
+      TcEpilogue e;
+      e.mode = TC_EPI_BWD;
+      e.act = below.act;
+      e.slope = (float)below.slope;
+      e.mask = c.at<uint32_t>(lay.mask[l - 1]);
+      e.planes = c.at<__nv_bfloat16>(lay.hp[cur ^ 1]);
+      e.n_planes = c.pr.pg2;
+      e.plane_stride = c.bn;
+      MW_TRY(tc_gemm(c.cache, operand(gz, c.B, d, c.pr.pg2, false), operand(Wp, d, d, c.pr.pw, true),
+                     c.B, d, d, e, c.st, s));
+      cur ^= 1;
+    }
+  }
+  return MW_OK;
+}
+
+}  // namespace mw

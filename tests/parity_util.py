@@ -68,3 +68,26 @@ def mask_disagreement(problem, gpu_words, ref):
 
 def grad_errors(gpu_dW, ref_dW):
     return [O.normwise_error(a.reshape(b.shape), b) for a, b in zip(gpu_dW, ref_dW)]
+
+
+def check_problem(p, tol, backend="simt", inverse_iters=0, resident=True, exact_masks=True, tau=0.0):
+    out = run_gpu(p, backend=backend, resident_inverse=resident, inverse_iters=inverse_iters)
+    assert out["status"] == 0 and out["bp_status"] == 0
+    ref_own = oracle_reference(p)
+    flips, worst = mask_disagreement(p, out["masks"], ref_own)
+    if exact_masks:
+        assert flips == 0
+        ref = ref_own
+    else:
+        assert worst <= tau, (flips, worst)
+        ref = oracle_reference(p, oracle_masks_from_words(p, out["masks"]))
+    errs = grad_errors(out["dW"], ref["dW"])
+    errs_bp = grad_errors(out["bp_dW"], ref["dW"])
+    assert O.normwise_error(out["g0"].reshape(ref["g0"].shape), ref["g0"]) <= tol
+    assert max(errs) <= tol, errs
+    assert max(errs_bp) <= tol, errs_bp
+    assert abs(out["loss"] - ref["loss"]) <= max(tol, 1e-12) * max(1.0, abs(ref["loss"]))
+    assert abs(out["bp_loss"] - ref["loss"]) <= max(tol, 1e-12) * max(1.0, abs(ref["loss"]))
+    return out, ref, errs
+
+

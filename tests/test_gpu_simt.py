@@ -6,8 +6,7 @@ import pytest
 from oracle import moonwalk_oracle as O
 from paper_2402_14212_b200 import binding as mwb
 from paper_2402_14212_b200 import synth as S
-from parity_util import (grad_errors, mask_disagreement, oracle_masks_from_words,
-                         oracle_reference, run_gpu)
+from parity_util import check_problem
 
 pytestmark = pytest.mark.gpu
 
@@ -80,27 +79,6 @@ def test_leaky_vijp_closed_form(rows, cols):
 # ---------------------------------------------------------------------------------------
 # whole path, fp64 (config 1 and ragged variants): masks bit-exact, gradients to 1e-9
 # ---------------------------------------------------------------------------------------
-def check_problem(p, tol, backend="simt", resident=True, exact_masks=True, tau=0.0):
-    out = run_gpu(p, backend=backend, resident_inverse=resident)
-    assert out["status"] == 0 and out["bp_status"] == 0
-    ref_own = oracle_reference(p)
-    flips, worst = mask_disagreement(p, out["masks"], ref_own)
-    if exact_masks:
-        assert flips == 0
-        ref = ref_own
-    else:
-        assert worst <= tau, (flips, worst)
-        ref = oracle_reference(p, oracle_masks_from_words(p, out["masks"]))
-    errs = grad_errors(out["dW"], ref["dW"])
-    errs_bp = grad_errors(out["bp_dW"], ref["dW"])
-    assert O.normwise_error(out["g0"].reshape(ref["g0"].shape), ref["g0"]) <= tol
-    assert max(errs) <= tol, errs
-    assert max(errs_bp) <= tol, errs_bp
-    assert abs(out["loss"] - ref["loss"]) <= max(tol, 1e-12) * max(1.0, abs(ref["loss"]))
-    assert abs(out["bp_loss"] - ref["loss"]) <= max(tol, 1e-12) * max(1.0, abs(ref["loss"]))
-    return out, ref, errs
-
-
 def test_config1_tiny_mlp_fp64():
     # literal Algorithm 1 (no re-seeding): 4 layers stay within 1e-9 in fp64
     check_problem(S.tiny_mlp(seed=0), 1e-9)
