@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the Moonwalk gradient step on B200.
+
+One "step" = one pass of the whole hot path over one batch: per-step preparation (W^-1 of every
+layer), Phase I + Phase II (mw_input_cotangent) and the forward sweep (mw_forward_sweep).
+Workload: config 2 of the baseline (64 square dense layers, width 1024, leaky-ReLU 0.1, batch 256,
+fp32, MSE), synthetic seeded data.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+N > 1 (under torchrun): independent replicas of the same step on every GPU, no data-path
+collective ("replicas only"); NCCL is used only for the barrier and the max over ranks.
+--impl reference times the CPU oracle (fp64, numpy) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "moonwalk_grad_samples_per_s"
+UNIT = "samples/s"
+NOMINAL_TF32_OVER_BF16 = 1.1 / 2.25      # dense tensor peaks, nominal ratio
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes per launch of the product kernel, from the committed ncu capture (None until measured)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def workload(name: str, seed: int = 0):
+    from paper_2402_14212_b200 import synth as S
+    if name == "deep_mlp":
+        return S.deep_mlp(seed=seed)
+    if name == "deep_mlp_small":
+        return S.deep_mlp(seed=seed, depth=8, n=256, batch=128)
+    if name == "mixed_mlp":
+        return S.mixed_mlp(seed=seed)
+    if name == "tiny_mlp":
+        return S.tiny_mlp(seed=seed)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def describe(p):
+    return {"workload": p.name, "layers": len(p.layers), "width": p.layers[0].n_in,
+            "batch": p.batch, "prec": p.prec, "loss": p.loss, "reseed_every": p.reseed_every,
+            "seed": p.seed}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for nme, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def time_oracle(p, seconds_target: float, max_reps: int = 50):
+    """Oracle (as it stands) on the host cores: Algorithm 1 with the same re-seed interval."""
+    from oracle import moonwalk_oracle as O
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        O.moonwalk(p.layers, p.params, p.x, p.target, p.loss, reseed_every=p.reseed_every)
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= seconds_target or reps >= max_reps:
+            break
+    return p.batch * reps / dt, reps, dt
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 0) for d in threadpool_info() if d.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from oracle import moonwalk_oracle as O
+    from paper_2402_14212_b200 import synth as S
+    p = workload(args.workload)
+    total = args.steps + args.warmup
+    t0 = time.perf_counter()
+    O.moonwalk(p.layers, p.params, p.x, p.target, p.loss, reseed_every=p.reseed_every)
+    t_full = time.perf_counter() - t0
+    budget = 150.0
+    b = p.batch
+    if t_full * total > budget:      # bounded sample: the first b rows of the batch
+        b = max(8, int(p.batch * budget / (t_full * total)))
+        b = min(b, p.batch)
+    x, t = p.x[:b], p.target[:b]
+
+    def step():
+        O.moonwalk(p.layers, p.params, x, t, p.loss, reseed_every=p.reseed_every)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = b * args.steps / dt
+    cores = blas_threads()
+    sample = f"{b} of {p.batch} samples per step, all {len(p.layers)} layers, fp64 numpy"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": describe(p),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2402_14212_b200 import binding as mwb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    p = workload(args.workload)
+    net = mwb.net_for(p, backend=args.backend)
+    params, x, target = mwb.to_device(p, dev)
+    ws = net.alloc_workspace("moonwalk", dev)
+    mw_bytes, bp_bytes, (mw_res, bp_res) = net.workspace_bytes()
+    g0 = torch.empty(x.shape, dtype=net.grad_dtype(), device=dev)
+    dW = [torch.empty(w.shape, dtype=net.grad_dtype(), device=dev) for w in params]
+    loss = torch.zeros(1, dtype=torch.float64, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        net.input_cotangent(params, x, target, ws, g0_out=g0, loss_out=loss)
+        net.forward_sweep(params, x, g0, ws, dW_out=dW)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    code, detail = net.last_device_status(ws)
+    if code != 0:
+        raise SystemExit(f"device status {code} {detail} during warm-up")
+
+    # ---- device-resident timing: K steps, events on the launching stream --------------------
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = mwb.launch_count()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    launches = mwb.launch_count() - launches0
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    t_ms = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    ms_max = float(t_ms.item())
+    value = p.batch * args.steps * world / (ms_max * 1e-3)
+
+    # ---- phase split (device timed, a few extra steps) --------------------------------------
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    reps = min(args.steps, 5)
+    t_cot = t_sweep = 0.0
+    for _ in range(reps):
+        ev[0].record(stream)
+        net.input_cotangent(params, x, target, ws, g0_out=g0, loss_out=loss)
+        ev[1].record(stream)
+        net.forward_sweep(params, x, g0, ws, dW_out=dW)
+        ev[2].record(stream)
+        torch.cuda.synchronize()
+        t_cot += ev[0].elapsed_time(ev[1])
+        t_sweep += ev[1].elapsed_time(ev[2])
+    t_cot /= reps
+    t_sweep /= reps
+
+    # ---- end to end through the C ABI with host buffers --------------------------------------
+    xh = x.cpu().pin_memory()
+    th = target.cpu().pin_memory()
+    lh = torch.zeros(1, dtype=torch.float64).pin_memory()
+    xd, td = torch.empty_like(x), torch.empty_like(target)
+    for _ in range(2):
+        net.gradient_step_host(params, xh, th, xd, td, g0, dW, loss, lh, ws)
+    barrier()
+    w0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(args.steps):
+        net.gradient_step_host(params, xh, th, xd, td, g0, dW, loss, lh, ws)
+    e1.record(stream)
+    barrier()
+    wall = time.perf_counter() - w0
+    ms_e2e = max(e0.elapsed_time(e1), 0.0)
+    t2 = torch.tensor([max(ms_e2e, wall * 1e3)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+    e2e_value = p.batch * args.steps * world / (float(t2.item()) * 1e-3)
+    h2d = xh.numel() * xh.element_size() + th.numel() * th.element_size()
+
+    # ---- roofline of the dominant kernel: per-launch events over the same K steps ------------
+    roof = None
+    if net.prec != "f64":
+        barrier()
+        mwb.profile_begin()
+        for _ in range(args.steps):
+            step()
+        prof = mwb.profile_end()
+        pk = peaks()
+        src = pk["_source"]
+        bf16_peak = float(pk.get("bf16_tflops_sustained", pk["bf16_tflops"]))
+        if p.prec == "f32":
+            peak = bf16_peak * NOMINAL_TF32_OVER_BF16
+            peak_note = f"{src} sustained bf16 x nominal tf32/bf16 ratio (fp32 products)"
+        else:
+            peak = bf16_peak
+            peak_note = f"{src} sustained bf16"
+        if prof["launches"]:
+            achieved = prof["flops"] / (prof["total_ms"] * 1e-3) / 1e12
+            executed = prof["mma_flops"] / (prof["total_ms"] * 1e-3) / 1e12
+            roof = {"bound": "tensor", "kernel": "tc_gemm_kernel (tcgen05, all layouts)",
+                    "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_source": peak_note,
+                    "launches_per_step": prof["launches"] / args.steps,
+                    "avg_launch_us": 1e3 * prof["total_ms"] / prof["launches"],
+                    "algorithmic_flops_per_launch": prof["flops"] / prof["launches"],
+                    "executed_bf16_tflops": executed, "executed_frac_of_bf16_peak": executed / bf16_peak,
+                    "kernel_time_share_of_step": prof["total_ms"] / (ms_max if world == 1 else ms)}
+
+    # ---- the oracle on the host cores (rank 0, single GPU only) -----------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, reps_o, dt = time_oracle(p, 10.0)
+        cpu = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": f"{reps_o} full steps ({p.batch} samples, {len(p.layers)} layers) in {dt:.1f} s, "
+                         "Algorithm 1 in fp64 numpy"}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_max / args.steps,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": {"f64": "f64", "f32": "f32 (bf16x3 split on tensor cores, fp32 accumulate)",
+                          "bf16_f32acc": "bf16 (fp32 accumulate)"}[p.prec]
+                if net_backend_is_tensor(net) else ("f64" if p.prec == "f64" else "f32"),
+                "data": "synthetic",
+                "config": dict(describe(p), parallelism=f"replicas x{world}" if world > 1 else "single GPU",
+                               l2="working set (weights, term planes, inverses, gradients) "
+                                  "far above the 126 MB L2; no flush between steps"),
+                "clocks": clocks, "gpu_launches": launches,
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": 8},
+                "roofline": roof, "cpu_baseline": cpu,
+                "phases_ms": {"prep_phase1_phase2": t_cot, "forward_sweep": t_sweep},
+                "memory_bytes": {"moonwalk_workspace": mw_bytes, "backprop_workspace": bp_bytes,
+                                 "moonwalk_residual": mw_res, "backprop_residual": bp_res,
+                                 "params": sum(w.numel() * w.element_size() for w in params),
+                                 "grads": sum(g.numel() * g.element_size() for g in dW)}}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def net_backend_is_tensor(net):
+    return net.prec != "f64" and all(l.kind == "dense" and l.n_in % 64 == 0 for l in net.layers)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="deep_mlp")
+    ap.add_argument("--backend", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -181,6 +181,31 @@ mw_status mw_gemm_split_bf16(const float* A, int32_t a_mn, const float* B, int32
                              int32_t M, int32_t N, int32_t K, int32_t terms, void* scratch,
                              size_t scratch_bytes, void* stream);
 
+/* ---- whole step from host buffers, and measurement hooks --------------------------------- */
+
+/* One Moonwalk gradient step (Algorithm 1 with Phases I-II in front) whose per-step inputs
+ * arrive in HOST memory: copies x and the loss target to the caller's device staging buffers
+ * (x_dev, target_dev), runs mw_input_cotangent and mw_forward_sweep, copies the loss back to
+ * loss_host and synchronises the stream.  params, dW_out, g0_dev, loss_dev, workspace: device,
+ * as in the calls above.  Use pinned host memory for asynchronous copies. */
+mw_status mw_gradient_step_host(mw_net* net, const void* const* params, const void* x_host,
+                                size_t x_bytes, const void* target_host, size_t target_bytes,
+                                void* x_dev, void* target_dev, void* g0_dev, void* const* dW_out,
+                                double* loss_dev, double* loss_host, void* workspace,
+                                size_t workspace_bytes, void* stream);
+
+/* Number of kernel launches this library has enqueued since it was loaded (host-side count;
+ * the paper has no counterpart: bookkeeping for benchmarks). */
+int64_t mw_launch_count(void);
+
+/* Between mw_profile_begin() and mw_profile_end() every launch of the tensor-core product
+ * kernel is bracketed by CUDA events on its stream.  mw_profile_end() waits for them and
+ * returns the summed kernel time, the number of launches, the algorithmic flops (2*M*N*K per
+ * product) and the flops the tensor cores executed (times the number of term pairs).  Not
+ * thread-safe; meant for benchmarks (the paper has no counterpart). */
+void mw_profile_begin(void);
+mw_status mw_profile_end(double* total_ms, int64_t* launches, double* flops, double* mma_flops);
+
 #ifdef __cplusplus
 }
 #endif

@@ -74,10 +74,14 @@ def lib() -> C.CDLL:
         L.mw_relu_fragment_compact.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp, vp, sz, vp]
         L.mw_activation_vijp.argtypes = [vp, vp, i64, i32, i32, C.c_float, vp, vp, vp, vp, vp]
         L.mw_gemm_split_bf16.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, vp, sz, vp]
-        for name in ("mw_step_host",):
-            if hasattr(L, name):
-                getattr(L, name).argtypes = [vp, C.POINTER(vp), vp, sz, vp, sz, vp, vp, vp,
-                                             C.POINTER(vp), vp, vp, vp, sz, vp]
+        L.mw_gradient_step_host.argtypes = [vp, C.POINTER(vp), vp, sz, vp, sz, vp, vp, vp,
+                                            C.POINTER(vp), vp, vp, vp, sz, vp]
+        L.mw_launch_count.argtypes = []
+        L.mw_launch_count.restype = C.c_int64
+        L.mw_profile_begin.argtypes = []
+        L.mw_profile_begin.restype = None
+        L.mw_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64),
+                                     C.POINTER(C.c_double), C.POINTER(C.c_double)]
         _lib = L
     return _lib
 
@@ -199,6 +203,17 @@ class Net:
                                            _stream_handle(stream)), "mw_backprop_reference")
         return dW_out
 
+    def gradient_step_host(self, params, x_host, target_host, x_dev, target_dev, g0_dev, dW_out,
+                           loss_dev, loss_host, workspace, stream=None):
+        """Whole step with the per-step inputs in (pinned) host memory; returns after the loss
+        has landed in `loss_host`."""
+        wp, wb = self._ws(workspace)
+        _check(lib().mw_gradient_step_host(
+            self._h, _ptr_array(params), _ptr(x_host), x_host.numel() * x_host.element_size(),
+            _ptr(target_host), target_host.numel() * target_host.element_size(), _ptr(x_dev),
+            _ptr(target_dev), _ptr(g0_dev), _ptr_array(dW_out), _ptr(loss_dev), _ptr(loss_host),
+            wp, wb, _stream_handle(stream)), "mw_gradient_step_host")
+
     def export_masks(self, workspace, layer: int, stream=None) -> np.ndarray:
         l = self.layers[layer]
         if l.kind == "conv2d":
@@ -219,6 +234,20 @@ class Net:
         detail = (C.c_uint32 * 4)()
         code = lib().mw_last_device_status(self._h, wp, _stream_handle(stream), detail)
         return code, list(detail)
+
+
+def launch_count() -> int:
+    return int(lib().mw_launch_count())
+
+
+def profile_begin():
+    lib().mw_profile_begin()
+
+
+def profile_end():
+    ms, n, fl, mfl = C.c_double(), C.c_int64(), C.c_double(), C.c_double()
+    _check(lib().mw_profile_end(C.byref(ms), C.byref(n), C.byref(fl), C.byref(mfl)), "mw_profile_end")
+    return dict(total_ms=ms.value, launches=int(n.value), flops=fl.value, mma_flops=mfl.value)
 
 
 # ---- stand-alone kernels -----------------------------------------------------------------

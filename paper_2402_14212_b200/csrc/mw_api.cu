@@ -7,9 +7,12 @@
 #include "mw_common.cuh"
 #include "mw_conv.cuh"
 #include "mw_net.cuh"
+#include "mw_tc_gemm.cuh"
 #include "mw_tensor.cuh"
 
 using namespace mw;
+
+long long mw::g_launch_count = 0;
 
 // ---------------------------------------------------------------------------------------
 // description and layout
@@ -600,4 +603,39 @@ extern "C" mw_status mw_activation_vijp(const float* gz, const uint32_t* words, 
   if (act == MW_ACT_LEAKY_RELU && !(slope != 0.f)) return MW_ERR_INVALID_ARG;
   return activation_vijp<float>(gz, words, rows, cols, act, (double)slope, off, vals, h_out, gz_out,
                                 (cudaStream_t)stream);
+}
+
+// ---------------------------------------------------------------------------------------
+// whole step from host buffers, and measurement hooks
+// ---------------------------------------------------------------------------------------
+extern "C" mw_status mw_gradient_step_host(mw_net* net, const void* const* params,
+                                           const void* x_host, size_t x_bytes,
+                                           const void* target_host, size_t target_bytes,
+                                           void* x_dev, void* target_dev, void* g0_dev,
+                                           void* const* dW_out, double* loss_dev,
+                                           double* loss_host, void* workspace,
+                                           size_t workspace_bytes, void* stream) {
+  if (!net || !x_host || !target_host || !x_dev || !target_dev || !g0_dev || !loss_dev || !loss_host)
+    return MW_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  MW_CUDA_OK(cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, s));
+  MW_CUDA_OK(cudaMemcpyAsync(target_dev, target_host, target_bytes, cudaMemcpyHostToDevice, s));
+  MW_TRY(mw_input_cotangent(net, params, x_dev, target_dev, g0_dev, loss_dev, workspace,
+                            workspace_bytes, stream));
+  MW_TRY(mw_forward_sweep(net, params, x_dev, g0_dev, dW_out, workspace, workspace_bytes, stream));
+  MW_CUDA_OK(cudaMemcpyAsync(loss_host, loss_dev, sizeof(double), cudaMemcpyDeviceToHost, s));
+  MW_CUDA_OK(cudaStreamSynchronize(s));
+  return MW_OK;
+}
+
+extern "C" int64_t mw_launch_count(void) { return (int64_t)g_launch_count; }
+
+extern "C" void mw_profile_begin(void) { tc_profile_begin(); }
+
+extern "C" mw_status mw_profile_end(double* total_ms, int64_t* launches, double* flops,
+                                    double* mma_flops) {
+  long long n = 0;
+  mw_status r = tc_profile_end(total_ms, &n, flops, mma_flops);
+  if (launches) *launches = (int64_t)n;
+  return r;
 }

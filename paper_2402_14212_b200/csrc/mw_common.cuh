@@ -40,7 +40,13 @@ __device__ __forceinline__ void record_error(DeviceStatus* st, unsigned int code
     if (s__ != MW_OK) return s__;    \
   } while (0)
 
-inline mw_status launch_ok() { return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA; }
+// Kernel launches enqueued by this library since load (host-side count, for the benchmark's
+// "gpu_launches" figure).  launch_ok(k) is called after k launches.
+extern long long g_launch_count;
+inline mw_status launch_ok(int k = 1) {
+  g_launch_count += k;
+  return cudaGetLastError() == cudaSuccess ? MW_OK : MW_ERR_CUDA;
+}
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }

@@ -204,7 +204,7 @@ mw_status conv_wgrad(const T* x, const T* gz, T* dw, T* scratch, int Bn, int H, 
   conv_wgrad_kernel<T><<<grid, 256, 0, s>>>(x, gz, scratch, Bn, H, W, Ci, Co, k, pad, slice);
   const int64_t n = (int64_t)R * Co;
   slice_sum_kernel<T><<<ceil_div(n, 256), 256, 0, s>>>(scratch, n, slices, dw);
-  return launch_ok();
+  return launch_ok(2);
 }
 
 // zero one k*k tap [Ci][Co] block

@@ -313,7 +313,7 @@ mw_status fragment_offsets(const uint32_t* words, int64_t rows, int cols, uint32
   const int wpr = (cols + 31) / 32;
   dead_count_kernel<<<grid_for(rows), kThreads, 0, s>>>(words, rows, cols, wpr, cnt);
   exclusive_scan_kernel<<<1, 1024, 0, s>>>(cnt, rows, off, total);
-  return launch_ok();
+  return launch_ok(2);
 }
 
 // one warp per row; MODE 0: compact h at dead units into vals; MODE 1: restore (activation vijp
@@ -457,14 +457,19 @@ mw_status loss_cotangent(const T* y, const void* target, int64_t rows, int cols,
     int blocks = (int)((n + kThreads - 1) / kThreads);
     if (blocks > kLossBlocks) blocks = kLossBlocks;
     sq_loss_kernel<T><<<blocks, kThreads, 0, s>>>(y, (const T*)target, n, (T)scale, h, partials);
-    if (loss_out)
+    if (loss_out) {
       final_sum_kernel<<<1, 32, 0, s>>>(partials, blocks,
                                         loss == MW_LOSS_HALF_SSE ? 0.5 : 1.0 / (double)n, loss_out);
+      ++g_launch_count;
+    }
   } else if (loss == MW_LOSS_XENT_MEAN) {
     if (rows > 1 << 20) return MW_ERR_UNSUPPORTED;
     xent_kernel<T><<<grid_for(rows), kThreads, 0, s>>>(y, (const int32_t*)target, rows, cols, h,
                                                        partials);
-    if (loss_out) final_sum_kernel<<<1, 32, 0, s>>>(partials, rows, 1.0 / (double)rows, loss_out);
+    if (loss_out) {
+      final_sum_kernel<<<1, 32, 0, s>>>(partials, rows, 1.0 / (double)rows, loss_out);
+      ++g_launch_count;
+    }
   } else {
     return MW_ERR_INVALID_ARG;
   }

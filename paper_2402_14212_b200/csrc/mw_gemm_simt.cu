@@ -218,6 +218,7 @@ mw_status inverse_newton_simt(const T* W, int n, int iters, T* X, T* scratch, De
   frob_scale_kernel<T><<<1, 1024, 0, s>>>(W, (int64_t)n * n, n, c);
   dim3 tg(ceil_div(n, 32), ceil_div(n, 32));
   scaled_transpose_kernel<T><<<tg, 256, 0, s>>>(W, n, c, X);
+  g_launch_count += 2;
   const size_t bytes = sizeof(T) * (size_t)n * n;
   for (int it = 0; it < iters; ++it) {
     MW_TRY(gemm_simt<T>(0, 0, n, n, n, 1.0, W, n, X, n, 0.0, P, n, s));         // P = W X

@@ -20,6 +20,7 @@
 
 #include <map>
 #include <tuple>
+#include <vector>
 
 #include "mw_tc_gemm.cuh"
 
@@ -430,6 +431,46 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
 
 }  // namespace
 
+// ---- optional per-launch timing of the product kernel (measurement hook) -----------------
+struct TcProfile {
+  bool on = false;
+  std::vector<cudaEvent_t> pool;      // pairs: [2i] before, [2i+1] after
+  size_t used = 0;
+  double flops = 0.0, mma_flops = 0.0;
+};
+static TcProfile g_prof;
+
+void tc_profile_begin() {
+  g_prof.on = true;
+  g_prof.used = 0;
+  g_prof.flops = g_prof.mma_flops = 0.0;
+}
+
+mw_status tc_profile_end(double* total_ms, long long* launches, double* flops, double* mma_flops) {
+  g_prof.on = false;
+  double ms = 0.0;
+  for (size_t i = 0; i + 1 < g_prof.used; i += 2) {
+    if (cudaEventSynchronize(g_prof.pool[i + 1]) != cudaSuccess) return MW_ERR_CUDA;
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, g_prof.pool[i], g_prof.pool[i + 1]) != cudaSuccess) return MW_ERR_CUDA;
+    ms += t;
+  }
+  if (total_ms) *total_ms = ms;
+  if (launches) *launches = (long long)(g_prof.used / 2);
+  if (flops) *flops = g_prof.flops;
+  if (mma_flops) *mma_flops = g_prof.mma_flops;
+  return MW_OK;
+}
+
+static cudaEvent_t prof_event() {
+  if (g_prof.used == g_prof.pool.size()) {
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    g_prof.pool.push_back(e);
+  }
+  return g_prof.pool[g_prof.used++];
+}
+
 struct TcMapCache {
   std::map<std::tuple<const void*, int, int, int, int64_t, int>, CUtensorMap> maps;
 };
@@ -517,17 +558,25 @@ mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int
   CUtensorMap ta, tb;
   MW_TRY(get_map(cache, A, A.mn_major ? 64 : BM, &ta));
   MW_TRY(get_map(cache, B, B.mn_major ? 64 : BNsel, &tb));
+  const bool prof = g_prof.on;
+  if (prof) {
+    cudaEventRecord(prof_event(), s);
+    g_prof.flops += 2.0 * M * N * K;
+    g_prof.mma_flops += 2.0 * M * N * K * np;
+  }
+  mw_status rc = MW_ERR_UNSUPPORTED;
 #define MW_TC_DISPATCH(AM, BMJ)                                              \
   if (A.mn_major == AM && B.mn_major == BMJ) {                               \
-    return bn128 ? launch_tc<AM, BMJ, 128>(ta, tb, prm, s)                   \
-                 : launch_tc<AM, BMJ, 64>(ta, tb, prm, s);                   \
+    rc = bn128 ? launch_tc<AM, BMJ, 128>(ta, tb, prm, s)                     \
+               : launch_tc<AM, BMJ, 64>(ta, tb, prm, s);                     \
   }
   MW_TC_DISPATCH(false, false)
   MW_TC_DISPATCH(false, true)
   MW_TC_DISPATCH(true, true)
   MW_TC_DISPATCH(true, false)
 #undef MW_TC_DISPATCH
-  return MW_ERR_UNSUPPORTED;
+  if (prof) cudaEventRecord(prof_event(), s);
+  return rc;
 }
 
 // ---------------------------------------------------------------------------------------

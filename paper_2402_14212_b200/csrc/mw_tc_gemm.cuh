@@ -64,6 +64,10 @@ void tc_cache_destroy(TcMapCache*);
 mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int M, int N, int K,
                   const TcEpilogue& epi, DeviceStatus* st, cudaStream_t s);
 
+// Per-launch timing of the product kernel (CUDA events around every launch while enabled).
+void tc_profile_begin();
+mw_status tc_profile_end(double* total_ms, long long* launches, double* flops, double* mma_flops);
+
 // fp32 [n] -> `planes` bf16 term planes (plane p at out + p*plane_stride)
 mw_status split_planes(const float* in, int64_t n, __nv_bfloat16* out, int planes,
                        int64_t plane_stride, cudaStream_t s);

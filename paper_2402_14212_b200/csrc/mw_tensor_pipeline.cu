@@ -178,7 +178,7 @@ mw_status newton_schulz(const Ctx& c, int l, const void* W, const __nv_bfloat16*
     frob_scale_kernel<__nv_bfloat16><<<1, 1024, 0, c.s>>>((const __nv_bfloat16*)W, c.nn, d, cscale);
     x0_kernel<__nv_bfloat16><<<dim3(d / 32, d / 32), 256, 0, c.s>>>((const __nv_bfloat16*)W, d, cscale, X);
   }
-  MW_TRY(launch_ok());
+  MW_TRY(launch_ok(2));
   int have = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;   // terms of X currently split
   MW_TRY(split_planes(X, c.nn, Xp[0], have, c.nn, c.s));
   int cur = 0;
@@ -197,6 +197,7 @@ mw_status newton_schulz(const Ctx& c, int l, const void* W, const __nv_bfloat16*
       // the update squares this residual: gate on it so a diverging layer is reported
       const double limit = c.n->opts.prec == MW_F32 ? 2e-3 : 2e-2;
       residual_gate_kernel<<<1, 32, 0, c.s>>>(sumsq, d, limit, c.st, l);
+      ++g_launch_count;
     }
     // X' = X + X R
     int next_terms = c.pr.ph;
