@@ -31,7 +31,7 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int kThreadsTc = 192;
-constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far above any legitimate wait
 constexpr int kMaxStages = 8;
 constexpr int kMaxPairs = 6;
 constexpr uint32_t kATileBytes = BM * BK * 2;  // one A term plane of one stage
@@ -71,12 +71,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// bounded wait; returns false (and records the timeout) when the limit is reached
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: try_wait suspends the thread in hardware until the phase completes or its own
+// time slice ends, so the loop does not burn issue slots and adds no wake-up latency.  The bound
+// is wall time (checked every 256 polls); on expiry the timeout is recorded and false returned.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, DeviceStatus* st,
                                           unsigned who) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+  uint64_t t0 = 0;
+  for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (i > 32) __nanosleep(64);
+    if ((i & 255u) == 255u) {
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) break;
+    }
   }
   record_error(st, MW_ERR_TIMEOUT, who, blockIdx.x, blockIdx.y, parity);
   return false;

@@ -65,22 +65,33 @@ int ns_schedule(const mw_net* n, NsStep* out) {
   return cnt;
 }
 
+// sum of squares of W: kFrobBlocks partial sums, then one block folds them in fixed order and
+// writes the Newton-Schulz start scale c = n / ||W||_F^2 (deterministic)
+constexpr int kFrobBlocks = 128;
 template <typename TW>
-__global__ void __launch_bounds__(1024)
-frob_scale_kernel(const TW* __restrict__ W, int64_t n2, int n, float* __restrict__ c_out) {
-  __shared__ double red[1024];
+__global__ void __launch_bounds__(256)
+frob_partial_kernel(const TW* __restrict__ W, int64_t n2, double* __restrict__ partial) {
+  __shared__ double red[256];
   double a = 0.0;
-  for (int64_t i = threadIdx.x; i < n2; i += 1024) {
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n2; i += (int64_t)gridDim.x * 256) {
     const double v = (double)to_f32(W[i]);
     a += v * v;
   }
   red[threadIdx.x] = a;
   __syncthreads();
-  for (int o = 512; o; o >>= 1) {
+  for (int o = 128; o; o >>= 1) {
     if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
     __syncthreads();
   }
-  if (threadIdx.x == 0) *c_out = red[0] > 0.0 ? (float)((double)n / red[0]) : 0.f;
+  if (threadIdx.x == 0) partial[blockIdx.x] = red[0];
+}
+__global__ void frob_final_kernel(const double* __restrict__ partial, int blocks, int n,
+                                  float* __restrict__ c_out) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    double a = 0.0;
+    for (int i = 0; i < blocks; ++i) a += partial[i];
+    *c_out = a > 0.0 ? (float)((double)n / a) : 0.f;
+  }
 }
 
 // X0 = c W^T (fp32) through a 32x32 shared tile
@@ -171,14 +182,17 @@ mw_status newton_schulz(const Ctx& c, int l, const void* W, const __nv_bfloat16*
   NsStep sched[16];
   const int steps = ns_schedule(c.n, sched);
   if (steps < 1) return MW_ERR_INVALID_ARG;
+  double* fpart = c.at<double>(lay.partials);
   if (c.n->opts.prec == MW_F32) {
-    frob_scale_kernel<float><<<1, 1024, 0, c.s>>>((const float*)W, c.nn, d, cscale);
+    frob_partial_kernel<float><<<kFrobBlocks, 256, 0, c.s>>>((const float*)W, c.nn, fpart);
+    frob_final_kernel<<<1, 32, 0, c.s>>>(fpart, kFrobBlocks, d, cscale);
     x0_kernel<float><<<dim3(d / 32, d / 32), 256, 0, c.s>>>((const float*)W, d, cscale, X);
   } else {
-    frob_scale_kernel<__nv_bfloat16><<<1, 1024, 0, c.s>>>((const __nv_bfloat16*)W, c.nn, d, cscale);
+    frob_partial_kernel<__nv_bfloat16><<<kFrobBlocks, 256, 0, c.s>>>((const __nv_bfloat16*)W, c.nn, fpart);
+    frob_final_kernel<<<1, 32, 0, c.s>>>(fpart, kFrobBlocks, d, cscale);
     x0_kernel<__nv_bfloat16><<<dim3(d / 32, d / 32), 256, 0, c.s>>>((const __nv_bfloat16*)W, d, cscale, X);
   }
-  MW_TRY(launch_ok(2));
+  MW_TRY(launch_ok(3));
   int have = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;   // terms of X currently split
   MW_TRY(split_planes(X, c.nn, Xp[0], have, c.nn, c.s));
   int cur = 0;

@@ -1,0 +1,52 @@
+"""Small, self-ending cases of single kernels for profiler captures.
+
+  python -m paper_2402_14212_b200.profile_cases gemm --M 256 --N 1024 --K 1024 --terms 3 --b-mn
+  python -m paper_2402_14212_b200.profile_cases pack --rows 65536 --cols 2048
+  python -m paper_2402_14212_b200.profile_cases fragments --rows 65536 --cols 2048
+
+Each case allocates its seeded inputs, runs the kernel `--reps` times and exits.
+"""
+from __future__ import annotations
+
+import argparse
+
+import numpy as np
+
+
+def main():
+    import torch
+    from . import binding as mwb
+    ap = argparse.ArgumentParser()
+    ap.add_argument("case", choices=["gemm", "pack", "fragments", "vijp"])
+    ap.add_argument("--M", type=int, default=256)
+    ap.add_argument("--N", type=int, default=1024)
+    ap.add_argument("--K", type=int, default=1024)
+    ap.add_argument("--terms", type=int, default=3)
+    ap.add_argument("--a-mn", action="store_true")
+    ap.add_argument("--b-mn", action="store_true")
+    ap.add_argument("--rows", type=int, default=65536)
+    ap.add_argument("--cols", type=int, default=2048)
+    ap.add_argument("--reps", type=int, default=3)
+    a = ap.parse_args()
+    g = torch.Generator(device="cuda").manual_seed(0)
+    if a.case == "gemm":
+        A = torch.randn((a.K, a.M) if a.a_mn else (a.M, a.K), device="cuda", generator=g)
+        B = torch.randn((a.K, a.N) if a.b_mn else (a.N, a.K), device="cuda", generator=g)
+        for _ in range(a.reps):
+            mwb.gemm_split_bf16(A, B, a.a_mn, a.b_mn, a.terms)
+    else:
+        z = torch.randn((a.rows, a.cols), device="cuda", generator=g)
+        h = torch.randn((a.rows, a.cols), device="cuda", generator=g)
+        for _ in range(a.reps):
+            words = mwb.pack_sign_bits(z)
+            if a.case == "fragments":
+                cnt, off, vals, total = mwb.relu_fragment_compact(h, words)
+                mwb.activation_vijp(h, words, "relu", 0.0, off, vals)
+            elif a.case == "vijp":
+                mwb.activation_vijp(h, words, "leaky_relu", 0.1)
+    torch.cuda.synchronize()
+    print("done", a.case)
+
+
+if __name__ == "__main__":
+    main()
