@@ -31,7 +31,7 @@ struct Layout {
   Region inv_scratch;
   // tensor-core backend operands (bf16 term planes)
   std::vector<Region> w_planes;              // split weights (MW_F32), per layer or one slot
-  Region xp[2], hp[2], gzp, ns_r, ns_x;      // activation / cotangent / g_z planes, NS scratch
+  Region xp[2], hp[2], gzp, ns_r, ns_x, ns_w; // activation / cotangent / g_z planes, NS scratch
 };
 
 }  // namespace mw

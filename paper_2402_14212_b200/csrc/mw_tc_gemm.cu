@@ -45,6 +45,7 @@ struct TcParams {
   int nacc;        // tensor-memory accumulators in use (each BN columns)
   int nbig;        // of those, the ones that take the leading (0,0) term, rotated over K blocks
   int tmem_cols;   // allocated columns: power of two >= nacc * BN
+  int a_batch_planes, b_batch_planes;
   TcEpilogue epi;
   DeviceStatus* st;
 };
@@ -90,7 +91,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, DeviceS
       else if (now - t0 > kWaitLimitNs) break;
     }
   }
-  record_error(st, MW_ERR_TIMEOUT, who, blockIdx.x, blockIdx.y, parity);
+  record_error(st, MW_ERR_TIMEOUT, who, blockIdx.x, blockIdx.y, blockIdx.z);
   return false;
 }
 
@@ -282,6 +283,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * BN;
   const int m0 = blockIdx.y * BM;
+  const int bz = blockIdx.z;
+  const int a_pl0 = bz * p.a_batch_planes, b_pl0 = bz * p.b_batch_planes;
   const int num_kb = (p.K + BK - 1) / BK;
   constexpr uint32_t kBTileBytes = BN * BK * 2;
   const uint32_t stage_bytes = p.pa * kATileBytes + p.pb * kBTileBytes;
@@ -323,10 +326,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int pl = 0; pl < p.pa; ++pl) {
           const uint32_t dst = sbase + (uint32_t)pl * kATileBytes;
           if (A_MN) {
-            tma_load_3d(dst, &tmA, fb, m0, kb * BK, pl);
-            tma_load_3d(dst + 8192u, &tmA, fb, m0 + 64, kb * BK, pl);
+            tma_load_3d(dst, &tmA, fb, m0, kb * BK, a_pl0 + pl);
+            tma_load_3d(dst + 8192u, &tmA, fb, m0 + 64, kb * BK, a_pl0 + pl);
           } else {
-            tma_load_3d(dst, &tmA, fb, kb * BK, m0, pl);
+            tma_load_3d(dst, &tmA, fb, kb * BK, m0, a_pl0 + pl);
           }
         }
         const uint32_t bbase = sbase + (uint32_t)p.pa * kATileBytes;
@@ -335,9 +338,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (B_MN) {
 #pragma unroll
             for (int h = 0; h < BN / 64; ++h)
-              tma_load_3d(dst + (uint32_t)h * 8192u, &tmB, fb, n0 + h * 64, kb * BK, pl);
+              tma_load_3d(dst + (uint32_t)h * 8192u, &tmB, fb, n0 + h * 64, kb * BK, b_pl0 + pl);
           } else {
-            tma_load_3d(dst, &tmB, fb, kb * BK, n0, pl);
+            tma_load_3d(dst, &tmB, fb, kb * BK, n0, b_pl0 + pl);
           }
         }
         ++issued;
@@ -386,6 +389,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int quarter = warp & 3;                 // tensor-memory lane quarter this warp may read
     const int row = m0 + quarter * 32 + lane;
     double sumsq_local = 0.0;
+    TcEpilogue epi = p.epi;           // this batch item's view of the outputs
+    if (bz) {
+      if (epi.addend) epi.addend += (int64_t)bz * epi.bs_f32;
+      if (epi.out_f32) epi.out_f32 += (int64_t)bz * epi.bs_f32;
+      if (epi.planes) epi.planes += (int64_t)bz * epi.bs_planes;
+      if (epi.planes2) epi.planes2 += (int64_t)bz * epi.bs_planes2;
+      if (epi.mask) epi.mask += (int64_t)bz * epi.bs_mask;
+      if (epi.sumsq) epi.sumsq += (int64_t)bz * epi.bs_sumsq;
+    }
     // every lane observes the barrier itself; the warp then takes one common decision so the
     // warp-wide tensor-memory loads below are never executed by part of a warp
     const bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&accum_bar), 0u, p.st, 3u));
@@ -402,11 +414,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] += t[i];
         }
-        if (row < p.M) epilogue_chunk(p.epi, p.N, row, n0 + c, v, sumsq_local);
+        if (row < p.M) epilogue_chunk(epi, p.N, row, n0 + c, v, sumsq_local);
       }
-      if (p.epi.mode == TC_EPI_RESID && p.epi.sumsq) {
+      if (epi.mode == TC_EPI_RESID && epi.sumsq) {
         for (int o = 16; o; o >>= 1) sumsq_local += __shfl_xor_sync(0xffffffffu, sumsq_local, o);
-        if (lane == 0) atomicAdd(p.epi.sumsq, sumsq_local);
+        if (lane == 0) atomicAdd(epi.sumsq, sumsq_local);
       }
     }
   }
@@ -489,8 +501,9 @@ struct TcMapCache {
 TcMapCache* tc_cache_create() { return new TcMapCache(); }
 void tc_cache_destroy(TcMapCache* c) { delete c; }
 
-static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, CUtensorMap* out) {
-  auto key = std::make_tuple(op.base, op.rows, op.cols, op.planes, op.plane_stride, box_rows);
+static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, int total_planes,
+                         CUtensorMap* out) {
+  auto key = std::make_tuple(op.base, op.rows, op.cols, total_planes, op.plane_stride, box_rows);
   if (cache) {
     auto it = cache->maps.find(key);
     if (it != cache->maps.end()) { *out = it->second; return MW_OK; }
@@ -498,9 +511,9 @@ static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, C
   auto fn = encode_fn();
   if (!fn) return MW_ERR_CUDA;
   if (((uintptr_t)op.base & 15u) || (op.cols % 8) != 0) return MW_ERR_INVALID_ARG;
-  const int64_t ps = op.planes > 1 ? op.plane_stride : (int64_t)op.rows * op.cols;
+  const int64_t ps = total_planes > 1 ? op.plane_stride : (int64_t)op.rows * op.cols;
   if (ps % 8 != 0) return MW_ERR_INVALID_ARG;
-  cuuint64_t dims[3] = {(cuuint64_t)op.cols, (cuuint64_t)op.rows, (cuuint64_t)op.planes};
+  cuuint64_t dims[3] = {(cuuint64_t)op.cols, (cuuint64_t)op.rows, (cuuint64_t)total_planes};
   cuuint64_t strides[2] = {(cuuint64_t)op.cols * 2, (cuuint64_t)ps * 2};
   cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
   cuuint32_t estr[3] = {1u, 1u, 1u};
@@ -513,7 +526,8 @@ static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, C
 }
 
 template <bool A_MN, bool B_MN, int BN>
-static mw_status launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParams& prm, cudaStream_t s) {
+static mw_status launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParams& prm, int batch,
+                           cudaStream_t s) {
   const uint32_t stage_bytes = prm.pa * kATileBytes + prm.pb * (BN * BK * 2);
   const uint32_t budget = 227u * 1024u - 2048u;   // static barriers + alignment slack
   int stages = (int)(budget / stage_bytes);
@@ -537,14 +551,15 @@ static mw_status launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParam
                                     cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024));
     attr_set = true;
   }
-  dim3 grid(prm.N / BN, (prm.M + BM - 1) / BM);
+  dim3 grid(prm.N / BN, (prm.M + BM - 1) / BM, batch);
   tc_gemm_kernel<A_MN, B_MN, BN><<<grid, kThreadsTc, smem, s>>>(ta, tb, prm);
   return launch_ok();
 }
 
 mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int M, int N, int K,
-                  const TcEpilogue& epi, DeviceStatus* st, cudaStream_t s) {
-  if (M <= 0 || N <= 0 || K <= 0) return MW_OK;
+                  const TcEpilogue& epi, DeviceStatus* st, cudaStream_t s, int batch) {
+  if (M <= 0 || N <= 0 || K <= 0 || batch <= 0) return MW_OK;
+  if (batch > 65535) return MW_ERR_UNSUPPORTED;
   if (N % 64 != 0) return MW_ERR_UNSUPPORTED;
   if (A.planes < 1 || A.planes > 3 || B.planes < 1 || B.planes > 3) return MW_ERR_INVALID_ARG;
   if (!A.mn_major && (K % 64 != 0)) return MW_ERR_UNSUPPORTED;
@@ -564,23 +579,27 @@ mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int
   prm.npairs = np;
   prm.epi = epi;
   prm.st = st;
-  const int tiles128 = (N % 128 == 0) ? (N / 128) * ((M + BM - 1) / BM) : 0;
+  prm.a_batch_planes = A.batch_planes ? A.batch_planes : A.planes;
+  prm.b_batch_planes = B.batch_planes ? B.batch_planes : B.planes;
+  const int a_total = batch > 1 ? (batch - 1) * prm.a_batch_planes + A.planes : A.planes;
+  const int b_total = batch > 1 ? (batch - 1) * prm.b_batch_planes + B.planes : B.planes;
+  const int tiles128 = (N % 128 == 0) ? (N / 128) * ((M + BM - 1) / BM) * batch : 0;
   const bool bn128 = tiles128 >= 120;
   const int BNsel = bn128 ? 128 : 64;
   CUtensorMap ta, tb;
-  MW_TRY(get_map(cache, A, A.mn_major ? 64 : BM, &ta));
-  MW_TRY(get_map(cache, B, B.mn_major ? 64 : BNsel, &tb));
+  MW_TRY(get_map(cache, A, A.mn_major ? 64 : BM, a_total, &ta));
+  MW_TRY(get_map(cache, B, B.mn_major ? 64 : BNsel, b_total, &tb));
   const bool prof = g_prof.on;
   if (prof) {
     cudaEventRecord(prof_event(), s);
-    g_prof.flops += 2.0 * M * N * K;
-    g_prof.mma_flops += 2.0 * M * N * K * np;
+    g_prof.flops += 2.0 * M * N * K * batch;
+    g_prof.mma_flops += 2.0 * M * N * K * np * batch;
   }
   mw_status rc = MW_ERR_UNSUPPORTED;
 #define MW_TC_DISPATCH(AM, BMJ)                                              \
   if (A.mn_major == AM && B.mn_major == BMJ) {                               \
-    rc = bn128 ? launch_tc<AM, BMJ, 128>(ta, tb, prm, s)                     \
-               : launch_tc<AM, BMJ, 64>(ta, tb, prm, s);                     \
+    rc = bn128 ? launch_tc<AM, BMJ, 128>(ta, tb, prm, batch, s)              \
+               : launch_tc<AM, BMJ, 64>(ta, tb, prm, batch, s);              \
   }
   MW_TC_DISPATCH(false, false)
   MW_TC_DISPATCH(false, true)
@@ -613,6 +632,44 @@ split_planes_kernel(const float* __restrict__ in, int64_t n4, __nv_bfloat16* __r
       reinterpret_cast<uint2*>(out + (int64_t)p * plane_stride)[i] = pk;
     }
   }
+}
+
+__global__ void __launch_bounds__(256)
+split_planes_batched_kernel(const float* __restrict__ in, int64_t n4, int64_t in_stride,
+                            __nv_bfloat16* __restrict__ out, int planes, int64_t plane_stride,
+                            int64_t out_stride) {
+  const float* src = in + (int64_t)blockIdx.y * in_stride;
+  __nv_bfloat16* dst = out + (int64_t)blockIdx.y * out_stride;
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n4; i += (int64_t)gridDim.x * 256) {
+    float4 v = reinterpret_cast<const float4*>(src)[i];
+    float r[4] = {v.x, v.y, v.z, v.w};
+    for (int p = 0; p < planes; ++p) {
+      __nv_bfloat16 b[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        b[j] = __float2bfloat16_rn(r[j]);
+        r[j] -= __bfloat162float(b[j]);
+      }
+      uint2 pk;
+      pk.x = (uint32_t)__bfloat16_as_ushort(b[0]) | ((uint32_t)__bfloat16_as_ushort(b[1]) << 16);
+      pk.y = (uint32_t)__bfloat16_as_ushort(b[2]) | ((uint32_t)__bfloat16_as_ushort(b[3]) << 16);
+      reinterpret_cast<uint2*>(dst + (int64_t)p * plane_stride)[i] = pk;
+    }
+  }
+}
+
+mw_status split_planes_batched(const float* in, int64_t n, int batch, int64_t in_stride,
+                               __nv_bfloat16* out, int planes, int64_t plane_stride,
+                               int64_t out_stride, cudaStream_t s) {
+  if (n == 0 || batch == 0) return MW_OK;
+  if (n % 4 != 0 || plane_stride % 4 != 0 || in_stride % 4 != 0 || out_stride % 4 != 0)
+    return MW_ERR_UNSUPPORTED;
+  int64_t bx = (n / 4 + 255) / 256;
+  const int64_t cap = (148 * 8 + batch - 1) / batch;
+  if (bx > cap) bx = cap < 1 ? 1 : cap;
+  split_planes_batched_kernel<<<dim3((unsigned)bx, (unsigned)batch), 256, 0, s>>>(
+      in, n / 4, in_stride, out, planes, plane_stride, out_stride);
+  return launch_ok();
 }
 
 mw_status split_planes(const float* in, int64_t n, __nv_bfloat16* out, int planes,

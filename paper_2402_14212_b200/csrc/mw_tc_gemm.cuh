@@ -25,6 +25,7 @@ struct TcOperand {
   int planes = 1;
   int64_t plane_stride = 0;     // elements between planes
   bool mn_major = false;
+  int batch_planes = 0;         // batched launch: planes between consecutive batch items (0 = planes)
 };
 
 enum TcEpiMode : int {
@@ -51,6 +52,11 @@ struct TcEpilogue {
   int act = MW_ACT_NONE;
   float slope = 1.f;
   double* sumsq = nullptr;             // TC_EPI_RESID: atomically accumulated ||v||_F^2
+  // batched launch (grid.z): element strides between consecutive batch items
+  int64_t bs_f32 = 0;                  // addend and out_f32
+  int64_t bs_planes = 0, bs_planes2 = 0;
+  int64_t bs_mask = 0;                 // words
+  int64_t bs_sumsq = 0;                // doubles
 };
 
 // Cache of encoded tensor maps (host side), owned by the caller of tc_gemm.
@@ -61,8 +67,11 @@ void tc_cache_destroy(TcMapCache*);
 // D[M][N] = sum over term pairs of A_i B_j^T-style products; see TcOperand for layouts.
 // Requirements: N % 64 == 0; K % 64 == 0 for K-major operands; inner dimensions % 64 == 0;
 // all bases 16-byte aligned (256 recommended).
+// batch > 1 runs `batch` independent products of the same shape in one launch (grid.z): batch
+// item b reads planes b*batch_planes + t of each operand and offsets the epilogue pointers by
+// b times the bs_* strides.
 mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int M, int N, int K,
-                  const TcEpilogue& epi, DeviceStatus* st, cudaStream_t s);
+                  const TcEpilogue& epi, DeviceStatus* st, cudaStream_t s, int batch = 1);
 
 // Per-launch timing of the product kernel (CUDA events around every launch while enabled).
 void tc_profile_begin();
@@ -71,5 +80,9 @@ mw_status tc_profile_end(double* total_ms, long long* launches, double* flops, d
 // fp32 [n] -> `planes` bf16 term planes (plane p at out + p*plane_stride)
 mw_status split_planes(const float* in, int64_t n, __nv_bfloat16* out, int planes,
                        int64_t plane_stride, cudaStream_t s);
+// batched: item b reads in + b*in_stride and writes out + b*out_stride
+mw_status split_planes_batched(const float* in, int64_t n, int batch, int64_t in_stride,
+                               __nv_bfloat16* out, int planes, int64_t plane_stride,
+                               int64_t out_stride, cudaStream_t s);
 
 }  // namespace mw

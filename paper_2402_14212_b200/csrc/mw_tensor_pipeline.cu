@@ -65,13 +65,17 @@ int ns_schedule(const mw_net* n, NsStep* out) {
   return cnt;
 }
 
-// sum of squares of W: kFrobBlocks partial sums, then one block folds them in fixed order and
-// writes the Newton-Schulz start scale c = n / ||W||_F^2 (deterministic)
+constexpr int kMaxGroup = 32;     // layers whose inverses are computed together
+struct PtrBatch { const void* p[kMaxGroup]; };
+
+// sum of squares of each W of the group: kFrobBlocks partial sums per matrix, then one thread
+// per matrix folds them in fixed order into the Newton-Schulz start scale c = n / ||W||_F^2
 constexpr int kFrobBlocks = 128;
 template <typename TW>
 __global__ void __launch_bounds__(256)
-frob_partial_kernel(const TW* __restrict__ W, int64_t n2, double* __restrict__ partial) {
+frob_partial_kernel(PtrBatch Ws, int64_t n2, double* __restrict__ partial) {
   __shared__ double red[256];
+  const TW* W = static_cast<const TW*>(Ws.p[blockIdx.y]);
   double a = 0.0;
   for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n2; i += (int64_t)gridDim.x * 256) {
     const double v = (double)to_f32(W[i]);
@@ -83,36 +87,77 @@ frob_partial_kernel(const TW* __restrict__ W, int64_t n2, double* __restrict__ p
     if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
     __syncthreads();
   }
-  if (threadIdx.x == 0) partial[blockIdx.x] = red[0];
+  if (threadIdx.x == 0) partial[blockIdx.y * kFrobBlocks + blockIdx.x] = red[0];
 }
-__global__ void frob_final_kernel(const double* __restrict__ partial, int blocks, int n,
+__global__ void frob_final_kernel(const double* __restrict__ partial, int group, int n,
                                   float* __restrict__ c_out) {
-  if (threadIdx.x == 0 && blockIdx.x == 0) {
+  const int g = threadIdx.x;
+  if (g < group) {
     double a = 0.0;
-    for (int i = 0; i < blocks; ++i) a += partial[i];
-    *c_out = a > 0.0 ? (float)((double)n / a) : 0.f;
+    for (int i = 0; i < kFrobBlocks; ++i) a += partial[g * kFrobBlocks + i];
+    c_out[g] = a > 0.0 ? (float)((double)n / a) : 0.f;
   }
 }
 
-// X0 = c W^T (fp32) through a 32x32 shared tile
+// X0 = c W^T (fp32) through a 32x32 shared tile; blockIdx.z = matrix of the group
 template <typename TW>
 __global__ void __launch_bounds__(256)
-x0_kernel(const TW* __restrict__ W, int n, const float* __restrict__ c, float* __restrict__ X) {
+x0_kernel(PtrBatch Ws, int n, const float* __restrict__ c, float* __restrict__ X) {
   __shared__ float tile[32][33];
+  const TW* W = static_cast<const TW*>(Ws.p[blockIdx.z]);
+  float* Xg = X + (int64_t)blockIdx.z * n * n;
   const int bx = blockIdx.x * 32, by = blockIdx.y * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   for (int r = ty; r < 32; r += 8) tile[r][tx] = to_f32(W[(int64_t)(by + r) * n + bx + tx]);
   __syncthreads();
-  const float cc = *c;
-  for (int r = ty; r < 32; r += 8) X[(int64_t)(bx + r) * n + by + tx] = cc * tile[tx][r];
+  const float cc = c[blockIdx.z];
+  for (int r = ty; r < 32; r += 8) Xg[(int64_t)(bx + r) * n + by + tx] = cc * tile[tx][r];
 }
 
-__global__ void residual_gate_kernel(const double* __restrict__ sumsq, int n, double limit,
-                                     DeviceStatus* st, int layer) {
-  if (threadIdx.x == 0 && blockIdx.x == 0) {
-    const double r = sqrt(*sumsq / (double)n);   // rms singular value of I - W X
-    if (!(r <= limit)) record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)layer, __float_as_uint((float)r), 3u, 0u);
+// fp32 weights of the group -> 3 bf16 term planes each (dst + g*3*n2)
+__global__ void __launch_bounds__(256)
+split_weights_kernel(PtrBatch Ws, int64_t n4, int64_t n2, __nv_bfloat16* __restrict__ dst0) {
+  const float* src = static_cast<const float*>(Ws.p[blockIdx.y]);
+  __nv_bfloat16* dst = dst0 + (int64_t)blockIdx.y * 3 * n2;
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n4; i += (int64_t)gridDim.x * 256) {
+    float4 v = reinterpret_cast<const float4*>(src)[i];
+    float r[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int p = 0; p < 3; ++p) {
+      __nv_bfloat16 b[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        b[j] = __float2bfloat16_rn(r[j]);
+        r[j] -= __bfloat162float(b[j]);
+      }
+      uint2 pk;
+      pk.x = (uint32_t)__bfloat16_as_ushort(b[0]) | ((uint32_t)__bfloat16_as_ushort(b[1]) << 16);
+      pk.y = (uint32_t)__bfloat16_as_ushort(b[2]) | ((uint32_t)__bfloat16_as_ushort(b[3]) << 16);
+      reinterpret_cast<uint2*>(dst + (int64_t)p * n2)[i] = pk;
+    }
   }
+}
+
+__global__ void residual_gate_kernel(const double* __restrict__ sumsq, int group, int n,
+                                     double limit, DeviceStatus* st, int layer0) {
+  const int g = threadIdx.x;
+  if (g < group) {
+    const double r = sqrt(sumsq[g] / (double)n);   // rms singular value of I - W X
+    if (!(r <= limit))
+      record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)(layer0 + g), __float_as_uint((float)r), 3u, 0u);
+  }
+}
+
+// layers per Newton-Schulz group: enough 128x128 tiles for several waves of the 148 SMs
+int ns_group(const mw_net* n) {
+  if (!n->opts.resident_inverse) return 1;
+  const int d = n->layers[0].n_in;
+  const int tiles = ((d + 127) / 128) * ((d + 127) / 128);
+  int g = 2048 / tiles;
+  if (g < 1) g = 1;
+  if (g > kMaxGroup) g = kMaxGroup;
+  if (g > n->L) g = n->L;
+  return g;
 }
 
 TcOperand operand(const void* base, int rows, int cols, int planes, bool mn) {
@@ -153,8 +198,8 @@ Ctx make_ctx(mw_net* n, const Layout& lay, void* ws, cudaStream_t s) {
   return c;
 }
 
-// weight operand of layer l with `terms` terms (MW_F32: split planes in the workspace, made here
-// unless resident and already made; bf16: the caller's array itself)
+// weight operand of layer l (MW_F32: split planes in the workspace, made here when `make`;
+// bf16: the caller's array itself)
 mw_status weight_planes(const Ctx& c, int l, const void* W, bool make, const __nv_bfloat16** out) {
   if (c.n->opts.prec == MW_F32) {
     __nv_bfloat16* p = c.at<__nv_bfloat16>(c.lay->w_planes[l]);
@@ -166,52 +211,83 @@ mw_status weight_planes(const Ctx& c, int l, const void* W, bool make, const __n
   return MW_OK;
 }
 
-// W^-1 of layer l into the layer's inverse region as `ph` term planes (row-major X = W^-1)
-mw_status newton_schulz(const Ctx& c, int l, const void* W, const __nv_bfloat16* Wp) {
+// W^-1 of layers [l0, l0+G) into their inverse regions as `ph` term planes (row-major
+// X = W^-1), all G layers advancing together in batched launches.  Also leaves the split weight
+// planes of those layers in w_planes (MW_F32).
+mw_status newton_schulz_group(const Ctx& c, int l0, int G, const void* const* params) {
   const Layout& lay = *c.lay;
   const int d = c.dim;
-  float* X = c.at<float>(lay.ns_x);
-  // ns_r holds the residual planes [3][n*n] followed by two iterate plane sets [2][3][n*n]
-  __nv_bfloat16* xbase = c.at<__nv_bfloat16>(lay.ns_r) + 3 * c.nn;
-  __nv_bfloat16* Xp[2] = {xbase, xbase + 3 * c.nn};
-  __nv_bfloat16* Rp = c.at<__nv_bfloat16>(lay.ns_r);
-  double* sumsq = reinterpret_cast<double*>(c.at<char>(lay.inv_scratch));
-  float* cscale = reinterpret_cast<float*>(c.at<char>(lay.inv_scratch) + 64);
-  __nv_bfloat16* dst = c.at<__nv_bfloat16>(lay.inv[l]);
+  const bool f32 = c.n->opts.prec == MW_F32;
+  float* X = c.at<float>(lay.ns_x);                             // [G][n*n]
+  __nv_bfloat16* Rp = c.at<__nv_bfloat16>(lay.ns_r);            // [G][3][n*n]
+  __nv_bfloat16* Xp[2] = {Rp + (int64_t)3 * G * c.nn, Rp + (int64_t)6 * G * c.nn};
+  char* sc = c.at<char>(lay.inv_scratch);
+  double* sumsq = reinterpret_cast<double*>(sc);                // [G]
+  float* cscale = reinterpret_cast<float*>(sc + 8 * kMaxGroup); // [G]
+  double* fpart = reinterpret_cast<double*>(sc + 12 * kMaxGroup + 64);   // [G][kFrobBlocks]
+  __nv_bfloat16* dst = c.at<__nv_bfloat16>(lay.inv[l0]);
+  const int64_t dst_stride = G > 1 ? (int64_t)(lay.inv[l0 + 1].off - lay.inv[l0].off) / 2 : 0;
+
+  PtrBatch wp{};
+  for (int g = 0; g < G; ++g) wp.p[g] = params[l0 + g];
+  // the weight operand of the residual product
+  const __nv_bfloat16* Wbase;
+  int w_batch_planes;
+  if (f32) {
+    __nv_bfloat16* w0 = c.at<__nv_bfloat16>(lay.w_planes[l0]);
+    int64_t bx = (c.nn / 4 + 255) / 256;
+    if (bx > 64) bx = 64;
+    split_weights_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(wp, c.nn / 4, c.nn, w0);
+    MW_TRY(launch_ok());
+    Wbase = w0;
+    w_batch_planes = G > 1 ? (int)((lay.w_planes[l0 + 1].off - lay.w_planes[l0].off) / (2 * c.nn)) : 3;
+  } else if (G == 1) {
+    Wbase = (const __nv_bfloat16*)params[l0];
+    w_batch_planes = 1;
+  } else {
+    __nv_bfloat16* stage = c.at<__nv_bfloat16>(lay.ns_w);        // [G][n*n] bf16 copies
+    for (int g = 0; g < G; ++g)
+      MW_CUDA_OK(cudaMemcpyAsync(stage + (int64_t)g * c.nn, params[l0 + g], 2 * c.nn,
+                                 cudaMemcpyDeviceToDevice, c.s));
+    Wbase = stage;
+    w_batch_planes = 1;
+  }
 
   NsStep sched[16];
   const int steps = ns_schedule(c.n, sched);
   if (steps < 1) return MW_ERR_INVALID_ARG;
-  double* fpart = c.at<double>(lay.partials);
-  if (c.n->opts.prec == MW_F32) {
-    frob_partial_kernel<float><<<kFrobBlocks, 256, 0, c.s>>>((const float*)W, c.nn, fpart);
-    frob_final_kernel<<<1, 32, 0, c.s>>>(fpart, kFrobBlocks, d, cscale);
-    x0_kernel<float><<<dim3(d / 32, d / 32), 256, 0, c.s>>>((const float*)W, d, cscale, X);
+  if (f32) {
+    frob_partial_kernel<float><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
+    frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
+    x0_kernel<float><<<dim3(d / 32, d / 32, G), 256, 0, c.s>>>(wp, d, cscale, X);
   } else {
-    frob_partial_kernel<__nv_bfloat16><<<kFrobBlocks, 256, 0, c.s>>>((const __nv_bfloat16*)W, c.nn, fpart);
-    frob_final_kernel<<<1, 32, 0, c.s>>>(fpart, kFrobBlocks, d, cscale);
-    x0_kernel<__nv_bfloat16><<<dim3(d / 32, d / 32), 256, 0, c.s>>>((const __nv_bfloat16*)W, d, cscale, X);
+    frob_partial_kernel<__nv_bfloat16><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
+    frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
+    x0_kernel<__nv_bfloat16><<<dim3(d / 32, d / 32, G), 256, 0, c.s>>>(wp, d, cscale, X);
   }
   MW_TRY(launch_ok(3));
-  int have = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;   // terms of X currently split
-  MW_TRY(split_planes(X, c.nn, Xp[0], have, c.nn, c.s));
+  const int first = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;
+  MW_TRY(split_planes_batched(X, c.nn, G, c.nn, Xp[0], first, c.nn, 3 * c.nn, c.s));
   int cur = 0;
   for (int it = 0; it < steps; ++it) {
     const bool last = it + 1 == steps;
     const int pw = c.pr.pw < sched[it].pr ? c.pr.pw : sched[it].pr;
     // R = I - W X
-    MW_CUDA_OK(cudaMemsetAsync(sumsq, 0, sizeof(double), c.s));
+    MW_CUDA_OK(cudaMemsetAsync(sumsq, 0, sizeof(double) * G, c.s));
     TcEpilogue er;
     er.mode = TC_EPI_RESID;
-    er.planes = Rp; er.n_planes = sched[it].pu; er.plane_stride = c.nn;
-    er.sumsq = sumsq;
-    MW_TRY(tc_gemm(c.cache, operand(Wp, d, d, pw, false), operand(Xp[cur], d, d, sched[it].pr, true),
-                   d, d, d, er, c.st, c.s));
+    er.planes = Rp; er.n_planes = sched[it].pu; er.plane_stride = c.nn; er.bs_planes = 3 * c.nn;
+    er.sumsq = sumsq; er.bs_sumsq = 1;
+    TcOperand wa = operand(Wbase, d, d, pw, false);
+    wa.batch_planes = w_batch_planes;
+    TcOperand xb = operand(Xp[cur], d, d, sched[it].pr, true);
+    xb.batch_planes = 3;
+    MW_TRY(tc_gemm(c.cache, wa, xb, d, d, d, er, c.st, c.s, G));
     if (last) {
       // the update squares this residual: gate on it so a diverging layer is reported
-      const double limit = c.n->opts.prec == MW_F32 ? 2e-3 : 2e-2;
-      residual_gate_kernel<<<1, 32, 0, c.s>>>(sumsq, d, limit, c.st, l);
-      ++g_launch_count;
+      const double limit = f32 ? 2e-3 : 2e-2;
+      residual_gate_kernel<<<1, kMaxGroup, 0, c.s>>>(sumsq, G, d, limit, c.st, l0);
+      MW_TRY(launch_ok());
     }
     // X' = X + X R
     int next_terms = c.pr.ph;
@@ -220,22 +296,19 @@ mw_status newton_schulz(const Ctx& c, int l, const void* W, const __nv_bfloat16*
     eu.mode = TC_EPI_PLAIN;
     eu.addend = X;
     eu.out_f32 = last ? nullptr : X;
+    eu.bs_f32 = c.nn;
     eu.planes = last ? dst : Xp[cur ^ 1];
     eu.n_planes = next_terms;
     eu.plane_stride = c.nn;
-    MW_TRY(tc_gemm(c.cache, operand(Xp[cur], d, d, sched[it].pu, false),
-                   operand(Rp, d, d, sched[it].pu, true), d, d, d, eu, c.st, c.s));
+    eu.bs_planes = last ? dst_stride : 3 * c.nn;
+    TcOperand xa = operand(Xp[cur], d, d, sched[it].pu, false);
+    xa.batch_planes = 3;
+    TcOperand rb = operand(Rp, d, d, sched[it].pu, true);
+    rb.batch_planes = 3;
+    MW_TRY(tc_gemm(c.cache, xa, rb, d, d, d, eu, c.st, c.s, G));
     cur ^= 1;
-    have = next_terms;
   }
-  (void)have;
   return MW_OK;
-}
-
-mw_status prep_layer(const Ctx& c, int l, const void* W, bool make_w) {
-  const __nv_bfloat16* Wp = nullptr;
-  MW_TRY(weight_planes(c, l, W, make_w, &Wp));
-  return newton_schulz(c, l, W, Wp);
 }
 
 // x0 (caller's array) as a K-major / MN-major operand base with px terms
@@ -359,9 +432,11 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
       Region slot = b.take(2 * (size_t)pr.ph * nn);
       for (int l = 0; l < L; ++l) lay.inv[l] = slot;
     }
-    lay.ns_x = b.take(4 * nn);
-    lay.ns_r = b.take(2 * 9 * nn);      // R planes [3] + two iterate plane sets [2][3]
-    lay.inv_scratch = b.take(256);
+    const size_t G = (size_t)ns_group(n);
+    lay.ns_x = b.take(4 * nn * G);
+    lay.ns_r = b.take(2 * 9 * nn * G);  // per group member: R planes [3] + two iterate plane sets
+    if (n->opts.prec != MW_F32 && G > 1) lay.ns_w = b.take(2 * nn * G);
+    lay.inv_scratch = b.take(12 * kMaxGroup + 64 + 8 * (size_t)kMaxGroup * kFrobBlocks);
   }
   lay.total = b.cur;
 }
@@ -383,8 +458,10 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
   const int L = n->L, d = c.dim;
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
   const bool resident = n->opts.resident_inverse != 0;
-  if (resident)
-    for (int l = 0; l < L; ++l) MW_TRY(prep_layer(c, l, params[l], true));
+  if (resident) {
+    const int G = ns_group(n);
+    for (int l = 0; l < L; l += G) MW_TRY(newton_schulz_group(c, l, (L - l) < G ? (L - l) : G, params));
+  }
   MW_TRY(forward_pass(c, params, x, false));                 // Phase I
   MW_TRY(loss_and_top(c, target, loss_out, true));
   // Phase II: g_z planes ping-pong between hp[0] and hp[1]
@@ -437,11 +514,8 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
     const mw_layer_desc& ld = n->layers[l];
     const uint32_t* words = c.at<uint32_t>(lay.mask[l]);
     const __nv_bfloat16* Wp = nullptr;
-    if (resident) MW_TRY(weight_planes(c, l, params[l], false, &Wp));
-    else {
-      MW_TRY(weight_planes(c, l, params[l], true, &Wp));
-      MW_TRY(newton_schulz(c, l, params[l], Wp));
-    }
+    if (!resident) MW_TRY(newton_schulz_group(c, l, 1, params));
+    MW_TRY(weight_planes(c, l, params[l], false, &Wp));
     const __nv_bfloat16* hin = c.at<__nv_bfloat16>(lay.hp[l & 1]);
     __nv_bfloat16* hout = c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]);
     __nv_bfloat16* xout = c.at<__nv_bfloat16>(lay.xp[(l + 1) & 1]);
