@@ -50,6 +50,7 @@ void build_layout(mw_net* n, bool backprop, Layout& lay) {
   lay.mask.resize(L);
   lay.frag_cnt.resize(L);
   lay.frag_off.resize(L);
+  lay.frag_rank.resize(L);
   lay.frag_vals.resize(L);
   lay.reseed.resize(L + 1);
   lay.stored_act.resize(L + 1);
@@ -74,6 +75,8 @@ void build_layout(mw_net* n, bool backprop, Layout& lay) {
       if (n->layers[l].act == MW_ACT_RELU) {
         lay.frag_cnt[l] = b.take(sizeof(uint32_t) * n->info[l].rows);
         lay.frag_off[l] = b.take(sizeof(uint32_t) * n->info[l].rows);
+        if (n->backend == MW_BACKEND_TENSOR)
+          lay.frag_rank[l] = b.take(sizeof(uint32_t) * n->info[l].rows * ((n->info[l].cols + 63) / 64));
         lay.frag_vals[l] = b.take((n->opts.prec == MW_F64 ? 8 : 4) * (size_t)n->info[l].out_elems);
       }
     }

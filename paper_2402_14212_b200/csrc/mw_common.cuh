@@ -88,6 +88,10 @@ mw_status activation_vijp(const T* gz, const uint32_t* words, int64_t rows, int 
 mw_status fragment_offsets(const uint32_t* words, int64_t rows, int cols, uint32_t* cnt,
                            uint32_t* off, uint32_t* total, void* scratch, size_t scratch_bytes,
                            cudaStream_t s);
+// the same index built by one CTA, plus rank[r][c/64] = dead units of row r before column
+// 64*(c/64) (cols % 64 == 0; meant for a few thousand rows)
+mw_status fragment_index(const uint32_t* words, int rows, int cols, uint32_t* cnt, uint32_t* off,
+                         uint32_t* rank, uint32_t* total, cudaStream_t s);
 template <typename T>
 mw_status fragment_compact(const T* h, const uint32_t* words, int64_t rows, int cols,
                            const uint32_t* off, T* vals, cudaStream_t s);

@@ -267,9 +267,8 @@ dead_count_kernel(const uint32_t* __restrict__ words, int64_t rows, int cols, in
 }
 
 // single CTA, chunked exclusive scan with a running carry (deterministic, integer exact)
-__global__ void __launch_bounds__(1024)
-exclusive_scan_kernel(const uint32_t* __restrict__ cnt, int64_t rows, uint32_t* __restrict__ off,
-                      uint32_t* __restrict__ total) {
+__device__ __forceinline__ void block_exclusive_scan(const uint32_t* cnt, int64_t rows,
+                                                     uint32_t* off, uint32_t* total) {
   __shared__ uint32_t warp_sums[32];
   __shared__ uint32_t carry_s;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -304,6 +303,44 @@ exclusive_scan_kernel(const uint32_t* __restrict__ cnt, int64_t rows, uint32_t* 
   if (tid == 0 && total) *total = carry_s;
 }
 
+__global__ void __launch_bounds__(1024)
+exclusive_scan_kernel(const uint32_t* __restrict__ cnt, int64_t rows, uint32_t* __restrict__ off,
+                      uint32_t* __restrict__ total) {
+  block_exclusive_scan(cnt, rows, off, total);
+}
+
+// One CTA builds the whole index of a ReLU layer's fragment stream from its sign words:
+// cnt[r] dead units of row r, rank[r][t] dead units of row r before column 64 t, off = exclusive
+// scan of cnt over rows.  cols % 64 == 0.
+__global__ void __launch_bounds__(1024)
+fragment_index_kernel(const uint32_t* __restrict__ words, int rows, int cols, uint32_t* cnt,
+                      uint32_t* __restrict__ off, uint32_t* __restrict__ rank,
+                      uint32_t* __restrict__ total) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const int wpr = cols >> 5, tiles = cols >> 6;
+  for (int r = wid; r < rows; r += 32) {
+    uint32_t carry = 0;
+    for (int t0 = 0; t0 < tiles; t0 += 32) {
+      const int t = t0 + lane;
+      uint32_t d = 0;
+      if (t < tiles) {
+        const uint2 w = *reinterpret_cast<const uint2*>(words + (int64_t)r * wpr + 2 * t);
+        d = 64u - __popc(w.x) - __popc(w.y);
+      }
+      uint32_t incl = d;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      if (t < tiles) rank[(int64_t)r * tiles + t] = carry + incl - d;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) cnt[r] = carry;
+  }
+  __syncthreads();
+  block_exclusive_scan(cnt, rows, off, total);
+}
+
 mw_status fragment_offsets(const uint32_t* words, int64_t rows, int cols, uint32_t* cnt,
                            uint32_t* off, uint32_t* total, void* scratch, size_t scratch_bytes,
                            cudaStream_t s) {
@@ -314,6 +351,14 @@ mw_status fragment_offsets(const uint32_t* words, int64_t rows, int cols, uint32
   dead_count_kernel<<<grid_for(rows), kThreads, 0, s>>>(words, rows, cols, wpr, cnt);
   exclusive_scan_kernel<<<1, 1024, 0, s>>>(cnt, rows, off, total);
   return launch_ok(2);
+}
+
+mw_status fragment_index(const uint32_t* words, int rows, int cols, uint32_t* cnt, uint32_t* off,
+                         uint32_t* rank, uint32_t* total, cudaStream_t s) {
+  if (rows == 0) return MW_OK;
+  if (cols % 64 != 0) return MW_ERR_UNSUPPORTED;
+  fragment_index_kernel<<<1, 1024, 0, s>>>(words, rows, cols, cnt, off, rank, total);
+  return launch_ok();
 }
 
 // one warp per row; MODE 0: compact h at dead units into vals; MODE 1: restore (activation vijp

@@ -24,14 +24,15 @@ struct Layout {
   size_t total = 0;
   size_t residual = 0;  // bytes that must survive between the phases
   Region status, partials;
-  std::vector<Region> mask, frag_cnt, frag_off, frag_vals, reseed, stored_act;
+  std::vector<Region> mask, frag_cnt, frag_off, frag_rank, frag_vals, reseed, stored_act;
   Region frag_total, h_last;
   Region act[2], cot[2], z, gz, aux0, aux1;  // aux: conv vijp iterate / h', wgrad partials
   std::vector<Region> inv;                   // per layer (resident) or all the same slot
   Region inv_scratch;
   // tensor-core backend operands (bf16 term planes)
   std::vector<Region> w_planes;              // split weights (MW_F32), per layer or one slot
-  Region xp[2], hp[2], gzp, ns_r, ns_x, ns_w; // activation / cotangent / g_z planes, NS scratch
+  Region xp[3], hp[2], gzp[2], ns_r, ns_x, ns_w; // activation / cotangent / g_z planes, NS scratch
+  Region split[3];                           // K-split meeting places of concurrently running products
 };
 
 }  // namespace mw

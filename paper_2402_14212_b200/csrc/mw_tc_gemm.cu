@@ -1,23 +1,31 @@
-// tcgen05 / TMA product kernel for sm_100a (see mw_tc_gemm.cuh for the role of each call).
+// tcgen05 / TMA product kernel for sm_100a (see mw_tc_gemm.cuh for the role of each product).
 //
-// One CTA computes one 128 x BN tile of D.  192 threads:
+// One launch runs a group of independent products.  Their output tiles (128 rows x bn columns,
+// optionally cut along K) form one list of work units, sorted by cost; the grid is persistent
+// (at most one CTA per SM) and CTA c takes units c, 2G-1-c, 2G+c, ... ("snake" order, which keeps
+// the per-CTA sums close).  192 threads per CTA:
 //   warp 0      TMA producer: stages the bf16 term planes of A and B for one 64-deep K block
-//               (cp.async.bulk.tensor, 128-byte swizzle, no multicast) and signals an mbarrier;
-//   warp 1      allocates tensor memory, then one lane issues tcgen05.mma (kind::f16, bf16 in,
-//               fp32 accumulate in tensor memory) for every term pair of the K block and commits
-//               the stage's "empty" barrier; after the last block commits the accumulator barrier;
-//   warps 2..5  epilogue: tcgen05.ld 32 columns at a time (one row per thread), apply the fused
-//               step (activation + sign word, vjp scaling, leaky vijp, residual, ...), store.
+//               (cp.async.bulk.tensor, 128-byte swizzle, no multicast) in a ring of shared-memory
+//               stages that runs on across units;
+//   warp 1      allocates tensor memory (two accumulator sets of 256 columns), then one lane
+//               issues tcgen05.mma (kind::f16, bf16 in, fp32 accumulate).  Term planes of B sit
+//               next to each other in a stage, so ONE instruction of width (planes x bn) forms
+//               the products of one A plane with several B planes; the cross products of equal
+//               order land in the same column block;
+//   warps 2..5  epilogue: tcgen05.ld 32 columns at a time (one row per thread), add the column
+//               blocks in registers (round to nearest), apply the fused step (activation + sign
+//               word, vjp scaling, activation vijp with the ReLU fragment stream, residual, ...)
+//               and store.  While they drain one accumulator set the next unit fills the other.
 //
 // Accuracy: the tensor core truncates its fp32 accumulator at every instruction, a bias that grows
-// with the number of instructions feeding one accumulator (measured: 1e-5 relative after 256
-// steps).  So the leading term product rotates over several accumulators (one per K block,
-// round robin), the small cross terms go to one of their own, and the epilogue adds them in
-// registers with round-to-nearest: fp32-accurate results at tensor-core speed.
+// with the number of instructions feeding one accumulator.  For fp32-accurate products the
+// leading term therefore alternates between two column blocks from one K block to the next, and
+// the small cross terms have blocks of their own.
 // Every wait is bounded; on expiry the kernel records MW_ERR_TIMEOUT and unwinds (tensor memory
 // is always released).
 #include <cudaTypedefs.h>
 
+#include <algorithm>
 #include <map>
 #include <tuple>
 #include <vector>
@@ -33,21 +41,42 @@ constexpr int BK = 64;
 constexpr int kThreadsTc = 192;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far above any legitimate wait
 constexpr int kMaxStages = 8;
-constexpr int kMaxPairs = 6;
+constexpr int kMaxOps = 6;
 constexpr uint32_t kATileBytes = BM * BK * 2;  // one A term plane of one stage
+constexpr int kSetCols = 256;                  // tensor-memory columns of one accumulator set
+constexpr int kTmemCols = 512;
 
-struct TcParams {
-  int M, N, K;
-  int pa, pb;
-  int npairs;
-  int pair_a[kMaxPairs], pair_b[kMaxPairs];
-  int stages;
-  int nacc;        // tensor-memory accumulators in use (each BN columns)
-  int nbig;        // of those, the ones that take the leading (0,0) term, rotated over K blocks
-  int tmem_cols;   // allocated columns: power of two >= nacc * BN
-  int a_batch_planes, b_batch_planes;
+// one tcgen05.mma per 16-deep K step: A plane at a_off16, `width` columns of B starting at b_off16
+struct TcOp {
+  uint32_t a_off16, b_off16;   // offsets inside a stage, in 16-byte units
+  uint32_t idesc;
+  uint16_t dcol;               // first accumulator column (inside the set)
+  uint16_t rot;                // added to dcol on odd K blocks (alternating leading block)
+  uint32_t first_kbs;          // the first K step of this many leading K blocks overwrites
+};
+
+struct alignas(64) TcProblem {
+  CUtensorMap tmA, tmB;
   TcEpilogue epi;
+  int M, N, K, num_kb, kb_per_split, split;
+  int bn, tiles_n, tiles_mn, unit_begin, unit_count;
+  int pa, pb, a_mn, b_mn, a_batch_planes, b_batch_planes;
+  uint32_t b_tile_bytes, tx_bytes;
+  int nops, nblocks;
+  float* split_partials;
+  unsigned int* split_counters;
+  TcOp ops[kMaxOps];
+};
+
+struct alignas(64) TcGroupParams {
+  int nprob, total_units, stages, pad0;
+  uint32_t stage_bytes, pad1;
   DeviceStatus* st;
+  TcProblem prob[kTcMaxGroup];
+};
+
+struct Unit {
+  int q, m0, n0, z, kb0, kb1, tl, ks;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -60,6 +89,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -78,20 +110,22 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 // Bounded wait: try_wait suspends the thread in hardware until the phase completes or its own
-// time slice ends, so the loop does not burn issue slots and adds no wake-up latency.  The bound
-// is wall time (checked every 256 polls); on expiry the timeout is recorded and false returned.
+// time slice ends.  The bound is wall time (checked every 256 polls); a wait also gives up when
+// another role of the CTA has already failed.  On expiry the timeout is recorded.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, DeviceStatus* st,
-                                          unsigned who) {
+                                          unsigned who, volatile int* abort_flag) {
   uint64_t t0 = 0;
   for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u) {
+      if (*abort_flag) return false;
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
       else if (now - t0 > kWaitLimitNs) break;
     }
   }
-  record_error(st, MW_ERR_TIMEOUT, who, blockIdx.x, blockIdx.y, blockIdx.z);
+  record_error(st, MW_ERR_TIMEOUT, who, blockIdx.x, 0u, 0u);
+  *abort_flag = 1;
   return false;
 }
 
@@ -104,23 +138,22 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       : "memory");
 }
 
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, bool mn_major, uint32_t lbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)((mn_major ? (lbo_bytes >> 4) : 1u) & 0x3FFFu) << 16;  // leading byte offset
-  d |= (uint64_t)((1024u >> 4) & 0x3FFFu) << 32;                         // stride byte offset
-  d |= (uint64_t)1 << 46;                                                // descriptor version
-  d |= (uint64_t)2 << 61;                                                // 128-byte swizzle
-  return d;
+// shared-memory operand descriptor, 128-byte swizzle: the upper word is constant, the lower word
+// holds the start address (and, for MN-major tiles, the distance between 64-element groups)
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo_base(bool mn_major) {
+  return (mn_major ? (8192u >> 4) : 1u) << 16;
 }
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo,
                                           uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %5};\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(tmem_d),
+      "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -134,8 +167,7 @@ __device__ __forceinline__ void tc_fence_after() {
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -147,9 +179,9 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // write 32 consecutive values as `planes` bf16 term planes (v is left holding the remainder)
@@ -175,6 +207,14 @@ __device__ __forceinline__ void store_f32x32(const float (&v)[32], float* dst) {
   float4* d4 = reinterpret_cast<float4*>(dst);
 #pragma unroll
   for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+}
+
+// position in the fragment stream of the first dead unit of (row, 32-column chunk at col0)
+__device__ __forceinline__ uint32_t frag_base(const TcEpilogue& e, int N, int row, int col0,
+                                              int64_t woff) {
+  uint32_t b = e.frag_off[row] + e.frag_rank[(int64_t)row * (N >> 6) + (col0 >> 6)];
+  if (col0 & 32) b += 32u - __popc(e.mask[woff - 1]);
+  return b;
 }
 
 // the fused step applied to one row chunk of 32 accumulator columns
@@ -235,9 +275,16 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int r
     }
     case TC_EPI_BWD: {
       if (e.out_f32) store_f32x32(v, e.out_f32 + off);
+      const uint32_t word = e.act != MW_ACT_NONE ? e.mask[woff] : 0xffffffffu;
+      if (e.act == MW_ACT_RELU && e.frag_vals) {
+        // fragments: the cotangent at dead units, in column order
+        uint32_t pos = frag_base(e, N, row, col0, woff);
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (!((word >> i) & 1u)) e.frag_vals[pos++] = v[i];
+      }
       if (e.n_planes) {
         if (e.act != MW_ACT_NONE) {
-          const uint32_t word = e.mask[woff];
           const float nf = e.act == MW_ACT_LEAKY_RELU ? e.slope : 0.f;
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = ((word >> i) & 1u) ? v[i] : nf * v[i];
@@ -247,19 +294,31 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int r
       break;
     }
     case TC_EPI_VIJP: {
-      if (e.out_f32) store_f32x32(v, e.out_f32 + off);
-      if (e.n_planes2) {
-        float h[32];
-        if (e.act == MW_ACT_LEAKY_RELU) {
-          const uint32_t word = e.mask[woff];
+      float h[32];
+      if (e.act == MW_ACT_LEAKY_RELU) {
+        const uint32_t word = e.mask[woff];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) h[i] = ((word >> i) & 1u) ? v[i] : v[i] / e.slope;
-        } else {
+        for (int i = 0; i < 32; ++i) h[i] = ((word >> i) & 1u) ? v[i] : v[i] / e.slope;
+      } else if (e.act == MW_ACT_RELU) {
+        // live units pass g_z on (phi' = 1); dead units take their stored cotangent back and
+        // contribute nothing to the weight vjp
+        const uint32_t word = e.mask[woff];
+        uint32_t pos = frag_base(e, N, row, col0, woff);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) h[i] = v[i];
+        for (int i = 0; i < 32; ++i) {
+          if ((word >> i) & 1u) {
+            h[i] = v[i];
+          } else {
+            h[i] = e.frag_vals[pos++];
+            v[i] = 0.f;
+          }
         }
-        store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, off);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) h[i] = v[i];
       }
+      if (e.out_f32) store_f32x32(h, e.out_f32 + off);
+      if (e.n_planes2) store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, off);
       if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off);
       break;
     }
@@ -268,26 +327,49 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int r
   }
 }
 
-template <bool A_MN, bool B_MN, int BN>
+// unit u of the sorted list -> product, tile, batch item and K range
+__device__ __forceinline__ void decode_unit(const TcGroupParams& p, int u, Unit& w) {
+  int q = 0;
+#pragma unroll
+  for (int i = 1; i < kTcMaxGroup; ++i)
+    if (i < p.nprob && u >= p.prob[i].unit_begin) q = i;
+  const TcProblem& P = p.prob[q];
+  const int local = u - P.unit_begin;
+  const int tl = local / P.split;
+  const int ks = local - tl * P.split;
+  const int z = tl / P.tiles_mn;
+  const int r = tl - z * P.tiles_mn;
+  const int mt = r / P.tiles_n;
+  w.q = q;
+  w.tl = tl;
+  w.ks = ks;
+  w.z = z;
+  w.m0 = mt * BM;
+  w.n0 = (r - mt * P.tiles_n) * P.bn;
+  w.kb0 = ks * P.kb_per_split;
+  const int e = w.kb0 + P.kb_per_split;
+  w.kb1 = e < P.num_kb ? e : P.num_kb;
+}
+
+// units of this CTA: round r takes index r*G + c (even r) or r*G + G-1-c (odd r)
+#define MW_FOR_MY_UNITS(p, u)                                                              \
+  for (int r_ = 0, u = 0; r_ * (int)gridDim.x < (p).total_units; ++r_)                   \
+    if ((u = r_ * (int)gridDim.x +                                                        \
+             ((r_ & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x)) <       \
+        (p).total_units)
+
 __global__ void __launch_bounds__(kThreadsTc, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ TcParams p) {
+tc_group_kernel(const __grid_constant__ TcGroupParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[kMaxStages];
   __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
-  __shared__ __align__(8) uint64_t accum_bar;
+  __shared__ __align__(8) uint64_t acc_full[2];
+  __shared__ __align__(8) uint64_t acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * BN;
-  const int m0 = blockIdx.y * BM;
-  const int bz = blockIdx.z;
-  const int a_pl0 = bz * p.a_batch_planes, b_pl0 = bz * p.b_batch_planes;
-  const int num_kb = (p.K + BK - 1) / BK;
-  constexpr uint32_t kBTileBytes = BN * BK * 2;
-  const uint32_t stage_bytes = p.pa * kATileBytes + p.pb * kBTileBytes;
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;  // 1024-byte aligned for the swizzle
 
   if (threadIdx.x == 0) {
@@ -295,7 +377,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
-    mbar_init(smem_u32(&accum_bar), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&acc_full[s]), 1);
+      mbar_init(smem_u32(&acc_empty[s]), 4);   // one arrival per epilogue warp
+    }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -303,7 +388,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(&tmem_slot)),
-                 "r"((uint32_t)p.tmem_cols)
+                 "r"((uint32_t)kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -311,114 +396,200 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot;
+  volatile int* abortp = &abort_flag;
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      int issued = 0;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % p.stages;
-        const uint32_t ph = (uint32_t)(kb / p.stages) & 1u;
-        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, p.st, 1u)) { abort_flag = 1; break; }
-        const uint32_t fb = smem_u32(&full_bar[s]);
-        mbar_expect_tx(fb, stage_bytes);
-        const uint32_t sbase = tiles + (uint32_t)s * stage_bytes;
-        for (int pl = 0; pl < p.pa; ++pl) {
-          const uint32_t dst = sbase + (uint32_t)pl * kATileBytes;
-          if (A_MN) {
-            tma_load_3d(dst, &tmA, fb, m0, kb * BK, a_pl0 + pl);
-            tma_load_3d(dst + 8192u, &tmA, fb, m0 + 64, kb * BK, a_pl0 + pl);
-          } else {
-            tma_load_3d(dst, &tmA, fb, kb * BK, m0, a_pl0 + pl);
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      MW_FOR_MY_UNITS(p, u) {
+        if (!ok) break;
+        Unit w;
+        decode_unit(p, u, w);
+        const TcProblem& P = p.prob[w.q];
+        const int a_pl0 = w.z * P.a_batch_planes, b_pl0 = w.z * P.b_batch_planes;
+        const int pa = P.pa, pb = P.pb, nbox = P.bn >> 6;
+        const bool a_mn = P.a_mn != 0, b_mn = P.b_mn != 0;
+        const uint32_t b_tile_bytes = P.b_tile_bytes, tx = P.tx_bytes;
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
+          if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, p.st, 1u, abortp)) { ok = false; break; }
+          const uint32_t fb = smem_u32(&full_bar[stage]);
+          mbar_expect_tx(fb, tx);
+          const uint32_t sbase = tiles + stage * p.stage_bytes;
+          const int k0 = kb * BK;
+          for (int pl = 0; pl < pa; ++pl) {
+            const uint32_t dst = sbase + (uint32_t)pl * kATileBytes;
+            if (a_mn) {
+              tma_load_3d(dst, &P.tmA, fb, w.m0, k0, a_pl0 + pl);
+              tma_load_3d(dst + 8192u, &P.tmA, fb, w.m0 + 64, k0, a_pl0 + pl);
+            } else {
+              tma_load_3d(dst, &P.tmA, fb, k0, w.m0, a_pl0 + pl);
+            }
           }
-        }
-        const uint32_t bbase = sbase + (uint32_t)p.pa * kATileBytes;
-        for (int pl = 0; pl < p.pb; ++pl) {
-          const uint32_t dst = bbase + (uint32_t)pl * kBTileBytes;
-          if (B_MN) {
-#pragma unroll
-            for (int h = 0; h < BN / 64; ++h)
-              tma_load_3d(dst + (uint32_t)h * 8192u, &tmB, fb, n0 + h * 64, kb * BK, b_pl0 + pl);
-          } else {
-            tma_load_3d(dst, &tmB, fb, kb * BK, n0, b_pl0 + pl);
+          const uint32_t bbase = sbase + (uint32_t)pa * kATileBytes;
+          for (int pl = 0; pl < pb; ++pl) {
+            const uint32_t dst = bbase + (uint32_t)pl * b_tile_bytes;
+            if (b_mn) {
+              for (int h = 0; h < nbox; ++h)
+                tma_load_3d(dst + (uint32_t)h * 8192u, &P.tmB, fb, w.n0 + h * 64, k0, b_pl0 + pl);
+            } else {
+              tma_load_3d(dst, &P.tmB, fb, k0, w.n0, b_pl0 + pl);
+            }
           }
+          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
         }
-        ++issued;
       }
-      (void)issued;
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) |
-                             ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) |
-                             ((uint32_t)(BM >> 4) << 24);
-      uint32_t written = 0;   // bit a: accumulator a already holds a partial sum
-      const int big_base = p.nacc - p.nbig;
+      uint32_t stage = 0, phase = 0;
+      int j = 0;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % p.stages;
-        const uint32_t ph = (uint32_t)(kb / p.stages) & 1u;
-        if (!mbar_wait(smem_u32(&full_bar[s]), ph, p.st, 2u)) { abort_flag = 1; ok = false; break; }
+      MW_FOR_MY_UNITS(p, u) {
+        if (!ok) break;
+        Unit w;
+        decode_unit(p, u, w);
+        const TcProblem& P = p.prob[w.q];
+        const uint32_t set = (uint32_t)j & 1u, aphase = ((uint32_t)j >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&acc_empty[set]), aphase ^ 1u, p.st, 2u, abortp)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t sbase = tiles + (uint32_t)s * stage_bytes;
-        const uint32_t bbase = sbase + (uint32_t)p.pa * kATileBytes;
-        for (int q = 0; q < p.npairs; ++q) {
-          const bool leading = p.pair_a[q] == 0 && p.pair_b[q] == 0;
-          const int acc = (leading || big_base == 0) ? big_base + kb % p.nbig : 0;
-          const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BN);
-          uint32_t accumulate = (written >> acc) & 1u;
-          written |= 1u << acc;
-          const uint64_t adesc0 = make_smem_desc(sbase + (uint32_t)p.pair_a[q] * kATileBytes, A_MN, 8192u);
-          const uint64_t bdesc0 = make_smem_desc(bbase + (uint32_t)p.pair_b[q] * kBTileBytes, B_MN, 8192u);
+        const uint32_t d_set = tmem_base + set * (uint32_t)kSetCols;
+        // the unit's instruction list, in registers
+        uint32_t oa[kMaxOps], ob[kMaxOps], oi[kMaxOps], od[kMaxOps], orot[kMaxOps], ofk[kMaxOps];
+        const int nops = P.nops;
+#pragma unroll
+        for (int o = 0; o < kMaxOps; ++o) {
+          const TcOp op = P.ops[o < nops ? o : 0];
+          oa[o] = op.a_off16 | desc_lo_base(P.a_mn != 0);
+          ob[o] = op.b_off16 | desc_lo_base(P.b_mn != 0);
+          oi[o] = op.idesc;
+          od[o] = d_set + op.dcol;
+          orot[o] = op.rot;
+          ofk[o] = op.first_kbs;
+        }
+        // K advance of 16 elements: 32 bytes along a K-major row, 16 rows of 128 bytes otherwise
+        const uint32_t a_kadv = P.a_mn ? (2048u >> 4) : (32u >> 4);
+        const uint32_t b_kadv = P.b_mn ? (2048u >> 4) : (32u >> 4);
+        const int nkb = w.kb1 - w.kb0;
+        for (int kbl = 0; kbl < nkb; ++kbl) {
+          if (!mbar_wait(smem_u32(&full_bar[stage]), phase, p.st, 3u, abortp)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sb16 = (tiles + stage * p.stage_bytes) >> 4;
+          const uint32_t odd = (uint32_t)kbl & 1u;
 #pragma unroll
           for (int k4 = 0; k4 < BK / 16; ++k4) {
-            // K-major: 16 elements = 32 bytes along the row; MN-major: 16 rows of 128 bytes
-            const uint64_t adesc = adesc0 + (uint64_t)((A_MN ? 2048u : 32u) >> 4) * (uint64_t)k4;
-            const uint64_t bdesc = bdesc0 + (uint64_t)((B_MN ? 2048u : 32u) >> 4) * (uint64_t)k4;
-            umma_bf16(tmem_d, adesc, bdesc, idesc, accumulate);
-            accumulate = 1;
+#pragma unroll
+            for (int o = 0; o < kMaxOps; ++o) {
+              if (o < nops) {
+                const uint32_t acc = (k4 == 0 && (uint32_t)kbl < ofk[o]) ? 0u : 1u;
+                umma_bf16(od[o] + (odd ? orot[o] : 0u), oa[o] + sb16 + (uint32_t)k4 * a_kadv,
+                          ob[o] + sb16 + (uint32_t)k4 * b_kadv, oi[o], acc);
+              }
+            }
           }
+          umma_commit(smem_u32(&empty_bar[stage]));  // frees the stage once these products retire
+          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
         }
-        umma_commit(smem_u32(&empty_bar[s]));  // frees the stage once these products retire
+        if (!ok) break;
+        umma_commit(smem_u32(&acc_full[set]));
+        ++j;
       }
-      if (ok) umma_commit(smem_u32(&accum_bar));
     }
   } else {
     // ---------------- epilogue (warps 2..5) ----------------
     const int quarter = warp & 3;                 // tensor-memory lane quarter this warp may read
-    const int row = m0 + quarter * 32 + lane;
-    double sumsq_local = 0.0;
-    TcEpilogue epi = p.epi;           // this batch item's view of the outputs
-    if (bz) {
-      if (epi.addend) epi.addend += (int64_t)bz * epi.bs_f32;
-      if (epi.out_f32) epi.out_f32 += (int64_t)bz * epi.bs_f32;
-      if (epi.planes) epi.planes += (int64_t)bz * epi.bs_planes;
-      if (epi.planes2) epi.planes2 += (int64_t)bz * epi.bs_planes2;
-      if (epi.mask) epi.mask += (int64_t)bz * epi.bs_mask;
-      if (epi.sumsq) epi.sumsq += (int64_t)bz * epi.bs_sumsq;
-    }
-    // every lane observes the barrier itself; the warp then takes one common decision so the
-    // warp-wide tensor-memory loads below are never executed by part of a warp
-    const bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&accum_bar), 0u, p.st, 3u));
-    tc_fence_after();
-    if (ok) {
+    int j = 0;
+    bool ok = true;
+    MW_FOR_MY_UNITS(p, u) {
+      if (!ok) break;
+      Unit w;
+      decode_unit(p, u, w);
+      const TcProblem& P = p.prob[w.q];
+      const uint32_t set = (uint32_t)j & 1u, aphase = ((uint32_t)j >> 1) & 1u;
+      // every lane observes the barrier itself; the warp then takes one common decision so the
+      // warp-wide tensor-memory loads below are never executed by part of a warp
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&acc_full[set]), aphase, p.st, 4u, abortp));
+      if (!ok) break;
+      tc_fence_after();
+      const int row = w.m0 + quarter * 32 + lane;
+      const int bn = P.bn, nblk = P.nblocks, N = P.N;
+      TcEpilogue epi = P.epi;           // this batch item's view of the outputs
+      if (w.z) {
+        const int64_t z = w.z;
+        if (epi.addend) epi.addend += z * epi.bs_f32;
+        if (epi.out_f32) epi.out_f32 += z * epi.bs_f32;
+        if (epi.planes) epi.planes += z * epi.bs_planes;
+        if (epi.planes2) epi.planes2 += z * epi.bs_planes2;
+        if (epi.mask) epi.mask += z * epi.bs_mask;
+        if (epi.sumsq) epi.sumsq += z * epi.bs_sumsq;
+      }
+      double sumsq_local = 0.0;
+      const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + set * (uint32_t)kSetCols;
+      const bool split = P.split > 1;
+      float* part = nullptr;
+      if (split)
+        part = P.split_partials + ((int64_t)w.tl * P.split + w.ks) * (int64_t)(BM * bn) +
+               (int64_t)(quarter * 32 + lane) * bn;
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = 0; c < bn; c += 32) {
+        if (w.n0 + c >= N) break;
+        uint32_t r0[32];
         float v[32];
-        const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c;
-        tmem_ld32(t0, v);
-        for (int a = 1; a < p.nacc; ++a) {
-          float t[32];
-          tmem_ld32(t0 + (uint32_t)(a * BN), t);
+        tmem_ld32_issue(t0 + (uint32_t)c, r0);
+        tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] += t[i];
+        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
+        for (int b = 1; b < nblk; ++b) {
+          tmem_ld32_issue(t0 + (uint32_t)(b * bn + c), r0);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] += __uint_as_float(r0[i]);
         }
-        if (row < p.M) epilogue_chunk(epi, p.N, row, n0 + c, v, sumsq_local);
+        if (split) store_f32x32(v, part + c);
+        else if (row < P.M) epilogue_chunk(epi, N, row, w.n0 + c, v, sumsq_local);
+      }
+      // this warp has read its part of the accumulator set: hand it back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&acc_empty[set]));
+      ++j;
+      if (split) {
+        // the warp that finds the other K pieces of its 32 rows complete adds all pieces in
+        // fixed order and applies the fused step
+        __threadfence();
+        __syncwarp();
+        unsigned int* cnt = P.split_counters + (int64_t)w.tl * 4 + quarter;
+        unsigned int old = 0;
+        if (lane == 0) old = atomicAdd(cnt, 1u);
+        old = __shfl_sync(0xffffffffu, old, 0);
+        if (old == (unsigned)P.split - 1u) {
+          __threadfence();
+          const float* p0 = P.split_partials + (int64_t)w.tl * P.split * (int64_t)(BM * bn) +
+                            (int64_t)(quarter * 32 + lane) * bn;
+#pragma unroll 1
+          for (int c = 0; c < bn; c += 32) {
+            if (w.n0 + c >= N) break;
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = 0.f;
+            for (int s = 0; s < P.split; ++s) {
+              const float4* q4 = reinterpret_cast<const float4*>(p0 + (int64_t)s * (BM * bn) + c);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float4 t = __ldcg(q4 + i);
+                v[4 * i] += t.x; v[4 * i + 1] += t.y; v[4 * i + 2] += t.z; v[4 * i + 3] += t.w;
+              }
+            }
+            if (row < P.M) epilogue_chunk(epi, N, row, w.n0 + c, v, sumsq_local);
+          }
+          if (lane == 0) *cnt = 0u;     // ready for the next launch
+        }
       }
       if (epi.mode == TC_EPI_RESID && epi.sumsq) {
         for (int o = 16; o; o >>= 1) sumsq_local += __shfl_xor_sync(0xffffffffu, sumsq_local, o);
-        if (lane == 0) atomicAdd(epi.sumsq, sumsq_local);
+        if (lane == 0 && sumsq_local != 0.0) atomicAdd(epi.sumsq, sumsq_local);
       }
     }
   }
@@ -431,7 +602,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (uint32_t i = 0; i < 4096u && !mbar_try_wait(smem_u32(&full_bar[s]), 0u); ++i) __nanosleep(256);
   }
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
                  : "memory");
   }
 }
@@ -453,7 +624,51 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+// tile width: as wide as the accumulator set allows for the number of term orders, narrowed while
+// the product alone cannot give every SM a tile
+int pick_bn(int pa, int pb, int M, int N, int batch) {
+  const int t = pa > pb ? pa : pb;
+  int bn = t == 1 ? 256 : (t == 2 ? 128 : 64);
+  const int tm = (M + BM - 1) / BM;
+  while (bn > 64 && (N % bn != 0 || (int64_t)tm * (N / bn) * batch < sm_count())) bn >>= 1;
+  return bn;
+}
+
 }  // namespace
+
+int tc_tile_n(int a_planes, int b_planes, int M, int N, int batch) {
+  return pick_bn(a_planes, b_planes, M, N, batch);
+}
+
+size_t tc_split_scratch_bytes(int a_planes, int b_planes, int M, int N, int batch, int split_k) {
+  if (split_k <= 1) return 0;
+  const int bn = pick_bn(a_planes, b_planes, M, N, batch);
+  const size_t tiles = (size_t)((M + BM - 1) / BM) * ((N + bn - 1) / bn) * batch;
+  return kTcSplitCounterBytes + align_up(tiles * split_k * BM * bn * sizeof(float), 256);
+}
+
+int tc_auto_split(int a_planes, int b_planes, int M, int N, int K, int batch) {
+  const int bn = pick_bn(a_planes, b_planes, M, N, batch);
+  const int64_t units = (int64_t)((M + BM - 1) / BM) * ((N + bn - 1) / bn) * batch;
+  const int sms = sm_count();
+  if (units * 5 >= (int64_t)sms * 3) return 1;
+  int s = (int)((sms + units - 1) / units);
+  const int num_kb = (K + BK - 1) / BK;
+  if (s > num_kb / 2) s = num_kb / 2;
+  if (s > 8) s = 8;
+  return s < 1 ? 1 : s;
+}
 
 // ---- optional per-launch timing of the product kernel (measurement hook) -----------------
 struct TcProfile {
@@ -525,115 +740,184 @@ static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, i
   return MW_OK;
 }
 
-template <bool A_MN, bool B_MN, int BN>
-static mw_status launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParams& prm, int batch,
-                           cudaStream_t s) {
-  const uint32_t stage_bytes = prm.pa * kATileBytes + prm.pb * (BN * BK * 2);
+namespace {
+
+uint32_t make_idesc(bool a_mn, bool b_mn, int n) {
+  // fp32 accumulate, bf16 A and B, major-ness of A and B, N / 8, M / 16
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+// the instruction list of one K step: one instruction per A plane covering the B planes whose
+// cross product with it is kept (i + j < max(pa, pb)); products of equal order i + j share a
+// column block.  Returns the tensor-core cycles of one K block (for sorting).
+double build_ops(TcProblem& P, bool rotate) {
+  const int pa = P.pa, pb = P.pb, bn = P.bn;
+  const int t = pa > pb ? pa : pb;
+  const int lead = rotate ? 1 : 0;            // extra column block for the alternating leading term
+  auto col = [&](int order) { return (order == 0 ? 0 : (order + lead)) * bn; };
+  const uint32_t b0 = (uint32_t)pa * kATileBytes;
+  bool init[8] = {false, false, false, false, false, false, false, false};
+  int n = 0;
+  double cycles = 0.0;
+  auto add = [&](int i, int j0, int cnt, int rot, int first) {
+    TcOp& o = P.ops[n++];
+    o.a_off16 = ((uint32_t)i * kATileBytes) >> 4;
+    o.b_off16 = (b0 + (uint32_t)j0 * P.b_tile_bytes) >> 4;
+    o.idesc = make_idesc(P.a_mn != 0, P.b_mn != 0, cnt * bn);
+    o.dcol = (uint16_t)col(i + j0);
+    o.rot = (uint16_t)rot;
+    o.first_kbs = (uint32_t)first;
+    const double w = cnt * bn;
+    cycles += 4.0 * std::max(w / 2.0, (128.0 + w) / 4.0);   // math vs shared-memory operand reads
+  };
+  for (int i = 0; i < pa; ++i) {
+    int cnt = pb < t - i ? pb : t - i;
+    if (cnt <= 0) continue;
+    int j0 = 0;
+    if (i == 0 && rotate) {
+      add(0, 0, 1, bn, 2);
+      init[0] = true;
+      j0 = 1;
+      --cnt;
+      if (cnt <= 0) continue;
+    }
+    // blocks i+j0 .. i+j0+cnt-1: one instruction when they are all fresh or all started
+    bool all_init = true, none_init = true;
+    for (int b = i + j0; b < i + j0 + cnt; ++b) {
+      if (init[b]) none_init = false; else all_init = false;
+    }
+    if (all_init || none_init) {
+      add(i, j0, cnt, 0, none_init ? 1 : 0);
+    } else {
+      for (int b = 0; b < cnt; ++b) add(i, j0 + b, 1, 0, init[i + j0 + b] ? 0 : 1);
+    }
+    for (int b = i + j0; b < i + j0 + cnt; ++b) init[b] = true;
+  }
+  P.nops = n;
+  P.nblocks = t + lead;
+  return cycles;
+}
+
+}  // namespace
+
+mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceStatus* st,
+                        cudaStream_t s) {
+  if (count < 1 || count > kTcMaxGroup) return MW_ERR_INVALID_ARG;
+  static thread_local TcGroupParams prm;
+  prm.nprob = 0;
+  prm.st = st;
+  double cost[kTcMaxGroup];
+  double flops = 0.0, mma_flops = 0.0;
+  uint32_t stage_bytes = 0;
+  for (int i = 0; i < count; ++i) {
+    const TcGemm& d = g[i];
+    if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.batch <= 0) continue;
+    if (d.N % 64 != 0) return MW_ERR_UNSUPPORTED;
+    // a ragged K tail is zero-filled by the copies of MN-major operands (K counts their rows)
+    if ((!d.A.mn_major || !d.B.mn_major) && d.K % 64 != 0) return MW_ERR_UNSUPPORTED;
+    if (d.A.planes < 1 || d.A.planes > 3 || d.B.planes < 1 || d.B.planes > 3) return MW_ERR_INVALID_ARG;
+    if (d.A.mn_major && (d.M % 64 != 0)) return MW_ERR_UNSUPPORTED;
+    TcProblem& P = prm.prob[prm.nprob];
+    P.M = d.M; P.N = d.N; P.K = d.K;
+    P.pa = d.A.planes; P.pb = d.B.planes;
+    P.a_mn = d.A.mn_major ? 1 : 0;
+    P.b_mn = d.B.mn_major ? 1 : 0;
+    P.a_batch_planes = d.A.batch_planes ? d.A.batch_planes : d.A.planes;
+    P.b_batch_planes = d.B.batch_planes ? d.B.batch_planes : d.B.planes;
+    P.bn = pick_bn(P.pa, P.pb, d.M, d.N, d.batch);
+    P.num_kb = (d.K + BK - 1) / BK;
+    int split = d.split_k > 1 ? d.split_k : 1;
+    if (split > P.num_kb) split = P.num_kb;
+    P.kb_per_split = (P.num_kb + split - 1) / split;
+    split = (P.num_kb + P.kb_per_split - 1) / P.kb_per_split;
+    P.split = split;
+    const int tiles_m = (d.M + BM - 1) / BM;
+    P.tiles_n = (d.N + P.bn - 1) / P.bn;
+    P.tiles_mn = tiles_m * P.tiles_n;
+    const int64_t units = (int64_t)P.tiles_mn * d.batch * split;
+    if (units > (1 << 30)) return MW_ERR_UNSUPPORTED;
+    P.unit_count = (int)units;
+    P.b_tile_bytes = (uint32_t)P.bn * BK * 2;
+    P.tx_bytes = (uint32_t)P.pa * kATileBytes + (uint32_t)P.pb * P.b_tile_bytes;
+    if (P.tx_bytes > stage_bytes) stage_bytes = P.tx_bytes;
+    const int t = P.pa > P.pb ? P.pa : P.pb;
+    // fp32-accurate products alternate the leading block (needs two K blocks per unit)
+    const bool rotate = t == 3 && P.pa == 3 && P.pb == 3 && P.kb_per_split >= 2 &&
+                        (P.num_kb - (split - 1) * P.kb_per_split) >= 2;
+    const double kb_cycles = build_ops(P, rotate);
+    cost[prm.nprob] = kb_cycles * P.kb_per_split;
+    P.epi = d.epi;
+    P.split_partials = nullptr;
+    P.split_counters = nullptr;
+    if (split > 1) {
+      if (!d.split_scratch || ((uintptr_t)d.split_scratch & 255u)) return MW_ERR_WORKSPACE;
+      const size_t tiles = (size_t)P.tiles_mn * d.batch;
+      if (tiles * 4 * sizeof(unsigned) > kTcSplitCounterBytes) return MW_ERR_UNSUPPORTED;
+      P.split_counters = static_cast<unsigned int*>(d.split_scratch);
+      P.split_partials = reinterpret_cast<float*>(static_cast<char*>(d.split_scratch) + kTcSplitCounterBytes);
+    }
+    const int a_total = d.batch > 1 ? (d.batch - 1) * P.a_batch_planes + d.A.planes : d.A.planes;
+    const int b_total = d.batch > 1 ? (d.batch - 1) * P.b_batch_planes + d.B.planes : d.B.planes;
+    MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA));
+    MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
+    int np = 0;
+    for (int a = 0; a < P.pa; ++a)
+      for (int b = 0; b < P.pb; ++b)
+        if (a + b < t) ++np;
+    flops += 2.0 * d.M * d.N * d.K * d.batch;
+    mma_flops += 2.0 * d.M * d.N * d.K * np * d.batch;
+    ++prm.nprob;
+  }
+  if (prm.nprob == 0) return MW_OK;
+  // costliest units first
+  for (int i = 1; i < prm.nprob; ++i)
+    for (int j = i; j > 0 && cost[j] > cost[j - 1]; --j) {
+      std::swap(cost[j], cost[j - 1]);
+      std::swap(prm.prob[j], prm.prob[j - 1]);
+    }
+  int total = 0;
+  for (int i = 0; i < prm.nprob; ++i) {
+    prm.prob[i].unit_begin = total;
+    total += prm.prob[i].unit_count;
+  }
+  prm.total_units = total;
+  prm.stage_bytes = stage_bytes;
   const uint32_t budget = 227u * 1024u - 2048u;   // static barriers + alignment slack
   int stages = (int)(budget / stage_bytes);
   if (stages > kMaxStages) stages = kMaxStages;
-  const int num_kb = (prm.K + BK - 1) / BK;
-  if (stages > num_kb) stages = num_kb < 1 ? 1 : num_kb;
-  if (stages < 1) return MW_ERR_UNSUPPORTED;
+  if (stages < 2) return MW_ERR_UNSUPPORTED;
   prm.stages = stages;
-  const int small = prm.npairs > 1 ? 1 : 0;
-  int nbig = 512 / BN - small;
-  if (nbig > num_kb) nbig = num_kb;
-  prm.nbig = nbig;
-  prm.nacc = nbig + small;
-  int cols = 32;
-  while (cols < prm.nacc * BN) cols *= 2;
-  prm.tmem_cols = cols;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   static bool attr_set = false;
   if (!attr_set) {
-    MW_CUDA_OK(cudaFuncSetAttribute(tc_gemm_kernel<A_MN, B_MN, BN>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024));
+    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    227 * 1024 - 1024));
     attr_set = true;
   }
-  dim3 grid(prm.N / BN, (prm.M + BM - 1) / BM, batch);
-  tc_gemm_kernel<A_MN, B_MN, BN><<<grid, kThreadsTc, smem, s>>>(ta, tb, prm);
-  return launch_ok();
+  const bool prof = g_prof.on;
+  if (prof) {
+    cudaEventRecord(prof_event(), s);
+    g_prof.flops += flops;
+    g_prof.mma_flops += mma_flops;
+  }
+  const int grid = total < sm_count() ? total : sm_count();
+  tc_group_kernel<<<grid, kThreadsTc, smem, s>>>(prm);
+  const mw_status rc = launch_ok();
+  if (prof) cudaEventRecord(prof_event(), s);
+  return rc;
 }
 
 mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int M, int N, int K,
                   const TcEpilogue& epi, DeviceStatus* st, cudaStream_t s, int batch) {
-  if (M <= 0 || N <= 0 || K <= 0 || batch <= 0) return MW_OK;
-  if (batch > 65535) return MW_ERR_UNSUPPORTED;
-  if (N % 64 != 0) return MW_ERR_UNSUPPORTED;
-  if (A.planes < 1 || A.planes > 3 || B.planes < 1 || B.planes > 3) return MW_ERR_INVALID_ARG;
-  if (!A.mn_major && (K % 64 != 0)) return MW_ERR_UNSUPPORTED;
-  if (!B.mn_major && (K % 64 != 0)) return MW_ERR_UNSUPPORTED;
-  if (A.mn_major && (M % 64 != 0)) return MW_ERR_UNSUPPORTED;
-  TcParams prm{};
-  prm.M = M; prm.N = N; prm.K = K;
-  prm.pa = A.planes; prm.pb = B.planes;
-  const int terms = A.planes > B.planes ? A.planes : B.planes;
-  int np = 0;
-  // smallest cross products first
-  for (int sum = terms - 1; sum >= 0; --sum)
-    for (int i = 0; i <= sum; ++i) {
-      const int j = sum - i;
-      if (i < A.planes && j < B.planes) { prm.pair_a[np] = i; prm.pair_b[np] = j; ++np; }
-    }
-  prm.npairs = np;
-  prm.epi = epi;
-  prm.st = st;
-  prm.a_batch_planes = A.batch_planes ? A.batch_planes : A.planes;
-  prm.b_batch_planes = B.batch_planes ? B.batch_planes : B.planes;
-  const int a_total = batch > 1 ? (batch - 1) * prm.a_batch_planes + A.planes : A.planes;
-  const int b_total = batch > 1 ? (batch - 1) * prm.b_batch_planes + B.planes : B.planes;
-  const int tiles128 = (N % 128 == 0) ? (N / 128) * ((M + BM - 1) / BM) * batch : 0;
-  const bool bn128 = tiles128 >= 120;
-  const int BNsel = bn128 ? 128 : 64;
-  CUtensorMap ta, tb;
-  MW_TRY(get_map(cache, A, A.mn_major ? 64 : BM, a_total, &ta));
-  MW_TRY(get_map(cache, B, B.mn_major ? 64 : BNsel, b_total, &tb));
-  const bool prof = g_prof.on;
-  if (prof) {
-    cudaEventRecord(prof_event(), s);
-    g_prof.flops += 2.0 * M * N * K * batch;
-    g_prof.mma_flops += 2.0 * M * N * K * np * batch;
-  }
-  mw_status rc = MW_ERR_UNSUPPORTED;
-#define MW_TC_DISPATCH(AM, BMJ)                                              \
-  if (A.mn_major == AM && B.mn_major == BMJ) {                               \
-    rc = bn128 ? launch_tc<AM, BMJ, 128>(ta, tb, prm, batch, s)              \
-               : launch_tc<AM, BMJ, 64>(ta, tb, prm, batch, s);              \
-  }
-  MW_TC_DISPATCH(false, false)
-  MW_TC_DISPATCH(false, true)
-  MW_TC_DISPATCH(true, true)
-  MW_TC_DISPATCH(true, false)
-#undef MW_TC_DISPATCH
-  if (prof) cudaEventRecord(prof_event(), s);
-  return rc;
+  TcGemm g;
+  g.A = A; g.B = B; g.M = M; g.N = N; g.K = K; g.batch = batch; g.epi = epi;
+  return tc_gemm_group(cache, &g, 1, st, s);
 }
 
 // ---------------------------------------------------------------------------------------
 // fp32 -> bf16 term planes
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-split_planes_kernel(const float* __restrict__ in, int64_t n4, __nv_bfloat16* __restrict__ out,
-                    int planes, int64_t plane_stride) {
-  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n4; i += (int64_t)gridDim.x * 256) {
-    float4 v = reinterpret_cast<const float4*>(in)[i];
-    float r[4] = {v.x, v.y, v.z, v.w};
-    for (int p = 0; p < planes; ++p) {
-      __nv_bfloat16 b[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        b[j] = __float2bfloat16_rn(r[j]);
-        r[j] -= __bfloat162float(b[j]);
-      }
-      uint2 pk;
-      pk.x = (uint32_t)__bfloat16_as_ushort(b[0]) | ((uint32_t)__bfloat16_as_ushort(b[1]) << 16);
-      pk.y = (uint32_t)__bfloat16_as_ushort(b[2]) | ((uint32_t)__bfloat16_as_ushort(b[3]) << 16);
-      reinterpret_cast<uint2*>(out + (int64_t)p * plane_stride)[i] = pk;
-    }
-  }
-}
-
 __global__ void __launch_bounds__(256)
 split_planes_batched_kernel(const float* __restrict__ in, int64_t n4, int64_t in_stride,
                             __nv_bfloat16* __restrict__ out, int planes, int64_t plane_stride,
@@ -674,12 +958,7 @@ mw_status split_planes_batched(const float* in, int64_t n, int batch, int64_t in
 
 mw_status split_planes(const float* in, int64_t n, __nv_bfloat16* out, int planes,
                        int64_t plane_stride, cudaStream_t s) {
-  if (n == 0) return MW_OK;
-  if (n % 4 != 0 || plane_stride % 4 != 0) return MW_ERR_UNSUPPORTED;
-  int64_t blocks = (n / 4 + 255) / 256;
-  if (blocks > 148 * 8) blocks = 148 * 8;
-  split_planes_kernel<<<(int)blocks, 256, 0, s>>>(in, n / 4, out, planes, plane_stride);
-  return launch_ok();
+  return split_planes_batched(in, n, 1, 0, out, planes, plane_stride, 0, s);
 }
 
 }  // namespace mw

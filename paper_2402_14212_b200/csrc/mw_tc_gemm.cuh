@@ -1,12 +1,15 @@
 // Tensor-core product core for sm_100a: TMA-staged operand tiles, tcgen05.mma with the
-// accumulator in tensor memory, fused epilogues.  Internal interface.
+// accumulators in tensor memory, fused epilogues.  Internal interface.
 //
-// Every dense step of the Moonwalk path is one call of tc_gemm():
+// Every dense step of the Moonwalk path is one product:
 //   Phase I / recompute   z   = x W^T         (A = x K-major,  B = W K-major)
 //   Phase II              h'  = g_z W         (A = g_z K-major, B = W MN-major)
 //   dense vijp            g_z = h W^-1        (A = h K-major,  B = W^-1 MN-major)       Eq. "h_i"
 //   weight vjp            dW  = g_z^T x       (A = g_z MN-major, B = x MN-major)        Eq. "g_i"
 //   Newton-Schulz         R = I - W X, X' = X + X R
+// and one launch of the persistent kernel runs a GROUP of up to kTcMaxGroup independent products
+// (for the forward sweep: the recompute and the vijp of layer l+1 together with the weight vjp of
+// layer l), its CTAs walking the union of their output tiles.
 //
 // An operand is a stack of 1..3 bf16 "term planes" whose sum is the value (term t holds the
 // bf16 rounding of what the earlier terms left over).  A product of an a-term and a b-term
@@ -19,21 +22,24 @@
 
 namespace mw {
 
+constexpr int kTcMaxGroup = 4;
+constexpr size_t kTcSplitCounterBytes = 65536;
+
 struct TcOperand {
   const void* base = nullptr;   // bf16 planes, each [rows][cols] row-major
   int rows = 0, cols = 0;       // K-major: rows = M or N, cols = K.  MN-major: rows = K, cols = M or N
   int planes = 1;
   int64_t plane_stride = 0;     // elements between planes
   bool mn_major = false;
-  int batch_planes = 0;         // batched launch: planes between consecutive batch items (0 = planes)
+  int batch_planes = 0;         // batched product: planes between consecutive batch items (0 = planes)
 };
 
 enum TcEpiMode : int {
   TC_EPI_PLAIN = 0,    // v = alpha*acc (+ addend);  out_f32 and/or planes
   TC_EPI_RESID = 1,    // v = (row == col) - acc;    planes; sum of squares -> sumsq
   TC_EPI_FWD = 2,      // z = acc; sign word written (write_mask) or read; x = phi(z) -> planes (+ out_f32)
-  TC_EPI_BWD = 3,      // h = acc -> out_f32 (optional); g = h * phi'(mask) -> planes
-  TC_EPI_VIJP = 4,     // g = acc; leaky: h = g or g/slope -> planes2 ; g -> planes (for the weight vjp)
+  TC_EPI_BWD = 3,      // h = acc -> out_f32 (optional), ReLU fragments (optional); g = h * phi'(mask) -> planes
+  TC_EPI_VIJP = 4,     // g = acc; activation vijp: h -> planes2 (+ out_f32); g (zero at dead ReLU units) -> planes
 };
 
 struct TcEpilogue {
@@ -52,26 +58,55 @@ struct TcEpilogue {
   int act = MW_ACT_NONE;
   float slope = 1.f;
   double* sumsq = nullptr;             // TC_EPI_RESID: atomically accumulated ||v||_F^2
-  // batched launch (grid.z): element strides between consecutive batch items
+  // ReLU fragment stream (Section 5.1 applied to ReLU): row r keeps the cotangent at its dead
+  // units from vals[frag_off[r]], in increasing column order; frag_rank[r][c/64] = number of
+  // dead units of row r before column 64*(c/64).  TC_EPI_BWD writes the stream, TC_EPI_VIJP
+  // reads it back.
+  const uint32_t* frag_off = nullptr;
+  const uint32_t* frag_rank = nullptr;
+  float* frag_vals = nullptr;
+  // batched product (one tile range per batch item): element strides between consecutive items
   int64_t bs_f32 = 0;                  // addend and out_f32
   int64_t bs_planes = 0, bs_planes2 = 0;
   int64_t bs_mask = 0;                 // words
   int64_t bs_sumsq = 0;                // doubles
 };
 
-// Cache of encoded tensor maps (host side), owned by the caller of tc_gemm.
+// One product of a group.
+struct TcGemm {
+  TcOperand A, B;
+  int M = 0, N = 0, K = 0;
+  int batch = 1;
+  TcEpilogue epi;
+  // K split: the K range of every output tile is cut into `split_k` pieces computed by
+  // different CTAs; partial tiles meet in `split_scratch` (kTcSplitCounterBytes of arrival
+  // counters, zero before the first use and left zero by every launch, then split_k * tiles *
+  // 128 * bn floats; see tc_split_scratch_bytes) and the warp that arrives last adds the pieces
+  // in fixed order, so the result does not depend on scheduling.  0 / 1 = no split.
+  int split_k = 1;
+  void* split_scratch = nullptr;
+};
+
+// Cache of encoded tensor maps (host side), owned by the caller.
 struct TcMapCache;
 TcMapCache* tc_cache_create();
 void tc_cache_destroy(TcMapCache*);
 
-// D[M][N] = sum over term pairs of A_i B_j^T-style products; see TcOperand for layouts.
-// Requirements: N % 64 == 0; K % 64 == 0 for K-major operands; inner dimensions % 64 == 0;
-// all bases 16-byte aligned (256 recommended).
-// batch > 1 runs `batch` independent products of the same shape in one launch (grid.z): batch
-// item b reads planes b*batch_planes + t of each operand and offsets the epilogue pointers by
-// b times the bs_* strides.
+// Requirements per product: N % 64 == 0; K % 64 == 0 unless both operands are MN-major; M % 64 == 0
+// for an MN-major A; all bases 16-byte aligned.  batch > 1 runs `batch` independent products of the same shape: item b reads
+// planes b*batch_planes + t of each operand and offsets the epilogue pointers by b times the
+// bs_* strides.
+mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceStatus* st,
+                        cudaStream_t s);
+// single product
 mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int M, int N, int K,
                   const TcEpilogue& epi, DeviceStatus* st, cudaStream_t s, int batch = 1);
+
+// tile width the kernel will use for this product, and the scratch a K split of it needs
+int tc_tile_n(int a_planes, int b_planes, int M, int N, int batch);
+size_t tc_split_scratch_bytes(int a_planes, int b_planes, int M, int N, int batch, int split_k);
+// K split that gives every SM a work unit when the product alone has too few tiles (1 = none)
+int tc_auto_split(int a_planes, int b_planes, int M, int N, int K, int batch);
 
 // Per-launch timing of the product kernel (CUDA events around every launch while enabled).
 void tc_profile_begin();

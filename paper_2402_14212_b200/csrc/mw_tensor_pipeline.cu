@@ -1,14 +1,18 @@
 // Tensor-core pipelines of the three calls for dense nets (MW_F32 and MW_BF16_F32ACC).
 //
-// Every matrix product is one launch of the tcgen05 kernel (mw_tc_gemm.cu) with the step's
+// Every matrix product runs on the persistent tcgen05 kernel (mw_tc_gemm.cu) with the step's
 // elementwise work fused into its epilogue:
 //   Phase I    z = x W^T          -> sign words + x_l term planes                (Section 4.1)
-//   Phase II   h_{l-1} = g_z W    -> h (fp32, where a store needs it) + next g_z term planes
+//   Phase II   h_{l-1} = g_z W    -> cotangent checkpoint (fp32) and ReLU fragment stream where
+//                                    the layer below asks for them + next g_z term planes
 //   prep       W^-1 by Newton-Schulz, X <- X + X (I - W X), low precision first
-//   sweep      recompute (as Phase I, reading the stored sign words)             (Algorithm 1)
-//              g_z = h W^-1       -> leaky vijp fused: h_l term planes + g_z term planes (Eq. "h_i")
-//              dW = g_z^T x       -> fp32 gradient                               (Eq. "g_i")
-// ReLU layers take the stand-alone fragment kernels after a plain fp32 epilogue.
+//   sweep      one launch per layer (Algorithm 1) carrying three independent products:
+//              recompute x_{l+1} (as Phase I, reading the stored sign words),
+//              g_z = h_l W^-1 with the activation's vijp behind it: h_{l+1} term planes (leaky:
+//              divide by the slope; ReLU: dead units take their fragment back) + g_z term planes
+//              (Eq. "h_i"), and the weight vjp of the layer before, dW = g_z^T x (Eq. "g_i").
+// Products with too few output tiles for the machine are cut along K (deterministic meeting in
+// the workspace).
 #include "mw_tc_gemm.cuh"
 #include "mw_tensor.cuh"
 
@@ -323,6 +327,28 @@ mw_status input_planes(const Ctx& c, const void* x, const __nv_bfloat16** out) {
   return MW_OK;
 }
 
+// one product of a launch; `slot` picks the K-split meeting place (products of one launch must
+// use different slots)
+TcGemm product(const Ctx& c, const TcOperand& A, const TcOperand& B, int M, int N, int K,
+               const TcEpilogue& e, int slot) {
+  TcGemm g;
+  g.A = A; g.B = B; g.M = M; g.N = N; g.K = K; g.epi = e;
+  g.split_k = tc_auto_split(A.planes, B.planes, M, N, K, 1);
+  if (g.split_k > 1) g.split_scratch = c.at<char>(c.lay->split[slot]);
+  return g;
+}
+
+mw_status run(const Ctx& c, const TcGemm* g, int count) {
+  return tc_gemm_group(c.cache, g, count, c.st, c.s);
+}
+
+mw_status clear_split_counters(const Ctx& c) {
+  for (int i = 0; i < 3; ++i)
+    if (c.lay->split[i].bytes)
+      MW_CUDA_OK(cudaMemsetAsync(c.at<char>(c.lay->split[i]), 0, kTcSplitCounterBytes, c.s));
+  return MW_OK;
+}
+
 // forward pass shared by Phase I and backprop's forward; y (fp32 network output) lands in lay.z
 mw_status forward_pass(const Ctx& c, const void* const* params, const void* x, bool store_acts) {
   const Layout& lay = *c.lay;
@@ -336,7 +362,7 @@ mw_status forward_pass(const Ctx& c, const void* const* params, const void* x, b
     // resident + Moonwalk: the planes were made by the prep at the top of mw_input_cotangent
     MW_TRY(weight_planes(c, l, params[l], !(resident && !store_acts), &Wp));
     __nv_bfloat16* xout = (store_acts && l + 1 < L) ? c.at<__nv_bfloat16>(lay.stored_act[l + 1])
-                                                   : c.at<__nv_bfloat16>(lay.xp[(l + 1) & 1]);
+                                                   : c.at<__nv_bfloat16>(lay.xp[(l + 1) % 3]);
     TcEpilogue e;
     e.mode = TC_EPI_FWD;
     e.mask = c.at<uint32_t>(lay.mask[l]);
@@ -348,11 +374,20 @@ mw_status forward_pass(const Ctx& c, const void* const* params, const void* x, b
     } else {
       e.out_f32 = c.at<float>(lay.z);
     }
-    MW_TRY(tc_gemm(c.cache, operand(xin, c.B, d, c.pr.px, false), operand(Wp, d, d, c.pr.pw, false),
-                   c.B, d, d, e, c.st, c.s));
+    TcGemm g = product(c, operand(xin, c.B, d, c.pr.px, false), operand(Wp, d, d, c.pr.pw, false),
+                       c.B, d, d, e, 0);
+    MW_TRY(run(c, &g, 1));
     xin = xout;
   }
   return MW_OK;
+}
+
+// index of layer l's fragment stream from its sign words
+mw_status relu_index(const Ctx& c, int l) {
+  const Layout& lay = *c.lay;
+  return fragment_index(c.at<uint32_t>(lay.mask[l]), c.B, c.dim, c.at<uint32_t>(lay.frag_cnt[l]),
+                        c.at<uint32_t>(lay.frag_off[l]), c.at<uint32_t>(lay.frag_rank[l]),
+                        c.at<uint32_t>(lay.frag_total) + l, c.s);
 }
 
 // top of the reverse pass: loss, h_L (fp32 in cot[0]) and g_z of the last layer as term planes
@@ -365,9 +400,7 @@ mw_status loss_and_top(const Ctx& c, const void* target, double* loss_out, bool 
                                c.at<double>(lay.partials), loss_out, c.s));
   const uint32_t* words = c.at<uint32_t>(lay.mask[L - 1]);
   if (fragments && ld.act == MW_ACT_RELU) {
-    MW_TRY(fragment_offsets(words, c.B, d, c.at<uint32_t>(lay.frag_cnt[L - 1]),
-                            c.at<uint32_t>(lay.frag_off[L - 1]),
-                            c.at<uint32_t>(lay.frag_total) + (L - 1), nullptr, 0, c.s));
+    MW_TRY(relu_index(c, L - 1));
     MW_TRY(fragment_compact<float>(h, words, c.B, d, c.at<uint32_t>(lay.frag_off[L - 1]),
                                    c.at<float>(lay.frag_vals[L - 1]), c.s));
   }
@@ -411,12 +444,27 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
   const size_t d = (size_t)n->layers[0].n_in;
   const size_t bn = (size_t)n->B * d, nn = d * d;
   const bool resident = n->opts.resident_inverse != 0;
-  lay.z = b.take(4 * bn);                                   // fp32 network output / g_z scratch
-  for (int i = 0; i < 2; ++i) lay.cot[i] = b.take(4 * bn);  // fp32 cotangent scratch
-  for (int i = 0; i < 2; ++i) lay.xp[i] = b.take(2 * (size_t)pr.px * bn);
+  lay.z = b.take(4 * bn);                                   // fp32 network output
+  for (int i = 0; i < 2; ++i) lay.cot[i] = b.take(4 * bn);  // fp32 cotangent scratch (loss top)
+  for (int i = 0; i < 3; ++i) lay.xp[i] = b.take(2 * (size_t)pr.px * bn);
   const int hpl = pr.ph > pr.pg2 ? pr.ph : pr.pg2;
   for (int i = 0; i < 2; ++i) lay.hp[i] = b.take(2 * (size_t)hpl * bn);
-  lay.gzp = b.take(2 * (size_t)(pr.pgw > pr.pg2 ? pr.pgw : pr.pg2) * bn);
+  for (int i = 0; i < 2; ++i) lay.gzp[i] = b.take(2 * (size_t)(pr.pgw > pr.pg2 ? pr.pgw : pr.pg2) * bn);
+  // K-split meeting places: slot 0 recompute / Phase I / Phase II, slot 1 vijp, slot 2 weight vjp
+  {
+    const int B = n->B, dd = (int)d;
+    auto need = [&](int pa, int pb, int M, int N, int K) {
+      return tc_split_scratch_bytes(pa, pb, M, N, 1, tc_auto_split(pa, pb, M, N, K, 1));
+    };
+    size_t s0 = need(pr.px, pr.pw, B, dd, dd);
+    const size_t s0b = need(pr.pg2, pr.pw, B, dd, dd);
+    if (s0b > s0) s0 = s0b;
+    const size_t s1 = need(pr.ph, pr.ph, B, dd, dd);
+    const size_t s2 = need(pr.pgw, pr.px, dd, dd, B);
+    if (s0) lay.split[0] = b.take(s0);
+    if (s1 && !backprop) lay.split[1] = b.take(s1);
+    if (s2) lay.split[2] = b.take(s2);
+  }
   if (n->opts.prec == MW_F32) {
     if (resident) {
       for (int l = 0; l < L; ++l) lay.w_planes[l] = b.take(2 * 3 * nn);
@@ -457,6 +505,7 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
   Ctx c = make_ctx(n, lay, ws, s);
   const int L = n->L, d = c.dim;
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
+  MW_TRY(clear_split_counters(c));
   const bool resident = n->opts.resident_inverse != 0;
   if (resident) {
     const int G = ns_group(n);
@@ -471,31 +520,28 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
     MW_TRY(weight_planes(c, l, params[l], !resident, &Wp));
     TcEpilogue e;
     e.mode = TC_EPI_BWD;
-    float* hf = nullptr;
     if (l == 0) {
-      hf = (float*)g0;
+      e.out_f32 = (float*)g0;
     } else {
       const mw_layer_desc& below = n->layers[l - 1];
-      if (is_reseed(n, l)) hf = c.at<float>(lay.reseed[l]);
-      else if (below.act == MW_ACT_RELU) hf = c.at<float>(lay.cot[0]);
+      if (is_reseed(n, l)) e.out_f32 = c.at<float>(lay.reseed[l]);
       e.act = below.act;
       e.slope = (float)below.slope;
       e.mask = c.at<uint32_t>(lay.mask[l - 1]);
       e.planes = c.at<__nv_bfloat16>(lay.hp[cur ^ 1]);
       e.n_planes = c.pr.pg2;
       e.plane_stride = c.bn;
+      if (below.act == MW_ACT_RELU) {
+        // the layer below is not submersive: keep the cotangent at its dead units (Section 5.1)
+        MW_TRY(relu_index(c, l - 1));
+        e.frag_off = c.at<uint32_t>(lay.frag_off[l - 1]);
+        e.frag_rank = c.at<uint32_t>(lay.frag_rank[l - 1]);
+        e.frag_vals = c.at<float>(lay.frag_vals[l - 1]);
+      }
     }
-    e.out_f32 = hf;
-    MW_TRY(tc_gemm(c.cache, operand(c.at<__nv_bfloat16>(lay.hp[cur]), c.B, d, c.pr.pg2, false),
-                   operand(Wp, d, d, c.pr.pw, true), c.B, d, d, e, c.st, s));
-    if (l > 0 && n->layers[l - 1].act == MW_ACT_RELU) {
-      const uint32_t* words = c.at<uint32_t>(lay.mask[l - 1]);
-      MW_TRY(fragment_offsets(words, c.B, d, c.at<uint32_t>(lay.frag_cnt[l - 1]),
-                              c.at<uint32_t>(lay.frag_off[l - 1]),
-                              c.at<uint32_t>(lay.frag_total) + (l - 1), nullptr, 0, s));
-      MW_TRY(fragment_compact<float>(hf, words, c.B, d, c.at<uint32_t>(lay.frag_off[l - 1]),
-                                     c.at<float>(lay.frag_vals[l - 1]), s));
-    }
+    TcGemm g = product(c, operand(c.at<__nv_bfloat16>(lay.hp[cur]), c.B, d, c.pr.pg2, false),
+                       operand(Wp, d, d, c.pr.pw, true), c.B, d, d, e, 0);
+    MW_TRY(run(c, &g, 1));
     cur ^= 1;
   }
   return MW_OK;
@@ -507,69 +553,74 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
   Ctx c = make_ctx(n, lay, ws, s);
   const int L = n->L, d = c.dim;
   const bool resident = n->opts.resident_inverse != 0;
-  const __nv_bfloat16* xin = nullptr;
-  MW_TRY(input_planes(c, x, &xin));
+  const __nv_bfloat16* x0p = nullptr;
+  MW_TRY(input_planes(c, x, &x0p));
   MW_TRY(split_planes((const float*)g0, c.bn, c.at<__nv_bfloat16>(lay.hp[0]), c.pr.ph, c.bn, s));
-  for (int l = 0; l < L; ++l) {
-    const mw_layer_desc& ld = n->layers[l];
-    const uint32_t* words = c.at<uint32_t>(lay.mask[l]);
-    const __nv_bfloat16* Wp = nullptr;
-    if (!resident) MW_TRY(newton_schulz_group(c, l, 1, params));
-    MW_TRY(weight_planes(c, l, params[l], false, &Wp));
-    const __nv_bfloat16* hin = c.at<__nv_bfloat16>(lay.hp[l & 1]);
-    __nv_bfloat16* hout = c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]);
-    __nv_bfloat16* xout = c.at<__nv_bfloat16>(lay.xp[(l + 1) & 1]);
-    __nv_bfloat16* gzp = c.at<__nv_bfloat16>(lay.gzp);
-    const bool more = l + 1 < L;
-    const bool reseed_next = more && is_reseed(n, l + 1);
-    // recompute x_{l+1} (not needed after the last layer)
-    if (more) {
-      TcEpilogue e;
-      e.mode = TC_EPI_FWD;
-      e.mask = const_cast<uint32_t*>(words);
-      e.write_mask = 0;
-      e.act = ld.act;
-      e.slope = (float)ld.slope;
-      e.planes = xout; e.n_planes = c.pr.px; e.plane_stride = c.bn;
-      MW_TRY(tc_gemm(c.cache, operand(xin, c.B, d, c.pr.px, false), operand(Wp, d, d, c.pr.pw, false),
-                     c.B, d, d, e, c.st, s));
+  auto xbuf = [&](int l) -> const __nv_bfloat16* {          // term planes of x_l
+    return l == 0 ? x0p : c.at<__nv_bfloat16>(lay.xp[l % 3]);
+  };
+  // launch l: recompute x_{l+1} and vijp of layer l, with the weight vjp of layer l-1
+  for (int l = 0; l <= L; ++l) {
+    TcGemm g[3];
+    int cnt = 0;
+    if (l < L) {
+      const mw_layer_desc& ld = n->layers[l];
+      uint32_t* words = c.at<uint32_t>(lay.mask[l]);
+      const bool more = l + 1 < L;
+      const bool reseed_next = more && is_reseed(n, l + 1);
+      if (!resident) MW_TRY(newton_schulz_group(c, l, 1, params));
+      if (reseed_next)   // the recursion restarts from the stored cotangent h_{l+1}
+        MW_TRY(split_planes(c.at<float>(lay.reseed[l + 1]), c.bn,
+                            c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]), c.pr.ph, c.bn, s));
+      if (more) {
+        const __nv_bfloat16* Wp = nullptr;
+        MW_TRY(weight_planes(c, l, params[l], false, &Wp));
+        TcEpilogue e;
+        e.mode = TC_EPI_FWD;
+        e.mask = words;
+        e.write_mask = 0;
+        e.act = ld.act;
+        e.slope = (float)ld.slope;
+        e.planes = c.at<__nv_bfloat16>(lay.xp[(l + 1) % 3]);
+        e.n_planes = c.pr.px;
+        e.plane_stride = c.bn;
+        g[cnt++] = product(c, operand(xbuf(l), c.B, d, c.pr.px, false),
+                           operand(Wp, d, d, c.pr.pw, false), c.B, d, d, e, 0);
+      }
+      if (dW[l] || (more && !reseed_next)) {
+        TcEpilogue e;
+        e.mode = TC_EPI_VIJP;
+        e.act = ld.act;
+        e.slope = (float)ld.slope;
+        e.mask = words;
+        if (ld.act == MW_ACT_RELU) {
+          e.frag_off = c.at<uint32_t>(lay.frag_off[l]);
+          e.frag_rank = c.at<uint32_t>(lay.frag_rank[l]);
+          e.frag_vals = c.at<float>(lay.frag_vals[l]);
+        }
+        if (more && !reseed_next) {
+          e.planes2 = c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]);
+          e.n_planes2 = c.pr.ph;
+          e.plane_stride2 = c.bn;
+        }
+        if (dW[l]) {
+          e.planes = c.at<__nv_bfloat16>(lay.gzp[l & 1]);
+          e.n_planes = c.pr.pgw;
+          e.plane_stride = c.bn;
+        }
+        g[cnt++] = product(c, operand(c.at<__nv_bfloat16>(lay.hp[l & 1]), c.B, d, c.pr.ph, false),
+                           operand(c.at<__nv_bfloat16>(lay.inv[l]), d, d, c.pr.ph, true), c.B, d, d,
+                           e, 1);
+      }
     }
-    // dense vijp g_z = h W^-1, with the activation's vijp behind it
-    const TcOperand hop = operand(hin, c.B, d, c.pr.ph, false);
-    const TcOperand iop = operand(c.at<__nv_bfloat16>(lay.inv[l]), d, d, c.pr.ph, true);
-    if (ld.act == MW_ACT_RELU) {
-      float* gzf = c.at<float>(lay.z);
-      float* hf = c.at<float>(lay.cot[1]);
+    if (l >= 1 && dW[l - 1]) {
       TcEpilogue e;
       e.mode = TC_EPI_PLAIN;
-      e.out_f32 = gzf;
-      MW_TRY(tc_gemm(c.cache, hop, iop, c.B, d, d, e, c.st, s));
-      MW_TRY(activation_vijp<float>(gzf, words, c.B, d, MW_ACT_RELU, 0.0,
-                                    c.at<uint32_t>(lay.frag_off[l]), c.at<float>(lay.frag_vals[l]),
-                                    hf, gzf, s));
-      if (more && !reseed_next) MW_TRY(split_planes(hf, c.bn, hout, c.pr.ph, c.bn, s));
-      if (dW[l]) MW_TRY(split_planes(gzf, c.bn, gzp, c.pr.pgw, c.bn, s));
-    } else {
-      TcEpilogue e;
-      e.mode = TC_EPI_VIJP;
-      e.act = ld.act;
-      e.slope = (float)ld.slope;
-      e.mask = const_cast<uint32_t*>(words);
-      if (more && !reseed_next) { e.planes2 = hout; e.n_planes2 = c.pr.ph; e.plane_stride2 = c.bn; }
-      if (dW[l]) { e.planes = gzp; e.n_planes = c.pr.pgw; e.plane_stride = c.bn; }
-      MW_TRY(tc_gemm(c.cache, hop, iop, c.B, d, d, e, c.st, s));
+      e.out_f32 = (float*)dW[l - 1];
+      g[cnt++] = product(c, operand(c.at<__nv_bfloat16>(lay.gzp[(l - 1) & 1]), c.B, d, c.pr.pgw, true),
+                         operand(xbuf(l - 1), c.B, d, c.pr.px, true), d, d, c.B, e, 2);
     }
-    if (reseed_next)
-      MW_TRY(split_planes(c.at<float>(lay.reseed[l + 1]), c.bn, hout, c.pr.ph, c.bn, s));
-    // weight vjp dW = g_z^T x
-    if (dW[l]) {
-      TcEpilogue e;
-      e.mode = TC_EPI_PLAIN;
-      e.out_f32 = (float*)dW[l];
-      MW_TRY(tc_gemm(c.cache, operand(gzp, c.B, d, c.pr.pgw, true), operand(xin, c.B, d, c.pr.px, true),
-                     d, d, c.B, e, c.st, s));
-    }
-    xin = xout;
+    if (cnt) MW_TRY(run(c, g, cnt));
   }
   return MW_OK;
 }
@@ -580,26 +631,23 @@ mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, c
   Ctx c = make_ctx(n, lay, ws, s);
   const int L = n->L, d = c.dim;
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
+  MW_TRY(clear_split_counters(c));
   MW_TRY(forward_pass(c, params, x, true));
   MW_TRY(loss_and_top(c, target, loss_out, false));
   const __nv_bfloat16* x0p = nullptr;
   if (n->opts.prec == MW_F32) x0p = c.at<__nv_bfloat16>(lay.xp[0]);   // split by forward_pass
   else x0p = (const __nv_bfloat16*)x;
-  const bool resident = n->opts.resident_inverse != 0;
   int cur = 0;
+  // one launch per layer: both vjps of layer l read the same g_z
   for (int l = L - 1; l >= 0; --l) {
     const __nv_bfloat16* gz = c.at<__nv_bfloat16>(lay.hp[cur]);
     const __nv_bfloat16* xl = l == 0 ? x0p : c.at<__nv_bfloat16>(lay.stored_act[l]);
-    if (dW[l]) {
-      TcEpilogue e;
-      e.mode = TC_EPI_PLAIN;
-      e.out_f32 = (float*)dW[l];
-      MW_TRY(tc_gemm(c.cache, operand(gz, c.B, d, c.pr.pgw, true), operand(xl, c.B, d, c.pr.px, true),
-                     d, d, c.B, e, c.st, s));
-    }
+    TcGemm g[2];
+    int cnt = 0;
     if (l > 0) {
       const __nv_bfloat16* Wp = nullptr;
-      MW_TRY(weight_planes(c, l, params[l], !resident, &Wp));
+      // resident: the planes made by forward_pass are still there (MW_F32)
+      MW_TRY(weight_planes(c, l, params[l], n->opts.resident_inverse == 0, &Wp));
       const mw_layer_desc& below = n->layers[l - 1];
       TcEpilogue e;
       e.mode = TC_EPI_BWD;
@@ -609,10 +657,18 @@ mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, c
       e.planes = c.at<__nv_bfloat16>(lay.hp[cur ^ 1]);
       e.n_planes = c.pr.pg2;
       e.plane_stride = c.bn;
-      MW_TRY(tc_gemm(c.cache, operand(gz, c.B, d, c.pr.pg2, false), operand(Wp, d, d, c.pr.pw, true),
-                     c.B, d, d, e, c.st, s));
-      cur ^= 1;
+      g[cnt++] = product(c, operand(gz, c.B, d, c.pr.pg2, false), operand(Wp, d, d, c.pr.pw, true),
+                         c.B, d, d, e, 0);
     }
+    if (dW[l]) {
+      TcEpilogue e;
+      e.mode = TC_EPI_PLAIN;
+      e.out_f32 = (float*)dW[l];
+      g[cnt++] = product(c, operand(gz, c.B, d, c.pr.pgw, true), operand(xl, c.B, d, c.pr.px, true),
+                         d, d, c.B, e, 2);
+    }
+    if (cnt) MW_TRY(run(c, g, cnt));
+    cur ^= 1;
   }
   return MW_OK;
 }
