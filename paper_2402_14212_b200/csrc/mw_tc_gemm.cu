@@ -385,6 +385,12 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (warp == 2 && lane < 2 * p.nprob) {
+    // start fetching the tensor maps before the first copy needs them
+    const TcProblem& P = p.prob[lane >> 1];
+    const CUtensorMap* tm = (lane & 1) ? &P.tmB : &P.tmA;
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
+  }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(&tmem_slot)),
@@ -527,16 +533,10 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       }
       double sumsq_local = 0.0;
       const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + set * (uint32_t)kSetCols;
-      const bool split = P.split > 1;
-      float* part = nullptr;
-      if (split)
-        part = P.split_partials + ((int64_t)w.tl * P.split + w.ks) * (int64_t)(BM * bn) +
-               (int64_t)(quarter * 32 + lane) * bn;
-#pragma unroll 1
-      for (int c = 0; c < bn; c += 32) {
-        if (w.n0 + c >= N) break;
+      const int nchunk = bn >> 5;
+      // sum of the column blocks of 32 accumulator columns starting at c
+      auto load_chunk = [&](int c, float (&v)[32]) {
         uint32_t r0[32];
-        float v[32];
         tmem_ld32_issue(t0 + (uint32_t)c, r0);
         tmem_ld_wait();
 #pragma unroll
@@ -547,46 +547,74 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] += __uint_as_float(r0[i]);
         }
-        if (split) store_f32x32(v, part + c);
-        else if (row < P.M) epilogue_chunk(epi, N, row, w.n0 + c, v, sumsq_local);
-      }
-      // this warp has read its part of the accumulator set: hand it back to the MMA issuer
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&acc_empty[set]));
-      ++j;
-      if (split) {
-        // the warp that finds the other K pieces of its 32 rows complete adds all pieces in
-        // fixed order and applies the fused step
+      };
+      bool fused_step = true;
+      if (P.split > 1) {
+        // K split: leave this piece of the tile in the meeting place, element (row, c + i) of
+        // piece s at ((s * nchunk + c / 32) * 32 + i) * 128 + row so that a warp writes whole lines
+        float* mine = P.split_partials + ((int64_t)w.tl * P.split + w.ks) * (int64_t)(BM * bn) +
+                      quarter * 32 + lane;
+#pragma unroll 1
+        for (int c = 0; c < bn; c += 32) {
+          if (w.n0 + c >= N) break;
+          float v[32];
+          load_chunk(c, v);
+          float* dst = mine + (int64_t)c * BM;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) dst[i * BM] = v[i];
+        }
         __threadfence();
         __syncwarp();
         unsigned int* cnt = P.split_counters + (int64_t)w.tl * 4 + quarter;
         unsigned int old = 0;
         if (lane == 0) old = atomicAdd(cnt, 1u);
         old = __shfl_sync(0xffffffffu, old, 0);
-        if (old == (unsigned)P.split - 1u) {
+        // the warp that finds the other pieces of its 32 rows complete adds all pieces in fixed
+        // order (its own straight from tensor memory) and applies the fused step
+        fused_step = old == (unsigned)P.split - 1u;
+        if (fused_step) {
           __threadfence();
-          const float* p0 = P.split_partials + (int64_t)w.tl * P.split * (int64_t)(BM * bn) +
-                            (int64_t)(quarter * 32 + lane) * bn;
-#pragma unroll 1
-          for (int c = 0; c < bn; c += 32) {
-            if (w.n0 + c >= N) break;
-            float v[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = 0.f;
-            for (int s = 0; s < P.split; ++s) {
-              const float4* q4 = reinterpret_cast<const float4*>(p0 + (int64_t)s * (BM * bn) + c);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const float4 t = __ldcg(q4 + i);
-                v[4 * i] += t.x; v[4 * i + 1] += t.y; v[4 * i + 2] += t.z; v[4 * i + 3] += t.w;
-              }
-            }
-            if (row < P.M) epilogue_chunk(epi, N, row, w.n0 + c, v, sumsq_local);
-          }
           if (lane == 0) *cnt = 0u;     // ready for the next launch
         }
       }
+      if (fused_step) {
+        const float* others = P.split > 1 ? P.split_partials + (int64_t)w.tl * P.split * (int64_t)(BM * bn) +
+                                                quarter * 32 + lane
+                                          : nullptr;
+#pragma unroll 1
+        for (int c = 0; c < bn; c += 32) {
+          if (w.n0 + c >= N) break;
+          float v[32];
+          if (P.split > 1) {
+            float own[32];
+            load_chunk(c, own);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = 0.f;
+            for (int sp = 0; sp < P.split; ++sp) {
+              if (sp == w.ks) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] += own[i];
+              } else {
+                const float* src = others + (int64_t)sp * (BM * bn) + (int64_t)c * BM;
+                float t[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) t[i] = __ldcg(src + i * BM);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] += t[i];
+              }
+            }
+          } else {
+            load_chunk(c, v);
+          }
+          if (row < P.M) epilogue_chunk(epi, N, row, w.n0 + c, v, sumsq_local);
+        }
+      }
+      (void)nchunk;
+      // this warp has read its part of the accumulator set: hand it back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&acc_empty[set]));
+      ++j;
       if (epi.mode == TC_EPI_RESID && epi.sumsq) {
         for (int o = 16; o; o >>= 1) sumsq_local += __shfl_xor_sync(0xffffffffu, sumsq_local, o);
         if (lane == 0 && sumsq_local != 0.0) atomicAdd(epi.sumsq, sumsq_local);
@@ -661,12 +689,11 @@ size_t tc_split_scratch_bytes(int a_planes, int b_planes, int M, int N, int batc
 int tc_auto_split(int a_planes, int b_planes, int M, int N, int K, int batch) {
   const int bn = pick_bn(a_planes, b_planes, M, N, batch);
   const int64_t units = (int64_t)((M + BM - 1) / BM) * ((N + bn - 1) / bn) * batch;
-  const int sms = sm_count();
-  if (units * 5 >= (int64_t)sms * 3) return 1;
-  int s = (int)((sms + units - 1) / units);
+  // as many pieces as keep every piece on an SM of its own, each at least four K blocks deep
+  int s = (int)(sm_count() / units);
   const int num_kb = (K + BK - 1) / BK;
-  if (s > num_kb / 2) s = num_kb / 2;
-  if (s > 8) s = 8;
+  if (s > num_kb / 4) s = num_kb / 4;
+  if (s > 4) s = 4;
   return s < 1 ? 1 : s;
 }
 
