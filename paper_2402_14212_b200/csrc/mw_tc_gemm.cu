@@ -327,6 +327,32 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int r
   }
 }
 
+// The instructions of one 64-deep K block, as straight-line code: the issuing lane runs alone on
+// its scheduler, so every branch and every dependent integer instruction in this loop costs
+// tens of cycles that the tensor pipe would otherwise spend on the next product.
+template <int NOPS>
+__device__ __forceinline__ void issue_k_block(const uint32_t (&oa)[kMaxOps], const uint32_t (&ob)[kMaxOps],
+                                              const uint32_t (&oi)[kMaxOps], const uint32_t (&od)[kMaxOps],
+                                              const uint32_t (&orot)[kMaxOps], const uint32_t (&ofk)[kMaxOps],
+                                              uint32_t sb16, uint32_t a_kadv, uint32_t b_kadv,
+                                              uint32_t kbl) {
+  uint32_t d[NOPS], a[NOPS], b[NOPS], first[NOPS];
+#pragma unroll
+  for (int o = 0; o < NOPS; ++o) {
+    d[o] = od[o] + ((kbl & 1u) ? orot[o] : 0u);
+    a[o] = oa[o] + sb16;
+    b[o] = ob[o] + sb16;
+    first[o] = kbl < ofk[o] ? 0u : 1u;
+  }
+#pragma unroll
+  for (int k4 = 0; k4 < BK / 16; ++k4) {
+#pragma unroll
+    for (int o = 0; o < NOPS; ++o)
+      umma_bf16(d[o], a[o] + (uint32_t)k4 * a_kadv, b[o] + (uint32_t)k4 * b_kadv, oi[o],
+                k4 == 0 ? first[o] : 1u);
+  }
+}
+
 // unit u of the sorted list -> product, tile, batch item and K range
 __device__ __forceinline__ void decode_unit(const TcGroupParams& p, int u, Unit& w) {
   int q = 0;
@@ -483,17 +509,13 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           if (!mbar_wait(smem_u32(&full_bar[stage]), phase, p.st, 3u, abortp)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sb16 = (tiles + stage * p.stage_bytes) >> 4;
-          const uint32_t odd = (uint32_t)kbl & 1u;
-#pragma unroll
-          for (int k4 = 0; k4 < BK / 16; ++k4) {
-#pragma unroll
-            for (int o = 0; o < kMaxOps; ++o) {
-              if (o < nops) {
-                const uint32_t acc = (k4 == 0 && (uint32_t)kbl < ofk[o]) ? 0u : 1u;
-                umma_bf16(od[o] + (odd ? orot[o] : 0u), oa[o] + sb16 + (uint32_t)k4 * a_kadv,
-                          ob[o] + sb16 + (uint32_t)k4 * b_kadv, oi[o], acc);
-              }
-            }
+          switch (nops) {
+            case 1: issue_k_block<1>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            case 2: issue_k_block<2>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            case 3: issue_k_block<3>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            case 4: issue_k_block<4>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            case 5: issue_k_block<5>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            default: issue_k_block<6>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
           }
           umma_commit(smem_u32(&empty_bar[stage]));  // frees the stage once these products retire
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
