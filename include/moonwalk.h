@@ -181,6 +181,28 @@ mw_status mw_gemm_split_bf16(const float* A, int32_t a_mn, const float* B, int32
                              int32_t M, int32_t N, int32_t K, int32_t terms, void* scratch,
                              size_t scratch_bytes, void* stream);
 
+/* The same product as mw_gemm_split_bf16 for callers that have no scratch buffer to lend and
+ * cannot allocate one when they call: code that runs inside a host framework whose memory pool
+ * owns the whole device (a direct cudaMalloc there fails or stalls every stream), and services
+ * with a fixed memory plan that forbid allocation after start-up.  (The paper has no counterpart;
+ * this is a convenience of the library.)
+ *   A, B, D, M, N, K, terms, a_mn, b_mn: exactly as in mw_gemm_split_bf16; the caller still owns
+ *   the inputs and the output.
+ * The scratch (status block + bf16 term planes of A and B) lives in an array built into the
+ * library, MW_GEMM_STATIC_SCRATCH_BYTES per GPU, held by every GPU that loads the library until
+ * the process exits.  Sizes that need more, 256 + 2*terms*(M*K + N*K) bytes (+ padding), are
+ * rejected with MW_ERR_WORKSPACE before any GPU work.  The call itself allocates nothing on host
+ * or device and frees nothing.
+ * The first call on a device looks up the array's device address (with that device current); make
+ * that first call before any stream capture begins.
+ * All calls on one GPU share the array, which keeps the previous call's contents; the entry point
+ * clears the part that must start at zero.  Two calls whose GPU work overlaps (different streams,
+ * or threads) race on it: serialise them.  Synchronises `stream` before returning. */
+#define MW_GEMM_STATIC_SCRATCH_BYTES (16u << 20)
+mw_status mw_gemm_split_bf16_static(const float* A, int32_t a_mn, const float* B, int32_t b_mn,
+                                    float* D, int32_t M, int32_t N, int32_t K, int32_t terms,
+                                    void* stream);
+
 /* ---- whole step from host buffers, and measurement hooks --------------------------------- */
 
 /* One Moonwalk gradient step (Algorithm 1 with Phases I-II in front) whose per-step inputs

@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
         L.mw_relu_fragment_compact.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp, vp, sz, vp]
         L.mw_activation_vijp.argtypes = [vp, vp, i64, i32, i32, C.c_float, vp, vp, vp, vp, vp]
         L.mw_gemm_split_bf16.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, vp, sz, vp]
+        L.mw_gemm_split_bf16_static.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, vp]
         L.mw_gradient_step_host.argtypes = [vp, C.POINTER(vp), vp, sz, vp, sz, vp, vp, vp,
                                             C.POINTER(vp), vp, vp, vp, sz, vp]
         L.mw_launch_count.argtypes = []
@@ -300,6 +301,24 @@ def gemm_split_bf16(A, B, a_mn: bool, b_mn: bool, terms: int, stream=None):
     _check(lib().mw_gemm_split_bf16(_ptr(A), int(a_mn), _ptr(B), int(b_mn), _ptr(D), M, N, K,
                                     int(terms), _ptr(scratch), scratch.numel(),
                                     _stream_handle(stream)), "mw_gemm_split_bf16")
+    return D
+
+
+GEMM_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def gemm_split_bf16_static(A, B, a_mn: bool, b_mn: bool, terms: int, stream=None):
+    """mw_gemm_split_bf16_static: the same product with the library's built-in scratch, for callers
+    that cannot allocate a scratch buffer.  Only the output tensor is created here (by torch, as
+    for every other call of this binding); the C entry point itself allocates nothing."""
+    import torch
+    M = A.shape[1] if a_mn else A.shape[0]
+    K = A.shape[0] if a_mn else A.shape[1]
+    N = B.shape[1] if b_mn else B.shape[0]
+    D = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    _check(lib().mw_gemm_split_bf16_static(_ptr(A), int(a_mn), _ptr(B), int(b_mn), _ptr(D), M, N, K,
+                                           int(terms), _stream_handle(stream)),
+           "mw_gemm_split_bf16_static")
     return D
 
 

@@ -1047,3 +1047,63 @@ extern "C" mw_status mw_gemm_split_bf16(const float* A, int32_t a_mn, const floa
   MW_CUDA_OK(cudaStreamSynchronize(s));
   return host.code == 0 ? MW_OK : (mw_status)host.code;
 }
+
+// ---------------------------------------------------------------------------------------
+// The same product for callers that cannot hand over scratch memory
+// ---------------------------------------------------------------------------------------
+namespace {
+
+// Scratch of mw_gemm_split_bf16_static: the status block and the bf16 term planes of both
+// operands.  One copy per GPU that loads the library, held until the process exits.
+constexpr size_t kStaticScratchBytes = MW_GEMM_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kStaticMaxDevices = 64;
+void* g_static_scratch_ptr[kStaticMaxDevices] = {};   // device address of the array, per device
+
+}  // namespace
+
+extern "C" mw_status mw_gemm_split_bf16_static(const float* A, int32_t a_mn, const float* B,
+                                               int32_t b_mn, float* D, int32_t M, int32_t N,
+                                               int32_t K, int32_t terms, void* stream) {
+  using namespace mw;
+  if (!A || !B || !D) return MW_ERR_INVALID_ARG;
+  if (terms < 1 || terms > 3 || M < 1 || N < 1 || K < 1) return MW_ERR_INVALID_ARG;
+  if (M % 64 || N % 64 || K % 64) return MW_ERR_UNSUPPORTED;
+  const size_t ea = (size_t)M * K, eb = (size_t)N * K;
+  const size_t need = 256 + 2 * (align_up((size_t)terms * ea, 128) + (size_t)terms * eb);
+  if (need > kStaticScratchBytes) return MW_ERR_WORKSPACE;   // beyond the built-in scratch
+  int dev = -1;
+  MW_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kStaticMaxDevices) return MW_ERR_UNSUPPORTED;
+  if (!g_static_scratch_ptr[dev]) {
+    // In host code the array's name stands for the symbol, not for device memory: ask the
+    // runtime for the address on the current device, once.
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return MW_ERR_CUDA;
+    g_static_scratch_ptr[dev] = p;
+  }
+  char* scratch = static_cast<char*>(g_static_scratch_ptr[dev]);
+  cudaStream_t s = (cudaStream_t)stream;
+  // the array keeps whatever the last call left: the status block has to start at zero, the
+  // planes are overwritten in full before they are read
+  DeviceStatus* st = reinterpret_cast<DeviceStatus*>(scratch);
+  MW_CUDA_OK(cudaMemsetAsync(st, 0, 256, s));
+  __nv_bfloat16* pa = reinterpret_cast<__nv_bfloat16*>(scratch + 256);
+  __nv_bfloat16* pb = pa + align_up((size_t)terms * ea, 128);
+  MW_TRY(split_planes(A, (int64_t)ea, pa, terms, (int64_t)ea, s));
+  MW_TRY(split_planes(B, (int64_t)eb, pb, terms, (int64_t)eb, s));
+  TcOperand oa, ob;
+  oa.base = pa; oa.planes = terms; oa.plane_stride = (int64_t)ea; oa.mn_major = a_mn != 0;
+  oa.rows = a_mn ? K : M; oa.cols = a_mn ? M : K;
+  ob.base = pb; ob.planes = terms; ob.plane_stride = (int64_t)eb; ob.mn_major = b_mn != 0;
+  ob.rows = b_mn ? K : N; ob.cols = b_mn ? N : K;
+  TcEpilogue e;
+  e.mode = TC_EPI_PLAIN;
+  e.out_f32 = D;
+  MW_TRY(tc_gemm(nullptr, oa, ob, M, N, K, e, st, s));
+  DeviceStatus host;
+  MW_CUDA_OK(cudaMemcpyAsync(&host, st, sizeof(host), cudaMemcpyDeviceToHost, s));
+  MW_CUDA_OK(cudaStreamSynchronize(s));
+  return host.code == 0 ? MW_OK : (mw_status)host.code;
+}
