@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES_PER_LAUNCH = None
 
 
-def workload(name: str, seed: int = 0):
+def workload(name: str, seed: int = 0, depth: int = 0):
     from paper_2402_14212_b200 import synth as S
     if name == "deep_mlp":
         return S.deep_mlp(seed=seed)
@@ -42,12 +42,21 @@ def workload(name: str, seed: int = 0):
         return S.deep_mlp(seed=seed, depth=8, n=256, batch=128)
     if name == "mixed_mlp":
         return S.mixed_mlp(seed=seed)
+    if name == "sweep_mlp":
+        return S.sweep_mlp(seed=seed, depth=depth or 32, pool=4)
+    if name == "submersive_cnn":
+        return S.submersive_cnn(seed=seed)
     if name == "tiny_mlp":
         return S.tiny_mlp(seed=seed)
     raise SystemExit(f"unknown workload {name}")
 
 
 def describe(p):
+    if p.layers[0].kind == "conv2d":
+        l0 = p.layers[0]
+        return {"workload": p.name, "layers": len(p.layers), "conv": f"{l0.k}x{l0.k}x{l0.C_in}x{l0.C_out}",
+                "image": f"{l0.H}x{l0.W}", "batch": p.batch, "prec": p.prec, "loss": p.loss,
+                "reseed_every": p.reseed_every, "conv_vijp_iters": p.conv_vijp_iters, "seed": p.seed}
     return {"workload": p.name, "layers": len(p.layers), "width": p.layers[0].n_in,
             "batch": p.batch, "prec": p.prec, "loss": p.loss, "reseed_every": p.reseed_every,
             "seed": p.seed}
@@ -146,7 +155,7 @@ def run_reference(args):
     import numpy as np
     from oracle import moonwalk_oracle as O
     from paper_2402_14212_b200 import synth as S
-    p = workload(args.workload)
+    p = workload(args.workload, depth=args.depth)
     total = args.steps + args.warmup
     t0 = time.perf_counter()
     O.moonwalk(p.layers, p.params, p.x, p.target, p.loss, reseed_every=p.reseed_every)
@@ -201,7 +210,7 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    p = workload(args.workload)
+    p = workload(args.workload, depth=args.depth)
     net = mwb.net_for(p, backend=args.backend)
     params, x, target = mwb.to_device(p, dev)
     ws = net.alloc_workspace("moonwalk", dev)
@@ -341,6 +350,105 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_depth_sweep(args):
+    """Config 5: dense leaky-ReLU MLP, width 4096, batch 1024, bf16 / fp32 accumulate, depth
+    doubling from 32.  Per depth: workspace and residual bytes of both methods (from the library's
+    own accounting), peak device bytes seen by the allocator, samples/s; and the largest depth whose
+    total (parameters + gradients + workspace) fits 64 GB, from the same accounting."""
+    import torch
+    from paper_2402_14212_b200 import binding as mwb
+    from paper_2402_14212_b200 import synth as S
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    n, batch, budget = 4096, 1024, 64e9
+    base = S.sweep_mlp(seed=0, depth=4, pool=4)
+    pool_dev = [torch.from_numpy(w).to(torch.bfloat16).to(dev) for w in base.params[:4]]
+    x = torch.from_numpy(base.x).to(torch.bfloat16).to(dev)
+    target = torch.from_numpy(base.target).to(torch.float32).to(dev)
+
+    def accounting(depth, resident):
+        layers = [base.layers[0]] * depth
+        net = mwb.Net(layers, batch, base.prec, base.loss, reseed_every=base.reseed_every,
+                      backend="tensor", resident_inverse=resident)
+        mw_b, bp_b, (mw_res, bp_res) = net.workspace_bytes()
+        return net, mw_b, bp_b, mw_res, bp_res
+
+    pbytes, gbytes = n * n * 2, n * n * 4
+    rows = []
+    depth = 32
+    while depth <= args.max_depth:
+        net, mw_b, bp_b, mw_res, bp_res = accounting(depth, False)
+        row = {"depth": depth, "params_bytes": depth * pbytes,
+               "moonwalk": {"workspace_bytes": mw_b, "residual_bytes": mw_res},
+               "backprop": {"workspace_bytes": bp_b, "residual_bytes": bp_res}}
+        # gradients streamed: layer l's dW lands in one of two rotating buffers (applied and
+        # dropped, Algorithm 1's last line), so the totals below exclude a full set of gradients
+        params = [pool_dev[l % 4].clone() for l in range(depth)]
+        dW2 = [torch.empty((n, n), dtype=torch.float32, device=dev) for _ in range(2)]
+        dW = [dW2[l & 1] for l in range(depth)]
+        g0 = torch.empty((batch, n), dtype=torch.float32, device=dev)
+        for which in ("moonwalk", "backprop"):
+            torch.cuda.synchronize()
+            torch.cuda.reset_peak_memory_stats(dev)
+            before = torch.cuda.memory_allocated(dev)
+            ws = net.alloc_workspace(which, dev)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+
+            def step():
+                if which == "moonwalk":
+                    net.input_cotangent(params, x, target, ws, g0_out=g0)
+                    net.forward_sweep(params, x, g0, ws, dW_out=dW)
+                else:
+                    net.backprop_reference(params, x, target, ws, dW_out=dW)
+
+            step()
+            code, detail = net.last_device_status(ws)
+            if code != 0:
+                raise SystemExit(f"device status {code} {detail} at depth {depth} ({which})")
+            reps = 2
+            ev[0].record()
+            for _ in range(reps):
+                step()
+            ev[1].record()
+            torch.cuda.synchronize()
+            ms = ev[0].elapsed_time(ev[1]) / reps
+            row[which].update({"ms_per_step": ms, "samples_per_s": batch / (ms * 1e-3),
+                               "peak_device_bytes": torch.cuda.max_memory_allocated(dev),
+                               "extra_over_params_and_inputs": torch.cuda.max_memory_allocated(dev) - before})
+            del ws
+        rows.append(row)
+        del params, dW, dW2, net
+        torch.cuda.empty_cache()
+        depth *= 2
+
+    def max_depth(which, keep_grads):
+        lo, hi = 1, 1 << 14
+        while lo < hi:
+            mid = (lo + hi + 1) // 2
+            _, mw_b, bp_b, _, _ = accounting(mid, False)
+            ws = mw_b if which == "moonwalk" else bp_b
+            total = mid * pbytes + ws + (mid * gbytes if keep_grads else 2 * gbytes)
+            if total <= budget:
+                lo = mid
+            else:
+                hi = mid - 1
+        return lo
+
+    out = {"workload": "depth sweep: dense leaky-ReLU MLP, width 4096, batch 1024, bf16 storage / fp32 accumulate",
+           "per_layer_bytes": {"params_bf16": pbytes, "grad_fp32": gbytes,
+                               "backprop_stored_activation_bf16": batch * n * 2,
+                               "moonwalk_sign_bits": batch * n // 8,
+                               "moonwalk_cotangent_checkpoint_fp32_every_K": batch * n * 4,
+                               "K": base.reseed_every},
+           "rows": rows,
+           "max_depth_under_64GB": {
+               "moonwalk_grads_streamed": max_depth("moonwalk", False),
+               "backprop_grads_streamed": max_depth("backprop", False),
+               "moonwalk_grads_kept": max_depth("moonwalk", True),
+               "backprop_grads_kept": max_depth("backprop", True)}}
+    print(json.dumps(out), flush=True)
+
+
 def net_backend_is_tensor(net):
     return net.prec != "f64" and all(l.kind == "dense" and l.n_in % 64 == 0 for l in net.layers)
 
@@ -354,8 +462,15 @@ def main():
     ap.add_argument("--workload", default="deep_mlp")
     ap.add_argument("--backend", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--depth", type=int, default=0, help="depth of the sweep_mlp workload")
+    ap.add_argument("--depth-sweep", action="store_true",
+                    help="config 5: peak memory and samples/s versus depth, Moonwalk against the "
+                         "in-library Backprop (prints one JSON object, not the benchmark line)")
+    ap.add_argument("--max-depth", type=int, default=512)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.depth_sweep:
+        run_depth_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

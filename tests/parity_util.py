@@ -73,7 +73,12 @@ def grad_errors(gpu_dW, ref_dW):
 def check_problem(p, tol, backend="simt", inverse_iters=0, resident=True, exact_masks=True, tau=0.0):
     out = run_gpu(p, backend=backend, resident_inverse=resident, inverse_iters=inverse_iters)
     assert out["status"] == 0 and out["bp_status"] == 0
-    ref_own = oracle_reference(p)
+    if exact_masks:
+        ref_own = oracle_reference(p)
+    else:
+        # only the oracle's own pre-activations are needed to judge the sign bits
+        _, _, zs = O.forward(p.layers, p.params, p.x)
+        ref_own = dict(z=zs)
     flips, worst = mask_disagreement(p, out["masks"], ref_own)
     if exact_masks:
         assert flips == 0

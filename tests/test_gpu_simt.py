@@ -114,6 +114,12 @@ def test_small_cnn_fp32_fixed_iterations_match_truncated_oracle():
     check_problem(p, 1e-4, exact_masks=False, tau=1e-4)
 
 
+def test_config3_submersive_cnn_full_size():
+    # 32 stride-1 3x3 convolutions, 64 channels, 32x32, batch 128, fp32, head + cross-entropy
+    p = S.submersive_cnn(seed=0)
+    check_problem(p, 1e-4, backend="auto", exact_masks=False, tau=1e-4)
+
+
 def test_sweep_requires_matching_cotangent_pass():
     torch = torch_cuda()
     p = S.tiny_mlp()

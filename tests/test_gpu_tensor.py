@@ -40,3 +40,18 @@ def test_config2_deep_mlp_full_size():
     # 64 layers, width 1024, batch 256, fp32: the benchmark's workload and launch configuration
     p = S.deep_mlp(seed=0)
     check_problem(p, 1e-4, backend="tensor", exact_masks=False, tau=1e-4)
+
+
+def test_config4_mixed_mlp_full_size():
+    # 128 layers, width 2048, batch 512, bf16 storage, alternating leaky-ReLU / ReLU with the
+    # fragment stream written and read back inside the product kernel's epilogues
+    p = S.mixed_mlp(seed=0)
+    out, ref, errs = check_problem(p, 2e-2, backend="tensor", exact_masks=False, tau=2e-2)
+    assert len(errs) == 128
+
+
+def test_config5_depth32_full_width():
+    # width 4096, batch 1024, bf16, depth 32 (the first point of the depth sweep); four distinct
+    # weight matrices cycled over the depth
+    p = S.sweep_mlp(seed=0, depth=32, pool=4)
+    check_problem(p, 2e-2, backend="tensor", exact_masks=False, tau=2e-2)
