@@ -49,20 +49,21 @@ def oracle_reference(problem, masks=None):
 
 
 def mask_disagreement(problem, gpu_words, ref):
-    """Hamming distance between GPU masks and the oracle's own masks, and the largest |z| (relative
-    to the row rms) at a disagreeing element."""
-    flips, worst = 0, 0.0
+    """Sign bits of the GPU against the signs of the oracle's pre-activations `ref["z"]`.  Returns
+    the Hamming distance and, per layer, the largest |z| (relative to the row rms) at a disagreeing
+    element (0 where the layer agrees everywhere)."""
+    flips, worst = 0, []
     for l, (layer, words) in enumerate(zip(problem.layers, gpu_words)):
-        if layer.act == "none":
-            continue
-        z = ref["z"][l].reshape(words.shape[0], -1)
-        mg = O.unpack_mask(words, z.shape[1])
-        mo = O.sign_mask(z)
-        d = mg != mo
-        if d.any():
-            flips += int(d.sum())
-            rms = np.sqrt((z * z).mean(axis=1, keepdims=True))
-            worst = max(worst, float((np.abs(z) / rms)[d].max()))
+        w = 0.0
+        if layer.act != "none":
+            z = ref["z"][l].reshape(words.shape[0], -1)
+            mg = O.unpack_mask(words, z.shape[1])
+            d = mg != O.sign_mask(z)
+            if d.any():
+                flips += int(d.sum())
+                rms = np.sqrt((z * z).mean(axis=1, keepdims=True))
+                w = float((np.abs(z) / rms)[d].max())
+        worst.append(w)
     return flips, worst
 
 
@@ -71,21 +72,22 @@ def grad_errors(gpu_dW, ref_dW):
 
 
 def check_problem(p, tol, backend="simt", inverse_iters=0, resident=True, exact_masks=True, tau=0.0):
+    """Whole path against the oracle.  exact_masks: the sign bits must equal the oracle's own.
+    Otherwise (fp32 / bf16 arithmetic) the oracle is evaluated on the GPU's exported bits (mask
+    replay) and a bit may contradict the sign of the oracle's pre-activation only where that
+    pre-activation is within rounding of zero: |z| <= tau * sqrt(l + 1) * rms(z_row) at layer l
+    (the per-layer rounding errors of the chain add up like a random walk along the depth)."""
     out = run_gpu(p, backend=backend, resident_inverse=resident, inverse_iters=inverse_iters)
     assert out["status"] == 0 and out["bp_status"] == 0
     if exact_masks:
-        ref_own = oracle_reference(p)
-    else:
-        # only the oracle's own pre-activations are needed to judge the sign bits
-        _, _, zs = O.forward(p.layers, p.params, p.x)
-        ref_own = dict(z=zs)
-    flips, worst = mask_disagreement(p, out["masks"], ref_own)
-    if exact_masks:
+        ref = oracle_reference(p)
+        flips, worst = mask_disagreement(p, out["masks"], ref)
         assert flips == 0
-        ref = ref_own
     else:
-        assert worst <= tau, (flips, worst)
         ref = oracle_reference(p, oracle_masks_from_words(p, out["masks"]))
+        flips, worst = mask_disagreement(p, out["masks"], ref)
+        for l, w in enumerate(worst):
+            assert w <= tau * np.sqrt(l + 1.0), (l, w, flips)
     errs = grad_errors(out["dW"], ref["dW"])
     errs_bp = grad_errors(out["bp_dW"], ref["dW"])
     assert O.normwise_error(out["g0"].reshape(ref["g0"].shape), ref["g0"]) <= tol
@@ -93,6 +95,5 @@ def check_problem(p, tol, backend="simt", inverse_iters=0, resident=True, exact_
     assert max(errs_bp) <= tol, errs_bp
     assert abs(out["loss"] - ref["loss"]) <= max(tol, 1e-12) * max(1.0, abs(ref["loss"]))
     assert abs(out["bp_loss"] - ref["loss"]) <= max(tol, 1e-12) * max(1.0, abs(ref["loss"]))
+    out["flips"], out["worst"] = flips, worst
     return out, ref, errs
-
-
