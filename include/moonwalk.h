@@ -181,6 +181,19 @@ mw_status mw_gemm_split_bf16(const float* A, int32_t a_mn, const float* B, int32
                              int32_t M, int32_t N, int32_t K, int32_t terms, void* scratch,
                              size_t scratch_bytes, void* stream);
 
+/* The three convolution steps of a stride-1, same-size, 64-channel layer on the tensor cores,
+ * exposed for unit parity tests (Lemma 1; Eq. "conv-vjp"; Eq. "g_i"):
+ *   op 0  forward        out[b,i',c'] = sum_{j,c} w[j,c,c'] a[b,i'+j-p,c]      a = x, b = w
+ *   op 1  TransposeConv  out[b,i,c]   = sum_{j,c'} w[j,c,c'] a[b,i+p-j,c']     a = h', b = w
+ *   op 2  weight vjp     out[j,c,c']  = sum_{b,i'} a[b,i'+j-p,c] b[b,i',c']    a = x, b = g_z
+ * Pixel arrays are channel-last float [images][H][W][64], kernels float [k][k][64][64], p = k/2,
+ * zero padding; all device memory.  terms as in mw_gemm_split_bf16.  Sizes: 128 % W == 0 (64 % W
+ * == 0 for op 2), H*W % 128 == 0, k odd.  scratch: device, 256-byte aligned, >= 1024 + 8*terms*
+ * (elements of a + elements of b) bytes (+ 32 * k*k*16 KiB for op 2).  Synchronises `stream`. */
+mw_status mw_conv2d_split_bf16(int32_t op, const float* a, const float* b, float* out,
+                               int32_t images, int32_t H, int32_t W, int32_t k, int32_t terms,
+                               void* scratch, size_t scratch_bytes, void* stream);
+
 /* The same product as mw_gemm_split_bf16 for callers that have no scratch buffer to lend and
  * cannot allocate one when they call: code that runs inside a host framework whose memory pool
  * owns the whole device (a direct cudaMalloc there fails or stalls every stream), and services

@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
         L.mw_relu_fragment_compact.argtypes = [vp, vp, i64, i32, vp, vp, vp, vp, vp, sz, vp]
         L.mw_activation_vijp.argtypes = [vp, vp, i64, i32, i32, C.c_float, vp, vp, vp, vp, vp]
         L.mw_gemm_split_bf16.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, vp, sz, vp]
+        L.mw_conv2d_split_bf16.argtypes = [i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, sz, vp]
         L.mw_gemm_split_bf16_static.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, vp]
         L.mw_gradient_step_host.argtypes = [vp, C.POINTER(vp), vp, sz, vp, sz, vp, vp, vp,
                                             C.POINTER(vp), vp, vp, vp, sz, vp]
@@ -302,6 +303,21 @@ def gemm_split_bf16(A, B, a_mn: bool, b_mn: bool, terms: int, stream=None):
                                     int(terms), _ptr(scratch), scratch.numel(),
                                     _stream_handle(stream)), "mw_gemm_split_bf16")
     return D
+
+
+def conv2d_split_bf16(op: int, a, b, k: int, terms: int, stream=None):
+    """op 0: conv(a = x, b = w); op 1: TransposeConv(a = h', b = w); op 2: weight vjp (a = x, b = g_z)."""
+    import torch
+    images, H, W, C = a.shape
+    assert C == 64
+    out = torch.empty((k, k, 64, 64) if op == 2 else (images, H, W, 64), dtype=torch.float32,
+                      device=a.device)
+    n = 1024 + 8 * terms * (a.numel() + b.numel()) + 32 * k * k * 16384 + 4096
+    scratch = torch.empty(n, dtype=torch.uint8, device=a.device)
+    _check(lib().mw_conv2d_split_bf16(op, _ptr(a), _ptr(b), _ptr(out), images, H, W, k, int(terms),
+                                      _ptr(scratch), scratch.numel(), _stream_handle(stream)),
+           "mw_conv2d_split_bf16")
+    return out
 
 
 GEMM_STATIC_SCRATCH_BYTES = 16 << 20

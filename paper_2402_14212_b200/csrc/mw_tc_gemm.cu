@@ -65,6 +65,8 @@ struct alignas(64) TcProblem {
   int nops, nblocks;
   float* split_partials;
   unsigned int* split_counters;
+  // convolution forms (TcConv)
+  int conv_mode, cH, cW, ck, cpad, csgn, cskip, b_tap_rows, cntaps;
   TcOp ops[kMaxOps];
 };
 
@@ -135,6 +137,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
       "%4, %5}], [%2];" ::"r"(dst),
       "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
+                                            int c0, int c1, int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
+      "%4, %5, %6, %7}], [%2];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
       : "memory");
 }
 
@@ -294,6 +305,17 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int r
       break;
     }
     case TC_EPI_VIJP: {
+      if (e.addend) {
+        const float4* a4 = reinterpret_cast<const float4*>(e.addend + off);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float4 a = a4[i];
+          v[4 * i] = fmaf(e.alpha, v[4 * i], a.x);
+          v[4 * i + 1] = fmaf(e.alpha, v[4 * i + 1], a.y);
+          v[4 * i + 2] = fmaf(e.alpha, v[4 * i + 2], a.z);
+          v[4 * i + 3] = fmaf(e.alpha, v[4 * i + 3], a.w);
+        }
+      }
       float h[32];
       if (e.act == MW_ACT_LEAKY_RELU) {
         const uint32_t word = e.mask[woff];
@@ -444,12 +466,46 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         const int pa = P.pa, pb = P.pb, nbox = P.bn >> 6;
         const bool a_mn = P.a_mn != 0, b_mn = P.b_mn != 0;
         const uint32_t b_tile_bytes = P.b_tile_bytes, tx = P.tx_bytes;
+        const int conv = P.conv_mode;
+        // convolution: image and first image row of the unit's pixel tile
+        int cb = 0, cy0 = 0;
+        if (conv == TC_CONV_PIXELS) {
+          const int hw = P.cH * P.cW;
+          cb = w.m0 / hw;
+          cy0 = (w.m0 - cb * hw) / P.cW;
+        }
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, p.st, 1u, abortp)) { ok = false; break; }
           const uint32_t fb = smem_u32(&full_bar[stage]);
           mbar_expect_tx(fb, tx);
           const uint32_t sbase = tiles + stage * p.stage_bytes;
-          const int k0 = kb * BK;
+          int k0 = kb * BK;
+          int bk0 = k0, bn0 = w.n0;       // B coordinates (K, N)
+          if (conv == TC_CONV_PIXELS) {
+            const int tap = (P.cskip >= 0 && kb >= P.cskip) ? kb + 1 : kb;
+            const int j0 = tap / P.ck, j1 = tap - j0 * P.ck;
+            const int dy = P.csgn * (j0 - P.cpad), dx = P.csgn * (j1 - P.cpad);
+            for (int pl = 0; pl < pa; ++pl)
+              tma_load_5d(sbase + (uint32_t)pl * kATileBytes, &P.tmA, fb, 0, dx, cy0 + dy, cb, a_pl0 + pl);
+            bk0 = tap * BK;
+            if (P.b_tap_rows) { bn0 = tap * BK + w.n0; bk0 = 0; }
+          } else if (conv == TC_CONV_WGRAD) {
+            // K block = 64 pixels of slice z; the two halves of the A tile are two taps
+            const int pix = (w.z * P.num_kb + kb) * BK;
+            const int hw = P.cH * P.cW;
+            const int b = pix / hw, y0 = (pix - b * hw) / P.cW;
+            const int t0 = 2 * (w.m0 / BM);
+            for (int hh = 0; hh < 2; ++hh) {
+              int tap = t0 + hh;
+              if (tap >= P.cntaps) tap = P.cntaps - 1;   // rows past the last tap are never stored
+              const int j0 = tap / P.ck, j1 = tap - j0 * P.ck;
+              for (int pl = 0; pl < pa; ++pl)
+                tma_load_5d(sbase + (uint32_t)pl * kATileBytes + (uint32_t)hh * 8192u, &P.tmA, fb, 0,
+                            j1 - P.cpad, y0 + j0 - P.cpad, b, pl);
+            }
+            bk0 = pix;
+            k0 = pix;
+          } else
           for (int pl = 0; pl < pa; ++pl) {
             const uint32_t dst = sbase + (uint32_t)pl * kATileBytes;
             if (a_mn) {
@@ -460,13 +516,14 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
             }
           }
           const uint32_t bbase = sbase + (uint32_t)pa * kATileBytes;
+          const int bz = conv == TC_CONV_WGRAD ? 0 : b_pl0;
           for (int pl = 0; pl < pb; ++pl) {
             const uint32_t dst = bbase + (uint32_t)pl * b_tile_bytes;
             if (b_mn) {
               for (int h = 0; h < nbox; ++h)
-                tma_load_3d(dst + (uint32_t)h * 8192u, &P.tmB, fb, w.n0 + h * 64, k0, b_pl0 + pl);
+                tma_load_3d(dst + (uint32_t)h * 8192u, &P.tmB, fb, bn0 + h * 64, bk0, bz + pl);
             } else {
-              tma_load_3d(dst, &P.tmB, fb, k0, w.n0, b_pl0 + pl);
+              tma_load_3d(dst, &P.tmB, fb, bk0, bn0, bz + pl);
             }
           }
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
@@ -789,6 +846,33 @@ static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, i
   return MW_OK;
 }
 
+// channel-last pixel array [images][H][W][64] per plane, read in boxes of `box_rows` image rows
+static mw_status get_map_conv(TcMapCache* cache, const TcOperand& op, int H, int W, int box_rows,
+                              int total_planes, CUtensorMap* out) {
+  auto key = std::make_tuple(op.base, op.rows, op.cols, total_planes, op.plane_stride,
+                             1000000 + W * 1000 + box_rows);
+  if (cache) {
+    auto it = cache->maps.find(key);
+    if (it != cache->maps.end()) { *out = it->second; return MW_OK; }
+  }
+  auto fn = encode_fn();
+  if (!fn) return MW_ERR_CUDA;
+  if (((uintptr_t)op.base & 15u) || op.cols != 64 || op.rows % (H * W) != 0) return MW_ERR_INVALID_ARG;
+  const int64_t ps = total_planes > 1 ? op.plane_stride : (int64_t)op.rows * op.cols;
+  if (ps % 8 != 0) return MW_ERR_INVALID_ARG;
+  const cuuint64_t images = (cuuint64_t)(op.rows / (H * W));
+  cuuint64_t dims[5] = {64u, (cuuint64_t)W, (cuuint64_t)H, images, (cuuint64_t)total_planes};
+  cuuint64_t strides[4] = {128u, (cuuint64_t)W * 128u, (cuuint64_t)H * W * 128u, (cuuint64_t)ps * 2};
+  cuuint32_t box[5] = {64u, (cuuint32_t)W, (cuuint32_t)box_rows, 1u, 1u};
+  cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(op.base), dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return MW_ERR_CUDA;
+  if (cache) cache->maps[key] = *out;
+  return MW_OK;
+}
+
 namespace {
 
 uint32_t make_idesc(bool a_mn, bool b_mn, int n) {
@@ -867,7 +951,22 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
     if ((!d.A.mn_major || !d.B.mn_major) && d.K % 64 != 0) return MW_ERR_UNSUPPORTED;
     if (d.A.planes < 1 || d.A.planes > 3 || d.B.planes < 1 || d.B.planes > 3) return MW_ERR_INVALID_ARG;
     if (d.A.mn_major && (d.M % 64 != 0)) return MW_ERR_UNSUPPORTED;
+    const TcConv& cv = d.conv;
+    if (cv.mode != TC_CONV_NONE) {
+      const int span = cv.mode == TC_CONV_PIXELS ? BM : BK;    // pixels per A box
+      if (cv.W < 1 || cv.H < 1 || span % cv.W != 0 || cv.H % (span / cv.W) != 0 || cv.k < 1 ||
+          cv.k * cv.k > 64 || d.N != 64)
+        return MW_ERR_UNSUPPORTED;
+      if (cv.mode == TC_CONV_PIXELS && (d.A.mn_major || d.M % (cv.H * cv.W) != 0 || d.batch != 1 ||
+                                        d.K % 64 != 0 || d.K / 64 > cv.k * cv.k))
+        return MW_ERR_UNSUPPORTED;
+      if (cv.mode == TC_CONV_WGRAD && (!d.A.mn_major || !d.B.mn_major || d.M != cv.k * cv.k * 64 ||
+                                       d.K % 64 != 0 || d.split_k > 1))
+        return MW_ERR_UNSUPPORTED;
+    }
     TcProblem& P = prm.prob[prm.nprob];
+    P.conv_mode = cv.mode; P.cH = cv.H; P.cW = cv.W; P.ck = cv.k; P.cpad = cv.pad; P.csgn = cv.sgn;
+    P.cskip = cv.skip_tap; P.b_tap_rows = cv.b_tap_rows; P.cntaps = cv.k * cv.k;
     P.M = d.M; P.N = d.N; P.K = d.K;
     P.pa = d.A.planes; P.pb = d.B.planes;
     P.a_mn = d.A.mn_major ? 1 : 0;
@@ -908,8 +1007,16 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
     }
     const int a_total = d.batch > 1 ? (d.batch - 1) * P.a_batch_planes + d.A.planes : d.A.planes;
     const int b_total = d.batch > 1 ? (d.batch - 1) * P.b_batch_planes + d.B.planes : d.B.planes;
-    MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA));
-    MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
+    if (cv.mode == TC_CONV_PIXELS) {
+      MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, BM / cv.W, a_total, &P.tmA));
+      MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
+    } else if (cv.mode == TC_CONV_WGRAD) {
+      MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, BK / cv.W, d.A.planes, &P.tmA));
+      MW_TRY(get_map(cache, d.B, 64, d.B.planes, &P.tmB));
+    } else {
+      MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA));
+      MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
+    }
     int np = 0;
     for (int a = 0; a < P.pa; ++a)
       for (int b = 0; b < P.pb; ++b)

@@ -39,7 +39,8 @@ enum TcEpiMode : int {
   TC_EPI_RESID = 1,    // v = (row == col) - acc;    planes; sum of squares -> sumsq
   TC_EPI_FWD = 2,      // z = acc; sign word written (write_mask) or read; x = phi(z) -> planes (+ out_f32)
   TC_EPI_BWD = 3,      // h = acc -> out_f32 (optional), ReLU fragments (optional); g = h * phi'(mask) -> planes
-  TC_EPI_VIJP = 4,     // g = acc; activation vijp: h -> planes2 (+ out_f32); g (zero at dead ReLU units) -> planes
+  TC_EPI_VIJP = 4,     // g = alpha*acc (+ addend); activation vijp: h -> planes2 (+ out_f32); g (zero at dead
+                       // ReLU units) -> planes
 };
 
 struct TcEpilogue {
@@ -72,12 +73,36 @@ struct TcEpilogue {
   int64_t bs_sumsq = 0;                // doubles
 };
 
+// Convolution forms of a product (stride 1, same size, 64 channels = one K block per tap).
+// The A operand is then a channel-last pixel array [B][H][W][64] per term plane, read through a
+// window shifted by the tap (out-of-image pixels read as zero: the padding of Lemma 1):
+//   TC_CONV_PIXELS  rows of A = pixels, K = (tap, channel): K block kb is tap kb (taps before
+//                   `skip_tap` keep their index, later ones move down by one) and reads pixel
+//                   (y + sgn*(j0 - pad), x + sgn*(j1 - pad)).  sgn = +1: forward convolution,
+//                   sgn = -1: TransposeConv (Eq. "conv-vjp").  B is indexed by the same tap.
+//   TC_CONV_WGRAD   weight vjp (Eq. "g_i" for a convolution): rows of the result = (tap, c), two
+//                   taps per 128-row tile; K = pixels; batch item z covers the K blocks
+//                   [z*K/64, (z+1)*K/64) of the pixel range, so that `batch` slices of the pixel sum
+//                   land in separate outputs.  A (MN-major) is the shifted activation, B (MN-major)
+//                   the cotangent [pixels][64].
+enum TcConvMode : int { TC_CONV_NONE = 0, TC_CONV_PIXELS = 1, TC_CONV_WGRAD = 2 };
+
+struct TcConv {
+  int mode = TC_CONV_NONE;
+  int H = 0, W = 0;         // image; 128 % W == 0 (64 % W == 0 for TC_CONV_WGRAD), H*W % 128 == 0
+  int k = 0, pad = 0;       // kernel k x k
+  int sgn = 1;
+  int skip_tap = -1;        // tap left out of the sum (the centre tap of the folded kernel), or -1
+  int b_tap_rows = 0;       // B is K-major with rows (tap, n): used by TransposeConv
+};
+
 // One product of a group.
 struct TcGemm {
   TcOperand A, B;
   int M = 0, N = 0, K = 0;
   int batch = 1;
   TcEpilogue epi;
+  TcConv conv;
   // K split: the K range of every output tile is cut into `split_k` pieces computed by
   // different CTAs; partial tiles meet in `split_scratch` (kTcSplitCounterBytes of arrival
   // counters, zero before the first use and left zero by every launch, then split_k * tiles *

@@ -1,0 +1,36 @@
+"""Convolution steps on the tensor cores against the oracle's plain definitions (Lemma 1,
+Eq. "conv-vjp", Eq. "g_i"), on the same seeded arrays."""
+import numpy as np
+import pytest
+
+from oracle import moonwalk_oracle as O
+from paper_2402_14212_b200 import binding as mwb
+
+pytestmark = pytest.mark.gpu
+
+TOL = {1: 2e-2, 2: 2e-4, 3: 2e-6}
+
+
+@pytest.mark.parametrize("terms", [1, 2, 3])
+@pytest.mark.parametrize("images,H,W,k", [(1, 4, 32, 3), (3, 8, 16, 3), (2, 16, 64, 3), (4, 32, 32, 3),
+                                          (2, 8, 32, 5), (1, 4, 32, 1)])
+def test_conv_products(images, H, W, k, terms):
+    import torch
+    assert torch.cuda.is_available()
+    rng = np.random.default_rng(images * 100 + H + W + k + terms)
+    x = rng.standard_normal((images, H, W, 64)).astype(np.float32)
+    g = rng.standard_normal((images, H, W, 64)).astype(np.float32)
+    w = (rng.standard_normal((k, k, 64, 64)) / np.sqrt(64 * k * k)).astype(np.float32)
+    # marks that a wrong shift, a transposed tap or a swapped channel pair would move
+    x[0, 0, 0, :] = 0.0; x[0, 0, 0, 1] = 3.0
+    w[0, k - 1, 1, 2] = 1.5
+    p = k // 2
+    xt, gt, wt = (torch.from_numpy(a).cuda() for a in (x, g, w))
+    x64, g64, w64 = x.astype(np.float64), g.astype(np.float64), w.astype(np.float64)
+    cases = [(0, xt, wt, O.conv_forward(x64, w64, 1, p)),
+             (1, gt, wt, O.transpose_conv(g64, w64, (H, W), 1, p)),
+             (2, xt, gt, O.conv_weight_vjp(x64, g64, k, 1, p))]
+    for op, a, b, ref in cases:
+        got = mwb.conv2d_split_bf16(op, a, b, k, terms).double().cpu().numpy()
+        err = np.abs(got - ref).max() / np.abs(ref).max()
+        assert err <= TOL[terms], (op, err)
