@@ -32,6 +32,9 @@ struct Layout {
   // tensor-core backend operands (bf16 term planes)
   std::vector<Region> w_planes;              // split weights (MW_F32), per layer or one slot
   Region xp[3], hp[2], gzp[2], ns_r, ns_x, ns_w; // activation / cotangent / g_z planes, NS scratch
+  // convolution nets on the tensor cores
+  std::vector<Region> cw, cwhat, cwinv;      // per layer: kernel, folded kernel, centre-tap inverse (term planes)
+  Region cwinv_f32, cwhat_f32, cg[2], chpf, cxf, cpart, clogits;
   Region split[3];                           // K-split meeting places of concurrently running products
 };
 

@@ -20,10 +20,6 @@ namespace mw {
 
 namespace {
 
-struct TensorState {
-  TcMapCache* cache = nullptr;
-};
-
 struct Prec {
   int px;    // activation / weight terms (recompute, Phase I)
   int ph;    // cotangent-chain terms (h and W^-1 in the dense vijp)
@@ -421,6 +417,7 @@ mw_status loss_and_top(const Ctx& c, const void* target, double* loss_out, bool 
 }  // namespace
 
 bool tensor_supported(const mw_net* n) {
+  if (n->layers[0].kind == MW_CONV2D) return conv_tensor_supported(n);
   if (n->opts.prec != MW_F32 && n->opts.prec != MW_BF16_F32ACC) return false;
   if (n->opts.loss == MW_LOSS_XENT_MEAN) return false;
   const int d = n->layers[0].n_in;
@@ -443,6 +440,10 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     TensorState* t = new TensorState();
     t->cache = tc_cache_create();
     n->tc = t;
+  }
+  if (n->layers[0].kind == MW_CONV2D) {
+    conv_tensor_layout(n, backprop, lay, start);
+    return;
   }
   const Prec pr = prec_of(n);
   const int L = n->L;
@@ -506,6 +507,8 @@ void tensor_destroy(mw_net* n) {
 mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const void* x,
                                  const void* target, void* g0, double* loss_out, void* ws,
                                  cudaStream_t s) {
+  if (n->layers[0].kind == MW_CONV2D)
+    return conv_tensor_input_cotangent(n, params, x, target, g0, loss_out, ws, s);
   const Layout& lay = n->mwl;
   Ctx c = make_ctx(n, lay, ws, s);
   const int L = n->L, d = c.dim;
@@ -554,6 +557,7 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
 
 mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void* x, const void* g0,
                                void* const* dW, void* ws, cudaStream_t s) {
+  if (n->layers[0].kind == MW_CONV2D) return conv_tensor_forward_sweep(n, params, x, g0, dW, ws, s);
   const Layout& lay = n->mwl;
   Ctx c = make_ctx(n, lay, ws, s);
   const int L = n->L, d = c.dim;
@@ -632,6 +636,8 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
 
 mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, const void* target,
                           void* const* dW, double* loss_out, void* ws, cudaStream_t s) {
+  if (n->layers[0].kind == MW_CONV2D)
+    return conv_tensor_backprop(n, params, x, target, dW, loss_out, ws, s);
   const Layout& lay = n->bpl;
   Ctx c = make_ctx(n, lay, ws, s);
   const int L = n->L, d = c.dim;

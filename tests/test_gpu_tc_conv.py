@@ -34,3 +34,17 @@ def test_conv_products(images, H, W, k, terms):
         got = mwb.conv2d_split_bf16(op, a, b, k, terms).double().cpu().numpy()
         err = np.abs(got - ref).max() / np.abs(ref).max()
         assert err <= TOL[terms], (op, err)
+
+
+# ---------------------------------------------------------------------------------------
+# whole path on the tensor-core convolution pipeline (fp32, 64 channels)
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("depth,H,W,batch,K,iters,resident", [(3, 8, 16, 2, 2, 10, True), (4, 4, 32, 3, 0, 12, True), (6, 4, 32, 2, 3, 10, True),
+                                                              (4, 16, 64, 1, 3, 10, False)])
+def test_small_cnn_fp32_tensor_path(depth, H, W, batch, K, iters, resident):
+    from paper_2402_14212_b200 import synth as S
+    from parity_util import check_problem
+    p = S.submersive_cnn(seed=depth, depth=depth, C=64, H=H, W=W, batch=batch, gamma=0.05, classes=10,
+                         reseed_every=K, conv_vijp_iters=iters, prec=S.F32)
+    out, ref, errs = check_problem(p, 1e-4, backend="tensor", resident=resident, exact_masks=False,
+                                   tau=1e-4)
