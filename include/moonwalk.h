@@ -88,7 +88,7 @@ typedef struct {
   int32_t resident_inverse;/* 1: mw_input_cotangent computes every layer's W^-1 (and split
                               operands) once and keeps them in the workspace; 0: the sweep
                               builds them layer by layer in a transient slot (lean memory) */
-  int32_t reserved;
+  int32_t reserved;        /* 0; 1 = run the forward sweep as a single launch (experimental)     */
 } mw_net_opts;
 
 /* Build a host-side description.  `batch` is fixed per net.  Returns MW_ERR_UNSUPPORTED for

@@ -81,7 +81,12 @@ void build_layout(mw_net* n, bool backprop, Layout& lay) {
       }
     }
     for (int l = 1; l < L; ++l)
-      if (is_reseed(n, l)) lay.reseed[l] = b.take((n->opts.prec == MW_F64 ? 8 : 4) * (size_t)n->info[l - 1].out_elems);
+      if (is_reseed(n, l)) {
+        // dense tensor-core nets keep the checkpoint as bf16 term planes (3 for MW_F32, 2 otherwise)
+        size_t per = n->opts.prec == MW_F64 ? 8 : 4;
+        if (n->backend == MW_BACKEND_TENSOR && n->layers[0].kind == MW_DENSE && n->opts.prec == MW_F32) per = 6;
+        lay.reseed[l] = b.take(per * (size_t)n->info[l - 1].out_elems);
+      }
     if (n->layers[L - 1].kind == MW_HEAD_LINEAR)
       lay.h_last = b.take((n->opts.prec == MW_F64 ? 8 : 4) * (size_t)n->info[L - 1].out_elems);
   } else {

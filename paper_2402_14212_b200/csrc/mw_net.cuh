@@ -35,6 +35,8 @@ struct Layout {
   // convolution nets on the tensor cores
   std::vector<Region> cw, cwhat, cwinv;      // per layer: kernel, folded kernel, centre-tap inverse (term planes)
   Region cwinv_f32, cwhat_f32, cg[2], chpf, cxf, cpart, clogits;
+  Region ns_sumsq;
+  Region prog_table[3], prog_done[3];        // product tables and completion counters of program launches
   Region split[3];                           // K-split meeting places of concurrently running products
 };
 

@@ -39,6 +39,7 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int kThreadsTc = 192;
+constexpr int kEpiWarps = 4;     // one per tensor-memory lane quarter
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far above any legitimate wait
 constexpr int kMaxStages = 8;
 constexpr int kMaxOps = 6;
@@ -67,13 +68,21 @@ struct alignas(64) TcProblem {
   unsigned int* split_counters;
   // convolution forms (TcConv)
   int conv_mode, cH, cW, ck, cpad, csgn, cskip, b_tap_rows, cntaps;
+  // program launches: products (by index) that must be complete before this one starts, and
+  // the number of warp arrivals that completes each of them (one per epilogue warp and tile)
+  int ndep, dep[3];
+  unsigned int dep_target[3];
   TcOp ops[kMaxOps];
 };
+
+constexpr int kMaxProgram = 768;   // products of one program launch
 
 struct alignas(64) TcGroupParams {
   int nprob, total_units, stages, pad0;
   uint32_t stage_bytes, pad1;
   DeviceStatus* st;
+  const TcProblem* table;     // program launch: the products live in global memory ...
+  unsigned int* done;         // ... and count their finished tiles here (zero at launch)
   TcProblem prob[kTcMaxGroup];
 };
 
@@ -127,6 +136,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, DeviceS
     }
   }
   record_error(st, MW_ERR_TIMEOUT, who, blockIdx.x, 0u, 0u);
+  *abort_flag = 1;
+  return false;
+}
+
+// Bounded wait for a product of the same (co-resident) launch: its tiles count themselves in
+// global memory.  Same bound and failure path as mbar_wait.
+__device__ __forceinline__ bool wait_done(const unsigned int* counter, unsigned int target,
+                                          DeviceStatus* st, volatile int* abort_flag) {
+  uint64_t t0 = 0;
+  for (uint32_t i = 0;; ++i) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= target) return true;
+    __nanosleep(40);
+    if ((i & 63u) == 63u) {
+      if (*abort_flag) return false;
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) break;
+    }
+  }
+  record_error(st, MW_ERR_TIMEOUT, 5u, blockIdx.x, target, 0u);
   *abort_flag = 1;
   return false;
 }
@@ -286,6 +317,12 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int r
     }
     case TC_EPI_BWD: {
       if (e.out_f32) store_f32x32(v, e.out_f32 + off);
+      if (e.n_planes2) {   // cotangent checkpoint as term planes (the sweep reads it as an operand)
+        float h[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) h[i] = v[i];
+        store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, off);
+      }
       const uint32_t word = e.act != MW_ACT_NONE ? e.mask[woff] : 0xffffffffu;
       if (e.act == MW_ACT_RELU && e.frag_vals) {
         // fragments: the cotangent at dead units, in column order
@@ -376,12 +413,10 @@ __device__ __forceinline__ void issue_k_block(const uint32_t (&oa)[kMaxOps], con
 }
 
 // unit u of the sorted list -> product, tile, batch item and K range
-__device__ __forceinline__ void decode_unit(const TcGroupParams& p, int u, Unit& w) {
-  int q = 0;
-#pragma unroll
-  for (int i = 1; i < kTcMaxGroup; ++i)
-    if (i < p.nprob && u >= p.prob[i].unit_begin) q = i;
-  const TcProblem& P = p.prob[q];
+__device__ __forceinline__ void decode_unit(const TcProblem* probs, const int* ub, int nprob, int u,
+                                            int& q, Unit& w) {
+  while (q + 1 < nprob && u >= ub[q + 1]) ++q;    // units come in increasing order
+  const TcProblem& P = probs[q];
   const int local = u - P.unit_begin;
   const int tl = local / P.split;
   const int ks = local - tl * P.split;
@@ -399,13 +434,25 @@ __device__ __forceinline__ void decode_unit(const TcGroupParams& p, int u, Unit&
   w.kb1 = e < P.num_kb ? e : P.num_kb;
 }
 
-// units of this CTA: round r takes index r*G + c (even r) or r*G + G-1-c (odd r)
-#define MW_FOR_MY_UNITS(p, u)                                                              \
-  for (int r_ = 0, u = 0; r_ * (int)gridDim.x < (p).total_units; ++r_)                   \
-    if ((u = r_ * (int)gridDim.x +                                                        \
-             ((r_ & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x)) <       \
-        (p).total_units)
+// Units of this CTA: round r takes index r*G + c (even r) or r*G + G-1-c (odd r); a program
+// launch takes r*G + c throughout, so that one CTA never holds two units of one short product
+// (they would run one after the other and hold up everything that waits for that product).
+// (Handing units out dynamically in list order was tried and is slower: CTAs pile up behind the
+// one product that is not complete yet.)
+template <bool kProgram>
+__device__ __forceinline__ int next_unit(const TcGroupParams& p, int& r) {
+  const int G = (int)gridDim.x, c = (int)blockIdx.x;
+  while (r * G < p.total_units) {
+    const int u = r * G + (((r & 1) && !kProgram) ? G - 1 - c : c);
+    ++r;
+    if (u < p.total_units) return u;
+  }
+  return -1;
+}
 
+// kProgram: the products live in global memory and wait for one another (program launch);
+// otherwise they are read straight from the kernel parameters
+template <bool kProgram>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 tc_group_kernel(const __grid_constant__ TcGroupParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -415,10 +462,14 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
   __shared__ __align__(8) uint64_t acc_empty[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
+  __shared__ int ub[kMaxProgram + 1];     // first unit of every product
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;  // 1024-byte aligned for the swizzle
+  const TcProblem* probs = kProgram ? p.table : p.prob;
+  const int nprob = p.nprob;
+  for (int i = threadIdx.x; i < nprob; i += kThreadsTc) ub[i] = probs[i].unit_begin;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -427,15 +478,15 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&acc_full[s]), 1);
-      mbar_init(smem_u32(&acc_empty[s]), 4);   // one arrival per epilogue warp
+      mbar_init(smem_u32(&acc_empty[s]), kEpiWarps);   // one arrival per epilogue warp
     }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 2 && lane < 2 * p.nprob) {
+  if (warp == 2 && lane < 2 * nprob && lane < 2 * kTcMaxGroup) {
     // start fetching the tensor maps before the first copy needs them
-    const TcProblem& P = p.prob[lane >> 1];
+    const TcProblem& P = probs[lane >> 1];
     const CUtensorMap* tm = (lane & 1) ? &P.tmB : &P.tmA;
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
   }
@@ -457,11 +508,21 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
       bool ok = true;
-      MW_FOR_MY_UNITS(p, u) {
+      int q = 0, rr = 0;
+      for (;;) {
         if (!ok) break;
+        const int u = next_unit<kProgram>(p, rr);
+        if (u < 0) break;
         Unit w;
-        decode_unit(p, u, w);
-        const TcProblem& P = p.prob[w.q];
+        decode_unit(probs, ub, nprob, u, q, w);
+        const TcProblem& P = probs[w.q];
+        if (kProgram && P.ndep) {
+          // program launch: the operands are written by earlier products of this same launch
+          for (int i = 0; i < P.ndep && ok; ++i)
+            ok = wait_done(p.done + P.dep[i], P.dep_target[i], p.st, abortp);
+          if (!ok) break;
+          asm volatile("fence.proxy.async;" ::: "memory");   // their stores, then our bulk copies
+        }
         const int a_pl0 = w.z * P.a_batch_planes, b_pl0 = w.z * P.b_batch_planes;
         const int pa = P.pa, pb = P.pb, nbox = P.bn >> 6;
         const bool a_mn = P.a_mn != 0, b_mn = P.b_mn != 0;
@@ -534,13 +595,15 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
-      int j = 0;
+      int j = 0, q = 0, rr = 0;
       bool ok = true;
-      MW_FOR_MY_UNITS(p, u) {
+      for (;;) {
         if (!ok) break;
+        const int u = next_unit<kProgram>(p, rr);
+        if (u < 0) break;
         Unit w;
-        decode_unit(p, u, w);
-        const TcProblem& P = p.prob[w.q];
+        decode_unit(probs, ub, nprob, u, q, w);
+        const TcProblem& P = probs[w.q];
         const uint32_t set = (uint32_t)j & 1u, aphase = ((uint32_t)j >> 1) & 1u;
         if (!mbar_wait(smem_u32(&acc_empty[set]), aphase ^ 1u, p.st, 2u, abortp)) { ok = false; break; }
         tc_fence_after();
@@ -585,13 +648,16 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
   } else {
     // ---------------- epilogue (warps 2..5) ----------------
     const int quarter = warp & 3;                 // tensor-memory lane quarter this warp may read
-    int j = 0;
+    const int half = 0;
+    int j = 0, q = 0, rr = 0;
     bool ok = true;
-    MW_FOR_MY_UNITS(p, u) {
+    for (;;) {
       if (!ok) break;
+      const int u = next_unit<kProgram>(p, rr);
+      if (u < 0) break;
       Unit w;
-      decode_unit(p, u, w);
-      const TcProblem& P = p.prob[w.q];
+      decode_unit(probs, ub, nprob, u, q, w);
+      const TcProblem& P = probs[w.q];
       const uint32_t set = (uint32_t)j & 1u, aphase = ((uint32_t)j >> 1) & 1u;
       // every lane observes the barrier itself; the warp then takes one common decision so the
       // warp-wide tensor-memory loads below are never executed by part of a warp
@@ -634,7 +700,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         float* mine = P.split_partials + ((int64_t)w.tl * P.split + w.ks) * (int64_t)(BM * bn) +
                       quarter * 32 + lane;
 #pragma unroll 1
-        for (int c = 0; c < bn; c += 32) {
+        for (int c = half * 32; c < bn; c += 32 * (kEpiWarps / 4)) {
           if (w.n0 + c >= N) break;
           float v[32];
           load_chunk(c, v);
@@ -644,7 +710,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         }
         __threadfence();
         __syncwarp();
-        unsigned int* cnt = P.split_counters + (int64_t)w.tl * 4 + quarter;
+        unsigned int* cnt = P.split_counters + (int64_t)w.tl * kEpiWarps + quarter * (kEpiWarps / 4) + half;
         unsigned int old = 0;
         if (lane == 0) old = atomicAdd(cnt, 1u);
         old = __shfl_sync(0xffffffffu, old, 0);
@@ -661,7 +727,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
                                                 quarter * 32 + lane
                                           : nullptr;
 #pragma unroll 1
-        for (int c = 0; c < bn; c += 32) {
+        for (int c = half * 32; c < bn; c += 32 * (kEpiWarps / 4)) {
           if (w.n0 + c >= N) break;
           float v[32];
           if (P.split > 1) {
@@ -669,17 +735,26 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
             load_chunk(c, own);
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = 0.f;
-            for (int sp = 0; sp < P.split; ++sp) {
-              if (sp == w.ks) {
+            // two pieces per round trip (all loads of a pair are in flight together), added in
+            // index order with this warp's own piece in its place
+            for (int sp = 0; sp < P.split; sp += 2) {
+              const bool has1 = sp + 1 < P.split;
+              const float* s0 = others + (int64_t)sp * (BM * bn) + (int64_t)c * BM;
+              const float* s1 = s0 + (int64_t)(BM * bn);
+              float t0[32], t1[32];
+              if (sp != w.ks) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] += own[i];
-              } else {
-                const float* src = others + (int64_t)sp * (BM * bn) + (int64_t)c * BM;
-                float t[32];
+                for (int i = 0; i < 32; ++i) t0[i] = __ldcg(s0 + i * BM);
+              }
+              if (has1 && sp + 1 != w.ks) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) t[i] = __ldcg(src + i * BM);
+                for (int i = 0; i < 32; ++i) t1[i] = __ldcg(s1 + i * BM);
+              }
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] += t[i];
+              for (int i = 0; i < 32; ++i) v[i] += sp == w.ks ? own[i] : t0[i];
+              if (has1) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] += sp + 1 == w.ks ? own[i] : t1[i];
               }
             }
           } else {
@@ -694,6 +769,12 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&acc_empty[set]));
       ++j;
+      if (kProgram && fused_step) {
+        // program launch: publish this warp's part of the tile to the products that wait for it
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(p.done + w.q, 1u);
+      }
       if (epi.mode == TC_EPI_RESID && epi.sumsq) {
         for (int o = 16; o; o >>= 1) sumsq_local += __shfl_xor_sync(0xffffffffu, sumsq_local, o);
         if (lane == 0 && sumsq_local != 0.0) atomicAdd(epi.sumsq, sumsq_local);
@@ -744,11 +825,11 @@ int sm_count() {
 
 // tile width: as wide as the accumulator set allows for the number of term orders, narrowed while
 // the product alone cannot give every SM a tile
-int pick_bn(int pa, int pb, int M, int N, int batch) {
+int pick_bn(int pa, int pb, int M, int N, int batch, bool wide = false) {
   const int t = pa > pb ? pa : pb;
   int bn = t == 1 ? 256 : (t == 2 ? 128 : 64);
   const int tm = (M + BM - 1) / BM;
-  while (bn > 64 && (N % bn != 0 || (int64_t)tm * (N / bn) * batch < sm_count())) bn >>= 1;
+  while (bn > 64 && (N % bn != 0 || (!wide && (int64_t)tm * (N / bn) * batch < sm_count()))) bn >>= 1;
   return bn;
 }
 
@@ -934,95 +1015,123 @@ double build_ops(TcProblem& P, bool rotate) {
 
 }  // namespace
 
+// fills P from d (everything but unit_begin); returns the tensor-core cycles of one unit
+static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P, double* unit_cost,
+                               double* flops, double* mma_flops) {
+  if (d.N % 64 != 0) return MW_ERR_UNSUPPORTED;
+  // a ragged K tail is zero-filled by the copies of MN-major operands (K counts their rows)
+  if ((!d.A.mn_major || !d.B.mn_major) && d.K % 64 != 0) return MW_ERR_UNSUPPORTED;
+  if (d.A.planes < 1 || d.A.planes > 3 || d.B.planes < 1 || d.B.planes > 3) return MW_ERR_INVALID_ARG;
+  if (d.A.mn_major && (d.M % 64 != 0)) return MW_ERR_UNSUPPORTED;
+  const TcConv& cv = d.conv;
+  if (cv.mode != TC_CONV_NONE) {
+    const int span = cv.mode == TC_CONV_PIXELS ? BM : BK;    // pixels per A box
+    if (cv.W < 1 || cv.H < 1 || span % cv.W != 0 || cv.H % (span / cv.W) != 0 || cv.k < 1 ||
+        cv.k * cv.k > 64 || d.N != 64)
+      return MW_ERR_UNSUPPORTED;
+    if (cv.mode == TC_CONV_PIXELS && (d.A.mn_major || d.M % (cv.H * cv.W) != 0 || d.batch != 1 ||
+                                      d.K % 64 != 0 || d.K / 64 > cv.k * cv.k))
+      return MW_ERR_UNSUPPORTED;
+    if (cv.mode == TC_CONV_WGRAD && (!d.A.mn_major || !d.B.mn_major || d.M != cv.k * cv.k * 64 ||
+                                     d.K % 64 != 0 || d.split_k > 1))
+      return MW_ERR_UNSUPPORTED;
+  }
+  P.conv_mode = cv.mode; P.cH = cv.H; P.cW = cv.W; P.ck = cv.k; P.cpad = cv.pad; P.csgn = cv.sgn;
+  P.cskip = cv.skip_tap; P.b_tap_rows = cv.b_tap_rows; P.cntaps = cv.k * cv.k;
+  P.ndep = 0;
+  P.M = d.M; P.N = d.N; P.K = d.K;
+  P.pa = d.A.planes; P.pb = d.B.planes;
+  P.a_mn = d.A.mn_major ? 1 : 0;
+  P.b_mn = d.B.mn_major ? 1 : 0;
+  P.a_batch_planes = d.A.batch_planes ? d.A.batch_planes : d.A.planes;
+  P.b_batch_planes = d.B.batch_planes ? d.B.batch_planes : d.B.planes;
+  P.bn = pick_bn(P.pa, P.pb, d.M, d.N, d.batch, d.wide_tiles != 0);
+  P.num_kb = (d.K + BK - 1) / BK;
+  int split = d.split_k > 1 ? d.split_k : 1;
+  if (split > P.num_kb) split = P.num_kb;
+  P.kb_per_split = (P.num_kb + split - 1) / split;
+  split = (P.num_kb + P.kb_per_split - 1) / P.kb_per_split;
+  P.split = split;
+  const int tiles_m = (d.M + BM - 1) / BM;
+  P.tiles_n = (d.N + P.bn - 1) / P.bn;
+  P.tiles_mn = tiles_m * P.tiles_n;
+  const int64_t units = (int64_t)P.tiles_mn * d.batch * split;
+  if (units > (1 << 30)) return MW_ERR_UNSUPPORTED;
+  P.unit_count = (int)units;
+  P.b_tile_bytes = (uint32_t)P.bn * BK * 2;
+  P.tx_bytes = (uint32_t)P.pa * kATileBytes + (uint32_t)P.pb * P.b_tile_bytes;
+  const int t = P.pa > P.pb ? P.pa : P.pb;
+  // fp32-accurate products alternate the leading block (needs two K blocks per unit)
+  const bool rotate = t == 3 && P.pa == 3 && P.pb == 3 && P.kb_per_split >= 2 &&
+                      (P.num_kb - (split - 1) * P.kb_per_split) >= 2;
+  const double kb_cycles = build_ops(P, rotate);
+  *unit_cost = kb_cycles * P.kb_per_split;
+  P.epi = d.epi;
+  P.split_partials = nullptr;
+  P.split_counters = nullptr;
+  if (split > 1) {
+    if (!d.split_scratch || ((uintptr_t)d.split_scratch & 255u)) return MW_ERR_WORKSPACE;
+    const size_t tiles = (size_t)P.tiles_mn * d.batch;
+    if (tiles * kEpiWarps * sizeof(unsigned) > kTcSplitCounterBytes) return MW_ERR_UNSUPPORTED;
+    P.split_counters = static_cast<unsigned int*>(d.split_scratch);
+    P.split_partials = reinterpret_cast<float*>(static_cast<char*>(d.split_scratch) + kTcSplitCounterBytes);
+  }
+  const int a_total = d.batch > 1 ? (d.batch - 1) * P.a_batch_planes + d.A.planes : d.A.planes;
+  const int b_total = d.batch > 1 ? (d.batch - 1) * P.b_batch_planes + d.B.planes : d.B.planes;
+  if (cv.mode == TC_CONV_PIXELS) {
+    MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, BM / cv.W, a_total, &P.tmA));
+    MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
+  } else if (cv.mode == TC_CONV_WGRAD) {
+    MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, BK / cv.W, d.A.planes, &P.tmA));
+    MW_TRY(get_map(cache, d.B, 64, d.B.planes, &P.tmB));
+  } else {
+    MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA));
+    MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
+  }
+  int np = 0;
+  for (int a = 0; a < P.pa; ++a)
+    for (int b = 0; b < P.pb; ++b)
+      if (a + b < t) ++np;
+  *flops += 2.0 * d.M * d.N * d.K * d.batch;
+  *mma_flops += 2.0 * d.M * d.N * d.K * np * d.batch;
+  return MW_OK;
+}
+
+static int stages_for(uint32_t stage_bytes) {
+  const uint32_t budget = 227u * 1024u - 8192u;   // static shared memory + alignment slack
+  int stages = (int)(budget / stage_bytes);
+  return stages > kMaxStages ? kMaxStages : stages;
+}
+
+static mw_status ensure_kernel_attr() {
+  static bool attr_set = false;
+  if (!attr_set) {
+    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    227 * 1024 - 6144));
+    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    227 * 1024 - 6144));
+    attr_set = true;
+  }
+  return MW_OK;
+}
+
 mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceStatus* st,
                         cudaStream_t s) {
   if (count < 1 || count > kTcMaxGroup) return MW_ERR_INVALID_ARG;
   static thread_local TcGroupParams prm;
   prm.nprob = 0;
   prm.st = st;
+  prm.table = nullptr;
+  prm.done = nullptr;
   double cost[kTcMaxGroup];
   double flops = 0.0, mma_flops = 0.0;
   uint32_t stage_bytes = 0;
   for (int i = 0; i < count; ++i) {
     const TcGemm& d = g[i];
     if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.batch <= 0) continue;
-    if (d.N % 64 != 0) return MW_ERR_UNSUPPORTED;
-    // a ragged K tail is zero-filled by the copies of MN-major operands (K counts their rows)
-    if ((!d.A.mn_major || !d.B.mn_major) && d.K % 64 != 0) return MW_ERR_UNSUPPORTED;
-    if (d.A.planes < 1 || d.A.planes > 3 || d.B.planes < 1 || d.B.planes > 3) return MW_ERR_INVALID_ARG;
-    if (d.A.mn_major && (d.M % 64 != 0)) return MW_ERR_UNSUPPORTED;
-    const TcConv& cv = d.conv;
-    if (cv.mode != TC_CONV_NONE) {
-      const int span = cv.mode == TC_CONV_PIXELS ? BM : BK;    // pixels per A box
-      if (cv.W < 1 || cv.H < 1 || span % cv.W != 0 || cv.H % (span / cv.W) != 0 || cv.k < 1 ||
-          cv.k * cv.k > 64 || d.N != 64)
-        return MW_ERR_UNSUPPORTED;
-      if (cv.mode == TC_CONV_PIXELS && (d.A.mn_major || d.M % (cv.H * cv.W) != 0 || d.batch != 1 ||
-                                        d.K % 64 != 0 || d.K / 64 > cv.k * cv.k))
-        return MW_ERR_UNSUPPORTED;
-      if (cv.mode == TC_CONV_WGRAD && (!d.A.mn_major || !d.B.mn_major || d.M != cv.k * cv.k * 64 ||
-                                       d.K % 64 != 0 || d.split_k > 1))
-        return MW_ERR_UNSUPPORTED;
-    }
     TcProblem& P = prm.prob[prm.nprob];
-    P.conv_mode = cv.mode; P.cH = cv.H; P.cW = cv.W; P.ck = cv.k; P.cpad = cv.pad; P.csgn = cv.sgn;
-    P.cskip = cv.skip_tap; P.b_tap_rows = cv.b_tap_rows; P.cntaps = cv.k * cv.k;
-    P.M = d.M; P.N = d.N; P.K = d.K;
-    P.pa = d.A.planes; P.pb = d.B.planes;
-    P.a_mn = d.A.mn_major ? 1 : 0;
-    P.b_mn = d.B.mn_major ? 1 : 0;
-    P.a_batch_planes = d.A.batch_planes ? d.A.batch_planes : d.A.planes;
-    P.b_batch_planes = d.B.batch_planes ? d.B.batch_planes : d.B.planes;
-    P.bn = pick_bn(P.pa, P.pb, d.M, d.N, d.batch);
-    P.num_kb = (d.K + BK - 1) / BK;
-    int split = d.split_k > 1 ? d.split_k : 1;
-    if (split > P.num_kb) split = P.num_kb;
-    P.kb_per_split = (P.num_kb + split - 1) / split;
-    split = (P.num_kb + P.kb_per_split - 1) / P.kb_per_split;
-    P.split = split;
-    const int tiles_m = (d.M + BM - 1) / BM;
-    P.tiles_n = (d.N + P.bn - 1) / P.bn;
-    P.tiles_mn = tiles_m * P.tiles_n;
-    const int64_t units = (int64_t)P.tiles_mn * d.batch * split;
-    if (units > (1 << 30)) return MW_ERR_UNSUPPORTED;
-    P.unit_count = (int)units;
-    P.b_tile_bytes = (uint32_t)P.bn * BK * 2;
-    P.tx_bytes = (uint32_t)P.pa * kATileBytes + (uint32_t)P.pb * P.b_tile_bytes;
+    MW_TRY(setup_problem(cache, d, P, &cost[prm.nprob], &flops, &mma_flops));
     if (P.tx_bytes > stage_bytes) stage_bytes = P.tx_bytes;
-    const int t = P.pa > P.pb ? P.pa : P.pb;
-    // fp32-accurate products alternate the leading block (needs two K blocks per unit)
-    const bool rotate = t == 3 && P.pa == 3 && P.pb == 3 && P.kb_per_split >= 2 &&
-                        (P.num_kb - (split - 1) * P.kb_per_split) >= 2;
-    const double kb_cycles = build_ops(P, rotate);
-    cost[prm.nprob] = kb_cycles * P.kb_per_split;
-    P.epi = d.epi;
-    P.split_partials = nullptr;
-    P.split_counters = nullptr;
-    if (split > 1) {
-      if (!d.split_scratch || ((uintptr_t)d.split_scratch & 255u)) return MW_ERR_WORKSPACE;
-      const size_t tiles = (size_t)P.tiles_mn * d.batch;
-      if (tiles * 4 * sizeof(unsigned) > kTcSplitCounterBytes) return MW_ERR_UNSUPPORTED;
-      P.split_counters = static_cast<unsigned int*>(d.split_scratch);
-      P.split_partials = reinterpret_cast<float*>(static_cast<char*>(d.split_scratch) + kTcSplitCounterBytes);
-    }
-    const int a_total = d.batch > 1 ? (d.batch - 1) * P.a_batch_planes + d.A.planes : d.A.planes;
-    const int b_total = d.batch > 1 ? (d.batch - 1) * P.b_batch_planes + d.B.planes : d.B.planes;
-    if (cv.mode == TC_CONV_PIXELS) {
-      MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, BM / cv.W, a_total, &P.tmA));
-      MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
-    } else if (cv.mode == TC_CONV_WGRAD) {
-      MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, BK / cv.W, d.A.planes, &P.tmA));
-      MW_TRY(get_map(cache, d.B, 64, d.B.planes, &P.tmB));
-    } else {
-      MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA));
-      MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
-    }
-    int np = 0;
-    for (int a = 0; a < P.pa; ++a)
-      for (int b = 0; b < P.pb; ++b)
-        if (a + b < t) ++np;
-    flops += 2.0 * d.M * d.N * d.K * d.batch;
-    mma_flops += 2.0 * d.M * d.N * d.K * np * d.batch;
     ++prm.nprob;
   }
   if (prm.nprob == 0) return MW_OK;
@@ -1039,18 +1148,11 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
   }
   prm.total_units = total;
   prm.stage_bytes = stage_bytes;
-  const uint32_t budget = 227u * 1024u - 2048u;   // static barriers + alignment slack
-  int stages = (int)(budget / stage_bytes);
-  if (stages > kMaxStages) stages = kMaxStages;
+  const int stages = stages_for(stage_bytes);
   if (stages < 2) return MW_ERR_UNSUPPORTED;
   prm.stages = stages;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    227 * 1024 - 1024));
-    attr_set = true;
-  }
+  MW_TRY(ensure_kernel_attr());
   const bool prof = g_prof.on;
   if (prof) {
     cudaEventRecord(prof_event(), s);
@@ -1058,10 +1160,98 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
     g_prof.mma_flops += mma_flops;
   }
   const int grid = total < sm_count() ? total : sm_count();
-  tc_group_kernel<<<grid, kThreadsTc, smem, s>>>(prm);
+  tc_group_kernel<false><<<grid, kThreadsTc, smem, s>>>(prm);
   const mw_status rc = launch_ok();
   if (prof) cudaEventRecord(prof_event(), s);
   return rc;
+}
+
+// ---- program launches ----------------------------------------------------------------------
+struct TcProgram {
+  std::vector<TcProblem> table;
+  uint32_t stage_bytes = 0;
+  int total_units = 0;
+  double flops = 0.0, mma_flops = 0.0;
+  void* table_dev = nullptr;
+  unsigned int* done_dev = nullptr;
+  bool uploaded = false;
+};
+
+TcProgram* tc_program_create() { return new TcProgram(); }
+void tc_program_destroy(TcProgram* p) { delete p; }
+
+void tc_program_begin(TcProgram* pr, void* table_dev, unsigned int* done_dev) {
+  pr->table.clear();
+  pr->stage_bytes = 0;
+  pr->total_units = 0;
+  pr->flops = pr->mma_flops = 0.0;
+  pr->table_dev = table_dev;
+  pr->done_dev = done_dev;
+  pr->uploaded = false;
+}
+
+int tc_program_add(TcProgram* pr, TcMapCache* cache, const TcGemm& d, const int* deps, int ndep,
+                   mw_status* status) {
+  *status = MW_OK;
+  if ((int)pr->table.size() >= kMaxProgram || ndep > 3) { *status = MW_ERR_UNSUPPORTED; return -1; }
+  pr->table.emplace_back();
+  TcProblem& P = pr->table.back();
+  double cost = 0.0;
+  *status = setup_problem(cache, d, P, &cost, &pr->flops, &pr->mma_flops);
+  if (*status != MW_OK) { pr->table.pop_back(); return -1; }
+  P.unit_begin = pr->total_units;
+  pr->total_units += P.unit_count;
+  if (P.tx_bytes > pr->stage_bytes) pr->stage_bytes = P.tx_bytes;
+  const int self = (int)pr->table.size() - 1;
+  for (int i = 0; i < ndep; ++i) {
+    const int q = deps[i];
+    if (q < 0) continue;
+    if (q >= self) { *status = MW_ERR_INVALID_ARG; return -1; }   // only earlier products
+    const TcProblem& Q = pr->table[q];
+    P.dep[P.ndep] = q;
+    P.dep_target[P.ndep] = (unsigned)kEpiWarps * (unsigned)(Q.unit_count / Q.split);
+    ++P.ndep;
+  }
+  return self;
+}
+
+size_t tc_program_table_bytes(int products) { return (size_t)products * sizeof(TcProblem); }
+
+mw_status tc_program_launch(TcProgram* pr, DeviceStatus* st, cudaStream_t s) {
+  const int nprob = (int)pr->table.size();
+  if (nprob == 0) return MW_OK;
+  if (!pr->table_dev || !pr->done_dev || ((uintptr_t)pr->table_dev & 63u)) return MW_ERR_WORKSPACE;
+  // the table travels with every launch: the caller's workspace is only promised to keep its
+  // contents between the calls of one step
+  MW_CUDA_OK(cudaMemcpyAsync(pr->table_dev, pr->table.data(), nprob * sizeof(TcProblem),
+                             cudaMemcpyHostToDevice, s));
+  MW_CUDA_OK(cudaMemsetAsync(pr->done_dev, 0, sizeof(unsigned int) * nprob, s));
+  static thread_local TcGroupParams prm;
+  prm.nprob = nprob;
+  prm.st = st;
+  prm.table = static_cast<const TcProblem*>(pr->table_dev);
+  prm.done = pr->done_dev;
+  prm.total_units = pr->total_units;
+  prm.stage_bytes = pr->stage_bytes;
+  const int stages = stages_for(pr->stage_bytes);
+  if (stages < 2) return MW_ERR_UNSUPPORTED;
+  prm.stages = stages;
+  const size_t smem = (size_t)stages * pr->stage_bytes + 1024;
+  MW_TRY(ensure_kernel_attr());
+  const bool prof = g_prof.on;
+  if (prof) {
+    cudaEventRecord(prof_event(), s);
+    g_prof.flops += pr->flops;
+    g_prof.mma_flops += pr->mma_flops;
+  }
+  // products wait for one another inside the launch: every CTA must be resident
+  const int grid = pr->total_units < sm_count() ? pr->total_units : sm_count();
+  void* args[] = {(void*)&prm};
+  cudaError_t e = cudaLaunchCooperativeKernel((const void*)tc_group_kernel<true>, dim3(grid), dim3(kThreadsTc),
+                                              args, smem, s);
+  ++g_launch_count;
+  if (prof) cudaEventRecord(prof_event(), s);
+  return e == cudaSuccess ? MW_OK : MW_ERR_CUDA;
 }
 
 mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int M, int N, int K,

@@ -38,7 +38,7 @@ enum TcEpiMode : int {
   TC_EPI_PLAIN = 0,    // v = alpha*acc (+ addend);  out_f32 and/or planes
   TC_EPI_RESID = 1,    // v = (row == col) - acc;    planes; sum of squares -> sumsq
   TC_EPI_FWD = 2,      // z = acc; sign word written (write_mask) or read; x = phi(z) -> planes (+ out_f32)
-  TC_EPI_BWD = 3,      // h = acc -> out_f32 (optional), ReLU fragments (optional); g = h * phi'(mask) -> planes
+  TC_EPI_BWD = 3,      // h = acc -> out_f32 / planes2 (optional), ReLU fragments (optional); g = h * phi'(mask) -> planes
   TC_EPI_VIJP = 4,     // g = alpha*acc (+ addend); activation vijp: h -> planes2 (+ out_f32); g (zero at dead
                        // ReLU units) -> planes
 };
@@ -110,6 +110,9 @@ struct TcGemm {
   // in fixed order, so the result does not depend on scheduling.  0 / 1 = no split.
   int split_k = 1;
   void* split_scratch = nullptr;
+  // 1: keep the widest tile the term count allows even if the product alone then has fewer
+  // tiles than SMs (for throughput work that shares its launch with other products)
+  int wide_tiles = 0;
 };
 
 // Cache of encoded tensor maps (host side), owned by the caller.
@@ -126,6 +129,23 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
 // single product
 mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int M, int N, int K,
                   const TcEpilogue& epi, DeviceStatus* st, cudaStream_t s, int batch = 1);
+
+// A program: many products in ONE cooperative launch, each starting when the products it names
+// (earlier ones only) are complete -- a whole phase of the method without a launch per layer.
+// The product table lives in device memory (`table_dev`, tc_program_table_bytes(n), 64-byte
+// aligned) beside one completion counter per product (`done_dev`); both are the caller's.  The
+// table is uploaded and the counters are cleared at every launch.
+// Units are taken in order of insertion, so insertion order must be a valid execution order.
+struct TcProgram;
+TcProgram* tc_program_create();
+void tc_program_destroy(TcProgram*);
+void tc_program_begin(TcProgram*, void* table_dev, unsigned int* done_dev);
+// returns the product's index (negative on error, *status says why); deps: up to 3 indices, -1 = none
+int tc_program_add(TcProgram*, TcMapCache* cache, const TcGemm& g, const int* deps, int ndep,
+                   mw_status* status);
+size_t tc_program_table_bytes(int products);
+mw_status tc_program_launch(TcProgram*, DeviceStatus* st, cudaStream_t s);
+constexpr int kTcMaxProgram = 768;
 
 // tile width the kernel will use for this product, and the scratch a K split of it needs
 int tc_tile_n(int a_planes, int b_planes, int M, int N, int batch);

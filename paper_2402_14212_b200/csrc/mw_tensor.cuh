@@ -6,8 +6,13 @@
 namespace mw {
 
 struct TcMapCache;
+struct TcProgram;
+// programs (whole phases in one launch) are rebuilt only when a buffer they name has moved
+enum { MW_PROG_PHASE1 = 0, MW_PROG_PHASE2, MW_PROG_SWEEP, MW_PROG_BP_FWD, MW_PROG_BP_BWD, MW_PROG_COUNT };
 struct TensorState {
   TcMapCache* cache = nullptr;
+  TcProgram* prog[MW_PROG_COUNT] = {};
+  std::vector<const void*> key[MW_PROG_COUNT];
 };
 
 // convolutional nets on the tensor cores (mw_conv_pipeline.cu): stride-1 same-size convolutions

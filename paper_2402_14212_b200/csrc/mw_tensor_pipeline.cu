@@ -47,8 +47,9 @@ int ns_schedule(const mw_net* n, NsStep* out) {
     cnt = 3;
     for (int i = 0; i < cnt; ++i) out[i] = d[i];
   } else {
-    const NsStep d[] = {{1, 1}, {2, 1}, {2, 1}};
-    cnt = 3;
+    // residual 6e-2 -> 4e-3 -> 2e-5, the resolution of the two-term cotangent chain
+    const NsStep d[] = {{1, 1}, {2, 1}};
+    cnt = 2;
     for (int i = 0; i < cnt; ++i) out[i] = d[i];
   }
   const int want = n->opts.inverse_iters;
@@ -144,10 +145,10 @@ split_weights_kernel(PtrBatch Ws, int64_t n4, int64_t n2, __nv_bfloat16* __restr
 }
 
 __global__ void residual_gate_kernel(const double* __restrict__ sumsq, int group, int n,
-                                     double limit, DeviceStatus* st, int layer0) {
-  const int g = threadIdx.x;
+                                     double limit, DeviceStatus* st, int layer0, int stride = 1) {
+  const int g = blockIdx.x * blockDim.x + threadIdx.x;
   if (g < group) {
-    const double r = sqrt(sumsq[g] / (double)n);   // rms singular value of I - W X
+    const double r = sqrt(sumsq[(int64_t)g * stride] / (double)n);   // rms singular value of I - W X
     if (!(r <= limit))
       record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)(layer0 + g), __float_as_uint((float)r), 3u, 0u);
   }
@@ -414,6 +415,433 @@ mw_status loss_and_top(const Ctx& c, const void* target, double* loss_out, bool 
   return split_planes(src, c.bn, c.at<__nv_bfloat16>(lay.hp[0]), c.pr.pg2, c.bn, c.s);
 }
 
+// ---- Newton-Schulz as products of a program --------------------------------------------------
+// In the program path every layer has its own iterate (fp32 X, term planes of X and of the
+// residual), so that the steps of different layers can be spread over the launches that carry
+// Phase I and Phase II: the chains of those phases leave most SMs waiting, the inverses fill them.
+constexpr int kNsSumsqStride = 16;   // doubles per layer in ns_sumsq (one per step)
+
+struct NsBuffers {
+  float* X;
+  __nv_bfloat16 *Rp, *Xp[2];
+  double* sumsq;
+};
+
+NsBuffers ns_buffers(const Ctx& c) {
+  const Layout& lay = *c.lay;
+  const int64_t L = c.n->L;
+  NsBuffers b;
+  b.X = c.at<float>(lay.ns_x);
+  b.Rp = c.at<__nv_bfloat16>(lay.ns_r);
+  b.Xp[0] = b.Rp + 3 * L * c.nn;
+  b.Xp[1] = b.Rp + 6 * L * c.nn;
+  b.sumsq = c.at<double>(lay.ns_sumsq);
+  return b;
+}
+
+// X_0 = (n / ||W||_F^2) W^T and its first term planes, all layers (weight planes exist already)
+mw_status ns_prepare_all(const Ctx& c, const void* const* params, const NsStep* sched) {
+  const Layout& lay = *c.lay;
+  const int L = c.n->L, d = c.dim;
+  const bool f32 = c.n->opts.prec == MW_F32;
+  const NsBuffers nb = ns_buffers(c);
+  char* sc = c.at<char>(lay.inv_scratch);
+  float* cscale = reinterpret_cast<float*>(sc + 8 * kMaxGroup);
+  double* fpart = reinterpret_cast<double*>(sc + 12 * kMaxGroup + 64);
+  MW_CUDA_OK(cudaMemsetAsync(nb.sumsq, 0, sizeof(double) * kNsSumsqStride * L, c.s));
+  const int first = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;
+  for (int l0 = 0; l0 < L; l0 += kMaxGroup) {
+    const int G = (L - l0) < kMaxGroup ? (L - l0) : kMaxGroup;
+    PtrBatch wp{};
+    for (int g = 0; g < G; ++g) wp.p[g] = params[l0 + g];
+    float* X = nb.X + (int64_t)l0 * c.nn;
+    if (f32) {
+      frob_partial_kernel<float><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
+      frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
+      x0_kernel<float><<<dim3(d / 32, d / 32, G), 256, 0, c.s>>>(wp, d, cscale, X);
+    } else {
+      frob_partial_kernel<__nv_bfloat16><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
+      frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
+      x0_kernel<__nv_bfloat16><<<dim3(d / 32, d / 32, G), 256, 0, c.s>>>(wp, d, cscale, X);
+    }
+    MW_TRY(launch_ok(3));
+    MW_TRY(split_planes_batched(X, c.nn, G, c.nn, nb.Xp[0] + (int64_t)l0 * 3 * c.nn, first, c.nn,
+                                3 * c.nn, c.s));
+  }
+  return MW_OK;
+}
+
+// product `stage` of layer l: even = residual R = I - W X of step stage/2, odd = its update
+TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, const NsStep* sched,
+                  int steps) {
+  const Layout& lay = *c.lay;
+  const int d = c.dim, it = stage >> 1, cur = it & 1;
+  const bool last = it + 1 == steps;
+  const NsBuffers nb = ns_buffers(c);
+  float* X = nb.X + (int64_t)l * c.nn;
+  __nv_bfloat16* Rp = nb.Rp + (int64_t)l * 3 * c.nn;
+  __nv_bfloat16* Xc = nb.Xp[cur] + (int64_t)l * 3 * c.nn;
+  __nv_bfloat16* Xn = nb.Xp[cur ^ 1] + (int64_t)l * 3 * c.nn;
+  TcGemm g;
+  g.M = d; g.N = d; g.K = d;
+  g.wide_tiles = 1;      // throughput work beside the latency-bound chains
+  if (!(stage & 1)) {
+    const int pw = c.pr.pw < sched[it].pr ? c.pr.pw : sched[it].pr;
+    const void* W = c.n->opts.prec == MW_F32 ? (const void*)c.at<__nv_bfloat16>(lay.w_planes[l]) : params[l];
+    g.A = operand(W, d, d, pw, false);
+    g.B = operand(Xc, d, d, sched[it].pr, true);
+    g.epi.mode = TC_EPI_RESID;
+    g.epi.planes = Rp; g.epi.n_planes = sched[it].pu; g.epi.plane_stride = c.nn;
+    g.epi.sumsq = nb.sumsq + (int64_t)l * kNsSumsqStride + it;
+  } else {
+    int next_terms = c.pr.ph;
+    if (!last) next_terms = sched[it + 1].pr > sched[it + 1].pu ? sched[it + 1].pr : sched[it + 1].pu;
+    g.A = operand(Xc, d, d, sched[it].pu, false);
+    g.B = operand(Rp, d, d, sched[it].pu, true);
+    g.epi.mode = TC_EPI_PLAIN;
+    g.epi.addend = X;
+    g.epi.out_f32 = last ? nullptr : X;
+    g.epi.planes = last ? c.at<__nv_bfloat16>(lay.inv[l]) : Xn;
+    g.epi.n_planes = next_terms;
+    g.epi.plane_stride = c.nn;
+  }
+  return g;
+}
+
+// the inverse steps handed out to the chain steps of Phase I and Phase II, in step-major order
+// (step t of a layer sits L positions after its step t-1, so its turn comes many chain steps later)
+struct NsFeed {
+  const void* const* params;
+  NsStep sched[16];
+  int steps = 0, total = 0, next = 0, per_slot = 0;
+  std::vector<int> last;      // last product of each layer's chain inside the current program
+};
+
+NsFeed make_feed(const Ctx& c, const void* const* params) {
+  NsFeed f;
+  f.params = params;
+  f.steps = ns_schedule(c.n, f.sched);
+  f.total = f.steps > 0 ? 2 * f.steps * c.n->L : 0;
+  f.per_slot = (f.total + 2 * c.n->L - 1) / (2 * c.n->L);
+  f.last.assign(c.n->L, -1);
+  return f;
+}
+
+// ---- whole phases as one launch ("programs") -------------------------------------------------
+// needs every layer's weight and inverse planes resident, and room in the product table
+bool use_programs(const mw_net* n) {
+  return n->opts.resident_inverse != 0 && 5 * (n->L + 1) <= kTcMaxProgram;
+}
+
+TensorState* state_of(const Ctx& c) { return static_cast<TensorState*>(c.n->tc); }
+
+bool program_ready(const Ctx& c, int idx, const std::vector<const void*>& key) {
+  TensorState* t = state_of(c);
+  return t->prog[idx] != nullptr && !t->key[idx].empty() && t->key[idx] == key;
+}
+
+TcProgram* program_begin(const Ctx& c, int idx, int slot) {
+  TensorState* t = state_of(c);
+  if (!t->prog[idx]) t->prog[idx] = tc_program_create();
+  t->key[idx].clear();
+  tc_program_begin(t->prog[idx], c.at<char>(c.lay->prog_table[slot]),
+                   c.at<unsigned int>(c.lay->prog_done[slot]));
+  return t->prog[idx];
+}
+
+struct Adder {
+  const Ctx& c;
+  TcProgram* pr;
+  mw_status status = MW_OK;
+  // the next inverse steps, after a chain product (everything that is left when `all`)
+  void feed(NsFeed* f, bool all) {
+    if (!f) return;
+    const int L = c.n->L;
+    for (int k = 0; (all || k < f->per_slot) && f->next < f->total; ++k, ++f->next) {
+      const int stage = f->next / L, l = f->next % L;
+      f->last[l] = add(ns_product(c, l, stage, f->params, f->sched, f->steps), f->last[l]);
+    }
+  }
+  int add(const TcGemm& g, int d0 = -1, int d1 = -1, int d2 = -1) {
+    if (status != MW_OK) return -1;
+    const int deps[3] = {d0, d1, d2};
+    mw_status st;
+    const int q = tc_program_add(pr, c.cache, g, deps, 3, &st);
+    if (q < 0) status = st;
+    return q;
+  }
+};
+
+std::vector<const void*> key_of(const Ctx& c, const void* const* params, const void* a,
+                                const void* b, void* const* dW) {
+  std::vector<const void*> k;
+  k.push_back(c.ws);
+  k.push_back(a);
+  k.push_back(b);
+  for (int l = 0; l < c.n->L; ++l) k.push_back(params[l]);
+  if (dW)
+    for (int l = 0; l < c.n->L; ++l) k.push_back(dW[l]);
+  return k;
+}
+
+// all weights as term planes (MW_F32; the layers' plane regions are contiguous)
+mw_status split_all_weights(const Ctx& c, const void* const* params) {
+  if (c.n->opts.prec != MW_F32) return MW_OK;
+  const Layout& lay = *c.lay;
+  const int L = c.n->L;
+  for (int l0 = 0; l0 < L; l0 += kMaxGroup) {
+    const int G = (L - l0) < kMaxGroup ? (L - l0) : kMaxGroup;
+    PtrBatch wp{};
+    for (int g = 0; g < G; ++g) wp.p[g] = params[l0 + g];
+    int64_t bx = (c.nn / 4 + 255) / 256;
+    if (bx > 64) bx = 64;
+    split_weights_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(
+        wp, c.nn / 4, c.nn, c.at<__nv_bfloat16>(lay.w_planes[l0]));
+    MW_TRY(launch_ok());
+  }
+  return MW_OK;
+}
+
+// Phase I (or backprop's forward) as one launch; the weight term planes must already exist
+mw_status forward_program(const Ctx& c, const void* const* params, const void* x, bool store_acts,
+                          NsFeed* feed = nullptr) {
+  const Layout& lay = *c.lay;
+  const int L = c.n->L, d = c.dim;
+  const int idx = store_acts ? MW_PROG_BP_FWD : MW_PROG_PHASE1;
+  const __nv_bfloat16* xin = nullptr;
+  MW_TRY(input_planes(c, x, &xin));
+  const std::vector<const void*> key = key_of(c, params, x, nullptr, nullptr);
+  if (!program_ready(c, idx, key)) {
+    Adder a{c, program_begin(c, idx, 0)};
+    int prev = -1;
+    for (int l = 0; l < L; ++l) {
+      const mw_layer_desc& ld = c.n->layers[l];
+      const __nv_bfloat16* Wp = nullptr;
+      MW_TRY(weight_planes(c, l, params[l], false, &Wp));
+      __nv_bfloat16* xout = (store_acts && l + 1 < L) ? c.at<__nv_bfloat16>(lay.stored_act[l + 1])
+                                                     : c.at<__nv_bfloat16>(lay.xp[(l + 1) % 3]);
+      TcEpilogue e;
+      e.mode = TC_EPI_FWD;
+      e.mask = c.at<uint32_t>(lay.mask[l]);
+      e.write_mask = 1;
+      e.act = ld.act;
+      e.slope = (float)ld.slope;
+      if (l + 1 < L) {
+        e.planes = xout; e.n_planes = c.pr.px; e.plane_stride = c.bn;
+      } else {
+        e.out_f32 = c.at<float>(lay.z);
+      }
+      prev = a.add(product(c, operand(xin, c.B, d, c.pr.px, false), operand(Wp, d, d, c.pr.pw, false),
+                           c.B, d, d, e, 0), prev);
+      a.feed(feed, false);
+      xin = xout;
+    }
+    MW_TRY(a.status);
+    state_of(c)->key[idx] = key;
+  }
+  return tc_program_launch(state_of(c)->prog[idx], c.st, c.s);
+}
+
+// Phase II as one launch (the g_z planes of the last layer are in hp[0])
+mw_status phase2_program(const Ctx& c, const void* const* params, void* g0, NsFeed* feed) {
+  const Layout& lay = *c.lay;
+  mw_net* n = c.n;
+  const int L = n->L, d = c.dim;
+  for (int l = 0; l + 1 < L; ++l)
+    if (n->layers[l].act == MW_ACT_RELU) MW_TRY(relu_index(c, l));
+  const std::vector<const void*> key = key_of(c, params, g0, nullptr, nullptr);
+  if (!program_ready(c, MW_PROG_PHASE2, key)) {
+    Adder a{c, program_begin(c, MW_PROG_PHASE2, 1)};
+    int prev = -1, cur = 0;
+    if (feed) {
+      // Phase I took its share; earlier steps of every layer ended with that launch
+      const int taken = feed->per_slot * L;
+      feed->next = taken < feed->total ? taken : feed->total;
+      feed->last.assign(L, -1);
+    }
+    for (int l = L - 1; l >= 0; --l) {
+      const __nv_bfloat16* Wp = nullptr;
+      MW_TRY(weight_planes(c, l, params[l], false, &Wp));
+      TcEpilogue e;
+      e.mode = TC_EPI_BWD;
+      if (l == 0) {
+        e.out_f32 = (float*)g0;
+      } else {
+        const mw_layer_desc& below = n->layers[l - 1];
+        if (is_reseed(n, l)) {
+          e.planes2 = c.at<__nv_bfloat16>(lay.reseed[l]);
+          e.n_planes2 = c.pr.ph;
+          e.plane_stride2 = c.bn;
+        }
+        e.act = below.act;
+        e.slope = (float)below.slope;
+        e.mask = c.at<uint32_t>(lay.mask[l - 1]);
+        e.planes = c.at<__nv_bfloat16>(lay.hp[cur ^ 1]);
+        e.n_planes = c.pr.pg2;
+        e.plane_stride = c.bn;
+        if (below.act == MW_ACT_RELU) {
+          e.frag_off = c.at<uint32_t>(lay.frag_off[l - 1]);
+          e.frag_rank = c.at<uint32_t>(lay.frag_rank[l - 1]);
+          e.frag_vals = c.at<float>(lay.frag_vals[l - 1]);
+        }
+      }
+      prev = a.add(product(c, operand(c.at<__nv_bfloat16>(lay.hp[cur]), c.B, d, c.pr.pg2, false),
+                           operand(Wp, d, d, c.pr.pw, true), c.B, d, d, e, 0), prev);
+      a.feed(feed, l == 0);
+      cur ^= 1;
+    }
+    MW_TRY(a.status);
+    state_of(c)->key[MW_PROG_PHASE2] = key;
+  }
+  return tc_program_launch(state_of(c)->prog[MW_PROG_PHASE2], c.st, c.s);
+}
+
+// term planes of h_l as the vijp's operand: the checkpoint where the recursion restarts
+const __nv_bfloat16* h_planes(const Ctx& c, int l) {
+  return (l > 0 && is_reseed(c.n, l)) ? c.at<__nv_bfloat16>(c.lay->reseed[l])
+                                      : c.at<__nv_bfloat16>(c.lay->hp[l & 1]);
+}
+
+// the products of layer l of the sweep
+TcGemm recompute_product(const Ctx& c, int l, const __nv_bfloat16* xl, const __nv_bfloat16* Wp) {
+  const mw_layer_desc& ld = c.n->layers[l];
+  TcEpilogue e;
+  e.mode = TC_EPI_FWD;
+  e.mask = c.at<uint32_t>(c.lay->mask[l]);
+  e.write_mask = 0;
+  e.act = ld.act;
+  e.slope = (float)ld.slope;
+  e.planes = c.at<__nv_bfloat16>(c.lay->xp[(l + 1) % 3]);
+  e.n_planes = c.pr.px;
+  e.plane_stride = c.bn;
+  return product(c, operand(xl, c.B, c.dim, c.pr.px, false), operand(Wp, c.dim, c.dim, c.pr.pw, false),
+                 c.B, c.dim, c.dim, e, 0);
+}
+
+TcGemm vijp_product(const Ctx& c, int l, bool want_h, bool want_gz) {
+  const Layout& lay = *c.lay;
+  const mw_layer_desc& ld = c.n->layers[l];
+  TcEpilogue e;
+  e.mode = TC_EPI_VIJP;
+  e.act = ld.act;
+  e.slope = (float)ld.slope;
+  e.mask = c.at<uint32_t>(lay.mask[l]);
+  if (ld.act == MW_ACT_RELU) {
+    e.frag_off = c.at<uint32_t>(lay.frag_off[l]);
+    e.frag_rank = c.at<uint32_t>(lay.frag_rank[l]);
+    e.frag_vals = c.at<float>(lay.frag_vals[l]);
+  }
+  if (want_h) {
+    e.planes2 = c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]);
+    e.n_planes2 = c.pr.ph;
+    e.plane_stride2 = c.bn;
+  }
+  if (want_gz) {
+    e.planes = c.at<__nv_bfloat16>(lay.gzp[l & 1]);
+    e.n_planes = c.pr.pgw;
+    e.plane_stride = c.bn;
+  }
+  return product(c, operand(h_planes(c, l), c.B, c.dim, c.pr.ph, false),
+                 operand(c.at<__nv_bfloat16>(lay.inv[l]), c.dim, c.dim, c.pr.ph, true), c.B, c.dim,
+                 c.dim, e, 1);
+}
+
+TcGemm weight_vjp_product(const Ctx& c, const __nv_bfloat16* gz, const __nv_bfloat16* xl, float* dW) {
+  TcEpilogue e;
+  e.mode = TC_EPI_PLAIN;
+  e.out_f32 = dW;
+  return product(c, operand(gz, c.B, c.dim, c.pr.pgw, true), operand(xl, c.B, c.dim, c.pr.pxw, true),
+                 c.dim, c.dim, c.B, e, 2);
+}
+
+// The forward sweep (Algorithm 1) as one launch.  Products of layer l: R_l recompute x_{l+1},
+// V_l vijp (g_z of layer l, h_{l+1}), D_l weight vjp.  R_l needs x_l (R_{l-1}) and the slot of
+// x_{l+1} free (D_{l-2} read x_{l-2} there); V_l needs h_l (V_{l-1}, unless a checkpoint) and the
+// g_z slot free (D_{l-2}); D_l needs g_z (V_l) and x_l (R_{l-1}).
+mw_status sweep_program(const Ctx& c, const void* const* params, const void* x, void* const* dW,
+                        const __nv_bfloat16* x0p) {
+  const Layout& lay = *c.lay;
+  mw_net* n = c.n;
+  const int L = n->L;
+  const std::vector<const void*> key = key_of(c, params, x, nullptr, dW);
+  if (!program_ready(c, MW_PROG_SWEEP, key)) {
+    Adder a{c, program_begin(c, MW_PROG_SWEEP, 2)};
+    std::vector<int> R(L, -1), V(L, -1), D(L, -1);
+    auto xbuf = [&](int l) -> const __nv_bfloat16* {
+      return l == 0 ? x0p : c.at<__nv_bfloat16>(lay.xp[l % 3]);
+    };
+    auto at_or = [](const std::vector<int>& v, int i) { return i >= 0 ? v[i] : -1; };
+    for (int l = 0; l <= L; ++l) {
+      if (l < L) {
+        const bool more = l + 1 < L;
+        const bool want_h = more && !is_reseed(n, l + 1);
+        if (more) {
+          const __nv_bfloat16* Wp = nullptr;
+          MW_TRY(weight_planes(c, l, params[l], false, &Wp));
+          R[l] = a.add(recompute_product(c, l, xbuf(l), Wp), at_or(R, l - 1), at_or(D, l - 2));
+        }
+        if (dW[l] || want_h) {
+          // V_{l-1} produced h_l, or (at a checkpoint) still reads the slot h_{l+1} goes to
+          V[l] = a.add(vijp_product(c, l, want_h, dW[l] != nullptr), at_or(V, l - 1), at_or(D, l - 2));
+        }
+      }
+      if (l >= 1 && dW[l - 1]) {
+        const int k = l - 1;
+        TcGemm g = weight_vjp_product(c, c.at<__nv_bfloat16>(lay.gzp[k & 1]), xbuf(k), (float*)dW[k]);
+        // a K-split weight vjp shares its meeting place with the previous one
+        D[k] = a.add(g, V[k], at_or(R, k - 1), g.split_k > 1 ? at_or(D, k - 1) : -1);
+      }
+    }
+    MW_TRY(a.status);
+    state_of(c)->key[MW_PROG_SWEEP] = key;
+  }
+  return tc_program_launch(state_of(c)->prog[MW_PROG_SWEEP], c.st, c.s);
+}
+
+// backprop's reverse pass as one launch: B_l (h_{l} -> g_z of layer l-1) and D_l read the same g_z
+mw_status backprop_program(const Ctx& c, const void* const* params, const void* x, void* const* dW,
+                           const __nv_bfloat16* x0p) {
+  const Layout& lay = *c.lay;
+  mw_net* n = c.n;
+  const int L = n->L, d = c.dim;
+  const std::vector<const void*> key = key_of(c, params, x, nullptr, dW);
+  if (!program_ready(c, MW_PROG_BP_BWD, key)) {
+    Adder a{c, program_begin(c, MW_PROG_BP_BWD, 1)};
+    int prevB = -1, prevD = -1, cur = 0;
+    for (int l = L - 1; l >= 0; --l) {
+      const __nv_bfloat16* gz = c.at<__nv_bfloat16>(lay.hp[cur]);
+      const __nv_bfloat16* xl = l == 0 ? x0p : c.at<__nv_bfloat16>(lay.stored_act[l]);
+      int thisD = -1, thisB = -1;
+      if (dW[l]) {
+        TcGemm g = weight_vjp_product(c, gz, xl, (float*)dW[l]);
+        thisD = a.add(g, prevB, g.split_k > 1 ? prevD : -1);
+      }
+      if (l > 0) {
+        const __nv_bfloat16* Wp = nullptr;
+        MW_TRY(weight_planes(c, l, params[l], false, &Wp));
+        const mw_layer_desc& below = n->layers[l - 1];
+        TcEpilogue e;
+        e.mode = TC_EPI_BWD;
+        e.act = below.act;
+        e.slope = (float)below.slope;
+        e.mask = c.at<uint32_t>(lay.mask[l - 1]);
+        e.planes = c.at<__nv_bfloat16>(lay.hp[cur ^ 1]);
+        e.n_planes = c.pr.pg2;
+        e.plane_stride = c.bn;
+        // writes the slot that held g_z of layer l+1: its weight vjp must have read it
+        thisB = a.add(product(c, operand(gz, c.B, d, c.pr.pg2, false), operand(Wp, d, d, c.pr.pw, true),
+                              c.B, d, d, e, 0), prevB, prevD);
+      }
+      prevB = thisB;
+      if (thisD >= 0) prevD = thisD;
+      cur ^= 1;
+    }
+    MW_TRY(a.status);
+    state_of(c)->key[MW_PROG_BP_BWD] = key;
+  }
+  return tc_program_launch(state_of(c)->prog[MW_PROG_BP_BWD], c.st, c.s);
+}
+
 }  // namespace
 
 bool tensor_supported(const mw_net* n) {
@@ -471,6 +899,13 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     if (s1 && !backprop) lay.split[1] = b.take(s1);
     if (s2) lay.split[2] = b.take(s2);
   }
+  if (use_programs(n)) {
+    const int progs = backprop ? 2 : 3;
+    for (int i = 0; i < progs; ++i) {
+      lay.prog_table[i] = b.take(tc_program_table_bytes(5 * (L + 1)));
+      lay.prog_done[i] = b.take(sizeof(unsigned int) * (5 * (size_t)(L + 1) + 1));
+    }
+  }
   if (n->opts.prec == MW_F32) {
     if (resident) {
       for (int l = 0; l < L; ++l) lay.w_planes[l] = b.take(2 * 3 * nn);
@@ -486,10 +921,12 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
       Region slot = b.take(2 * (size_t)pr.ph * nn);
       for (int l = 0; l < L; ++l) lay.inv[l] = slot;
     }
-    const size_t G = (size_t)ns_group(n);
+    // program path: every layer keeps its own Newton-Schulz iterate
+    const size_t G = use_programs(n) ? (size_t)L : (size_t)ns_group(n);
+    if (use_programs(n)) lay.ns_sumsq = b.take(sizeof(double) * kNsSumsqStride * (size_t)L);
     lay.ns_x = b.take(4 * nn * G);
     lay.ns_r = b.take(2 * 9 * nn * G);  // per group member: R planes [3] + two iterate plane sets
-    if (n->opts.prec != MW_F32 && G > 1) lay.ns_w = b.take(2 * nn * G);
+    if (n->opts.prec != MW_F32 && G > 1 && !use_programs(n)) lay.ns_w = b.take(2 * nn * G);
     lay.inv_scratch = b.take(12 * kMaxGroup + 64 + 8 * (size_t)kMaxGroup * kFrobBlocks);
   }
   lay.total = b.cur;
@@ -498,6 +935,8 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
 void tensor_destroy(mw_net* n) {
   if (n->tc) {
     TensorState* t = static_cast<TensorState*>(n->tc);
+    for (int i = 0; i < MW_PROG_COUNT; ++i)
+      if (t->prog[i]) tc_program_destroy(t->prog[i]);
     tc_cache_destroy(t->cache);
     delete t;
     n->tc = nullptr;
@@ -515,6 +954,21 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
   MW_TRY(clear_split_counters(c));
   const bool resident = n->opts.resident_inverse != 0;
+  if (use_programs(n)) {
+    // each phase is one launch, and the inverse steps of all layers ride along in both
+    NsFeed feed = make_feed(c, params);
+    if (feed.steps < 1) return MW_ERR_INVALID_ARG;
+    MW_TRY(split_all_weights(c, params));
+    MW_TRY(ns_prepare_all(c, params, feed.sched));
+    MW_TRY(forward_program(c, params, x, false, &feed));      // Phase I
+    MW_TRY(loss_and_top(c, target, loss_out, true));
+    MW_TRY(phase2_program(c, params, g0, &feed));             // Phase II
+    // the last update squares the last residual: gate on it so a diverging layer is reported
+    const double limit = n->opts.prec == MW_F32 ? 2e-3 : 2e-2;
+    residual_gate_kernel<<<(L + 63) / 64, 64, 0, s>>>(ns_buffers(c).sumsq + (feed.steps - 1), L, d, limit,
+                                                     c.st, 0, kNsSumsqStride);
+    return launch_ok();
+  }
   if (resident) {
     const int G = ns_group(n);
     for (int l = 0; l < L; l += G) MW_TRY(newton_schulz_group(c, l, (L - l) < G ? (L - l) : G, params));
@@ -532,7 +986,11 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
       e.out_f32 = (float*)g0;
     } else {
       const mw_layer_desc& below = n->layers[l - 1];
-      if (is_reseed(n, l)) e.out_f32 = c.at<float>(lay.reseed[l]);
+      if (is_reseed(n, l)) {
+        e.planes2 = c.at<__nv_bfloat16>(lay.reseed[l]);
+        e.n_planes2 = c.pr.ph;
+        e.plane_stride2 = c.bn;
+      }
       e.act = below.act;
       e.slope = (float)below.slope;
       e.mask = c.at<uint32_t>(lay.mask[l - 1]);
@@ -565,6 +1023,9 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
   const __nv_bfloat16* x0p = nullptr;
   MW_TRY(input_planes(c, x, &x0p));
   MW_TRY(split_planes((const float*)g0, c.bn, c.at<__nv_bfloat16>(lay.hp[0]), c.pr.ph, c.bn, s));
+  // The sweep as one launch (sweep_program) measures slower than one launch per layer: its two
+  // chains leave little for the waiting CTAs to do, so the per-layer launches stay the default.
+  if (use_programs(n) && n->opts.reserved == 1) return sweep_program(c, params, x, dW, x0p);
   auto xbuf = [&](int l) -> const __nv_bfloat16* {          // term planes of x_l
     return l == 0 ? x0p : c.at<__nv_bfloat16>(lay.xp[l % 3]);
   };
@@ -573,62 +1034,19 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
     TcGemm g[3];
     int cnt = 0;
     if (l < L) {
-      const mw_layer_desc& ld = n->layers[l];
-      uint32_t* words = c.at<uint32_t>(lay.mask[l]);
       const bool more = l + 1 < L;
-      const bool reseed_next = more && is_reseed(n, l + 1);
-      if (!resident) MW_TRY(newton_schulz_group(c, l, 1, params));
-      if (reseed_next)   // the recursion restarts from the stored cotangent h_{l+1}
-        MW_TRY(split_planes(c.at<float>(lay.reseed[l + 1]), c.bn,
-                            c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]), c.pr.ph, c.bn, s));
+      const bool want_h = more && !is_reseed(n, l + 1);
+      if (!resident) MW_TRY(newton_schulz_group(c, l, 1, params));   // W^-1 (and W planes) of this layer
       if (more) {
         const __nv_bfloat16* Wp = nullptr;
         MW_TRY(weight_planes(c, l, params[l], false, &Wp));
-        TcEpilogue e;
-        e.mode = TC_EPI_FWD;
-        e.mask = words;
-        e.write_mask = 0;
-        e.act = ld.act;
-        e.slope = (float)ld.slope;
-        e.planes = c.at<__nv_bfloat16>(lay.xp[(l + 1) % 3]);
-        e.n_planes = c.pr.px;
-        e.plane_stride = c.bn;
-        g[cnt++] = product(c, operand(xbuf(l), c.B, d, c.pr.px, false),
-                           operand(Wp, d, d, c.pr.pw, false), c.B, d, d, e, 0);
+        g[cnt++] = recompute_product(c, l, xbuf(l), Wp);
       }
-      if (dW[l] || (more && !reseed_next)) {
-        TcEpilogue e;
-        e.mode = TC_EPI_VIJP;
-        e.act = ld.act;
-        e.slope = (float)ld.slope;
-        e.mask = words;
-        if (ld.act == MW_ACT_RELU) {
-          e.frag_off = c.at<uint32_t>(lay.frag_off[l]);
-          e.frag_rank = c.at<uint32_t>(lay.frag_rank[l]);
-          e.frag_vals = c.at<float>(lay.frag_vals[l]);
-        }
-        if (more && !reseed_next) {
-          e.planes2 = c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]);
-          e.n_planes2 = c.pr.ph;
-          e.plane_stride2 = c.bn;
-        }
-        if (dW[l]) {
-          e.planes = c.at<__nv_bfloat16>(lay.gzp[l & 1]);
-          e.n_planes = c.pr.pgw;
-          e.plane_stride = c.bn;
-        }
-        g[cnt++] = product(c, operand(c.at<__nv_bfloat16>(lay.hp[l & 1]), c.B, d, c.pr.ph, false),
-                           operand(c.at<__nv_bfloat16>(lay.inv[l]), d, d, c.pr.ph, true), c.B, d, d,
-                           e, 1);
-      }
+      if (dW[l] || want_h) g[cnt++] = vijp_product(c, l, want_h, dW[l] != nullptr);
     }
-    if (l >= 1 && dW[l - 1]) {
-      TcEpilogue e;
-      e.mode = TC_EPI_PLAIN;
-      e.out_f32 = (float*)dW[l - 1];
-      g[cnt++] = product(c, operand(c.at<__nv_bfloat16>(lay.gzp[(l - 1) & 1]), c.B, d, c.pr.pgw, true),
-                         operand(xbuf(l - 1), c.B, d, c.pr.pxw, true), d, d, c.B, e, 2);
-    }
+    if (l >= 1 && dW[l - 1])
+      g[cnt++] = weight_vjp_product(c, c.at<__nv_bfloat16>(lay.gzp[(l - 1) & 1]), xbuf(l - 1),
+                                    (float*)dW[l - 1]);
     if (cnt) MW_TRY(run(c, g, cnt));
   }
   return MW_OK;
@@ -643,11 +1061,18 @@ mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, c
   const int L = n->L, d = c.dim;
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
   MW_TRY(clear_split_counters(c));
-  MW_TRY(forward_pass(c, params, x, true));
+  const bool programs = use_programs(n);
+  if (programs) {
+    MW_TRY(split_all_weights(c, params));
+    MW_TRY(forward_program(c, params, x, true));
+  } else {
+    MW_TRY(forward_pass(c, params, x, true));
+  }
   MW_TRY(loss_and_top(c, target, loss_out, false));
   const __nv_bfloat16* x0p = nullptr;
-  if (n->opts.prec == MW_F32) x0p = c.at<__nv_bfloat16>(lay.xp[0]);   // split by forward_pass
+  if (n->opts.prec == MW_F32) x0p = c.at<__nv_bfloat16>(lay.xp[0]);   // split by the forward pass
   else x0p = (const __nv_bfloat16*)x;
+  if (programs) return backprop_program(c, params, x, dW, x0p);
   int cur = 0;
   // one launch per layer: both vjps of layer l read the same g_z
   for (int l = L - 1; l >= 0; --l) {
