@@ -30,8 +30,10 @@ METRIC = "moonwalk_grad_samples_per_s"
 UNIT = "samples/s"
 NOMINAL_TF32_OVER_BF16 = 1.1 / 2.25      # dense tensor peaks, nominal ratio
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes per launch of the product kernel, from the committed ncu capture (None until measured)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM bytes (read + written) per launch of the product kernel, averaged over the launches of this
+# benchmark's default workload (603 captured launches; profiles/tc_group_kernel_traffic_deep_mlp.md).
+# Other workloads have no capture: their `traffic` is null.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"deep_mlp": 115.6e6}
 
 
 def workload(name: str, seed: int = 0, depth: int = 0):
@@ -190,6 +192,19 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def aggregate_replicas(ms_local: float, batch: int, steps: int, world: int, device=None):
+    """Whole-job throughput of `world` independent replicas: all samples over the slowest rank's
+    time (max over ranks through torch.distributed when world > 1)."""
+    import torch
+    ms_max = float(ms_local)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_max = float(t.item())
+    return batch * steps * world / (ms_max * 1e-3), ms_max
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -244,11 +259,7 @@ def run_ours(args):
     launches = mwb.launch_count() - launches0
     clocks = sampler.stop()
     ms = e0.elapsed_time(e1)
-    t_ms = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    ms_max = float(t_ms.item())
-    value = p.batch * args.steps * world / (ms_max * 1e-3)
+    value, ms_max = aggregate_replicas(ms, p.batch, args.steps, world, dev)
 
     # ---- phase split (device timed, a few extra steps) --------------------------------------
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
@@ -282,10 +293,7 @@ def run_ours(args):
     barrier()
     wall = time.perf_counter() - w0
     ms_e2e = max(e0.elapsed_time(e1), 0.0)
-    t2 = torch.tensor([max(ms_e2e, wall * 1e3)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-    e2e_value = p.batch * args.steps * world / (float(t2.item()) * 1e-3)
+    e2e_value, _ = aggregate_replicas(max(ms_e2e, wall * 1e3), p.batch, args.steps, world, dev)
     h2d = xh.numel() * xh.element_size() + th.numel() * th.element_size()
 
     # ---- roofline of the dominant kernel: per-launch events over the same K steps ------------
@@ -308,9 +316,9 @@ def run_ours(args):
         if prof["launches"]:
             achieved = prof["flops"] / (prof["total_ms"] * 1e-3) / 1e12
             executed = prof["mma_flops"] / (prof["total_ms"] * 1e-3) / 1e12
-            roof = {"bound": "tensor", "kernel": "tc_gemm_kernel (tcgen05, all layouts)",
+            roof = {"bound": "tensor", "kernel": "tc_group_kernel (tcgen05 products: programs and grouped launches)",
                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                    "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_source": peak_note,
+                    "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(p.name), "peak_source": peak_note,
                     "launches_per_step": prof["launches"] / args.steps,
                     "avg_launch_us": 1e3 * prof["total_ms"] / prof["launches"],
                     "algorithmic_flops_per_launch": prof["flops"] / prof["launches"],

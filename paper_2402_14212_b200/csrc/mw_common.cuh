@@ -112,6 +112,12 @@ mw_status gemm_simt(int ta, int tb, int M, int N, int K, double alpha, const T* 
 // Gauss-Jordan inverse with partial pivoting of one n x n matrix, n <= 64, one CTA, fp64 inside.
 template <typename T>
 mw_status inverse_small(const T* W, int n, T* Winv, DeviceStatus* st, int layer, cudaStream_t s);
+// the same for up to kSmallBatch matrices at once (one CTA each): matrix b = Ws.p[b] + offset
+constexpr int kSmallBatch = 32;
+struct SmallBatch { const void* p[kSmallBatch]; };
+template <typename T>
+mw_status inverse_small_batch(const SmallBatch& Ws, int count, int64_t offset, int n, T* Winv,
+                              DeviceStatus* st, int layer0, cudaStream_t s);
 // X <- X (2I - W X) style Newton-Schulz on CUDA cores (any n); scratch >= 2 n^2 elements.
 template <typename T>
 mw_status inverse_newton_simt(const T* W, int n, int iters, T* X, T* scratch, DeviceStatus* st,

@@ -57,30 +57,91 @@ int update_terms(int t, int T) {
   return left < 4 ? 3 : (left < 7 ? 2 : 1);
 }
 
-// w^[tap] = Winv w[tap] for tap != centre, zero at the centre; one block per (tap, row)
+// w^[tap] = Winv w[tap] for tap != centre, zero at the centre; one block per (tap, row, layer)
 __global__ void __launch_bounds__(64)
-fold_kernel(const float* __restrict__ w, const float* __restrict__ winv, int centre,
-            float* __restrict__ what) {
+fold_kernel(SmallBatch ws, const float* __restrict__ winv0, int centre, int64_t we,
+            float* __restrict__ what0) {
   const int tap = blockIdx.x, c = blockIdx.y, cp = threadIdx.x;
+  const float* w = static_cast<const float*>(ws.p[blockIdx.z]);
+  const float* winv = winv0 + (int64_t)blockIdx.z * 4096;
+  float* what = what0 + (int64_t)blockIdx.z * we;
   float a = 0.f;
   if (tap != centre)
     for (int m = 0; m < 64; ++m) a = fmaf(winv[c * 64 + m], w[((int64_t)tap * 64 + m) * 64 + cp], a);
   what[((int64_t)tap * 64 + c) * 64 + cp] = a;
 }
 
-// per-step preparation of layer l: kernel term planes, centre-tap inverse, folded kernel
-mw_status prep_layer(const CCtx& c, int l, const float* w, bool inverse) {
+// per-step preparation of layers [l0, l0 + G): kernel term planes, centre-tap inverses, folded
+// kernels, G <= kSmallBatch layers per launch
+mw_status prep_layers(const CCtx& c, int l0, int G, const void* const* params, bool inverse) {
   const Layout& lay = *c.lay;
-  MW_TRY(split_planes(w, c.we, c.at<__nv_bfloat16>(lay.cw[l]), 3, c.we, c.s));
+  for (int g = 0; g < G; ++g)
+    MW_TRY(split_planes((const float*)params[l0 + g], c.we, c.at<__nv_bfloat16>(lay.cw[l0 + g]), 3, c.we, c.s));
   if (!inverse) return MW_OK;
   const int centre = c.g.pad * c.g.k + c.g.pad;
-  float* winv = c.at<float>(lay.cwinv_f32);
-  float* what = c.at<float>(lay.cwhat_f32);
-  MW_TRY(inverse_small<float>(w + (int64_t)centre * 4096, 64, winv, c.st, l, c.s));
-  fold_kernel<<<dim3(c.g.k * c.g.k, 64), 64, 0, c.s>>>(w, winv, centre, what);
+  float* winv = c.at<float>(lay.cwinv_f32);      // [kSmallBatch][64*64]
+  float* what = c.at<float>(lay.cwhat_f32);      // [kSmallBatch][k*k*64*64]
+  SmallBatch ws{};
+  for (int g = 0; g < G; ++g) ws.p[g] = params[l0 + g];
+  MW_TRY(inverse_small_batch<float>(ws, G, (int64_t)centre * 4096, 64, winv, c.st, l0, c.s));
+  fold_kernel<<<dim3(c.g.k * c.g.k, 64, G), 64, 0, c.s>>>(ws, winv, centre, c.we, what);
   MW_TRY(launch_ok());
-  MW_TRY(split_planes(winv, 4096, c.at<__nv_bfloat16>(lay.cwinv[l]), 3, 4096, c.s));
-  return split_planes(what, c.we, c.at<__nv_bfloat16>(lay.cwhat[l]), 3, c.we, c.s);
+  for (int g = 0; g < G; ++g) {
+    MW_TRY(split_planes(winv + (int64_t)g * 4096, 4096, c.at<__nv_bfloat16>(lay.cwinv[l0 + g]), 3, 4096, c.s));
+    MW_TRY(split_planes(what + (int64_t)g * c.we, c.we, c.at<__nv_bfloat16>(lay.cwhat[l0 + g]), 3, c.we, c.s));
+  }
+  return MW_OK;
+}
+
+mw_status prep_layer(const CCtx& c, int l, const void* const* params, bool inverse) {
+  return prep_layers(c, l, 1, params, inverse);
+}
+
+// ---- the linear head (a few outputs over a very long row) on CUDA cores -------------------
+// logits[b][o] = sum_k x[b][k] W[o][k]: one CTA per (o, b)
+__global__ void __launch_bounds__(256)
+head_forward_kernel(const float* __restrict__ x, const float* __restrict__ W, int64_t nf, int no,
+                    float* __restrict__ logits) {
+  __shared__ float red[256];
+  const int o = blockIdx.x, b = blockIdx.y;
+  const float4* xr = reinterpret_cast<const float4*>(x + (int64_t)b * nf);
+  const float4* wr = reinterpret_cast<const float4*>(W + (int64_t)o * nf);
+  float a = 0.f;
+  for (int64_t i = threadIdx.x; i < nf / 4; i += 256) {
+    const float4 u = xr[i], v = wr[i];
+    a = fmaf(u.x, v.x, fmaf(u.y, v.y, fmaf(u.z, v.z, fmaf(u.w, v.w, a))));
+  }
+  red[threadIdx.x] = a;
+  __syncthreads();
+  for (int s = 128; s; s >>= 1) {
+    if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) logits[(int64_t)b * no + o] = red[0];
+}
+
+// h[b][k] = sum_o hl[b][o] W[o][k]
+__global__ void __launch_bounds__(256)
+head_backward_kernel(const float* __restrict__ hl, const float* __restrict__ W, int64_t nf, int no,
+                     float* __restrict__ h) {
+  const int b = blockIdx.y;
+  const int64_t k = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (k >= nf) return;
+  float a = 0.f;
+  for (int o = 0; o < no; ++o) a = fmaf(hl[(int64_t)b * no + o], W[(int64_t)o * nf + k], a);
+  h[(int64_t)b * nf + k] = a;
+}
+
+// dW[o][k] = sum_b hl[b][o] x[b][k]
+__global__ void __launch_bounds__(256)
+head_wgrad_kernel(const float* __restrict__ hl, const float* __restrict__ x, int64_t nf, int no, int B,
+                  float* __restrict__ dW) {
+  const int o = blockIdx.y;
+  const int64_t k = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (k >= nf) return;
+  float a = 0.f;
+  for (int b = 0; b < B; ++b) a = fmaf(hl[(int64_t)b * no + o], x[(int64_t)b * nf + k], a);
+  dW[(int64_t)o * nf + k] = a;
 }
 
 // Phase I (or backprop's forward).  x_{l+1} planes go to the stores (backprop) or rotate; the
@@ -89,9 +150,11 @@ mw_status conv_forward_pass(const CCtx& c, const void* const* params, const void
   const Layout& lay = *c.lay;
   MW_TRY(split_planes((const float*)x, c.P, c.at<__nv_bfloat16>(lay.xp[0]), 3, c.P, c.s));
   const __nv_bfloat16* xin = c.at<__nv_bfloat16>(lay.xp[0]);
+  for (int l0 = 0; l0 < c.Lc; l0 += kSmallBatch)
+    MW_TRY(prep_layers(c, l0, (c.Lc - l0) < kSmallBatch ? (c.Lc - l0) : kSmallBatch, params,
+                       !store_acts && c.n->opts.resident_inverse));
   for (int l = 0; l < c.Lc; ++l) {
     const mw_layer_desc& ld = c.n->layers[l];
-    MW_TRY(prep_layer(c, l, (const float*)params[l], !store_acts && c.n->opts.resident_inverse));
     const bool last = l + 1 == c.Lc;
     __nv_bfloat16* xout = (store_acts && l + 1 < c.n->L) ? c.at<__nv_bfloat16>(lay.stored_act[l + 1])
                                                         : c.at<__nv_bfloat16>(lay.xp[(l + 1) % 3]);
@@ -122,15 +185,18 @@ mw_status conv_loss_top(const CCtx& c, const void* const* params, const void* ta
     const mw_layer_desc& hd = c.n->layers[L - 1];
     float* logits = c.at<float>(lay.clogits);
     float* hl = logits + (int64_t)c.n->B * hd.n_out;
-    MW_TRY(gemm_simt<float>(0, 1, c.n->B, hd.n_out, hd.n_in, 1.0, xf, hd.n_in, (const float*)params[L - 1],
-                            hd.n_in, 0.0, logits, hd.n_out, c.s));
+    if (hd.n_in % 4 != 0) return MW_ERR_UNSUPPORTED;
+    head_forward_kernel<<<dim3(hd.n_out, c.n->B), 256, 0, c.s>>>(xf, (const float*)params[L - 1], hd.n_in,
+                                                               hd.n_out, logits);
+    MW_TRY(launch_ok());
     MW_TRY(loss_cotangent<float>(logits, target, c.n->B, hd.n_out, c.n->opts.loss, hl,
                                  c.at<double>(lay.partials), loss_out, c.s));
     if (keep_head_cotangent)
       MW_CUDA_OK(cudaMemcpyAsync(c.at<float>(lay.h_last), hl, sizeof(float) * c.n->B * hd.n_out,
                                  cudaMemcpyDeviceToDevice, c.s));
-    MW_TRY(gemm_simt<float>(0, 0, c.n->B, hd.n_in, hd.n_out, 1.0, hl, hd.n_out, (const float*)params[L - 1],
-                            hd.n_in, 0.0, h, hd.n_in, c.s));
+    head_backward_kernel<<<dim3((unsigned)((hd.n_in + 255) / 256), c.n->B), 256, 0, c.s>>>(
+        hl, (const float*)params[L - 1], hd.n_in, hd.n_out, h);
+    MW_TRY(launch_ok());
   } else {
     MW_TRY(loss_cotangent<float>(xf, target, c.g.pixels(), 64, c.n->opts.loss, h,
                                  c.at<double>(lay.partials), loss_out, c.s));
@@ -207,8 +273,8 @@ void conv_tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
       lay.cwhat[l] = b.take(2 * 3 * we);
       lay.cwinv[l] = b.take(2 * 3 * 4096);
     }
-    lay.cwinv_f32 = b.take(4 * 4096);
-    lay.cwhat_f32 = b.take(4 * we);
+    lay.cwinv_f32 = b.take(4 * 4096 * (size_t)kSmallBatch);
+    lay.cwhat_f32 = b.take(4 * we * (size_t)kSmallBatch);
   }
   lay.total = b.cur;
 }
@@ -268,7 +334,7 @@ mw_status conv_tensor_forward_sweep(mw_net* n, const void* const* params, const 
     const bool more = l + 1 < Lc;
     const bool reseed_next = (more || c.head) && is_reseed(n, l + 1);
     const bool want_h = more && !reseed_next;
-    if (!resident) MW_TRY(prep_layer(c, l, (const float*)params[l], true));
+    if (!resident) MW_TRY(prep_layer(c, l, params, true));
     // recompute x_{l+1} (the last one in fp32, for the head's weight vjp)
     if (more || (c.head && dW[L - 1])) {
       TcEpilogue e;
@@ -338,8 +404,9 @@ mw_status conv_tensor_forward_sweep(mw_net* n, const void* const* params, const 
   if (c.head && dW[L - 1]) {
     // the head has no vijp: its output cotangent is the loss cotangent itself
     const mw_layer_desc& hd = n->layers[L - 1];
-    MW_TRY(gemm_simt<float>(1, 0, hd.n_out, hd.n_in, n->B, 1.0, c.at<float>(lay.h_last), hd.n_out,
-                            c.at<float>(lay.cxf), hd.n_in, 0.0, (float*)dW[L - 1], hd.n_in, s));
+    head_wgrad_kernel<<<dim3((unsigned)((hd.n_in + 255) / 256), hd.n_out), 256, 0, s>>>(
+        c.at<float>(lay.h_last), c.at<float>(lay.cxf), hd.n_in, hd.n_out, n->B, (float*)dW[L - 1]);
+    MW_TRY(launch_ok());
   }
   return MW_OK;
 }
@@ -356,8 +423,9 @@ mw_status conv_tensor_backprop(mw_net* n, const void* const* params, const void*
   if (c.head && dW[L - 1]) {
     const mw_layer_desc& hd = n->layers[L - 1];
     const float* hl = c.at<float>(lay.clogits) + (int64_t)n->B * hd.n_out;
-    MW_TRY(gemm_simt<float>(1, 0, hd.n_out, hd.n_in, n->B, 1.0, hl, hd.n_out, c.at<float>(lay.cxf),
-                            hd.n_in, 0.0, (float*)dW[L - 1], hd.n_in, s));
+    head_wgrad_kernel<<<dim3((unsigned)((hd.n_in + 255) / 256), hd.n_out), 256, 0, s>>>(
+        hl, c.at<float>(lay.cxf), hd.n_in, hd.n_out, n->B, (float*)dW[L - 1]);
+    MW_TRY(launch_ok());
   }
   MW_TRY(conv_top_gz(c));
   int cur = 0;

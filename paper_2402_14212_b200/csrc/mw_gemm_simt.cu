@@ -86,9 +86,8 @@ mw_status gemm_simt(int ta, int tb, int M, int N, int K, double alpha, const T* 
 // Gauss-Jordan with partial pivoting, one CTA, n <= 64, double arithmetic in shared memory
 // ---------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256)
-inverse_small_kernel(const T* __restrict__ W, int n, T* __restrict__ Winv, DeviceStatus* st,
-                     int layer) {
+__device__ __forceinline__ void inverse_small_body(const T* __restrict__ W, int n, T* __restrict__ Winv,
+                                                   DeviceStatus* st, int layer) {
   extern __shared__ double aug[];  // [n][2n]
   __shared__ int piv_s;
   __shared__ double pval_s;
@@ -138,6 +137,22 @@ inverse_small_kernel(const T* __restrict__ W, int n, T* __restrict__ Winv, Devic
 }
 
 template <typename T>
+__global__ void __launch_bounds__(256)
+inverse_small_kernel(const T* __restrict__ W, int n, T* __restrict__ Winv, DeviceStatus* st,
+                     int layer) {
+  inverse_small_body<T>(W, n, Winv, st, layer);
+}
+
+// one CTA per matrix: matrix b is Ws.p[b] + offset, its inverse lands at Winv + b*n*n
+template <typename T>
+__global__ void __launch_bounds__(256)
+inverse_small_batch_kernel(SmallBatch Ws, int64_t offset, int n, T* __restrict__ Winv,
+                           DeviceStatus* st, int layer0) {
+  inverse_small_body<T>(static_cast<const T*>(Ws.p[blockIdx.x]) + offset, n,
+                        Winv + (int64_t)blockIdx.x * n * n, st, layer0 + (int)blockIdx.x);
+}
+
+template <typename T>
 mw_status inverse_small(const T* W, int n, T* Winv, DeviceStatus* st, int layer, cudaStream_t s) {
   if (n < 1 || n > 64) return MW_ERR_UNSUPPORTED;
   const size_t smem = sizeof(double) * n * 2 * n;
@@ -150,6 +165,23 @@ mw_status inverse_small(const T* W, int n, T* Winv, DeviceStatus* st, int layer,
   inverse_small_kernel<T><<<1, 256, smem, s>>>(W, n, Winv, st, layer);
   return launch_ok();
 }
+
+template <typename T>
+mw_status inverse_small_batch(const SmallBatch& Ws, int count, int64_t offset, int n, T* Winv,
+                              DeviceStatus* st, int layer0, cudaStream_t s) {
+  if (n < 1 || n > 64 || count < 1 || count > kSmallBatch) return MW_ERR_UNSUPPORTED;
+  const size_t smem = sizeof(double) * n * 2 * n;
+  static bool attr_done = false;
+  if (!attr_done) {
+    MW_CUDA_OK(cudaFuncSetAttribute(inverse_small_batch_kernel<T>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
+    attr_done = true;
+  }
+  inverse_small_batch_kernel<T><<<count, 256, smem, s>>>(Ws, offset, n, Winv, st, layer0);
+  return launch_ok();
+}
+template mw_status inverse_small_batch<float>(const SmallBatch&, int, int64_t, int, float*,
+                                              DeviceStatus*, int, cudaStream_t);
 
 // ---------------------------------------------------------------------------------------
 // Newton-Schulz on CUDA cores: X <- 2X - X (W X), X_0 = (n / ||W||_F^2) W^T
