@@ -823,13 +823,14 @@ int sm_count() {
   return n;
 }
 
-// tile width: as wide as the accumulator set allows for the number of term orders, narrowed while
-// the product alone cannot give every SM a tile
+// tile width: as wide as the accumulator set allows for the number of term orders.  Narrower
+// tiles would give a small product more CTAs, but instructions below 128 columns are issue bound
+// (about 57 cycles each whatever their width); a product that needs more CTAs is cut along K.
 int pick_bn(int pa, int pb, int M, int N, int batch, bool wide = false) {
+  (void)M; (void)batch; (void)wide;
   const int t = pa > pb ? pa : pb;
   int bn = t == 1 ? 256 : (t == 2 ? 128 : 64);
-  const int tm = (M + BM - 1) / BM;
-  while (bn > 64 && (N % bn != 0 || (!wide && (int64_t)tm * (N / bn) * batch < sm_count()))) bn >>= 1;
+  while (bn > 64 && N % bn != 0) bn >>= 1;
   return bn;
 }
 
@@ -849,6 +850,8 @@ size_t tc_split_scratch_bytes(int a_planes, int b_planes, int M, int N, int batc
 int tc_auto_split(int a_planes, int b_planes, int M, int N, int K, int batch) {
   const int bn = pick_bn(a_planes, b_planes, M, N, batch);
   const int64_t units = (int64_t)((M + BM - 1) / BM) * ((N + bn - 1) / bn) * batch;
+  // only 64-column tiles are cut: the pieces of a wider tile are too costly to add up
+  if (bn > 64) return 1;
   // as many pieces as keep every piece on an SM of its own, each at least four K blocks deep
   int s = (int)(sm_count() / units);
   const int num_kb = (K + BK - 1) / BK;
