@@ -392,11 +392,66 @@ fragment_row_kernel(const T* __restrict__ src, const uint32_t* __restrict__ word
   }
 }
 
+// float rows of a multiple of 128 columns: one warp per row, 128 columns (four sign words, one
+// float4 per lane) per step, so that a warp keeps several 512-byte requests in flight; a lane's
+// position in the stream = row offset + dead units of the earlier segments and words + dead bits
+// below its nibble
+template <int MODE>
+__global__ void __launch_bounds__(kThreads)
+fragment_row_vec4_kernel(const float* __restrict__ src, const uint32_t* __restrict__ words,
+                         int64_t rows, int cols, const uint32_t* __restrict__ off,
+                         float* __restrict__ vals, float* __restrict__ h_out,
+                         float* __restrict__ gz_out) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp0 = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * kThreads) >> 5;
+  const int nseg = cols >> 7, wpr = cols >> 5;
+  const int wi = lane >> 3;
+  const unsigned sh = 4u * (unsigned)(lane & 7);
+  for (int64_t r = warp0; r < rows; r += nwarps) {
+    uint32_t base = off[r];
+#pragma unroll 4
+    for (int seg = 0; seg < nseg; ++seg) {
+      const int64_t e0 = r * cols + seg * 128 + lane * 4;
+      float4 v = *reinterpret_cast<const float4*>(src + e0);
+      const unsigned dead_w = ~words[r * wpr + seg * 4 + wi];
+      const unsigned c0 = __popc(__shfl_sync(0xffffffffu, dead_w, 0));
+      const unsigned c1 = __popc(__shfl_sync(0xffffffffu, dead_w, 8));
+      const unsigned c2 = __popc(__shfl_sync(0xffffffffu, dead_w, 16));
+      const unsigned c3 = __popc(__shfl_sync(0xffffffffu, dead_w, 24));
+      const unsigned before = (wi > 0 ? c0 : 0u) + (wi > 1 ? c1 : 0u) + (wi > 2 ? c2 : 0u) +
+                              __popc(dead_w & ((1u << sh) - 1u));
+      const unsigned nib = (dead_w >> sh) & 0xFu;
+      uint32_t pos = base + before;
+      if (MODE == 0) {
+        if (nib & 1u) vals[pos++] = v.x;
+        if (nib & 2u) vals[pos++] = v.y;
+        if (nib & 4u) vals[pos++] = v.z;
+        if (nib & 8u) vals[pos++] = v.w;
+      } else {
+        float4 h = v;
+        if (nib & 1u) { h.x = vals[pos++]; v.x = 0.f; }
+        if (nib & 2u) { h.y = vals[pos++]; v.y = 0.f; }
+        if (nib & 4u) { h.z = vals[pos++]; v.z = 0.f; }
+        if (nib & 8u) { h.w = vals[pos++]; v.w = 0.f; }
+        *reinterpret_cast<float4*>(h_out + e0) = h;
+        if (gz_out) *reinterpret_cast<float4*>(gz_out + e0) = v;
+      }
+      base += c0 + c1 + c2 + c3;
+    }
+  }
+}
+
 template <typename T>
 mw_status fragment_compact(const T* h, const uint32_t* words, int64_t rows, int cols,
                            const uint32_t* off, T* vals, cudaStream_t s) {
   if (rows == 0 || cols == 0) return MW_OK;
   const int wpr = (cols + 31) / 32;
+  if (vec_ok<T>(h, h, cols)) {
+    fragment_row_vec4_kernel<0><<<grid_for(rows), kThreads, 0, s>>>(
+        (const float*)h, words, rows, cols, off, (float*)vals, nullptr, nullptr);
+    return launch_ok();
+  }
   fragment_row_kernel<T, 0><<<grid_for(rows), kThreads, 0, s>>>(h, words, rows, cols, wpr, off,
                                                                 vals, nullptr, nullptr);
   return launch_ok();
@@ -410,8 +465,13 @@ mw_status activation_vijp(const T* gz, const uint32_t* words, int64_t rows, int 
   const int wpr = (cols + 31) / 32;
   if (act == MW_ACT_RELU) {
     if (!off || !vals) return MW_ERR_INVALID_ARG;
-    fragment_row_kernel<T, 1><<<grid_for(rows), kThreads, 0, s>>>(
-        gz, words, rows, cols, wpr, off, const_cast<T*>(vals), h_out, gz_out);
+    if (vec_ok<T>(gz, h_out, cols) && (!gz_out || ((uintptr_t)gz_out % 16 == 0)))
+      fragment_row_vec4_kernel<1><<<grid_for(rows), kThreads, 0, s>>>(
+          (const float*)gz, words, rows, cols, off, (float*)const_cast<T*>(vals), (float*)h_out,
+          (float*)gz_out);
+    else
+      fragment_row_kernel<T, 1><<<grid_for(rows), kThreads, 0, s>>>(
+          gz, words, rows, cols, wpr, off, const_cast<T*>(vals), h_out, gz_out);
   } else if (act == MW_ACT_LEAKY_RELU) {
     if (vec_ok<T>(gz, h_out, cols)) {
       const int64_t nseg = rows * (cols / 128);
