@@ -467,6 +467,10 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;  // 1024-byte aligned for the swizzle
+  // Launched with programmatic stream serialisation, this grid may start while the previous
+  // kernel of the stream is still finishing: everything up to the waits below (barriers, tensor
+  // memory, tensor-map prefetch) then overlaps that kernel's tail.  Let the next one do the same.
+  if (!kProgram) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const TcProblem* probs = kProgram ? p.table : p.prob;
   const int nprob = p.nprob;
   for (int i = threadIdx.x; i < nprob; i += kThreadsTc) ub[i] = probs[i].unit_begin;
@@ -509,6 +513,8 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       int q = 0, rr = 0;
+      // operands may come from the previous kernel of the stream
+      if (!kProgram) asm volatile("griddepcontrol.wait;" ::: "memory");
       for (;;) {
         if (!ok) break;
         const int u = next_unit<kProgram>(p, rr);
@@ -651,6 +657,9 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     const int half = 0;
     int j = 0, q = 0, rr = 0;
     bool ok = true;
+    // sign words, addends, fragments read here and everything stored here may be in use by the
+    // previous kernel of the stream
+    if (!kProgram) asm volatile("griddepcontrol.wait;" ::: "memory");
     for (;;) {
       if (!ok) break;
       const int u = next_unit<kProgram>(p, rr);
@@ -1163,8 +1172,19 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
     g_prof.mma_flops += mma_flops;
   }
   const int grid = total < sm_count() ? total : sm_count();
-  tc_group_kernel<false><<<grid, kThreadsTc, smem, s>>>(prm);
-  const mw_status rc = launch_ok();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreadsTc);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, tc_group_kernel<false>, prm);
+  ++g_launch_count;
+  const mw_status rc = le == cudaSuccess ? MW_OK : MW_ERR_CUDA;
   if (prof) cudaEventRecord(prof_event(), s);
   return rc;
 }
