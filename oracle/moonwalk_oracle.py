@@ -25,7 +25,9 @@ the output cotangent at every dead unit, row by row in increasing column
 order; the stride-1 same-size convolution's vijp is the unique solution of
 Eq. "conv-vjp" for h', computed with the paper's relation
 w_centre h'_{i'} = h_{i'} - TransposeConv(h', w~)_{i'} used as a fixed-point
-iteration with the whole C x C centre tap as the pivot block.
+iteration with the whole C x C centre tap as the pivot block; a convolution
+that meets Lemma 1 (stride above padding, triangular anchor tap) takes the
+lemma's elimination itself, which is exact.
 
 Pinned by tests/test_oracle_*.py: finite differences, Moonwalk == Backprop,
 vjp(vijp(h)) == h, closed-form leaky-ReLU inverse, explicit-Jacobian brute
@@ -189,8 +191,63 @@ def vijp_conv_fixed_point(layer, w, h, tol=1e-14, max_iters=400, iters=None, tra
     return g
 
 
+def submersive_conditions(layer, w):
+    """Lemma 1, conditions (i)-(iii), for one spatial size n x n' per dimension; returns the
+    list of violated conditions (empty = submersive by the lemma)."""
+    k, s, p = layer.k, layer.stride, layer.pad
+    bad = []
+    for n in (layer.H, layer.W):
+        n_out = (n + 2 * p - k) // s + 1
+        if not (k > p and s > p and n > s * (n_out - 1)):
+            bad.append("(i) spatial bounds")
+            break
+    m, mp = w.shape[2], w.shape[3]
+    anchor = w[p, p] if k > p else np.zeros((m, mp))
+    if mp > m or np.any(np.triu(anchor, 1) != 0.0):          # entries with c < c'
+        bad.append("(ii) channel-wise triangularity")
+    if np.any(np.diagonal(anchor)[:mp] == 0.0):
+        bad.append("(iii) diagonal support")
+    return bad
+
+
+def vijp_conv_submersive(layer, w, h):
+    """vijp of a convolution that meets Lemma 1, by the elimination of its proof: in
+    lexicographic order of (i', c'),
+        w[p, c', c'] h'[i', c'] = h[s i', c'] - TransposeConv(h', w~)[s i', c'],
+    w~ = w with the diagonal of the anchor tap w[p] zeroed; every h' entry that appears on the
+    right with a non-zero coefficient has a smaller index and is already known.  Terms from
+    other pixels (taps j with p - j a non-zero multiple of s) are taken first, then the
+    channels of pixel i' itself are eliminated one after the other through the triangular
+    anchor tap (Algorithm 2).  h: [B, H, W, m] -> h': [B, H', W', m']."""
+    bad = submersive_conditions(layer, w)
+    if bad:
+        raise ValueError("not submersive by Lemma 1: " + ", ".join(bad))
+    k, s, p = layer.k, layer.stride, layer.pad
+    B = h.shape[0]
+    Ho, Wo = layer.out_hw()
+    mp = w.shape[3]
+    hp = np.zeros((B, Ho, Wo, mp))
+    for i0 in range(Ho):
+        for i1 in range(Wo):
+            r = h[:, s * i0, s * i1, :mp].copy()
+            for j0 in range(k):
+                for j1 in range(k):
+                    d0, d1 = p - j0, p - j1
+                    if (d0 == 0 and d1 == 0) or d0 % s != 0 or d1 % s != 0:
+                        continue                      # anchor tap, or a zero of the dilated h'
+                    q0, q1 = i0 + d0 // s, i1 + d1 // s
+                    if 0 <= q0 < Ho and 0 <= q1 < Wo:
+                        r -= hp[:, q0, q1, :] @ w[j0, j1, :mp, :].T
+            for c in range(mp):
+                v = r[:, c] - hp[:, i0, i1, :c] @ w[p, p, c, :c]
+                hp[:, i0, i1, c] = v / w[p, p, c, c]
+    return hp
+
+
 def vijp_linear(layer, w, h, conv_iters=None):
     if layer.kind == CONV2D:
+        if layer.stride > layer.pad:
+            return vijp_conv_submersive(layer, w, h)
         return vijp_conv_fixed_point(layer, w, h, iters=conv_iters)
     return vijp_dense(w, h)
 
@@ -354,8 +411,7 @@ def forward_sweep(layers, params, x0, g0, store, conv_iters=None):
         if layer.kind == HEAD:
             gz = store["h_last"]                      # no vijp through a non-square last layer
         else:
-            gz = vijp_linear(layer, w, h.reshape(z.shape) if layer.kind == CONV2D else h,
-                             conv_iters).reshape(z.shape)
+            gz = vijp_linear(layer, w, h, conv_iters).reshape(z.shape)
         m = ms[l]
         if layer.act == ACT_RELU:
             gz = np.where(m, gz, 0.0)                 # phi' = 0: exact zeros at dead units

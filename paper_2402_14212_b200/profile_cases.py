@@ -3,6 +3,7 @@
   python -m paper_2402_14212_b200.profile_cases gemm --M 256 --N 1024 --K 1024 --terms 3 --b-mn
   python -m paper_2402_14212_b200.profile_cases pack --rows 65536 --cols 2048
   python -m paper_2402_14212_b200.profile_cases fragments --rows 65536 --cols 2048
+  python -m paper_2402_14212_b200.profile_cases conv --images 512 --op 1 --terms 2
 
 Each case allocates its seeded inputs, runs the kernel `--reps` times and exits.
 """
@@ -17,7 +18,7 @@ def main():
     import torch
     from . import binding as mwb
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["gemm", "pack", "fragments", "vijp"])
+    ap.add_argument("case", choices=["gemm", "pack", "fragments", "vijp", "conv"])
     ap.add_argument("--M", type=int, default=256)
     ap.add_argument("--N", type=int, default=1024)
     ap.add_argument("--K", type=int, default=1024)
@@ -27,6 +28,8 @@ def main():
     ap.add_argument("--rows", type=int, default=65536)
     ap.add_argument("--cols", type=int, default=2048)
     ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--images", type=int, default=512)
+    ap.add_argument("--op", type=int, default=0, help="0 conv, 1 TransposeConv, 2 weight vjp")
     a = ap.parse_args()
     g = torch.Generator(device="cuda").manual_seed(0)
     if a.case == "gemm":
@@ -34,6 +37,15 @@ def main():
         B = torch.randn((a.K, a.N) if a.b_mn else (a.N, a.K), device="cuda", generator=g)
         for _ in range(a.reps):
             mwb.gemm_split_bf16(A, B, a.a_mn, a.b_mn, a.terms)
+    elif a.case == "conv":
+        # 3x3, 64 channels, 32 x 32 images, channel-last: the convolutional configuration's layer
+        x = torch.randn((a.images, 32, 32, 64), device="cuda", generator=g)
+        if a.op == 2:
+            b = torch.randn((a.images, 32, 32, 64), device="cuda", generator=g)
+        else:
+            b = torch.randn((3, 3, 64, 64), device="cuda", generator=g)
+        for _ in range(a.reps):
+            mwb.conv2d_split_bf16(a.op, x, b, 3, a.terms)
     else:
         z = torch.randn((a.rows, a.cols), device="cuda", generator=g)
         h = torch.randn((a.rows, a.cols), device="cuda", generator=g)

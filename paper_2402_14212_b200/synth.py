@@ -189,6 +189,44 @@ def submersive_cnn(seed=0, depth=32, C=64, H=32, W=32, batch=128, gamma=0.05, cl
                    reseed_every=reseed_every, conv_vijp_iters=conv_vijp_iters, seed=seed)
 
 
+def strided_cnn(seed=0, depth=8, C=128, H=256, W=256, batch=128, gamma=0.5, reseed_every=4,
+                prec=F32) -> Problem:
+    """The fully submersive CNN of the paper's experiments (Section "Fully Parallel Submersive 2D
+    CNN"): `depth` 3x3 convolutions with C channels, stride 2, padding 1 and leaky-ReLU 0.1,
+    each halving the resolution, on a batch of H x W x C inputs (the paper: 256 x 256 x 128,
+    batch 128, up to 8 layers).
+
+    w = gamma * N(0, 2/(9*C)) (He scale) with the anchor tap w[1, 1] made lower triangular in
+    (c, c') with unit diagonal (Lemma 1 (ii), (iii); Algorithm 2 normalises the diagonal to 1).
+    Loss: mean squared error of the last feature map against a Gaussian target (the paper pools
+    and projects to a scalar; any scalar loss of the output serves).
+    """
+    rng = np.random.default_rng(seed)
+    layers, params = [], []
+    he = np.sqrt(2.0 / (9 * C))
+    h, wd = H, W
+    for l in range(depth):
+        w = gamma * he * rng.standard_normal((3, 3, C, C))
+        w[1, 1] = np.tril(w[1, 1], -1) + np.eye(C)
+        lay = Layer(CONV2D, ACT_LEAKY, 0.1, h * wd * C, 0, H=h, W=wd, C_in=C, C_out=C, k=3,
+                    stride=2, pad=1)
+        ho, wo = lay.out_hw()
+        lay.n_out = ho * wo * C
+        layers.append(lay)
+        params.append(round_storage(w, prec))
+        h, wd = ho, wo
+    if batch * H * W * C > (1 << 26):
+        # large inputs: draw in fp32 directly (an fp64 copy would not fit comfortably)
+        x = rng.standard_normal((batch, H, W, C), dtype=np.float32)
+        if prec == BF16:
+            x = bf16_bits_to_f64(round_to_bf16_bits(x)).reshape(x.shape).astype(np.float32)
+    else:
+        x = round_storage(rng.standard_normal((batch, H, W, C)), prec)
+    t = round_storage(rng.standard_normal((batch, h, wd, C)), F32 if prec == BF16 else prec)
+    return Problem("strided_cnn", layers, params, x, t, LOSS_MSE_MEAN, prec, batch,
+                   reseed_every=reseed_every, seed=seed)
+
+
 def random_preacts(seed: int, rows: int, cols: int, zero_frac: float = 0.01) -> np.ndarray:
     """fp32 pre-activation-like array with exact zeros, negative zeros and a NaN sprinkled in
     (inputs for the sign-bit pack / fragment compaction unit tests)."""

@@ -140,6 +140,90 @@ def test_conv_vijp_equals_dense_solve_on_explicit_jacobian():
     assert 1e-12 < np.abs(g3.ravel() - g_ref).max() < 0.5
 
 
+def submersive_kernel(rng, k, p, C, Cp, scale=0.4):
+    """Random kernel meeting Lemma 1 (ii), (iii): anchor tap zero for c < c', non-zero diagonal."""
+    w = scale * rng.standard_normal((k, k, C, Cp))
+    a = np.tril(w[p, p])                                   # keeps c >= c'
+    a[np.arange(Cp), np.arange(Cp)] = 1.0 + 0.3 * rng.random(Cp)
+    w[p, p] = a
+    return w
+
+
+@pytest.mark.parametrize("k,s,p,H,C,Cp", [(3, 2, 1, 8, 4, 4), (3, 2, 1, 6, 5, 3), (5, 2, 1, 9, 3, 3),
+                                          (4, 3, 2, 8, 3, 2), (3, 2, 0, 7, 3, 3)])
+def test_submersive_conv_vijp_against_explicit_jacobian(k, s, p, H, C, Cp):
+    # Lemma 1: the Jacobian J of the layer has a right inverse and the elimination recovers h'
+    # from h = h' J.  J is built index by index from the defining sum, not from the oracle.
+    rng = np.random.default_rng(100 * k + 10 * s + p)
+    w = submersive_kernel(rng, k, p, C, Cp)
+    layer = S.Layer(S.CONV2D, S.ACT_LEAKY, 0.1, H=H, W=H, C_in=C, C_out=Cp, k=k, stride=s, pad=p)
+    assert O.submersive_conditions(layer, w) == []
+    Ho, Wo = layer.out_hw()
+    n_in, n_out = H * H * C, Ho * Wo * Cp
+    Jm = np.zeros((n_out, n_in))
+    for i in range(n_in):
+        e = np.zeros(n_in); e[i] = 1.0
+        Jm[:, i] = conv_by_loops(e.reshape(1, H, H, C), w, s, p).ravel()
+    assert np.linalg.matrix_rank(Jm) == n_out               # submersive: full row rank
+    B = 3
+    hp = rng.standard_normal((B, Ho, Wo, Cp))
+    h = (hp.reshape(B, -1) @ Jm).reshape(B, H, H, C)        # vjp through the explicit Jacobian
+    got = O.vijp_conv_submersive(layer, w, h)
+    assert got.shape == hp.shape
+    assert np.allclose(got, hp, atol=1e-10)
+    # the same through the oracle's own TransposeConv: vijp(vjp(h')) = h'
+    assert np.allclose(O.vijp_conv_submersive(layer, w, O.transpose_conv(hp, w, (H, H), s, p)), hp,
+                       atol=1e-10)
+    # and it is a right inverse of J on the row space: vijp(h) J = h
+    assert np.allclose((got.reshape(B, -1) @ Jm).reshape(h.shape), h, atol=1e-10)
+
+
+def test_submersive_conv_vijp_special_cases():
+    rng = np.random.default_rng(3)
+    H, C = 8, 4
+    layer = S.Layer(S.CONV2D, S.ACT_LEAKY, 0.1, H=H, W=H, C_in=C, C_out=C, k=3, stride=2, pad=1)
+    # identity anchor tap alone: the layer subsamples, so does its vijp
+    w = np.zeros((3, 3, C, C)); w[1, 1] = np.eye(C)
+    h = rng.standard_normal((2, H, H, C))
+    assert np.array_equal(O.vijp_conv_submersive(layer, w, h), h[:, ::2, ::2, :])
+    # k = 3, s = 2, p = 1: at the positions s*i' only the anchor tap reaches h, so the vijp is a
+    # per-pixel triangular solve of  g A^T = h[s i']  (A = w[p, p] indexed [c][c'])
+    w = submersive_kernel(rng, 3, 1, C, C)
+    g = O.vijp_conv_submersive(layer, w, h)
+    ref = np.linalg.solve(w[1, 1], h[:, ::2, ::2, :].reshape(-1, C).T).T.reshape(g.shape)
+    assert np.allclose(g, ref, atol=1e-12)
+    # violations of the lemma are reported, not silently solved
+    wb = w.copy(); wb[1, 1, 0, 2] = 0.5                     # c < c'
+    assert "(ii) channel-wise triangularity" in O.submersive_conditions(layer, wb)
+    with pytest.raises(ValueError):
+        O.vijp_conv_submersive(layer, wb, h)
+    wb = w.copy(); wb[1, 1, 1, 1] = 0.0
+    assert "(iii) diagonal support" in O.submersive_conditions(layer, wb)
+    same = S.Layer(S.CONV2D, S.ACT_LEAKY, 0.1, H=H, W=H, C_in=C, C_out=C, k=3, stride=1, pad=1)
+    assert "(i) spatial bounds" in O.submersive_conditions(same, w)
+
+
+@pytest.mark.parametrize("K", [0, 2])
+def test_moonwalk_equals_backprop_strided_cnn(K):
+    p = S.strided_cnn(seed=2, depth=3, C=4, H=16, W=16, batch=2, gamma=1.0, reseed_every=K, prec=S.F64)
+    assert [l.out_hw() for l in p.layers] == [(8, 8), (4, 4), (2, 2)]
+    for l, w in zip(p.layers, p.params):
+        assert O.submersive_conditions(l, w) == []
+    ref = O.backprop(p.layers, p.params, p.x, p.target, p.loss)
+    mw = O.moonwalk(p.layers, p.params, p.x, p.target, p.loss, reseed_every=K)
+    for l in range(3):
+        assert O.normwise_error(mw["dW"][l], ref["dW"][l]) < 1e-9
+        assert O.normwise_error(mw["h"][l + 1], ref["h"][l + 1]) < 1e-9
+    # finite differences on a few kernel entries (the loss of the strided net itself)
+    check_off_kinks(p.layers, p.params, p.x, margin=1e-5)
+    rng = np.random.default_rng(4)
+    for l in range(3):
+        for _ in range(4):
+            idx = tuple(int(v) for v in (rng.integers(0, 3), rng.integers(0, 3), rng.integers(0, 4), rng.integers(0, 4)))
+            fd = fd_grad(p.layers, p.params, p.x, p.target, p.loss, l, idx)
+            assert abs(fd - ref["dW"][l][idx]) <= 1e-7 * max(1.0, abs(fd))
+
+
 def test_dense_vijp_is_right_inverse_and_leaky_closed_form():
     rng = np.random.default_rng(2)
     n, B = 12, 5
