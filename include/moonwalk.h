@@ -194,6 +194,23 @@ mw_status mw_conv2d_split_bf16(int32_t op, const float* a, const float* b, float
                                int32_t images, int32_t H, int32_t W, int32_t k, int32_t terms,
                                void* scratch, size_t scratch_bytes, void* stream);
 
+/* The same three steps for a k x k convolution with C channels in and out (C a multiple of 64),
+ * stride s and zero padding p (Lemma 1's general form; Section "Fully Parallel Submersive 2D CNN"
+ * uses k = 3, s = 2, p = 1, C = 128): Ho = (H + 2p - k)/s + 1, Wo likewise,
+ *   op 0  out[images][Ho][Wo][C] = sum_{j,c} w[j,c,c'] a[b, s i' + j - p, c]      a = x [images][H][W][C], b = w
+ *   op 1  out[images][H][W][C]   = sum_{j,c'} w[j,c,c'] hbar'[b, i + p - j, c']   a = h' [images][Ho][Wo][C], b = w;
+ *         hbar' is h' dilated by s (Eq. "conv-vjp").  s = 1 (k = 2p + 1), or s = 2 with H = 2 Ho, W = 2 Wo.
+ *   op 2  out[k][k][C][C]        = sum_{b,i'} a[b, s i' + j - p, c] b[b, i', c']   a = x, b = g_z [images][Ho][Wo][C]
+ * A tile of 128 consecutive product pixels (64 for op 2) must be part of an image row, whole rows
+ * of one image, or whole images (widths and heights that are powers of two up to 256 qualify);
+ * images*Ho*Wo % 64 == 0 for op 2.  Otherwise MW_ERR_UNSUPPORTED.  scratch: device, 256-byte
+ * aligned, >= 1024 + 8*terms*(elements of a + elements of b) + (op 2: 128 * k*k*C*C) bytes.
+ * Synchronises `stream`. */
+mw_status mw_conv2d_strided_split_bf16(int32_t op, const float* a, const float* b, float* out,
+                                       int32_t images, int32_t H, int32_t W, int32_t C, int32_t k,
+                                       int32_t stride, int32_t pad, int32_t terms, void* scratch,
+                                       size_t scratch_bytes, void* stream);
+
 /* The same product as mw_gemm_split_bf16 for callers that have no scratch buffer to lend and
  * cannot allocate one when they call: code that runs inside a host framework whose memory pool
  * owns the whole device (a direct cudaMalloc there fails or stalls every stream), and services

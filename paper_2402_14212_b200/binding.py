@@ -75,6 +75,8 @@ def lib() -> C.CDLL:
         L.mw_activation_vijp.argtypes = [vp, vp, i64, i32, i32, C.c_float, vp, vp, vp, vp, vp]
         L.mw_gemm_split_bf16.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, vp, sz, vp]
         L.mw_conv2d_split_bf16.argtypes = [i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, sz, vp]
+        L.mw_conv2d_strided_split_bf16.argtypes = [i32, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32,
+                                                   i32, vp, sz, vp]
         L.mw_gemm_split_bf16_static.argtypes = [vp, i32, vp, i32, vp, i32, i32, i32, i32, vp]
         L.mw_gradient_step_host.argtypes = [vp, C.POINTER(vp), vp, sz, vp, sz, vp, vp, vp,
                                             C.POINTER(vp), vp, vp, vp, sz, vp]
@@ -317,6 +319,28 @@ def conv2d_split_bf16(op: int, a, b, k: int, terms: int, stream=None):
     _check(lib().mw_conv2d_split_bf16(op, _ptr(a), _ptr(b), _ptr(out), images, H, W, k, int(terms),
                                       _ptr(scratch), scratch.numel(), _stream_handle(stream)),
            "mw_conv2d_split_bf16")
+    return out
+
+
+def conv2d_strided_split_bf16(op: int, a, b, k: int, stride: int, pad: int, terms: int, in_hw=None,
+                              stream=None):
+    """op 0: conv(a = x, b = w); op 1: TransposeConv(a = h', b = w) back to the `in_hw` image;
+    op 2: weight vjp (a = x, b = g_z).  Channel-last float tensors, C channels in and out."""
+    import torch
+    images, Ha, Wa, C = a.shape
+    if op == 1:
+        H, W = in_hw
+    else:
+        H, W = Ha, Wa
+    Ho, Wo = (H + 2 * pad - k) // stride + 1, (W + 2 * pad - k) // stride + 1
+    shape = {0: (images, Ho, Wo, C), 1: (images, H, W, C), 2: (k, k, C, C)}[op]
+    out = torch.empty(shape, dtype=torch.float32, device=a.device)
+    n = 1024 + 8 * terms * (a.numel() + b.numel()) + 128 * k * k * C * C + 4096
+    scratch = torch.empty(n, dtype=torch.uint8, device=a.device)
+    _check(lib().mw_conv2d_strided_split_bf16(op, _ptr(a), _ptr(b), _ptr(out), images, H, W, C, k,
+                                              stride, pad, int(terms), _ptr(scratch), scratch.numel(),
+                                              _stream_handle(stream)),
+           "mw_conv2d_strided_split_bf16")
     return out
 
 

@@ -32,11 +32,12 @@ int conv_wgrad_tensor_slices(int64_t pixels) {
   return 1;
 }
 
-TcOperand pixel_operand(const void* planes, int64_t pixels, int terms, int64_t plane_stride, bool mn) {
+TcOperand pixel_operand(const void* planes, int64_t pixels, int terms, int64_t plane_stride, bool mn,
+                        int channels) {
   TcOperand o;
   o.base = planes;
   o.rows = (int)pixels;
-  o.cols = 64;
+  o.cols = channels;
   o.planes = terms;
   o.plane_stride = plane_stride;
   o.mn_major = mn;
@@ -46,15 +47,62 @@ TcOperand pixel_operand(const void* planes, int64_t pixels, int terms, int64_t p
 TcGemm conv_forward_product(const ConvGeom& g, const __nv_bfloat16* x_planes, int xt,
                             const __nv_bfloat16* w_planes, int wt, const TcEpilogue& e) {
   TcGemm p;
-  p.A = pixel_operand(x_planes, g.pixels(), xt, g.pixels() * 64, false);
+  const int C = g.C;
+  p.A = pixel_operand(x_planes, g.pixels(), xt, g.pixels() * C, false, C);
   // w[tap][ci][co]: K = (tap, ci) rows, N = co contiguous
-  p.B.base = w_planes; p.B.rows = g.k * g.k * 64; p.B.cols = 64; p.B.planes = wt;
-  p.B.plane_stride = (int64_t)g.k * g.k * 4096; p.B.mn_major = true;
-  p.M = (int)g.pixels(); p.N = 64; p.K = g.k * g.k * 64;
+  p.B.base = w_planes; p.B.rows = g.k * g.k * C; p.B.cols = C; p.B.planes = wt;
+  p.B.plane_stride = g.kernel_elems(); p.B.mn_major = true;
+  p.M = (int)g.out_pixels(); p.N = C; p.K = g.k * g.k * C;
   p.epi = e;
   p.conv.mode = TC_CONV_PIXELS; p.conv.H = g.H; p.conv.W = g.W; p.conv.k = g.k; p.conv.pad = g.pad;
+  p.conv.C = C; p.conv.stride = g.stride; p.conv.Ho = g.Ho(); p.conv.Wo = g.Wo();
   p.conv.sgn = 1;
+  if (g.stride != 1) {
+    // window of output pixel i' starts at stride*i' + j - pad
+    int n = 0;
+    for (int j0 = 0; j0 < g.k; ++j0)
+      for (int j1 = 0; j1 < g.k; ++j1, ++n) {
+        p.conv.dy[n] = (signed char)(j0 - g.pad);
+        p.conv.dx[n] = (signed char)(j1 - g.pad);
+        p.conv.tb[n] = (signed char)n;
+      }
+    p.conv.ntaps = n;
+  }
   return p;
+}
+
+bool conv_transpose_class_product(const ConvGeom& g, int py, int px, const __nv_bfloat16* g_planes,
+                                  int gt, const __nv_bfloat16* w_planes, int wt, const TcEpilogue& e,
+                                  TcGemm* out) {
+  TcGemm p;
+  const int C = g.C, s = g.stride, Ho = g.Ho(), Wo = g.Wo();
+  p.A = pixel_operand(g_planes, g.out_pixels(), gt, g.out_pixels() * C, false, C);
+  // w[tap][c][c']: for one tap N = c rows, K = c' contiguous
+  p.B.base = w_planes; p.B.rows = g.k * g.k * C; p.B.cols = C; p.B.planes = wt;
+  p.B.plane_stride = g.kernel_elems(); p.B.mn_major = false;
+  p.conv.mode = TC_CONV_PIXELS; p.conv.H = Ho; p.conv.W = Wo; p.conv.C = C; p.conv.stride = 1;
+  p.conv.Ho = Ho; p.conv.Wo = Wo; p.conv.k = g.k; p.conv.pad = g.pad; p.conv.b_tap_rows = 1;
+  int n = 0;
+  for (int j0 = 0; j0 < g.k; ++j0) {
+    const int vy = py + g.pad - j0;
+    if (((vy % s) + s) % s != 0) continue;
+    for (int j1 = 0; j1 < g.k; ++j1) {
+      const int vx = px + g.pad - j1;
+      if (((vx % s) + s) % s != 0) continue;
+      // h[s y + py] takes w[j] h'[(s y + py + pad - j) / s] = h'[y + vy / s]
+      p.conv.dy[n] = (signed char)(vy >= 0 ? vy / s : -((-vy) / s));
+      p.conv.dx[n] = (signed char)(vx >= 0 ? vx / s : -((-vx) / s));
+      p.conv.tb[n] = (signed char)(j0 * g.k + j1);
+      ++n;
+    }
+  }
+  if (n == 0) return false;
+  p.conv.ntaps = n;
+  p.M = (int)g.out_pixels(); p.N = C; p.K = n * C;
+  p.epi = e;
+  p.epi.remap_s = s; p.epi.remap_ho = Ho; p.epi.remap_wo = Wo; p.epi.remap_py = py; p.epi.remap_px = px;
+  *out = p;
+  return true;
 }
 
 TcGemm conv_transpose_product(const ConvGeom& g, const __nv_bfloat16* g_planes, int gt,
@@ -77,20 +125,22 @@ TcGemm conv_transpose_product(const ConvGeom& g, const __nv_bfloat16* g_planes, 
 mw_status conv_wgrad_tensor(TcMapCache* cache, const ConvGeom& g, const __nv_bfloat16* x_planes,
                             const __nv_bfloat16* gz_planes, int terms, float* partials, float* dw,
                             DeviceStatus* st, cudaStream_t s) {
-  const int slices = conv_wgrad_tensor_slices(g.pixels());
-  const int rows = g.k * g.k * 64;
+  const int slices = conv_wgrad_tensor_slices(g.out_pixels());
+  const int C = g.C;
+  const int rows = g.k * g.k * C;
   TcGemm p;
-  p.A = pixel_operand(x_planes, g.pixels(), terms, g.pixels() * 64, true);
-  p.B = pixel_operand(gz_planes, g.pixels(), terms, g.pixels() * 64, true);
-  p.M = rows; p.N = 64; p.K = (int)(g.pixels() / slices);
+  p.A = pixel_operand(x_planes, g.pixels(), terms, g.pixels() * C, true, C);
+  p.B = pixel_operand(gz_planes, g.out_pixels(), terms, g.out_pixels() * C, true, C);
+  p.M = rows; p.N = C; p.K = (int)(g.out_pixels() / slices);
   p.batch = slices;
   p.epi.mode = TC_EPI_PLAIN;
   p.epi.out_f32 = slices > 1 ? partials : dw;
-  p.epi.bs_f32 = (int64_t)rows * 64;
+  p.epi.bs_f32 = (int64_t)rows * C;
   p.conv.mode = TC_CONV_WGRAD; p.conv.H = g.H; p.conv.W = g.W; p.conv.k = g.k; p.conv.pad = g.pad;
+  p.conv.C = C; p.conv.stride = g.stride; p.conv.Ho = g.Ho(); p.conv.Wo = g.Wo();
   MW_TRY(tc_gemm_group(cache, &p, 1, st, s));
   if (slices > 1) {
-    const int64_t n = (int64_t)rows * 64;
+    const int64_t n = (int64_t)rows * C;
     slice_sum_f32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(partials, n, n, slices, dw);
     MW_TRY(launch_ok());
   }
@@ -102,62 +152,91 @@ mw_status conv_wgrad_tensor(TcMapCache* cache, const ConvGeom& g, const __nv_bfl
 // ---------------------------------------------------------------------------------------
 // C ABI: the three convolution products, exposed for unit parity tests
 // ---------------------------------------------------------------------------------------
-extern "C" mw_status mw_conv2d_split_bf16(int32_t op, const float* a, const float* b, float* out,
-                                          int32_t images, int32_t H, int32_t W, int32_t k,
-                                          int32_t terms, void* scratch, size_t scratch_bytes,
-                                          void* stream) {
+extern "C" mw_status mw_conv2d_strided_split_bf16(int32_t op, const float* a, const float* b, float* out,
+                                                  int32_t images, int32_t H, int32_t W, int32_t C,
+                                                  int32_t k, int32_t stride, int32_t pad, int32_t terms,
+                                                  void* scratch, size_t scratch_bytes, void* stream) {
   using namespace mw;
   if (!a || !b || !out || !scratch) return MW_ERR_INVALID_ARG;
-  if (op < 0 || op > 2 || terms < 1 || terms > 3 || images < 1 || H < 1 || W < 1 || k < 1 || !(k & 1))
+  if (op < 0 || op > 2 || terms < 1 || terms > 3 || images < 1 || H < 1 || W < 1 || k < 1 || C < 64 ||
+      C % 64 != 0 || stride < 1 || pad < 0 || pad >= k || H + 2 * pad < k || W + 2 * pad < k)
     return MW_ERR_INVALID_ARG;
-  ConvGeom g{images, H, W, k, k / 2};
-  const int64_t px = g.pixels();
-  const int64_t ea = px * 64;                                   // pixel array
-  const int64_t ew = (int64_t)k * k * 4096;                     // kernel
-  const int64_t eb = op == 2 ? ea : ew;
-  const int slices = conv_wgrad_tensor_slices(px);
-  const size_t need = 256 + 2 * (size_t)terms * (align_up((size_t)ea, 128) + align_up((size_t)eb, 128)) +
-                      (op == 2 ? (size_t)slices * ew * 4 : 0) + 512;
+  ConvGeom g{images, H, W, k, pad, C, stride};
+  const int64_t pin = g.pixels() * C, pout = g.out_pixels() * C;  // elements of the two pixel arrays
+  const int64_t ew = g.kernel_elems();
+  const int64_t ea = op == 1 ? pout : pin;
+  const int64_t eb = op == 2 ? pout : ew;
+  const int slices = conv_wgrad_tensor_slices(g.out_pixels());
+  const size_t sa = align_up((size_t)ea, 128), sb = align_up((size_t)eb, 128);
+  const size_t need = 256 + 2 * (size_t)terms * (sa + sb) + (op == 2 ? (size_t)slices * ew * 4 : 0) + 512;
   if (((uintptr_t)scratch & 255u) || scratch_bytes < need) return MW_ERR_WORKSPACE;
+  if (op == 1 && stride > 1 && (stride > 2 || H != stride * g.Ho() || W != stride * g.Wo()))
+    return MW_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)stream;
   DeviceStatus* st = reinterpret_cast<DeviceStatus*>(scratch);
   MW_CUDA_OK(cudaMemsetAsync(st, 0, 256, s));
   __nv_bfloat16* pa = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(scratch) + 256);
-  __nv_bfloat16* pb = pa + (size_t)terms * align_up((size_t)ea, 128);
-  float* partials = reinterpret_cast<float*>(pb + (size_t)terms * align_up((size_t)eb, 128));
-  MW_TRY(split_planes(a, ea, pa, terms, (int64_t)align_up((size_t)ea, 128), s));
-  MW_TRY(split_planes(b, eb, pb, terms, (int64_t)align_up((size_t)eb, 128), s));
-  mw_status rc;
+  __nv_bfloat16* pb = pa + (size_t)terms * sa;
+  float* partials = reinterpret_cast<float*>(pb + (size_t)terms * sb);
+  MW_TRY(split_planes(a, ea, pa, terms, (int64_t)sa, s));
+  MW_TRY(split_planes(b, eb, pb, terms, (int64_t)sb, s));
+  mw_status rc = MW_OK;
+  TcEpilogue e;
+  e.mode = TC_EPI_PLAIN;
+  e.out_f32 = out;
   if (op == 2) {
-    // planes are spaced by the padded size: rebuild the operands with that stride
+    // the planes here are spaced by the padded sizes: build the product with those strides
+    const int rows = k * k * C;
     TcGemm p;
-    p.A = pixel_operand(pa, px, terms, (int64_t)align_up((size_t)ea, 128), true);
-    p.B = pixel_operand(pb, px, terms, (int64_t)align_up((size_t)eb, 128), true);
-    const int rows = k * k * 64;
-    p.M = rows; p.N = 64; p.K = (int)(px / slices); p.batch = slices;
+    p.A = pixel_operand(pa, g.pixels(), terms, (int64_t)sa, true, C);
+    p.B = pixel_operand(pb, g.out_pixels(), terms, (int64_t)sb, true, C);
+    p.M = rows; p.N = C; p.K = (int)(g.out_pixels() / slices); p.batch = slices;
     p.epi.mode = TC_EPI_PLAIN;
     p.epi.out_f32 = slices > 1 ? partials : out;
-    p.epi.bs_f32 = (int64_t)rows * 64;
-    p.conv.mode = TC_CONV_WGRAD; p.conv.H = H; p.conv.W = W; p.conv.k = k; p.conv.pad = k / 2;
+    p.epi.bs_f32 = (int64_t)rows * C;
+    p.conv.mode = TC_CONV_WGRAD; p.conv.H = H; p.conv.W = W; p.conv.k = k; p.conv.pad = pad;
+    p.conv.C = C; p.conv.stride = stride; p.conv.Ho = g.Ho(); p.conv.Wo = g.Wo();
     rc = tc_gemm_group(nullptr, &p, 1, st, s);
     if (rc == MW_OK && slices > 1) {
-      const int64_t n = (int64_t)rows * 64;
+      const int64_t n = (int64_t)rows * C;
       slice_sum_f32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(partials, n, n, slices, out);
       rc = launch_ok();
     }
-  } else {
-    TcEpilogue e;
-    e.mode = TC_EPI_PLAIN;
-    e.out_f32 = out;
-    TcGemm p = op == 0 ? conv_forward_product(g, pa, terms, pb, terms, e)
-                       : conv_transpose_product(g, pa, terms, pb, terms, false, e);
-    p.A.plane_stride = (int64_t)align_up((size_t)ea, 128);
-    p.B.plane_stride = (int64_t)align_up((size_t)eb, 128);
+  } else if (op == 0) {
+    TcGemm p = conv_forward_product(g, pa, terms, pb, terms, e);
+    p.A.plane_stride = (int64_t)sa;
+    p.B.plane_stride = (int64_t)sb;
     rc = tc_gemm_group(nullptr, &p, 1, st, s);
+  } else if (stride == 1) {
+    if (2 * pad + 1 != k) return MW_ERR_UNSUPPORTED;
+    TcGemm p = conv_transpose_product(g, pa, terms, pb, terms, false, e);
+    p.A.plane_stride = (int64_t)sa;
+    p.B.plane_stride = (int64_t)sb;
+    rc = tc_gemm_group(nullptr, &p, 1, st, s);
+  } else {
+    TcGemm cls[4];
+    int n = 0;
+    for (int py = 0; py < stride; ++py)
+      for (int px = 0; px < stride; ++px) {
+        if (!conv_transpose_class_product(g, py, px, pa, terms, pb, terms, e, &cls[n])) return MW_ERR_UNSUPPORTED;
+        cls[n].A.plane_stride = (int64_t)sa;
+        cls[n].B.plane_stride = (int64_t)sb;
+        ++n;
+      }
+    rc = tc_gemm_group(nullptr, cls, n, st, s);
   }
   MW_TRY(rc);
   DeviceStatus host;
   MW_CUDA_OK(cudaMemcpyAsync(&host, st, sizeof(host), cudaMemcpyDeviceToHost, s));
   MW_CUDA_OK(cudaStreamSynchronize(s));
   return host.code == 0 ? MW_OK : (mw_status)host.code;
+}
+
+extern "C" mw_status mw_conv2d_split_bf16(int32_t op, const float* a, const float* b, float* out,
+                                          int32_t images, int32_t H, int32_t W, int32_t k,
+                                          int32_t terms, void* scratch, size_t scratch_bytes,
+                                          void* stream) {
+  if (k < 1 || !(k & 1)) return MW_ERR_INVALID_ARG;
+  return mw_conv2d_strided_split_bf16(op, a, b, out, images, H, W, 64, k, 1, k / 2, terms, scratch,
+                                      scratch_bytes, stream);
 }

@@ -67,7 +67,8 @@ struct alignas(64) TcProblem {
   float* split_partials;
   unsigned int* split_counters;
   // convolution forms (TcConv)
-  int conv_mode, cH, cW, ck, cpad, csgn, cskip, b_tap_rows, cntaps;
+  int conv_mode, cHo, cWo, ck, cpad, cstride, ccb, b_tap_rows, cntaps;
+  signed char tdy[28], tdx[28], ttb[28];
   // program launches: products (by index) that must be complete before this one starts, and
   // the number of warp arrivals that completes each of them (one per epilogue warp and tile)
   int ndep, dep[3];
@@ -534,12 +535,14 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         const bool a_mn = P.a_mn != 0, b_mn = P.b_mn != 0;
         const uint32_t b_tile_bytes = P.b_tile_bytes, tx = P.tx_bytes;
         const int conv = P.conv_mode;
-        // convolution: image and first image row of the unit's pixel tile
-        int cb = 0, cy0 = 0;
+        // convolution: image, row and column of the first pixel of the unit's tile
+        int cb = 0, cy0 = 0, cx0 = 0;
         if (conv == TC_CONV_PIXELS) {
-          const int hw = P.cH * P.cW;
+          const int hw = P.cHo * P.cWo;
           cb = w.m0 / hw;
-          cy0 = (w.m0 - cb * hw) / P.cW;
+          const int rem = w.m0 - cb * hw;
+          cy0 = rem / P.cWo;
+          cx0 = rem - cy0 * P.cWo;
         }
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, p.st, 1u, abortp)) { ok = false; break; }
@@ -549,26 +552,29 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           int k0 = kb * BK;
           int bk0 = k0, bn0 = w.n0;       // B coordinates (K, N)
           if (conv == TC_CONV_PIXELS) {
-            const int tap = (P.cskip >= 0 && kb >= P.cskip) ? kb + 1 : kb;
-            const int j0 = tap / P.ck, j1 = tap - j0 * P.ck;
-            const int dy = P.csgn * (j0 - P.cpad), dx = P.csgn * (j1 - P.cpad);
+            const int t = kb / P.ccb, cblk = kb - t * P.ccb;
+            const int dy = P.tdy[t], dx = P.tdx[t], tb = P.ttb[t];
             for (int pl = 0; pl < pa; ++pl)
-              tma_load_5d(sbase + (uint32_t)pl * kATileBytes, &P.tmA, fb, 0, dx, cy0 + dy, cb, a_pl0 + pl);
-            bk0 = tap * BK;
-            if (P.b_tap_rows) { bn0 = tap * BK + w.n0; bk0 = 0; }
+              tma_load_5d(sbase + (uint32_t)pl * kATileBytes, &P.tmA, fb, cblk * BK, P.cstride * cx0 + dx,
+                          P.cstride * cy0 + dy, cb, a_pl0 + pl);
+            bk0 = (tb * P.ccb + cblk) * BK;
+            if (P.b_tap_rows) { bn0 = tb * P.N + w.n0; bk0 = cblk * BK; }
           } else if (conv == TC_CONV_WGRAD) {
-            // K block = 64 pixels of slice z; the two halves of the A tile are two taps
+            // K block = 64 pixels of slice z; the two halves of the A tile are two blocks of 64
+            // rows (tap, channel block)
             const int pix = (w.z * P.num_kb + kb) * BK;
-            const int hw = P.cH * P.cW;
-            const int b = pix / hw, y0 = (pix - b * hw) / P.cW;
-            const int t0 = 2 * (w.m0 / BM);
+            const int hw = P.cHo * P.cWo;
+            const int b = pix / hw, rem = pix - b * hw;
+            const int y0 = rem / P.cWo, x0 = rem - y0 * P.cWo;
+            const int r0 = 2 * (w.m0 / BM);
             for (int hh = 0; hh < 2; ++hh) {
-              int tap = t0 + hh;
+              int tap = (r0 + hh) / P.ccb;
+              const int cblk = (r0 + hh) - tap * P.ccb;
               if (tap >= P.cntaps) tap = P.cntaps - 1;   // rows past the last tap are never stored
               const int j0 = tap / P.ck, j1 = tap - j0 * P.ck;
               for (int pl = 0; pl < pa; ++pl)
-                tma_load_5d(sbase + (uint32_t)pl * kATileBytes + (uint32_t)hh * 8192u, &P.tmA, fb, 0,
-                            j1 - P.cpad, y0 + j0 - P.cpad, b, pl);
+                tma_load_5d(sbase + (uint32_t)pl * kATileBytes + (uint32_t)hh * 8192u, &P.tmA, fb, cblk * BK,
+                            P.cstride * x0 + j1 - P.cpad, P.cstride * y0 + j0 - P.cpad, b, pl);
             }
             bk0 = pix;
             k0 = pix;
@@ -676,6 +682,14 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       const int row = w.m0 + quarter * 32 + lane;
       const int bn = P.bn, nblk = P.nblocks, N = P.N;
       TcEpilogue epi = P.epi;           // this batch item's view of the outputs
+      int orow = row;                   // where the row's outputs live
+      if (epi.remap_s) {
+        const int hw = epi.remap_ho * epi.remap_wo;
+        const int b = row / hw, rem = row - b * hw;
+        const int y = rem / epi.remap_wo, x = rem - y * epi.remap_wo;
+        orow = (b * epi.remap_ho * epi.remap_s + epi.remap_s * y + epi.remap_py) *
+                   (epi.remap_wo * epi.remap_s) + epi.remap_s * x + epi.remap_px;
+      }
       if (w.z) {
         const int64_t z = w.z;
         if (epi.addend) epi.addend += z * epi.bs_f32;
@@ -769,7 +783,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           } else {
             load_chunk(c, v);
           }
-          if (row < P.M) epilogue_chunk(epi, N, row, w.n0 + c, v, sumsq_local);
+          if (row < P.M) epilogue_chunk(epi, N, orow, w.n0 + c, v, sumsq_local);
         }
       }
       (void)nchunk;
@@ -910,14 +924,14 @@ static cudaEvent_t prof_event() {
 }
 
 struct TcMapCache {
-  std::map<std::tuple<const void*, int, int, int, int64_t, int>, CUtensorMap> maps;
+  std::map<std::tuple<const void*, int, int, int, int64_t, int64_t>, CUtensorMap> maps;
 };
 TcMapCache* tc_cache_create() { return new TcMapCache(); }
 void tc_cache_destroy(TcMapCache* c) { delete c; }
 
 static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, int total_planes,
                          CUtensorMap* out) {
-  auto key = std::make_tuple(op.base, op.rows, op.cols, total_planes, op.plane_stride, box_rows);
+  auto key = std::make_tuple(op.base, op.rows, op.cols, total_planes, op.plane_stride, (int64_t)box_rows);
   if (cache) {
     auto it = cache->maps.find(key);
     if (it != cache->maps.end()) { *out = it->second; return MW_OK; }
@@ -939,25 +953,30 @@ static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, i
   return MW_OK;
 }
 
-// channel-last pixel array [images][H][W][64] per plane, read in boxes of `box_rows` image rows
-static mw_status get_map_conv(TcMapCache* cache, const TcOperand& op, int H, int W, int box_rows,
-                              int total_planes, CUtensorMap* out) {
+// channel-last pixel array [images][H][W][C] per plane, read in boxes of 64 channels of bx x by
+// pixels (every `stride`-th one in both directions) of bi images
+static mw_status get_map_conv(TcMapCache* cache, const TcOperand& op, int H, int W, int bx, int by,
+                              int bi, int stride, int total_planes, CUtensorMap* out) {
+  const int C = op.cols;
   auto key = std::make_tuple(op.base, op.rows, op.cols, total_planes, op.plane_stride,
-                             1000000 + W * 1000 + box_rows);
+                             ((int64_t)1 << 62) + (((((int64_t)W * 4096 + H) * 512 + bx) * 512 + by) * 512 + bi) * 8 + stride);
   if (cache) {
     auto it = cache->maps.find(key);
     if (it != cache->maps.end()) { *out = it->second; return MW_OK; }
   }
   auto fn = encode_fn();
   if (!fn) return MW_ERR_CUDA;
-  if (((uintptr_t)op.base & 15u) || op.cols != 64 || op.rows % (H * W) != 0) return MW_ERR_INVALID_ARG;
+  if (((uintptr_t)op.base & 15u) || C % 64 != 0 || op.rows % (H * W) != 0) return MW_ERR_INVALID_ARG;
   const int64_t ps = total_planes > 1 ? op.plane_stride : (int64_t)op.rows * op.cols;
   if (ps % 8 != 0) return MW_ERR_INVALID_ARG;
+  // a strided box spans stride * count pixels and loads every stride-th of them
+  if (bx * stride > 256 || by * stride > 256 || bi > 256) return MW_ERR_UNSUPPORTED;
   const cuuint64_t images = (cuuint64_t)(op.rows / (H * W));
-  cuuint64_t dims[5] = {64u, (cuuint64_t)W, (cuuint64_t)H, images, (cuuint64_t)total_planes};
-  cuuint64_t strides[4] = {128u, (cuuint64_t)W * 128u, (cuuint64_t)H * W * 128u, (cuuint64_t)ps * 2};
-  cuuint32_t box[5] = {64u, (cuuint32_t)W, (cuuint32_t)box_rows, 1u, 1u};
-  cuuint32_t estr[5] = {1u, 1u, 1u, 1u, 1u};
+  const cuuint64_t pb = (cuuint64_t)C * 2;     // bytes of one pixel
+  cuuint64_t dims[5] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, images, (cuuint64_t)total_planes};
+  cuuint64_t strides[4] = {pb, (cuuint64_t)W * pb, (cuuint64_t)H * W * pb, (cuuint64_t)ps * 2};
+  cuuint32_t box[5] = {64u, (cuuint32_t)(bx * stride), (cuuint32_t)(by * stride), (cuuint32_t)bi, 1u};
+  cuuint32_t estr[5] = {1u, (cuuint32_t)stride, (cuuint32_t)stride, 1u, 1u};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(op.base), dims, strides,
                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -1036,20 +1055,47 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   if (d.A.planes < 1 || d.A.planes > 3 || d.B.planes < 1 || d.B.planes > 3) return MW_ERR_INVALID_ARG;
   if (d.A.mn_major && (d.M % 64 != 0)) return MW_ERR_UNSUPPORTED;
   const TcConv& cv = d.conv;
+  int cbx = 0, cby = 0, cbi = 0;          // pixels, rows, images of one A box
+  P.conv_mode = cv.mode;
   if (cv.mode != TC_CONV_NONE) {
     const int span = cv.mode == TC_CONV_PIXELS ? BM : BK;    // pixels per A box
-    if (cv.W < 1 || cv.H < 1 || span % cv.W != 0 || cv.H % (span / cv.W) != 0 || cv.k < 1 ||
-        cv.k * cv.k > 64 || d.N != 64)
+    const int Ho = cv.Ho ? cv.Ho : cv.H, Wo = cv.Wo ? cv.Wo : cv.W;
+    const int C = d.A.cols;
+    if (cv.W < 1 || cv.H < 1 || Ho < 1 || Wo < 1 || cv.stride < 1 || cv.stride > 4 || C != cv.C ||
+        C % 64 != 0 || cv.k < 0 || cv.k * cv.k > kTcMaxTaps || cv.ntaps < 0 || cv.ntaps > kTcMaxTaps)
       return MW_ERR_UNSUPPORTED;
-    if (cv.mode == TC_CONV_PIXELS && (d.A.mn_major || d.M % (cv.H * cv.W) != 0 || d.batch != 1 ||
-                                      d.K % 64 != 0 || d.K / 64 > cv.k * cv.k))
-      return MW_ERR_UNSUPPORTED;
-    if (cv.mode == TC_CONV_WGRAD && (!d.A.mn_major || !d.B.mn_major || d.M != cv.k * cv.k * 64 ||
-                                     d.K % 64 != 0 || d.split_k > 1))
-      return MW_ERR_UNSUPPORTED;
+    cbx = Wo < span ? Wo : span;
+    if (span % cbx != 0 || Wo % cbx != 0) return MW_ERR_UNSUPPORTED;
+    cby = span / cbx < Ho ? span / cbx : Ho;
+    if (Ho % cby != 0) return MW_ERR_UNSUPPORTED;
+    cbi = span / (cbx * cby);
+    if (cbx * cby * cbi != span) return MW_ERR_UNSUPPORTED;
+    P.cHo = Ho; P.cWo = Wo; P.cstride = cv.stride; P.ccb = C / 64;
+    P.ck = cv.k; P.cpad = cv.pad; P.b_tap_rows = cv.b_tap_rows;
+    if (cv.mode == TC_CONV_PIXELS) {
+      int nt = 0;
+      if (cv.ntaps > 0) {
+        for (; nt < cv.ntaps; ++nt) { P.tdy[nt] = cv.dy[nt]; P.tdx[nt] = cv.dx[nt]; P.ttb[nt] = cv.tb[nt]; }
+      } else {
+        for (int tap = 0; tap < cv.k * cv.k; ++tap) {
+          if (tap == cv.skip_tap) continue;
+          const int j0 = tap / cv.k, j1 = tap - j0 * cv.k;
+          P.tdy[nt] = (signed char)(cv.sgn * (j0 - cv.pad));
+          P.tdx[nt] = (signed char)(cv.sgn * (j1 - cv.pad));
+          P.ttb[nt] = (signed char)tap;
+          ++nt;
+        }
+      }
+      P.cntaps = nt;
+      if (nt < 1 || d.A.mn_major || d.M % (Ho * Wo) != 0 || d.batch != 1 || d.K != nt * C)
+        return MW_ERR_UNSUPPORTED;
+    } else {
+      P.cntaps = cv.k * cv.k;
+      if (cv.k < 1 || !d.A.mn_major || !d.B.mn_major || d.M != cv.k * cv.k * C || d.K % 64 != 0 ||
+          d.split_k > 1)
+        return MW_ERR_UNSUPPORTED;
+    }
   }
-  P.conv_mode = cv.mode; P.cH = cv.H; P.cW = cv.W; P.ck = cv.k; P.cpad = cv.pad; P.csgn = cv.sgn;
-  P.cskip = cv.skip_tap; P.b_tap_rows = cv.b_tap_rows; P.cntaps = cv.k * cv.k;
   P.ndep = 0;
   P.M = d.M; P.N = d.N; P.K = d.K;
   P.pa = d.A.planes; P.pb = d.B.planes;
@@ -1091,10 +1137,10 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   const int a_total = d.batch > 1 ? (d.batch - 1) * P.a_batch_planes + d.A.planes : d.A.planes;
   const int b_total = d.batch > 1 ? (d.batch - 1) * P.b_batch_planes + d.B.planes : d.B.planes;
   if (cv.mode == TC_CONV_PIXELS) {
-    MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, BM / cv.W, a_total, &P.tmA));
+    MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, cbx, cby, cbi, cv.stride, a_total, &P.tmA));
     MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
   } else if (cv.mode == TC_CONV_WGRAD) {
-    MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, BK / cv.W, d.A.planes, &P.tmA));
+    MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, cbx, cby, cbi, cv.stride, d.A.planes, &P.tmA));
     MW_TRY(get_map(cache, d.B, 64, d.B.planes, &P.tmB));
   } else {
     MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA));

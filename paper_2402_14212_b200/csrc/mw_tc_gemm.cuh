@@ -71,29 +71,43 @@ struct TcEpilogue {
   int64_t bs_planes = 0, bs_planes2 = 0;
   int64_t bs_mask = 0;                 // words
   int64_t bs_sumsq = 0;                // doubles
+  // row scatter (remap_s > 0): row r of the product is pixel (b, y, x) of a remap_ho x remap_wo
+  // image and its outputs (and sign words) live at pixel (b, remap_s*y + remap_py,
+  // remap_s*x + remap_px) of the remap_s times larger image: one parity class of a strided
+  // TransposeConv
+  int remap_s = 0, remap_ho = 0, remap_wo = 0, remap_py = 0, remap_px = 0;
 };
 
-// Convolution forms of a product (stride 1, same size, 64 channels = one K block per tap).
-// The A operand is then a channel-last pixel array [B][H][W][64] per term plane, read through a
-// window shifted by the tap (out-of-image pixels read as zero: the padding of Lemma 1):
-//   TC_CONV_PIXELS  rows of A = pixels, K = (tap, channel): K block kb is tap kb (taps before
-//                   `skip_tap` keep their index, later ones move down by one) and reads pixel
-//                   (y + sgn*(j0 - pad), x + sgn*(j1 - pad)).  sgn = +1: forward convolution,
-//                   sgn = -1: TransposeConv (Eq. "conv-vjp").  B is indexed by the same tap.
-//   TC_CONV_WGRAD   weight vjp (Eq. "g_i" for a convolution): rows of the result = (tap, c), two
-//                   taps per 128-row tile; K = pixels; batch item z covers the K blocks
+// Convolution forms of a product.  The A operand is then a channel-last pixel array
+// [images][H][W][C] per term plane (C a multiple of 64: one K block per tap and 64 channels),
+// read through a window that starts at `stride` times the product's own pixel plus an offset
+// (out-of-image pixels read as zero: the padding of Lemma 1).  The product's pixels form images
+// of Ho x Wo; a tile covers part of a row, whole rows of one image, or whole images.
+//   TC_CONV_PIXELS  rows of A = pixels (b, y, x) of the Ho x Wo image, K = (window, channel).
+//                   Window t reads pixel (stride*y + dy[t], stride*x + dx[t]) and the B block
+//                   tb[t].  With ntaps = 0 the list is derived from k, pad, sgn, skip_tap: every
+//                   tap (j0, j1) but skip_tap, offset sgn*(j - pad), B block = tap.  sgn = +1:
+//                   forward convolution (Lemma 1), sgn = -1: TransposeConv (Eq. "conv-vjp").
+//   TC_CONV_WGRAD   weight vjp (Eq. "g_i" for a convolution): rows of the result = (tap, c);
+//                   K = pixels of the Ho x Wo image; batch item z covers the K blocks
 //                   [z*K/64, (z+1)*K/64) of the pixel range, so that `batch` slices of the pixel sum
-//                   land in separate outputs.  A (MN-major) is the shifted activation, B (MN-major)
-//                   the cotangent [pixels][64].
+//                   land in separate outputs.  A (MN-major) is the activation read at
+//                   stride*pixel + tap - pad, B (MN-major) the cotangent [pixels][N].
 enum TcConvMode : int { TC_CONV_NONE = 0, TC_CONV_PIXELS = 1, TC_CONV_WGRAD = 2 };
+constexpr int kTcMaxTaps = 25;
 
 struct TcConv {
   int mode = TC_CONV_NONE;
-  int H = 0, W = 0;         // image; 128 % W == 0 (64 % W == 0 for TC_CONV_WGRAD), H*W % 128 == 0
-  int k = 0, pad = 0;       // kernel k x k
+  int H = 0, W = 0;         // image of the pixel array A reads
+  int C = 64;               // its channels
+  int stride = 1;
+  int Ho = 0, Wo = 0;       // image of the product's pixels (0: H, W)
+  int k = 0, pad = 0;       // kernel k x k (k*k <= kTcMaxTaps)
   int sgn = 1;
   int skip_tap = -1;        // tap left out of the sum (the centre tap of the folded kernel), or -1
-  int b_tap_rows = 0;       // B is K-major with rows (tap, n): used by TransposeConv
+  int b_tap_rows = 0;       // B is K-major with rows (block, n): used by TransposeConv
+  int ntaps = 0;            // explicit window list (TC_CONV_PIXELS)
+  signed char dy[kTcMaxTaps] = {}, dx[kTcMaxTaps] = {}, tb[kTcMaxTaps] = {};
 };
 
 // One product of a group.

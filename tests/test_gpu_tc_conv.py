@@ -48,3 +48,33 @@ def test_small_cnn_fp32_tensor_path(depth, H, W, batch, K, iters, resident):
                          reseed_every=K, conv_vijp_iters=iters, prec=S.F32)
     out, ref, errs = check_problem(p, 1e-4, backend="tensor", resident=resident, exact_masks=False,
                                    tau=1e-4)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("terms", [1, 3])
+@pytest.mark.parametrize("images,H,W,C", [(2, 16, 16, 128), (1, 64, 64, 128), (4, 8, 8, 64), (16, 4, 4, 128),
+                                          (64, 2, 2, 128), (1, 256, 256, 64), (3, 32, 16, 128)])
+def test_strided_conv_products(images, H, W, C, terms):
+    """3x3, stride 2, padding 1 (the paper's submersive layer): forward, TransposeConv through its
+    four parity classes, weight vjp; tiles that are part of a row, rows of an image, whole images."""
+    import torch
+    from paper_2402_14212_b200 import binding as mwb
+    rng = np.random.default_rng(images * 1000 + H)
+    k, s, p = 3, 2, 1
+    Ho, Wo = (H + 2 * p - k) // s + 1, (W + 2 * p - k) // s + 1
+    x = rng.standard_normal((images, H, W, C)).astype(np.float32)
+    w = (rng.standard_normal((k, k, C, C)) / np.sqrt(C * k * k)).astype(np.float32)
+    g = rng.standard_normal((images, Ho, Wo, C)).astype(np.float32)
+    w[0, 2, 1, 2] = 1.5
+    xt, wt, gt = (torch.from_numpy(v).cuda() for v in (x, w, g))
+    x64, w64, g64 = x.astype(np.float64), w.astype(np.float64), g.astype(np.float64)
+    tol = {1: 2e-2, 3: 2e-6}[terms]
+    cases = [(0, xt, wt, None, O.conv_forward(x64, w64, s, p)),
+             (1, gt, wt, (H, W), O.transpose_conv(g64, w64, (H, W), s, p))]
+    if (images * Ho * Wo) % 64 == 0:
+        cases.append((2, xt, gt, None, O.conv_weight_vjp(x64, g64, k, s, p)))
+    for op, a, b, hw, ref in cases:
+        got = mwb.conv2d_strided_split_bf16(op, a, b, k, s, p, terms, in_hw=hw).double().cpu().numpy()
+        assert got.shape == ref.shape
+        err = np.abs(got - ref).max() / np.abs(ref).max()
+        assert err < tol, (op, err)
