@@ -221,7 +221,8 @@ class Net:
     def export_masks(self, workspace, layer: int, stream=None) -> np.ndarray:
         l = self.layers[layer]
         if l.kind == "conv2d":
-            rows, cols = self.batch * l.H * l.W, l.C_out
+            ho, wo = l.out_hw()
+            rows, cols = self.batch * ho * wo, l.C_out
         else:
             rows, cols = self.batch, l.n_out
         wpr = (cols + 31) // 32

@@ -34,9 +34,15 @@ bool valid_layer(const mw_layer_desc& d, int idx, int L) {
   if (d.act < MW_ACT_NONE || d.act > MW_ACT_RELU) return false;
   if (d.kind == MW_DENSE) return d.n_in > 0 && d.n_in == d.n_out;
   if (d.kind == MW_HEAD_LINEAR) return idx == L - 1 && d.n_in > 0 && d.n_out > 0 && d.act == MW_ACT_NONE;
-  if (d.kind == MW_CONV2D)
-    return d.H > 0 && d.W > 0 && d.C_in > 0 && d.C_in == d.C_out && d.stride == 1 && d.k >= 1 &&
-           d.k == 2 * d.pad + 1;
+  if (d.kind == MW_CONV2D) {
+    if (!(d.H > 0 && d.W > 0 && d.C_in > 0 && d.C_in == d.C_out && d.k >= 1 && d.pad >= 0 && d.stride >= 1))
+      return false;
+    // same-size stride-1 layers (vijp by iteration on the centre tap), or Lemma 1 (i)
+    if (d.stride == 1) return d.k == 2 * d.pad + 1;
+    if (!(d.k > d.pad && d.stride > d.pad && d.H + 2 * d.pad >= d.k && d.W + 2 * d.pad >= d.k)) return false;
+    const int Ho = (d.H + 2 * d.pad - d.k) / d.stride + 1, Wo = (d.W + 2 * d.pad - d.k) / d.stride + 1;
+    return d.H > d.stride * (Ho - 1) && d.W > d.stride * (Wo - 1);
+  }
   return false;
 }
 
@@ -165,9 +171,10 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
     const mw_layer_desc& d = n->layers[l];
     LayerInfo& li = n->info[l];
     if (d.kind == MW_CONV2D) {
-      li.rows = (int64_t)batch * d.H * d.W;
+      const int Ho = (d.H + 2 * d.pad - d.k) / d.stride + 1, Wo = (d.W + 2 * d.pad - d.k) / d.stride + 1;
+      li.rows = (int64_t)batch * Ho * Wo;
       li.cols = d.C_out;
-      li.in_elems = li.rows * d.C_in;
+      li.in_elems = (int64_t)batch * d.H * d.W * d.C_in;
       li.out_elems = li.rows * d.C_out;
       li.w_elems = (int64_t)d.k * d.k * d.C_in * d.C_out;
       li.inv_n = d.C_in;
@@ -201,6 +208,15 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
   if (n->backend == MW_BACKEND_SIMT && opts->prec == MW_BF16_F32ACC) {
     delete n;
     return MW_ERR_UNSUPPORTED;
+  }
+  // strided convolutions only have the tensor-core path; a conv net is all of one kind
+  for (int l = 0; l < n_layers; ++l) {
+    const mw_layer_desc& d = n->layers[l];
+    if (d.kind == MW_CONV2D && (d.stride != n->layers[0].stride || n->layers[0].kind != MW_CONV2D ||
+                                (d.stride != 1 && n->backend != MW_BACKEND_TENSOR))) {
+      delete n;
+      return MW_ERR_UNSUPPORTED;
+    }
   }
   build_layout(n, false, n->mwl);
   build_layout(n, true, n->bpl);

@@ -28,6 +28,19 @@ mw_status conv_tensor_backprop(mw_net* n, const void* const* params, const void*
                                const void* target, void* const* dW, double* loss_out, void* ws,
                                cudaStream_t s);
 
+// the fully submersive strided CNN (mw_sconv_pipeline.cu): stride-2 convolutions meeting Lemma 1
+// with 64 or 128 channels, leaky-ReLU or no activation, MW_F32, loss on the last feature map
+bool sconv_tensor_supported(const mw_net* n);
+void sconv_tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start);
+mw_status sconv_tensor_input_cotangent(mw_net* n, const void* const* params, const void* x,
+                                       const void* target, void* g0, double* loss_out, void* ws,
+                                       cudaStream_t s);
+mw_status sconv_tensor_forward_sweep(mw_net* n, const void* const* params, const void* x,
+                                     const void* g0, void* const* dW, void* ws, cudaStream_t s);
+mw_status sconv_tensor_backprop(mw_net* n, const void* const* params, const void* x,
+                                const void* target, void* const* dW, double* loss_out, void* ws,
+                                cudaStream_t s);
+
 // true when every layer of the net has a tensor-core path (dense, sizes multiples of 64,
 // MW_F32 or MW_BF16_F32ACC)
 bool tensor_supported(const mw_net* n);

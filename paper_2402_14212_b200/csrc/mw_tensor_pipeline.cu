@@ -845,7 +845,8 @@ mw_status backprop_program(const Ctx& c, const void* const* params, const void* 
 }  // namespace
 
 bool tensor_supported(const mw_net* n) {
-  if (n->layers[0].kind == MW_CONV2D) return conv_tensor_supported(n);
+  if (n->layers[0].kind == MW_CONV2D)
+    return n->layers[0].stride == 1 ? conv_tensor_supported(n) : sconv_tensor_supported(n);
   if (n->opts.prec != MW_F32 && n->opts.prec != MW_BF16_F32ACC) return false;
   if (n->opts.loss == MW_LOSS_XENT_MEAN) return false;
   const int d = n->layers[0].n_in;
@@ -870,7 +871,8 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     n->tc = t;
   }
   if (n->layers[0].kind == MW_CONV2D) {
-    conv_tensor_layout(n, backprop, lay, start);
+    if (n->layers[0].stride == 1) conv_tensor_layout(n, backprop, lay, start);
+    else sconv_tensor_layout(n, backprop, lay, start);
     return;
   }
   const Prec pr = prec_of(n);
@@ -947,7 +949,8 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
                                  const void* target, void* g0, double* loss_out, void* ws,
                                  cudaStream_t s) {
   if (n->layers[0].kind == MW_CONV2D)
-    return conv_tensor_input_cotangent(n, params, x, target, g0, loss_out, ws, s);
+    return n->layers[0].stride == 1 ? conv_tensor_input_cotangent(n, params, x, target, g0, loss_out, ws, s)
+                                    : sconv_tensor_input_cotangent(n, params, x, target, g0, loss_out, ws, s);
   const Layout& lay = n->mwl;
   Ctx c = make_ctx(n, lay, ws, s);
   const int L = n->L, d = c.dim;
@@ -1015,7 +1018,9 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
 
 mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void* x, const void* g0,
                                void* const* dW, void* ws, cudaStream_t s) {
-  if (n->layers[0].kind == MW_CONV2D) return conv_tensor_forward_sweep(n, params, x, g0, dW, ws, s);
+  if (n->layers[0].kind == MW_CONV2D)
+    return n->layers[0].stride == 1 ? conv_tensor_forward_sweep(n, params, x, g0, dW, ws, s)
+                                    : sconv_tensor_forward_sweep(n, params, x, g0, dW, ws, s);
   const Layout& lay = n->mwl;
   Ctx c = make_ctx(n, lay, ws, s);
   const int L = n->L, d = c.dim;
@@ -1055,7 +1060,8 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
 mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, const void* target,
                           void* const* dW, double* loss_out, void* ws, cudaStream_t s) {
   if (n->layers[0].kind == MW_CONV2D)
-    return conv_tensor_backprop(n, params, x, target, dW, loss_out, ws, s);
+    return n->layers[0].stride == 1 ? conv_tensor_backprop(n, params, x, target, dW, loss_out, ws, s)
+                                    : sconv_tensor_backprop(n, params, x, target, dW, loss_out, ws, s);
   const Layout& lay = n->bpl;
   Ctx c = make_ctx(n, lay, ws, s);
   const int L = n->L, d = c.dim;

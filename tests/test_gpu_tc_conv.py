@@ -78,3 +78,35 @@ def test_strided_conv_products(images, H, W, C, terms):
         assert got.shape == ref.shape
         err = np.abs(got - ref).max() / np.abs(ref).max()
         assert err < tol, (op, err)
+
+
+# ---------------------------------------------------------------------------------------
+# whole path on the fully submersive strided CNN (3x3, stride 2, padding 1; Lemma 1, Algorithm 2)
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("depth,C,H,W,batch,K", [(4, 128, 32, 32, 16, 2), (3, 64, 64, 32, 4, 0),
+                                                 (5, 128, 32, 32, 64, 4), (2, 128, 128, 128, 1, 0)])
+def test_strided_cnn_fp32_tensor_path(depth, C, H, W, batch, K):
+    from paper_2402_14212_b200 import synth as S
+    from parity_util import check_problem
+    p = S.strided_cnn(seed=depth, depth=depth, C=C, H=H, W=W, batch=batch, gamma=0.5, reseed_every=K,
+                      prec=S.F32)
+    out, ref, errs = check_problem(p, 1e-4, backend="tensor", exact_masks=False, tau=1e-4)
+    # the literal Algorithm 1 with Lemma 1's elimination as the vijp reaches the same gradients
+    mw = O.moonwalk(p.layers, p.params, p.x, p.target, p.loss, reseed_every=K,
+                    masks=[m.reshape(z.shape) for m, z in zip(ref["masks"], ref["z"])])
+    for l in range(depth):
+        assert O.normwise_error(mw["dW"][l], ref["dW"][l]) < 1e-7
+
+
+def test_strided_cnn_rejects_non_submersive_anchor():
+    """An anchor tap with an entry above the diagonal violates Lemma 1 (ii): the device status says so."""
+    import torch
+    from paper_2402_14212_b200 import synth as S
+    p = S.strided_cnn(seed=1, depth=2, C=64, H=16, W=16, batch=4, gamma=0.5, reseed_every=0, prec=S.F32)
+    p.params[1][1, 1, 0, 3] = 0.25
+    net = mwb.net_for(p, backend="tensor")
+    params, x, target = mwb.to_device(p)
+    ws = net.alloc_workspace("both")
+    net.input_cotangent(params, x, target, ws)
+    code, detail = net.last_device_status(ws)
+    assert code == mwb.STATUS_NAMES.index("MW_ERR_NOT_SUBMERSIVE")
