@@ -48,6 +48,12 @@ def workload(name: str, seed: int = 0, depth: int = 0):
         return S.sweep_mlp(seed=seed, depth=depth or 32, pool=4)
     if name == "submersive_cnn":
         return S.submersive_cnn(seed=seed)
+    if name == "strided_cnn":
+        # the paper's own convolutional experiment: 256 x 256 x 128 inputs, batch 128, 3x3 stride-2
+        # submersive layers (`depth` of them, 8 by default: down to 1 x 1)
+        return S.strided_cnn(seed=seed, depth=depth or 8)
+    if name == "strided_cnn_small":
+        return S.strided_cnn(seed=seed, depth=depth or 4, H=64, W=64, batch=16)
     if name == "tiny_mlp":
         return S.tiny_mlp(seed=seed)
     raise SystemExit(f"unknown workload {name}")
@@ -57,7 +63,7 @@ def describe(p):
     if p.layers[0].kind == "conv2d":
         l0 = p.layers[0]
         return {"workload": p.name, "layers": len(p.layers), "conv": f"{l0.k}x{l0.k}x{l0.C_in}x{l0.C_out}",
-                "image": f"{l0.H}x{l0.W}", "batch": p.batch, "prec": p.prec, "loss": p.loss,
+                "image": f"{l0.H}x{l0.W}", "stride": l0.stride, "batch": p.batch, "prec": p.prec, "loss": p.loss,
                 "reseed_every": p.reseed_every, "conv_vijp_iters": p.conv_vijp_iters, "seed": p.seed}
     return {"workload": p.name, "layers": len(p.layers), "width": p.layers[0].n_in,
             "batch": p.batch, "prec": p.prec, "loss": p.loss, "reseed_every": p.reseed_every,
@@ -128,17 +134,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def time_oracle(p, seconds_target: float, max_reps: int = 50):
-    """Oracle (as it stands) on the host cores: Algorithm 1 with the same re-seed interval."""
+def time_oracle(p, seconds_target: float, max_reps: int = 50, samples: int = 0):
+    """Oracle (as it stands) on the host cores: Algorithm 1 with the same re-seed interval, on the
+    first `samples` rows of the batch (0 = the whole batch)."""
+    import numpy as np
     from oracle import moonwalk_oracle as O
+    b = samples or p.batch
+    x, t = np.asarray(p.x[:b], dtype=np.float64), p.target[:b]
     reps, t0 = 0, time.perf_counter()
     while True:
-        O.moonwalk(p.layers, p.params, p.x, p.target, p.loss, reseed_every=p.reseed_every)
+        O.moonwalk(p.layers, p.params, x, t, p.loss, reseed_every=p.reseed_every)
         reps += 1
         dt = time.perf_counter() - t0
         if dt >= seconds_target or reps >= max_reps:
             break
-    return p.batch * reps / dt, reps, dt
+    return b * reps / dt, reps, dt, b
 
 
 def blas_threads():
@@ -159,15 +169,16 @@ def run_reference(args):
     from paper_2402_14212_b200 import synth as S
     p = workload(args.workload, depth=args.depth)
     total = args.steps + args.warmup
+    # cost of one sample, then as many rows of the batch as the time budget allows
+    probe = 1 if p.layers[0].kind == "conv2d" else min(8, p.batch)
     t0 = time.perf_counter()
-    O.moonwalk(p.layers, p.params, p.x, p.target, p.loss, reseed_every=p.reseed_every)
-    t_full = time.perf_counter() - t0
+    O.moonwalk(p.layers, p.params, np.asarray(p.x[:probe], dtype=np.float64), p.target[:probe], p.loss,
+               reseed_every=p.reseed_every)
+    t_one = (time.perf_counter() - t0) / probe
     budget = 150.0
-    b = p.batch
-    if t_full * total > budget:      # bounded sample: the first b rows of the batch
-        b = max(8, int(p.batch * budget / (t_full * total)))
-        b = min(b, p.batch)
-    x, t = p.x[:b], p.target[:b]
+    b = int(budget / (t_one * total))
+    b = max(1, min(b, p.batch))
+    x, t = np.asarray(p.x[:b], dtype=np.float64), p.target[:b]
 
     def step():
         O.moonwalk(p.layers, p.params, x, t, p.loss, reseed_every=p.reseed_every)
@@ -277,6 +288,20 @@ def run_ours(args):
     t_cot /= reps
     t_sweep /= reps
 
+    # ---- the library's own backprop on the same inputs (optional: needs its workspace too) ----
+    t_bp = None
+    if args.with_backprop:
+        ws_bp = net.alloc_workspace("backprop", dev)
+        for _ in range(2):
+            net.backprop_reference(params, x, target, ws_bp, dW_out=dW)
+        ev[0].record(stream)
+        for _ in range(reps):
+            net.backprop_reference(params, x, target, ws_bp, dW_out=dW)
+        ev[1].record(stream)
+        torch.cuda.synchronize()
+        t_bp = ev[0].elapsed_time(ev[1]) / reps
+        del ws_bp
+
     # ---- end to end through the C ABI with host buffers --------------------------------------
     xh = x.cpu().pin_memory()
     th = target.cpu().pin_memory()
@@ -328,9 +353,10 @@ def run_ours(args):
     # ---- the oracle on the host cores (rank 0, single GPU only) -----------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, reps_o, dt = time_oracle(p, 10.0)
+        # the large convolutional workload is sampled: one image of the batch through all layers
+        v, reps_o, dt, b_o = time_oracle(p, 10.0, samples=1 if p.name == "strided_cnn" else 0)
         cpu = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-               "sample": f"{reps_o} full steps ({p.batch} samples, {len(p.layers)} layers) in {dt:.1f} s, "
+               "sample": f"{reps_o} steps of {b_o} of {p.batch} samples, all {len(p.layers)} layers, in {dt:.1f} s, "
                          "Algorithm 1 in fp64 numpy"}
 
     if rank == 0:
@@ -348,7 +374,7 @@ def run_ours(args):
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": 8},
                 "roofline": roof, "cpu_baseline": cpu,
-                "phases_ms": {"prep_phase1_phase2": t_cot, "forward_sweep": t_sweep},
+                "phases_ms": {"prep_phase1_phase2": t_cot, "forward_sweep": t_sweep, "backprop": t_bp},
                 "memory_bytes": {"moonwalk_workspace": mw_bytes, "backprop_workspace": bp_bytes,
                                  "moonwalk_residual": mw_res, "backprop_residual": bp_res,
                                  "params": sum(w.numel() * w.element_size() for w in params),
@@ -470,6 +496,8 @@ def main():
     ap.add_argument("--workload", default="deep_mlp")
     ap.add_argument("--backend", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--with-backprop", action="store_true",
+                    help="also time mw_backprop_reference on the same inputs (phases_ms.backprop)")
     ap.add_argument("--depth", type=int, default=0, help="depth of the sweep_mlp workload")
     ap.add_argument("--depth-sweep", action="store_true",
                     help="config 5: peak memory and samples/s versus depth, Moonwalk against the "
