@@ -203,7 +203,10 @@ mw_status loss_top(const SCtx& c, const void* target, double* loss_out) {
 
 // h_l = TransposeConv(g_z(l), w_l) through its parity classes, one launch; `e` is the epilogue of
 // every class
-mw_status transpose_classes(const SCtx& c, int l, const __nv_bfloat16* gz, const TcEpilogue& e) {
+// `checkpoint` (optional): term planes of h_l at the pixels (s*y, s*x), which is all the vijp of
+// layer l reads of it; they are the rows of class (0, 0)
+mw_status transpose_classes(const SCtx& c, int l, const __nv_bfloat16* gz, const TcEpilogue& e,
+                            __nv_bfloat16* checkpoint) {
   const ConvGeom g = c.geom(l);
   TcGemm cls[kTcMaxGroup];
   int n = 0;
@@ -212,6 +215,10 @@ mw_status transpose_classes(const SCtx& c, int l, const __nv_bfloat16* gz, const
       if (n == kTcMaxGroup) return MW_ERR_UNSUPPORTED;
       if (!conv_transpose_class_product(g, py, px, gz, 3, c.at<__nv_bfloat16>(c.lay->cw[l]), 3, e, &cls[n]))
         return MW_ERR_UNSUPPORTED;
+      if (checkpoint && py == 0 && px == 0) {
+        TcEpilogue& ce = cls[n].epi;
+        ce.planes2 = checkpoint; ce.n_planes2 = 3; ce.plane_stride2 = c.out_elems(l); ce.compact2 = 1;
+      }
       ++n;
     }
   return tc_gemm_group(c.cache, cls, n, c.st, c.s);
@@ -235,7 +242,6 @@ mw_status backward_pass(const SCtx& c, void* g0, void* const* dW, bool checkpoin
       e.out_f32 = (float*)g0;
     } else {
       const mw_layer_desc& below = c.n->layers[l - 1];
-      if (checkpoints && is_reseed(c.n, l)) e.out_f32 = c.at<float>(lay.reseed[l]);
       e.act = below.act;
       e.slope = (float)below.slope;
       e.mask = c.at<uint32_t>(lay.mask[l - 1]);
@@ -243,7 +249,8 @@ mw_status backward_pass(const SCtx& c, void* g0, void* const* dW, bool checkpoin
       e.n_planes = 3;
       e.plane_stride = c.in_elems(l);
     }
-    MW_TRY(transpose_classes(c, l, gz, e));
+    MW_TRY(transpose_classes(c, l, gz, e, l > 0 && checkpoints && is_reseed(c.n, l)
+                                                ? c.at<__nv_bfloat16>(lay.reseed[l]) : nullptr));
     cur ^= 1;
   }
   return MW_OK;
@@ -326,7 +333,7 @@ mw_status sconv_tensor_forward_sweep(mw_net* n, const void* const* params, const
   const Layout& lay = n->mwl;
   SCtx c = make_sctx(n, lay, ws, s);
   const int L = c.L, C = c.C;
-  MW_TRY(split_planes((const float*)x, c.in_elems(0), x_planes(c, 0), 3, c.in_elems(0), s));
+  (void)x;   // its term planes (xp[0]) are still those Phase I made from the same x
   {
     // only the pixels s*i' of the input cotangent enter the vijp: split those
     const mw_layer_desc& d = n->layers[0];
@@ -336,12 +343,13 @@ mw_status sconv_tensor_forward_sweep(mw_net* n, const void* const* params, const
         (const float*)g0, Ho, Wo, d.stride, C / 4, n4, c.at<__nv_bfloat16>(lay.hp[0]), 3, c.out_elems(0));
     MW_TRY(launch_ok());
   }
+  const __nv_bfloat16* hcur = c.at<__nv_bfloat16>(lay.hp[0]);
   for (int l = 0; l < L; ++l) {
     const mw_layer_desc& ld = n->layers[l];
     const ConvGeom g = c.geom(l);
     uint32_t* words = c.at<uint32_t>(lay.mask[l]);
     const __nv_bfloat16* xin = x_planes(c, l);
-    const __nv_bfloat16* hin = c.at<__nv_bfloat16>(lay.hp[l & 1]);
+    const __nv_bfloat16* hin = hcur;
     __nv_bfloat16* hout = c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]);
     const bool more = l + 1 < L;
     const bool reseed_next = more && is_reseed(n, l + 1);
@@ -363,25 +371,23 @@ mw_status sconv_tensor_forward_sweep(mw_net* n, const void* const* params, const
       p.B.base = c.at<__nv_bfloat16>(lay.cwinv[l]); p.B.rows = C; p.B.cols = C; p.B.planes = 3;
       p.B.plane_stride = (int64_t)C * C; p.B.mn_major = false;
       p.M = (int)g.out_pixels(); p.N = C; p.K = C;
-      if (l == 0) {
-        p.A = pixel_operand(hin, g.out_pixels(), 3, c.out_elems(0), false, C);     // already subsampled
-      } else {
-        p.A = pixel_operand(hin, g.pixels(), 3, c.in_elems(l), false, C);
-        p.conv.mode = TC_CONV_PIXELS; p.conv.H = g.H; p.conv.W = g.W; p.conv.C = C;
-        p.conv.stride = g.stride; p.conv.Ho = g.Ho(); p.conv.Wo = g.Wo();
-        p.conv.ntaps = 1;                               // the window is the pixel s*i' itself
-      }
+      // h_l is kept at the pixels s*i' only (all that the elimination reads)
+      p.A = pixel_operand(hin, g.out_pixels(), 3, c.out_elems(l), false, C);
       TcEpilogue& e = p.epi;
       e.mode = TC_EPI_VIJP;
       e.act = ld.act;
       e.slope = (float)ld.slope;
       e.mask = words;
-      if (want_h) { e.planes2 = hout; e.n_planes2 = 3; e.plane_stride2 = c.out_elems(l); }
+      if (want_h) {
+        const mw_layer_desc& nd = n->layers[l + 1];
+        e.planes2 = hout; e.n_planes2 = 3; e.plane_stride2 = c.out_elems(l + 1);
+        e.sub2_s = nd.stride; e.sub2_h = nd.H; e.sub2_w = nd.W;
+      }
       if (dW[l]) { e.planes = c.at<__nv_bfloat16>(lay.cg[0]); e.n_planes = 2; e.plane_stride = c.out_elems(l); }
       MW_TRY(tc_gemm_group(c.cache, &p, 1, c.st, s));
     }
-    if (reseed_next)   // the recursion restarts from the stored cotangent h_{l+1}
-      MW_TRY(split_planes(c.at<float>(lay.reseed[l + 1]), c.out_elems(l), hout, 3, c.out_elems(l), s));
+    // the recursion restarts from the stored cotangent h_{l+1} (term planes) where there is one
+    hcur = reseed_next ? c.at<__nv_bfloat16>(lay.reseed[l + 1]) : hout;
     if (dW[l])
       MW_TRY(conv_wgrad_tensor(c.cache, g, xin, c.at<__nv_bfloat16>(lay.cg[0]), 2, c.at<float>(lay.cpart),
                                (float*)dW[l], c.st, s));

@@ -261,7 +261,8 @@ __device__ __forceinline__ uint32_t frag_base(const TcEpilogue& e, int N, int ro
 }
 
 // the fused step applied to one row chunk of 32 accumulator columns
-__device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int row, int col0,
+// (`prow`: the row inside the product, `row`: where its outputs live; they differ under a scatter)
+__device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int prow, int row, int col0,
                                                float (&v)[32], double& sumsq_local) {
   const int64_t off = (int64_t)row * N + col0;
   const int64_t woff = (int64_t)row * (N >> 5) + (col0 >> 5);
@@ -322,7 +323,8 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int r
         float h[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) h[i] = v[i];
-        store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, off);
+        store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2,
+                       e.compact2 ? (int64_t)prow * N + col0 : off);
       }
       const uint32_t word = e.act != MW_ACT_NONE ? e.mask[woff] : 0xffffffffu;
       if (e.act == MW_ACT_RELU && e.frag_vals) {
@@ -378,7 +380,20 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int r
         for (int i = 0; i < 32; ++i) h[i] = v[i];
       }
       if (e.out_f32) store_f32x32(h, e.out_f32 + off);
-      if (e.n_planes2) store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, off);
+      if (e.n_planes2) {
+        if (e.sub2_s) {
+          const int hw = e.sub2_h * e.sub2_w;
+          const int b = prow / hw, rem = prow - b * hw;
+          const int y = rem / e.sub2_w, x = rem - y * e.sub2_w;
+          if (y % e.sub2_s == 0 && x % e.sub2_s == 0) {
+            const int64_t r2 = ((int64_t)b * (e.sub2_h / e.sub2_s) + y / e.sub2_s) * (e.sub2_w / e.sub2_s) +
+                               x / e.sub2_s;
+            store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, r2 * N + col0);
+          }
+        } else {
+          store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, off);
+        }
+      }
       if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off);
       break;
     }
@@ -783,7 +798,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           } else {
             load_chunk(c, v);
           }
-          if (row < P.M) epilogue_chunk(epi, N, orow, w.n0 + c, v, sumsq_local);
+          if (row < P.M) epilogue_chunk(epi, N, row, orow, w.n0 + c, v, sumsq_local);
         }
       }
       (void)nchunk;

@@ -76,6 +76,12 @@ struct TcEpilogue {
   // remap_s*x + remap_px) of the remap_s times larger image: one parity class of a strided
   // TransposeConv
   int remap_s = 0, remap_ho = 0, remap_wo = 0, remap_py = 0, remap_px = 0;
+  // TC_EPI_BWD with a row scatter: planes2 is addressed by the product's own row all the same
+  // (the class of the pixels (s*y, s*x) written densely: all that a strided vijp reads of h)
+  int compact2 = 0;
+  // TC_EPI_VIJP (sub2_s > 0): the rows are pixels of sub2_h x sub2_w images and planes2 keeps
+  // only the pixels (sub2_s*y, sub2_s*x), densely: [images][sub2_h/s][sub2_w/s][N]
+  int sub2_s = 0, sub2_h = 0, sub2_w = 0;
 };
 
 // Convolution forms of a product.  The A operand is then a channel-last pixel array
