@@ -110,3 +110,47 @@ def test_strided_cnn_rejects_non_submersive_anchor():
     net.input_cotangent(params, x, target, ws)
     code, detail = net.last_device_status(ws)
     assert code == mwb.STATUS_NAMES.index("MW_ERR_NOT_SUBMERSIVE")
+
+
+def test_strided_cnn_full_size():
+    """The paper's experiment at full size (256 x 256 x 128 inputs, batch 128, 8 stride-2 layers), in
+    the launch configuration the benchmark times.  The oracle handles the batch in slices (samples
+    are independent but for the batch sums of dW and of the loss), replaying the GPU's sign bits."""
+    import torch
+    from paper_2402_14212_b200 import synth as S
+    from parity_util import run_gpu
+    p = S.strided_cnn(seed=0)
+    out = run_gpu(p, backend="tensor", backprop=False)
+    assert out["status"] == 0
+    L, B = len(p.layers), p.batch
+    n_last = p.target[0].size
+    dW = [np.zeros_like(w) for w in p.params]
+    loss, g0_err, worst = 0.0, 0.0, [0.0] * L
+    step = 8
+    for b0 in range(0, B, step):
+        sl = slice(b0, b0 + step)
+        masks = []
+        for l, layer in enumerate(p.layers):
+            ho, wo = layer.out_hw()
+            words = out["masks"][l].reshape(B, ho * wo, -1)[sl].reshape(step * ho * wo, -1)
+            masks.append(O.unpack_mask(words, layer.C_out).reshape(step, ho, wo, layer.C_out))
+        x = np.asarray(p.x[sl], dtype=np.float64)
+        ref = O.backprop(p.layers, p.params, x, p.target[sl], p.loss, masks=masks)
+        # mse_mean divides by the elements of ITS batch: rescale the slice to the whole batch
+        f = step / B
+        loss += ref["loss"] * f
+        for l in range(L):
+            dW[l] += ref["dW"][l] * f
+            z = ref["z"][l].reshape(-1, p.layers[l].C_out)
+            d = masks[l].reshape(z.shape) != O.sign_mask(z)
+            if d.any():
+                rms = np.sqrt((z * z).mean(axis=1, keepdims=True))
+                worst[l] = max(worst[l], float((np.abs(z) / rms)[d].max()))
+        g = out["g0"][sl].reshape(ref["g0"].shape)
+        g0_err = max(g0_err, float(np.abs(g - ref["g0"] * f).max()))
+    g0_scale = float(np.abs(out["g0"]).max())
+    assert g0_err <= 1e-4 * g0_scale, g0_err / g0_scale
+    for l in range(L):
+        assert worst[l] <= 1e-4 * np.sqrt(l + 1.0), (l, worst[l])
+        assert O.normwise_error(out["dW"][l], dW[l]) <= 1e-4, l
+    assert abs(out["loss"] - loss) <= 1e-4 * abs(loss)
