@@ -241,13 +241,16 @@ def run_ours(args):
     params, x, target = mwb.to_device(p, dev)
     ws = net.alloc_workspace("moonwalk", dev)
     mw_bytes, bp_bytes, (mw_res, bp_res) = net.workspace_bytes()
-    g0 = torch.empty(x.shape, dtype=net.grad_dtype(), device=dev)
+    # nets of strided submersive convolutions keep the part of g0 that the sweep reads inside the
+    # workspace (mw_input_cotangent with g0_out = NULL); the others hand g0 over in full
+    lean = p.layers[0].kind == "conv2d" and p.layers[0].stride != 1 and not args.full_g0
+    g0 = None if lean else torch.empty(x.shape, dtype=net.grad_dtype(), device=dev)
     dW = [torch.empty(w.shape, dtype=net.grad_dtype(), device=dev) for w in params]
     loss = torch.zeros(1, dtype=torch.float64, device=dev)
     stream = torch.cuda.current_stream()
 
     def step():
-        net.input_cotangent(params, x, target, ws, g0_out=g0, loss_out=loss)
+        net.input_cotangent(params, x, target, ws, g0_out=g0, loss_out=loss, keep_seed=lean)
         net.forward_sweep(params, x, g0, ws, dW_out=dW)
 
     for _ in range(max(args.warmup, 3)):
@@ -278,7 +281,7 @@ def run_ours(args):
     t_cot = t_sweep = 0.0
     for _ in range(reps):
         ev[0].record(stream)
-        net.input_cotangent(params, x, target, ws, g0_out=g0, loss_out=loss)
+        net.input_cotangent(params, x, target, ws, g0_out=g0, loss_out=loss, keep_seed=lean)
         ev[1].record(stream)
         net.forward_sweep(params, x, g0, ws, dW_out=dW)
         ev[2].record(stream)
@@ -496,6 +499,8 @@ def main():
     ap.add_argument("--workload", default="deep_mlp")
     ap.add_argument("--backend", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--full-g0", action="store_true",
+                    help="strided CNN workloads: have mw_input_cotangent return g0 in full")
     ap.add_argument("--with-backprop", action="store_true",
                     help="also time mw_backprop_reference on the same inputs (phases_ms.backprop)")
     ap.add_argument("--depth", type=int, default=0, help="depth of the sweep_mlp workload")

@@ -92,8 +92,12 @@ typedef struct {
 } mw_net_opts;
 
 /* Build a host-side description.  `batch` is fixed per net.  Returns MW_ERR_UNSUPPORTED for
- * shapes outside: dense layers square; convolutions stride 1, k = 2*pad+1, C_in = C_out;
- * head only as the last layer; all layers of one net share `prec`. */
+ * shapes outside: dense layers square; convolutions with C_in = C_out, either stride 1 with
+ * k = 2*pad+1 (same size), or every layer of the net meeting Lemma 1 (i) with stride 2 (the
+ * paper's submersive CNN: MW_F32, 64 or 128 channels, k - 1 - pad < 2, even image sizes, a
+ * loss on the last feature map; conditions (ii) and (iii) on the anchor tap w[pad][pad] are
+ * checked on the device every step: MW_ERR_NOT_SUBMERSIVE); head only as the last layer; all
+ * layers of one net share `prec`. */
 mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers, int32_t batch,
                         const mw_net_opts* opts, mw_net** out);
 void mw_net_destroy(mw_net* net);
@@ -109,7 +113,11 @@ mw_status mw_workspace_bytes(const mw_net* net, size_t* moonwalk_bytes, size_t* 
  *   params       host array of n_layers DEVICE pointers to the weights (read-only).
  *   x            device, [B][n_0] (or NHWC), storage type of `prec`.
  *   loss_target  device, see mw_loss.
- *   g0_out       device, [B][n_0], double (MW_F64) or float.
+ *   g0_out       device, [B][n_0], double (MW_F64) or float.  May be NULL for a net of strided
+ *                submersive convolutions: the vijp of such a layer (Lemma 1) reads the input
+ *                cotangent at the pixels (s*y, s*x) only, so only those are then computed
+ *                (one ninth of the first layer's TransposeConv for k = 3) and kept in the
+ *                workspace; call mw_forward_sweep with g0 = NULL.
  *   loss_out     device pointer to one double receiving J, or NULL.
  * Also fills the workspace with the residual stores the sweep consumes. */
 mw_status mw_input_cotangent(mw_net* net, const void* const* params, const void* x,
@@ -120,7 +128,10 @@ mw_status mw_input_cotangent(mw_net* net, const void* const* params, const void*
  *   dW_out  host array of n_layers DEVICE pointers, each shaped like its weight, double
  *           (MW_F64) or float; overwritten.  A NULL entry skips storing that layer's gradient
  *           (gradients need not coexist, Section 4.3 last paragraph but one).
- * Requires the workspace last written by mw_input_cotangent on the same net (MW_ERR_STATE). */
+ *   g0      the result of mw_input_cotangent; NULL where that call allows g0_out = NULL: the sweep
+ *           then starts from the part of g0 that call left in the workspace.
+ * Requires the workspace last written by mw_input_cotangent on the same net, with the same x,
+ * unchanged since (MW_ERR_STATE where that can be told). */
 mw_status mw_forward_sweep(mw_net* net, const void* const* params, const void* x, const void* g0,
                            void* const* dW_out, void* workspace, size_t workspace_bytes,
                            void* stream);
@@ -189,7 +200,7 @@ mw_status mw_gemm_split_bf16(const float* A, int32_t a_mn, const float* B, int32
  * Pixel arrays are channel-last float [images][H][W][64], kernels float [k][k][64][64], p = k/2,
  * zero padding; all device memory.  terms as in mw_gemm_split_bf16.  Sizes: 128 % W == 0 (64 % W
  * == 0 for op 2), H*W % 128 == 0, k odd.  scratch: device, 256-byte aligned, >= 1024 + 8*terms*
- * (elements of a + elements of b) bytes (+ 32 * k*k*16 KiB for op 2).  Synchronises `stream`. */
+ * (elements of a + elements of b) bytes (+ 256 * k*k*16 KiB for op 2).  Synchronises `stream`. */
 mw_status mw_conv2d_split_bf16(int32_t op, const float* a, const float* b, float* out,
                                int32_t images, int32_t H, int32_t W, int32_t k, int32_t terms,
                                void* scratch, size_t scratch_bytes, void* stream);
@@ -204,7 +215,7 @@ mw_status mw_conv2d_split_bf16(int32_t op, const float* a, const float* b, float
  * A tile of 128 consecutive product pixels (64 for op 2) must be part of an image row, whole rows
  * of one image, or whole images (widths and heights that are powers of two up to 256 qualify);
  * images*Ho*Wo % 64 == 0 for op 2.  Otherwise MW_ERR_UNSUPPORTED.  scratch: device, 256-byte
- * aligned, >= 1024 + 8*terms*(elements of a + elements of b) + (op 2: 128 * k*k*C*C) bytes.
+ * aligned, >= 1024 + 8*terms*(elements of a + elements of b) + (op 2: 1024 * k*k*C*C) bytes.
  * Synchronises `stream`. */
 mw_status mw_conv2d_strided_split_bf16(int32_t op, const float* a, const float* b, float* out,
                                        int32_t images, int32_t H, int32_t W, int32_t C, int32_t k,

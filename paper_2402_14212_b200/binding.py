@@ -176,9 +176,12 @@ class Net:
         return ap, workspace.numel() - (ap - p)
 
     # ---- the three calls ------------------------------------------------------------------
-    def input_cotangent(self, params, x, target, workspace, g0_out=None, loss_out=None, stream=None):
+    def input_cotangent(self, params, x, target, workspace, g0_out=None, loss_out=None, stream=None,
+                        keep_seed=False):
+        """keep_seed (nets of strided submersive convolutions only): g0 is not returned; the part
+        of it that the sweep reads stays in the workspace (call forward_sweep with g0 = None)."""
         import torch
-        if g0_out is None:
+        if g0_out is None and not keep_seed:
             g0_out = torch.empty(x.shape, dtype=self.grad_dtype(), device=x.device)
         wp, wb = self._ws(workspace)
         _check(lib().mw_input_cotangent(self._h, _ptr_array(params), _ptr(x), _ptr(target),
@@ -315,7 +318,7 @@ def conv2d_split_bf16(op: int, a, b, k: int, terms: int, stream=None):
     assert C == 64
     out = torch.empty((k, k, 64, 64) if op == 2 else (images, H, W, 64), dtype=torch.float32,
                       device=a.device)
-    n = 1024 + 8 * terms * (a.numel() + b.numel()) + 32 * k * k * 16384 + 4096
+    n = 1024 + 8 * terms * (a.numel() + b.numel()) + 256 * k * k * 16384 + 4096
     scratch = torch.empty(n, dtype=torch.uint8, device=a.device)
     _check(lib().mw_conv2d_split_bf16(op, _ptr(a), _ptr(b), _ptr(out), images, H, W, k, int(terms),
                                       _ptr(scratch), scratch.numel(), _stream_handle(stream)),
@@ -336,7 +339,7 @@ def conv2d_strided_split_bf16(op: int, a, b, k: int, stride: int, pad: int, term
     Ho, Wo = (H + 2 * pad - k) // stride + 1, (W + 2 * pad - k) // stride + 1
     shape = {0: (images, Ho, Wo, C), 1: (images, H, W, C), 2: (k, k, C, C)}[op]
     out = torch.empty(shape, dtype=torch.float32, device=a.device)
-    n = 1024 + 8 * terms * (a.numel() + b.numel()) + 128 * k * k * C * C + 4096
+    n = 1024 + 8 * terms * (a.numel() + b.numel()) + 1024 * k * k * C * C + 4096
     scratch = torch.empty(n, dtype=torch.uint8, device=a.device)
     _check(lib().mw_conv2d_strided_split_bf16(op, _ptr(a), _ptr(b), _ptr(out), images, H, W, C, k,
                                               stride, pad, int(terms), _ptr(scratch), scratch.numel(),

@@ -220,6 +220,7 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
   }
   build_layout(n, false, n->mwl);
   build_layout(n, true, n->bpl);
+  n->lean_seed = n->backend == MW_BACKEND_TENSOR && n->layers[0].kind == MW_CONV2D && n->layers[0].stride != 1;
   *out = n;
   return MW_OK;
 }
@@ -496,7 +497,8 @@ mw_status simt_backprop(mw_net* n, const void* const* params, const T* x, const 
 extern "C" mw_status mw_input_cotangent(mw_net* net, const void* const* params, const void* x,
                                         const void* loss_target, void* g0_out, double* loss_out,
                                         void* workspace, size_t workspace_bytes, void* stream) {
-  if (!net || !params || !x || !loss_target || !g0_out) return MW_ERR_INVALID_ARG;
+  if (!net || !params || !x || !loss_target) return MW_ERR_INVALID_ARG;
+  if (!g0_out && !net->lean_seed) return MW_ERR_INVALID_ARG;
   for (int l = 0; l < net->L; ++l)
     if (!params[l]) return MW_ERR_INVALID_ARG;
   MW_TRY(check_ws(workspace, workspace_bytes, net->mwl.total));
@@ -521,7 +523,8 @@ extern "C" mw_status mw_input_cotangent(mw_net* net, const void* const* params, 
 extern "C" mw_status mw_forward_sweep(mw_net* net, const void* const* params, const void* x,
                                       const void* g0, void* const* dW_out, void* workspace,
                                       size_t workspace_bytes, void* stream) {
-  if (!net || !params || !x || !g0 || !dW_out) return MW_ERR_INVALID_ARG;
+  if (!net || !params || !x || !dW_out) return MW_ERR_INVALID_ARG;
+  if (!g0 && !net->lean_seed) return MW_ERR_INVALID_ARG;
   for (int l = 0; l < net->L; ++l)
     if (!params[l]) return MW_ERR_INVALID_ARG;
   MW_TRY(check_ws(workspace, workspace_bytes, net->mwl.total));
@@ -639,8 +642,8 @@ extern "C" mw_status mw_gradient_step_host(mw_net* net, const void* const* param
                                            void* const* dW_out, double* loss_dev,
                                            double* loss_host, void* workspace,
                                            size_t workspace_bytes, void* stream) {
-  if (!net || !x_host || !target_host || !x_dev || !target_dev || !g0_dev || !loss_dev || !loss_host)
-    return MW_ERR_INVALID_ARG;
+  if (!net || !x_host || !target_host || !x_dev || !target_dev || !loss_dev || !loss_host)
+    return MW_ERR_INVALID_ARG;   // g0_dev: as g0_out of mw_input_cotangent
   cudaStream_t s = (cudaStream_t)stream;
   MW_CUDA_OK(cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, s));
   MW_CUDA_OK(cudaMemcpyAsync(target_dev, target_host, target_bytes, cudaMemcpyHostToDevice, s));

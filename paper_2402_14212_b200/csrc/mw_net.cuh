@@ -34,7 +34,7 @@ struct Layout {
   Region xp[3], hp[2], gzp[2], ns_r, ns_x, ns_w; // activation / cotangent / g_z planes, NS scratch
   // convolution nets on the tensor cores
   std::vector<Region> cw, cwhat, cwinv;      // per layer: kernel, folded kernel, centre-tap inverse (term planes)
-  Region cwinv_f32, cwhat_f32, cg[2], chpf, cxf, cpart, clogits;
+  Region cwinv_f32, cwhat_f32, cg[2], chpf, cxf, cpart, clogits, cseed;
   Region ns_sumsq;
   Region prog_table[3], prog_done[3];        // product tables and completion counters of program launches
   Region split[3];                           // K-split meeting places of concurrently running products
@@ -54,6 +54,7 @@ struct mw_net {
   const void* ws_done = nullptr;   // workspace that holds a finished Phase I+II
   const void* x_done = nullptr;
   void* tc = nullptr;              // tensor-core backend private state
+  bool lean_seed = false;          // the net can keep the sweep's seed itself (g0 optional)
 };
 
 namespace mw {

@@ -205,13 +205,15 @@ mw_status loss_top(const SCtx& c, const void* target, double* loss_out) {
 // every class
 // `checkpoint` (optional): term planes of h_l at the pixels (s*y, s*x), which is all the vijp of
 // layer l reads of it; they are the rows of class (0, 0)
+// With `only_checkpoint` nothing but those pixels is computed (one class, one ninth of the work).
 mw_status transpose_classes(const SCtx& c, int l, const __nv_bfloat16* gz, const TcEpilogue& e,
-                            __nv_bfloat16* checkpoint) {
+                            __nv_bfloat16* checkpoint, bool only_checkpoint = false) {
   const ConvGeom g = c.geom(l);
   TcGemm cls[kTcMaxGroup];
   int n = 0;
   for (int py = 0; py < g.stride; ++py)
     for (int px = 0; px < g.stride; ++px) {
+      if (only_checkpoint && (py || px)) continue;
       if (n == kTcMaxGroup) return MW_ERR_UNSUPPORTED;
       if (!conv_transpose_class_product(g, py, px, gz, 3, c.at<__nv_bfloat16>(c.lay->cw[l]), 3, e, &cls[n]))
         return MW_ERR_UNSUPPORTED;
@@ -226,7 +228,7 @@ mw_status transpose_classes(const SCtx& c, int l, const __nv_bfloat16* gz, const
 
 // the backward walk shared by Phase II and backprop: for l = L-1 .. 0 (optionally the weight
 // vjp of layer l first) h_l -> g0 / checkpoint, g_z(l-1) planes
-mw_status backward_pass(const SCtx& c, void* g0, void* const* dW, bool checkpoints) {
+mw_status backward_pass(const SCtx& c, void* g0, __nv_bfloat16* seed, void* const* dW, bool checkpoints) {
   const Layout& lay = *c.lay;
   int cur = 0;
   for (int l = c.L - 1; l >= 0; --l) {
@@ -235,11 +237,15 @@ mw_status backward_pass(const SCtx& c, void* g0, void* const* dW, bool checkpoin
       const __nv_bfloat16* xl = l == 0 ? x_planes(c, 0) : c.at<__nv_bfloat16>(lay.stored_act[l]);
       MW_TRY(conv_wgrad_tensor(c.cache, c.geom(l), xl, gz, 2, c.at<float>(lay.cpart), (float*)dW[l], c.st, c.s));
     }
-    if (l == 0 && !g0) break;
+    if (l == 0 && !g0 && !seed) break;
     TcEpilogue e;
     e.mode = TC_EPI_BWD;
     if (l == 0) {
+      // the input cotangent: in full when the caller wants it; the sweep itself only needs its
+      // pixels (s*y, s*x), kept as term planes
       e.out_f32 = (float*)g0;
+      MW_TRY(transpose_classes(c, 0, gz, e, seed, g0 == nullptr));
+      break;
     } else {
       const mw_layer_desc& below = c.n->layers[l - 1];
       e.act = below.act;
@@ -310,6 +316,8 @@ void sconv_tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
   lay.cpart = b.take(part);
   if (!backprop) {
     lay.cg[0] = b.take(2 * 2 * P1);                     // g_z planes of the sweep (two terms)
+    lay.cseed = b.take(2 * 3 * P1);                     // h_0 at the pixels (s*y, s*x): survives to the sweep
+    lay.residual += 2 * 3 * P1;
     for (int l = 0; l < L; ++l) lay.cwinv[l] = b.take(2 * 3 * (size_t)C * C);
     lay.cwinv_f32 = b.take(4 * (size_t)C * C * kSmallBatch);
   }
@@ -324,7 +332,7 @@ mw_status sconv_tensor_input_cotangent(mw_net* n, const void* const* params, con
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
   MW_TRY(forward_pass(c, params, x, false));          // Phase I (+ per-step preparation)
   MW_TRY(loss_top(c, target, loss_out));
-  return backward_pass(c, g0, nullptr, true);          // Phase II
+  return backward_pass(c, g0, c.at<__nv_bfloat16>(lay.cseed), nullptr, true);   // Phase II
 }
 
 mw_status sconv_tensor_forward_sweep(mw_net* n, const void* const* params, const void* x,
@@ -334,7 +342,8 @@ mw_status sconv_tensor_forward_sweep(mw_net* n, const void* const* params, const
   SCtx c = make_sctx(n, lay, ws, s);
   const int L = c.L, C = c.C;
   (void)x;   // its term planes (xp[0]) are still those Phase I made from the same x
-  {
+  const __nv_bfloat16* hcur = c.at<__nv_bfloat16>(lay.cseed);   // Phase II's own seed
+  if (g0) {
     // only the pixels s*i' of the input cotangent enter the vijp: split those
     const mw_layer_desc& d = n->layers[0];
     const int Ho = d.H / d.stride, Wo = d.W / d.stride;
@@ -342,15 +351,15 @@ mw_status sconv_tensor_forward_sweep(mw_net* n, const void* const* params, const
     split_subsampled_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(
         (const float*)g0, Ho, Wo, d.stride, C / 4, n4, c.at<__nv_bfloat16>(lay.hp[0]), 3, c.out_elems(0));
     MW_TRY(launch_ok());
+    hcur = c.at<__nv_bfloat16>(lay.hp[0]);
   }
-  const __nv_bfloat16* hcur = c.at<__nv_bfloat16>(lay.hp[0]);
   for (int l = 0; l < L; ++l) {
     const mw_layer_desc& ld = n->layers[l];
     const ConvGeom g = c.geom(l);
     uint32_t* words = c.at<uint32_t>(lay.mask[l]);
     const __nv_bfloat16* xin = x_planes(c, l);
     const __nv_bfloat16* hin = hcur;
-    __nv_bfloat16* hout = c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]);
+    __nv_bfloat16* hout = c.at<__nv_bfloat16>(lay.hp[(l + 1) & 1]);   // l = 0 reads hp[0] or the seed
     const bool more = l + 1 < L;
     const bool reseed_next = more && is_reseed(n, l + 1);
     const bool want_h = more && !reseed_next;
@@ -403,7 +412,7 @@ mw_status sconv_tensor_backprop(mw_net* n, const void* const* params, const void
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
   MW_TRY(forward_pass(c, params, x, true));
   MW_TRY(loss_top(c, target, loss_out));
-  return backward_pass(c, nullptr, dW, false);
+  return backward_pass(c, nullptr, nullptr, dW, false);
 }
 
 }  // namespace mw

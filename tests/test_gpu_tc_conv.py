@@ -98,6 +98,31 @@ def test_strided_cnn_fp32_tensor_path(depth, C, H, W, batch, K):
         assert O.normwise_error(mw["dW"][l], ref["dW"][l]) < 1e-7
 
 
+def test_strided_cnn_lean_seed_gives_the_same_gradients():
+    """With g0_out = NULL only the pixels (s y, s x) of the input cotangent are computed and kept in
+    the workspace; the sweep started from them returns the same gradients (the seed holds the same
+    values, split into term planes by the product's epilogue instead of a separate kernel)."""
+    import torch
+    from paper_2402_14212_b200 import synth as S
+    p = S.strided_cnn(seed=3, depth=4, C=128, H=32, W=32, batch=16, gamma=0.5, reseed_every=2, prec=S.F32)
+    net = mwb.net_for(p, backend="tensor")
+    params, x, target = mwb.to_device(p)
+    ws = net.alloc_workspace("moonwalk")
+    g0 = net.input_cotangent(params, x, target, ws)
+    dW_full = [d.clone() for d in net.forward_sweep(params, x, g0, ws)]
+    assert net.input_cotangent(params, x, target, ws, keep_seed=True) is None
+    dW_lean = net.forward_sweep(params, x, None, ws)
+    assert net.last_device_status(ws)[0] == 0
+    for a, b in zip(dW_full, dW_lean):
+        assert float((a - b).abs().max()) <= 1e-6 * float(a.abs().max())
+    # a dense net has no such part to keep: g0 is required
+    q = S.deep_mlp(seed=0, depth=2, n=64, batch=64)
+    dn = mwb.net_for(q, backend="tensor")
+    qp, qx, qt = mwb.to_device(q)
+    with pytest.raises(mwb.MwError):
+        dn.input_cotangent(qp, qx, qt, dn.alloc_workspace("moonwalk"), keep_seed=True)
+
+
 def test_strided_cnn_rejects_non_submersive_anchor():
     """An anchor tap with an entry above the diagonal violates Lemma 1 (ii): the device status says so."""
     import torch
