@@ -124,6 +124,18 @@ mw_status mw_input_cotangent(mw_net* net, const void* const* params, const void*
                              const void* loss_target, void* g0_out, double* loss_out,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/* Phase III with the last line of Algorithm 1 ("apply g_i to theta_i") fused into the weight vjp:
+ * params_out[l] = params[l] - lr * g_l for every layer, written by the epilogue of the product that
+ * forms g_l, so that no gradient buffer exists (gradients need not coexist, Section 4.3).
+ * params_out[l] (device, float, shaped like the weight) may be params[l] itself: the products of
+ * the sweep read the term planes Phase I made of the weights, never params again (with
+ * resident_inverse = 0 layer l's weight is read just before its own update).  A NULL entry skips
+ * that layer.  MW_F32 nets on the tensor-core backend; otherwise MW_ERR_UNSUPPORTED.  Other
+ * arguments, requirements and errors as for mw_forward_sweep. */
+mw_status mw_forward_sweep_apply(mw_net* net, const void* const* params, const void* x,
+                                 const void* g0, double lr, void* const* params_out,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
 /* Phase III (Algorithm 1): all parameter gradients from x and g0.
  *   dW_out  host array of n_layers DEVICE pointers, each shaped like its weight, double
  *           (MW_F64) or float; overwritten.  A NULL entry skips storing that layer's gradient

@@ -397,10 +397,11 @@ def input_cotangent(layers, params, x0, target, loss, reseed_every=0, masks=None
     return h, store
 
 
-def forward_sweep(layers, params, x0, g0, store, conv_iters=None):
+def forward_sweep(layers, params, x0, g0, store, conv_iters=None, apply=None):
     """Phase III = the loop body of Algorithm 1: x_i = f_i(x_{i-1}); h_i = vijp(f_i, x_{i-1},
-    h_{i-1}) (Eq. "h_i"); g_i = vjp(f_i, theta_i, h_i) (Eq. "g_i").  The last layer's output
-    cotangent is the loss cotangent itself when that layer has no vijp (classification head)."""
+    h_{i-1}) (Eq. "h_i"); g_i = vjp(f_i, theta_i, h_i) (Eq. "g_i"); "apply g_i to theta_i":
+    `apply(i, g_i)` is called as soon as g_i exists.  The last layer's output cotangent is the
+    loss cotangent itself when that layer has no vijp (classification head)."""
     L = len(layers)
     ms = store["masks"]
     x, h = x0, g0
@@ -422,12 +423,29 @@ def forward_sweep(layers, params, x0, g0, store, conv_iters=None):
         else:
             hn = gz
         dW[l] = linear_vjp_param(layer, x, gz)
+        if apply is not None:
+            apply(l, dW[l])
         x = act_forward(z, layer, m)
         h = hn
         if (l + 1) in store["reseed"]:
             h = store["reseed"][l + 1]
         hs.append(h)
     return dict(dW=dW, h=hs)
+
+
+def moonwalk_sgd_step(layers, params, x0, target, loss, lr, reseed_every=0, masks=None,
+                      conv_iters=None):
+    """One step of gradient descent with Algorithm 1 as printed: every g_i is applied to theta_i
+    (theta_i <- theta_i - lr g_i) the moment it is formed and then dropped.  Layer i's own
+    parameters are not read again after that, so the result equals theta - lr grad J."""
+    g0, store = input_cotangent(layers, params, x0, target, loss, reseed_every, masks)
+    new = [np.array(p, dtype=np.float64) for p in params]
+
+    def apply(i, g):
+        new[i] = new[i] - lr * g
+
+    forward_sweep(layers, params, x0, g0, store, conv_iters, apply=apply)
+    return new
 
 
 def moonwalk(layers, params, x0, target, loss, reseed_every=0, masks=None, conv_iters=None):

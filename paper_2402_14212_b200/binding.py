@@ -65,6 +65,7 @@ def lib() -> C.CDLL:
         L.mw_workspace_bytes.argtypes = [vp, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
         L.mw_input_cotangent.argtypes = [vp, C.POINTER(vp), vp, vp, vp, vp, vp, sz, vp]
         L.mw_forward_sweep.argtypes = [vp, C.POINTER(vp), vp, vp, C.POINTER(vp), vp, sz, vp]
+        L.mw_forward_sweep_apply.argtypes = [vp, C.POINTER(vp), vp, vp, C.c_double, C.POINTER(vp), vp, sz, vp]
         L.mw_backprop_reference.argtypes = [vp, C.POINTER(vp), vp, vp, C.POINTER(vp), vp, vp, sz, vp]
         L.mw_export_masks.argtypes = [vp, vp, i32, vp, sz, C.POINTER(i32), C.POINTER(i32), vp]
         L.mw_last_device_status.argtypes = [vp, vp, vp, C.POINTER(C.c_uint32)]
@@ -198,6 +199,16 @@ class Net:
                                       _ptr_array(dW_out), wp, wb, _stream_handle(stream)),
                "mw_forward_sweep")
         return dW_out
+
+    def forward_sweep_apply(self, params, x, g0, lr: float, workspace, params_out=None, stream=None):
+        """theta_l <- theta_l - lr * g_l inside the sweep; in place unless `params_out` is given."""
+        if params_out is None:
+            params_out = params
+        wp, wb = self._ws(workspace)
+        _check(lib().mw_forward_sweep_apply(self._h, _ptr_array(params), _ptr(x), _ptr(g0), float(lr),
+                                            _ptr_array(params_out), wp, wb, _stream_handle(stream)),
+               "mw_forward_sweep_apply")
+        return params_out
 
     def backprop_reference(self, params, x, target, workspace, dW_out=None, loss_out=None,
                            stream=None):

@@ -539,6 +539,18 @@ extern "C" mw_status mw_forward_sweep(mw_net* net, const void* const* params, co
                                    workspace, s);
 }
 
+extern "C" mw_status mw_forward_sweep_apply(mw_net* net, const void* const* params, const void* x,
+                                            const void* g0, double lr, void* const* params_out,
+                                            void* workspace, size_t workspace_bytes, void* stream) {
+  if (!net || !params || !params_out) return MW_ERR_INVALID_ARG;
+  if (net->backend != MW_BACKEND_TENSOR || net->opts.prec != MW_F32) return MW_ERR_UNSUPPORTED;
+  net->apply_params = params;
+  net->apply_lr = (float)lr;
+  const mw_status r = mw_forward_sweep(net, params, x, g0, params_out, workspace, workspace_bytes, stream);
+  net->apply_params = nullptr;
+  return r;
+}
+
 extern "C" mw_status mw_backprop_reference(mw_net* net, const void* const* params, const void* x,
                                            const void* loss_target, void* const* dW_out,
                                            double* loss_out, void* workspace,

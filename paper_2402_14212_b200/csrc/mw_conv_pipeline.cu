@@ -135,13 +135,13 @@ head_backward_kernel(const float* __restrict__ hl, const float* __restrict__ W, 
 // dW[o][k] = sum_b hl[b][o] x[b][k]
 __global__ void __launch_bounds__(256)
 head_wgrad_kernel(const float* __restrict__ hl, const float* __restrict__ x, int64_t nf, int no, int B,
-                  float* __restrict__ dW) {
+                  float* __restrict__ dW, const float* theta = nullptr, float lr = 0.f) {
   const int o = blockIdx.y;
   const int64_t k = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (k >= nf) return;
   float a = 0.f;
   for (int b = 0; b < B; ++b) a = fmaf(hl[(int64_t)b * no + o], x[(int64_t)b * nf + k], a);
-  dW[(int64_t)o * nf + k] = a;
+  dW[(int64_t)o * nf + k] = theta ? fmaf(-lr, a, theta[(int64_t)o * nf + k]) : a;   // fused update
 }
 
 // Phase I (or backprop's forward).  x_{l+1} planes go to the stores (backprop) or rotate; the
@@ -399,13 +399,15 @@ mw_status conv_tensor_forward_sweep(mw_net* n, const void* const* params, const 
     // weight vjp
     if (dW[l])
       MW_TRY(conv_wgrad_tensor(c.cache, c.g, xin, c.at<__nv_bfloat16>(lay.cg[T & 1]), 2,
-                               c.at<float>(lay.cpart), (float*)dW[l], c.st, s));
+                               c.at<float>(lay.cpart), (float*)dW[l], c.st, s,
+                               n->apply_params ? (const float*)n->apply_params[l] : nullptr, n->apply_lr));
   }
   if (c.head && dW[L - 1]) {
     // the head has no vijp: its output cotangent is the loss cotangent itself
     const mw_layer_desc& hd = n->layers[L - 1];
     head_wgrad_kernel<<<dim3((unsigned)((hd.n_in + 255) / 256), hd.n_out), 256, 0, s>>>(
-        c.at<float>(lay.h_last), c.at<float>(lay.cxf), hd.n_in, hd.n_out, n->B, (float*)dW[L - 1]);
+        c.at<float>(lay.h_last), c.at<float>(lay.cxf), hd.n_in, hd.n_out, n->B, (float*)dW[L - 1],
+        n->apply_params ? (const float*)n->apply_params[L - 1] : nullptr, n->apply_lr);
     MW_TRY(launch_ok());
   }
   return MW_OK;

@@ -15,12 +15,12 @@ namespace {
 
 __global__ void __launch_bounds__(256)
 slice_sum_f32_kernel(const float* __restrict__ part, int64_t n, int64_t stride, int slices,
-                     float* __restrict__ out) {
+                     float* __restrict__ out, const float* theta = nullptr, float lr = 0.f) {
   const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (i >= n) return;
   float a = 0.f;
   for (int z = 0; z < slices; ++z) a += part[(int64_t)z * stride + i];   // fixed order
-  out[i] = a;
+  out[i] = theta ? fmaf(-lr, a, theta[i]) : a;
 }
 
 }  // namespace
@@ -130,7 +130,7 @@ TcGemm conv_transpose_product(const ConvGeom& g, const __nv_bfloat16* g_planes, 
 
 mw_status conv_wgrad_tensor(TcMapCache* cache, const ConvGeom& g, const __nv_bfloat16* x_planes,
                             const __nv_bfloat16* gz_planes, int terms, float* partials, float* dw,
-                            DeviceStatus* st, cudaStream_t s) {
+                            DeviceStatus* st, cudaStream_t s, const float* theta, float lr) {
   const int slices = conv_wgrad_tensor_slices(g.out_pixels());
   const int C = g.C;
   const int rows = g.k * g.k * C;
@@ -142,12 +142,13 @@ mw_status conv_wgrad_tensor(TcMapCache* cache, const ConvGeom& g, const __nv_bfl
   p.epi.mode = TC_EPI_PLAIN;
   p.epi.out_f32 = slices > 1 ? partials : dw;
   p.epi.bs_f32 = (int64_t)rows * C;
+  if (theta && slices == 1) { p.epi.alpha = -lr; p.epi.addend = theta; }
   p.conv.mode = TC_CONV_WGRAD; p.conv.H = g.H; p.conv.W = g.W; p.conv.k = g.k; p.conv.pad = g.pad;
   p.conv.C = C; p.conv.stride = g.stride; p.conv.Ho = g.Ho(); p.conv.Wo = g.Wo();
   MW_TRY(tc_gemm_group(cache, &p, 1, st, s));
   if (slices > 1) {
     const int64_t n = (int64_t)rows * C;
-    slice_sum_f32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(partials, n, n, slices, dw);
+    slice_sum_f32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(partials, n, n, slices, dw, theta, lr);
     MW_TRY(launch_ok());
   }
   return MW_OK;

@@ -37,8 +37,10 @@ bool conv_transpose_class_product(const ConvGeom& g, int py, int px, const __nv_
 // dw[k*k][C][C] = sum over output pixels; `partials` holds conv_wgrad_tensor_slices(out pixels)
 // copies of dw
 int conv_wgrad_tensor_slices(int64_t pixels);
+// With `theta` given the result is theta - lr * dw instead (fused parameter update).
 mw_status conv_wgrad_tensor(TcMapCache* cache, const ConvGeom& g, const __nv_bfloat16* x_planes,
                             const __nv_bfloat16* gz_planes, int terms, float* partials, float* dw,
-                            DeviceStatus* st, cudaStream_t s);
+                            DeviceStatus* st, cudaStream_t s, const float* theta = nullptr,
+                            float lr = 0.f);
 
 }  // namespace mw

@@ -55,6 +55,10 @@ struct mw_net {
   const void* x_done = nullptr;
   void* tc = nullptr;              // tensor-core backend private state
   bool lean_seed = false;          // the net can keep the sweep's seed itself (g0 optional)
+  // mw_forward_sweep_apply in progress: the weight vjp's epilogue writes theta - apply_lr * g
+  // (theta = apply_params[l]) instead of g
+  const void* const* apply_params = nullptr;
+  float apply_lr = 0.f;
 };
 
 namespace mw {

@@ -399,7 +399,8 @@ mw_status sconv_tensor_forward_sweep(mw_net* n, const void* const* params, const
     hcur = reseed_next ? c.at<__nv_bfloat16>(lay.reseed[l + 1]) : hout;
     if (dW[l])
       MW_TRY(conv_wgrad_tensor(c.cache, g, xin, c.at<__nv_bfloat16>(lay.cg[0]), 2, c.at<float>(lay.cpart),
-                               (float*)dW[l], c.st, s));
+                               (float*)dW[l], c.st, s,
+                               n->apply_params ? (const float*)n->apply_params[l] : nullptr, n->apply_lr));
   }
   return MW_OK;
 }

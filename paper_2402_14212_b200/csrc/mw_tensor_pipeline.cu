@@ -746,10 +746,16 @@ TcGemm vijp_product(const Ctx& c, int l, bool want_h, bool want_gz) {
                  c.dim, e, 1);
 }
 
-TcGemm weight_vjp_product(const Ctx& c, const __nv_bfloat16* gz, const __nv_bfloat16* xl, float* dW) {
+// `layer`: whose gradient this is (for the fused parameter update, Algorithm 1's last line)
+TcGemm weight_vjp_product(const Ctx& c, const __nv_bfloat16* gz, const __nv_bfloat16* xl, float* dW,
+                          int layer = -1) {
   TcEpilogue e;
   e.mode = TC_EPI_PLAIN;
   e.out_f32 = dW;
+  if (c.n->apply_params && layer >= 0) {
+    e.alpha = -c.n->apply_lr;
+    e.addend = static_cast<const float*>(c.n->apply_params[layer]);
+  }
   return product(c, operand(gz, c.B, c.dim, c.pr.pgw, true), operand(xl, c.B, c.dim, c.pr.pxw, true),
                  c.dim, c.dim, c.B, e, 2);
 }
@@ -1030,7 +1036,7 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
   MW_TRY(split_planes((const float*)g0, c.bn, c.at<__nv_bfloat16>(lay.hp[0]), c.pr.ph, c.bn, s));
   // The sweep as one launch (sweep_program) measures slower than one launch per layer: its two
   // chains leave little for the waiting CTAs to do, so the per-layer launches stay the default.
-  if (use_programs(n) && n->opts.reserved == 1) return sweep_program(c, params, x, dW, x0p);
+  if (use_programs(n) && n->opts.reserved == 1 && !n->apply_params) return sweep_program(c, params, x, dW, x0p);
   auto xbuf = [&](int l) -> const __nv_bfloat16* {          // term planes of x_l
     return l == 0 ? x0p : c.at<__nv_bfloat16>(lay.xp[l % 3]);
   };
@@ -1051,7 +1057,7 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
     }
     if (l >= 1 && dW[l - 1])
       g[cnt++] = weight_vjp_product(c, c.at<__nv_bfloat16>(lay.gzp[(l - 1) & 1]), xbuf(l - 1),
-                                    (float*)dW[l - 1]);
+                                    (float*)dW[l - 1], l - 1);
     if (cnt) MW_TRY(run(c, g, cnt));
   }
   return MW_OK;

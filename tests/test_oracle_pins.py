@@ -271,6 +271,23 @@ def test_moonwalk_equals_backprop_cnn():
         assert O.normwise_error(mw["dW"][l], ref["dW"][l]) < 1e-9
 
 
+def test_sgd_step_through_the_sweep():
+    # Algorithm 1's last line: applying g_i as it appears equals theta - lr * grad J, and to first
+    # order lowers the loss by lr * |grad J|^2 (Taylor)
+    p = S.dense_chain("t", 24, 4, 8, S.F64, S.LOSS_MSE_MEAN, [S.ACT_LEAKY], 0.1,
+                      lambda rng, n, l: S.orthogonal(rng, n) + 0.05 * rng.standard_normal((n, n)) / np.sqrt(n),
+                      9, 2)
+    ref = O.backprop(p.layers, p.params, p.x, p.target, p.loss)
+    lr = 1e-3
+    new = O.moonwalk_sgd_step(p.layers, p.params, p.x, p.target, p.loss, lr, reseed_every=2)
+    for w, g, wn in zip(p.params, ref["dW"], new):
+        assert np.allclose(wn, w - lr * g, rtol=0, atol=1e-12 * lr)
+    J0 = ref["loss"]
+    J1 = O.loss_and_cotangent(O.forward(p.layers, new, p.x)[0][-1], p.target, p.loss)[0]
+    g2 = sum(float((g * g).sum()) for g in ref["dW"])
+    assert abs((J0 - J1) - lr * g2) <= 0.05 * lr * g2
+
+
 def test_cotangent_recursion_error_grows_with_depth():
     # the forward recursion amplifies rounding error layer by layer (leaky slope 0.1): an
     # invariant of the method that fixes the need for re-seeding, reproducible in fp64
