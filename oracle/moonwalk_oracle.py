@@ -39,7 +39,7 @@ from __future__ import annotations
 
 import numpy as np
 
-DENSE, CONV2D, HEAD = "dense", "conv2d", "head"
+DENSE, CONV2D, HEAD, CONV1D = "dense", "conv2d", "head", "conv1d"
 ACT_NONE, ACT_LEAKY, ACT_RELU = "none", "leaky_relu", "relu"
 
 
@@ -128,7 +128,50 @@ def conv_weight_vjp(x, gz, k, stride, pad):
     return dw
 
 
+def conv1d_forward(x, w, stride, pad):
+    """Lemma 1 with one spatial dimension: x'[i', c'] = sum_{j, c} w[j, c, c'] x[s i' + j - p, c].
+    x: [B, N, C], w: [k, C, C']."""
+    B, N, C = x.shape
+    k = w.shape[0]
+    No = (N + 2 * pad - k) // stride + 1
+    xp = np.zeros((B, N + 2 * pad, C))
+    xp[:, pad:pad + N, :] = x
+    out = np.zeros((B, No, w.shape[2]))
+    for j in range(k):
+        out += xp[:, j:j + stride * (No - 1) + 1:stride, :] @ w[j]
+    return out
+
+
+def transpose_conv1d(hp, w, n, stride, pad):
+    """Eq. "conv-vjp" with one spatial dimension: h[i, c] = sum_{j, c'} w[j, c, c'] hbar'[i + p - j, c']."""
+    B, No, Cp = hp.shape
+    k = w.shape[0]
+    m = k
+    hb = np.zeros((B, n + 2 * m, Cp))
+    hb[:, m:m + stride * (No - 1) + 1:stride, :] = hp
+    h = np.zeros((B, n, w.shape[1]))
+    for j in range(k):
+        o = m + pad - j
+        h += hb[:, o:o + n, :] @ w[j].T
+    return h
+
+
+def conv1d_weight_vjp(x, gz, k, stride, pad):
+    """dw[j, c, c'] = sum_{b, i'} x[b, s i' + j - p, c] gz[b, i', c']."""
+    B, N, C = x.shape
+    _, No, Cp = gz.shape
+    xp = np.zeros((B, N + 2 * pad, C))
+    xp[:, pad:pad + N, :] = x
+    dw = np.zeros((k, C, Cp))
+    g2 = gz.reshape(-1, Cp)
+    for j in range(k):
+        dw[j] = xp[:, j:j + stride * (No - 1) + 1:stride, :].reshape(-1, C).T @ g2
+    return dw
+
+
 def linear_forward(layer, w, x):
+    if layer.kind == CONV1D:
+        return conv1d_forward(x, w, layer.stride, layer.pad)
     if layer.kind == CONV2D:
         return conv_forward(x, w, layer.stride, layer.pad)
     x2 = x.reshape(x.shape[0], -1)
@@ -137,6 +180,8 @@ def linear_forward(layer, w, x):
 
 def linear_vjp_input(layer, w, g, in_shape):
     """vjp(f, x, g) of the linear part (Section 3.1)."""
+    if layer.kind == CONV1D:
+        return transpose_conv1d(g, w, layer.W, layer.stride, layer.pad)
     if layer.kind == CONV2D:
         return transpose_conv(g, w, (layer.H, layer.W), layer.stride, layer.pad)
     return (g @ w).reshape(in_shape)
@@ -144,6 +189,8 @@ def linear_vjp_input(layer, w, g, in_shape):
 
 def linear_vjp_param(layer, x, g):
     """vjp(f, theta, g) of the linear part: Eq. "g_i"."""
+    if layer.kind == CONV1D:
+        return conv1d_weight_vjp(x, g, layer.k, layer.stride, layer.pad)
     if layer.kind == CONV2D:
         return conv_weight_vjp(x, g, layer.k, layer.stride, layer.pad)
     return g.T @ x.reshape(x.shape[0], -1)
@@ -244,7 +291,51 @@ def vijp_conv_submersive(layer, w, h):
     return hp
 
 
+def conv1d_fragments(hp, k, block):
+    """Fragmental checkpoint of an output cotangent h' [B, N, C'] (Section 5.1): the first k - 1
+    positions of every block of `block` positions; [B, N / block, k - 1, C']."""
+    B, N, Cp = hp.shape
+    assert N % block == 0 and block >= k - 1
+    return hp.reshape(B, N // block, block, Cp)[:, :, :k - 1, :].copy()
+
+
+def vijp_conv1d_fragmental(layer, w, h, frags, block):
+    """Stride-1 convolution with padding 1 (Section 5.1, Appendix "Fragmental Gradient
+    Checkpointing"): the reverse pass reads h[i] = sum_j w[j] h'[i + 1 - j], whose newest unknown
+    is h'[i + 1] with coefficient w[0], lower triangular in (c, c') with a non-zero diagonal (the
+    paper normalises it to 1).  Given the first k - 1 positions of a block, the rest follow one
+    position after the other,
+        w[0] h'[i + 1] = h[i] - sum_{j >= 1} w[j] h'[i + 1 - j],
+    channel by channel through the triangle; blocks are independent of one another.
+    h: [B, N, C], frags: [B, N / block, k - 1, C'] -> h': [B, N, C']."""
+    k = layer.k
+    assert layer.stride == 1 and layer.pad == 1
+    w0 = w[0]
+    if np.any(np.triu(w0, 1) != 0.0) or np.any(np.diagonal(w0) == 0.0):
+        raise ValueError("tap 0 must be lower triangular in (c, c') with a non-zero diagonal")
+    B, N, C = h.shape
+    Cp = w.shape[2]
+    nb = N // block
+    hp = np.zeros((B, N, Cp))
+    for b in range(nb):
+        base = b * block
+        hp[:, base:base + k - 1, :] = frags[:, b]
+        for t in range(k - 1, block):
+            i = base + t - 1                       # the equation of h[i] yields h'[i + 1]
+            r = h[:, i, :Cp].copy()
+            for j in range(1, k):
+                q = i + 1 - j
+                if q >= 0:
+                    r -= hp[:, q, :] @ w[j, :Cp, :].T
+            for c in range(Cp):
+                v = r[:, c] - hp[:, i + 1, :c] @ w0[c, :c]
+                hp[:, i + 1, c] = v / w0[c, c]
+    return hp
+
+
 def vijp_linear(layer, w, h, conv_iters=None):
+    if layer.kind == CONV1D:
+        raise ValueError("a stride-1 1-D convolution needs its fragments: vijp_conv1d_fragmental")
     if layer.kind == CONV2D:
         if layer.stride > layer.pad:
             return vijp_conv_submersive(layer, w, h)
@@ -361,7 +452,7 @@ def relu_restore(gz, mask2d, off, vals):
 # ----------------------------------------------------------------------------
 # Algorithm 1 (Moonwalk), mixed mode: Phases I, II, III of Section 4.1
 # ----------------------------------------------------------------------------
-def input_cotangent(layers, params, x0, target, loss, reseed_every=0, masks=None):
+def input_cotangent(layers, params, x0, target, loss, reseed_every=0, masks=None, frag_block=0):
     """Phase I + Phase II.  Phase I keeps only the sign bits.  Phase II walks back computing
     input cotangents only; on the way it writes (a) the ReLU fragments and (b) a full cotangent
     checkpoint h_l for every l that is a multiple of `reseed_every` (0 < l < L)."""
@@ -376,12 +467,15 @@ def input_cotangent(layers, params, x0, target, loss, reseed_every=0, masks=None
         ms.append(m)
         x = act_forward(z, layer, m)
     J, h = loss_and_cotangent(x, target, loss)
-    store = dict(masks=ms, fragments={}, reseed={}, loss=J, h_last=h)
+    store = dict(masks=ms, fragments={}, reseed={}, loss=J, h_last=h, conv_fragments={},
+                 frag_block=frag_block)
     in_shapes = [x0.shape]
     for layer in layers[:-1]:
         if layer.kind == CONV2D:
             ho, wo = layer.out_hw()
             in_shapes.append((x0.shape[0], ho, wo, layer.C_out))
+        elif layer.kind == CONV1D:
+            in_shapes.append((x0.shape[0], layer.out_hw()[1], layer.C_out))
         else:
             in_shapes.append((x0.shape[0], layer.n_out))
     for l in range(L - 1, -1, -1):                                  # Phase II
@@ -392,6 +486,9 @@ def input_cotangent(layers, params, x0, target, loss, reseed_every=0, masks=None
         if reseed_every and (l + 1) % reseed_every == 0 and (l + 1) < L:
             store["reseed"][l + 1] = h.copy()
         gz = h * act_derivative(layer, ms[l])
+        if layer.kind == CONV1D:
+            # the convolution's own output cotangent g_z is what its vijp has to rebuild
+            store["conv_fragments"][l] = conv1d_fragments(gz, layer.k, frag_block)
         h = linear_vjp_input(layer, params[l], gz, in_shapes[l])
     store["g0"] = h
     return h, store
@@ -411,6 +508,8 @@ def forward_sweep(layers, params, x0, g0, store, conv_iters=None, apply=None):
         z = linear_forward(layer, w, x)
         if layer.kind == HEAD:
             gz = store["h_last"]                      # no vijp through a non-square last layer
+        elif layer.kind == CONV1D:
+            gz = vijp_conv1d_fragmental(layer, w, h, store["conv_fragments"][l], store["frag_block"])
         else:
             gz = vijp_linear(layer, w, h, conv_iters).reshape(z.shape)
         m = ms[l]
@@ -448,8 +547,9 @@ def moonwalk_sgd_step(layers, params, x0, target, loss, lr, reseed_every=0, mask
     return new
 
 
-def moonwalk(layers, params, x0, target, loss, reseed_every=0, masks=None, conv_iters=None):
-    g0, store = input_cotangent(layers, params, x0, target, loss, reseed_every, masks)
+def moonwalk(layers, params, x0, target, loss, reseed_every=0, masks=None, conv_iters=None,
+             frag_block=0):
+    g0, store = input_cotangent(layers, params, x0, target, loss, reseed_every, masks, frag_block)
     out = forward_sweep(layers, params, x0, g0, store, conv_iters)
     out.update(loss=store["loss"], g0=g0, masks=store["masks"], store=store)
     return out

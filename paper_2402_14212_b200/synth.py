@@ -23,7 +23,7 @@ import numpy as np
 
 # layer kinds / activations / losses / precisions (strings on the Python side;
 # the C-ABI enums carry the same names)
-DENSE, CONV2D, HEAD = "dense", "conv2d", "head"
+DENSE, CONV2D, HEAD, CONV1D = "dense", "conv2d", "head", "conv1d"
 ACT_NONE, ACT_LEAKY, ACT_RELU = "none", "leaky_relu", "relu"
 LOSS_HALF_SSE, LOSS_MSE_MEAN, LOSS_XENT_MEAN = "half_sse", "mse_mean", "xent_mean"
 F64, F32, BF16 = "f64", "f32", "bf16_f32acc"
@@ -46,8 +46,10 @@ class Layer:
     pad: int = 0
 
     def out_hw(self):
-        ho = (self.H + 2 * self.pad - self.k) // self.stride + 1
         wo = (self.W + 2 * self.pad - self.k) // self.stride + 1
+        if self.kind == CONV1D:
+            return 1, wo
+        ho = (self.H + 2 * self.pad - self.k) // self.stride + 1
         return ho, wo
 
 
@@ -63,6 +65,7 @@ class Problem:
     batch: int
     reseed_every: int = 4
     conv_vijp_iters: int = 0
+    frag_block: int = 0               # block size of the fragmental checkpoints of 1-D convolutions
     seed: int = 0
     notes: dict = field(default_factory=dict)
 
@@ -225,6 +228,32 @@ def strided_cnn(seed=0, depth=8, C=128, H=256, W=256, batch=128, gamma=0.5, rese
     t = round_storage(rng.standard_normal((batch, h, wd, C)), F32 if prec == BF16 else prec)
     return Problem("strided_cnn", layers, params, x, t, LOSS_MSE_MEAN, prec, batch,
                    reseed_every=reseed_every, seed=seed)
+
+
+def fragmental_cnn1d(seed=0, depth=8, C=256, N=2048, batch=128, block=4, gamma=0.5, reseed_every=4,
+                     prec=F32) -> Problem:
+    """The 1-D CNN of the paper's fragmental-checkpointing experiment: `depth` convolutions with
+    k = 3, stride 1, padding 1 on N x C sequences (the paper: 2048 x 256), leaky-ReLU 0.1, shape
+    kept across the layers; the output cotangent of every convolution is checkpointed at the first
+    2 positions of each block of `block` positions.
+
+    w[j, c, c'] for a [N, C] layer (H = 1, W = N): w = gamma * N(0, 2/(3*C)) with tap 0 made lower
+    triangular in (c, c') with unit diagonal (Section 5.1's assumptions).  Loss: mean squared error
+    against a Gaussian target.
+    """
+    rng = np.random.default_rng(seed)
+    layers, params = [], []
+    he = np.sqrt(2.0 / (3 * C))
+    for l in range(depth):
+        w = gamma * he * rng.standard_normal((3, C, C))
+        w[0] = np.tril(w[0], -1) + np.eye(C)
+        layers.append(Layer(CONV1D, ACT_LEAKY, 0.1, N * C, N * C, H=1, W=N, C_in=C, C_out=C, k=3,
+                            stride=1, pad=1))
+        params.append(round_storage(w, prec))
+    x = round_storage(rng.standard_normal((batch, N, C)), prec)
+    t = round_storage(rng.standard_normal((batch, N, C)), F32 if prec == BF16 else prec)
+    return Problem("fragmental_cnn1d", layers, params, x, t, LOSS_MSE_MEAN, prec, batch,
+                   reseed_every=reseed_every, frag_block=block, seed=seed)
 
 
 def random_preacts(seed: int, rows: int, cols: int, zero_frac: float = 0.01) -> np.ndarray:

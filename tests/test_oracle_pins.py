@@ -271,6 +271,85 @@ def test_moonwalk_equals_backprop_cnn():
         assert O.normwise_error(mw["dW"][l], ref["dW"][l]) < 1e-9
 
 
+def conv1d_by_loops(x, w, s, p):
+    B, N, C = x.shape
+    k, Cp = w.shape[0], w.shape[2]
+    No = (N + 2 * p - k) // s + 1
+    out = np.zeros((B, No, Cp))
+    for b in range(B):
+        for i in range(No):
+            for cp in range(Cp):
+                acc = 0.0
+                for j in range(k):
+                    a = s * i + j - p
+                    if 0 <= a < N:
+                        for c in range(C):
+                            acc += w[j, c, cp] * x[b, a, c]
+                out[b, i, cp] = acc
+    return out
+
+
+@pytest.mark.parametrize("block", [4, 8, 16])
+def test_fragmental_conv1d_vijp_against_explicit_jacobian(block):
+    # Section 5.1: with the first k - 1 positions of every block stored, the rest of the output
+    # cotangent follows from the input cotangent.  J is built index by index from Lemma 1's sum.
+    rng = np.random.default_rng(block)
+    N, C, B, k = 16, 3, 2, 3
+    w = 0.4 * rng.standard_normal((k, C, C))
+    w[0] = np.tril(w[0], -1) + np.diag(1.0 + 0.2 * rng.random(C))
+    layer = S.Layer(S.CONV1D, S.ACT_LEAKY, 0.1, H=1, W=N, C_in=C, C_out=C, k=k, stride=1, pad=1)
+    x = rng.standard_normal((B, N, C))
+    assert np.allclose(O.conv1d_forward(x, w, 1, 1), conv1d_by_loops(x, w, 1, 1), atol=1e-13)
+    n = N * C
+    Jm = np.zeros((n, n))
+    for i in range(n):
+        e = np.zeros(n); e[i] = 1.0
+        Jm[:, i] = conv1d_by_loops(e.reshape(1, N, C), w, 1, 1).ravel()
+    hp = rng.standard_normal((B, N, C))
+    h = (hp.reshape(B, -1) @ Jm).reshape(B, N, C)
+    assert np.allclose(O.transpose_conv1d(hp, w, N, 1, 1), h, atol=1e-12)
+    frags = O.conv1d_fragments(hp, k, block)
+    assert frags.shape == (B, N // block, k - 1, C)
+    assert frags.size * block == hp.size * (k - 1)              # the (k - 1) / block memory ratio
+    got = O.vijp_conv1d_fragmental(layer, w, h, frags, block)
+    assert np.allclose(got, hp, atol=1e-9)
+    # weight vjp against finite differences
+    g = rng.standard_normal((B, N, C))
+    dw = O.conv1d_weight_vjp(x, g, k, 1, 1)
+    for idx in [(0, 0, 0), (1, 2, 1), (2, 1, 2)]:
+        wp, wm = w.copy(), w.copy()
+        wp[idx] += 1e-6; wm[idx] -= 1e-6
+        fd = ((O.conv1d_forward(x, wp, 1, 1) - O.conv1d_forward(x, wm, 1, 1)) * g).sum() / 2e-6
+        assert abs(fd - dw[idx]) <= 1e-8
+    # wrong fragments give a wrong cotangent (the stored part is really used)
+    bad = O.vijp_conv1d_fragmental(layer, w, h, frags + 1e-3, block)
+    assert np.abs(bad - hp).max() > 1e-4
+
+
+def test_fragment_sizes_match_the_papers_example():
+    # Section 5.1: a 1024 x 64 residual, k = 3: B = 4 keeps 512 x 64, B = 16 keeps one eighth
+    hp = np.zeros((1, 1024, 64))
+    assert O.conv1d_fragments(hp, 3, 4).size == 512 * 64
+    assert O.conv1d_fragments(hp, 3, 16).size * 8 == hp.size
+
+
+@pytest.mark.parametrize("block,K", [(4, 0), (16, 2)])
+def test_moonwalk_equals_backprop_fragmental_cnn1d(block, K):
+    p = S.fragmental_cnn1d(seed=block, depth=3, C=4, N=32, batch=2, block=block, gamma=0.5,
+                           reseed_every=K, prec=S.F64)
+    ref = O.backprop(p.layers, p.params, p.x, p.target, p.loss)
+    mw = O.moonwalk(p.layers, p.params, p.x, p.target, p.loss, reseed_every=K, frag_block=block)
+    for l in range(3):
+        assert O.normwise_error(mw["dW"][l], ref["dW"][l]) < 1e-9
+    check_off_kinks(p.layers, p.params, p.x, margin=1e-6)
+    rng = np.random.default_rng(1)
+    for l in range(3):
+        for _ in range(4):
+            idx = tuple(int(v) for v in (rng.integers(0, 3), rng.integers(0, 4), rng.integers(0, 4)))
+            fd = fd_grad(p.layers, p.params, p.x, p.target, p.loss, l, idx)
+            assert abs(fd - ref["dW"][l][idx]) <= 1e-7 * max(1.0, abs(fd))
+
+
 def test_sgd_step_through_the_sweep():
     # Algorithm 1's last line: applying g_i as it appears equals theta - lr * grad J, and to first
     # order lowers the loss by lr * |grad J|^2 (Taylor)
