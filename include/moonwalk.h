@@ -50,7 +50,9 @@ typedef enum {
   MW_ERR_CUDA = 7            /* a CUDA runtime / driver call failed                      */
 } mw_status;
 
-typedef enum { MW_DENSE = 0, MW_CONV2D = 1, MW_HEAD_LINEAR = 2 } mw_kind;
+/* MW_CONV1D: a convolution along one dimension, [W positions][C channels] per sample (H = 1),
+ * kernel w[k][c_in][c_out]; its reverse pass is undone with fragmental checkpoints (Section 5.1). */
+typedef enum { MW_DENSE = 0, MW_CONV2D = 1, MW_HEAD_LINEAR = 2, MW_CONV1D = 3 } mw_kind;
 typedef enum { MW_ACT_NONE = 0, MW_ACT_LEAKY_RELU = 1, MW_ACT_RELU = 2 } mw_act;
 
 /* Storage / arithmetic:
@@ -89,6 +91,9 @@ typedef struct {
                               operands) once and keeps them in the workspace; 0: the sweep
                               builds them layer by layer in a transient slot (lean memory) */
   int32_t reserved;        /* 0; 1 = run the forward sweep as a single launch (experimental)     */
+  int32_t frag_block;      /* MW_CONV1D nets: Phase II keeps the output cotangent of every
+                              convolution at the first k - 1 positions of each block of this
+                              many positions (2..64, dividing W); Phase III rebuilds the rest  */
 } mw_net_opts;
 
 /* Build a host-side description.  `batch` is fixed per net.  Returns MW_ERR_UNSUPPORTED for
@@ -96,8 +101,10 @@ typedef struct {
  * k = 2*pad+1 (same size), or every layer of the net meeting Lemma 1 (i) with stride 2 (the
  * paper's submersive CNN: MW_F32, 64 or 128 channels, k - 1 - pad < 2, even image sizes, a
  * loss on the last feature map; conditions (ii) and (iii) on the anchor tap w[pad][pad] are
- * checked on the device every step: MW_ERR_NOT_SUBMERSIVE); head only as the last layer; all
- * layers of one net share `prec`. */
+ * checked on the device every step: MW_ERR_NOT_SUBMERSIVE); MW_CONV1D nets: every layer k = 3,
+ * stride 1, padding 1, the same W (a multiple of 128) and C (64..256, a multiple of 64), MW_F32,
+ * tap 0 lower triangular in (c_in, c_out) with a non-zero diagonal (checked on the device);
+ * head only as the last layer; all layers of one net share `prec`. */
 mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers, int32_t batch,
                         const mw_net_opts* opts, mw_net** out);
 void mw_net_destroy(mw_net* net);

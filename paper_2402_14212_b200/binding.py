@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libmoonwalk.so")
 MW_OK = 0
 STATUS_NAMES = ["MW_OK", "MW_ERR_INVALID_ARG", "MW_ERR_UNSUPPORTED", "MW_ERR_WORKSPACE",
                 "MW_ERR_STATE", "MW_ERR_NOT_SUBMERSIVE", "MW_ERR_TIMEOUT", "MW_ERR_CUDA"]
-KIND = {"dense": 0, "conv2d": 1, "head": 2}
+KIND = {"dense": 0, "conv2d": 1, "head": 2, "conv1d": 3}
 ACT = {"none": 0, "leaky_relu": 1, "relu": 2}
 PREC = {"f64": 0, "f32": 1, "bf16_f32acc": 2}
 LOSS = {"half_sse": 0, "mse_mean": 1, "xent_mean": 2}
@@ -44,7 +44,7 @@ class NetOpts(C.Structure):
     _fields_ = [("prec", C.c_int32), ("loss", C.c_int32), ("reseed_every", C.c_int32),
                 ("conv_vijp_iters", C.c_int32), ("backend", C.c_int32),
                 ("inverse_iters", C.c_int32), ("resident_inverse", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("reserved", C.c_int32), ("frag_block", C.c_int32)]
 
 
 _lib = None
@@ -127,13 +127,14 @@ class Net:
 
     def __init__(self, layers, batch: int, prec: str, loss: str, reseed_every: int = 4,
                  conv_vijp_iters: int = 10, backend: str = "auto", inverse_iters: int = 0,
-                 resident_inverse: bool = True):
+                 resident_inverse: bool = True, frag_block: int = 0):
         self.layers = list(layers)
         self.batch = int(batch)
         self.prec, self.loss = prec, loss
         self._h = C.c_void_p()
         opts = NetOpts(PREC[prec], LOSS[loss], int(reseed_every), int(conv_vijp_iters),
-                       BACKEND[backend], int(inverse_iters), int(bool(resident_inverse)), 0)
+                       BACKEND[backend], int(inverse_iters), int(bool(resident_inverse)), 0,
+                       int(frag_block))
         descs = make_layer_descs(self.layers)
         _check(lib().mw_net_create(descs, len(self.layers), self.batch, C.byref(opts),
                                    C.byref(self._h)), "mw_net_create")
@@ -234,7 +235,7 @@ class Net:
 
     def export_masks(self, workspace, layer: int, stream=None) -> np.ndarray:
         l = self.layers[layer]
-        if l.kind == "conv2d":
+        if l.kind in ("conv2d", "conv1d"):
             ho, wo = l.out_hw()
             rows, cols = self.batch * ho * wo, l.C_out
         else:
@@ -396,4 +397,5 @@ def to_device(problem, device="cuda"):
 def net_for(problem, backend="auto", resident_inverse=True, inverse_iters=0) -> Net:
     return Net(problem.layers, problem.batch, problem.prec, problem.loss,
                reseed_every=problem.reseed_every, conv_vijp_iters=problem.conv_vijp_iters,
-               backend=backend, inverse_iters=inverse_iters, resident_inverse=resident_inverse)
+               backend=backend, inverse_iters=inverse_iters, resident_inverse=resident_inverse,
+               frag_block=getattr(problem, "frag_block", 0))

@@ -34,6 +34,9 @@ bool valid_layer(const mw_layer_desc& d, int idx, int L) {
   if (d.act < MW_ACT_NONE || d.act > MW_ACT_RELU) return false;
   if (d.kind == MW_DENSE) return d.n_in > 0 && d.n_in == d.n_out;
   if (d.kind == MW_HEAD_LINEAR) return idx == L - 1 && d.n_in > 0 && d.n_out > 0 && d.act == MW_ACT_NONE;
+  if (d.kind == MW_CONV1D)
+    return d.H == 1 && d.W > 0 && d.C_in > 0 && d.C_in == d.C_out && d.k >= 2 && d.stride == 1 && d.pad == 1 &&
+           d.k == 3;
   if (d.kind == MW_CONV2D) {
     if (!(d.H > 0 && d.W > 0 && d.C_in > 0 && d.C_in == d.C_out && d.k >= 1 && d.pad >= 0 && d.stride >= 1))
       return false;
@@ -151,11 +154,11 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
   if (!layers || !opts || !out || n_layers < 1 || batch < 1) return MW_ERR_INVALID_ARG;
   if (opts->prec < MW_F64 || opts->prec > MW_BF16_F32ACC) return MW_ERR_INVALID_ARG;
   if (opts->loss < MW_LOSS_HALF_SSE || opts->loss > MW_LOSS_XENT_MEAN) return MW_ERR_INVALID_ARG;
-  if (opts->reseed_every < 0 || opts->conv_vijp_iters < 0 || opts->inverse_iters < 0)
+  if (opts->reseed_every < 0 || opts->conv_vijp_iters < 0 || opts->inverse_iters < 0 || opts->frag_block < 0)
     return MW_ERR_INVALID_ARG;
   if (opts->backend < MW_BACKEND_AUTO || opts->backend > MW_BACKEND_TENSOR) return MW_ERR_INVALID_ARG;
   for (int l = 0; l < n_layers; ++l) {
-    if (layers[l].kind < MW_DENSE || layers[l].kind > MW_HEAD_LINEAR) return MW_ERR_INVALID_ARG;
+    if (layers[l].kind < MW_DENSE || layers[l].kind > MW_CONV1D) return MW_ERR_INVALID_ARG;
     if (!valid_layer(layers[l], l, n_layers)) return MW_ERR_UNSUPPORTED;
   }
   mw_net* n = new (std::nothrow) mw_net();
@@ -170,7 +173,14 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
   for (int l = 0; l < n_layers; ++l) {
     const mw_layer_desc& d = n->layers[l];
     LayerInfo& li = n->info[l];
-    if (d.kind == MW_CONV2D) {
+    if (d.kind == MW_CONV1D) {
+      li.rows = (int64_t)batch * d.W;
+      li.cols = d.C_out;
+      li.in_elems = li.rows * d.C_in;
+      li.out_elems = li.rows * d.C_out;
+      li.w_elems = (int64_t)d.k * d.C_in * d.C_out;
+      li.inv_n = d.C_in;
+    } else if (d.kind == MW_CONV2D) {
       const int Ho = (d.H + 2 * d.pad - d.k) / d.stride + 1, Wo = (d.W + 2 * d.pad - d.k) / d.stride + 1;
       li.rows = (int64_t)batch * Ho * Wo;
       li.cols = d.C_out;
@@ -193,7 +203,8 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
     }
     prev_out = li.out_elems;
   }
-  if (opts->loss == MW_LOSS_XENT_MEAN && n->layers[n_layers - 1].kind == MW_CONV2D) {
+  if (opts->loss == MW_LOSS_XENT_MEAN && n->layers[n_layers - 1].kind != MW_HEAD_LINEAR &&
+      n->layers[n_layers - 1].kind != MW_DENSE) {
     delete n;
     return MW_ERR_UNSUPPORTED;
   }
@@ -209,9 +220,14 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
     delete n;
     return MW_ERR_UNSUPPORTED;
   }
-  // strided convolutions only have the tensor-core path; a conv net is all of one kind
+  // strided and 1-D convolutions only have the tensor-core path; a conv net is all of one kind
   for (int l = 0; l < n_layers; ++l) {
     const mw_layer_desc& d = n->layers[l];
+    if ((d.kind == MW_CONV1D || n->layers[0].kind == MW_CONV1D) &&
+        (d.kind != n->layers[0].kind || n->backend != MW_BACKEND_TENSOR)) {
+      delete n;
+      return MW_ERR_UNSUPPORTED;
+    }
     if (d.kind == MW_CONV2D && (d.stride != n->layers[0].stride || n->layers[0].kind != MW_CONV2D ||
                                 (d.stride != 1 && n->backend != MW_BACKEND_TENSOR))) {
       delete n;

@@ -29,6 +29,12 @@ slice_sum_f32_kernel(const float* __restrict__ part, int64_t n, int64_t stride, 
 // core truncates its fp32 accumulator at every instruction, a bias that grows with the length of
 // one accumulation (about 1e-4 relative after 1024 K blocks) and that the fixed-order sum of the
 // slices, in round-to-nearest fp32, does not have.
+mw_status conv_slice_sum(const float* part, int64_t n, int slices, float* out, const float* theta,
+                         float lr, cudaStream_t s) {
+  slice_sum_f32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(part, n, n, slices, out, theta, lr);
+  return launch_ok();
+}
+
 int conv_wgrad_tensor_slices(int64_t pixels) {
   const int64_t blocks = pixels / 64;
   for (int s = 256; s > 32; s >>= 1)

@@ -37,6 +37,9 @@ bool conv_transpose_class_product(const ConvGeom& g, int py, int px, const __nv_
 // dw[k*k][C][C] = sum over output pixels; `partials` holds conv_wgrad_tensor_slices(out pixels)
 // copies of dw
 int conv_wgrad_tensor_slices(int64_t pixels);
+// out[i] = sum over the slices (in order) of part[z*n + i]; with `theta`: theta[i] - lr * that sum
+mw_status conv_slice_sum(const float* part, int64_t n, int slices, float* out, const float* theta,
+                         float lr, cudaStream_t s);
 // With `theta` given the result is theta - lr * dw instead (fused parameter update).
 mw_status conv_wgrad_tensor(TcMapCache* cache, const ConvGeom& g, const __nv_bfloat16* x_planes,
                             const __nv_bfloat16* gz_planes, int terms, float* partials, float* dw,

@@ -34,6 +34,7 @@ struct Layout {
   Region xp[3], hp[2], gzp[2], ns_r, ns_x, ns_w; // activation / cotangent / g_z planes, NS scratch
   // convolution nets on the tensor cores
   std::vector<Region> cw, cwhat, cwinv;      // per layer: kernel, folded kernel, centre-tap inverse (term planes)
+  std::vector<Region> cfrag;                 // per layer: fragmental checkpoints of a 1-D convolution
   Region cwinv_f32, cwhat_f32, cg[2], chpf, cxf, cpart, clogits, cseed;
   Region ns_sumsq;
   Region prog_table[3], prog_done[3];        // product tables and completion counters of program launches

@@ -67,7 +67,7 @@ struct alignas(64) TcProblem {
   float* split_partials;
   unsigned int* split_counters;
   // convolution forms (TcConv)
-  int conv_mode, cHo, cWo, ck, cpad, cstride, ccb, b_tap_rows, cntaps;
+  int conv_mode, cHo, cWo, ck, cpad, cstride, ccb, b_tap_rows, cntaps, c1d;
   signed char tdy[28], tdx[28], ttb[28];
   // program launches: products (by index) that must be complete before this one starts, and
   // the number of warp arrivals that completes each of them (one per epilogue warp and tile)
@@ -264,7 +264,7 @@ __device__ __forceinline__ uint32_t frag_base(const TcEpilogue& e, int N, int ro
 // (`prow`: the row inside the product, `row`: where its outputs live; they differ under a scatter)
 __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int prow, int row, int col0,
                                                float (&v)[32], double& sumsq_local) {
-  const int64_t off = (int64_t)row * N + col0;
+  const int64_t off = (int64_t)row * (e.ld ? e.ld : (int64_t)N) + col0;
   const int64_t woff = (int64_t)row * (N >> 5) + (col0 >> 5);
   switch (e.mode) {
     case TC_EPI_PLAIN: {
@@ -586,10 +586,11 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
               int tap = (r0 + hh) / P.ccb;
               const int cblk = (r0 + hh) - tap * P.ccb;
               if (tap >= P.cntaps) tap = P.cntaps - 1;   // rows past the last tap are never stored
-              const int j0 = tap / P.ck, j1 = tap - j0 * P.ck;
+              const int j0 = P.c1d ? 0 : tap / P.ck, j1 = tap - j0 * P.ck;
+              const int oy = P.c1d ? 0 : j0 - P.cpad;
               for (int pl = 0; pl < pa; ++pl)
                 tma_load_5d(sbase + (uint32_t)pl * kATileBytes + (uint32_t)hh * 8192u, &P.tmA, fb, cblk * BK,
-                            P.cstride * x0 + j1 - P.cpad, P.cstride * y0 + j0 - P.cpad, b, pl);
+                            P.cstride * x0 + j1 - P.cpad, P.cstride * y0 + oy, b, pl);
             }
             bk0 = pix;
             k0 = pix;
@@ -946,18 +947,20 @@ void tc_cache_destroy(TcMapCache* c) { delete c; }
 
 static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, int total_planes,
                          CUtensorMap* out) {
-  auto key = std::make_tuple(op.base, op.rows, op.cols, total_planes, op.plane_stride, (int64_t)box_rows);
+  const int64_t ld = op.ld ? op.ld : op.cols;
+  auto key = std::make_tuple(op.base, op.rows, op.cols, total_planes, op.plane_stride,
+                             (int64_t)box_rows + (ld << 12));
   if (cache) {
     auto it = cache->maps.find(key);
     if (it != cache->maps.end()) { *out = it->second; return MW_OK; }
   }
   auto fn = encode_fn();
   if (!fn) return MW_ERR_CUDA;
-  if (((uintptr_t)op.base & 15u) || (op.cols % 8) != 0) return MW_ERR_INVALID_ARG;
-  const int64_t ps = total_planes > 1 ? op.plane_stride : (int64_t)op.rows * op.cols;
+  if (((uintptr_t)op.base & 15u) || (op.cols % 8) != 0 || (ld % 8) != 0 || ld < op.cols) return MW_ERR_INVALID_ARG;
+  const int64_t ps = total_planes > 1 ? op.plane_stride : (int64_t)op.rows * ld;
   if (ps % 8 != 0) return MW_ERR_INVALID_ARG;
   cuuint64_t dims[3] = {(cuuint64_t)op.cols, (cuuint64_t)op.rows, (cuuint64_t)total_planes};
-  cuuint64_t strides[2] = {(cuuint64_t)op.cols * 2, (cuuint64_t)ps * 2};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)ps * 2};
   cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
   cuuint32_t estr[3] = {1u, 1u, 1u};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(op.base), dims, strides,
@@ -1072,6 +1075,7 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   const TcConv& cv = d.conv;
   int cbx = 0, cby = 0, cbi = 0;          // pixels, rows, images of one A box
   P.conv_mode = cv.mode;
+  P.c1d = 0;
   if (cv.mode != TC_CONV_NONE) {
     const int span = cv.mode == TC_CONV_PIXELS ? BM : BK;    // pixels per A box
     const int Ho = cv.Ho ? cv.Ho : cv.H, Wo = cv.Wo ? cv.Wo : cv.W;
@@ -1105,8 +1109,9 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
       if (nt < 1 || d.A.mn_major || d.M % (Ho * Wo) != 0 || d.batch != 1 || d.K != nt * C)
         return MW_ERR_UNSUPPORTED;
     } else {
-      P.cntaps = cv.k * cv.k;
-      if (cv.k < 1 || !d.A.mn_major || !d.B.mn_major || d.M != cv.k * cv.k * C || d.K % 64 != 0 ||
+      P.cntaps = cv.one_d ? cv.k : cv.k * cv.k;
+      P.c1d = cv.one_d;
+      if (cv.k < 1 || !d.A.mn_major || !d.B.mn_major || d.M != P.cntaps * C || d.K % 64 != 0 ||
           d.split_k > 1)
         return MW_ERR_UNSUPPORTED;
     }

@@ -32,6 +32,7 @@ struct TcOperand {
   int64_t plane_stride = 0;     // elements between planes
   bool mn_major = false;
   int batch_planes = 0;         // batched product: planes between consecutive batch items (0 = planes)
+  int64_t ld = 0;               // elements between consecutive rows (0 = cols): a window of wider rows
 };
 
 enum TcEpiMode : int {
@@ -78,6 +79,9 @@ struct TcEpilogue {
   int remap_s = 0, remap_ho = 0, remap_wo = 0, remap_py = 0, remap_px = 0;
   // TC_EPI_BWD with a row scatter: planes2 is addressed by the product's own row all the same
   // (the class of the pixels (s*y, s*x) written densely: all that a strided vijp reads of h)
+  // elements between consecutive rows of addend, out_f32 and planes (0 = N): outputs that are a
+  // column window of wider rows
+  int64_t ld = 0;
   int compact2 = 0;
   // TC_EPI_VIJP (sub2_s > 0): the rows are pixels of sub2_h x sub2_w images and planes2 keeps
   // only the pixels (sub2_s*y, sub2_s*x), densely: [images][sub2_h/s][sub2_w/s][N]
@@ -112,6 +116,7 @@ struct TcConv {
   int sgn = 1;
   int skip_tap = -1;        // tap left out of the sum (the centre tap of the folded kernel), or -1
   int b_tap_rows = 0;       // B is K-major with rows (block, n): used by TransposeConv
+  int one_d = 0;            // TC_CONV_WGRAD: the kernel is 1 x k (taps along x only, no row offset)
   int ntaps = 0;            // explicit window list (TC_CONV_PIXELS)
   signed char dy[kTcMaxTaps] = {}, dx[kTcMaxTaps] = {}, tb[kTcMaxTaps] = {};
 };

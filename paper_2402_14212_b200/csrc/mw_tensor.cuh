@@ -41,6 +41,18 @@ mw_status sconv_tensor_backprop(mw_net* n, const void* const* params, const void
                                 const void* target, void* const* dW, double* loss_out, void* ws,
                                 cudaStream_t s);
 
+// the 1-D CNN with fragmental checkpoints (mw_conv1d_pipeline.cu): k = 3, stride 1, padding 1
+bool conv1d_tensor_supported(const mw_net* n);
+void conv1d_tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start);
+mw_status conv1d_tensor_input_cotangent(mw_net* n, const void* const* params, const void* x,
+                                        const void* target, void* g0, double* loss_out, void* ws,
+                                        cudaStream_t s);
+mw_status conv1d_tensor_forward_sweep(mw_net* n, const void* const* params, const void* x,
+                                      const void* g0, void* const* dW, void* ws, cudaStream_t s);
+mw_status conv1d_tensor_backprop(mw_net* n, const void* const* params, const void* x,
+                                 const void* target, void* const* dW, double* loss_out, void* ws,
+                                 cudaStream_t s);
+
 // true when every layer of the net has a tensor-core path (dense, sizes multiples of 64,
 // MW_F32 or MW_BF16_F32ACC)
 bool tensor_supported(const mw_net* n);

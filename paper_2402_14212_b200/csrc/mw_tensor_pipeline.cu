@@ -851,6 +851,7 @@ mw_status backprop_program(const Ctx& c, const void* const* params, const void* 
 }  // namespace
 
 bool tensor_supported(const mw_net* n) {
+  if (n->layers[0].kind == MW_CONV1D) return conv1d_tensor_supported(n);
   if (n->layers[0].kind == MW_CONV2D)
     return n->layers[0].stride == 1 ? conv_tensor_supported(n) : sconv_tensor_supported(n);
   if (n->opts.prec != MW_F32 && n->opts.prec != MW_BF16_F32ACC) return false;
@@ -875,6 +876,10 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     TensorState* t = new TensorState();
     t->cache = tc_cache_create();
     n->tc = t;
+  }
+  if (n->layers[0].kind == MW_CONV1D) {
+    conv1d_tensor_layout(n, backprop, lay, start);
+    return;
   }
   if (n->layers[0].kind == MW_CONV2D) {
     if (n->layers[0].stride == 1) conv_tensor_layout(n, backprop, lay, start);
@@ -954,6 +959,8 @@ void tensor_destroy(mw_net* n) {
 mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const void* x,
                                  const void* target, void* g0, double* loss_out, void* ws,
                                  cudaStream_t s) {
+  if (n->layers[0].kind == MW_CONV1D)
+    return conv1d_tensor_input_cotangent(n, params, x, target, g0, loss_out, ws, s);
   if (n->layers[0].kind == MW_CONV2D)
     return n->layers[0].stride == 1 ? conv_tensor_input_cotangent(n, params, x, target, g0, loss_out, ws, s)
                                     : sconv_tensor_input_cotangent(n, params, x, target, g0, loss_out, ws, s);
@@ -1024,6 +1031,7 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
 
 mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void* x, const void* g0,
                                void* const* dW, void* ws, cudaStream_t s) {
+  if (n->layers[0].kind == MW_CONV1D) return conv1d_tensor_forward_sweep(n, params, x, g0, dW, ws, s);
   if (n->layers[0].kind == MW_CONV2D)
     return n->layers[0].stride == 1 ? conv_tensor_forward_sweep(n, params, x, g0, dW, ws, s)
                                     : sconv_tensor_forward_sweep(n, params, x, g0, dW, ws, s);
@@ -1065,6 +1073,8 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
 
 mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, const void* target,
                           void* const* dW, double* loss_out, void* ws, cudaStream_t s) {
+  if (n->layers[0].kind == MW_CONV1D)
+    return conv1d_tensor_backprop(n, params, x, target, dW, loss_out, ws, s);
   if (n->layers[0].kind == MW_CONV2D)
     return n->layers[0].stride == 1 ? conv_tensor_backprop(n, params, x, target, dW, loss_out, ws, s)
                                     : sconv_tensor_backprop(n, params, x, target, dW, loss_out, ws, s);

@@ -34,7 +34,9 @@ def oracle_masks_from_words(problem, words_list):
     """GPU-exported words -> boolean masks shaped like each layer's z (for mask replay)."""
     ms = []
     for layer, words in zip(problem.layers, words_list):
-        if layer.kind == "conv2d":
+        if layer.kind == "conv1d":
+            m = O.unpack_mask(words, layer.C_out).reshape(problem.batch, layer.out_hw()[1], layer.C_out)
+        elif layer.kind == "conv2d":
             ho, wo = layer.out_hw()
             m = O.unpack_mask(words, layer.C_out).reshape(problem.batch, ho, wo, layer.C_out)
         else:

@@ -179,3 +179,33 @@ def test_strided_cnn_full_size():
         assert worst[l] <= 1e-4 * np.sqrt(l + 1.0), (l, worst[l])
         assert O.normwise_error(out["dW"][l], dW[l]) <= 1e-4, l
     assert abs(out["loss"] - loss) <= 1e-4 * abs(loss)
+
+
+# ---------------------------------------------------------------------------------------
+# whole path on the 1-D CNN with fragmental checkpoints (Section 5.1; k = 3, stride 1, padding 1)
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("depth,C,N,batch,block,K", [(3, 64, 128, 2, 4, 0), (4, 256, 256, 2, 16, 2),
+                                                     (5, 128, 128, 4, 8, 4), (2, 64, 256, 1, 2, 0),
+                                                     (3, 128, 128, 2, 64, 0)])
+def test_fragmental_cnn1d_fp32_tensor_path(depth, C, N, batch, block, K):
+    from paper_2402_14212_b200 import synth as S
+    from parity_util import check_problem
+    p = S.fragmental_cnn1d(seed=depth, depth=depth, C=C, N=N, batch=batch, block=block, reseed_every=K,
+                           prec=S.F32)
+    out, ref, errs = check_problem(p, 1e-4, backend="tensor", exact_masks=False, tau=1e-4)
+    # the residual store holds (k - 1) / block of one cotangent per layer, in fp32, beside the sign bits
+    _, _, (mw_res, bp_res) = out["net"].workspace_bytes()
+    frag_bytes = depth * 4 * batch * N * C * 2 // block
+    assert mw_res >= frag_bytes
+
+
+def test_fragmental_cnn1d_rejects_a_full_tap0():
+    from paper_2402_14212_b200 import synth as S
+    p = S.fragmental_cnn1d(seed=1, depth=2, C=64, N=128, batch=2, block=4, reseed_every=0, prec=S.F32)
+    p.params[0][0, 2, 5] = 0.5                       # c < c': tap 0 is no longer triangular
+    net = mwb.net_for(p, backend="tensor")
+    params, x, target = mwb.to_device(p)
+    ws = net.alloc_workspace("both")
+    net.input_cotangent(params, x, target, ws)
+    code, detail = net.last_device_status(ws)
+    assert code == mwb.STATUS_NAMES.index("MW_ERR_NOT_SUBMERSIVE")
