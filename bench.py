@@ -36,7 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {"deep_mlp": 115.6e6}
 
 
-def workload(name: str, seed: int = 0, depth: int = 0):
+def workload(name: str, seed: int = 0, depth: int = 0, block: int = 0):
     from paper_2402_14212_b200 import synth as S
     if name == "deep_mlp":
         return S.deep_mlp(seed=seed)
@@ -54,12 +54,21 @@ def workload(name: str, seed: int = 0, depth: int = 0):
         return S.strided_cnn(seed=seed, depth=depth or 8)
     if name == "strided_cnn_small":
         return S.strided_cnn(seed=seed, depth=depth or 4, H=64, W=64, batch=16)
+    if name == "fragmental_cnn1d":
+        # the paper's 1-D experiment: 2048 x 256 sequences, batch 128, k = 3 stride-1 convolutions,
+        # output cotangents checkpointed at 2 of every `block` positions
+        return S.fragmental_cnn1d(seed=seed, depth=depth or 16, block=block or 4)
     if name == "tiny_mlp":
         return S.tiny_mlp(seed=seed)
     raise SystemExit(f"unknown workload {name}")
 
 
 def describe(p):
+    if p.layers[0].kind == "conv1d":
+        l0 = p.layers[0]
+        return {"workload": p.name, "layers": len(p.layers), "conv": f"{l0.k}x{l0.C_in}x{l0.C_out}",
+                "sequence": f"{l0.W}x{l0.C_in}", "stride": 1, "batch": p.batch, "prec": p.prec,
+                "loss": p.loss, "reseed_every": p.reseed_every, "frag_block": p.frag_block, "seed": p.seed}
     if p.layers[0].kind == "conv2d":
         l0 = p.layers[0]
         return {"workload": p.name, "layers": len(p.layers), "conv": f"{l0.k}x{l0.k}x{l0.C_in}x{l0.C_out}",
@@ -143,7 +152,7 @@ def time_oracle(p, seconds_target: float, max_reps: int = 50, samples: int = 0):
     x, t = np.asarray(p.x[:b], dtype=np.float64), p.target[:b]
     reps, t0 = 0, time.perf_counter()
     while True:
-        O.moonwalk(p.layers, p.params, x, t, p.loss, reseed_every=p.reseed_every)
+        O.moonwalk(p.layers, p.params, x, t, p.loss, reseed_every=p.reseed_every, frag_block=p.frag_block)
         reps += 1
         dt = time.perf_counter() - t0
         if dt >= seconds_target or reps >= max_reps:
@@ -167,13 +176,13 @@ def run_reference(args):
     import numpy as np
     from oracle import moonwalk_oracle as O
     from paper_2402_14212_b200 import synth as S
-    p = workload(args.workload, depth=args.depth)
+    p = workload(args.workload, depth=args.depth, block=args.frag_block)
     total = args.steps + args.warmup
     # cost of one sample, then as many rows of the batch as the time budget allows
-    probe = 1 if p.layers[0].kind == "conv2d" else min(8, p.batch)
+    probe = 1 if p.layers[0].kind in ("conv2d", "conv1d") else min(8, p.batch)
     t0 = time.perf_counter()
     O.moonwalk(p.layers, p.params, np.asarray(p.x[:probe], dtype=np.float64), p.target[:probe], p.loss,
-               reseed_every=p.reseed_every)
+               reseed_every=p.reseed_every, frag_block=p.frag_block)
     t_one = (time.perf_counter() - t0) / probe
     budget = 150.0
     b = int(budget / (t_one * total))
@@ -181,7 +190,7 @@ def run_reference(args):
     x, t = np.asarray(p.x[:b], dtype=np.float64), p.target[:b]
 
     def step():
-        O.moonwalk(p.layers, p.params, x, t, p.loss, reseed_every=p.reseed_every)
+        O.moonwalk(p.layers, p.params, x, t, p.loss, reseed_every=p.reseed_every, frag_block=p.frag_block)
 
     for _ in range(args.warmup):
         step()
@@ -236,7 +245,7 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    p = workload(args.workload, depth=args.depth)
+    p = workload(args.workload, depth=args.depth, block=args.frag_block)
     net = mwb.net_for(p, backend=args.backend)
     params, x, target = mwb.to_device(p, dev)
     ws = net.alloc_workspace("moonwalk", dev)
@@ -357,7 +366,7 @@ def run_ours(args):
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         # the large convolutional workload is sampled: one image of the batch through all layers
-        v, reps_o, dt, b_o = time_oracle(p, 10.0, samples=1 if p.name == "strided_cnn" else 0)
+        v, reps_o, dt, b_o = time_oracle(p, 10.0, samples=1 if p.name in ("strided_cnn", "fragmental_cnn1d") else 0)
         cpu = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                "sample": f"{reps_o} steps of {b_o} of {p.batch} samples, all {len(p.layers)} layers, in {dt:.1f} s, "
                          "Algorithm 1 in fp64 numpy"}
@@ -503,7 +512,8 @@ def main():
                     help="strided CNN workloads: have mw_input_cotangent return g0 in full")
     ap.add_argument("--with-backprop", action="store_true",
                     help="also time mw_backprop_reference on the same inputs (phases_ms.backprop)")
-    ap.add_argument("--depth", type=int, default=0, help="depth of the sweep_mlp workload")
+    ap.add_argument("--depth", type=int, default=0, help="depth of the sweep_mlp / CNN workloads")
+    ap.add_argument("--frag-block", type=int, default=0, help="block size of the fragmental_cnn1d workload")
     ap.add_argument("--depth-sweep", action="store_true",
                     help="config 5: peak memory and samples/s versus depth, Moonwalk against the "
                          "in-library Backprop (prints one JSON object, not the benchmark line)")
