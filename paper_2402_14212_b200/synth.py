@@ -230,7 +230,7 @@ def strided_cnn(seed=0, depth=8, C=128, H=256, W=256, batch=128, gamma=0.5, rese
                    reseed_every=reseed_every, seed=seed)
 
 
-def fragmental_cnn1d(seed=0, depth=8, C=256, N=2048, batch=128, block=4, gamma=0.5, reseed_every=4,
+def fragmental_cnn1d(seed=0, depth=8, C=256, N=2048, batch=128, block=4, gamma=0.3, reseed_every=4,
                      prec=F32) -> Problem:
     """The 1-D CNN of the paper's fragmental-checkpointing experiment: `depth` convolutions with
     k = 3, stride 1, padding 1 on N x C sequences (the paper: 2048 x 256), leaky-ReLU 0.1, shape

@@ -209,3 +209,40 @@ def test_fragmental_cnn1d_rejects_a_full_tap0():
     net.input_cotangent(params, x, target, ws)
     code, detail = net.last_device_status(ws)
     assert code == mwb.STATUS_NAMES.index("MW_ERR_NOT_SUBMERSIVE")
+
+
+def test_fragmental_cnn1d_full_size():
+    """The paper's 1-D experiment at its size (2048 x 256 sequences, batch 128; 8 layers, blocks of
+    16 positions: the longest reconstruction the paper uses), in the launch configuration the
+    benchmark times.  The oracle takes the batch in slices, replaying the GPU's sign bits."""
+    from paper_2402_14212_b200 import synth as S
+    from parity_util import run_gpu
+    p = S.fragmental_cnn1d(seed=0, depth=8, block=16)
+    out = run_gpu(p, backend="tensor", backprop=False)
+    assert out["status"] == 0
+    L, B = len(p.layers), p.batch
+    dW = [np.zeros_like(w) for w in p.params]
+    loss, g0_err, worst = 0.0, 0.0, [0.0] * L
+    step = 16
+    for b0 in range(0, B, step):
+        sl = slice(b0, b0 + step)
+        masks = []
+        for l, layer in enumerate(p.layers):
+            words = out["masks"][l].reshape(B, layer.W, -1)[sl].reshape(step * layer.W, -1)
+            masks.append(O.unpack_mask(words, layer.C_out).reshape(step, layer.W, layer.C_out))
+        ref = O.backprop(p.layers, p.params, p.x[sl], p.target[sl], p.loss, masks=masks)
+        f = step / B                       # mse_mean divides by the elements of ITS batch
+        loss += ref["loss"] * f
+        for l in range(L):
+            dW[l] += ref["dW"][l] * f
+            z = ref["z"][l].reshape(-1, p.layers[l].C_out)
+            d = masks[l].reshape(z.shape) != O.sign_mask(z)
+            if d.any():
+                rms = np.sqrt((z * z).mean(axis=1, keepdims=True))
+                worst[l] = max(worst[l], float((np.abs(z) / rms)[d].max()))
+        g0_err = max(g0_err, float(np.abs(out["g0"][sl].reshape(ref["g0"].shape) - ref["g0"] * f).max()))
+    assert g0_err <= 1e-4 * float(np.abs(out["g0"]).max())
+    for l in range(L):
+        assert worst[l] <= 1e-4 * np.sqrt(l + 1.0), (l, worst[l])
+        assert O.normwise_error(out["dW"][l], dW[l]) <= 1e-4, l
+    assert abs(out["loss"] - loss) <= 1e-4 * abs(loss)
