@@ -47,13 +47,14 @@ C1 make_c1(mw_net* n, const Layout& lay, void* ws, cudaStream_t s) {
 }
 
 // ---- small kernels ---------------------------------------------------------------------------
-// inverse of the lower triangular tap 0 of up to kSmallBatch layers: one CTA per layer, one thread
-// per column, x_i = (delta_ij - sum_{m<i} A[i][m] x_m) / A[i][i] in double (scratch: n*n per layer)
-__global__ void __launch_bounds__(256)
-tri_inverse_kernel(SmallBatch ws, int n, double* __restrict__ scratch0, float* __restrict__ inv0,
-                   DeviceStatus* st, int layer0) {
+// inverse of the lower triangular tap 0 of up to kSmallBatch layers: CTA (layer, group of 64
+// columns), one thread per column, x_i = (delta_ij - sum_{m<i} A[i][m] x_m) / A[i][i] in double,
+// the columns of the group in shared memory ([n][64] doubles)
+constexpr int kTriCols = 64;
+__global__ void __launch_bounds__(kTriCols)
+tri_inverse_kernel(SmallBatch ws, int n, float* __restrict__ inv0, DeviceStatus* st, int layer0) {
+  extern __shared__ double xs[];            // [n][kTriCols]
   const float* A = static_cast<const float*>(ws.p[blockIdx.x]);
-  double* xs = scratch0 + (int64_t)blockIdx.x * n * n;
   float* inv = inv0 + (int64_t)blockIdx.x * n * n;
   __shared__ int bad;
   if (threadIdx.x == 0) bad = 0;
@@ -65,18 +66,31 @@ tri_inverse_kernel(SmallBatch ws, int n, double* __restrict__ scratch0, float* _
   }
   __syncthreads();
   if (bad) {
-    if (threadIdx.x == 0)
+    if (threadIdx.x == 0 && blockIdx.y == 0)
       record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)(layer0 + blockIdx.x), 0u, 3u, 0u);
     return;
   }
-  for (int j = threadIdx.x; j < n; j += blockDim.x) {
-    for (int i = 0; i < n; ++i) {
-      double a = i == j ? 1.0 : 0.0;
-      if (i > j)
-        for (int m = j; m < i; ++m) a -= (double)A[i * n + m] * xs[(int64_t)m * n + j];
-      xs[(int64_t)i * n + j] = i < j ? 0.0 : a / (double)A[i * n + i];
+  const int t = threadIdx.x, j = blockIdx.y * kTriCols + t;
+  if (j >= n) return;
+  for (int i = 0; i < n; ++i) {
+    double a = i == j ? 1.0 : 0.0;
+    if (i > j) {
+      const float* Ai = A + (int64_t)i * n;
+      for (int m = j; m < i; ++m) a -= (double)Ai[m] * xs[m * kTriCols + t];
     }
-    for (int i = 0; i < n; ++i) inv[i * n + j] = (float)xs[(int64_t)i * n + j];
+    const double x = i < j ? 0.0 : a / (double)A[(int64_t)i * n + i];
+    xs[i * kTriCols + t] = x;
+    inv[(int64_t)i * n + j] = (float)x;
+  }
+}
+
+// eight bf16 values of one 128-bit load, as floats
+__device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
   }
 }
 
@@ -84,7 +98,7 @@ tri_inverse_kernel(SmallBatch ws, int n, double* __restrict__ scratch0, float* _
 // reconstruction step, whose K runs over the k - 1 previous positions, oldest first
 __global__ void __launch_bounds__(256)
 fold1d_kernel(SmallBatch ws, const float* __restrict__ inv0, int C, int k, float* __restrict__ fold0) {
-  const int c = blockIdx.x, q = blockIdx.y, cp = threadIdx.x + blockIdx.z * 0;
+  const int c = blockIdx.x, q = blockIdx.y, cp = threadIdx.x;
   const float* w = static_cast<const float*>(ws.p[blockIdx.z]);
   const float* inv = inv0 + (int64_t)blockIdx.z * C * C;
   float* fold = fold0 + (int64_t)blockIdx.z * C * (k - 1) * C;
@@ -96,55 +110,90 @@ fold1d_kernel(SmallBatch ws, const float* __restrict__ inv0, int C, int k, float
   }
 }
 
-// fragments of g (term planes, [rows = samples*N][C]) -> fp32 [samples*N/blk][keep*C]
+// fragments of g (term planes, [rows = samples*N][C]) -> fp32 [samples*N/blk][keep*C]; eight
+// channels per thread (C a multiple of 8)
 __global__ void __launch_bounds__(256)
 frag_gather_kernel(const __nv_bfloat16* __restrict__ planes, int n_planes, int64_t plane_stride, int C,
-                   int blk, int keep, int64_t total, float* __restrict__ frags) {
-  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;   // over [blocks][keep][C]
-  if (i >= total) return;
-  const int c = (int)(i % C);
-  const int64_t r = i / C;
+                   int blk, int keep, int64_t total8, float* __restrict__ frags) {
+  const int64_t i8 = (int64_t)blockIdx.x * 256 + threadIdx.x;   // over [blocks][keep][C / 8]
+  if (i8 >= total8) return;
+  const int C8 = C >> 3;
+  const int c = (int)(i8 % C8) * 8;
+  const int64_t r = i8 / C8;
   const int q = (int)(r % keep);
   const int64_t b = r / keep;
   const int64_t src = (b * blk + q) * C + c;
-  float a = 0.f;
-  for (int p = n_planes - 1; p >= 0; --p) a += __bfloat162float(planes[(int64_t)p * plane_stride + src]);
-  frags[i] = a;
+  float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int p = n_planes - 1; p >= 0; --p) {
+    float f[8];
+    unpack8(*reinterpret_cast<const uint4*>(planes + (int64_t)p * plane_stride + src), f);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) a[k] += f[k];
+  }
+  float4* dst = reinterpret_cast<float4*>(frags + i8 * 8);
+  dst[0] = make_float4(a[0], a[1], a[2], a[3]);
+  dst[1] = make_float4(a[4], a[5], a[6], a[7]);
 }
 
 // the inverse: fp32 fragments -> term planes at the first `keep` positions of every block
 __global__ void __launch_bounds__(256)
-frag_scatter_kernel(const float* __restrict__ frags, int C, int blk, int keep, int64_t total,
+frag_scatter_kernel(const float* __restrict__ frags, int C, int blk, int keep, int64_t total8,
                     __nv_bfloat16* __restrict__ planes, int n_planes, int64_t plane_stride) {
-  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  if (i >= total) return;
-  const int c = (int)(i % C);
-  const int64_t r = i / C;
+  const int64_t i8 = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i8 >= total8) return;
+  const int C8 = C >> 3;
+  const int c = (int)(i8 % C8) * 8;
+  const int64_t r = i8 / C8;
   const int q = (int)(r % keep);
   const int64_t b = r / keep;
   const int64_t dst = (b * blk + q) * C + c;
-  float rem = frags[i];
+  const float4* src = reinterpret_cast<const float4*>(frags + i8 * 8);
+  const float4 u = src[0], v = src[1];
+  float a[8] = {u.x, u.y, u.z, u.w, v.x, v.y, v.z, v.w};
   for (int p = 0; p < n_planes; ++p) {
-    const __nv_bfloat16 t = __float2bfloat16_rn(rem);
-    rem -= __bfloat162float(t);
-    planes[(int64_t)p * plane_stride + dst] = t;
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const __nv_bfloat16 t0 = __float2bfloat16_rn(a[2 * k]), t1 = __float2bfloat16_rn(a[2 * k + 1]);
+      a[2 * k] -= __bfloat162float(t0);
+      a[2 * k + 1] -= __bfloat162float(t1);
+      w[k] = (uint32_t)__bfloat16_as_ushort(t0) | ((uint32_t)__bfloat16_as_ushort(t1) << 16);
+    }
+    *reinterpret_cast<uint4*>(planes + (int64_t)p * plane_stride + dst) = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
-// leaky-ReLU vijp on term planes: h = g where the sign bit is set, g / slope elsewhere
+// leaky-ReLU vijp on term planes (n and the plane strides multiples of 8; 128-bit accesses)
 __global__ void __launch_bounds__(256)
 planes_leaky_vijp_kernel(const __nv_bfloat16* __restrict__ g, int gp, int64_t gs,
-                         const uint32_t* __restrict__ words, int act, float slope, int64_t n,
+                         const uint32_t* __restrict__ words, int act, float slope, int64_t n8,
                          __nv_bfloat16* __restrict__ h, int hp, int64_t hs) {
-  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  if (i >= n) return;
-  float a = 0.f;
-  for (int p = gp - 1; p >= 0; --p) a += __bfloat162float(g[(int64_t)p * gs + i]);
-  if (act == MW_ACT_LEAKY_RELU && !((words[i >> 5] >> (i & 31)) & 1u)) a = a / slope;
+  const int64_t i8 = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i8 >= n8) return;
+  const int64_t i = i8 * 8;
+  float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int p = gp - 1; p >= 0; --p) {
+    float f[8];
+    unpack8(*reinterpret_cast<const uint4*>(g + (int64_t)p * gs + i), f);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) a[k] += f[k];
+  }
+  if (act == MW_ACT_LEAKY_RELU) {
+    const uint32_t bits = words[i >> 5] >> (i & 31);
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (!((bits >> k) & 1u)) a[k] = a[k] / slope;
+  }
   for (int p = 0; p < hp; ++p) {
-    const __nv_bfloat16 t = __float2bfloat16_rn(a);
-    a -= __bfloat162float(t);
-    h[(int64_t)p * hs + i] = t;
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const __nv_bfloat16 t0 = __float2bfloat16_rn(a[2 * k]), t1 = __float2bfloat16_rn(a[2 * k + 1]);
+      a[2 * k] -= __bfloat162float(t0);
+      a[2 * k + 1] -= __bfloat162float(t1);
+      w[k] = (uint32_t)__bfloat16_as_ushort(t0) | ((uint32_t)__bfloat16_as_ushort(t1) << 16);
+    }
+    *reinterpret_cast<uint4*>(h + (int64_t)p * hs + i) = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
@@ -214,15 +263,21 @@ mw_status prep(const C1& c, const void* const* params, bool inverse) {
   for (int l = 0; l < c.L; ++l)
     MW_TRY(split_planes((const float*)params[l], c.we, c.at<__nv_bfloat16>(lay.cw[l]), 3, c.we, c.s));
   if (!inverse) return MW_OK;
+  static bool attr_done = false;
+  if (!attr_done) {
+    MW_CUDA_OK(cudaFuncSetAttribute(tri_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)(sizeof(double) * 256 * kTriCols)));
+    attr_done = true;
+  }
   float* inv = c.at<float>(lay.cwinv_f32);        // [kSmallBatch][C*C]
   float* fold = c.at<float>(lay.cwhat_f32);       // [kSmallBatch][C][(k-1)*C]
-  double* scratch = c.at<double>(lay.inv_scratch);
   const int64_t fe = (int64_t)C * (c.k - 1) * C;
   for (int l0 = 0; l0 < c.L; l0 += kSmallBatch) {
     const int G = c.L - l0 < kSmallBatch ? c.L - l0 : kSmallBatch;
     SmallBatch ws{};
     for (int g = 0; g < G; ++g) ws.p[g] = params[l0 + g];
-    tri_inverse_kernel<<<G, 256, 0, c.s>>>(ws, C, scratch, inv, c.st, l0);
+    tri_inverse_kernel<<<dim3(G, (C + kTriCols - 1) / kTriCols), kTriCols, sizeof(double) * C * kTriCols, c.s>>>(
+        ws, C, inv, c.st, l0);
     MW_TRY(launch_ok());
     fold1d_kernel<<<dim3(C, c.k - 1, G), 256, 0, c.s>>>(ws, inv, C, c.k, fold);
     MW_TRY(launch_ok());
@@ -289,9 +344,9 @@ mw_status backward_pass(const C1& c, void* g0, void* const* dW, bool moonwalk) {
     const __nv_bfloat16* gz = c.at<__nv_bfloat16>(lay.hp[cur]);
     if (moonwalk) {
       // fragmental checkpoint of this layer's g_z: the first k - 1 positions of every block
-      const int64_t total = frag_elems(c);
-      frag_gather_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c.s>>>(
-          gz, 3, c.P, c.C, c.blk, c.k - 1, total, c.at<float>(lay.cfrag[l]));
+      const int64_t total8 = frag_elems(c) / 8;
+      frag_gather_kernel<<<(unsigned)((total8 + 255) / 256), 256, 0, c.s>>>(
+          gz, 3, c.P, c.C, c.blk, c.k - 1, total8, c.at<float>(lay.cfrag[l]));
       MW_TRY(launch_ok());
     }
     if (dW && dW[l]) {
@@ -372,7 +427,6 @@ void conv1d_tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     }
     lay.cwinv_f32 = b.take(4 * (size_t)C * C * kSmallBatch);
     lay.cwhat_f32 = b.take(4 * (size_t)C * (k - 1) * C * kSmallBatch);
-    lay.inv_scratch = b.take(8 * (size_t)C * C * kSmallBatch);
   }
   lay.total = b.cur;
 }
@@ -431,9 +485,9 @@ mw_status conv1d_tensor_forward_sweep(mw_net* n, const void* const* params, cons
         MW_TRY(tc_gemm_group(c.cache, &p, 1, c.st, s));
       }
       {
-        const int64_t total = frag_elems(c);
-        frag_scatter_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
-            c.at<float>(lay.cfrag[l]), C, blk, k - 1, total, gzp, 3, c.P);
+        const int64_t total8 = frag_elems(c) / 8;
+        frag_scatter_kernel<<<(unsigned)((total8 + 255) / 256), 256, 0, s>>>(
+            c.at<float>(lay.cfrag[l]), C, blk, k - 1, total8, gzp, 3, c.P);
         MW_TRY(launch_ok());
       }
       // position t of every block from positions t-2, t-1 (adjacent in memory: K = 2 C)
@@ -454,8 +508,8 @@ mw_status conv1d_tensor_forward_sweep(mw_net* n, const void* const* params, cons
         MW_TRY(tc_gemm_group(c.cache, &p, 1, c.st, s));
       }
       if (want_h) {
-        planes_leaky_vijp_kernel<<<(unsigned)((c.P + 255) / 256), 256, 0, s>>>(
-            gzp, 3, c.P, words, ld.act, (float)ld.slope, c.P, hout, 3, c.P);
+        planes_leaky_vijp_kernel<<<(unsigned)((c.P / 8 + 255) / 256), 256, 0, s>>>(
+            gzp, 3, c.P, words, ld.act, (float)ld.slope, c.P / 8, hout, 3, c.P);
         MW_TRY(launch_ok());
       }
     }
