@@ -499,6 +499,55 @@ def net_backend_is_tensor(net):
     return net.prec != "f64" and all(l.kind == "dense" and l.n_in % 64 == 0 for l in net.layers)
 
 
+def memory_table(budget_bytes: float = 24e9):
+    """The paper's memory experiments from the library's own accounting (mw_workspace_bytes; no GPU
+    work): workspace and between-phase residual bytes of Moonwalk and of the in-library Backprop for
+    the 2-D submersive CNN over its depth and for the 1-D CNN with fragmental checkpoints over depth
+    and block size, and the largest 1-D depth whose total (workspace + parameters + gradients + input
+    and target) stays under `budget_bytes` (the paper's GPU has 24 GB)."""
+    from paper_2402_14212_b200 import binding as mwb
+    from paper_2402_14212_b200 import synth as S
+
+    def strided_layers(depth, C=128, H=256):
+        out, h = [], H
+        for _ in range(depth):
+            lay = S.Layer(S.CONV2D, S.ACT_LEAKY, 0.1, h * h * C, 0, H=h, W=h, C_in=C, C_out=C, k=3, stride=2, pad=1)
+            ho, wo = lay.out_hw()
+            lay.n_out = ho * wo * C
+            out.append(lay)
+            h = ho
+        return out
+
+    def conv1d_layers(depth, C=256, N=2048):
+        return [S.Layer(S.CONV1D, S.ACT_LEAKY, 0.1, N * C, N * C, H=1, W=N, C_in=C, C_out=C, k=3, stride=1, pad=1)
+                for _ in range(depth)]
+
+    def row(layers, batch, **kw):
+        net = mwb.Net(layers, batch, S.F32, S.LOSS_MSE_MEAN, backend="tensor", reseed_every=4, **kw)
+        mw_b, bp_b, (mw_res, bp_res) = net.workspace_bytes()
+        w = sum(4 * l.k * l.k * l.C_in * l.C_out if l.kind == S.CONV2D else 4 * l.k * l.C_in * l.C_out
+                for l in layers)
+        io = 4 * batch * (layers[0].n_in + layers[-1].n_out)
+        net.close()
+        return {"depth": len(layers), "moonwalk_workspace": mw_b, "backprop_workspace": bp_b,
+                "moonwalk_residual": mw_res, "backprop_residual": bp_res, "params": w, "grads": w,
+                "inputs": io, "moonwalk_total": mw_b + 2 * w + io, "backprop_total": bp_b + 2 * w + io}
+
+    table = {"budget_bytes": budget_bytes, "strided_cnn": [row(strided_layers(d), 128) for d in range(1, 9)],
+             "fragmental_cnn1d": {}}
+    for blk in (4, 16):
+        rows = [row(conv1d_layers(d), 128, frag_block=blk) for d in (2, 4, 8, 16, 22, 32)]
+        # totals grow linearly in depth: walk up to the budget
+        fit = {}
+        for which in ("moonwalk_total", "backprop_total"):
+            d = 1
+            while d < 4096 and row(conv1d_layers(d + 1), 128, frag_block=blk)[which] <= budget_bytes:
+                d += 1 if d < 64 else 16
+            fit[which.replace("_total", "_max_depth")] = d
+        table["fragmental_cnn1d"][f"block_{blk}"] = {"rows": rows, **fit}
+    return table
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -518,8 +567,13 @@ def main():
                     help="config 5: peak memory and samples/s versus depth, Moonwalk against the "
                          "in-library Backprop (prints one JSON object, not the benchmark line)")
     ap.add_argument("--max-depth", type=int, default=512)
+    ap.add_argument("--memory-table", action="store_true",
+                    help="the paper's CNN memory experiments from the library's byte accounting "
+                         "(prints one JSON object; runs without a GPU)")
     args = ap.parse_args()
-    if args.depth_sweep:
+    if args.memory_table:
+        print(json.dumps(memory_table()), flush=True)
+    elif args.depth_sweep:
         run_depth_sweep(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -4,6 +4,7 @@
   python -m paper_2402_14212_b200.profile_cases pack --rows 65536 --cols 2048
   python -m paper_2402_14212_b200.profile_cases fragments --rows 65536 --cols 2048
   python -m paper_2402_14212_b200.profile_cases conv --images 512 --op 1 --terms 2
+  python -m paper_2402_14212_b200.profile_cases sconv --images 16 --op 0 --terms 3
 
 Each case allocates its seeded inputs, runs the kernel `--reps` times and exits.
 """
@@ -18,7 +19,7 @@ def main():
     import torch
     from . import binding as mwb
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["gemm", "pack", "fragments", "vijp", "conv"])
+    ap.add_argument("case", choices=["gemm", "pack", "fragments", "vijp", "conv", "sconv"])
     ap.add_argument("--M", type=int, default=256)
     ap.add_argument("--N", type=int, default=1024)
     ap.add_argument("--K", type=int, default=1024)
@@ -37,6 +38,17 @@ def main():
         B = torch.randn((a.K, a.N) if a.b_mn else (a.N, a.K), device="cuda", generator=g)
         for _ in range(a.reps):
             mwb.gemm_split_bf16(A, B, a.a_mn, a.b_mn, a.terms)
+    elif a.case == "sconv":
+        # 3x3, stride 2, padding 1, 128 channels on 256 x 256 images: the first layer of the paper's CNN
+        x = torch.randn((a.images, 256, 256, 128), device="cuda", generator=g)
+        if a.op == 1:
+            x = torch.randn((a.images, 128, 128, 128), device="cuda", generator=g)
+        if a.op == 2:
+            b = torch.randn((a.images, 128, 128, 128), device="cuda", generator=g)
+        else:
+            b = torch.randn((3, 3, 128, 128), device="cuda", generator=g)
+        for _ in range(a.reps):
+            mwb.conv2d_strided_split_bf16(a.op, x, b, 3, 2, 1, a.terms, in_hw=(256, 256))
     elif a.case == "conv":
         # 3x3, 64 channels, 32 x 32 images, channel-last: the convolutional configuration's layer
         x = torch.randn((a.images, 32, 32, 64), device="cuda", generator=g)

@@ -54,6 +54,48 @@ def test_net_create_rejects_bad_descriptions():
                 2, S.F32, S.LOSS_MSE_MEAN)
 
 
+def test_net_create_convolution_families():
+    def sconv(H, C=128, k=3, s=2, p=1, act=S.ACT_LEAKY):
+        l = S.Layer(S.CONV2D, act, 0.1, H=H, W=H, C_in=C, C_out=C, k=k, stride=s, pad=p)
+        ho, wo = l.out_hw()
+        l.n_in, l.n_out = H * H * C, ho * wo * C
+        return l
+    # the paper's submersive CNN: stride 2, padding 1, halving resolution
+    net = mwb.Net([sconv(32), sconv(16), sconv(8)], 16, S.F32, S.LOSS_MSE_MEAN)
+    mw_b, bp_b, (mw_res, bp_res) = net.workspace_bytes()
+    assert mw_b > mw_res > 0 and bp_res > 0
+    # its first call may leave g0 out; a dense net's may not (checked before any GPU work)
+    L = mwb.lib()
+    arr = (C.c_void_p * 3)(1, 1, 1)
+    assert L.mw_input_cotangent(net._h, arr, 1, 1, None, None, None, 1 << 30, None) == 3   # reaches the workspace check
+    dense = mwb.net_for(S.tiny_mlp())
+    arr4 = (C.c_void_p * 4)(1, 1, 1, 1)
+    assert L.mw_input_cotangent(dense._h, arr4, 1, 1, None, None, 256, 1 << 30, None) == 1
+    for bad in ([sconv(32), sconv(8)],                 # resolutions do not chain
+                [sconv(32, C=96)],                     # channels not a multiple of 64
+                [sconv(30)],                           # 15 x 15 output: tiles are not boxes
+                [sconv(32, k=5)],                      # taps of other pixels reach the positions s*i'
+                [sconv(32, act=S.ACT_RELU)]):
+        with pytest.raises(mwb.MwError):
+            mwb.Net(bad, 16, S.F32, S.LOSS_MSE_MEAN)
+    with pytest.raises(mwb.MwError):
+        mwb.Net([sconv(32)], 16, S.F64, S.LOSS_MSE_MEAN)          # tensor cores only: fp32 nets
+    # 1-D convolutions need a block size for their fragmental checkpoints
+    c1 = [S.Layer(S.CONV1D, S.ACT_LEAKY, 0.1, 128 * 64, 128 * 64, H=1, W=128, C_in=64, C_out=64, k=3,
+                  stride=1, pad=1) for _ in range(3)]
+    with pytest.raises(mwb.MwError):
+        mwb.Net(c1, 4, S.F32, S.LOSS_MSE_MEAN)
+    with pytest.raises(mwb.MwError):
+        mwb.Net(c1, 4, S.F32, S.LOSS_MSE_MEAN, frag_block=3)      # does not divide the length
+    n4 = mwb.Net(c1, 4, S.F32, S.LOSS_MSE_MEAN, frag_block=4)
+    n16 = mwb.Net(c1, 4, S.F32, S.LOSS_MSE_MEAN, frag_block=16)
+    r4, r16 = n4.workspace_bytes()[2][0], n16.workspace_bytes()[2][0]
+    frag = lambda blk: 3 * 4 * 4 * 128 * 64 * 2 // blk
+    assert r4 - r16 == frag(4) - frag(16)              # fragments: 2 of every `block` positions, fp32
+    # the fused update is for fp32 nets on the tensor cores
+    assert L.mw_forward_sweep_apply(dense._h, arr4, 1, 1, 0.1, arr4, 256, 1 << 30, None) == 2
+
+
 def test_workspace_sizes_and_residual_accounting():
     p = S.deep_mlp(depth=8, n=128, batch=64, reseed_every=4)
     net = mwb.net_for(p, backend="simt")
