@@ -75,8 +75,18 @@ tri_inverse_kernel(SmallBatch ws, int n, float* __restrict__ inv0, DeviceStatus*
   for (int i = 0; i < n; ++i) {
     double a = i == j ? 1.0 : 0.0;
     if (i > j) {
+      // four independent partial sums: the chain of dependent fp64 adds is what takes the time
       const float* Ai = A + (int64_t)i * n;
-      for (int m = j; m < i; ++m) a -= (double)Ai[m] * xs[m * kTriCols + t];
+      double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+      int m = j;
+      for (; m + 3 < i; m += 4) {
+        s0 += (double)__ldg(Ai + m) * xs[m * kTriCols + t];
+        s1 += (double)__ldg(Ai + m + 1) * xs[(m + 1) * kTriCols + t];
+        s2 += (double)__ldg(Ai + m + 2) * xs[(m + 2) * kTriCols + t];
+        s3 += (double)__ldg(Ai + m + 3) * xs[(m + 3) * kTriCols + t];
+      }
+      for (; m < i; ++m) s0 += (double)__ldg(Ai + m) * xs[m * kTriCols + t];
+      a -= (s0 + s1) + (s2 + s3);
     }
     const double x = i < j ? 0.0 : a / (double)A[(int64_t)i * n + i];
     xs[i * kTriCols + t] = x;
