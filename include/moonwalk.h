@@ -137,8 +137,11 @@ mw_status mw_input_cotangent(mw_net* net, const void* const* params, const void*
  * params_out[l] (device, float, shaped like the weight) may be params[l] itself: the products of
  * the sweep read the term planes Phase I made of the weights, never params again (with
  * resident_inverse = 0 layer l's weight is read just before its own update).  A NULL entry skips
- * that layer.  MW_F32 nets on the tensor-core backend; otherwise MW_ERR_UNSUPPORTED.  Other
- * arguments, requirements and errors as for mw_forward_sweep. */
+ * that layer.  In nets whose convolutions are constrained to a triangular tap (Lemma 1 (ii);
+ * Section 5.1 for MW_CONV1D) the entries that the constraint fixes at zero are not parameters
+ * (Section "Constrained Convolutions") and stay zero.  MW_F32 nets on the tensor-core backend;
+ * otherwise MW_ERR_UNSUPPORTED.  Other arguments, requirements and errors as for
+ * mw_forward_sweep. */
 mw_status mw_forward_sweep_apply(mw_net* net, const void* const* params, const void* x,
                                  const void* g0, double lr, void* const* params_out,
                                  void* workspace, size_t workspace_bytes, void* stream);

@@ -532,16 +532,29 @@ def forward_sweep(layers, params, x0, g0, store, conv_iters=None, apply=None):
     return dict(dW=dW, h=hs)
 
 
+def trainable_entries(layer, w):
+    """Section "Constrained Convolutions": layers are parameterised so that the conditions of their
+    vijp hold by construction.  The entries that Lemma 1 (ii) fixes at zero (anchor tap w[p], c < c')
+    -- for the stride-1 1-D convolution of Section 5.1 those of tap 0 -- are not parameters.
+    Returns 1.0 at trainable entries, 0.0 at fixed ones."""
+    m = np.ones(w.shape)
+    if layer.kind == CONV2D and layer.stride > layer.pad:
+        m[layer.pad, layer.pad] = np.tril(np.ones(w.shape[2:]))
+    elif layer.kind == CONV1D:
+        m[0] = np.tril(np.ones(w.shape[1:]))
+    return m
+
+
 def moonwalk_sgd_step(layers, params, x0, target, loss, lr, reseed_every=0, masks=None,
-                      conv_iters=None):
+                      conv_iters=None, frag_block=0):
     """One step of gradient descent with Algorithm 1 as printed: every g_i is applied to theta_i
     (theta_i <- theta_i - lr g_i) the moment it is formed and then dropped.  Layer i's own
     parameters are not read again after that, so the result equals theta - lr grad J."""
-    g0, store = input_cotangent(layers, params, x0, target, loss, reseed_every, masks)
+    g0, store = input_cotangent(layers, params, x0, target, loss, reseed_every, masks, frag_block)
     new = [np.array(p, dtype=np.float64) for p in params]
 
     def apply(i, g):
-        new[i] = new[i] - lr * g
+        new[i] = new[i] - lr * g * trainable_entries(layers[i], params[i])
 
     forward_sweep(layers, params, x0, g0, store, conv_iters, apply=apply)
     return new

@@ -525,7 +525,11 @@ mw_status conv1d_tensor_forward_sweep(mw_net* n, const void* const* params, cons
     }
     if (reseed_next)
       MW_TRY(split_planes(c.at<float>(lay.reseed[l + 1]), c.P, hout, 3, c.P, s));
-    if (dW[l]) MW_TRY(wgrad(c, xin, gzp, c.P, (float*)dW[l], l));
+    if (dW[l]) {
+      MW_TRY(wgrad(c, xin, gzp, c.P, (float*)dW[l], l));
+      if (n->apply_params)   // the zeros of tap 0 are structure, not parameters
+        MW_TRY(conv_zero_fixed_entries((float*)dW[l], 0, C, s));
+    }
   }
   return MW_OK;
 }

@@ -29,6 +29,19 @@ slice_sum_f32_kernel(const float* __restrict__ part, int64_t n, int64_t stride, 
 // core truncates its fp32 accumulator at every instruction, a bias that grows with the length of
 // one accumulation (about 1e-4 relative after 1024 K blocks) and that the fixed-order sum of the
 // slices, in round-to-nearest fp32, does not have.
+__global__ void __launch_bounds__(256)
+zero_above_diagonal_kernel(float* __restrict__ tap, int C) {
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= C * C) return;
+  const int c = i / C, cp = i - c * C;
+  if (c < cp) tap[i] = 0.f;
+}
+
+mw_status conv_zero_fixed_entries(float* w, int64_t offset, int C, cudaStream_t s) {
+  zero_above_diagonal_kernel<<<(C * C + 255) / 256, 256, 0, s>>>(w + offset, C);
+  return launch_ok();
+}
+
 mw_status conv_slice_sum(const float* part, int64_t n, int slices, float* out, const float* theta,
                          float lr, cudaStream_t s) {
   slice_sum_f32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(part, n, n, slices, out, theta, lr);

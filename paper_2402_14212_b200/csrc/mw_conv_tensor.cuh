@@ -37,6 +37,10 @@ bool conv_transpose_class_product(const ConvGeom& g, int py, int px, const __nv_
 // dw[k*k][C][C] = sum over output pixels; `partials` holds conv_wgrad_tensor_slices(out pixels)
 // copies of dw
 int conv_wgrad_tensor_slices(int64_t pixels);
+// Constrained parameterisation (Section "Constrained Convolutions"): the entries of the C x C tap
+// at w + offset that Lemma 1 (ii) fixes (c < c') are not parameters; after a fused update they are
+// put back to zero.
+mw_status conv_zero_fixed_entries(float* w, int64_t offset, int C, cudaStream_t s);
 // out[i] = sum over the slices (in order) of part[z*n + i]; with `theta`: theta[i] - lr * that sum
 mw_status conv_slice_sum(const float* part, int64_t n, int slices, float* out, const float* theta,
                          float lr, cudaStream_t s);

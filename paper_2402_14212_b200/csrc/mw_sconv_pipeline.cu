@@ -401,6 +401,8 @@ mw_status sconv_tensor_forward_sweep(mw_net* n, const void* const* params, const
       MW_TRY(conv_wgrad_tensor(c.cache, g, xin, c.at<__nv_bfloat16>(lay.cg[0]), 2, c.at<float>(lay.cpart),
                                (float*)dW[l], c.st, s,
                                n->apply_params ? (const float*)n->apply_params[l] : nullptr, n->apply_lr));
+    if (dW[l] && n->apply_params)   // the zeros of the anchor tap are structure, not parameters
+      MW_TRY(conv_zero_fixed_entries((float*)dW[l], (int64_t)(ld.pad * ld.k + ld.pad) * C * C, C, s));
   }
   return MW_OK;
 }

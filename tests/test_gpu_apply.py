@@ -59,3 +59,41 @@ def test_fused_update_unsupported_precisions():
     g0 = net.input_cotangent(params, x, target, ws)
     with pytest.raises(mwb.MwError):
         net.forward_sweep_apply(params, x, g0, 0.1, ws)
+
+
+@pytest.mark.parametrize("name", ["dense", "strided", "conv1d"])
+def test_gradient_descent_loop_follows_the_oracle(name):
+    """A few steps of plain gradient descent with the update fused into the sweep, in place: the loss
+    falls, and it falls the way the oracle's own loop (fp64, Algorithm 1 with theta_i updated as g_i
+    appears) says it should."""
+    import torch
+    if name == "dense":
+        p = S.deep_mlp(seed=5, depth=4, n=128, batch=64, reseed_every=2)
+    elif name == "strided":
+        p = S.strided_cnn(seed=5, depth=3, C=64, H=32, W=32, batch=4, gamma=0.5, reseed_every=2, prec=S.F32)
+    else:
+        p = S.fragmental_cnn1d(seed=5, depth=3, C=64, N=128, batch=4, block=8, reseed_every=2, prec=S.F32)
+    g = O.backprop(p.layers, p.params, p.x, p.target, p.loss)["dW"]
+    lr = 0.02 * max(float(np.abs(w).max()) for w in p.params) / max(float(np.abs(d).max()) for d in g)
+    steps = 4
+    theta = [np.array(w) for w in p.params]
+    want = []
+    for _ in range(steps):
+        want.append(O.backprop(p.layers, theta, p.x, p.target, p.loss)["loss"])
+        theta = O.moonwalk_sgd_step(p.layers, theta, p.x, p.target, p.loss, lr, reseed_every=p.reseed_every,
+                                    frag_block=p.frag_block)
+    net = mwb.net_for(p, backend="tensor")
+    params, x, target = mwb.to_device(p)
+    ws = net.alloc_workspace("moonwalk")
+    loss = torch.zeros(1, dtype=torch.float64, device="cuda")
+    got = []
+    for _ in range(steps):
+        g0 = net.input_cotangent(params, x, target, ws, loss_out=loss)
+        got.append(float(loss.item()))
+        net.forward_sweep_apply(params, x, g0, lr, ws)
+    assert net.last_device_status(ws)[0] == 0
+    assert all(b < a for a, b in zip(got, got[1:]))
+    for a, b in zip(got, want):
+        assert abs(a - b) <= 2e-4 * abs(b), (got, want)
+    for w, t in zip(params, theta):
+        assert O.normwise_error(w.double().cpu().numpy().reshape(t.shape), t) <= 1e-4

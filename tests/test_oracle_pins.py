@@ -367,6 +367,25 @@ def test_sgd_step_through_the_sweep():
     assert abs((J0 - J1) - lr * g2) <= 0.05 * lr * g2
 
 
+def test_sgd_step_keeps_constrained_convolutions_submersive():
+    # Section "Constrained Convolutions": the zeros that Lemma 1 (ii) demands are structure, not
+    # parameters; a step moves every other entry by -lr * gradient and leaves the layer submersive
+    p = S.strided_cnn(seed=6, depth=2, C=4, H=8, W=8, batch=2, gamma=1.0, reseed_every=0, prec=S.F64)
+    ref = O.backprop(p.layers, p.params, p.x, p.target, p.loss)
+    new = O.moonwalk_sgd_step(p.layers, p.params, p.x, p.target, p.loss, 0.5)
+    for layer, w, g, wn in zip(p.layers, p.params, ref["dW"], new):
+        assert O.submersive_conditions(layer, wn) == []
+        fixed = np.zeros(w.shape, dtype=bool)
+        fixed[1, 1] = np.triu(np.ones((4, 4), dtype=bool), 1)
+        assert np.abs(g[fixed]).max() > 0                       # the raw gradient is not zero there
+        assert np.array_equal(wn[fixed], w[fixed])
+        assert np.allclose(wn[~fixed], (w - 0.5 * g)[~fixed], rtol=0, atol=1e-13)
+    q = S.fragmental_cnn1d(seed=6, depth=2, C=4, N=16, batch=2, block=4, reseed_every=0, prec=S.F64)
+    new = O.moonwalk_sgd_step(q.layers, q.params, q.x, q.target, q.loss, 0.5, frag_block=4)
+    for w, wn in zip(q.params, new):
+        assert np.all(np.triu(wn[0], 1) == 0.0) and np.abs(wn[1] - w[1]).max() > 0
+
+
 def test_cotangent_recursion_error_grows_with_depth():
     # the forward recursion amplifies rounding error layer by layer (leaky slope 0.1): an
     # invariant of the method that fixes the need for re-seeding, reproducible in fp64
