@@ -42,7 +42,7 @@ typedef struct mw_net mw_net; /* opaque, host side; owns no device memory */
 typedef enum {
   MW_OK = 0,
   MW_ERR_INVALID_ARG = 1,    /* null pointer, bad enum, inconsistent sizes               */
-  MW_ERR_UNSUPPORTED = 2,    /* layer / size combination this build has no kernel for   */
+  MW_ERR_UNSUPPORTED = 2,    /* layer / size combination the library has no kernel for  */
   MW_ERR_WORKSPACE = 3,      /* workspace null, misaligned (256 B) or too small          */
   MW_ERR_STATE = 4,          /* sweep called without a matching mw_input_cotangent       */
   MW_ERR_NOT_SUBMERSIVE = 5, /* a layer's Jacobian could not be inverted to tolerance    */
