@@ -50,11 +50,13 @@ CCtx make_cctx(mw_net* n, const Layout& lay, void* ws, cudaStream_t s) {
   return c;
 }
 
-// terms of the operands of update t (1-based) of `T`: the last four updates are fp32-accurate,
-// the three before them carry two terms, earlier ones one
+// terms of the operands of update t (1-based) of `T`: the last two updates are fp32-accurate, the
+// three before them carry two terms, earlier ones one.  An update's rounding error (4e-3, 1.5e-5,
+// 1e-7 relative for 1, 2, 3 terms) is contracted by the later updates (0.14 each for the default
+// kernels): two later updates take a two-term error to 3e-7, five take a one-term error there.
 int update_terms(int t, int T) {
   const int left = T - t;
-  return left < 4 ? 3 : (left < 7 ? 2 : 1);
+  return left < 2 ? 3 : (left < 5 ? 2 : 1);
 }
 
 // w^[tap] = Winv w[tap] for tap != centre, zero at the centre; one block per (tap, row, layer)

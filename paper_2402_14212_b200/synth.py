@@ -168,7 +168,7 @@ def sweep_mlp(seed=0, depth=32, n=4096, batch=1024, reseed_every=4, prec=BF16,
 
 
 def submersive_cnn(seed=0, depth=32, C=64, H=32, W=32, batch=128, gamma=0.05, classes=10,
-                   reseed_every=4, conv_vijp_iters=10, prec=F32) -> Problem:
+                   reseed_every=4, conv_vijp_iters=8, prec=F32) -> Problem:
     """Config 3: stride-1 3x3 same-size convolutions with a dominant identity centre tap.
 
     w = delta_centre * I + gamma * N(0, 2/(9*C)) (He scale), leaky 0.1, linear head
