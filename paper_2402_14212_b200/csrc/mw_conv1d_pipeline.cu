@@ -247,7 +247,7 @@ TcGemm transpose_product(const C1& c, const __nv_bfloat16* g, const __nv_bfloat1
 mw_status wgrad(const C1& c, const __nv_bfloat16* x, const __nv_bfloat16* g, int64_t g_stride, float* dw,
                 int layer) {
   const int64_t px = c.P / c.C;
-  const int slices = conv_wgrad_tensor_slices(px);
+  const int slices = conv_wgrad_tensor_slices(px, c.C, c.k);
   const int rows = c.k * c.C;
   TcGemm p;
   p.A = pixel_operand(x, px, 2, c.P, true, c.C);
@@ -427,7 +427,7 @@ void conv1d_tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
   for (int i = 0; i < 2; ++i) lay.hp[i] = b.take(2 * 3 * P);
   lay.cw.resize(L); lay.cwinv.resize(L); lay.cwhat.resize(L);
   for (int l = 0; l < L; ++l) lay.cw[l] = b.take(2 * 3 * we);
-  lay.cpart = b.take(4 * (size_t)conv_wgrad_tensor_slices((int64_t)n->B * d.W) * we);
+  lay.cpart = b.take(4 * (size_t)conv_wgrad_tensor_slices((int64_t)n->B * d.W, C, k) * we);
   if (!backprop) {
     lay.cg[0] = b.take(2 * 3 * P);                      // g_z rebuilt block by block (three terms)
     lay.chpf = b.take(4 * P);                           // c = h W0^-T

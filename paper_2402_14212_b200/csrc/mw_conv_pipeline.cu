@@ -267,7 +267,7 @@ void conv_tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
   lay.cw.resize(L); lay.cwhat.resize(L); lay.cwinv.resize(L);
   for (int l = 0; l < Lc; ++l) lay.cw[l] = b.take(2 * 3 * we);
   if (head) lay.clogits = b.take(4 * 2 * (size_t)n->B * n->layers[L - 1].n_out);
-  lay.cpart = b.take(4 * (size_t)conv_wgrad_tensor_slices((int64_t)n->B * d.H * d.W) * we);
+  lay.cpart = b.take(4 * (size_t)conv_wgrad_tensor_slices((int64_t)n->B * d.H * d.W, 64, d.k * d.k) * we);
   if (!backprop) {
     for (int i = 0; i < 2; ++i) lay.cg[i] = b.take(2 * 3 * P);
     lay.chpf = b.take(4 * P);

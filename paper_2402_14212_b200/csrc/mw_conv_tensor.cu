@@ -25,10 +25,6 @@ slice_sum_f32_kernel(const float* __restrict__ part, int64_t n, int64_t stride, 
 
 }  // namespace
 
-// Slices of the pixel sum.  A slice is at most 128 K blocks where the sum is long: the tensor
-// core truncates its fp32 accumulator at every instruction, a bias that grows with the length of
-// one accumulation (about 1e-4 relative after 1024 K blocks) and that the fixed-order sum of the
-// slices, in round-to-nearest fp32, does not have.
 __global__ void __launch_bounds__(256)
 zero_above_diagonal_kernel(float* __restrict__ tap, int C) {
   const int i = blockIdx.x * 256 + threadIdx.x;
@@ -48,13 +44,30 @@ mw_status conv_slice_sum(const float* part, int64_t n, int slices, float* out, c
   return launch_ok();
 }
 
-int conv_wgrad_tensor_slices(int64_t pixels) {
+// Slices of the pixel sum.  A slice is at most 128 K blocks where the sum is long: the tensor
+// core truncates its fp32 accumulator at every instruction, a bias that grows with the length of
+// one accumulation (about 1e-4 relative after 1024 K blocks) and that the fixed-order sum of the
+// slices, in round-to-nearest fp32, does not have.
+int conv_wgrad_tensor_slices(int64_t pixels, int C, int taps) {
   const int64_t blocks = pixels / 64;
-  for (int s = 256; s > 32; s >>= 1)
-    if (blocks % s == 0 && blocks / s >= 64) return s;
-  for (int s = 32; s > 1; s >>= 1)
-    if (blocks % s == 0 && blocks / s >= 4) return s;
-  return 1;
+  // output tiles of one slice: 128 rows (tap, channel) x all C columns (two-term operands)
+  const int tiles = ((taps * C + 127) / 128) * (C % 128 == 0 ? C / 128 : C / 64);
+  const int sms = 148;
+  // Among the powers of two that divide the K blocks (at most 128 K blocks per slice where the sum
+  // is long enough, at least 4), the one with the shortest estimated time: waves of `sms` units,
+  // each unit about 6 us of set-up and epilogue plus 0.8 us per K block.
+  int best = 1;
+  double best_t = 1e30;
+  for (int s = 1; s <= 256; s <<= 1) {
+    if (blocks % s != 0) break;
+    const int64_t kb = blocks / s;
+    if (s > 1 && kb < 4) break;
+    const double waves = (double)(((int64_t)tiles * s + sms - 1) / sms);
+    double t = waves * (6.0 + 0.8 * (double)kb);
+    if (kb > 128) t *= 4.0;     // long accumulations lose accuracy (see above): strongly disfavoured
+    if (t < best_t) { best_t = t; best = s; }
+  }
+  return best;
 }
 
 TcOperand pixel_operand(const void* planes, int64_t pixels, int terms, int64_t plane_stride, bool mn,
@@ -150,8 +163,8 @@ TcGemm conv_transpose_product(const ConvGeom& g, const __nv_bfloat16* g_planes, 
 mw_status conv_wgrad_tensor(TcMapCache* cache, const ConvGeom& g, const __nv_bfloat16* x_planes,
                             const __nv_bfloat16* gz_planes, int terms, float* partials, float* dw,
                             DeviceStatus* st, cudaStream_t s, const float* theta, float lr) {
-  const int slices = conv_wgrad_tensor_slices(g.out_pixels());
   const int C = g.C;
+  const int slices = conv_wgrad_tensor_slices(g.out_pixels(), C, g.k * g.k);
   const int rows = g.k * g.k * C;
   TcGemm p;
   p.A = pixel_operand(x_planes, g.pixels(), terms, g.pixels() * C, true, C);
@@ -192,7 +205,7 @@ extern "C" mw_status mw_conv2d_strided_split_bf16(int32_t op, const float* a, co
   const int64_t ew = g.kernel_elems();
   const int64_t ea = op == 1 ? pout : pin;
   const int64_t eb = op == 2 ? pout : ew;
-  const int slices = conv_wgrad_tensor_slices(g.out_pixels());
+  const int slices = conv_wgrad_tensor_slices(g.out_pixels(), C, k * k);
   const size_t sa = align_up((size_t)ea, 128), sb = align_up((size_t)eb, 128);
   const size_t need = 256 + 2 * (size_t)terms * (sa + sb) + (op == 2 ? (size_t)slices * ew * 4 : 0) + 512;
   if (((uintptr_t)scratch & 255u) || scratch_bytes < need) return MW_ERR_WORKSPACE;

@@ -36,7 +36,7 @@ bool conv_transpose_class_product(const ConvGeom& g, int py, int px, const __nv_
                                   TcGemm* out);
 // dw[k*k][C][C] = sum over output pixels; `partials` holds conv_wgrad_tensor_slices(out pixels)
 // copies of dw
-int conv_wgrad_tensor_slices(int64_t pixels);
+int conv_wgrad_tensor_slices(int64_t pixels, int C = 64, int taps = 9);
 // Constrained parameterisation (Section "Constrained Convolutions"): the entries of the C x C tap
 // at w + offset that Lemma 1 (ii) fixes (c < c') are not parameters; after a fused update they are
 // put back to zero.

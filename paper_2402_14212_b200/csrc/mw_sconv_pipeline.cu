@@ -303,7 +303,7 @@ void sconv_tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
   for (int l = 0; l < L; ++l) {
     const size_t w = (size_t)n->info[l].w_elems;
     if (w > we) we = w;
-    const size_t p = 4 * (size_t)conv_wgrad_tensor_slices(n->info[l].rows) * w;
+    const size_t p = 4 * (size_t)conv_wgrad_tensor_slices(n->info[l].rows, C, n->layers[l].k * n->layers[l].k) * w;
     if (p > part) part = p;
   }
   for (int i = 0; i < 2; ++i) lay.cot[i] = b.take(4 * PL);

@@ -68,6 +68,7 @@ struct alignas(64) TcProblem {
   unsigned int* split_counters;
   // convolution forms (TcConv)
   int conv_mode, cHo, cWo, ck, cpad, cstride, ccb, b_tap_rows, cntaps, c1d;
+  int cbx, cby, cbi;           // pixels, rows and images of one A box
   signed char tdy[28], tdx[28], ttb[28];
   // program launches: products (by index) that must be complete before this one starts, and
   // the number of warp arrivals that completes each of them (one per epilogue warp and tile)
@@ -559,6 +560,28 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           cy0 = rem / P.cWo;
           cx0 = rem - cy0 * P.cWo;
         }
+        // weight vjp: the window of each half of the A tile (constant over the K blocks) and the
+        // position of the unit's first K block; the divisions are kept out of the K loop, where
+        // this single lane's integer work is what paces the copies
+        int wg_c0[2] = {0, 0}, wg_ox[2] = {0, 0}, wg_oy[2] = {0, 0};
+        int wg_b = 0, wg_y = 0, wg_x = 0;
+        if (conv == TC_CONV_WGRAD) {
+          const int r0 = 2 * (w.m0 / BM);
+          for (int hh = 0; hh < 2; ++hh) {
+            int tap = (r0 + hh) / P.ccb;
+            wg_c0[hh] = ((r0 + hh) - tap * P.ccb) * BK;
+            if (tap >= P.cntaps) tap = P.cntaps - 1;   // rows past the last tap are never stored
+            const int j0 = P.c1d ? 0 : tap / P.ck, j1 = tap - j0 * P.ck;
+            wg_ox[hh] = j1 - P.cpad;
+            wg_oy[hh] = P.c1d ? 0 : j0 - P.cpad;
+          }
+          const int pix = (w.z * P.num_kb + w.kb0) * BK;
+          const int hw = P.cHo * P.cWo;
+          wg_b = pix / hw;
+          const int rem = pix - wg_b * hw;
+          wg_y = rem / P.cWo;
+          wg_x = rem - wg_y * P.cWo;
+        }
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, p.st, 1u, abortp)) { ok = false; break; }
           const uint32_t fb = smem_u32(&full_bar[stage]);
@@ -575,22 +598,19 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
             bk0 = (tb * P.ccb + cblk) * BK;
             if (P.b_tap_rows) { bn0 = tb * P.N + w.n0; bk0 = cblk * BK; }
           } else if (conv == TC_CONV_WGRAD) {
-            // K block = 64 pixels of slice z; the two halves of the A tile are two blocks of 64
-            // rows (tap, channel block)
+            // K block = 64 pixels of slice z (one box: part of a row, rows, or images); the two
+            // halves of the A tile are two blocks of 64 rows (tap, channel block)
             const int pix = (w.z * P.num_kb + kb) * BK;
-            const int hw = P.cHo * P.cWo;
-            const int b = pix / hw, rem = pix - b * hw;
-            const int y0 = rem / P.cWo, x0 = rem - y0 * P.cWo;
-            const int r0 = 2 * (w.m0 / BM);
-            for (int hh = 0; hh < 2; ++hh) {
-              int tap = (r0 + hh) / P.ccb;
-              const int cblk = (r0 + hh) - tap * P.ccb;
-              if (tap >= P.cntaps) tap = P.cntaps - 1;   // rows past the last tap are never stored
-              const int j0 = P.c1d ? 0 : tap / P.ck, j1 = tap - j0 * P.ck;
-              const int oy = P.c1d ? 0 : j0 - P.cpad;
+            for (int hh = 0; hh < 2; ++hh)
               for (int pl = 0; pl < pa; ++pl)
-                tma_load_5d(sbase + (uint32_t)pl * kATileBytes + (uint32_t)hh * 8192u, &P.tmA, fb, cblk * BK,
-                            P.cstride * x0 + j1 - P.cpad, P.cstride * y0 + oy, b, pl);
+                tma_load_5d(sbase + (uint32_t)pl * kATileBytes + (uint32_t)hh * 8192u, &P.tmA, fb, wg_c0[hh],
+                            P.cstride * wg_x + wg_ox[hh], P.cstride * wg_y + wg_oy[hh], wg_b, pl);
+            // next box
+            wg_x += P.cbx;
+            if (wg_x >= P.cWo) {
+              wg_x = 0;
+              wg_y += P.cby;
+              if (wg_y >= P.cHo) { wg_y = 0; wg_b += P.cbi; }
             }
             bk0 = pix;
             k0 = pix;
@@ -1090,6 +1110,7 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
     cbi = span / (cbx * cby);
     if (cbx * cby * cbi != span) return MW_ERR_UNSUPPORTED;
     P.cHo = Ho; P.cWo = Wo; P.cstride = cv.stride; P.ccb = C / 64;
+    P.cbx = cbx; P.cby = cby; P.cbi = cbi;
     P.ck = cv.k; P.cpad = cv.pad; P.b_tap_rows = cv.b_tap_rows;
     if (cv.mode == TC_CONV_PIXELS) {
       int nt = 0;
