@@ -563,6 +563,11 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         // weight vjp: the window of each half of the A tile (constant over the K blocks) and the
         // position of the unit's first K block; the divisions are kept out of the K loop, where
         // this single lane's integer work is what paces the copies
+        int px_t = 0, px_c = 0;      // window and channel block of the next K block (TC_CONV_PIXELS)
+        if (conv == TC_CONV_PIXELS) {
+          px_t = w.kb0 / P.ccb;
+          px_c = w.kb0 - px_t * P.ccb;
+        }
         int wg_c0[2] = {0, 0}, wg_ox[2] = {0, 0}, wg_oy[2] = {0, 0};
         int wg_b = 0, wg_y = 0, wg_x = 0;
         if (conv == TC_CONV_WGRAD) {
@@ -590,7 +595,8 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           int k0 = kb * BK;
           int bk0 = k0, bn0 = w.n0;       // B coordinates (K, N)
           if (conv == TC_CONV_PIXELS) {
-            const int t = kb / P.ccb, cblk = kb - t * P.ccb;
+            const int t = px_t, cblk = px_c;
+            if (++px_c == P.ccb) { px_c = 0; ++px_t; }
             const int dy = P.tdy[t], dx = P.tdx[t], tb = P.ttb[t];
             for (int pl = 0; pl < pa; ++pl)
               tma_load_5d(sbase + (uint32_t)pl * kATileBytes, &P.tmA, fb, cblk * BK, P.cstride * cx0 + dx,
