@@ -246,3 +246,24 @@ def test_fragmental_cnn1d_full_size():
         assert worst[l] <= 1e-4 * np.sqrt(l + 1.0), (l, worst[l])
         assert O.normwise_error(out["dW"][l], dW[l]) <= 1e-4, l
     assert abs(out["loss"] - loss) <= 1e-4 * abs(loss)
+
+
+@pytest.mark.parametrize("family", ["strided", "conv1d"])
+def test_cnn_sweep_skips_layers_without_an_output(family):
+    """A NULL entry of dW_out skips that layer's weight vjp (gradients need not coexist, Section 4.3);
+    the other layers' gradients are unchanged, bit for bit."""
+    import torch
+    from paper_2402_14212_b200 import synth as S
+    if family == "strided":
+        p = S.strided_cnn(seed=7, depth=4, C=64, H=32, W=32, batch=16, gamma=0.5, reseed_every=2, prec=S.F32)
+    else:
+        p = S.fragmental_cnn1d(seed=7, depth=4, C=64, N=128, batch=4, block=8, reseed_every=2, prec=S.F32)
+    net = mwb.net_for(p, backend="tensor")
+    params, x, target = mwb.to_device(p)
+    ws = net.alloc_workspace("moonwalk")
+    g0 = net.input_cotangent(params, x, target, ws)
+    full = [d.clone() for d in net.forward_sweep(params, x, g0, ws)]
+    some = [None, torch.zeros_like(params[1]), None, torch.zeros_like(params[3])]
+    net.forward_sweep(params, x, g0, ws, dW_out=some)
+    assert net.last_device_status(ws)[0] == 0
+    assert torch.equal(some[1], full[1]) and torch.equal(some[3], full[3])
