@@ -52,6 +52,8 @@ def workload(name: str, seed: int = 0, depth: int = 0, block: int = 0):
         # the paper's own convolutional experiment: 256 x 256 x 128 inputs, batch 128, 3x3 stride-2
         # submersive layers (`depth` of them, 8 by default: down to 1 x 1)
         return S.strided_cnn(seed=seed, depth=depth or 8)
+    if name == "strided_cnn_bf16":
+        return S.strided_cnn(seed=seed, depth=depth or 8, prec=S.BF16)
     if name == "strided_cnn_small":
         return S.strided_cnn(seed=seed, depth=depth or 4, H=64, W=64, batch=16)
     if name == "fragmental_cnn1d":

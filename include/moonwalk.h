@@ -99,7 +99,7 @@ typedef struct {
 /* Build a host-side description.  `batch` is fixed per net.  Returns MW_ERR_UNSUPPORTED for
  * shapes outside: dense layers square; convolutions with C_in = C_out, either stride 1 with
  * k = 2*pad+1 (same size), or every layer of the net meeting Lemma 1 (i) with stride 2 (the
- * paper's submersive CNN: MW_F32, 64 or 128 channels, k - 1 - pad < 2, even image sizes, a
+ * paper's submersive CNN: MW_F32 or MW_BF16_F32ACC, 64 or 128 channels, k - 1 - pad < 2, even image sizes, a
  * loss on the last feature map; conditions (ii) and (iii) on the anchor tap w[pad][pad] are
  * checked on the device every step: MW_ERR_NOT_SUBMERSIVE); MW_CONV1D nets: every layer k = 3,
  * stride 1, padding 1, the same W (a multiple of 128) and C (64..256, a multiple of 64), MW_F32,
