@@ -60,6 +60,8 @@ def workload(name: str, seed: int = 0, depth: int = 0, block: int = 0):
         # the paper's 1-D experiment: 2048 x 256 sequences, batch 128, k = 3 stride-1 convolutions,
         # output cotangents checkpointed at 2 of every `block` positions
         return S.fragmental_cnn1d(seed=seed, depth=depth or 16, block=block or 4)
+    if name == "fragmental_cnn1d_bf16":
+        return S.fragmental_cnn1d(seed=seed, depth=depth or 16, block=block or 4, prec=S.BF16)
     if name == "tiny_mlp":
         return S.tiny_mlp(seed=seed)
     raise SystemExit(f"unknown workload {name}")

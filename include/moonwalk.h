@@ -102,7 +102,8 @@ typedef struct {
  * paper's submersive CNN: MW_F32 or MW_BF16_F32ACC, 64 or 128 channels, k - 1 - pad < 2, even image sizes, a
  * loss on the last feature map; conditions (ii) and (iii) on the anchor tap w[pad][pad] are
  * checked on the device every step: MW_ERR_NOT_SUBMERSIVE); MW_CONV1D nets: every layer k = 3,
- * stride 1, padding 1, the same W (a multiple of 128) and C (64..256, a multiple of 64), MW_F32,
+ * stride 1, padding 1, the same W (a multiple of 128) and C (64..256, a multiple of 64), MW_F32 or
+ * MW_BF16_F32ACC,
  * tap 0 lower triangular in (c_in, c_out) with a non-zero diagonal (checked on the device);
  * head only as the last layer; all layers of one net share `prec`. */
 mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers, int32_t batch,

@@ -29,14 +29,24 @@ struct C1 {
   TcMapCache* cache;
   DeviceStatus* st;
   int L, C, N, k, blk;
+  // bf16 terms per operand: MW_F32 three on the chains and two in the weight vjp; MW_BF16_F32ACC:
+  // x and w are bf16 in memory and serve as their own single plane, cotangents and W0^-1 two terms
+  bool bf16;
+  int px, pw, pg, pwg;
+  const void* const* params;
+  const void* x;
   int64_t P;          // elements of one activation: B * N * C
   int64_t we;         // elements of one kernel: k * C * C
   template <typename T> T* at(const Region& r) const { return mw::at<T>(ws, r); }
 };
 
-C1 make_c1(mw_net* n, const Layout& lay, void* ws, cudaStream_t s) {
+C1 make_c1(mw_net* n, const Layout& lay, void* ws, cudaStream_t s, const void* const* params,
+           const void* x) {
   C1 c;
   c.n = n; c.lay = &lay; c.ws = ws; c.s = s;
+  c.params = params; c.x = x;
+  c.bf16 = n->opts.prec == MW_BF16_F32ACC;
+  c.px = c.bf16 ? 1 : 3; c.pw = c.px; c.pg = c.bf16 ? 2 : 3; c.pwg = c.bf16 ? 1 : 2;
   c.cache = static_cast<TensorState*>(n->tc)->cache;
   c.st = status_of(ws, lay);
   const mw_layer_desc& d = n->layers[0];
@@ -51,17 +61,21 @@ C1 make_c1(mw_net* n, const Layout& lay, void* ws, cudaStream_t s) {
 // columns), one thread per column, x_i = (delta_ij - sum_{m<i} A[i][m] x_m) / A[i][i] in double,
 // the columns of the group in shared memory ([n][64] doubles)
 constexpr int kTriCols = 64;
+__device__ __forceinline__ float ld_f(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float ld_f(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+template <typename T>
 __global__ void __launch_bounds__(kTriCols)
 tri_inverse_kernel(SmallBatch ws, int n, float* __restrict__ inv0, DeviceStatus* st, int layer0) {
   extern __shared__ double xs[];            // [n][kTriCols]
-  const float* A = static_cast<const float*>(ws.p[blockIdx.x]);
+  const T* A = static_cast<const T*>(ws.p[blockIdx.x]);
   float* inv = inv0 + (int64_t)blockIdx.x * n * n;
   __shared__ int bad;
   if (threadIdx.x == 0) bad = 0;
   __syncthreads();
   for (int e = threadIdx.x; e < n * n; e += blockDim.x) {
     const int i = e / n, j = e - i * n;
-    const float v = A[e];
+    const float v = ld_f(A + e);
     if ((j > i && v != 0.f) || (j == i && !(fabsf(v) > 0.f))) bad = 1;
   }
   __syncthreads();
@@ -76,19 +90,19 @@ tri_inverse_kernel(SmallBatch ws, int n, float* __restrict__ inv0, DeviceStatus*
     double a = i == j ? 1.0 : 0.0;
     if (i > j) {
       // four independent partial sums: the chain of dependent fp64 adds is what takes the time
-      const float* Ai = A + (int64_t)i * n;
+      const T* Ai = A + (int64_t)i * n;
       double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
       int m = j;
       for (; m + 3 < i; m += 4) {
-        s0 += (double)__ldg(Ai + m) * xs[m * kTriCols + t];
-        s1 += (double)__ldg(Ai + m + 1) * xs[(m + 1) * kTriCols + t];
-        s2 += (double)__ldg(Ai + m + 2) * xs[(m + 2) * kTriCols + t];
-        s3 += (double)__ldg(Ai + m + 3) * xs[(m + 3) * kTriCols + t];
+        s0 += (double)ld_f(Ai + m) * xs[m * kTriCols + t];
+        s1 += (double)ld_f(Ai + m + 1) * xs[(m + 1) * kTriCols + t];
+        s2 += (double)ld_f(Ai + m + 2) * xs[(m + 2) * kTriCols + t];
+        s3 += (double)ld_f(Ai + m + 3) * xs[(m + 3) * kTriCols + t];
       }
-      for (; m < i; ++m) s0 += (double)__ldg(Ai + m) * xs[m * kTriCols + t];
+      for (; m < i; ++m) s0 += (double)ld_f(Ai + m) * xs[m * kTriCols + t];
       a -= (s0 + s1) + (s2 + s3);
     }
-    const double x = i < j ? 0.0 : a / (double)A[(int64_t)i * n + i];
+    const double x = i < j ? 0.0 : a / (double)ld_f(A + (int64_t)i * n + i);
     xs[i * kTriCols + t] = x;
     inv[(int64_t)i * n + j] = (float)x;
   }
@@ -106,16 +120,17 @@ __device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
 
 // fold[c][(q, c')] = sum_m W0inv[c][m] w[k-1-q][m][c'], q = 0 .. k-2: the B operand of a
 // reconstruction step, whose K runs over the k - 1 previous positions, oldest first
+template <typename T>
 __global__ void __launch_bounds__(256)
 fold1d_kernel(SmallBatch ws, const float* __restrict__ inv0, int C, int k, float* __restrict__ fold0) {
   const int c = blockIdx.x, q = blockIdx.y, cp = threadIdx.x;
-  const float* w = static_cast<const float*>(ws.p[blockIdx.z]);
+  const T* w = static_cast<const T*>(ws.p[blockIdx.z]);
   const float* inv = inv0 + (int64_t)blockIdx.z * C * C;
   float* fold = fold0 + (int64_t)blockIdx.z * C * (k - 1) * C;
-  const float* wj = w + (int64_t)(k - 1 - q) * C * C;
+  const T* wj = w + (int64_t)(k - 1 - q) * C * C;
   for (int t = cp; t < C; t += blockDim.x) {
     float a = 0.f;
-    for (int m = 0; m < C; ++m) a = fmaf(inv[c * C + m], wj[(int64_t)m * C + t], a);
+    for (int m = 0; m < C; ++m) a = fmaf(inv[c * C + m], ld_f(wj + (int64_t)m * C + t), a);
     fold[((int64_t)c * (k - 1) + q) * C + t] = a;
   }
 }
@@ -224,8 +239,8 @@ TcConv window_list(const C1& c, bool transpose) {
 
 TcGemm forward_product(const C1& c, const __nv_bfloat16* x, const __nv_bfloat16* w, const TcEpilogue& e) {
   TcGemm p;
-  p.A = pixel_operand(x, c.P / c.C, 3, c.P, false, c.C);
-  p.B.base = w; p.B.rows = c.k * c.C; p.B.cols = c.C; p.B.planes = 3; p.B.plane_stride = c.we;
+  p.A = pixel_operand(x, c.P / c.C, c.px, c.P, false, c.C);
+  p.B.base = w; p.B.rows = c.k * c.C; p.B.cols = c.C; p.B.planes = c.pw; p.B.plane_stride = c.we;
   p.B.mn_major = true;                                        // w[j][ci][co]: K = (j, ci), N = co
   p.M = (int)(c.P / c.C); p.N = c.C; p.K = c.k * c.C;
   p.epi = e;
@@ -235,8 +250,8 @@ TcGemm forward_product(const C1& c, const __nv_bfloat16* x, const __nv_bfloat16*
 
 TcGemm transpose_product(const C1& c, const __nv_bfloat16* g, const __nv_bfloat16* w, const TcEpilogue& e) {
   TcGemm p;
-  p.A = pixel_operand(g, c.P / c.C, 3, c.P, false, c.C);
-  p.B.base = w; p.B.rows = c.k * c.C; p.B.cols = c.C; p.B.planes = 3; p.B.plane_stride = c.we;
+  p.A = pixel_operand(g, c.P / c.C, c.pg, c.P, false, c.C);
+  p.B.base = w; p.B.rows = c.k * c.C; p.B.cols = c.C; p.B.planes = c.pw; p.B.plane_stride = c.we;
   p.B.mn_major = false;                                       // rows (j, c), K = c'
   p.M = (int)(c.P / c.C); p.N = c.C; p.K = c.k * c.C;
   p.epi = e;
@@ -250,8 +265,8 @@ mw_status wgrad(const C1& c, const __nv_bfloat16* x, const __nv_bfloat16* g, int
   const int slices = conv_wgrad_tensor_slices(px, c.C, c.k);
   const int rows = c.k * c.C;
   TcGemm p;
-  p.A = pixel_operand(x, px, 2, c.P, true, c.C);
-  p.B = pixel_operand(g, px, 2, g_stride, true, c.C);
+  p.A = pixel_operand(x, px, c.pwg, c.P, true, c.C);
+  p.B = pixel_operand(g, px, c.pwg, g_stride, true, c.C);
   p.M = rows; p.N = c.C; p.K = (int)(px / slices); p.batch = slices;
   p.epi.mode = TC_EPI_PLAIN;
   float* part = c.at<float>(c.lay->cpart);
@@ -270,12 +285,15 @@ mw_status wgrad(const C1& c, const __nv_bfloat16* x, const __nv_bfloat16* g, int
 mw_status prep(const C1& c, const void* const* params, bool inverse) {
   const Layout& lay = *c.lay;
   const int C = c.C;
-  for (int l = 0; l < c.L; ++l)
-    MW_TRY(split_planes((const float*)params[l], c.we, c.at<__nv_bfloat16>(lay.cw[l]), 3, c.we, c.s));
+  if (!c.bf16)
+    for (int l = 0; l < c.L; ++l)
+      MW_TRY(split_planes((const float*)params[l], c.we, c.at<__nv_bfloat16>(lay.cw[l]), 3, c.we, c.s));
   if (!inverse) return MW_OK;
   static bool attr_done = false;
   if (!attr_done) {
-    MW_CUDA_OK(cudaFuncSetAttribute(tri_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    MW_CUDA_OK(cudaFuncSetAttribute(tri_inverse_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)(sizeof(double) * 256 * kTriCols)));
+    MW_CUDA_OK(cudaFuncSetAttribute(tri_inverse_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)(sizeof(double) * 256 * kTriCols)));
     attr_done = true;
   }
@@ -286,28 +304,41 @@ mw_status prep(const C1& c, const void* const* params, bool inverse) {
     const int G = c.L - l0 < kSmallBatch ? c.L - l0 : kSmallBatch;
     SmallBatch ws{};
     for (int g = 0; g < G; ++g) ws.p[g] = params[l0 + g];
-    tri_inverse_kernel<<<dim3(G, (C + kTriCols - 1) / kTriCols), kTriCols, sizeof(double) * C * kTriCols, c.s>>>(
-        ws, C, inv, c.st, l0);
-    MW_TRY(launch_ok());
-    fold1d_kernel<<<dim3(C, c.k - 1, G), 256, 0, c.s>>>(ws, inv, C, c.k, fold);
+    const dim3 tg(G, (C + kTriCols - 1) / kTriCols);
+    const size_t tsm = sizeof(double) * C * kTriCols;
+    if (c.bf16) {
+      tri_inverse_kernel<__nv_bfloat16><<<tg, kTriCols, tsm, c.s>>>(ws, C, inv, c.st, l0);
+      MW_TRY(launch_ok());
+      fold1d_kernel<__nv_bfloat16><<<dim3(C, c.k - 1, G), 256, 0, c.s>>>(ws, inv, C, c.k, fold);
+    } else {
+      tri_inverse_kernel<float><<<tg, kTriCols, tsm, c.s>>>(ws, C, inv, c.st, l0);
+      MW_TRY(launch_ok());
+      fold1d_kernel<float><<<dim3(C, c.k - 1, G), 256, 0, c.s>>>(ws, inv, C, c.k, fold);
+    }
     MW_TRY(launch_ok());
     for (int g = 0; g < G; ++g) {
-      MW_TRY(split_planes(inv + (int64_t)g * C * C, (int64_t)C * C, c.at<__nv_bfloat16>(lay.cwinv[l0 + g]), 3,
+      MW_TRY(split_planes(inv + (int64_t)g * C * C, (int64_t)C * C, c.at<__nv_bfloat16>(lay.cwinv[l0 + g]), c.pg,
                           (int64_t)C * C, c.s));
-      MW_TRY(split_planes(fold + (int64_t)g * fe, fe, c.at<__nv_bfloat16>(lay.cwhat[l0 + g]), 3, fe, c.s));
+      MW_TRY(split_planes(fold + (int64_t)g * fe, fe, c.at<__nv_bfloat16>(lay.cwhat[l0 + g]), c.pg, fe, c.s));
     }
   }
   return MW_OK;
 }
 
 __nv_bfloat16* x_planes(const C1& c, int l) {
+  // a bf16 input is its own (single) term plane
+  if (l == 0 && c.bf16) return const_cast<__nv_bfloat16*>(static_cast<const __nv_bfloat16*>(c.x));
   return c.at<__nv_bfloat16>(l == 0 ? c.lay->xp[0] : c.lay->xp[1 + ((l - 1) & 1)]);
+}
+
+const __nv_bfloat16* w_planes(const C1& c, int l) {
+  return c.bf16 ? static_cast<const __nv_bfloat16*>(c.params[l]) : c.at<__nv_bfloat16>(c.lay->cw[l]);
 }
 
 mw_status forward_pass(const C1& c, const void* const* params, const void* x, bool store_acts) {
   const Layout& lay = *c.lay;
   MW_TRY(prep(c, params, !store_acts));
-  MW_TRY(split_planes((const float*)x, c.P, x_planes(c, 0), 3, c.P, c.s));
+  if (!c.bf16) MW_TRY(split_planes((const float*)x, c.P, x_planes(c, 0), 3, c.P, c.s));
   const __nv_bfloat16* xin = x_planes(c, 0);
   for (int l = 0; l < c.L; ++l) {
     const mw_layer_desc& ld = c.n->layers[l];
@@ -319,9 +350,9 @@ mw_status forward_pass(const C1& c, const void* const* params, const void* x, bo
     e.write_mask = 1;
     e.act = ld.act;
     e.slope = (float)ld.slope;
-    if (!last) { e.planes = xout; e.n_planes = 3; e.plane_stride = c.P; }
+    if (!last) { e.planes = xout; e.n_planes = c.px; e.plane_stride = c.P; }
     else e.out_f32 = c.at<float>(lay.cxf);
-    TcGemm g = forward_product(c, xin, c.at<__nv_bfloat16>(lay.cw[l]), e);
+    TcGemm g = forward_product(c, xin, w_planes(c, l), e);
     MW_TRY(tc_gemm_group(c.cache, &g, 1, c.st, c.s));
     xin = xout;
   }
@@ -342,7 +373,7 @@ mw_status loss_top(const C1& c, const void* target, double* loss_out) {
     MW_TRY(scale_by_mask<float>(h, c.at<uint32_t>(lay.mask[l]), rows, c.C, ld.act, ld.slope, g, c.s));
     src = g;
   }
-  return split_planes(src, c.P, c.at<__nv_bfloat16>(lay.hp[0]), 3, c.P, c.s);
+  return split_planes(src, c.P, c.at<__nv_bfloat16>(lay.hp[0]), c.pg, c.P, c.s);
 }
 
 int64_t frag_elems(const C1& c) { return c.P / c.blk * (c.k - 1); }
@@ -356,7 +387,7 @@ mw_status backward_pass(const C1& c, void* g0, void* const* dW, bool moonwalk) {
       // fragmental checkpoint of this layer's g_z: the first k - 1 positions of every block
       const int64_t total8 = frag_elems(c) / 8;
       frag_gather_kernel<<<(unsigned)((total8 + 255) / 256), 256, 0, c.s>>>(
-          gz, 3, c.P, c.C, c.blk, c.k - 1, total8, c.at<float>(lay.cfrag[l]));
+          gz, c.pg, c.P, c.C, c.blk, c.k - 1, total8, c.at<float>(lay.cfrag[l]));
       MW_TRY(launch_ok());
     }
     if (dW && dW[l]) {
@@ -375,10 +406,10 @@ mw_status backward_pass(const C1& c, void* g0, void* const* dW, bool moonwalk) {
       e.slope = (float)below.slope;
       e.mask = c.at<uint32_t>(lay.mask[l - 1]);
       e.planes = c.at<__nv_bfloat16>(lay.hp[cur ^ 1]);
-      e.n_planes = 3;
+      e.n_planes = c.pg;
       e.plane_stride = c.P;
     }
-    TcGemm g = transpose_product(c, gz, c.at<__nv_bfloat16>(lay.cw[l]), e);
+    TcGemm g = transpose_product(c, gz, w_planes(c, l), e);
     MW_TRY(tc_gemm_group(c.cache, &g, 1, c.st, c.s));
     cur ^= 1;
   }
@@ -388,7 +419,7 @@ mw_status backward_pass(const C1& c, void* g0, void* const* dW, bool moonwalk) {
 }  // namespace
 
 bool conv1d_tensor_supported(const mw_net* n) {
-  if (n->opts.prec != MW_F32 || n->opts.loss == MW_LOSS_XENT_MEAN) return false;
+  if ((n->opts.prec != MW_F32 && n->opts.prec != MW_BF16_F32ACC) || n->opts.loss == MW_LOSS_XENT_MEAN) return false;
   const mw_layer_desc& d0 = n->layers[0];
   const int blk = n->opts.frag_block;
   if (d0.C_in < 64 || d0.C_in % 64 != 0 || d0.C_in > 256) return false;
@@ -423,17 +454,20 @@ void conv1d_tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
   }
   for (int i = 0; i < 2; ++i) lay.cot[i] = b.take(4 * P);
   lay.cxf = b.take(4 * P);
-  for (int i = 0; i < 3; ++i) lay.xp[i] = b.take(2 * 3 * P);
-  for (int i = 0; i < 2; ++i) lay.hp[i] = b.take(2 * 3 * P);
+  const bool bf16 = n->opts.prec == MW_BF16_F32ACC;
+  const size_t px = bf16 ? 1 : 3, pg = bf16 ? 2 : 3;
+  lay.xp[0] = b.take(bf16 ? 256 : 2 * 3 * P);
+  for (int i = 1; i < 3; ++i) lay.xp[i] = b.take(2 * px * P);
+  for (int i = 0; i < 2; ++i) lay.hp[i] = b.take(2 * pg * P);
   lay.cw.resize(L); lay.cwinv.resize(L); lay.cwhat.resize(L);
-  for (int l = 0; l < L; ++l) lay.cw[l] = b.take(2 * 3 * we);
+  for (int l = 0; l < L; ++l) lay.cw[l] = b.take(bf16 ? 256 : 2 * 3 * we);
   lay.cpart = b.take(4 * (size_t)conv_wgrad_tensor_slices((int64_t)n->B * d.W, C, k) * we);
   if (!backprop) {
-    lay.cg[0] = b.take(2 * 3 * P);                      // g_z rebuilt block by block (three terms)
+    lay.cg[0] = b.take(2 * pg * P);                     // g_z rebuilt block by block
     lay.chpf = b.take(4 * P);                           // c = h W0^-T
     for (int l = 0; l < L; ++l) {
-      lay.cwinv[l] = b.take(2 * 3 * (size_t)C * C);
-      lay.cwhat[l] = b.take(2 * 3 * (size_t)C * (k - 1) * C);
+      lay.cwinv[l] = b.take(2 * pg * (size_t)C * C);
+      lay.cwhat[l] = b.take(2 * pg * (size_t)C * (k - 1) * C);
     }
     lay.cwinv_f32 = b.take(4 * (size_t)C * C * kSmallBatch);
     lay.cwhat_f32 = b.take(4 * (size_t)C * (k - 1) * C * kSmallBatch);
@@ -445,7 +479,7 @@ mw_status conv1d_tensor_input_cotangent(mw_net* n, const void* const* params, co
                                         const void* target, void* g0, double* loss_out, void* ws,
                                         cudaStream_t s) {
   const Layout& lay = n->mwl;
-  C1 c = make_c1(n, lay, ws, s);
+  C1 c = make_c1(n, lay, ws, s, params, x);
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
   MW_TRY(forward_pass(c, params, x, false));          // Phase I (+ per-step preparation)
   MW_TRY(loss_top(c, target, loss_out));
@@ -454,12 +488,12 @@ mw_status conv1d_tensor_input_cotangent(mw_net* n, const void* const* params, co
 
 mw_status conv1d_tensor_forward_sweep(mw_net* n, const void* const* params, const void* x,
                                       const void* g0, void* const* dW, void* ws, cudaStream_t s) {
-  (void)params; (void)x;   // the term planes of x (xp[0]) are still those Phase I made
+  // the term planes of an fp32 x (xp[0]) are still those Phase I made
   const Layout& lay = n->mwl;
-  C1 c = make_c1(n, lay, ws, s);
+  C1 c = make_c1(n, lay, ws, s, params, x);
   const int L = c.L, C = c.C, blk = c.blk, k = c.k;
   const int64_t rows = c.P / C;                       // samples * N
-  MW_TRY(split_planes((const float*)g0, c.P, c.at<__nv_bfloat16>(lay.hp[0]), 3, c.P, s));
+  MW_TRY(split_planes((const float*)g0, c.P, c.at<__nv_bfloat16>(lay.hp[0]), c.pg, c.P, s));
   __nv_bfloat16* gzp = c.at<__nv_bfloat16>(lay.cg[0]);
   float* cst = c.at<float>(lay.chpf);
   for (int l = 0; l < L; ++l) {
@@ -478,16 +512,16 @@ mw_status conv1d_tensor_forward_sweep(mw_net* n, const void* const* params, cons
       e.write_mask = 0;
       e.act = ld.act;
       e.slope = (float)ld.slope;
-      e.planes = x_planes(c, l + 1); e.n_planes = 3; e.plane_stride = c.P;
-      TcGemm p = forward_product(c, xin, c.at<__nv_bfloat16>(lay.cw[l]), e);
+      e.planes = x_planes(c, l + 1); e.n_planes = c.px; e.plane_stride = c.P;
+      TcGemm p = forward_product(c, xin, w_planes(c, l), e);
       MW_TRY(tc_gemm_group(c.cache, &p, 1, c.st, s));
     }
     if (dW[l] || want_h) {
       {
         // c = h W0^-T at every position
         TcGemm p;
-        p.A = pixel_operand(hin, rows, 3, c.P, false, C);
-        p.B.base = c.at<__nv_bfloat16>(lay.cwinv[l]); p.B.rows = C; p.B.cols = C; p.B.planes = 3;
+        p.A = pixel_operand(hin, rows, c.pg, c.P, false, C);
+        p.B.base = c.at<__nv_bfloat16>(lay.cwinv[l]); p.B.rows = C; p.B.cols = C; p.B.planes = c.pg;
         p.B.plane_stride = (int64_t)C * C; p.B.mn_major = false;
         p.M = (int)rows; p.N = C; p.K = C;
         p.epi.mode = TC_EPI_PLAIN;
@@ -497,7 +531,7 @@ mw_status conv1d_tensor_forward_sweep(mw_net* n, const void* const* params, cons
       {
         const int64_t total8 = frag_elems(c) / 8;
         frag_scatter_kernel<<<(unsigned)((total8 + 255) / 256), 256, 0, s>>>(
-            c.at<float>(lay.cfrag[l]), C, blk, k - 1, total8, gzp, 3, c.P);
+            c.at<float>(lay.cfrag[l]), C, blk, k - 1, total8, gzp, c.pg, c.P);
         MW_TRY(launch_ok());
       }
       // position t of every block from positions t-2, t-1 (adjacent in memory: K = 2 C)
@@ -505,26 +539,26 @@ mw_status conv1d_tensor_forward_sweep(mw_net* n, const void* const* params, cons
         TcGemm p;
         p.A.base = gzp + (int64_t)(t - (k - 1)) * C;
         p.A.rows = (int)(rows / blk); p.A.cols = (k - 1) * C; p.A.ld = (int64_t)blk * C;
-        p.A.planes = 3; p.A.plane_stride = c.P; p.A.mn_major = false;
-        p.B.base = c.at<__nv_bfloat16>(lay.cwhat[l]); p.B.rows = C; p.B.cols = (k - 1) * C; p.B.planes = 3;
+        p.A.planes = c.pg; p.A.plane_stride = c.P; p.A.mn_major = false;
+        p.B.base = c.at<__nv_bfloat16>(lay.cwhat[l]); p.B.rows = C; p.B.cols = (k - 1) * C; p.B.planes = c.pg;
         p.B.plane_stride = (int64_t)C * (k - 1) * C; p.B.mn_major = false;
         p.M = (int)(rows / blk); p.N = C; p.K = (k - 1) * C;
         TcEpilogue& e = p.epi;
         e.mode = TC_EPI_PLAIN;
         e.alpha = -1.f;
         e.addend = cst + (int64_t)(t - 1) * C;
-        e.planes = gzp + (int64_t)t * C; e.n_planes = 3; e.plane_stride = c.P;
+        e.planes = gzp + (int64_t)t * C; e.n_planes = c.pg; e.plane_stride = c.P;
         e.ld = (int64_t)blk * C;
         MW_TRY(tc_gemm_group(c.cache, &p, 1, c.st, s));
       }
       if (want_h) {
         planes_leaky_vijp_kernel<<<(unsigned)((c.P / 8 + 255) / 256), 256, 0, s>>>(
-            gzp, 3, c.P, words, ld.act, (float)ld.slope, c.P / 8, hout, 3, c.P);
+            gzp, c.pg, c.P, words, ld.act, (float)ld.slope, c.P / 8, hout, c.pg, c.P);
         MW_TRY(launch_ok());
       }
     }
     if (reseed_next)
-      MW_TRY(split_planes(c.at<float>(lay.reseed[l + 1]), c.P, hout, 3, c.P, s));
+      MW_TRY(split_planes(c.at<float>(lay.reseed[l + 1]), c.P, hout, c.pg, c.P, s));
     if (dW[l]) {
       MW_TRY(wgrad(c, xin, gzp, c.P, (float*)dW[l], l));
       if (n->apply_params)   // the zeros of tap 0 are structure, not parameters
@@ -538,7 +572,7 @@ mw_status conv1d_tensor_backprop(mw_net* n, const void* const* params, const voi
                                  const void* target, void* const* dW, double* loss_out, void* ws,
                                  cudaStream_t s) {
   const Layout& lay = n->bpl;
-  C1 c = make_c1(n, lay, ws, s);
+  C1 c = make_c1(n, lay, ws, s, params, x);
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
   MW_TRY(forward_pass(c, params, x, true));
   MW_TRY(loss_top(c, target, loss_out));

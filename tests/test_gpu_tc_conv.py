@@ -211,6 +211,17 @@ def test_fragmental_cnn1d_fp32_tensor_path(depth, C, N, batch, block, K):
     assert mw_res >= frag_bytes
 
 
+@pytest.mark.parametrize("depth,C,N,batch,block,K", [(3, 64, 128, 2, 4, 0), (4, 256, 256, 2, 16, 2),
+                                                     (5, 128, 128, 4, 8, 4)])
+def test_fragmental_cnn1d_bf16_tensor_path(depth, C, N, batch, block, K):
+    """bf16 inputs and weights, fp32 accumulation, two-term cotangents; bar 2e-2."""
+    from paper_2402_14212_b200 import synth as S
+    from parity_util import check_problem
+    p = S.fragmental_cnn1d(seed=depth, depth=depth, C=C, N=N, batch=batch, block=block, reseed_every=K,
+                           prec=S.BF16)
+    check_problem(p, 2e-2, backend="tensor", exact_masks=False, tau=2e-2)
+
+
 def test_fragmental_cnn1d_rejects_a_full_tap0():
     from paper_2402_14212_b200 import synth as S
     p = S.fragmental_cnn1d(seed=1, depth=2, C=64, N=128, batch=2, block=4, reseed_every=0, prec=S.F32)
