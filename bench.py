@@ -8,6 +8,13 @@ fp32, MSE), synthetic seeded data.  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
 
+Workloads: deep_mlp (default, config 2), deep_mlp_small, mixed_mlp (config 4), sweep_mlp --depth D
+(config 5), submersive_cnn (config 3), tiny_mlp (config 1); the paper's own convolutional experiments
+strided_cnn [--depth D] (stride-2 submersive layers) and fragmental_cnn1d [--depth D --frag-block B]
+(1-D, fragmental checkpoints), their bf16 forms strided_cnn_bf16 / fragmental_cnn1d_bf16, and
+strided_cnn_small.  --with-backprop adds the time of the library's own Backprop; --depth-sweep and
+--memory-table print the memory studies instead of the benchmark line.
+
 N > 1 (under torchrun): independent replicas of the same step on every GPU, no data-path
 collective ("replicas only"); NCCL is used only for the barrier and the max over ranks.
 --impl reference times the CPU oracle (fp64, numpy) on the host cores instead.
