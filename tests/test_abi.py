@@ -96,6 +96,20 @@ def test_net_create_convolution_families():
     assert L.mw_forward_sweep_apply(dense._h, arr4, 1, 1, 0.1, arr4, 256, 1 << 30, None) == 2
 
 
+def test_nets_can_be_created_and_destroyed_repeatedly():
+    # host objects only (descriptions, layouts, tensor-map caches): no device memory is involved
+    probs = [S.deep_mlp(depth=4, n=128, batch=64), S.mixed_mlp(depth=4, n=128, batch=64),
+             S.strided_cnn(depth=2, C=64, H=16, W=16, batch=16), S.fragmental_cnn1d(depth=2, C=64, N=128, batch=2)]
+    sizes = []
+    for _ in range(50):
+        for p in probs:
+            net = mwb.net_for(p, backend="tensor")
+            sizes.append(net.workspace_bytes()[0])
+            net.close()
+            net.close()                      # closing twice is harmless
+    assert sizes[:4] == sizes[-4:]
+
+
 def test_workspace_sizes_and_residual_accounting():
     p = S.deep_mlp(depth=8, n=128, batch=64, reseed_every=4)
     net = mwb.net_for(p, backend="simt")
