@@ -290,3 +290,35 @@ def test_cnn_sweep_skips_layers_without_an_output(family):
     net.forward_sweep(params, x, g0, ws, dW_out=some)
     assert net.last_device_status(ws)[0] == 0
     assert torch.equal(some[1], full[1]) and torch.equal(some[3], full[3])
+
+
+@pytest.mark.parametrize("family", ["strided", "conv1d"])
+def test_cnn_calls_can_be_repeated(family):
+    """The sweep may be run again on the same workspace, and a whole step again after it, with the
+    same results bit for bit (nothing a call needs is consumed by it)."""
+    import torch
+    from paper_2402_14212_b200 import synth as S
+    if family == "strided":
+        p = S.strided_cnn(seed=8, depth=3, C=64, H=32, W=32, batch=4, gamma=0.5, reseed_every=2, prec=S.F32)
+    else:
+        p = S.fragmental_cnn1d(seed=8, depth=3, C=64, N=128, batch=4, block=4, reseed_every=2, prec=S.F32)
+    net = mwb.net_for(p, backend="tensor")
+    params, x, target = mwb.to_device(p)
+    ws = net.alloc_workspace("moonwalk")
+    g0 = net.input_cotangent(params, x, target, ws)
+    first = [d.clone() for d in net.forward_sweep(params, x, g0, ws)]
+    again = net.forward_sweep(params, x, g0, ws)
+    for a, b in zip(first, again):
+        assert torch.equal(a, b)
+    g0b = net.input_cotangent(params, x, target, ws)
+    third = net.forward_sweep(params, x, g0b, ws)
+    assert torch.equal(g0, g0b)
+    for a, b in zip(first, third):
+        assert torch.equal(a, b)
+    # a sweep on a workspace that backprop has overwritten is refused
+    wsb = net.alloc_workspace("both")
+    g0c = net.input_cotangent(params, x, target, wsb)
+    net.backprop_reference(params, x, target, wsb)
+    with pytest.raises(mwb.MwError) as e:
+        net.forward_sweep(params, x, g0c, wsb)
+    assert e.value.code == mwb.STATUS_NAMES.index("MW_ERR_STATE")
