@@ -360,8 +360,11 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
       float h[32];
       if (e.act == MW_ACT_LEAKY_RELU) {
         const uint32_t word = e.mask[woff];
+        // one division per chunk: the inverse derivative is applied as a product with the
+        // correctly rounded reciprocal of the slope (within an ulp of the quotient)
+        const float rs = 1.f / e.slope;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) h[i] = ((word >> i) & 1u) ? v[i] : v[i] / e.slope;
+        for (int i = 0; i < 32; ++i) h[i] = ((word >> i) & 1u) ? v[i] : v[i] * rs;
       } else if (e.act == MW_ACT_RELU) {
         // live units pass g_z on (phi' = 1); dead units take their stored cotangent back and
         // contribute nothing to the weight vjp
