@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (read + written) per launch of the product kernel, averaged over the launches of this
 # benchmark's default workload (670 captured launches; profiles/tc_group_kernel_traffic_deep_mlp.md).
 # Other workloads have no capture: their `traffic` is null.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"deep_mlp": 115.7e6}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"deep_mlp": 115.4e6}
 
 
 def workload(name: str, seed: int = 0, depth: int = 0, block: int = 0):
