@@ -90,7 +90,7 @@ typedef struct {
   int32_t resident_inverse;/* 1: mw_input_cotangent computes every layer's W^-1 (and split
                               operands) once and keeps them in the workspace; 0: the sweep
                               builds them layer by layer in a transient slot (lean memory) */
-  int32_t reserved;        /* 0; 1 = run the forward sweep as a single launch (experimental)     */
+  int32_t reserved;        /* must be 0                                                      */
   int32_t frag_block;      /* MW_CONV1D nets: Phase II keeps the output cotangent of every
                               convolution at the first k - 1 positions of each block of this
                               many positions (2..64, dividing W); Phase III rebuilds the rest  */
@@ -291,6 +291,14 @@ int64_t mw_launch_count(void);
  * thread-safe; meant for benchmarks (the paper has no counterpart). */
 void mw_profile_begin(void);
 mw_status mw_profile_end(double* total_ms, int64_t* launches, double* flops, double* mma_flops);
+
+/* The tensor-core product kernel has two forms: one CTA per 128-row tile, and a pair of CTAs (a
+ * cluster of two SMs, tcgen05 cta_group::2) per 256-row tile that stage half of the B tile each.
+ * Launches whose products all qualify (operands of at most two bf16 terms, M a multiple of 256,
+ * N of 128) use the pair form.  enable = 0 turns it off for the launches that follow, 1 (the
+ * default) turns it back on; returns the previous setting.  Process-wide; for comparisons and
+ * tests (the paper has no counterpart). */
+int32_t mw_set_pair_mode(int32_t enable);
 
 #ifdef __cplusplus
 }

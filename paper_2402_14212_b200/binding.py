@@ -83,6 +83,8 @@ def lib() -> C.CDLL:
                                             C.POINTER(vp), vp, vp, vp, sz, vp]
         L.mw_launch_count.argtypes = []
         L.mw_launch_count.restype = C.c_int64
+        L.mw_set_pair_mode.argtypes = [i32]
+        L.mw_set_pair_mode.restype = i32
         L.mw_profile_begin.argtypes = []
         L.mw_profile_begin.restype = None
         L.mw_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64),
@@ -258,6 +260,11 @@ class Net:
 
 def launch_count() -> int:
     return int(lib().mw_launch_count())
+
+
+def set_pair_mode(enable: bool) -> bool:
+    """Turn the CTA-pair form of the product kernel on or off; returns the previous setting."""
+    return bool(lib().mw_set_pair_mode(int(bool(enable))))
 
 
 def profile_begin():

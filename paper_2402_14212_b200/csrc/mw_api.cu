@@ -32,6 +32,8 @@ struct Bump {
 
 bool valid_layer(const mw_layer_desc& d, int idx, int L) {
   if (d.act < MW_ACT_NONE || d.act > MW_ACT_RELU) return false;
+  // a leaky-ReLU of slope 0 is a ReLU: not submersive, its vijp would divide by zero
+  if (d.act == MW_ACT_LEAKY_RELU && !(d.slope != 0.0 && d.slope - d.slope == 0.0)) return false;
   if (d.kind == MW_DENSE) return d.n_in > 0 && d.n_in == d.n_out;
   if (d.kind == MW_HEAD_LINEAR) return idx == L - 1 && d.n_in > 0 && d.n_out > 0 && d.act == MW_ACT_NONE;
   if (d.kind == MW_CONV1D)
@@ -157,6 +159,7 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
   if (opts->reseed_every < 0 || opts->conv_vijp_iters < 0 || opts->inverse_iters < 0 || opts->frag_block < 0)
     return MW_ERR_INVALID_ARG;
   if (opts->backend < MW_BACKEND_AUTO || opts->backend > MW_BACKEND_TENSOR) return MW_ERR_INVALID_ARG;
+  if (opts->reserved != 0) return MW_ERR_INVALID_ARG;
   for (int l = 0; l < n_layers; ++l) {
     if (layers[l].kind < MW_DENSE || layers[l].kind > MW_CONV1D) return MW_ERR_INVALID_ARG;
     if (!valid_layer(layers[l], l, n_layers)) return MW_ERR_UNSUPPORTED;
@@ -684,6 +687,8 @@ extern "C" mw_status mw_gradient_step_host(mw_net* net, const void* const* param
 }
 
 extern "C" int64_t mw_launch_count(void) { return (int64_t)g_launch_count; }
+
+extern "C" int32_t mw_set_pair_mode(int32_t enable) { return tc_set_pair_mode(enable); }
 
 extern "C" void mw_profile_begin(void) { tc_profile_begin(); }
 

@@ -23,6 +23,16 @@
 // the small cross terms have blocks of their own.
 // Every wait is bounded; on expiry the kernel records MW_ERR_TIMEOUT and unwinds (tensor memory
 // is always released).
+//
+// Pair form (kPair): two CTAs of a cluster (two SMs) own one 256-row tile.  Each stages its own
+// 128 rows of A and HALF of the B tile; one lane of the even CTA issues tcgen05.mma.cta_group::2,
+// which reads both halves of B from the two shared memories and writes each CTA's 128 rows of the
+// accumulator into that CTA's tensor memory.  B then crosses the L2-to-SM path once per 256 rows
+// instead of once per 128.  Copies of both CTAs complete on the even CTA's barrier (plain
+// cp.async.bulk.tensor with .cta_group::2; nothing is multicast), the commits that free a stage or
+// publish an accumulator set arrive at both CTAs, and the odd CTA's epilogue warps hand the set
+// back with a remote arrive.  Operands of at most two terms; every cross product is its own
+// instruction of the tile's width (a stacked instruction would interleave the halves of the planes).
 #include <cudaTypedefs.h>
 
 #include <algorithm>
@@ -40,7 +50,7 @@ constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int kThreadsTc = 192;
 constexpr int kEpiWarps = 4;     // one per tensor-memory lane quarter
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far above any legitimate wait
+constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;   // 2 s: far above any legitimate wait
 constexpr int kMaxStages = 8;
 constexpr int kMaxOps = 6;
 constexpr uint32_t kATileBytes = BM * BK * 2;  // one A term plane of one stage
@@ -61,8 +71,9 @@ struct alignas(64) TcProblem {
   TcEpilogue epi;
   int M, N, K, num_kb, kb_per_split, split;
   int bn, tiles_n, tiles_mn, unit_begin, unit_count;
+  int bm;                      // rows of one tile: 128, or 256 in the pair form
   int pa, pb, a_mn, b_mn, a_batch_planes, b_batch_planes;
-  uint32_t b_tile_bytes, tx_bytes;
+  uint32_t b_tile_bytes, tx_bytes;   // per CTA: in the pair form a CTA stages half of the B tile
   int nops, nblocks;
   float* split_partials;
   unsigned int* split_counters;
@@ -82,6 +93,7 @@ constexpr int kMaxProgram = 768;   // products of one program launch
 struct alignas(64) TcGroupParams {
   int nprob, total_units, stages, pad0;
   uint32_t stage_bytes, pad1;
+  uint64_t wait_limit_ns;     // bound of every device-side wait
   DeviceStatus* st;
   const TcProblem* table;     // program launch: the products live in global memory ...
   unsigned int* done;         // ... and count their finished tiles here (zero at launch)
@@ -106,15 +118,47 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// arrive at a barrier of another CTA of the cluster (`bar` is a shared::cluster address)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// shared::cluster address of this CTA's shared-memory address `addr` inside CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// all threads of all CTAs of the cluster
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// kCluster: the phase may have been completed from another CTA of the cluster
+template <bool kCluster>
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
+  if (kCluster) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+  }
   return ok != 0;
 }
 __device__ __forceinline__ uint64_t global_timer_ns() {
@@ -122,30 +166,35 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+// what every bounded wait of a CTA shares
+struct WaitCtx {
+  DeviceStatus* st;
+  volatile int* abort_flag;
+  uint64_t limit_ns;
+};
 // Bounded wait: try_wait suspends the thread in hardware until the phase completes or its own
 // time slice ends.  The bound is wall time (checked every 256 polls); a wait also gives up when
 // another role of the CTA has already failed.  On expiry the timeout is recorded.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, DeviceStatus* st,
-                                          unsigned who, volatile int* abort_flag) {
+template <bool kCluster>
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& wc, unsigned who) {
   uint64_t t0 = 0;
   for (uint32_t i = 0;; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait<kCluster>(bar, parity)) return true;
     if ((i & 255u) == 255u) {
-      if (*abort_flag) return false;
+      if (*wc.abort_flag) return false;
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) break;
+      else if (now - t0 > wc.limit_ns) break;
     }
   }
-  record_error(st, MW_ERR_TIMEOUT, who, blockIdx.x, 0u, 0u);
-  *abort_flag = 1;
+  record_error(wc.st, MW_ERR_TIMEOUT, who, blockIdx.x, 0u, 0u);
+  *wc.abort_flag = 1;
   return false;
 }
 
 // Bounded wait for a product of the same (co-resident) launch: its tiles count themselves in
 // global memory.  Same bound and failure path as mbar_wait.
-__device__ __forceinline__ bool wait_done(const unsigned int* counter, unsigned int target,
-                                          DeviceStatus* st, volatile int* abort_flag) {
+__device__ __forceinline__ bool wait_done(const unsigned int* counter, unsigned int target, const WaitCtx& wc) {
   uint64_t t0 = 0;
   for (uint32_t i = 0;; ++i) {
     unsigned int v;
@@ -153,24 +202,36 @@ __device__ __forceinline__ bool wait_done(const unsigned int* counter, unsigned 
     if (v >= target) return true;
     __nanosleep(40);
     if ((i & 63u) == 63u) {
-      if (*abort_flag) return false;
+      if (*wc.abort_flag) return false;
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) break;
+      else if (now - t0 > wc.limit_ns) break;
     }
   }
-  record_error(st, MW_ERR_TIMEOUT, 5u, blockIdx.x, target, 0u);
-  *abort_flag = 1;
+  record_error(wc.st, MW_ERR_TIMEOUT, 5u, blockIdx.x, target, 0u);
+  *wc.abort_flag = 1;
   return false;
 }
 
+// Bulk tensor copies into this CTA's shared memory.  kPair: the completion bytes are counted on
+// `bar`, a shared::cluster address that may lie in the other CTA of the pair (.cta_group::2); the
+// data itself always lands in the executing CTA.  No copy is multicast.
+template <bool kPair>
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
                                             int c0, int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
-      "%4, %5}], [%2];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-      : "memory");
+  if (kPair) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
+        "%4, %5}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+  } else {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
+        "%4, %5}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+  }
 }
 
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
@@ -189,20 +250,44 @@ __device__ __forceinline__ uint32_t desc_lo_base(bool mn_major) {
   return (mn_major ? (8192u >> 4) : 1u) << 16;
 }
 
+// kPair: one instruction for both CTAs of the pair (256 rows); the descriptors name the same
+// offsets in both shared memories, the accumulator address the same columns in both tensor memories
+template <bool kPair>
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo,
                                           uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-      "mov.b64 da, {%1, %5};\n\t"
-      "mov.b64 db, {%2, %5};\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(tmem_d),
-      "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
-      : "memory");
+  if (kPair) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(tmem_d),
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(tmem_d),
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+        : "memory");
+  }
 }
+// arrive at `bar` once the products issued so far have retired; kPair: at the barrier at this
+// offset in BOTH CTAs of the pair (the arrival is sent to two CTAs; no data is)
+template <bool kPair>
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-               : "memory");
+  if (kPair) {
+    asm volatile(
+        "{\n\t.reg .b16 m;\n\tmov.b16 m, 3;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n\t}" ::"r"(bar)
+        : "memory");
+  } else {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+  }
 }
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -409,7 +494,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
 // The instructions of one 64-deep K block, as straight-line code: the issuing lane runs alone on
 // its scheduler, so every branch and every dependent integer instruction in this loop costs
 // tens of cycles that the tensor pipe would otherwise spend on the next product.
-template <int NOPS>
+template <int NOPS, bool kPair>
 __device__ __forceinline__ void issue_k_block(const uint32_t (&oa)[kMaxOps], const uint32_t (&ob)[kMaxOps],
                                               const uint32_t (&oi)[kMaxOps], const uint32_t (&od)[kMaxOps],
                                               const uint32_t (&orot)[kMaxOps], const uint32_t (&ofk)[kMaxOps],
@@ -427,8 +512,8 @@ __device__ __forceinline__ void issue_k_block(const uint32_t (&oa)[kMaxOps], con
   for (int k4 = 0; k4 < BK / 16; ++k4) {
 #pragma unroll
     for (int o = 0; o < NOPS; ++o)
-      umma_bf16(d[o], a[o] + (uint32_t)k4 * a_kadv, b[o] + (uint32_t)k4 * b_kadv, oi[o],
-                k4 == 0 ? first[o] : 1u);
+      umma_bf16<kPair>(d[o], a[o] + (uint32_t)k4 * a_kadv, b[o] + (uint32_t)k4 * b_kadv, oi[o],
+                       k4 == 0 ? first[o] : 1u);
   }
 }
 
@@ -447,21 +532,22 @@ __device__ __forceinline__ void decode_unit(const TcProblem* probs, const int* u
   w.tl = tl;
   w.ks = ks;
   w.z = z;
-  w.m0 = mt * BM;
+  w.m0 = mt * P.bm;
   w.n0 = (r - mt * P.tiles_n) * P.bn;
   w.kb0 = ks * P.kb_per_split;
   const int e = w.kb0 + P.kb_per_split;
   w.kb1 = e < P.num_kb ? e : P.num_kb;
 }
 
-// Units of this CTA: round r takes index r*G + c (even r) or r*G + G-1-c (odd r); a program
-// launch takes r*G + c throughout, so that one CTA never holds two units of one short product
-// (they would run one after the other and hold up everything that waits for that product).
+// Units of this CTA (pair form: of this pair of CTAs): round r takes index r*G + c (even r) or
+// r*G + G-1-c (odd r); a program launch takes r*G + c throughout, so that one CTA never holds two
+// units of one short product (they would run one after the other and hold up everything that
+// waits for that product).
 // (Handing units out dynamically in list order was tried and is slower: CTAs pile up behind the
 // one product that is not complete yet.)
-template <bool kProgram>
+template <bool kProgram, bool kPair>
 __device__ __forceinline__ int next_unit(const TcGroupParams& p, int& r) {
-  const int G = (int)gridDim.x, c = (int)blockIdx.x;
+  const int G = (int)(gridDim.x >> (kPair ? 1 : 0)), c = (int)(blockIdx.x >> (kPair ? 1 : 0));
   while (r * G < p.total_units) {
     const int u = r * G + (((r & 1) && !kProgram) ? G - 1 - c : c);
     ++r;
@@ -471,8 +557,9 @@ __device__ __forceinline__ int next_unit(const TcGroupParams& p, int& r) {
 }
 
 // kProgram: the products live in global memory and wait for one another (program launch);
-// otherwise they are read straight from the kernel parameters
-template <bool kProgram>
+// otherwise they are read straight from the kernel parameters.
+// kPair: launched as clusters of two CTAs that share every tile (see the top of the file).
+template <bool kProgram, bool kPair>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 tc_group_kernel(const __grid_constant__ TcGroupParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -486,6 +573,8 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  // pair form: rank 0 (the even CTA) issues the products and owns the barriers both CTAs report to
+  const uint32_t rank = kPair ? cluster_cta_rank() : 0u;
   const uint32_t tiles = (smem_u32(smem_raw) + 1023u) & ~1023u;  // 1024-byte aligned for the swizzle
   // Launched with programmatic stream serialisation, this grid may start while the previous
   // kernel of the stream is still finishing: everything up to the waits below (barriers, tensor
@@ -502,7 +591,8 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&acc_full[s]), 1);
-      mbar_init(smem_u32(&acc_empty[s]), kEpiWarps);   // one arrival per epilogue warp
+      // one arrival per epilogue warp (of both CTAs in the pair form)
+      mbar_init(smem_u32(&acc_empty[s]), kEpiWarps * (kPair ? 2 : 1));
     }
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -515,17 +605,32 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     smem_u32(&tmem_slot)),
-                 "r"((uint32_t)kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    // pair form: the same warp of both CTAs allocates, and both get the same columns
+    if (kPair) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                       smem_u32(&tmem_slot)),
+                   "r"((uint32_t)kTmemCols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                       smem_u32(&tmem_slot)),
+                   "r"((uint32_t)kTmemCols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  // pair form: no copy may complete on, and no warp may arrive at, a barrier of the other CTA
+  // before that CTA has initialised it
+  if (kPair) cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot;
-  volatile int* abortp = &abort_flag;
+  WaitCtx wc;
+  wc.st = p.st;
+  wc.abort_flag = &abort_flag;
+  wc.limit_ns = p.wait_limit_ns;
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -537,23 +642,27 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       if (!kProgram) asm volatile("griddepcontrol.wait;" ::: "memory");
       for (;;) {
         if (!ok) break;
-        const int u = next_unit<kProgram>(p, rr);
+        const int u = next_unit<kProgram, kPair>(p, rr);
         if (u < 0) break;
         Unit w;
         decode_unit(probs, ub, nprob, u, q, w);
         const TcProblem& P = probs[w.q];
         if (kProgram && P.ndep) {
           // program launch: the operands are written by earlier products of this same launch
-          for (int i = 0; i < P.ndep && ok; ++i)
-            ok = wait_done(p.done + P.dep[i], P.dep_target[i], p.st, abortp);
+          for (int i = 0; i < P.ndep && ok; ++i) ok = wait_done(p.done + P.dep[i], P.dep_target[i], wc);
           if (!ok) break;
           asm volatile("fence.proxy.async;" ::: "memory");   // their stores, then our bulk copies
         }
         const int a_pl0 = w.z * P.a_batch_planes, b_pl0 = w.z * P.b_batch_planes;
-        const int pa = P.pa, pb = P.pb, nbox = P.bn >> 6;
+        const int pa = P.pa, pb = P.pb;
         const bool a_mn = P.a_mn != 0, b_mn = P.b_mn != 0;
         const uint32_t b_tile_bytes = P.b_tile_bytes, tx = P.tx_bytes;
-        const int conv = P.conv_mode;
+        // this CTA's rows of A and columns of B (pair form: its half of the tile)
+        const int am0 = w.m0 + (kPair ? (int)rank * BM : 0);
+        const int bcols = kPair ? (P.bn >> 1) : P.bn;
+        const int bn_first = w.n0 + (kPair ? (int)rank * bcols : 0);
+        const int nbox = bcols >> 6;
+        const int conv = kPair ? (int)TC_CONV_NONE : P.conv_mode;
         // convolution: image, row and column of the first pixel of the unit's tile
         int cb = 0, cy0 = 0, cx0 = 0;
         if (conv == TC_CONV_PIXELS) {
@@ -591,12 +700,18 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           wg_x = rem - wg_y * P.cWo;
         }
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
-          if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, p.st, 1u, abortp)) { ok = false; break; }
-          const uint32_t fb = smem_u32(&full_bar[stage]);
-          mbar_expect_tx(fb, tx);
+          if (!mbar_wait<kPair>(smem_u32(&empty_bar[stage]), phase ^ 1u, wc, 1u)) { ok = false; break; }
+          // the bytes of both CTAs are counted on the even CTA's barrier, which expects them all
+          uint32_t fb = smem_u32(&full_bar[stage]);
+          if (kPair) {
+            if (rank == 0) mbar_expect_tx(fb, 2u * tx);
+            fb = map_to_cta(fb, 0u);
+          } else {
+            mbar_expect_tx(fb, tx);
+          }
           const uint32_t sbase = tiles + stage * p.stage_bytes;
           int k0 = kb * BK;
-          int bk0 = k0, bn0 = w.n0;       // B coordinates (K, N)
+          int bk0 = k0, bn0 = bn_first;       // B coordinates (K, N)
           if (conv == TC_CONV_PIXELS) {
             const int t = px_t, cblk = px_c;
             if (++px_c == P.ccb) { px_c = 0; ++px_t; }
@@ -627,10 +742,10 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           for (int pl = 0; pl < pa; ++pl) {
             const uint32_t dst = sbase + (uint32_t)pl * kATileBytes;
             if (a_mn) {
-              tma_load_3d(dst, &P.tmA, fb, w.m0, k0, a_pl0 + pl);
-              tma_load_3d(dst + 8192u, &P.tmA, fb, w.m0 + 64, k0, a_pl0 + pl);
+              tma_load_3d<kPair>(dst, &P.tmA, fb, am0, k0, a_pl0 + pl);
+              tma_load_3d<kPair>(dst + 8192u, &P.tmA, fb, am0 + 64, k0, a_pl0 + pl);
             } else {
-              tma_load_3d(dst, &P.tmA, fb, k0, w.m0, a_pl0 + pl);
+              tma_load_3d<kPair>(dst, &P.tmA, fb, k0, am0, a_pl0 + pl);
             }
           }
           const uint32_t bbase = sbase + (uint32_t)pa * kATileBytes;
@@ -639,9 +754,9 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
             const uint32_t dst = bbase + (uint32_t)pl * b_tile_bytes;
             if (b_mn) {
               for (int h = 0; h < nbox; ++h)
-                tma_load_3d(dst + (uint32_t)h * 8192u, &P.tmB, fb, bn0 + h * 64, bk0, bz + pl);
+                tma_load_3d<kPair>(dst + (uint32_t)h * 8192u, &P.tmB, fb, bn0 + h * 64, bk0, bz + pl);
             } else {
-              tma_load_3d(dst, &P.tmB, fb, bk0, bn0, bz + pl);
+              tma_load_3d<kPair>(dst, &P.tmB, fb, bk0, bn0, bz + pl);
             }
           }
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
@@ -649,20 +764,20 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    // ---------------- MMA issuer (pair form: of the even CTA only) ----------------
+    if (lane == 0 && rank == 0) {
       uint32_t stage = 0, phase = 0;
       int j = 0, q = 0, rr = 0;
       bool ok = true;
       for (;;) {
         if (!ok) break;
-        const int u = next_unit<kProgram>(p, rr);
+        const int u = next_unit<kProgram, kPair>(p, rr);
         if (u < 0) break;
         Unit w;
         decode_unit(probs, ub, nprob, u, q, w);
         const TcProblem& P = probs[w.q];
         const uint32_t set = (uint32_t)j & 1u, aphase = ((uint32_t)j >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&acc_empty[set]), aphase ^ 1u, p.st, 2u, abortp)) { ok = false; break; }
+        if (!mbar_wait<kPair>(smem_u32(&acc_empty[set]), aphase ^ 1u, wc, 2u)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_set = tmem_base + set * (uint32_t)kSetCols;
         // the unit's instruction list, in registers
@@ -683,22 +798,22 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         const uint32_t b_kadv = P.b_mn ? (2048u >> 4) : (32u >> 4);
         const int nkb = w.kb1 - w.kb0;
         for (int kbl = 0; kbl < nkb; ++kbl) {
-          if (!mbar_wait(smem_u32(&full_bar[stage]), phase, p.st, 3u, abortp)) { ok = false; break; }
+          if (!mbar_wait<kPair>(smem_u32(&full_bar[stage]), phase, wc, 3u)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sb16 = (tiles + stage * p.stage_bytes) >> 4;
           switch (nops) {
-            case 1: issue_k_block<1>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            case 2: issue_k_block<2>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            case 3: issue_k_block<3>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            case 4: issue_k_block<4>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            case 5: issue_k_block<5>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            default: issue_k_block<6>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            case 1: issue_k_block<1, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            case 2: issue_k_block<2, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            case 3: issue_k_block<3, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            case 4: issue_k_block<4, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            case 5: issue_k_block<5, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
+            default: issue_k_block<6, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
           }
-          umma_commit(smem_u32(&empty_bar[stage]));  // frees the stage once these products retire
+          umma_commit<kPair>(smem_u32(&empty_bar[stage]));  // frees the stage once these products retire
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit(smem_u32(&acc_full[set]));
+        umma_commit<kPair>(smem_u32(&acc_full[set]));
         ++j;
       }
     }
@@ -713,7 +828,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     if (!kProgram) asm volatile("griddepcontrol.wait;" ::: "memory");
     for (;;) {
       if (!ok) break;
-      const int u = next_unit<kProgram>(p, rr);
+      const int u = next_unit<kProgram, kPair>(p, rr);
       if (u < 0) break;
       Unit w;
       decode_unit(probs, ub, nprob, u, q, w);
@@ -721,10 +836,11 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       const uint32_t set = (uint32_t)j & 1u, aphase = ((uint32_t)j >> 1) & 1u;
       // every lane observes the barrier itself; the warp then takes one common decision so the
       // warp-wide tensor-memory loads below are never executed by part of a warp
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&acc_full[set]), aphase, p.st, 4u, abortp));
+      ok = __all_sync(0xffffffffu, mbar_wait<kPair>(smem_u32(&acc_full[set]), aphase, wc, 4u));
       if (!ok) break;
       tc_fence_after();
-      const int row = w.m0 + quarter * 32 + lane;
+      // pair form: this CTA's tensor memory holds rows rank*128 .. rank*128+127 of the tile
+      const int row = w.m0 + (kPair ? (int)rank * BM : 0) + quarter * 32 + lane;
       const int bn = P.bn, nblk = P.nblocks, N = P.N;
       TcEpilogue epi = P.epi;           // this batch item's view of the outputs
       int orow = row;                   // where the row's outputs live
@@ -746,7 +862,6 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       }
       double sumsq_local = 0.0;
       const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + set * (uint32_t)kSetCols;
-      const int nchunk = bn >> 5;
       // sum of the column blocks of 32 accumulator columns starting at c
       auto load_chunk = [&](int c, float (&v)[32]) {
         uint32_t r0[32];
@@ -762,7 +877,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         }
       };
       bool fused_step = true;
-      if (P.split > 1) {
+      if (!kPair && P.split > 1) {
         // K split: leave this piece of the tile in the meeting place, element (row, c + i) of
         // piece s at ((s * nchunk + c / 32) * 32 + i) * 128 + row so that a warp writes whole lines
         float* mine = P.split_partials + ((int64_t)w.tl * P.split + w.ks) * (int64_t)(BM * bn) +
@@ -791,14 +906,15 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         }
       }
       if (fused_step) {
-        const float* others = P.split > 1 ? P.split_partials + (int64_t)w.tl * P.split * (int64_t)(BM * bn) +
-                                                quarter * 32 + lane
-                                          : nullptr;
+        const bool split = !kPair && P.split > 1;
+        const float* others = split ? P.split_partials + (int64_t)w.tl * P.split * (int64_t)(BM * bn) +
+                                          quarter * 32 + lane
+                                    : nullptr;
 #pragma unroll 1
         for (int c = half * 32; c < bn; c += 32 * (kEpiWarps / 4)) {
           if (w.n0 + c >= N) break;
           float v[32];
-          if (P.split > 1) {
+          if (split) {
             float own[32];
             load_chunk(c, own);
 #pragma unroll
@@ -831,35 +947,47 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           if (row < P.M) epilogue_chunk(epi, N, row, orow, w.n0 + c, v, sumsq_local);
         }
       }
-      (void)nchunk;
       // this warp has read its part of the accumulator set: hand it back to the MMA issuer
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&acc_empty[set]));
+      if (lane == 0) {
+        if (kPair && rank != 0) mbar_arrive_cluster(map_to_cta(smem_u32(&acc_empty[set]), 0u));
+        else mbar_arrive(smem_u32(&acc_empty[set]));
+      }
       ++j;
+      if (epi.mode == TC_EPI_RESID && epi.sumsq && fused_step) {
+        // this warp's share of ||v||_F^2 goes to a slot of its own (fixed-order sum by the reader)
+        for (int o = 16; o; o >>= 1) sumsq_local += __shfl_xor_sync(0xffffffffu, sumsq_local, o);
+        if (lane == 0)
+          epi.sumsq[((int64_t)(row >> 7) * P.tiles_n + w.n0 / bn) * kEpiWarps + quarter] = sumsq_local;
+      }
       if (kProgram && fused_step) {
         // program launch: publish this warp's part of the tile to the products that wait for it
         __threadfence();
         __syncwarp();
         if (lane == 0) atomicAdd(p.done + w.q, 1u);
       }
-      if (epi.mode == TC_EPI_RESID && epi.sumsq) {
-        for (int o = 16; o; o >>= 1) sumsq_local += __shfl_xor_sync(0xffffffffu, sumsq_local, o);
-        if (lane == 0 && sumsq_local != 0.0) atomicAdd(epi.sumsq, sumsq_local);
-      }
     }
   }
   tc_fence_before();
   __syncthreads();
-  tc_fence_after();
   if (warp == 0 && lane == 0 && abort_flag) {
     // a wait ran out: give copies still in flight a bounded time to land before the CTA retires
     for (int s = 0; s < p.stages; ++s)
-      for (uint32_t i = 0; i < 4096u && !mbar_try_wait(smem_u32(&full_bar[s]), 0u); ++i) __nanosleep(256);
+      for (uint32_t i = 0; i < 4096u && !mbar_try_wait<kPair>(smem_u32(&full_bar[s]), 0u); ++i) __nanosleep(256);
   }
+  // pair form: neither CTA may retire (or give up its tensor memory) while the other may still
+  // arrive at its barriers or have products running on both tensor memories; every role of both
+  // CTAs gets here through bounded waits
+  if (kPair) cluster_sync_all();
+  tc_fence_after();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
-                 : "memory");
+    if (kPair)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
+                   : "memory");
   }
 }
 
@@ -880,15 +1008,23 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
+constexpr int kMaxDevices = 64;
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+  return dev;
+}
+
+// SMs of the current device (cached per device)
 int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
+  static int n[kMaxDevices] = {};
+  const int dev = current_device();
+  if (n[dev] == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    n[dev] = v;
   }
-  return n;
+  return n[dev];
 }
 
 // tile width: as wide as the accumulator set allows for the number of term orders.  Narrower
@@ -900,6 +1036,19 @@ int pick_bn(int pa, int pb, int M, int N, int batch, bool wide = false) {
   int bn = t == 1 ? 256 : (t == 2 ? 128 : 64);
   while (bn > 64 && N % bn != 0) bn >>= 1;
   return bn;
+}
+
+// 0: never use the pair form, 1: wherever a launch qualifies (default)
+int g_pair_mode = 1;
+
+// Can this product run in the pair form?  Operands of at most two terms (the accumulator blocks
+// of a 128-column tile then fit one set), tiles at least 128 columns wide (each CTA stages whole
+// 64-column boxes of its half), whole 256-row tiles, no convolution window, no K split.
+bool pair_capable(const TcGemm& d) {
+  if (d.conv.mode != TC_CONV_NONE || d.split_k > 1) return false;
+  if (d.A.planes > 2 || d.B.planes > 2) return false;
+  if (d.M % 256 != 0 || d.N % 128 != 0) return false;
+  return pick_bn(d.A.planes, d.B.planes, d.M, d.N, d.batch) >= 128;
 }
 
 }  // namespace
@@ -1034,10 +1183,38 @@ static mw_status get_map_conv(TcMapCache* cache, const TcOperand& op, int H, int
 
 namespace {
 
-uint32_t make_idesc(bool a_mn, bool b_mn, int n) {
-  // fp32 accumulate, bf16 A and B, major-ness of A and B, N / 8, M / 16
+uint32_t make_idesc(bool a_mn, bool b_mn, int n, int m = BM) {
+  // fp32 accumulate, bf16 A and B, major-ness of A and B, N / 8, M / 16 (M = 256: both CTAs of a pair)
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// Pair form: one instruction per kept cross product (i, j), 256 rows x bn columns; the products
+// of order i + j accumulate in column block i + j.  Each CTA's stage holds its half of every B
+// plane, b_tile_bytes apart.  Returns the tensor-core cycles of one K block.
+double build_ops_pair(TcProblem& P) {
+  const int pa = P.pa, pb = P.pb, bn = P.bn;
+  const int t = pa > pb ? pa : pb;
+  const uint32_t b0 = (uint32_t)pa * kATileBytes;
+  bool init[4] = {false, false, false, false};
+  int n = 0;
+  double cycles = 0.0;
+  for (int i = 0; i < pa; ++i)
+    for (int j = 0; j < pb; ++j) {
+      if (i + j >= t) continue;
+      TcOp& o = P.ops[n++];
+      o.a_off16 = ((uint32_t)i * kATileBytes) >> 4;
+      o.b_off16 = (b0 + (uint32_t)j * P.b_tile_bytes) >> 4;
+      o.idesc = make_idesc(P.a_mn != 0, P.b_mn != 0, bn, 2 * BM);
+      o.dcol = (uint16_t)((i + j) * bn);
+      o.rot = 0;
+      o.first_kbs = init[i + j] ? 0u : 1u;
+      init[i + j] = true;
+      cycles += 4.0 * (bn / 2.0);
+    }
+  P.nops = n;
+  P.nblocks = t;
+  return cycles;
 }
 
 // the instruction list of one K step: one instruction per A plane covering the B planes whose
@@ -1095,7 +1272,8 @@ double build_ops(TcProblem& P, bool rotate) {
 
 // fills P from d (everything but unit_begin); returns the tensor-core cycles of one unit
 static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P, double* unit_cost,
-                               double* flops, double* mma_flops) {
+                               double* flops, double* mma_flops, bool pair = false) {
+  if (pair && !pair_capable(d)) return MW_ERR_UNSUPPORTED;
   if (d.N % 64 != 0) return MW_ERR_UNSUPPORTED;
   // a ragged K tail is zero-filled by the copies of MN-major operands (K counts their rows)
   if ((!d.A.mn_major || !d.B.mn_major) && d.K % 64 != 0) return MW_ERR_UNSUPPORTED;
@@ -1160,19 +1338,21 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   P.kb_per_split = (P.num_kb + split - 1) / split;
   split = (P.num_kb + P.kb_per_split - 1) / P.kb_per_split;
   P.split = split;
-  const int tiles_m = (d.M + BM - 1) / BM;
+  P.bm = pair ? 2 * BM : BM;
+  const int tiles_m = (d.M + P.bm - 1) / P.bm;
   P.tiles_n = (d.N + P.bn - 1) / P.bn;
   P.tiles_mn = tiles_m * P.tiles_n;
   const int64_t units = (int64_t)P.tiles_mn * d.batch * split;
   if (units > (1 << 30)) return MW_ERR_UNSUPPORTED;
   P.unit_count = (int)units;
-  P.b_tile_bytes = (uint32_t)P.bn * BK * 2;
+  const int b_cols = pair ? P.bn / 2 : P.bn;     // columns of the B tile one CTA stages
+  P.b_tile_bytes = (uint32_t)b_cols * BK * 2;
   P.tx_bytes = (uint32_t)P.pa * kATileBytes + (uint32_t)P.pb * P.b_tile_bytes;
   const int t = P.pa > P.pb ? P.pa : P.pb;
   // fp32-accurate products alternate the leading block (needs two K blocks per unit)
   const bool rotate = t == 3 && P.pa == 3 && P.pb == 3 && P.kb_per_split >= 2 &&
                       (P.num_kb - (split - 1) * P.kb_per_split) >= 2;
-  const double kb_cycles = build_ops(P, rotate);
+  const double kb_cycles = pair ? build_ops_pair(P) : build_ops(P, rotate);
   *unit_cost = kb_cycles * P.kb_per_split;
   P.epi = d.epi;
   P.split_partials = nullptr;
@@ -1194,7 +1374,7 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
     MW_TRY(get_map(cache, d.B, 64, d.B.planes, &P.tmB));
   } else {
     MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA));
-    MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : P.bn, b_total, &P.tmB));
+    MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : b_cols, b_total, &P.tmB));
   }
   int np = 0;
   for (int a = 0; a < P.pa; ++a)
@@ -1211,26 +1391,101 @@ static int stages_for(uint32_t stage_bytes) {
   return stages > kMaxStages ? kMaxStages : stages;
 }
 
+// the opt-in to large dynamic shared memory belongs to the device: once per device and kernel
 static mw_status ensure_kernel_attr() {
-  static bool attr_set = false;
-  if (!attr_set) {
-    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    227 * 1024 - 6144));
-    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    227 * 1024 - 6144));
-    attr_set = true;
+  static bool attr_set[kMaxDevices] = {};
+  const int dev = current_device();
+  if (!attr_set[dev]) {
+    const int bytes = 227 * 1024 - 6144;
+    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    attr_set[dev] = true;
   }
   return MW_OK;
+}
+
+// bound of the device-side waits of the launches that follow (test hook; 0 restores the default)
+static uint64_t g_wait_limit_ns = kDefaultWaitLimitNs;
+
+// CTA pairs that can be resident at once (cached per device); 0 when clusters cannot be launched
+static int max_pairs(size_t smem) {
+  static int n[kMaxDevices] = {};
+  const int dev = current_device();
+  if (n[dev] == 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (unsigned)sm_count());
+    cfg.blockDim = dim3(kThreadsTc);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int c = 0;
+    if (cudaOccupancyMaxActiveClusters(&c, tc_group_kernel<true, true>, &cfg) != cudaSuccess || c < 1) {
+      cudaGetLastError();
+      c = -1;
+    }
+    if (c > sm_count() / 2) c = sm_count() / 2;
+    n[dev] = c;
+  }
+  return n[dev] > 0 ? n[dev] : 0;
+}
+
+// launch of one of the four kernel forms; `coop`: every CTA must be resident (program launches)
+static cudaError_t launch_kernel(bool program, bool pair, int grid, size_t smem, cudaStream_t s,
+                                 const TcGroupParams& prm) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kThreadsTc);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  if (program) {
+    attr[na].id = cudaLaunchAttributeCooperative;
+    attr[na].val.cooperative = 1;
+  } else {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+  }
+  ++na;
+  if (pair) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 2;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  if (program) return pair ? cudaLaunchKernelEx(&cfg, tc_group_kernel<true, true>, prm)
+                           : cudaLaunchKernelEx(&cfg, tc_group_kernel<true, false>, prm);
+  return pair ? cudaLaunchKernelEx(&cfg, tc_group_kernel<false, true>, prm)
+              : cudaLaunchKernelEx(&cfg, tc_group_kernel<false, false>, prm);
 }
 
 mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceStatus* st,
                         cudaStream_t s) {
   if (count < 1 || count > kTcMaxGroup) return MW_ERR_INVALID_ARG;
+  MW_TRY(ensure_kernel_attr());
+  // the pair form when every product of the launch qualifies
+  bool pair = g_pair_mode != 0 && max_pairs(200 * 1024) > 0;
+  for (int i = 0; i < count && pair; ++i) {
+    const TcGemm& d = g[i];
+    if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.batch <= 0) continue;
+    pair = pair_capable(d);
+  }
   static thread_local TcGroupParams prm;
   prm.nprob = 0;
   prm.st = st;
   prm.table = nullptr;
   prm.done = nullptr;
+  prm.wait_limit_ns = g_wait_limit_ns;
   double cost[kTcMaxGroup];
   double flops = 0.0, mma_flops = 0.0;
   uint32_t stage_bytes = 0;
@@ -1238,7 +1493,7 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
     const TcGemm& d = g[i];
     if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.batch <= 0) continue;
     TcProblem& P = prm.prob[prm.nprob];
-    MW_TRY(setup_problem(cache, d, P, &cost[prm.nprob], &flops, &mma_flops));
+    MW_TRY(setup_problem(cache, d, P, &cost[prm.nprob], &flops, &mma_flops, pair));
     if (P.tx_bytes > stage_bytes) stage_bytes = P.tx_bytes;
     ++prm.nprob;
   }
@@ -1260,25 +1515,16 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
   if (stages < 2) return MW_ERR_UNSUPPORTED;
   prm.stages = stages;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  MW_TRY(ensure_kernel_attr());
   const bool prof = g_prof.on;
   if (prof) {
     cudaEventRecord(prof_event(), s);
     g_prof.flops += flops;
     g_prof.mma_flops += mma_flops;
   }
-  const int grid = total < sm_count() ? total : sm_count();
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kThreadsTc);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  const cudaError_t le = cudaLaunchKernelEx(&cfg, tc_group_kernel<false>, prm);
+  // persistent grid: one CTA (or one pair of CTAs) per unit, at most what the device holds at once
+  const int slots = pair ? max_pairs(smem) : sm_count();
+  const int grid = (total < slots ? total : slots) * (pair ? 2 : 1);
+  const cudaError_t le = launch_kernel(false, pair, grid, smem, s, prm);
   ++g_launch_count;
   const mw_status rc = le == cudaSuccess ? MW_OK : MW_ERR_CUDA;
   if (prof) cudaEventRecord(prof_event(), s);
@@ -1294,12 +1540,14 @@ struct TcProgram {
   void* table_dev = nullptr;
   unsigned int* done_dev = nullptr;
   bool uploaded = false;
+  bool pair = false;          // every product in the pair form (clusters of two CTAs)
 };
 
 TcProgram* tc_program_create() { return new TcProgram(); }
 void tc_program_destroy(TcProgram* p) { delete p; }
 
-void tc_program_begin(TcProgram* pr, void* table_dev, unsigned int* done_dev) {
+void tc_program_begin(TcProgram* pr, void* table_dev, unsigned int* done_dev, bool pair) {
+  pr->pair = pair && g_pair_mode != 0 && ensure_kernel_attr() == MW_OK && max_pairs(200 * 1024) > 0;
   pr->table.clear();
   pr->stage_bytes = 0;
   pr->total_units = 0;
@@ -1316,7 +1564,7 @@ int tc_program_add(TcProgram* pr, TcMapCache* cache, const TcGemm& d, const int*
   pr->table.emplace_back();
   TcProblem& P = pr->table.back();
   double cost = 0.0;
-  *status = setup_problem(cache, d, P, &cost, &pr->flops, &pr->mma_flops);
+  *status = setup_problem(cache, d, P, &cost, &pr->flops, &pr->mma_flops, pr->pair);
   if (*status != MW_OK) { pr->table.pop_back(); return -1; }
   P.unit_begin = pr->total_units;
   pr->total_units += P.unit_count;
@@ -1328,7 +1576,8 @@ int tc_program_add(TcProgram* pr, TcMapCache* cache, const TcGemm& d, const int*
     if (q >= self) { *status = MW_ERR_INVALID_ARG; return -1; }   // only earlier products
     const TcProblem& Q = pr->table[q];
     P.dep[P.ndep] = q;
-    P.dep_target[P.ndep] = (unsigned)kEpiWarps * (unsigned)(Q.unit_count / Q.split);
+    // one arrival per epilogue warp and tile (of both CTAs in the pair form)
+    P.dep_target[P.ndep] = (unsigned)kEpiWarps * (pr->pair ? 2u : 1u) * (unsigned)(Q.unit_count / Q.split);
     ++P.ndep;
   }
   return self;
@@ -1352,6 +1601,7 @@ mw_status tc_program_launch(TcProgram* pr, DeviceStatus* st, cudaStream_t s) {
   prm.done = pr->done_dev;
   prm.total_units = pr->total_units;
   prm.stage_bytes = pr->stage_bytes;
+  prm.wait_limit_ns = g_wait_limit_ns;
   const int stages = stages_for(pr->stage_bytes);
   if (stages < 2) return MW_ERR_UNSUPPORTED;
   prm.stages = stages;
@@ -1363,14 +1613,30 @@ mw_status tc_program_launch(TcProgram* pr, DeviceStatus* st, cudaStream_t s) {
     g_prof.flops += pr->flops;
     g_prof.mma_flops += pr->mma_flops;
   }
-  // products wait for one another inside the launch: every CTA must be resident
-  const int grid = pr->total_units < sm_count() ? pr->total_units : sm_count();
-  void* args[] = {(void*)&prm};
-  cudaError_t e = cudaLaunchCooperativeKernel((const void*)tc_group_kernel<true>, dim3(grid), dim3(kThreadsTc),
-                                              args, smem, s);
+  // products wait for one another inside the launch: every CTA must be resident (cooperative launch)
+  const int slots = pr->pair ? max_pairs(smem) : sm_count();
+  if (slots < 1) return MW_ERR_CUDA;
+  const int grid = (pr->total_units < slots ? pr->total_units : slots) * (pr->pair ? 2 : 1);
+  const cudaError_t e = launch_kernel(true, pr->pair, grid, smem, s, prm);
   ++g_launch_count;
   if (prof) cudaEventRecord(prof_event(), s);
   return e == cudaSuccess ? MW_OK : MW_ERR_CUDA;
+}
+
+bool tc_pair_ok(int a_planes, int b_planes, int M, int N) {
+  TcGemm d;
+  d.A.planes = a_planes; d.B.planes = b_planes; d.M = M; d.N = N; d.K = 64;
+  return g_pair_mode != 0 && pair_capable(d);
+}
+int tc_set_pair_mode(int mode) {
+  const int old = g_pair_mode;
+  g_pair_mode = mode != 0;
+  return old;
+}
+void tc_set_wait_limit_ns(uint64_t ns) { g_wait_limit_ns = ns ? ns : kDefaultWaitLimitNs; }
+size_t tc_sumsq_slots(int a_planes, int b_planes, int M, int N) {
+  const int bn = pick_bn(a_planes, b_planes, M, N, 1);
+  return (size_t)((M + BM - 1) / BM) * ((N + bn - 1) / bn) * kEpiWarps;
 }
 
 mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int M, int N, int K,
@@ -1414,7 +1680,7 @@ mw_status split_planes_batched(const float* in, int64_t n, int batch, int64_t in
   if (n % 4 != 0 || plane_stride % 4 != 0 || in_stride % 4 != 0 || out_stride % 4 != 0)
     return MW_ERR_UNSUPPORTED;
   int64_t bx = (n / 4 + 255) / 256;
-  const int64_t cap = (148 * 8 + batch - 1) / batch;
+  const int64_t cap = ((int64_t)sm_count() * 8 + batch - 1) / batch;
   if (bx > cap) bx = cap < 1 ? 1 : cap;
   split_planes_batched_kernel<<<dim3((unsigned)bx, (unsigned)batch), 256, 0, s>>>(
       in, n / 4, in_stride, out, planes, plane_stride, out_stride);

@@ -59,7 +59,9 @@ struct TcEpilogue {
   int write_mask = 0;
   int act = MW_ACT_NONE;
   float slope = 1.f;
-  double* sumsq = nullptr;             // TC_EPI_RESID: atomically accumulated ||v||_F^2
+  // TC_EPI_RESID: ||v||_F^2 in pieces, one slot per 128-row block, column tile and epilogue warp
+  // (tc_sumsq_slots of them; each is written, none accumulated: the reader adds them in order)
+  double* sumsq = nullptr;
   // ReLU fragment stream (Section 5.1 applied to ReLU): row r keeps the cotangent at its dead
   // units from vals[frag_off[r]], in increasing column order; frag_rank[r][c/64] = number of
   // dead units of row r before column 64*(c/64).  TC_EPI_BWD writes the stream, TC_EPI_VIJP
@@ -164,7 +166,8 @@ mw_status tc_gemm(TcMapCache* cache, const TcOperand& A, const TcOperand& B, int
 struct TcProgram;
 TcProgram* tc_program_create();
 void tc_program_destroy(TcProgram*);
-void tc_program_begin(TcProgram*, void* table_dev, unsigned int* done_dev);
+// pair: run every product in the pair form (each must satisfy tc_pair_ok, else tc_program_add fails)
+void tc_program_begin(TcProgram*, void* table_dev, unsigned int* done_dev, bool pair = false);
 // returns the product's index (negative on error, *status says why); deps: up to 3 indices, -1 = none
 int tc_program_add(TcProgram*, TcMapCache* cache, const TcGemm& g, const int* deps, int ndep,
                    mw_status* status);
@@ -177,6 +180,15 @@ int tc_tile_n(int a_planes, int b_planes, int M, int N, int batch);
 size_t tc_split_scratch_bytes(int a_planes, int b_planes, int M, int N, int batch, int split_k);
 // K split that gives every SM a work unit when the product alone has too few tiles (1 = none)
 int tc_auto_split(int a_planes, int b_planes, int M, int N, int K, int batch);
+
+// Pair form: two CTAs (a cluster of two SMs) share every 256-row tile and each stages half of the
+// B tile.  Grouped launches choose it by themselves when every product of the launch qualifies.
+bool tc_pair_ok(int a_planes, int b_planes, int M, int N);
+int tc_set_pair_mode(int mode);           // 0: never (for comparisons), 1: where it qualifies; returns the old mode
+// bound of the device-side waits of later launches (0 = default, 2 s)
+void tc_set_wait_limit_ns(uint64_t ns);
+// slots of TcEpilogue::sumsq for one product
+size_t tc_sumsq_slots(int a_planes, int b_planes, int M, int N);
 
 // Per-launch timing of the product kernel (CUDA events around every launch while enabled).
 void tc_profile_begin();

@@ -8,7 +8,7 @@ namespace mw {
 struct TcMapCache;
 struct TcProgram;
 // programs (whole phases in one launch) are rebuilt only when a buffer they name has moved
-enum { MW_PROG_PHASE1 = 0, MW_PROG_PHASE2, MW_PROG_SWEEP, MW_PROG_BP_FWD, MW_PROG_BP_BWD, MW_PROG_COUNT };
+enum { MW_PROG_PHASE1 = 0, MW_PROG_PHASE2, MW_PROG_BP_FWD, MW_PROG_BP_BWD, MW_PROG_COUNT };
 struct TensorState {
   TcMapCache* cache = nullptr;
   TcProgram* prog[MW_PROG_COUNT] = {};

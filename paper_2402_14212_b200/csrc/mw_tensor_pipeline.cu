@@ -144,15 +144,31 @@ split_weights_kernel(PtrBatch Ws, int64_t n4, int64_t n2, __nv_bfloat16* __restr
   }
 }
 
-__global__ void residual_gate_kernel(const double* __restrict__ sumsq, int group, int n,
-                                     double limit, DeviceStatus* st, int layer0, int stride = 1) {
-  const int g = blockIdx.x * blockDim.x + threadIdx.x;
-  if (g < group) {
-    const double r = sqrt(sumsq[(int64_t)g * stride] / (double)n);   // rms singular value of I - W X
+// One CTA per matrix: adds the `slots` pieces of ||I - W X||_F^2 that the residual product's
+// epilogue warps left (always in the same order, so the decision does not depend on scheduling)
+// and reports the layer when the rms singular value of the residual exceeds `limit`.
+__global__ void __launch_bounds__(256)
+residual_gate_kernel(const double* __restrict__ pieces, int64_t stride, int64_t slots, int n,
+                     double limit, DeviceStatus* st, int layer0) {
+  __shared__ double red[256];
+  const double* mine = pieces + (int64_t)blockIdx.x * stride;
+  double a = 0.0;
+  for (int64_t i = threadIdx.x; i < slots; i += 256) a += mine[i];
+  red[threadIdx.x] = a;
+  __syncthreads();
+  for (int o = 128; o; o >>= 1) {
+    if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const double r = sqrt(red[0] / (double)n);   // rms singular value of I - W X
     if (!(r <= limit))
-      record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)(layer0 + g), __float_as_uint((float)r), 3u, 0u);
+      record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)(layer0 + blockIdx.x), __float_as_uint((float)r), 3u, 0u);
   }
 }
+
+// slots of ||R||_F^2 pieces per matrix, for the narrowest tile a residual product may use
+size_t gate_slots(int d) { return (size_t)(d / 128 + 1) * (d / 64) * 4; }
 
 // layers per Newton-Schulz group: enough 128x128 tiles for several waves of the 148 SMs
 int ns_group(const mw_net* n) {
@@ -228,9 +244,9 @@ mw_status newton_schulz_group(const Ctx& c, int l0, int G, const void* const* pa
   __nv_bfloat16* Rp = c.at<__nv_bfloat16>(lay.ns_r);            // [G][3][n*n]
   __nv_bfloat16* Xp[2] = {Rp + (int64_t)3 * G * c.nn, Rp + (int64_t)6 * G * c.nn};
   char* sc = c.at<char>(lay.inv_scratch);
-  double* sumsq = reinterpret_cast<double*>(sc);                // [G]
   float* cscale = reinterpret_cast<float*>(sc + 8 * kMaxGroup); // [G]
   double* fpart = reinterpret_cast<double*>(sc + 12 * kMaxGroup + 64);   // [G][kFrobBlocks]
+  double* sumsq = c.at<double>(lay.ns_sumsq);                   // [G][gate_slots]
   __nv_bfloat16* dst = c.at<__nv_bfloat16>(lay.inv[l0]);
   const int64_t dst_stride = G > 1 ? (int64_t)(lay.inv[l0 + 1].off - lay.inv[l0].off) / 2 : 0;
 
@@ -279,11 +295,10 @@ mw_status newton_schulz_group(const Ctx& c, int l0, int G, const void* const* pa
     const bool last = it + 1 == steps;
     const int pw = c.pr.pw < sched[it].pr ? c.pr.pw : sched[it].pr;
     // R = I - W X
-    MW_CUDA_OK(cudaMemsetAsync(sumsq, 0, sizeof(double) * G, c.s));
     TcEpilogue er;
     er.mode = TC_EPI_RESID;
     er.planes = Rp; er.n_planes = sched[it].pu; er.plane_stride = c.nn; er.bs_planes = 3 * c.nn;
-    er.sumsq = sumsq; er.bs_sumsq = 1;
+    if (last) { er.sumsq = sumsq; er.bs_sumsq = (int64_t)gate_slots(d); }
     TcOperand wa = operand(Wbase, d, d, pw, false);
     wa.batch_planes = w_batch_planes;
     TcOperand xb = operand(Xp[cur], d, d, sched[it].pr, true);
@@ -292,7 +307,8 @@ mw_status newton_schulz_group(const Ctx& c, int l0, int G, const void* const* pa
     if (last) {
       // the update squares this residual: gate on it so a diverging layer is reported
       const double limit = f32 ? 2e-3 : 2e-2;
-      residual_gate_kernel<<<1, kMaxGroup, 0, c.s>>>(sumsq, G, d, limit, c.st, l0);
+      residual_gate_kernel<<<G, 256, 0, c.s>>>(sumsq, (int64_t)gate_slots(d),
+                                               (int64_t)tc_sumsq_slots(pw, sched[it].pr, d, d), d, limit, c.st, l0);
       MW_TRY(launch_ok());
     }
     // X' = X + X R
@@ -419,7 +435,6 @@ mw_status loss_and_top(const Ctx& c, const void* target, double* loss_out, bool 
 // In the program path every layer has its own iterate (fp32 X, term planes of X and of the
 // residual), so that the steps of different layers can be spread over the launches that carry
 // Phase I and Phase II: the chains of those phases leave most SMs waiting, the inverses fill them.
-constexpr int kNsSumsqStride = 16;   // doubles per layer in ns_sumsq (one per step)
 
 struct NsBuffers {
   float* X;
@@ -448,7 +463,6 @@ mw_status ns_prepare_all(const Ctx& c, const void* const* params, const NsStep* 
   char* sc = c.at<char>(lay.inv_scratch);
   float* cscale = reinterpret_cast<float*>(sc + 8 * kMaxGroup);
   double* fpart = reinterpret_cast<double*>(sc + 12 * kMaxGroup + 64);
-  MW_CUDA_OK(cudaMemsetAsync(nb.sumsq, 0, sizeof(double) * kNsSumsqStride * L, c.s));
   const int first = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;
   for (int l0 = 0; l0 < L; l0 += kMaxGroup) {
     const int G = (L - l0) < kMaxGroup ? (L - l0) : kMaxGroup;
@@ -492,7 +506,8 @@ TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, con
     g.B = operand(Xc, d, d, sched[it].pr, true);
     g.epi.mode = TC_EPI_RESID;
     g.epi.planes = Rp; g.epi.n_planes = sched[it].pu; g.epi.plane_stride = c.nn;
-    g.epi.sumsq = nb.sumsq + (int64_t)l * kNsSumsqStride + it;
+    // only the last residual is gated (the update that follows squares it)
+    if (last) g.epi.sumsq = nb.sumsq + (int64_t)l * (int64_t)gate_slots(d);
   } else {
     int next_terms = c.pr.ph;
     if (!last) next_terms = sched[it + 1].pr > sched[it + 1].pu ? sched[it + 1].pr : sched[it + 1].pu;
@@ -540,12 +555,18 @@ bool program_ready(const Ctx& c, int idx, const std::vector<const void*>& key) {
   return t->prog[idx] != nullptr && !t->key[idx].empty() && t->key[idx] == key;
 }
 
+// every product of a dense bf16 net (batch x width and width x width outputs, at most two terms
+// per operand) can run in the pair form when both sizes are multiples of 256
+bool net_pair(const Ctx& c) {
+  return c.n->opts.prec != MW_F32 && tc_pair_ok(2, 2, c.B, c.dim) && tc_pair_ok(2, 2, c.dim, c.dim);
+}
+
 TcProgram* program_begin(const Ctx& c, int idx, int slot) {
   TensorState* t = state_of(c);
   if (!t->prog[idx]) t->prog[idx] = tc_program_create();
   t->key[idx].clear();
   tc_program_begin(t->prog[idx], c.at<char>(c.lay->prog_table[slot]),
-                   c.at<unsigned int>(c.lay->prog_done[slot]));
+                   c.at<unsigned int>(c.lay->prog_done[slot]), net_pair(c));
   return t->prog[idx];
 }
 
@@ -760,50 +781,6 @@ TcGemm weight_vjp_product(const Ctx& c, const __nv_bfloat16* gz, const __nv_bflo
                  c.dim, c.dim, c.B, e, 2);
 }
 
-// The forward sweep (Algorithm 1) as one launch.  Products of layer l: R_l recompute x_{l+1},
-// V_l vijp (g_z of layer l, h_{l+1}), D_l weight vjp.  R_l needs x_l (R_{l-1}) and the slot of
-// x_{l+1} free (D_{l-2} read x_{l-2} there); V_l needs h_l (V_{l-1}, unless a checkpoint) and the
-// g_z slot free (D_{l-2}); D_l needs g_z (V_l) and x_l (R_{l-1}).
-mw_status sweep_program(const Ctx& c, const void* const* params, const void* x, void* const* dW,
-                        const __nv_bfloat16* x0p) {
-  const Layout& lay = *c.lay;
-  mw_net* n = c.n;
-  const int L = n->L;
-  const std::vector<const void*> key = key_of(c, params, x, nullptr, dW);
-  if (!program_ready(c, MW_PROG_SWEEP, key)) {
-    Adder a{c, program_begin(c, MW_PROG_SWEEP, 2)};
-    std::vector<int> R(L, -1), V(L, -1), D(L, -1);
-    auto xbuf = [&](int l) -> const __nv_bfloat16* {
-      return l == 0 ? x0p : c.at<__nv_bfloat16>(lay.xp[l % 3]);
-    };
-    auto at_or = [](const std::vector<int>& v, int i) { return i >= 0 ? v[i] : -1; };
-    for (int l = 0; l <= L; ++l) {
-      if (l < L) {
-        const bool more = l + 1 < L;
-        const bool want_h = more && !is_reseed(n, l + 1);
-        if (more) {
-          const __nv_bfloat16* Wp = nullptr;
-          MW_TRY(weight_planes(c, l, params[l], false, &Wp));
-          R[l] = a.add(recompute_product(c, l, xbuf(l), Wp), at_or(R, l - 1), at_or(D, l - 2));
-        }
-        if (dW[l] || want_h) {
-          // V_{l-1} produced h_l, or (at a checkpoint) still reads the slot h_{l+1} goes to
-          V[l] = a.add(vijp_product(c, l, want_h, dW[l] != nullptr), at_or(V, l - 1), at_or(D, l - 2));
-        }
-      }
-      if (l >= 1 && dW[l - 1]) {
-        const int k = l - 1;
-        TcGemm g = weight_vjp_product(c, c.at<__nv_bfloat16>(lay.gzp[k & 1]), xbuf(k), (float*)dW[k]);
-        // a K-split weight vjp shares its meeting place with the previous one
-        D[k] = a.add(g, V[k], at_or(R, k - 1), g.split_k > 1 ? at_or(D, k - 1) : -1);
-      }
-    }
-    MW_TRY(a.status);
-    state_of(c)->key[MW_PROG_SWEEP] = key;
-  }
-  return tc_program_launch(state_of(c)->prog[MW_PROG_SWEEP], c.st, c.s);
-}
-
 // backprop's reverse pass as one launch: B_l (h_{l} -> g_z of layer l-1) and D_l read the same g_z
 mw_status backprop_program(const Ctx& c, const void* const* params, const void* x, void* const* dW,
                            const __nv_bfloat16* x0p) {
@@ -913,7 +890,7 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     if (s2) lay.split[2] = b.take(s2);
   }
   if (use_programs(n)) {
-    const int progs = backprop ? 2 : 3;
+    const int progs = 2;     // Phase I / Phase II, or backprop's forward / reverse pass
     for (int i = 0; i < progs; ++i) {
       lay.prog_table[i] = b.take(tc_program_table_bytes(5 * (L + 1)));
       lay.prog_done[i] = b.take(sizeof(unsigned int) * (5 * (size_t)(L + 1) + 1));
@@ -936,7 +913,7 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     }
     // program path: every layer keeps its own Newton-Schulz iterate
     const size_t G = use_programs(n) ? (size_t)L : (size_t)ns_group(n);
-    if (use_programs(n)) lay.ns_sumsq = b.take(sizeof(double) * kNsSumsqStride * (size_t)L);
+    lay.ns_sumsq = b.take(sizeof(double) * gate_slots((int)d) * G);
     lay.ns_x = b.take(4 * nn * G);
     lay.ns_r = b.take(2 * 9 * nn * G);  // per group member: R planes [3] + two iterate plane sets
     if (n->opts.prec != MW_F32 && G > 1 && !use_programs(n)) lay.ns_w = b.take(2 * nn * G);
@@ -981,8 +958,10 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
     MW_TRY(phase2_program(c, params, g0, &feed));             // Phase II
     // the last update squares the last residual: gate on it so a diverging layer is reported
     const double limit = n->opts.prec == MW_F32 ? 2e-3 : 2e-2;
-    residual_gate_kernel<<<(L + 63) / 64, 64, 0, s>>>(ns_buffers(c).sumsq + (feed.steps - 1), L, d, limit,
-                                                     c.st, 0, kNsSumsqStride);
+    const NsStep lastst = feed.sched[feed.steps - 1];
+    const int pw = c.pr.pw < lastst.pr ? c.pr.pw : lastst.pr;
+    residual_gate_kernel<<<L, 256, 0, s>>>(ns_buffers(c).sumsq, (int64_t)gate_slots(d),
+                                           (int64_t)tc_sumsq_slots(pw, lastst.pr, d, d), d, limit, c.st, 0);
     return launch_ok();
   }
   if (resident) {
@@ -1042,9 +1021,8 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
   const __nv_bfloat16* x0p = nullptr;
   MW_TRY(input_planes(c, x, &x0p));
   MW_TRY(split_planes((const float*)g0, c.bn, c.at<__nv_bfloat16>(lay.hp[0]), c.pr.ph, c.bn, s));
-  // The sweep as one launch (sweep_program) measures slower than one launch per layer: its two
-  // chains leave little for the waiting CTAs to do, so the per-layer launches stay the default.
-  if (use_programs(n) && n->opts.reserved == 1 && !n->apply_params) return sweep_program(c, params, x, dW, x0p);
+  // one launch per layer (the whole sweep as a single program launch measured slower: its two
+  // chains leave little for the waiting CTAs to do)
   auto xbuf = [&](int l) -> const __nv_bfloat16* {          // term planes of x_l
     return l == 0 ? x0p : c.at<__nv_bfloat16>(lay.xp[l % 3]);
   };
