@@ -74,6 +74,14 @@ struct alignas(64) TcProblem {
   int bm;                      // rows of one tile: 128, or 256 in the pair form
   int pa, pb, a_mn, b_mn, a_batch_planes, b_batch_planes;
   uint32_t b_tile_bytes, tx_bytes;   // per CTA: in the pair form a CTA stages half of the B tile
+  // layout of a stage and the copies that fill it (operands without a convolution window):
+  //   K-major operand   [plane][rows][64 k]: one box {64, rows, planes} per K block;
+  //   MN-major operand  [64-column group][plane][64 k][64] when one box may span the planes
+  //                     (*_tma_pl = 1), else [plane][group][64 k][64] with a box per plane.
+  uint32_t a_pl_bytes, b_pl_bytes;   // between the planes of an operand inside a stage
+  uint32_t a_h_bytes, b_h_bytes;     // between the 64-column groups of an MN-major operand
+  uint32_t a_desc_base, b_desc_base; // descriptor low word without the address (group distance << 16)
+  int a_tma_pl, b_tma_pl;            // copies per 64-column group (or per K-major tile): 1 or the plane count
   int nops, nblocks;
   float* split_partials;
   unsigned int* split_counters;
@@ -246,9 +254,6 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm,
 // shared-memory operand descriptor, 128-byte swizzle: the upper word is constant, the lower word
 // holds the start address (and, for MN-major tiles, the distance between 64-element groups)
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint32_t desc_lo_base(bool mn_major) {
-  return (mn_major ? (8192u >> 4) : 1u) << 16;
-}
 
 // kPair: one instruction for both CTAs of the pair (256 rows); the descriptors name the same
 // offsets in both shared memories, the accumulator address the same columns in both tensor memories
@@ -491,30 +496,62 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
   }
 }
 
-// The instructions of one 64-deep K block, as straight-line code: the issuing lane runs alone on
-// its scheduler, so every branch and every dependent integer instruction in this loop costs
-// tens of cycles that the tensor pipe would otherwise spend on the next product.
+// The K loop of one unit on the issuing lane.  A tcgen05.mma is accepted only while at most one
+// earlier instruction is still running, so whatever this lane executes between the last
+// instruction of a K block and the first of the next must fit into the run time of one
+// instruction (128 cycles at 256 columns) or the tensor pipe idles.  Hence: straight-line code
+// specialised by the instruction count, all addresses advanced by additions, and the barrier of
+// the NEXT stage polled (and the next K block's operands prepared) between the first K step and
+// the other three of the current block, where the latency is hidden behind the running products.
+struct MmaRing {
+  uint32_t stage, phase, stages;
+  uint32_t sb16, tiles16, stage16;        // operand base of the stage (16-byte units), ring start, stage size
+  uint32_t full, empty, full0, empty0;    // barriers of the stage, and of stage 0
+};
+
 template <int NOPS, bool kPair>
-__device__ __forceinline__ void issue_k_block(const uint32_t (&oa)[kMaxOps], const uint32_t (&ob)[kMaxOps],
-                                              const uint32_t (&oi)[kMaxOps], const uint32_t (&od)[kMaxOps],
-                                              const uint32_t (&orot)[kMaxOps], const uint32_t (&ofk)[kMaxOps],
-                                              uint32_t sb16, uint32_t a_kadv, uint32_t b_kadv,
-                                              uint32_t kbl) {
-  uint32_t d[NOPS], a[NOPS], b[NOPS], first[NOPS];
+__device__ __forceinline__ bool mma_unit(MmaRing& r, const TcOp* ops, uint32_t d_set, uint32_t a_base,
+                                         uint32_t b_base, uint32_t a_kadv, uint32_t b_kadv, int nkb,
+                                         const WaitCtx& wc) {
+  uint32_t oa[NOPS], ob[NOPS], oi[NOPS], od[NOPS], orot[NOPS], ofk[NOPS];
 #pragma unroll
   for (int o = 0; o < NOPS; ++o) {
-    d[o] = od[o] + ((kbl & 1u) ? orot[o] : 0u);
-    a[o] = oa[o] + sb16;
-    b[o] = ob[o] + sb16;
-    first[o] = kbl < ofk[o] ? 0u : 1u;
+    const TcOp op = ops[o];
+    oa[o] = op.a_off16 | a_base;
+    ob[o] = op.b_off16 | b_base;
+    oi[o] = op.idesc;
+    od[o] = d_set + op.dcol;
+    orot[o] = op.rot;
+    ofk[o] = op.first_kbs;
   }
+  bool ready = mbar_try_wait<kPair>(r.full, r.phase);
+  for (int kbl = 0; kbl < nkb; ++kbl) {
+    if (!ready && !mbar_wait<kPair>(r.full, r.phase, wc, 3u)) return false;
+    tc_fence_after();
+    uint32_t d[NOPS], a[NOPS], b[NOPS];
 #pragma unroll
-  for (int k4 = 0; k4 < BK / 16; ++k4) {
+    for (int o = 0; o < NOPS; ++o) {
+      d[o] = od[o] + ((kbl & 1) ? orot[o] : 0u);
+      a[o] = oa[o] + r.sb16;
+      b[o] = ob[o] + r.sb16;
+      umma_bf16<kPair>(d[o], a[o], b[o], oi[o], (uint32_t)kbl < ofk[o] ? 0u : 1u);
+    }
+    // the ring moves on while the first products run
+    const uint32_t freed = r.empty;
+    r.sb16 += r.stage16; r.full += 8u; r.empty += 8u;
+    if (++r.stage == r.stages) {
+      r.stage = 0; r.phase ^= 1u; r.sb16 = r.tiles16; r.full = r.full0; r.empty = r.empty0;
+    }
+    ready = (kbl + 1 < nkb) && mbar_try_wait<kPair>(r.full, r.phase);
 #pragma unroll
-    for (int o = 0; o < NOPS; ++o)
-      umma_bf16<kPair>(d[o], a[o] + (uint32_t)k4 * a_kadv, b[o] + (uint32_t)k4 * b_kadv, oi[o],
-                       k4 == 0 ? first[o] : 1u);
+    for (int k4 = 1; k4 < BK / 16; ++k4) {
+#pragma unroll
+      for (int o = 0; o < NOPS; ++o)
+        umma_bf16<kPair>(d[o], a[o] + (uint32_t)k4 * a_kadv, b[o] + (uint32_t)k4 * b_kadv, oi[o], 1u);
+    }
+    umma_commit<kPair>(freed);   // frees the stage once these products retire
   }
+  return true;
 }
 
 // unit u of the sorted list -> product, tile, batch item and K range
@@ -699,16 +736,56 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           wg_y = rem / P.cWo;
           wg_x = rem - wg_y * P.cWo;
         }
+        if (conv == TC_CONV_NONE) {
+          // Lean loop of the plain products.  This lane runs alone: whatever it computes between
+          // two copies delays the copies, so everything that does not change is hoisted and the
+          // barrier of the NEXT stage is polled while this stage's copies are being issued.
+          const CUtensorMap* tmA = &P.tmA;
+          const CUtensorMap* tmB = &P.tmB;
+          const uint32_t a_pl_bytes = P.a_pl_bytes, a_h_bytes = P.a_h_bytes;
+          const uint32_t b_pl_bytes = P.b_pl_bytes, b_h_bytes = P.b_h_bytes;
+          const int a_loops = P.a_tma_pl, b_loops = P.b_tma_pl;
+          const uint32_t b_off = (uint32_t)pa * kATileBytes;
+          const uint32_t txe = kPair ? 2u * tx : tx;
+          const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+          // pair form: the bytes of both CTAs are counted on the even CTA's barrier, which expects them all
+          const uint32_t full0_remote = kPair ? map_to_cta(full0, 0u) : full0;
+          const uint32_t stages = (uint32_t)p.stages, stage_bytes = p.stage_bytes;
+          uint32_t sbase = tiles + stage * stage_bytes;
+          bool ready = mbar_try_wait<kPair>(empty0 + 8u * stage, phase ^ 1u);
+          int k0 = w.kb0 * BK;
+          for (int kb = w.kb0; kb < w.kb1; ++kb, k0 += BK) {
+            if (!ready && !mbar_wait<kPair>(empty0 + 8u * stage, phase ^ 1u, wc, 1u)) { ok = false; break; }
+            if (!kPair || rank == 0) mbar_expect_tx(full0 + 8u * stage, txe);
+            const uint32_t fb = full0_remote + 8u * stage;
+            for (int pl = 0; pl < a_loops; ++pl) {
+              const uint32_t dst = sbase + (uint32_t)pl * a_pl_bytes;
+              if (a_mn) {
+                tma_load_3d<kPair>(dst, tmA, fb, am0, k0, a_pl0 + pl);
+                tma_load_3d<kPair>(dst + a_h_bytes, tmA, fb, am0 + 64, k0, a_pl0 + pl);
+              } else {
+                tma_load_3d<kPair>(dst, tmA, fb, k0, am0, a_pl0 + pl);
+              }
+            }
+            for (int pl = 0; pl < b_loops; ++pl) {
+              const uint32_t dst = sbase + b_off + (uint32_t)pl * b_pl_bytes;
+              if (b_mn) {
+                for (int h = 0; h < nbox; ++h)
+                  tma_load_3d<kPair>(dst + (uint32_t)h * b_h_bytes, tmB, fb, bn_first + h * 64, k0, b_pl0 + pl);
+              } else {
+                tma_load_3d<kPair>(dst, tmB, fb, k0, bn_first, b_pl0 + pl);
+              }
+            }
+            sbase += stage_bytes;
+            if (++stage == stages) { stage = 0; phase ^= 1u; sbase = tiles; }
+            ready = mbar_try_wait<kPair>(empty0 + 8u * stage, phase ^ 1u);
+          }
+          continue;
+        }
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           if (!mbar_wait<kPair>(smem_u32(&empty_bar[stage]), phase ^ 1u, wc, 1u)) { ok = false; break; }
-          // the bytes of both CTAs are counted on the even CTA's barrier, which expects them all
-          uint32_t fb = smem_u32(&full_bar[stage]);
-          if (kPair) {
-            if (rank == 0) mbar_expect_tx(fb, 2u * tx);
-            fb = map_to_cta(fb, 0u);
-          } else {
-            mbar_expect_tx(fb, tx);
-          }
+          const uint32_t fb = smem_u32(&full_bar[stage]);
+          mbar_expect_tx(fb, tx);
           const uint32_t sbase = tiles + stage * p.stage_bytes;
           int k0 = kb * BK;
           int bk0 = k0, bn0 = bn_first;       // B coordinates (K, N)
@@ -721,7 +798,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
                           P.cstride * cy0 + dy, cb, a_pl0 + pl);
             bk0 = (tb * P.ccb + cblk) * BK;
             if (P.b_tap_rows) { bn0 = tb * P.N + w.n0; bk0 = cblk * BK; }
-          } else if (conv == TC_CONV_WGRAD) {
+          } else {
             // K block = 64 pixels of slice z (one box: part of a row, rows, or images); the two
             // halves of the A tile are two blocks of 64 rows (tap, channel block)
             const int pix = (w.z * P.num_kb + kb) * BK;
@@ -738,15 +815,6 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
             }
             bk0 = pix;
             k0 = pix;
-          } else
-          for (int pl = 0; pl < pa; ++pl) {
-            const uint32_t dst = sbase + (uint32_t)pl * kATileBytes;
-            if (a_mn) {
-              tma_load_3d<kPair>(dst, &P.tmA, fb, am0, k0, a_pl0 + pl);
-              tma_load_3d<kPair>(dst + 8192u, &P.tmA, fb, am0 + 64, k0, a_pl0 + pl);
-            } else {
-              tma_load_3d<kPair>(dst, &P.tmA, fb, k0, am0, a_pl0 + pl);
-            }
           }
           const uint32_t bbase = sbase + (uint32_t)pa * kATileBytes;
           const int bz = conv == TC_CONV_WGRAD ? 0 : b_pl0;
@@ -754,9 +822,9 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
             const uint32_t dst = bbase + (uint32_t)pl * b_tile_bytes;
             if (b_mn) {
               for (int h = 0; h < nbox; ++h)
-                tma_load_3d<kPair>(dst + (uint32_t)h * 8192u, &P.tmB, fb, bn0 + h * 64, bk0, bz + pl);
+                tma_load_3d<false>(dst + (uint32_t)h * 8192u, &P.tmB, fb, bn0 + h * 64, bk0, bz + pl);
             } else {
-              tma_load_3d<kPair>(dst, &P.tmB, fb, bk0, bn0, bz + pl);
+              tma_load_3d<false>(dst, &P.tmB, fb, bk0, bn0, bz + pl);
             }
           }
           if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
@@ -766,51 +834,34 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
   } else if (warp == 1) {
     // ---------------- MMA issuer (pair form: of the even CTA only) ----------------
     if (lane == 0 && rank == 0) {
-      uint32_t stage = 0, phase = 0;
+      MmaRing ring;
+      ring.stage = 0; ring.phase = 0; ring.stages = (uint32_t)p.stages;
+      ring.tiles16 = tiles >> 4; ring.stage16 = p.stage_bytes >> 4; ring.sb16 = ring.tiles16;
+      ring.full0 = smem_u32(&full_bar[0]); ring.empty0 = smem_u32(&empty_bar[0]);
+      ring.full = ring.full0; ring.empty = ring.empty0;
       int j = 0, q = 0, rr = 0;
-      bool ok = true;
       for (;;) {
-        if (!ok) break;
         const int u = next_unit<kProgram, kPair>(p, rr);
         if (u < 0) break;
         Unit w;
         decode_unit(probs, ub, nprob, u, q, w);
         const TcProblem& P = probs[w.q];
         const uint32_t set = (uint32_t)j & 1u, aphase = ((uint32_t)j >> 1) & 1u;
-        if (!mbar_wait<kPair>(smem_u32(&acc_empty[set]), aphase ^ 1u, wc, 2u)) { ok = false; break; }
+        if (!mbar_wait<kPair>(smem_u32(&acc_empty[set]), aphase ^ 1u, wc, 2u)) break;
         tc_fence_after();
         const uint32_t d_set = tmem_base + set * (uint32_t)kSetCols;
-        // the unit's instruction list, in registers
-        uint32_t oa[kMaxOps], ob[kMaxOps], oi[kMaxOps], od[kMaxOps], orot[kMaxOps], ofk[kMaxOps];
-        const int nops = P.nops;
-#pragma unroll
-        for (int o = 0; o < kMaxOps; ++o) {
-          const TcOp op = P.ops[o < nops ? o : 0];
-          oa[o] = op.a_off16 | desc_lo_base(P.a_mn != 0);
-          ob[o] = op.b_off16 | desc_lo_base(P.b_mn != 0);
-          oi[o] = op.idesc;
-          od[o] = d_set + op.dcol;
-          orot[o] = op.rot;
-          ofk[o] = op.first_kbs;
-        }
         // K advance of 16 elements: 32 bytes along a K-major row, 16 rows of 128 bytes otherwise
         const uint32_t a_kadv = P.a_mn ? (2048u >> 4) : (32u >> 4);
         const uint32_t b_kadv = P.b_mn ? (2048u >> 4) : (32u >> 4);
         const int nkb = w.kb1 - w.kb0;
-        for (int kbl = 0; kbl < nkb; ++kbl) {
-          if (!mbar_wait<kPair>(smem_u32(&full_bar[stage]), phase, wc, 3u)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t sb16 = (tiles + stage * p.stage_bytes) >> 4;
-          switch (nops) {
-            case 1: issue_k_block<1, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            case 2: issue_k_block<2, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            case 3: issue_k_block<3, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            case 4: issue_k_block<4, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            case 5: issue_k_block<5, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-            default: issue_k_block<6, kPair>(oa, ob, oi, od, orot, ofk, sb16, a_kadv, b_kadv, (uint32_t)kbl); break;
-          }
-          umma_commit<kPair>(smem_u32(&empty_bar[stage]));  // frees the stage once these products retire
-          if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1u; }
+        bool ok;
+        switch (P.nops) {
+          case 1: ok = mma_unit<1, kPair>(ring, P.ops, d_set, P.a_desc_base, P.b_desc_base, a_kadv, b_kadv, nkb, wc); break;
+          case 2: ok = mma_unit<2, kPair>(ring, P.ops, d_set, P.a_desc_base, P.b_desc_base, a_kadv, b_kadv, nkb, wc); break;
+          case 3: ok = mma_unit<3, kPair>(ring, P.ops, d_set, P.a_desc_base, P.b_desc_base, a_kadv, b_kadv, nkb, wc); break;
+          case 4: ok = mma_unit<4, kPair>(ring, P.ops, d_set, P.a_desc_base, P.b_desc_base, a_kadv, b_kadv, nkb, wc); break;
+          case 5: ok = mma_unit<5, kPair>(ring, P.ops, d_set, P.a_desc_base, P.b_desc_base, a_kadv, b_kadv, nkb, wc); break;
+          default: ok = mma_unit<6, kPair>(ring, P.ops, d_set, P.a_desc_base, P.b_desc_base, a_kadv, b_kadv, nkb, wc); break;
         }
         if (!ok) break;
         umma_commit<kPair>(smem_u32(&acc_full[set]));
@@ -1124,10 +1175,10 @@ TcMapCache* tc_cache_create() { return new TcMapCache(); }
 void tc_cache_destroy(TcMapCache* c) { delete c; }
 
 static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, int total_planes,
-                         CUtensorMap* out) {
+                         CUtensorMap* out, int box_planes = 1) {
   const int64_t ld = op.ld ? op.ld : op.cols;
   auto key = std::make_tuple(op.base, op.rows, op.cols, total_planes, op.plane_stride,
-                             (int64_t)box_rows + (ld << 12));
+                             (int64_t)box_rows + ((int64_t)box_planes << 10) + (ld << 12));
   if (cache) {
     auto it = cache->maps.find(key);
     if (it != cache->maps.end()) { *out = it->second; return MW_OK; }
@@ -1139,7 +1190,7 @@ static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, i
   if (ps % 8 != 0) return MW_ERR_INVALID_ARG;
   cuuint64_t dims[3] = {(cuuint64_t)op.cols, (cuuint64_t)op.rows, (cuuint64_t)total_planes};
   cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)ps * 2};
-  cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, 1u};
+  cuuint32_t box[3] = {64u, (cuuint32_t)box_rows, (cuuint32_t)box_planes};
   cuuint32_t estr[3] = {1u, 1u, 1u};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(op.base), dims, strides,
                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1203,14 +1254,14 @@ double build_ops_pair(TcProblem& P) {
     for (int j = 0; j < pb; ++j) {
       if (i + j >= t) continue;
       TcOp& o = P.ops[n++];
-      o.a_off16 = ((uint32_t)i * kATileBytes) >> 4;
-      o.b_off16 = (b0 + (uint32_t)j * P.b_tile_bytes) >> 4;
+      o.a_off16 = ((uint32_t)i * P.a_pl_bytes) >> 4;
+      o.b_off16 = (b0 + (uint32_t)j * P.b_pl_bytes) >> 4;
       o.idesc = make_idesc(P.a_mn != 0, P.b_mn != 0, bn, 2 * BM);
       o.dcol = (uint16_t)((i + j) * bn);
       o.rot = 0;
       o.first_kbs = init[i + j] ? 0u : 1u;
       init[i + j] = true;
-      cycles += 4.0 * (bn / 2.0);
+      cycles += 4.0 * std::max(bn / 2.0, 88.0);
     }
   P.nops = n;
   P.nblocks = t;
@@ -1231,14 +1282,14 @@ double build_ops(TcProblem& P, bool rotate) {
   double cycles = 0.0;
   auto add = [&](int i, int j0, int cnt, int rot, int first) {
     TcOp& o = P.ops[n++];
-    o.a_off16 = ((uint32_t)i * kATileBytes) >> 4;
-    o.b_off16 = (b0 + (uint32_t)j0 * P.b_tile_bytes) >> 4;
+    o.a_off16 = ((uint32_t)i * P.a_pl_bytes) >> 4;
+    o.b_off16 = (b0 + (uint32_t)j0 * P.b_pl_bytes) >> 4;
     o.idesc = make_idesc(P.a_mn != 0, P.b_mn != 0, cnt * bn);
     o.dcol = (uint16_t)col(i + j0);
     o.rot = (uint16_t)rot;
     o.first_kbs = (uint32_t)first;
     const double w = cnt * bn;
-    cycles += 4.0 * std::max(w / 2.0, (128.0 + w) / 4.0);   // math vs shared-memory operand reads
+    cycles += 4.0 * std::max(w / 2.0, 88.0);   // an instruction takes at least 88 cycles whatever its width
   };
   for (int i = 0; i < pa; ++i) {
     int cnt = pb < t - i ? pb : t - i;
@@ -1348,6 +1399,18 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   const int b_cols = pair ? P.bn / 2 : P.bn;     // columns of the B tile one CTA stages
   P.b_tile_bytes = (uint32_t)b_cols * BK * 2;
   P.tx_bytes = (uint32_t)P.pa * kATileBytes + (uint32_t)P.pb * P.b_tile_bytes;
+  // stage layout and copies (see TcProblem).  Convolution windows keep a box per plane.
+  const bool plain = cv.mode == TC_CONV_NONE;
+  P.a_tma_pl = plain ? 1 : P.pa;
+  P.a_h_bytes = (P.a_mn && plain) ? (uint32_t)P.pa * 8192u : 8192u;
+  P.a_pl_bytes = (P.a_mn && plain) ? 8192u : kATileBytes;
+  // an instruction that spans several B planes (single form) needs each plane's groups adjacent
+  const bool b_span = plain && (!P.b_mn || pair || P.pb == 1);
+  P.b_tma_pl = b_span ? 1 : P.pb;
+  P.b_h_bytes = (P.b_mn && b_span) ? (uint32_t)P.pb * 8192u : 8192u;
+  P.b_pl_bytes = (P.b_mn && b_span) ? 8192u : P.b_tile_bytes;
+  P.a_desc_base = (P.a_mn ? (P.a_h_bytes >> 4) : 1u) << 16;
+  P.b_desc_base = (P.b_mn ? (P.b_h_bytes >> 4) : 1u) << 16;
   const int t = P.pa > P.pb ? P.pa : P.pb;
   // fp32-accurate products alternate the leading block (needs two K blocks per unit)
   const bool rotate = t == 3 && P.pa == 3 && P.pb == 3 && P.kb_per_split >= 2 &&
@@ -1373,8 +1436,8 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
     MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, cbx, cby, cbi, cv.stride, d.A.planes, &P.tmA));
     MW_TRY(get_map(cache, d.B, 64, d.B.planes, &P.tmB));
   } else {
-    MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA));
-    MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : b_cols, b_total, &P.tmB));
+    MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA, P.pa));
+    MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : b_cols, b_total, &P.tmB, b_span ? P.pb : 1));
   }
   int np = 0;
   for (int a = 0; a < P.pa; ++a)
