@@ -31,7 +31,7 @@ struct Layout {
   Region inv_scratch;
   // tensor-core backend operands (bf16 term planes)
   std::vector<Region> w_planes;              // split weights (MW_F32), per layer or one slot
-  Region xp[3], hp[2], gzp[2], ns_r, ns_x, ns_w; // activation / cotangent / g_z planes, NS scratch
+  Region xp[5], hp[2], gzp[4], ns_r, ns_x, ns_w; // activation / cotangent / g_z planes (rings), NS scratch
   // convolution nets on the tensor cores
   std::vector<Region> cw, cwhat, cwinv;      // per layer: kernel, folded kernel, centre-tap inverse (term planes)
   std::vector<Region> cfrag;                 // per layer: fragmental checkpoints of a 1-D convolution

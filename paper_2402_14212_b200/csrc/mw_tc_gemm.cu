@@ -91,8 +91,9 @@ struct alignas(64) TcProblem {
   signed char tdy[28], tdx[28], ttb[28];
   // program launches: products (by index) that must be complete before this one starts, and
   // the number of warp arrivals that completes each of them (one per epilogue warp and tile)
-  int ndep, dep[3];
-  unsigned int dep_target[3];
+  int ndep, dep[kTcMaxDeps];
+  unsigned int dep_target[kTcMaxDeps];
+  int done2;                   // a second counter this product's tiles report to (a group), or -1
   TcOp ops[kMaxOps];
 };
 
@@ -639,7 +640,8 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     // start fetching the tensor maps before the first copy needs them
     const TcProblem& P = probs[lane >> 1];
     const CUtensorMap* tm = (lane & 1) ? &P.tmB : &P.tmA;
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
+    if (P.unit_count > 0)     // (a group entry of a program has no maps)
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
   }
   if (warp == 1) {
     // pair form: the same warp of both CTAs allocates, and both get the same columns
@@ -1016,7 +1018,10 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         // program launch: publish this warp's part of the tile to the products that wait for it
         __threadfence();
         __syncwarp();
-        if (lane == 0) atomicAdd(p.done + w.q, 1u);
+        if (lane == 0) {
+          atomicAdd(p.done + w.q, 1u);
+          if (P.done2 >= 0) atomicAdd(p.done + P.done2, 1u);
+        }
       }
     }
   }
@@ -1376,6 +1381,7 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
     }
   }
   P.ndep = 0;
+  P.done2 = -1;
   P.M = d.M; P.N = d.N; P.K = d.K;
   P.pa = d.A.planes; P.pb = d.B.planes;
   P.a_mn = d.A.mn_major ? 1 : 0;
@@ -1604,6 +1610,7 @@ struct TcProgram {
   unsigned int* done_dev = nullptr;
   bool uploaded = false;
   bool pair = false;          // every product in the pair form (clusters of two CTAs)
+  std::vector<unsigned> target;   // arrivals that complete each table entry (product or group)
 };
 
 TcProgram* tc_program_create() { return new TcProgram(); }
@@ -1612,6 +1619,7 @@ void tc_program_destroy(TcProgram* p) { delete p; }
 void tc_program_begin(TcProgram* pr, void* table_dev, unsigned int* done_dev, bool pair) {
   pr->pair = pair && g_pair_mode != 0 && ensure_kernel_attr() == MW_OK && max_pairs(200 * 1024) > 0;
   pr->table.clear();
+  pr->target.clear();
   pr->stage_bytes = 0;
   pr->total_units = 0;
   pr->flops = pr->mma_flops = 0.0;
@@ -1621,9 +1629,9 @@ void tc_program_begin(TcProgram* pr, void* table_dev, unsigned int* done_dev, bo
 }
 
 int tc_program_add(TcProgram* pr, TcMapCache* cache, const TcGemm& d, const int* deps, int ndep,
-                   mw_status* status) {
+                   mw_status* status, int group) {
   *status = MW_OK;
-  if ((int)pr->table.size() >= kMaxProgram || ndep > 3) { *status = MW_ERR_UNSUPPORTED; return -1; }
+  if ((int)pr->table.size() >= kMaxProgram || ndep > kTcMaxDeps) { *status = MW_ERR_UNSUPPORTED; return -1; }
   pr->table.emplace_back();
   TcProblem& P = pr->table.back();
   double cost = 0.0;
@@ -1633,17 +1641,38 @@ int tc_program_add(TcProgram* pr, TcMapCache* cache, const TcGemm& d, const int*
   pr->total_units += P.unit_count;
   if (P.tx_bytes > pr->stage_bytes) pr->stage_bytes = P.tx_bytes;
   const int self = (int)pr->table.size() - 1;
+  // one arrival per epilogue warp and tile (of both CTAs in the pair form)
+  const unsigned arrivals = (unsigned)kEpiWarps * (pr->pair ? 2u : 1u) * (unsigned)(P.unit_count / P.split);
+  pr->target.push_back(arrivals);
+  if (group >= 0) {
+    if (group >= self || pr->table[group].unit_count != 0) { *status = MW_ERR_INVALID_ARG; return -1; }
+    P.done2 = group;
+    pr->target[group] += arrivals;
+  }
   for (int i = 0; i < ndep; ++i) {
     const int q = deps[i];
     if (q < 0) continue;
-    if (q >= self) { *status = MW_ERR_INVALID_ARG; return -1; }   // only earlier products
-    const TcProblem& Q = pr->table[q];
+    if (q >= self) { *status = MW_ERR_INVALID_ARG; return -1; }   // only earlier entries
     P.dep[P.ndep] = q;
-    // one arrival per epilogue warp and tile (of both CTAs in the pair form)
-    P.dep_target[P.ndep] = (unsigned)kEpiWarps * (pr->pair ? 2u : 1u) * (unsigned)(Q.unit_count / Q.split);
+    P.dep_target[P.ndep] = 0;     // filled in at launch, when the groups are complete
     ++P.ndep;
   }
   return self;
+}
+
+int tc_program_add_group(TcProgram* pr) {
+  if ((int)pr->table.size() >= kMaxProgram) return -1;
+  pr->table.emplace_back();
+  TcProblem& P = pr->table.back();
+  P = TcProblem();
+  P.unit_begin = pr->total_units;
+  P.unit_count = 0;
+  P.split = 1;
+  P.tiles_mn = 1;
+  P.tiles_n = 1;
+  P.done2 = -1;
+  pr->target.push_back(0u);
+  return (int)pr->table.size() - 1;
 }
 
 size_t tc_program_table_bytes(int products) { return (size_t)products * sizeof(TcProblem); }
@@ -1652,6 +1681,8 @@ mw_status tc_program_launch(TcProgram* pr, DeviceStatus* st, cudaStream_t s) {
   const int nprob = (int)pr->table.size();
   if (nprob == 0) return MW_OK;
   if (!pr->table_dev || !pr->done_dev || ((uintptr_t)pr->table_dev & 63u)) return MW_ERR_WORKSPACE;
+  for (TcProblem& P : pr->table)
+    for (int i = 0; i < P.ndep; ++i) P.dep_target[i] = pr->target[P.dep[i]];
   // the table travels with every launch: the caller's workspace is only promised to keep its
   // contents between the calls of one step
   MW_CUDA_OK(cudaMemcpyAsync(pr->table_dev, pr->table.data(), nprob * sizeof(TcProblem),

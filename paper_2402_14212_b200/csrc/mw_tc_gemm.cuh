@@ -23,6 +23,7 @@
 namespace mw {
 
 constexpr int kTcMaxGroup = 4;
+constexpr int kTcMaxDeps = 4;
 constexpr size_t kTcSplitCounterBytes = 65536;
 
 struct TcOperand {
@@ -168,9 +169,14 @@ TcProgram* tc_program_create();
 void tc_program_destroy(TcProgram*);
 // pair: run every product in the pair form (each must satisfy tc_pair_ok, else tc_program_add fails)
 void tc_program_begin(TcProgram*, void* table_dev, unsigned int* done_dev, bool pair = false);
-// returns the product's index (negative on error, *status says why); deps: up to 3 indices, -1 = none
+// returns the product's index (negative on error, *status says why); deps: up to kTcMaxDeps
+// indices of earlier entries (products or groups), -1 = none.  group: index of a group entry
+// (tc_program_add_group) that this product's tiles also report to, or -1: a later product that
+// names the group waits for all its members.
 int tc_program_add(TcProgram*, TcMapCache* cache, const TcGemm& g, const int* deps, int ndep,
-                   mw_status* status);
+                   mw_status* status, int group = -1);
+// an entry without work that stands for "all products added to it"; add it before its members
+int tc_program_add_group(TcProgram*);
 size_t tc_program_table_bytes(int products);
 mw_status tc_program_launch(TcProgram*, DeviceStatus* st, cudaStream_t s);
 constexpr int kTcMaxProgram = 768;

@@ -13,6 +13,9 @@ struct TensorState {
   TcMapCache* cache = nullptr;
   TcProgram* prog[MW_PROG_COUNT] = {};
   std::vector<const void*> key[MW_PROG_COUNT];
+  // the forward sweep as chained programs, one per run of layers that fits a product table
+  std::vector<TcProgram*> sweep;
+  std::vector<const void*> sweep_key;
 };
 
 // convolutional nets on the tensor cores (mw_conv_pipeline.cu): stride-1 same-size convolutions

@@ -204,6 +204,10 @@ struct Ctx {
   int B, dim;          // batch, width
   int64_t bn;          // B * width
   int64_t nn;          // width^2
+  // rings of the sweep: x_l lives in xp[l % nx], g_z of layer l in gzp[l % ngz].  3 and 2 slots
+  // are what one launch per layer needs; the chained sweep runs several layers at once and uses
+  // 5 and 4, so that a slot is reused only by a product three layers behind its last reader
+  int nx = 3, ngz = 2;
   template <typename T> T* at(const Region& r) const { return mw::at<T>(ws, r); }
 };
 
@@ -561,6 +565,13 @@ bool net_pair(const Ctx& c) {
   return c.n->opts.prec != MW_F32 && tc_pair_ok(2, 2, c.B, c.dim) && tc_pair_ok(2, 2, c.dim, c.dim);
 }
 
+// sizes at which the sweep may run as chains (the workspace then holds the longer rings)
+bool chain_sizes(const mw_net* n) {
+  const int d = n->layers[0].n_in;
+  return n->opts.prec != MW_F32 && n->opts.resident_inverse != 0 && n->B % 256 == 0 && d % 256 == 0 &&
+         5 * (n->L + 1) <= kTcMaxProgram;
+}
+
 TcProgram* program_begin(const Ctx& c, int idx, int slot) {
   TensorState* t = state_of(c);
   if (!t->prog[idx]) t->prog[idx] = tc_program_create();
@@ -583,12 +594,20 @@ struct Adder {
       f->last[l] = add(ns_product(c, l, stage, f->params, f->sched, f->steps), f->last[l]);
     }
   }
-  int add(const TcGemm& g, int d0 = -1, int d1 = -1, int d2 = -1) {
+  int add(const TcGemm& g, int d0 = -1, int d1 = -1, int d2 = -1) { return add_to(g, -1, d0, d1, d2); }
+  // the same, the product also reporting to the group entry `group` (-1: none)
+  int add_to(const TcGemm& g, int group, int d0 = -1, int d1 = -1, int d2 = -1) {
     if (status != MW_OK) return -1;
     const int deps[3] = {d0, d1, d2};
     mw_status st;
-    const int q = tc_program_add(pr, c.cache, g, deps, 3, &st);
+    const int q = tc_program_add(pr, c.cache, g, deps, 3, &st, group);
     if (q < 0) status = st;
+    return q;
+  }
+  int group() {
+    if (status != MW_OK) return -1;
+    const int q = tc_program_add_group(pr);
+    if (q < 0) status = MW_ERR_UNSUPPORTED;
     return q;
   }
 };
@@ -732,7 +751,7 @@ TcGemm recompute_product(const Ctx& c, int l, const __nv_bfloat16* xl, const __n
   e.write_mask = 0;
   e.act = ld.act;
   e.slope = (float)ld.slope;
-  e.planes = c.at<__nv_bfloat16>(c.lay->xp[(l + 1) % 3]);
+  e.planes = c.at<__nv_bfloat16>(c.lay->xp[(l + 1) % c.nx]);
   e.n_planes = c.pr.px;
   e.plane_stride = c.bn;
   return product(c, operand(xl, c.B, c.dim, c.pr.px, false), operand(Wp, c.dim, c.dim, c.pr.pw, false),
@@ -758,7 +777,7 @@ TcGemm vijp_product(const Ctx& c, int l, bool want_h, bool want_gz) {
     e.plane_stride2 = c.bn;
   }
   if (want_gz) {
-    e.planes = c.at<__nv_bfloat16>(lay.gzp[l & 1]);
+    e.planes = c.at<__nv_bfloat16>(lay.gzp[l % c.ngz]);
     e.n_planes = c.pr.pgw;
     e.plane_stride = c.bn;
   }
@@ -780,6 +799,100 @@ TcGemm weight_vjp_product(const Ctx& c, const __nv_bfloat16* gz, const __nv_bflo
   return product(c, operand(gz, c.B, c.dim, c.pr.pgw, true), operand(xl, c.B, c.dim, c.pr.pxw, true),
                  c.dim, c.dim, c.B, e, 2);
 }
+
+// ---- the forward sweep as chains of one program launch ---------------------------------------
+// Algorithm 1 walks the layers in order, but the rows of the batch never meet before the weight
+// vjp: block m of `rb` rows of h_{l+1} and x_{l+1} needs block m of h_l and x_l only.  The sweep is
+// therefore B / rb independent chains of products
+//   V_{l,m}  (g_z, h_{l+1})[rows m] = vijp of layer l applied to h_l[rows m]      (Eq. "h_i")
+//   R_{l,m}  x_{l+1}[rows m] = phi(x_l[rows m] W_l^T)                               (recompute)
+// plus, per layer, D_l = g_z^T x_l over all rows (Eq. "g_i"), which needs the whole of V_l and of
+// R_{l-1} (two group counters) and feeds nothing.  One launch carries the layers [l0, l1): a
+// chain's next product sits hundreds of list positions behind the one it waits for, so the CTAs
+// rarely wait, and there is no launch boundary (with its idle tail) per layer.
+mw_status sweep_chain_program(const Ctx& c0, TcProgram* pr, int l0, int l1, const void* const* params,
+                              void* const* dW, const __nv_bfloat16* x0p, bool pair) {
+  Ctx c = c0;
+  c.nx = 5;
+  c.ngz = 4;
+  const Layout& lay = *c.lay;
+  mw_net* n = c.n;
+  const int L = n->L, d = c.dim;
+  const int rb = pair ? 256 : 128, mt = c.B / rb;
+  tc_program_begin(pr, c.at<char>(lay.prog_table[0]), c.at<unsigned int>(lay.prog_done[0]), pair);
+  Adder a{c, pr};
+  auto xbuf = [&](int l) -> const __nv_bfloat16* {
+    return l == 0 ? x0p : c.at<__nv_bfloat16>(lay.xp[l % c.nx]);
+  };
+  const int64_t blk = (int64_t)rb * d;                 // elements of one row block
+  const int nl = l1 - l0;
+  std::vector<int> GV((size_t)nl, -1), GR((size_t)nl, -1), D((size_t)nl, -1);
+  // the latest product of each chain (layers that need no vijp leave a gap in the V chain: the
+  // next V still follows the last one, which orders every reuse of the h slots of its rows)
+  std::vector<int> Vprev((size_t)mt, -1), Rprev((size_t)mt, -1);
+  int gz_reader[4] = {-1, -1, -1, -1};   // the latest weight vjp that read each g_z slot
+  auto at_or = [&](const std::vector<int>& v, int l) { return l >= l0 && l < l1 ? v[(size_t)(l - l0)] : -1; };
+  auto weight_vjp = [&](int k) {
+    if (!dW[k]) return;
+    const TcGemm g = weight_vjp_product(c, c.at<__nv_bfloat16>(lay.gzp[k % c.ngz]), xbuf(k), (float*)dW[k], k);
+    // g_z of layer k (all of V_k) and x_k (all of R_{k-1}); a K-split product shares its meeting
+    // place with the previous weight vjp
+    D[(size_t)(k - l0)] = a.add(g, at_or(GV, k), at_or(GR, k - 1), g.split_k > 1 ? at_or(D, k - 1) : -1);
+    gz_reader[k % c.ngz] = D[(size_t)(k - l0)];
+  };
+  for (int l = l0; l < l1; ++l) {
+    const bool more = l + 1 < L;
+    const bool want_h = more && !is_reseed(n, l + 1);
+    const bool want_v = dW[l] != nullptr || want_h;
+    if (want_v) {
+      GV[(size_t)(l - l0)] = a.group();
+      const TcGemm full = vijp_product(c, l, want_h, dW[l] != nullptr);
+      for (int m = 0; m < mt; ++m) {
+        TcGemm g = full;
+        g.M = rb;
+        g.A.base = static_cast<const __nv_bfloat16*>(full.A.base) + m * blk;
+        g.A.rows = rb;
+        TcEpilogue& e = g.epi;
+        e.mask += (int64_t)m * rb * (d / 32);
+        if (e.frag_off) { e.frag_off += (int64_t)m * rb; e.frag_rank += (int64_t)m * rb * (d / 64); }
+        if (e.planes) e.planes += m * blk;
+        if (e.planes2) e.planes2 += m * blk;
+        // the chain's last V made h_l[rows m] (or, at a checkpoint, was the last to use the slot
+        // h_{l+1} goes to); the g_z slot this product overwrites must have been read
+        Vprev[(size_t)m] = a.add_to(g, GV[(size_t)(l - l0)], Vprev[(size_t)m], gz_reader[l % c.ngz]);
+      }
+    }
+    if (more) {
+      GR[(size_t)(l - l0)] = a.group();
+      const __nv_bfloat16* Wp = nullptr;
+      MW_TRY(weight_planes(c, l, params[l], false, &Wp));
+      const TcGemm full = recompute_product(c, l, xbuf(l), Wp);
+      for (int m = 0; m < mt; ++m) {
+        TcGemm g = full;
+        g.M = rb;
+        g.A.base = static_cast<const __nv_bfloat16*>(full.A.base) + m * blk;
+        g.A.rows = rb;
+        g.epi.mask += (int64_t)m * rb * (d / 32);
+        g.epi.planes += m * blk;
+        // R_{l-1,m} made x_l[rows m]; the slot x_{l+1} goes to held x_{l+1-nx}, which the weight
+        // vjp of that layer read
+        Rprev[(size_t)m] = a.add_to(g, GR[(size_t)(l - l0)], Rprev[(size_t)m], at_or(D, l + 1 - c.nx));
+      }
+    }
+    // the weight vjp of the layer before comes after this layer's chain products in the list:
+    // by then its g_z is usually complete
+    if (l - 1 >= l0) weight_vjp(l - 1);
+    MW_TRY(a.status);
+  }
+  weight_vjp(l1 - 1);
+  return a.status;
+}
+
+// 1: nets that qualify run the sweep as chained programs (0: one launch per layer, for comparisons)
+int g_sweep_chains = 1;
+
+// entries of the product table per layer of a chained sweep
+int chain_entries_per_layer(const Ctx& c, bool pair) { return 2 * (c.B / (pair ? 256 : 128)) + 3; }
 
 // backprop's reverse pass as one launch: B_l (h_{l} -> g_z of layer l-1) and D_l read the same g_z
 mw_status backprop_program(const Ctx& c, const void* const* params, const void* x, void* const* dW,
@@ -870,10 +983,13 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
   const bool resident = n->opts.resident_inverse != 0;
   lay.z = b.take(4 * bn);                                   // fp32 network output
   for (int i = 0; i < 2; ++i) lay.cot[i] = b.take(4 * bn);  // fp32 cotangent scratch (loss top)
-  for (int i = 0; i < 3; ++i) lay.xp[i] = b.take(2 * (size_t)pr.px * bn);
+  // (two more x slots and two more g_z slots where the sweep runs as chains: see Ctx)
+  const bool chains = !backprop && chain_sizes(n);
+  for (int i = 0; i < (chains ? 5 : 3); ++i) lay.xp[i] = b.take(2 * (size_t)pr.px * bn);
   const int hpl = pr.ph > pr.pg2 ? pr.ph : pr.pg2;
   for (int i = 0; i < 2; ++i) lay.hp[i] = b.take(2 * (size_t)hpl * bn);
-  for (int i = 0; i < 2; ++i) lay.gzp[i] = b.take(2 * (size_t)(pr.pgw > pr.pg2 ? pr.pgw : pr.pg2) * bn);
+  for (int i = 0; i < (chains ? 4 : 2); ++i)
+    lay.gzp[i] = b.take(2 * (size_t)(pr.pgw > pr.pg2 ? pr.pgw : pr.pg2) * bn);
   // K-split meeting places: slot 0 recompute / Phase I / Phase II, slot 1 vijp, slot 2 weight vjp
   {
     const int B = n->B, dd = (int)d;
@@ -891,9 +1007,11 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
   }
   if (use_programs(n)) {
     const int progs = 2;     // Phase I / Phase II, or backprop's forward / reverse pass
+    // (table 0 also holds the chained forward sweep: up to kTcMaxProgram entries)
     for (int i = 0; i < progs; ++i) {
-      lay.prog_table[i] = b.take(tc_program_table_bytes(5 * (L + 1)));
-      lay.prog_done[i] = b.take(sizeof(unsigned int) * (5 * (size_t)(L + 1) + 1));
+      const size_t entries = (i == 0 && !backprop) ? (size_t)kTcMaxProgram : 5 * (size_t)(L + 1);
+      lay.prog_table[i] = b.take(tc_program_table_bytes((int)entries));
+      lay.prog_done[i] = b.take(sizeof(unsigned int) * (entries + 1));
     }
   }
   if (n->opts.prec == MW_F32) {
@@ -927,6 +1045,7 @@ void tensor_destroy(mw_net* n) {
     TensorState* t = static_cast<TensorState*>(n->tc);
     for (int i = 0; i < MW_PROG_COUNT; ++i)
       if (t->prog[i]) tc_program_destroy(t->prog[i]);
+    for (TcProgram* pr : t->sweep) tc_program_destroy(pr);
     tc_cache_destroy(t->cache);
     delete t;
     n->tc = nullptr;
@@ -1021,8 +1140,31 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
   const __nv_bfloat16* x0p = nullptr;
   MW_TRY(input_planes(c, x, &x0p));
   MW_TRY(split_planes((const float*)g0, c.bn, c.at<__nv_bfloat16>(lay.hp[0]), c.pr.ph, c.bn, s));
-  // one launch per layer (the whole sweep as a single program launch measured slower: its two
-  // chains leave little for the waiting CTAs to do)
+  // Nets whose products all run in the pair form (bf16 storage, sizes multiples of 256): the sweep
+  // as chains of products inside program launches, as many layers per launch as the table holds.
+  if (use_programs(n) && chain_sizes(n) && !n->apply_params && net_pair(c) && g_sweep_chains) {
+    TensorState* t = state_of(c);
+    const int per_layer = chain_entries_per_layer(c, true);
+    const int chunk = (kTcMaxProgram - 4) / per_layer;
+    if (chunk >= 1) {
+      const int nchunks = (L + chunk - 1) / chunk;
+      const std::vector<const void*> key = key_of(c, params, x, nullptr, dW);
+      if (t->sweep_key != key || (int)t->sweep.size() != nchunks) {
+        t->sweep_key.clear();
+        while ((int)t->sweep.size() < nchunks) t->sweep.push_back(tc_program_create());
+        while ((int)t->sweep.size() > nchunks) { tc_program_destroy(t->sweep.back()); t->sweep.pop_back(); }
+        for (int i = 0; i < nchunks; ++i) {
+          const int l0 = i * chunk, l1 = l0 + chunk < L ? l0 + chunk : L;
+          MW_TRY(sweep_chain_program(c, t->sweep[(size_t)i], l0, l1, params, dW, x0p, true));
+        }
+        t->sweep_key = key;
+      }
+      for (TcProgram* pr : t->sweep) MW_TRY(tc_program_launch(pr, c.st, c.s));
+      return MW_OK;
+    }
+  }
+  // otherwise one launch per layer (for nets of small products the whole sweep as one program
+  // launch measured slower: its chains leave little for the waiting CTAs to do)
   auto xbuf = [&](int l) -> const __nv_bfloat16* {          // term planes of x_l
     return l == 0 ? x0p : c.at<__nv_bfloat16>(lay.xp[l % 3]);
   };

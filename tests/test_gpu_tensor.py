@@ -55,3 +55,42 @@ def test_config5_depth32_full_width():
     # weight matrices cycled over the depth
     p = S.sweep_mlp(seed=0, depth=32, pool=4)
     check_problem(p, 2e-2, backend="tensor", exact_masks=False, tau=2e-2)
+
+
+@pytest.mark.parametrize("pair", [True, False])
+@pytest.mark.parametrize("n,depth,batch,K", [(256, 8, 256, 4), (512, 10, 512, 4), (256, 9, 768, 3)])
+def test_bf16_mixed_pair_sizes(n, depth, batch, K, pair):
+    """Sizes at which every product qualifies for the CTA-pair form (batch and width multiples of
+    256): the sweep then runs as chains of row blocks inside program launches.  The same nets with
+    the pair form switched off take the one-launch-per-layer path; both against the oracle."""
+    from paper_2402_14212_b200 import binding as mwb
+    old = mwb.set_pair_mode(pair)
+    try:
+        p = S.mixed_mlp(seed=4, depth=depth, n=n, batch=batch, reseed_every=K, prec=S.BF16)
+        check_problem(p, 2e-2, backend="tensor", exact_masks=False, tau=2e-2)
+    finally:
+        mwb.set_pair_mode(old)
+
+
+def test_bf16_pair_sizes_gradients_skipped():
+    """dW_out entries left out (gradients need not coexist): the chained sweep drops the weight vjp
+    of those layers and still carries the cotangent through them."""
+    import torch
+    from paper_2402_14212_b200 import binding as mwb
+    from oracle import moonwalk_oracle as O
+    from parity_util import oracle_masks_from_words
+    p = S.sweep_mlp(seed=5, depth=7, n=256, batch=256, reseed_every=3, prec=S.BF16)
+    net = mwb.net_for(p, backend="tensor")
+    params, x, target = mwb.to_device(p)
+    ws = net.alloc_workspace("moonwalk")
+    g0 = net.input_cotangent(params, x, target, ws)
+    keep = [0, 2, 3, 6]
+    dW = [torch.zeros(w.shape, dtype=torch.float32, device="cuda") if l in keep else None
+          for l, w in enumerate(params)]
+    net.forward_sweep(params, x, g0, ws, dW_out=dW)
+    code, detail = net.last_device_status(ws)
+    assert code == 0, detail
+    masks = oracle_masks_from_words(p, [net.export_masks(ws, l) for l in range(len(p.layers))])
+    ref = O.backprop(p.layers, p.params, p.x, p.target, p.loss, masks=masks)
+    for l in keep:
+        assert O.normwise_error(dW[l].double().cpu().numpy(), ref["dW"][l]) <= 2e-2, l
