@@ -54,6 +54,7 @@ constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;   // 2 s: far above any 
 constexpr int kMaxStages = 8;
 constexpr int kMaxOps = 6;
 constexpr uint32_t kATileBytes = BM * BK * 2;  // one A term plane of one stage
+constexpr uint32_t kEpiStageBytes = 4096;       // one 32 x 32 fp32 block (or two bf16 blocks) per epilogue warp
 constexpr int kSetCols = 256;                  // tensor-memory columns of one accumulator set
 constexpr int kTmemCols = 512;
 
@@ -68,20 +69,21 @@ struct TcOp {
 
 struct alignas(64) TcProblem {
   CUtensorMap tmA, tmB;
+  // maps of the outputs for the epilogue's bulk stores: fp32 output, term planes, second planes
+  // (out_tma bit 0, 1, 2: the map exists)
+  CUtensorMap tmO, tmP, tmP2;
+  int out_tma;
   TcEpilogue epi;
   int M, N, K, num_kb, kb_per_split, split;
   int bn, tiles_n, tiles_mn, unit_begin, unit_count;
   int bm;                      // rows of one tile: 128, or 256 in the pair form
   int pa, pb, a_mn, b_mn, a_batch_planes, b_batch_planes;
   uint32_t b_tile_bytes, tx_bytes;   // per CTA: in the pair form a CTA stages half of the B tile
-  // layout of a stage and the copies that fill it (operands without a convolution window):
-  //   K-major operand   [plane][rows][64 k]: one box {64, rows, planes} per K block;
-  //   MN-major operand  [64-column group][plane][64 k][64] when one box may span the planes
-  //                     (*_tma_pl = 1), else [plane][group][64 k][64] with a box per plane.
-  uint32_t a_pl_bytes, b_pl_bytes;   // between the planes of an operand inside a stage
-  uint32_t a_h_bytes, b_h_bytes;     // between the 64-column groups of an MN-major operand
+  // Layout of a stage (operands without a convolution window): every operand arrives with ONE
+  // copy per K block.  K-major: [plane][rows][64 k], box {64 k, rows, planes} of the array seen as
+  // (k, row, plane).  MN-major: [plane][64-column group][64 k][64], box {64, 64 k, groups, planes}
+  // of the array seen as (column inside its group, k, group, plane).
   uint32_t a_desc_base, b_desc_base; // descriptor low word without the address (group distance << 16)
-  int a_tma_pl, b_tma_pl;            // copies per 64-column group (or per K-major tile): 1 or the plane count
   int nops, nblocks;
   float* split_partials;
   unsigned int* split_counters;
@@ -103,6 +105,8 @@ struct alignas(64) TcGroupParams {
   int nprob, total_units, stages, pad0;
   uint32_t stage_bytes, pad1;
   uint64_t wait_limit_ns;     // bound of every device-side wait
+  uint32_t epi_stage_off;     // byte offset (from the first stage) of the epilogue's transposition
+  uint32_t pad2;              // buffers, kEpiStageBytes per epilogue warp; 0 = none
   DeviceStatus* st;
   const TcProblem* table;     // program launch: the products live in global memory ...
   unsigned int* done;         // ... and count their finished tiles here (zero at launch)
@@ -243,6 +247,24 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm,
   }
 }
 
+template <bool kPair>
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
+                                            int c0, int c1, int c2, int c3) {
+  if (kPair) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
+        "%4, %5, %6}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+  } else {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, "
+        "%4, %5, %6}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+  }
+}
+
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar,
                                             int c0, int c1, int c2, int c3, int c4) {
   asm volatile(
@@ -319,9 +341,58 @@ __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// write 32 consecutive values as `planes` bf16 term planes (v is left holding the remainder)
+// How an epilogue warp writes its 32 x 32 blocks.  Direct: every lane stores its own row (16-byte
+// stores; a warp instruction then touches 32 different lines, one sector-sized piece each, which the
+// load/store unit works off at about one piece per cycle).  Bulk (`sbuf` != 0): the block is laid
+// into the warp's shared-memory buffer as 32 rows of 64 bytes (32 bf16 or 16 fp32 values) in the
+// 64-byte swizzle of a tensor map (conflict-free 16-byte stores) and one lane hands it to the copy
+// engine (cp.async.bulk.tensor, shared -> global), which writes whole lines and clips rows beyond
+// the product.  The buffer holds two such blocks used in turn: a block is rewritten once the
+// engine has read it, i.e. when at most one later hand-over of this lane is still unread.
+struct EpiOut {
+  uint32_t sbuf = 0;                 // 4 KB, 1024-byte aligned; 0 = direct stores only
+  const CUtensorMap* m_f32 = nullptr;   // fp32 output  (col, row, batch item), blocks of 16 columns
+  const CUtensorMap* m_pl = nullptr;    // term planes  (col, row, plane, batch item), blocks of 32 columns
+  const CUtensorMap* m_pl2 = nullptr;   // second set of term planes
+  int row0 = 0;                      // first row of the warp's block
+  int z = 0;                         // batch item
+  uint32_t half = 0;                 // which 2 KB half the next block takes
+};
+
+__device__ __forceinline__ void bulk_wait_read_all() {
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_wait_read_but_one() {
+  asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() {
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_3d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(tm)),
+               "r"(src), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_store_4d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(tm)),
+               "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// write 32 consecutive values as `planes` bf16 term planes (v is left holding the remainder).
+// Direct (map == nullptr, only lanes with `valid` rows store) or through the copy engine (all
+// lanes of the warp take part; block (col0, eo.row0) of every plane).
 __device__ __forceinline__ void store_planes32(float (&v)[32], __nv_bfloat16* base, int planes,
-                                               int64_t plane_stride, int64_t off) {
+                                               int64_t plane_stride, int64_t off, bool valid,
+                                               const CUtensorMap* map, EpiOut& eo, int col0) {
+  const int lane = threadIdx.x & 31;
   for (int p = 0; p < planes; ++p) {
     uint32_t pk[16];
 #pragma unroll
@@ -332,16 +403,58 @@ __device__ __forceinline__ void store_planes32(float (&v)[32], __nv_bfloat16* ba
       v[2 * i + 1] -= __bfloat162float(b);
       pk[i] = (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
     }
-    uint4* dst = reinterpret_cast<uint4*>(base + (int64_t)p * plane_stride + off);
+    if (map == nullptr) {
+      if (valid) {
+        uint4* dst = reinterpret_cast<uint4*>(base + (int64_t)p * plane_stride + off);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+        for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+      }
+      continue;
+    }
+    // rows of 64 bytes in the 64-byte swizzle: 16-byte piece c of row r sits at c ^ ((r >> 1) & 3)
+    if (lane == 0) bulk_wait_read_but_one();
+    __syncwarp();
+    const uint32_t tile = eo.sbuf + eo.half * 2048u;
+    eo.half ^= 1u;
+    const uint32_t rowp = tile + (uint32_t)lane * 64u;
+    const uint32_t sw = ((uint32_t)lane >> 1) & 3u;
+#pragma unroll
+    for (uint32_t c = 0; c < 4; ++c)
+      st_shared_v4(rowp + ((c ^ sw) << 4), pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) bulk_store_4d(map, tile, col0, eo.row0, p, eo.z);
   }
 }
 
-__device__ __forceinline__ void store_f32x32(const float (&v)[32], float* dst) {
-  float4* d4 = reinterpret_cast<float4*>(dst);
+// 32 consecutive fp32 values of this lane's row: direct (16-byte stores of the lanes with `valid`
+// rows) or through the copy engine (all lanes; block (col0, eo.row0))
+__device__ __forceinline__ void store_f32x32(const float (&v)[32], float* dst, bool valid, EpiOut& eo, int col0) {
+  if (eo.m_f32 == nullptr) {
+    if (valid) {
+      float4* d4 = reinterpret_cast<float4*>(dst);
 #pragma unroll
-  for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+      for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    }
+    return;
+  }
+  const int lane = threadIdx.x & 31;
+  const uint32_t sw = ((uint32_t)lane >> 1) & 3u;
+#pragma unroll
+  for (int hh = 0; hh < 2; ++hh) {       // two blocks of 16 columns: rows of 64 bytes, as for bf16
+    if (lane == 0) bulk_wait_read_but_one();
+    __syncwarp();
+    const uint32_t tile = eo.sbuf + eo.half * 2048u;
+    eo.half ^= 1u;
+    const uint32_t rowp = tile + (uint32_t)lane * 64u;
+#pragma unroll
+    for (uint32_t c = 0; c < 4; ++c)
+      st_shared_v4(rowp + ((c ^ sw) << 4), __float_as_uint(v[16 * hh + 4 * c]), __float_as_uint(v[16 * hh + 4 * c + 1]),
+                   __float_as_uint(v[16 * hh + 4 * c + 2]), __float_as_uint(v[16 * hh + 4 * c + 3]));
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) bulk_store_3d(eo.m_f32, tile, col0 + 16 * hh, eo.row0, eo.z);
+  }
 }
 
 // position in the fragment stream of the first dead unit of (row, 32-column chunk at col0)
@@ -353,73 +466,78 @@ __device__ __forceinline__ uint32_t frag_base(const TcEpilogue& e, int N, int ro
 }
 
 // the fused step applied to one row chunk of 32 accumulator columns
-// (`prow`: the row inside the product, `row`: where its outputs live; they differ under a scatter)
+// (`prow`: the row inside the product, `row`: where its outputs live; they differ under a scatter;
+// `valid`: the row exists.  With bulk output every lane of the warp comes here, rows beyond the
+// product included: they touch no global memory and the copy engine clips their part of a block.)
+// `mword`: the row's sign word of this chunk, fetched ahead of the accumulator (modes that read it)
 __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int prow, int row, int col0,
-                                               float (&v)[32], double& sumsq_local) {
-  const int64_t off = (int64_t)row * (e.ld ? e.ld : (int64_t)N) + col0;
+                                               float (&v)[32], double& sumsq_local, bool valid, EpiOut& eo,
+                                               uint32_t mword) {
+  const int64_t ldo = e.ld ? e.ld : (int64_t)N;
+  const int64_t off = (int64_t)row * ldo + col0;
   const int64_t woff = (int64_t)row * (N >> 5) + (col0 >> 5);
   switch (e.mode) {
     case TC_EPI_PLAIN: {
       if (e.addend) {
-        const float4* a4 = reinterpret_cast<const float4*>(e.addend + off);
+        if (valid) {
+          const float4* a4 = reinterpret_cast<const float4*>(e.addend + off);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float4 a = a4[i];
-          v[4 * i] = fmaf(e.alpha, v[4 * i], a.x);
-          v[4 * i + 1] = fmaf(e.alpha, v[4 * i + 1], a.y);
-          v[4 * i + 2] = fmaf(e.alpha, v[4 * i + 2], a.z);
-          v[4 * i + 3] = fmaf(e.alpha, v[4 * i + 3], a.w);
+          for (int i = 0; i < 8; ++i) {
+            float4 a = a4[i];
+            v[4 * i] = fmaf(e.alpha, v[4 * i], a.x);
+            v[4 * i + 1] = fmaf(e.alpha, v[4 * i + 1], a.y);
+            v[4 * i + 2] = fmaf(e.alpha, v[4 * i + 2], a.z);
+            v[4 * i + 3] = fmaf(e.alpha, v[4 * i + 3], a.w);
+          }
         }
       } else if (e.alpha != 1.f) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] *= e.alpha;
       }
-      if (e.out_f32) store_f32x32(v, e.out_f32 + off);
-      if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off);
+      if (e.out_f32) store_f32x32(v, e.out_f32 + off, valid, eo, col0);
+      if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0);
       break;
     }
     case TC_EPI_RESID: {
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
         v[i] = ((col0 + i) == row ? 1.f : 0.f) - v[i];
-        sumsq_local += (double)v[i] * (double)v[i];
+        if (valid) sumsq_local += (double)v[i] * (double)v[i];
       }
-      if (e.out_f32) store_f32x32(v, e.out_f32 + off);
-      if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off);
+      if (e.out_f32) store_f32x32(v, e.out_f32 + off, valid, eo, col0);
+      if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0);
       break;
     }
     case TC_EPI_FWD: {
-      uint32_t word;
+      uint32_t word = 0xffffffffu;
       if (e.write_mask) {
-        word = 0;
-        if (e.act == MW_ACT_NONE) {
-          word = 0xffffffffu;
-        } else {
+        if (e.act != MW_ACT_NONE) {
+          word = 0;
 #pragma unroll
           for (int i = 0; i < 32; ++i) word |= (v[i] > 0.f ? 1u : 0u) << i;
         }
-        e.mask[woff] = word;
-      } else {
-        word = e.act == MW_ACT_NONE ? 0xffffffffu : e.mask[woff];
+        if (valid) e.mask[woff] = word;
+      } else if (e.act != MW_ACT_NONE && valid) {
+        word = mword;
       }
       const float nf = e.act == MW_ACT_LEAKY_RELU ? e.slope : (e.act == MW_ACT_RELU ? 0.f : 1.f);
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = ((word >> i) & 1u) ? v[i] : nf * v[i];
-      if (e.out_f32) store_f32x32(v, e.out_f32 + off);
-      if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off);
+      if (e.out_f32) store_f32x32(v, e.out_f32 + off, valid, eo, col0);
+      if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0);
       break;
     }
     case TC_EPI_BWD: {
-      if (e.out_f32) store_f32x32(v, e.out_f32 + off);
+      if (e.out_f32) store_f32x32(v, e.out_f32 + off, valid, eo, col0);
       if (e.n_planes2) {   // cotangent checkpoint as term planes (the sweep reads it as an operand)
         float h[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) h[i] = v[i];
         store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2,
-                       e.compact2 ? (int64_t)prow * N + col0 : off);
+                       e.compact2 ? (int64_t)prow * N + col0 : off, valid, eo.m_pl2, eo, col0);
       }
-      const uint32_t word = e.act != MW_ACT_NONE ? e.mask[woff] : 0xffffffffu;
-      if (e.act == MW_ACT_RELU && e.frag_vals) {
+      const uint32_t word = (e.act != MW_ACT_NONE && valid) ? mword : 0xffffffffu;
+      if (e.act == MW_ACT_RELU && e.frag_vals && valid) {
         // fragments: the cotangent at dead units, in column order
         uint32_t pos = frag_base(e, N, row, col0, woff);
 #pragma unroll
@@ -432,12 +550,12 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = ((word >> i) & 1u) ? v[i] : nf * v[i];
         }
-        store_planes32(v, e.planes, e.n_planes, e.plane_stride, off);
+        store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0);
       }
       break;
     }
     case TC_EPI_VIJP: {
-      if (e.addend) {
+      if (e.addend && valid) {
         const float4* a4 = reinterpret_cast<const float4*>(e.addend + off);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -450,7 +568,7 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
       }
       float h[32];
       if (e.act == MW_ACT_LEAKY_RELU) {
-        const uint32_t word = e.mask[woff];
+        const uint32_t word = valid ? mword : 0xffffffffu;
         // one division per chunk: the inverse derivative is applied as a product with the
         // correctly rounded reciprocal of the slope (within an ulp of the quotient)
         const float rs = 1.f / e.slope;
@@ -459,8 +577,8 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
       } else if (e.act == MW_ACT_RELU) {
         // live units pass g_z on (phi' = 1); dead units take their stored cotangent back and
         // contribute nothing to the weight vjp
-        const uint32_t word = e.mask[woff];
-        uint32_t pos = frag_base(e, N, row, col0, woff);
+        const uint32_t word = valid ? mword : 0xffffffffu;
+        uint32_t pos = valid ? frag_base(e, N, row, col0, woff) : 0u;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           if ((word >> i) & 1u) {
@@ -474,22 +592,22 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
 #pragma unroll
         for (int i = 0; i < 32; ++i) h[i] = v[i];
       }
-      if (e.out_f32) store_f32x32(h, e.out_f32 + off);
+      if (e.out_f32) store_f32x32(h, e.out_f32 + off, valid, eo, col0);
       if (e.n_planes2) {
         if (e.sub2_s) {
           const int hw = e.sub2_h * e.sub2_w;
           const int b = prow / hw, rem = prow - b * hw;
           const int y = rem / e.sub2_w, x = rem - y * e.sub2_w;
-          if (y % e.sub2_s == 0 && x % e.sub2_s == 0) {
+          if (valid && y % e.sub2_s == 0 && x % e.sub2_s == 0) {
             const int64_t r2 = ((int64_t)b * (e.sub2_h / e.sub2_s) + y / e.sub2_s) * (e.sub2_w / e.sub2_s) +
                                x / e.sub2_s;
-            store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, r2 * N + col0);
+            store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, r2 * N + col0, true, nullptr, eo, col0);
           }
         } else {
-          store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, off);
+          store_planes32(h, e.planes2, e.n_planes2, e.plane_stride2, off, valid, eo.m_pl2, eo, col0);
         }
       }
-      if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off);
+      if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0);
       break;
     }
     default:
@@ -744,9 +862,6 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           // barrier of the NEXT stage is polled while this stage's copies are being issued.
           const CUtensorMap* tmA = &P.tmA;
           const CUtensorMap* tmB = &P.tmB;
-          const uint32_t a_pl_bytes = P.a_pl_bytes, a_h_bytes = P.a_h_bytes;
-          const uint32_t b_pl_bytes = P.b_pl_bytes, b_h_bytes = P.b_h_bytes;
-          const int a_loops = P.a_tma_pl, b_loops = P.b_tma_pl;
           const uint32_t b_off = (uint32_t)pa * kATileBytes;
           const uint32_t txe = kPair ? 2u * tx : tx;
           const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
@@ -760,24 +875,10 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
             if (!ready && !mbar_wait<kPair>(empty0 + 8u * stage, phase ^ 1u, wc, 1u)) { ok = false; break; }
             if (!kPair || rank == 0) mbar_expect_tx(full0 + 8u * stage, txe);
             const uint32_t fb = full0_remote + 8u * stage;
-            for (int pl = 0; pl < a_loops; ++pl) {
-              const uint32_t dst = sbase + (uint32_t)pl * a_pl_bytes;
-              if (a_mn) {
-                tma_load_3d<kPair>(dst, tmA, fb, am0, k0, a_pl0 + pl);
-                tma_load_3d<kPair>(dst + a_h_bytes, tmA, fb, am0 + 64, k0, a_pl0 + pl);
-              } else {
-                tma_load_3d<kPair>(dst, tmA, fb, k0, am0, a_pl0 + pl);
-              }
-            }
-            for (int pl = 0; pl < b_loops; ++pl) {
-              const uint32_t dst = sbase + b_off + (uint32_t)pl * b_pl_bytes;
-              if (b_mn) {
-                for (int h = 0; h < nbox; ++h)
-                  tma_load_3d<kPair>(dst + (uint32_t)h * b_h_bytes, tmB, fb, bn_first + h * 64, k0, b_pl0 + pl);
-              } else {
-                tma_load_3d<kPair>(dst, tmB, fb, k0, bn_first, b_pl0 + pl);
-              }
-            }
+            if (a_mn) tma_load_4d<kPair>(sbase, tmA, fb, 0, k0, am0 >> 6, a_pl0);
+            else tma_load_3d<kPair>(sbase, tmA, fb, k0, am0, a_pl0);
+            if (b_mn) tma_load_4d<kPair>(sbase + b_off, tmB, fb, 0, k0, bn_first >> 6, b_pl0);
+            else tma_load_3d<kPair>(sbase + b_off, tmB, fb, k0, bn_first, b_pl0);
             sbase += stage_bytes;
             if (++stage == stages) { stage = 0; phase ^= 1u; sbase = tiles; }
             ready = mbar_try_wait<kPair>(empty0 + 8u * stage, phase ^ 1u);
@@ -874,6 +975,9 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     // ---------------- epilogue (warps 2..5) ----------------
     const int quarter = warp & 3;                 // tensor-memory lane quarter this warp may read
     const int half = 0;
+    // this warp's buffer for bulk stores (0: none, direct stores)
+    const uint32_t epi_sbuf = p.epi_stage_off ? tiles + p.epi_stage_off + (uint32_t)quarter * kEpiStageBytes : 0u;
+    bool bulk_used = false;
     int j = 0, q = 0, rr = 0;
     bool ok = true;
     // sign words, addends, fragments read here and everything stored here may be in use by the
@@ -887,11 +991,6 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       decode_unit(probs, ub, nprob, u, q, w);
       const TcProblem& P = probs[w.q];
       const uint32_t set = (uint32_t)j & 1u, aphase = ((uint32_t)j >> 1) & 1u;
-      // every lane observes the barrier itself; the warp then takes one common decision so the
-      // warp-wide tensor-memory loads below are never executed by part of a warp
-      ok = __all_sync(0xffffffffu, mbar_wait<kPair>(smem_u32(&acc_full[set]), aphase, wc, 4u));
-      if (!ok) break;
-      tc_fence_after();
       // pair form: this CTA's tensor memory holds rows rank*128 .. rank*128+127 of the tile
       const int row = w.m0 + (kPair ? (int)rank * BM : 0) + quarter * 32 + lane;
       const int bn = P.bn, nblk = P.nblocks, N = P.N;
@@ -913,7 +1012,40 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         if (epi.mask) epi.mask += z * epi.bs_mask;
         if (epi.sumsq) epi.sumsq += z * epi.bs_sumsq;
       }
+      // The row's sign words of this tile are fetched now, while the products are still running:
+      // read inside the chunk loop, each would put a trip to global memory on the epilogue's
+      // critical path.  (Sign words are never written by the launch that reads them.)
+      uint32_t mw[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) mw[i] = 0xffffffffu;
+      if (epi.mask && epi.act != MW_ACT_NONE && row < P.M &&
+          ((epi.mode == TC_EPI_FWD && !epi.write_mask) || epi.mode == TC_EPI_BWD || epi.mode == TC_EPI_VIJP)) {
+        const uint32_t* mrow = epi.mask + (int64_t)orow * (N >> 5) + (w.n0 >> 5);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (32 * i < bn && w.n0 + 32 * i < N) mw[i] = mrow[i];
+      }
+      // every lane observes the barrier itself; the warp then takes one common decision so the
+      // warp-wide tensor-memory loads below are never executed by part of a warp
+      ok = __all_sync(0xffffffffu, mbar_wait<kPair>(smem_u32(&acc_full[set]), aphase, wc, 4u));
+      if (!ok) break;
+      tc_fence_after();
       double sumsq_local = 0.0;
+      EpiOut eo;
+      if (epi_sbuf && P.out_tma) {
+        // the copy engine must have read what the previous unit left in the buffer
+        if (bulk_used) {
+          if (lane == 0) bulk_wait_read_all();
+          __syncwarp();
+        }
+        bulk_used = true;
+        eo.sbuf = epi_sbuf;
+        eo.m_f32 = (P.out_tma & 1) ? &P.tmO : nullptr;
+        eo.m_pl = (P.out_tma & 2) ? &P.tmP : nullptr;
+        eo.m_pl2 = (P.out_tma & 4) ? &P.tmP2 : nullptr;
+        eo.row0 = row - lane;
+        eo.z = w.z;
+      }
       const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + set * (uint32_t)kSetCols;
       // sum of the column blocks of 32 accumulator columns starting at c
       auto load_chunk = [&](int c, float (&v)[32]) {
@@ -997,7 +1129,12 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
           } else {
             load_chunk(c, v);
           }
-          if (row < P.M) epilogue_chunk(epi, N, row, orow, w.n0 + c, v, sumsq_local);
+          if (row < P.M || eo.sbuf) {
+            const int ci = c >> 5;      // the chunk's sign word, by selection (no indexed registers)
+            const uint32_t lo = ci & 2 ? (ci & 1 ? mw[3] : mw[2]) : (ci & 1 ? mw[1] : mw[0]);
+            const uint32_t hi = ci & 2 ? (ci & 1 ? mw[7] : mw[6]) : (ci & 1 ? mw[5] : mw[4]);
+            epilogue_chunk(epi, N, row, orow, w.n0 + c, v, sumsq_local, row < P.M, eo, ci & 4 ? hi : lo);
+          }
         }
       }
       // this warp has read its part of the accumulator set: hand it back to the MMA issuer
@@ -1016,6 +1153,11 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       }
       if (kProgram && fused_step) {
         // program launch: publish this warp's part of the tile to the products that wait for it
+        // (bulk stores must have been written, not just read from the buffer)
+        if (eo.sbuf) {
+          if (lane == 0) bulk_wait_all();
+          __syncwarp();
+        }
         __threadfence();
         __syncwarp();
         if (lane == 0) {
@@ -1025,6 +1167,8 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       }
     }
   }
+  // bulk stores of this thread complete before the CTA retires
+  if (warp >= 2 && lane == 0) bulk_wait_all();
   tc_fence_before();
   __syncthreads();
   if (warp == 0 && lane == 0 && abort_flag) {
@@ -1096,6 +1240,8 @@ int pick_bn(int pa, int pb, int M, int N, int batch, bool wide = false) {
 
 // 0: never use the pair form, 1: wherever a launch qualifies (default)
 int g_pair_mode = 1;
+// 1: epilogues hand plain outputs to the copy engine (0: per-lane stores everywhere)
+int g_bulk_epilogue = 1;
 
 // Can this product run in the pair form?  Operands of at most two terms (the accumulator blocks
 // of a 128-column tile then fit one set), tiles at least 128 columns wide (each CTA stages whole
@@ -1205,6 +1351,83 @@ static mw_status get_map(TcMapCache* cache, const TcOperand& op, int box_rows, i
   return MW_OK;
 }
 
+// MN-major operand [rows = K][cols] per plane, seen as (column inside its group of 64, k, group,
+// plane): one box {64, 64, groups, planes} lands as [plane][group][64 k][64], the layout the
+// product's operand descriptors expect (groups 8 KB apart)
+static mw_status get_map_mn(TcMapCache* cache, const TcOperand& op, int groups, int total_planes,
+                            int box_planes, CUtensorMap* out) {
+  const int64_t ld = op.ld ? op.ld : op.cols;
+  auto key = std::make_tuple(op.base, op.rows, op.cols, total_planes, op.plane_stride,
+                             ((int64_t)1 << 61) + groups + ((int64_t)box_planes << 10) + (ld << 12));
+  if (cache) {
+    auto it = cache->maps.find(key);
+    if (it != cache->maps.end()) { *out = it->second; return MW_OK; }
+  }
+  auto fn = encode_fn();
+  if (!fn) return MW_ERR_CUDA;
+  if (((uintptr_t)op.base & 15u) || (op.cols % 64) != 0 || (ld % 8) != 0 || ld < op.cols) return MW_ERR_INVALID_ARG;
+  const int64_t ps = total_planes > 1 ? op.plane_stride : (int64_t)op.rows * ld;
+  if (ps % 8 != 0) return MW_ERR_INVALID_ARG;
+  cuuint64_t dims[4] = {64u, (cuuint64_t)op.rows, (cuuint64_t)(op.cols / 64), (cuuint64_t)total_planes};
+  cuuint64_t strides[3] = {(cuuint64_t)ld * 2, 128u, (cuuint64_t)ps * 2};
+  cuuint32_t box[4] = {64u, 64u, (cuuint32_t)groups, (cuuint32_t)box_planes};
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(op.base), dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return MW_ERR_CUDA;
+  if (cache) cache->maps[key] = *out;
+  return MW_OK;
+}
+
+// Output of a product for the epilogue's bulk stores: [rows][cols] with `ld` elements between rows,
+// `planes` of them `plane_stride` apart, `batch` items `batch_stride` apart; blocks of 32 rows of 64
+// bytes (32 bf16 or 16 fp32 columns) in the 64-byte swizzle, which makes the epilogue's 16-byte
+// shared-memory stores conflict-free.  Returns false when the array does not qualify.
+static bool get_out_map(TcMapCache* cache, const void* base, bool f32, int rows, int cols, int64_t ld,
+                        int planes, int64_t plane_stride, int batch, int64_t batch_stride, CUtensorMap* out) {
+  const int64_t es = f32 ? 4 : 2;
+  if (!base || ((uintptr_t)base & 15u) || cols % 32 != 0 || (ld * es) % 16 != 0 || ld < cols) return false;
+  if (planes < 1) planes = 1;
+  if (batch < 1) batch = 1;
+  if (planes > 1 && ((plane_stride * es) % 16 != 0 || plane_stride <= 0)) return false;
+  if (batch > 1 && ((batch_stride * es) % 16 != 0 || batch_stride <= 0)) return false;
+  auto key = std::make_tuple(base, rows, cols, planes * 4096 + batch, plane_stride,
+                             ((int64_t)1 << 60) + (f32 ? 1 : 0) + (ld << 4) + (batch_stride << 34));
+  if (cache) {
+    auto it = cache->maps.find(key);
+    if (it != cache->maps.end()) { *out = it->second; return true; }
+  }
+  auto fn = encode_fn();
+  if (!fn) return false;
+  // strides of dimensions of extent 1 are never used but must be valid
+  const int64_t s_row = ld * es;
+  const int64_t s_pl = planes > 1 ? plane_stride * es : s_row * rows;
+  const int64_t s_b = batch > 1 ? batch_stride * es : s_pl * planes;
+  CUresult r;
+  if (f32) {
+    if (planes != 1) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)batch};
+    cuuint64_t strides[2] = {(cuuint64_t)s_row, (cuuint64_t)s_b};
+    cuuint32_t box[3] = {16u, 32u, 1u};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    cuuint64_t dims[4] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)planes, (cuuint64_t)batch};
+    cuuint64_t strides[3] = {(cuuint64_t)s_row, (cuuint64_t)s_pl, (cuuint64_t)s_b};
+    cuuint32_t box[4] = {32u, 32u, 1u, 1u};
+    cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
+  if (r != CUDA_SUCCESS) return false;
+  if (cache) cache->maps[key] = *out;
+  return true;
+}
+
 // channel-last pixel array [images][H][W][C] per plane, read in boxes of 64 channels of bx x by
 // pixels (every `stride`-th one in both directions) of bi images
 static mw_status get_map_conv(TcMapCache* cache, const TcOperand& op, int H, int W, int bx, int by,
@@ -1259,8 +1482,8 @@ double build_ops_pair(TcProblem& P) {
     for (int j = 0; j < pb; ++j) {
       if (i + j >= t) continue;
       TcOp& o = P.ops[n++];
-      o.a_off16 = ((uint32_t)i * P.a_pl_bytes) >> 4;
-      o.b_off16 = (b0 + (uint32_t)j * P.b_pl_bytes) >> 4;
+      o.a_off16 = ((uint32_t)i * kATileBytes) >> 4;
+      o.b_off16 = (b0 + (uint32_t)j * P.b_tile_bytes) >> 4;
       o.idesc = make_idesc(P.a_mn != 0, P.b_mn != 0, bn, 2 * BM);
       o.dcol = (uint16_t)((i + j) * bn);
       o.rot = 0;
@@ -1287,8 +1510,8 @@ double build_ops(TcProblem& P, bool rotate) {
   double cycles = 0.0;
   auto add = [&](int i, int j0, int cnt, int rot, int first) {
     TcOp& o = P.ops[n++];
-    o.a_off16 = ((uint32_t)i * P.a_pl_bytes) >> 4;
-    o.b_off16 = (b0 + (uint32_t)j0 * P.b_pl_bytes) >> 4;
+    o.a_off16 = ((uint32_t)i * kATileBytes) >> 4;
+    o.b_off16 = (b0 + (uint32_t)j0 * P.b_tile_bytes) >> 4;
     o.idesc = make_idesc(P.a_mn != 0, P.b_mn != 0, cnt * bn);
     o.dcol = (uint16_t)col(i + j0);
     o.rot = (uint16_t)rot;
@@ -1405,18 +1628,8 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   const int b_cols = pair ? P.bn / 2 : P.bn;     // columns of the B tile one CTA stages
   P.b_tile_bytes = (uint32_t)b_cols * BK * 2;
   P.tx_bytes = (uint32_t)P.pa * kATileBytes + (uint32_t)P.pb * P.b_tile_bytes;
-  // stage layout and copies (see TcProblem).  Convolution windows keep a box per plane.
-  const bool plain = cv.mode == TC_CONV_NONE;
-  P.a_tma_pl = plain ? 1 : P.pa;
-  P.a_h_bytes = (P.a_mn && plain) ? (uint32_t)P.pa * 8192u : 8192u;
-  P.a_pl_bytes = (P.a_mn && plain) ? 8192u : kATileBytes;
-  // an instruction that spans several B planes (single form) needs each plane's groups adjacent
-  const bool b_span = plain && (!P.b_mn || pair || P.pb == 1);
-  P.b_tma_pl = b_span ? 1 : P.pb;
-  P.b_h_bytes = (P.b_mn && b_span) ? (uint32_t)P.pb * 8192u : 8192u;
-  P.b_pl_bytes = (P.b_mn && b_span) ? 8192u : P.b_tile_bytes;
-  P.a_desc_base = (P.a_mn ? (P.a_h_bytes >> 4) : 1u) << 16;
-  P.b_desc_base = (P.b_mn ? (P.b_h_bytes >> 4) : 1u) << 16;
+  P.a_desc_base = (P.a_mn ? (8192u >> 4) : 1u) << 16;
+  P.b_desc_base = (P.b_mn ? (8192u >> 4) : 1u) << 16;
   const int t = P.pa > P.pb ? P.pa : P.pb;
   // fp32-accurate products alternate the leading block (needs two K blocks per unit)
   const bool rotate = t == 3 && P.pa == 3 && P.pb == 3 && P.kb_per_split >= 2 &&
@@ -1424,6 +1637,21 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   const double kb_cycles = pair ? build_ops_pair(P) : build_ops(P, rotate);
   *unit_cost = kb_cycles * P.kb_per_split;
   P.epi = d.epi;
+  // bulk stores for outputs that are plain [M][N] arrays (no row scatter, no sub-sampling)
+  P.out_tma = 0;
+  if (g_bulk_epilogue && d.epi.remap_s == 0) {
+    const TcEpilogue& e = d.epi;
+    const int64_t ldo = e.ld ? e.ld : (int64_t)d.N;
+    if (e.out_f32 && get_out_map(cache, e.out_f32, true, d.M, d.N, ldo, 1, 0, d.batch, e.bs_f32, &P.tmO))
+      P.out_tma |= 1;
+    if (e.n_planes && get_out_map(cache, e.planes, false, d.M, d.N, ldo, e.n_planes, e.plane_stride, d.batch,
+                                  e.bs_planes, &P.tmP))
+      P.out_tma |= 2;
+    if (e.n_planes2 && !e.compact2 && !e.sub2_s &&
+        get_out_map(cache, e.planes2, false, d.M, d.N, ldo, e.n_planes2, e.plane_stride2, d.batch, e.bs_planes2,
+                    &P.tmP2))
+      P.out_tma |= 4;
+  }
   P.split_partials = nullptr;
   P.split_counters = nullptr;
   if (split > 1) {
@@ -1442,8 +1670,11 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
     MW_TRY(get_map_conv(cache, d.A, cv.H, cv.W, cbx, cby, cbi, cv.stride, d.A.planes, &P.tmA));
     MW_TRY(get_map(cache, d.B, 64, d.B.planes, &P.tmB));
   } else {
-    MW_TRY(get_map(cache, d.A, d.A.mn_major ? 64 : BM, a_total, &P.tmA, P.pa));
-    MW_TRY(get_map(cache, d.B, d.B.mn_major ? 64 : b_cols, b_total, &P.tmB, b_span ? P.pb : 1));
+    // one box per operand and K block, spanning its planes (and, MN-major, its column groups)
+    if (d.A.mn_major) MW_TRY(get_map_mn(cache, d.A, BM / 64, a_total, P.pa, &P.tmA));
+    else MW_TRY(get_map(cache, d.A, BM, a_total, &P.tmA, P.pa));
+    if (d.B.mn_major) MW_TRY(get_map_mn(cache, d.B, b_cols / 64, b_total, P.pb, &P.tmB));
+    else MW_TRY(get_map(cache, d.B, b_cols, b_total, &P.tmB, P.pb));
   }
   int np = 0;
   for (int a = 0; a < P.pa; ++a)
@@ -1460,12 +1691,23 @@ static int stages_for(uint32_t stage_bytes) {
   return stages > kMaxStages ? kMaxStages : stages;
 }
 
+constexpr int kMaxDynamicSmem = 227 * 1024 - 6144;
+
+// the epilogue's transposition buffers go behind the stages when the ring leaves room for them
+static uint32_t epi_stage_offset(int stages, uint32_t stage_bytes, size_t* smem) {
+  const size_t need = (size_t)kEpiWarps * kEpiStageBytes;
+  if (*smem + need > (size_t)kMaxDynamicSmem) return 0;
+  const uint32_t off = (uint32_t)stages * stage_bytes;
+  *smem += need;
+  return off;
+}
+
 // the opt-in to large dynamic shared memory belongs to the device: once per device and kernel
 static mw_status ensure_kernel_attr() {
   static bool attr_set[kMaxDevices] = {};
   const int dev = current_device();
   if (!attr_set[dev]) {
-    const int bytes = 227 * 1024 - 6144;
+    const int bytes = kMaxDynamicSmem;
     MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
     MW_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
@@ -1583,7 +1825,8 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
   const int stages = stages_for(stage_bytes);
   if (stages < 2) return MW_ERR_UNSUPPORTED;
   prm.stages = stages;
-  const size_t smem = (size_t)stages * stage_bytes + 1024;
+  size_t smem = (size_t)stages * stage_bytes + 1024;
+  prm.epi_stage_off = epi_stage_offset(stages, stage_bytes, &smem);
   const bool prof = g_prof.on;
   if (prof) {
     cudaEventRecord(prof_event(), s);
@@ -1699,7 +1942,8 @@ mw_status tc_program_launch(TcProgram* pr, DeviceStatus* st, cudaStream_t s) {
   const int stages = stages_for(pr->stage_bytes);
   if (stages < 2) return MW_ERR_UNSUPPORTED;
   prm.stages = stages;
-  const size_t smem = (size_t)stages * pr->stage_bytes + 1024;
+  size_t smem = (size_t)stages * pr->stage_bytes + 1024;
+  prm.epi_stage_off = epi_stage_offset(stages, pr->stage_bytes, &smem);
   MW_TRY(ensure_kernel_attr());
   const bool prof = g_prof.on;
   if (prof) {
