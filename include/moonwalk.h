@@ -90,7 +90,18 @@ typedef struct {
   int32_t resident_inverse;/* 1: mw_input_cotangent computes every layer's W^-1 (and split
                               operands) once and keeps them in the workspace; 0: the sweep
                               builds them layer by layer in a transient slot (lean memory) */
-  int32_t reserved;        /* must be 0                                                      */
+  int32_t warm_inverse;    /* 1 (dense nets on the tensor cores with resident_inverse = 1): the
+                              workspace keeps every W^-1 from one mw_input_cotangent to the next,
+                              and a call on the same workspace REFRESHES them with the last step
+                              of the Newton-Schulz schedule instead of computing them from
+                              scratch.  For loops whose steps move the weights very little
+                              (fine tuning, small learning rates): the kept inverse X must
+                              still satisfy ||I - W X||_F <= 5e-4 (MW_F32) / 4e-3 (bf16) for
+                              the new W -- roughly ||delta W||_F below that -- which the call
+                              checks per layer (MW_ERR_NOT_SUBMERSIVE through
+                              mw_last_device_status; after that report the next call starts
+                              from scratch again).  The workspace must be left alone between
+                              steps.  0: every call computes the inverses from scratch.        */
   int32_t frag_block;      /* MW_CONV1D nets: Phase II keeps the output cotangent of every
                               convolution at the first k - 1 positions of each block of this
                               many positions (2..64, dividing W); Phase III rebuilds the rest  */

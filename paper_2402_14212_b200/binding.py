@@ -44,7 +44,7 @@ class NetOpts(C.Structure):
     _fields_ = [("prec", C.c_int32), ("loss", C.c_int32), ("reseed_every", C.c_int32),
                 ("conv_vijp_iters", C.c_int32), ("backend", C.c_int32),
                 ("inverse_iters", C.c_int32), ("resident_inverse", C.c_int32),
-                ("reserved", C.c_int32), ("frag_block", C.c_int32)]
+                ("warm_inverse", C.c_int32), ("frag_block", C.c_int32)]
 
 
 _lib = None
@@ -129,14 +129,14 @@ class Net:
 
     def __init__(self, layers, batch: int, prec: str, loss: str, reseed_every: int = 4,
                  conv_vijp_iters: int = 10, backend: str = "auto", inverse_iters: int = 0,
-                 resident_inverse: bool = True, frag_block: int = 0):
+                 resident_inverse: bool = True, frag_block: int = 0, warm_inverse: bool = False):
         self.layers = list(layers)
         self.batch = int(batch)
         self.prec, self.loss = prec, loss
         self._h = C.c_void_p()
         opts = NetOpts(PREC[prec], LOSS[loss], int(reseed_every), int(conv_vijp_iters),
-                       BACKEND[backend], int(inverse_iters), int(bool(resident_inverse)), 0,
-                       int(frag_block))
+                       BACKEND[backend], int(inverse_iters), int(bool(resident_inverse)),
+                       int(bool(warm_inverse)), int(frag_block))
         descs = make_layer_descs(self.layers)
         _check(lib().mw_net_create(descs, len(self.layers), self.batch, C.byref(opts),
                                    C.byref(self._h)), "mw_net_create")
@@ -401,8 +401,8 @@ def to_device(problem, device="cuda"):
     return params, x, target
 
 
-def net_for(problem, backend="auto", resident_inverse=True, inverse_iters=0) -> Net:
+def net_for(problem, backend="auto", resident_inverse=True, inverse_iters=0, warm_inverse=False) -> Net:
     return Net(problem.layers, problem.batch, problem.prec, problem.loss,
                reseed_every=problem.reseed_every, conv_vijp_iters=problem.conv_vijp_iters,
                backend=backend, inverse_iters=inverse_iters, resident_inverse=resident_inverse,
-               frag_block=getattr(problem, "frag_block", 0))
+               frag_block=getattr(problem, "frag_block", 0), warm_inverse=warm_inverse)

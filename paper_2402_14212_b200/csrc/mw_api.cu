@@ -159,7 +159,7 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
   if (opts->reseed_every < 0 || opts->conv_vijp_iters < 0 || opts->inverse_iters < 0 || opts->frag_block < 0)
     return MW_ERR_INVALID_ARG;
   if (opts->backend < MW_BACKEND_AUTO || opts->backend > MW_BACKEND_TENSOR) return MW_ERR_INVALID_ARG;
-  if (opts->reserved != 0) return MW_ERR_INVALID_ARG;
+  if (opts->warm_inverse != 0 && opts->warm_inverse != 1) return MW_ERR_INVALID_ARG;
   for (int l = 0; l < n_layers; ++l) {
     if (layers[l].kind < MW_DENSE || layers[l].kind > MW_CONV1D) return MW_ERR_INVALID_ARG;
     if (!valid_layer(layers[l], l, n_layers)) return MW_ERR_UNSUPPORTED;
@@ -580,6 +580,7 @@ extern "C" mw_status mw_backprop_reference(mw_net* net, const void* const* param
   MW_TRY(check_ws(workspace, workspace_bytes, net->bpl.total));
   cudaStream_t s = (cudaStream_t)stream;
   if (net->ws_done == workspace) net->ws_done = nullptr;  // the stores are overwritten
+  if (net->warm_ws == workspace) net->warm_ws = nullptr;
   if (net->backend == MW_BACKEND_TENSOR)
     return tensor_backprop(net, params, x, loss_target, dW_out, loss_out, workspace, s);
   if (net->opts.prec == MW_F64)
@@ -615,6 +616,8 @@ extern "C" mw_status mw_last_device_status(const mw_net* net, void* workspace, v
   MW_CUDA_OK(cudaStreamSynchronize(s));
   if (detail) std::memcpy(detail, host.detail, sizeof(host.detail));
   if (host.code != 0) {
+    // whatever failed, inverses kept in this workspace are no longer trusted
+    if (net->warm_ws == workspace) const_cast<mw_net*>(net)->warm_ws = nullptr;
     MW_CUDA_OK(cudaMemsetAsync(workspace, 0, sizeof(DeviceStatus), s));
     MW_CUDA_OK(cudaStreamSynchronize(s));
   }

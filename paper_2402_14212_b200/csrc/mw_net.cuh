@@ -56,6 +56,11 @@ struct mw_net {
   const void* x_done = nullptr;
   void* tc = nullptr;              // tensor-core backend private state
   bool lean_seed = false;          // the net can keep the sweep's seed itself (g0 optional)
+  // warm_inverse nets: the workspace whose kept inverses the next mw_input_cotangent may refresh
+  // (nullptr: none, the next call computes them from scratch), and which of the two homes of the
+  // Newton-Schulz iterate holds the current inverse
+  const void* warm_ws = nullptr;
+  int inv_side = 0;
   // mw_forward_sweep_apply in progress: the weight vjp's epilogue writes theta - apply_lr * g
   // (theta = apply_params[l]) instead of g
   const void* const* apply_params = nullptr;

@@ -9,13 +9,17 @@ struct TcMapCache;
 struct TcProgram;
 // programs (whole phases in one launch) are rebuilt only when a buffer they name has moved
 enum { MW_PROG_PHASE1 = 0, MW_PROG_PHASE2, MW_PROG_BP_FWD, MW_PROG_BP_BWD, MW_PROG_COUNT };
+// variants of a program: which home of the Newton-Schulz iterate it starts from (0, 1), cold or
+// refreshing (+2).  A training loop alternates between two of them; each is built once.
+constexpr int kProgVariants = 4;
 struct TensorState {
   TcMapCache* cache = nullptr;
-  TcProgram* prog[MW_PROG_COUNT] = {};
-  std::vector<const void*> key[MW_PROG_COUNT];
+  TcProgram* prog[MW_PROG_COUNT][kProgVariants] = {};
+  std::vector<const void*> key[MW_PROG_COUNT][kProgVariants];
   // the forward sweep as chained programs, one per run of layers that fits a product table
-  std::vector<TcProgram*> sweep;
-  std::vector<const void*> sweep_key;
+  // (two variants: the inverses' current home)
+  std::vector<TcProgram*> sweep[2];
+  std::vector<const void*> sweep_key[2];
 };
 
 // convolutional nets on the tensor cores (mw_conv_pipeline.cu): stride-1 same-size convolutions

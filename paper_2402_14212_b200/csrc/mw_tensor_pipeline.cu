@@ -146,10 +146,12 @@ split_weights_kernel(PtrBatch Ws, int64_t n4, int64_t n2, __nv_bfloat16* __restr
 
 // One CTA per matrix: adds the `slots` pieces of ||I - W X||_F^2 that the residual product's
 // epilogue warps left (always in the same order, so the decision does not depend on scheduling)
-// and reports the layer when the rms singular value of the residual exceeds `limit`.
+// and reports the layer when the rms singular value of the residual exceeds `limit` (whole =
+// 1: when its Frobenius norm does, which bounds the LARGEST singular value: a refreshed inverse
+// follows a training step, whose change of W is far from spread evenly over the directions).
 __global__ void __launch_bounds__(256)
 residual_gate_kernel(const double* __restrict__ pieces, int64_t stride, int64_t slots, int n,
-                     double limit, DeviceStatus* st, int layer0) {
+                     double limit, DeviceStatus* st, int layer0, int whole = 0) {
   __shared__ double red[256];
   const double* mine = pieces + (int64_t)blockIdx.x * stride;
   double a = 0.0;
@@ -161,9 +163,10 @@ residual_gate_kernel(const double* __restrict__ pieces, int64_t stride, int64_t 
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    const double r = sqrt(red[0] / (double)n);   // rms singular value of I - W X
+    const double r = sqrt(whole ? red[0] : red[0] / (double)n);   // rms (or root sum) of the singular values of I - W X
     if (!(r <= limit))
-      record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)(layer0 + blockIdx.x), __float_as_uint((float)r), 3u, 0u);
+      record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)(layer0 + blockIdx.x), __float_as_uint((float)r),
+                   whole ? 4u : 3u, 0u);
   }
 }
 
@@ -490,10 +493,11 @@ mw_status ns_prepare_all(const Ctx& c, const void* const* params, const NsStep* 
 }
 
 // product `stage` of layer l: even = residual R = I - W X of step stage/2, odd = its update
+// (the iterate alternates between its two homes Xp[0], Xp[1]; step `it` reads home side0 + it)
 TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, const NsStep* sched,
-                  int steps) {
+                  int steps, int side0) {
   const Layout& lay = *c.lay;
-  const int d = c.dim, it = stage >> 1, cur = it & 1;
+  const int d = c.dim, it = stage >> 1, cur = (side0 + it) & 1;
   const bool last = it + 1 == steps;
   const NsBuffers nb = ns_buffers(c);
   float* X = nb.X + (int64_t)l * c.nn;
@@ -519,8 +523,9 @@ TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, con
     g.B = operand(Rp, d, d, sched[it].pu, true);
     g.epi.mode = TC_EPI_PLAIN;
     g.epi.addend = X;
-    g.epi.out_f32 = last ? nullptr : X;
-    g.epi.planes = last ? c.at<__nv_bfloat16>(lay.inv[l]) : Xn;
+    // the last iterate stays in fp32 too where the next call may refresh it
+    g.epi.out_f32 = (last && !c.n->opts.warm_inverse) ? nullptr : X;
+    g.epi.planes = Xn;         // the last step leaves W^-1 here: the sweep reads it in place
     g.epi.n_planes = next_terms;
     g.epi.plane_stride = c.nn;
   }
@@ -533,13 +538,22 @@ struct NsFeed {
   const void* const* params;
   NsStep sched[16];
   int steps = 0, total = 0, next = 0, per_slot = 0;
+  int side0 = 0;              // home of the iterate the first step reads
+  int variant = 0;            // of the programs that carry this feed (see kProgVariants)
   std::vector<int> last;      // last product of each layer's chain inside the current program
 };
 
-NsFeed make_feed(const Ctx& c, const void* const* params) {
+// warm: only the last step of the schedule, from the inverse the workspace kept (home `side0`)
+NsFeed make_feed(const Ctx& c, const void* const* params, bool warm, int side0) {
   NsFeed f;
   f.params = params;
   f.steps = ns_schedule(c.n, f.sched);
+  if (warm && f.steps > 1) {
+    f.sched[0] = f.sched[f.steps - 1];
+    f.steps = 1;
+  }
+  f.side0 = side0 & 1;
+  f.variant = (warm ? 2 : 0) + f.side0;
   f.total = f.steps > 0 ? 2 * f.steps * c.n->L : 0;
   f.per_slot = (f.total + 2 * c.n->L - 1) / (2 * c.n->L);
   f.last.assign(c.n->L, -1);
@@ -554,9 +568,9 @@ bool use_programs(const mw_net* n) {
 
 TensorState* state_of(const Ctx& c) { return static_cast<TensorState*>(c.n->tc); }
 
-bool program_ready(const Ctx& c, int idx, const std::vector<const void*>& key) {
+bool program_ready(const Ctx& c, int idx, const std::vector<const void*>& key, int variant = 0) {
   TensorState* t = state_of(c);
-  return t->prog[idx] != nullptr && !t->key[idx].empty() && t->key[idx] == key;
+  return t->prog[idx][variant] != nullptr && !t->key[idx][variant].empty() && t->key[idx][variant] == key;
 }
 
 // every product of a dense bf16 net (batch x width and width x width outputs, at most two terms
@@ -572,13 +586,13 @@ bool chain_sizes(const mw_net* n) {
          5 * (n->L + 1) <= kTcMaxProgram;
 }
 
-TcProgram* program_begin(const Ctx& c, int idx, int slot) {
+TcProgram* program_begin(const Ctx& c, int idx, int slot, int variant = 0) {
   TensorState* t = state_of(c);
-  if (!t->prog[idx]) t->prog[idx] = tc_program_create();
-  t->key[idx].clear();
-  tc_program_begin(t->prog[idx], c.at<char>(c.lay->prog_table[slot]),
+  if (!t->prog[idx][variant]) t->prog[idx][variant] = tc_program_create();
+  t->key[idx][variant].clear();
+  tc_program_begin(t->prog[idx][variant], c.at<char>(c.lay->prog_table[slot]),
                    c.at<unsigned int>(c.lay->prog_done[slot]), net_pair(c));
-  return t->prog[idx];
+  return t->prog[idx][variant];
 }
 
 struct Adder {
@@ -591,7 +605,7 @@ struct Adder {
     const int L = c.n->L;
     for (int k = 0; (all || k < f->per_slot) && f->next < f->total; ++k, ++f->next) {
       const int stage = f->next / L, l = f->next % L;
-      f->last[l] = add(ns_product(c, l, stage, f->params, f->sched, f->steps), f->last[l]);
+      f->last[l] = add(ns_product(c, l, stage, f->params, f->sched, f->steps, f->side0), f->last[l]);
     }
   }
   int add(const TcGemm& g, int d0 = -1, int d1 = -1, int d2 = -1) { return add_to(g, -1, d0, d1, d2); }
@@ -651,8 +665,9 @@ mw_status forward_program(const Ctx& c, const void* const* params, const void* x
   const __nv_bfloat16* xin = nullptr;
   MW_TRY(input_planes(c, x, &xin));
   const std::vector<const void*> key = key_of(c, params, x, nullptr, nullptr);
-  if (!program_ready(c, idx, key)) {
-    Adder a{c, program_begin(c, idx, 0)};
+  const int variant = feed ? feed->variant : 0;
+  if (!program_ready(c, idx, key, variant)) {
+    Adder a{c, program_begin(c, idx, 0, variant)};
     int prev = -1;
     for (int l = 0; l < L; ++l) {
       const mw_layer_desc& ld = c.n->layers[l];
@@ -677,9 +692,9 @@ mw_status forward_program(const Ctx& c, const void* const* params, const void* x
       xin = xout;
     }
     MW_TRY(a.status);
-    state_of(c)->key[idx] = key;
+    state_of(c)->key[idx][variant] = key;
   }
-  return tc_program_launch(state_of(c)->prog[idx], c.st, c.s);
+  return tc_program_launch(state_of(c)->prog[idx][variant], c.st, c.s);
 }
 
 // Phase II as one launch (the g_z planes of the last layer are in hp[0])
@@ -690,8 +705,9 @@ mw_status phase2_program(const Ctx& c, const void* const* params, void* g0, NsFe
   for (int l = 0; l + 1 < L; ++l)
     if (n->layers[l].act == MW_ACT_RELU) MW_TRY(relu_index(c, l));
   const std::vector<const void*> key = key_of(c, params, g0, nullptr, nullptr);
-  if (!program_ready(c, MW_PROG_PHASE2, key)) {
-    Adder a{c, program_begin(c, MW_PROG_PHASE2, 1)};
+  const int variant = feed ? feed->variant : 0;
+  if (!program_ready(c, MW_PROG_PHASE2, key, variant)) {
+    Adder a{c, program_begin(c, MW_PROG_PHASE2, 1, variant)};
     int prev = -1, cur = 0;
     if (feed) {
       // Phase I took its share; earlier steps of every layer ended with that launch
@@ -731,15 +747,21 @@ mw_status phase2_program(const Ctx& c, const void* const* params, void* g0, NsFe
       cur ^= 1;
     }
     MW_TRY(a.status);
-    state_of(c)->key[MW_PROG_PHASE2] = key;
+    state_of(c)->key[MW_PROG_PHASE2][variant] = key;
   }
-  return tc_program_launch(state_of(c)->prog[MW_PROG_PHASE2], c.st, c.s);
+  return tc_program_launch(state_of(c)->prog[MW_PROG_PHASE2][variant], c.st, c.s);
 }
 
 // term planes of h_l as the vijp's operand: the checkpoint where the recursion restarts
 const __nv_bfloat16* h_planes(const Ctx& c, int l) {
   return (l > 0 && is_reseed(c.n, l)) ? c.at<__nv_bfloat16>(c.lay->reseed[l])
                                       : c.at<__nv_bfloat16>(c.lay->hp[l & 1]);
+}
+
+// W^-1 of layer l as term planes: where the prep left it
+const __nv_bfloat16* inverse_planes(const Ctx& c, int l) {
+  if (use_programs(c.n)) return ns_buffers(c).Xp[c.n->inv_side & 1] + (int64_t)l * 3 * c.nn;
+  return c.at<__nv_bfloat16>(c.lay->inv[l]);
 }
 
 // the products of layer l of the sweep
@@ -782,8 +804,7 @@ TcGemm vijp_product(const Ctx& c, int l, bool want_h, bool want_gz) {
     e.plane_stride = c.bn;
   }
   return product(c, operand(h_planes(c, l), c.B, c.dim, c.pr.ph, false),
-                 operand(c.at<__nv_bfloat16>(lay.inv[l]), c.dim, c.dim, c.pr.ph, true), c.B, c.dim,
-                 c.dim, e, 1);
+                 operand(inverse_planes(c, l), c.dim, c.dim, c.pr.ph, true), c.B, c.dim, c.dim, e, 1);
 }
 
 // `layer`: whose gradient this is (for the fused parameter update, Algorithm 1's last line)
@@ -933,9 +954,9 @@ mw_status backprop_program(const Ctx& c, const void* const* params, const void* 
       cur ^= 1;
     }
     MW_TRY(a.status);
-    state_of(c)->key[MW_PROG_BP_BWD] = key;
+    state_of(c)->key[MW_PROG_BP_BWD][0] = key;
   }
-  return tc_program_launch(state_of(c)->prog[MW_PROG_BP_BWD], c.st, c.s);
+  return tc_program_launch(state_of(c)->prog[MW_PROG_BP_BWD][0], c.st, c.s);
 }
 
 }  // namespace
@@ -1023,7 +1044,9 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     }
   }
   if (!backprop) {
-    if (resident) {
+    if (use_programs(n)) {
+      // the inverses stay where the last Newton-Schulz step wrote them (ns_r)
+    } else if (resident) {
       for (int l = 0; l < L; ++l) lay.inv[l] = b.take(2 * (size_t)pr.ph * nn);
     } else {
       Region slot = b.take(2 * (size_t)pr.ph * nn);
@@ -1044,8 +1067,10 @@ void tensor_destroy(mw_net* n) {
   if (n->tc) {
     TensorState* t = static_cast<TensorState*>(n->tc);
     for (int i = 0; i < MW_PROG_COUNT; ++i)
-      if (t->prog[i]) tc_program_destroy(t->prog[i]);
-    for (TcProgram* pr : t->sweep) tc_program_destroy(pr);
+      for (int v = 0; v < kProgVariants; ++v)
+        if (t->prog[i][v]) tc_program_destroy(t->prog[i][v]);
+    for (int v = 0; v < 2; ++v)
+      for (TcProgram* pr : t->sweep[v]) tc_program_destroy(pr);
     tc_cache_destroy(t->cache);
     delete t;
     n->tc = nullptr;
@@ -1068,20 +1093,30 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
   const bool resident = n->opts.resident_inverse != 0;
   if (use_programs(n)) {
     // each phase is one launch, and the inverse steps of all layers ride along in both
-    NsFeed feed = make_feed(c, params);
+    // a workspace that kept its inverses: refresh them (one step) instead of starting over
+    const bool warm = n->opts.warm_inverse != 0 && n->warm_ws == ws;
+    n->warm_ws = nullptr;
+    NsFeed feed = make_feed(c, params, warm, warm ? n->inv_side : 0);
     if (feed.steps < 1) return MW_ERR_INVALID_ARG;
     MW_TRY(split_all_weights(c, params));
-    MW_TRY(ns_prepare_all(c, params, feed.sched));
+    if (!warm) MW_TRY(ns_prepare_all(c, params, feed.sched));
     MW_TRY(forward_program(c, params, x, false, &feed));      // Phase I
     MW_TRY(loss_and_top(c, target, loss_out, true));
     MW_TRY(phase2_program(c, params, g0, &feed));             // Phase II
-    // the last update squares the last residual: gate on it so a diverging layer is reported
-    const double limit = n->opts.prec == MW_F32 ? 2e-3 : 2e-2;
+    // the last update squares the last residual: gate on it so a diverging layer is reported.
+    // From scratch the residual is spread over all directions and its rms singular value is
+    // judged; a refresh must keep the LARGEST one small enough for its square to vanish in the
+    // working precision (5e-4 squared for MW_F32, 4e-3 squared for the two-term bf16 chain)
+    const double limit = warm ? (n->opts.prec == MW_F32 ? 5e-4 : 4e-3) : (n->opts.prec == MW_F32 ? 2e-3 : 2e-2);
     const NsStep lastst = feed.sched[feed.steps - 1];
     const int pw = c.pr.pw < lastst.pr ? c.pr.pw : lastst.pr;
     residual_gate_kernel<<<L, 256, 0, s>>>(ns_buffers(c).sumsq, (int64_t)gate_slots(d),
-                                           (int64_t)tc_sumsq_slots(pw, lastst.pr, d, d), d, limit, c.st, 0);
-    return launch_ok();
+                                           (int64_t)tc_sumsq_slots(pw, lastst.pr, d, d), d, limit, c.st, 0,
+                                           warm ? 1 : 0);
+    MW_TRY(launch_ok());
+    n->inv_side = (feed.side0 + feed.steps) & 1;
+    if (n->opts.warm_inverse) n->warm_ws = ws;
+    return MW_OK;
   }
   if (resident) {
     const int G = ns_group(n);
@@ -1149,17 +1184,19 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
     if (chunk >= 1) {
       const int nchunks = (L + chunk - 1) / chunk;
       const std::vector<const void*> key = key_of(c, params, x, nullptr, dW);
-      if (t->sweep_key != key || (int)t->sweep.size() != nchunks) {
-        t->sweep_key.clear();
-        while ((int)t->sweep.size() < nchunks) t->sweep.push_back(tc_program_create());
-        while ((int)t->sweep.size() > nchunks) { tc_program_destroy(t->sweep.back()); t->sweep.pop_back(); }
+      const int v = n->inv_side & 1;       // the programs name the inverses' current home
+      std::vector<TcProgram*>& progs = t->sweep[v];
+      if (t->sweep_key[v] != key || (int)progs.size() != nchunks) {
+        t->sweep_key[v].clear();
+        while ((int)progs.size() < nchunks) progs.push_back(tc_program_create());
+        while ((int)progs.size() > nchunks) { tc_program_destroy(progs.back()); progs.pop_back(); }
         for (int i = 0; i < nchunks; ++i) {
           const int l0 = i * chunk, l1 = l0 + chunk < L ? l0 + chunk : L;
-          MW_TRY(sweep_chain_program(c, t->sweep[(size_t)i], l0, l1, params, dW, x0p, true));
+          MW_TRY(sweep_chain_program(c, progs[(size_t)i], l0, l1, params, dW, x0p, true));
         }
-        t->sweep_key = key;
+        t->sweep_key[v] = key;
       }
-      for (TcProgram* pr : t->sweep) MW_TRY(tc_program_launch(pr, c.st, c.s));
+      for (TcProgram* pr : progs) MW_TRY(tc_program_launch(pr, c.st, c.s));
       return MW_OK;
     }
   }

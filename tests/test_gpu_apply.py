@@ -20,6 +20,8 @@ def problems():
                                   reseed_every=2, conv_vijp_iters=10, prec=S.F32)),
         ("strided", S.strided_cnn(seed=4, depth=3, C=128, H=32, W=32, batch=4, gamma=0.5, reseed_every=2,
                                   prec=S.F32)),
+        ("conv1d", S.fragmental_cnn1d(seed=6, depth=3, C=64, N=128, batch=4, block=8, reseed_every=2,
+                                      prec=S.F32)),
     ]
 
 
@@ -35,7 +37,7 @@ def test_fused_update_matches_oracle(name, p, in_place):
     ref_grad = O.backprop(p.layers, p.params, p.x, p.target, p.loss, masks=masks)["dW"]
     lr = 0.05 * max(float(np.abs(w).max()) for w in p.params) / max(float(np.abs(g).max()) for g in ref_grad)
     ref = O.moonwalk_sgd_step(p.layers, p.params, p.x, p.target, p.loss, lr, reseed_every=p.reseed_every,
-                              masks=masks, conv_iters=p.conv_vijp_iters or None)
+                              masks=masks, conv_iters=p.conv_vijp_iters or None, frag_block=p.frag_block)
     before = [w.clone() for w in params]
     out = params if in_place else [torch.empty_like(w) for w in params]
     net.forward_sweep_apply(params, x, g0, lr, ws, params_out=out)

@@ -222,6 +222,26 @@ def test_fragmental_cnn1d_bf16_tensor_path(depth, C, N, batch, block, K):
     check_problem(p, 2e-2, backend="tensor", exact_masks=False, tau=2e-2)
 
 
+def test_fragmental_cnn1d_stronger_taps_stated_bar():
+    """The same net with the off-diagonal taps scaled by gamma = 0.5 instead of the recipe's 0.3 and
+    the longest blocks (16): the block recursion g[i+1] = W0^-1 (h[i] - w1 g[i] - w2 g[i-1]) then
+    amplifies fp32 rounding along its 14 steps by more than the four layers between cotangent
+    checkpoints can absorb, and the layers just before a checkpoint land above the 1e-4 bar that the
+    recipe's own weights meet (measured at the paper's size with seed 0: 1.4e-4; on this smaller
+    net with seed 2: 1.1e-4 and 2.7e-4 at layers 3 and 7, below 2e-5 elsewhere).  The case is kept
+    with the bar it does meet, 5e-4, so that a regression of the recursion still shows."""
+    from paper_2402_14212_b200 import synth as S
+    from parity_util import check_problem
+    p = S.fragmental_cnn1d(seed=2, depth=8, C=256, N=512, batch=8, block=16, gamma=0.5, reseed_every=4,
+                           prec=S.F32)
+    out, ref, errs = check_problem(p, 5e-4, backend="tensor", exact_masks=False, tau=1e-4)
+    assert max(errs[:3]) <= 1e-4          # away from the end of a checkpoint interval the bar holds
+    # blocks of 4 (the paper's main setting) stay inside the 1e-4 bar at the same gamma
+    p4 = S.fragmental_cnn1d(seed=2, depth=8, C=256, N=512, batch=8, block=4, gamma=0.5, reseed_every=4,
+                            prec=S.F32)
+    check_problem(p4, 1e-4, backend="tensor", exact_masks=False, tau=1e-4)
+
+
 def test_fragmental_cnn1d_rejects_a_full_tap0():
     from paper_2402_14212_b200 import synth as S
     p = S.fragmental_cnn1d(seed=1, depth=2, C=64, N=128, batch=2, block=4, reseed_every=0, prec=S.F32)
@@ -234,13 +254,16 @@ def test_fragmental_cnn1d_rejects_a_full_tap0():
     assert code == mwb.STATUS_NAMES.index("MW_ERR_NOT_SUBMERSIVE")
 
 
-def test_fragmental_cnn1d_full_size():
-    """The paper's 1-D experiment at its size (2048 x 256 sequences, batch 128; 8 layers, blocks of
-    16 positions: the longest reconstruction the paper uses), in the launch configuration the
-    benchmark times.  The oracle takes the batch in slices, replaying the GPU's sign bits."""
+@pytest.mark.parametrize("depth,block,prec,tol", [(8, 16, "f32", 1e-4), (16, 4, "f32", 1e-4),
+                                                  (16, 4, "bf16_f32acc", 2e-2)])
+def test_fragmental_cnn1d_full_size(depth, block, prec, tol):
+    """The paper's 1-D experiment at its size (2048 x 256 sequences, batch 128): 8 layers with blocks
+    of 16 positions (the longest reconstruction the paper uses), and the benchmark's own workload --
+    16 layers, blocks of 4 -- in fp32 and in bf16, in the launch configuration the benchmark times.
+    The oracle takes the batch in slices, replaying the GPU's sign bits."""
     from paper_2402_14212_b200 import synth as S
     from parity_util import run_gpu
-    p = S.fragmental_cnn1d(seed=0, depth=8, block=16)
+    p = S.fragmental_cnn1d(seed=0, depth=depth, block=block, prec=prec)
     out = run_gpu(p, backend="tensor", backprop=False)
     assert out["status"] == 0
     L, B = len(p.layers), p.batch
@@ -264,11 +287,11 @@ def test_fragmental_cnn1d_full_size():
                 rms = np.sqrt((z * z).mean(axis=1, keepdims=True))
                 worst[l] = max(worst[l], float((np.abs(z) / rms)[d].max()))
         g0_err = max(g0_err, float(np.abs(out["g0"][sl].reshape(ref["g0"].shape) - ref["g0"] * f).max()))
-    assert g0_err <= 1e-4 * float(np.abs(out["g0"]).max())
+    assert g0_err <= tol * float(np.abs(out["g0"]).max())
     for l in range(L):
-        assert worst[l] <= 1e-4 * np.sqrt(l + 1.0), (l, worst[l])
-        assert O.normwise_error(out["dW"][l], dW[l]) <= 1e-4, l
-    assert abs(out["loss"] - loss) <= 1e-4 * abs(loss)
+        assert worst[l] <= tol * np.sqrt(l + 1.0), (l, worst[l])
+        assert O.normwise_error(out["dW"][l], dW[l]) <= tol, l
+    assert abs(out["loss"] - loss) <= tol * abs(loss)
 
 
 @pytest.mark.parametrize("family", ["strided", "conv1d"])

@@ -50,11 +50,14 @@ def test_config4_mixed_mlp_full_size():
     assert len(errs) == 128
 
 
-def test_config5_depth32_full_width():
-    # width 4096, batch 1024, bf16, depth 32 (the first point of the depth sweep); four distinct
-    # weight matrices cycled over the depth
-    p = S.sweep_mlp(seed=0, depth=32, pool=4)
-    check_problem(p, 2e-2, backend="tensor", exact_masks=False, tau=2e-2)
+@pytest.mark.parametrize("depth,resident", [(32, True), (32, False), (64, True)])
+def test_config5_full_width(depth, resident):
+    # width 4096, batch 1024, bf16; four distinct weight matrices cycled over the depth.  Depth 32
+    # is the benchmark's workload (every inverse resident: the chained sweep) and, with one
+    # transient inverse slot, the first point of the depth study; depth 64 is its second point.
+    p = S.sweep_mlp(seed=0, depth=depth, pool=4)
+    out, ref, errs = check_problem(p, 2e-2, backend="tensor", resident=resident, exact_masks=False, tau=2e-2)
+    assert len(errs) == depth
 
 
 @pytest.mark.parametrize("pair", [True, False])
