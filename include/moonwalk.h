@@ -107,7 +107,15 @@ typedef struct {
                               many positions (2..64, dividing W); Phase III rebuilds the rest  */
 } mw_net_opts;
 
-/* Build a host-side description.  `batch` is fixed per net.  Returns MW_ERR_UNSUPPORTED for
+/* Build a host-side description.  `batch` is fixed per net.
+ * Dense layers must be invertible (the vijp of Section 3.1 is g_z = h W^-1).  The CUDA-core
+ * backend inverts with pivoted elimination (widths up to 64) and accepts any invertible W.  The
+ * tensor-core backend iterates X <- X + X (I - W X) from X_0 = (n / ||W||_F^2) W^T in a fixed
+ * number of steps: it converges while sigma_max(W)^2 < 2 mean(sigma_i^2) and reaches working
+ * precision in its default schedule when ||I - W X_0|| is about 0.15 or less, i.e. for weights
+ * near a multiple of an orthogonal matrix (mw_net_opts.inverse_iters adds steps).  Outside that
+ * domain the layer is reported per step as MW_ERR_NOT_SUBMERSIVE, never answered silently.
+ * Returns MW_ERR_UNSUPPORTED for
  * shapes outside: dense layers square; convolutions with C_in = C_out, either stride 1 with
  * k = 2*pad+1 (same size), or every layer of the net meeting Lemma 1 (i) with stride 2 (the
  * paper's submersive CNN: MW_F32 or MW_BF16_F32ACC, 64 or 128 channels, k - 1 - pad < 2, even image sizes, a
@@ -303,6 +311,17 @@ int64_t mw_launch_count(void);
 void mw_profile_begin(void);
 mw_status mw_profile_end(double* total_ms, int64_t* launches, double* flops, double* mma_flops);
 
+/* Self-test of the bounded device-side waits (failure detection): launches one small product that
+ * depends on something no product of its launch ever completes, with every wait of that launch
+ * bounded by limit_ms (1..1000) instead of the usual 2 s.  The waiting lane must give up, record
+ * MW_ERR_TIMEOUT and unwind the CTA (other roles leave, tensor memory is released) so that the
+ * kernel ends and the context stays usable.  *timed_out_status receives the status the launch
+ * recorded (MW_ERR_TIMEOUT when the path works); the return value is that of the host calls.
+ * scratch: device, 256-byte aligned, >= 256 KiB; the status block inside it is cleared again.
+ * Synchronises `stream`.  (The paper has no counterpart.) */
+mw_status mw_selftest_bounded_wait(void* scratch, size_t scratch_bytes, uint32_t limit_ms,
+                                   int32_t* timed_out_status, void* stream);
+
 /* The tensor-core product kernel has two forms: one CTA per 128-row tile, and a pair of CTAs (a
  * cluster of two SMs, tcgen05 cta_group::2) per 256-row tile that stage half of the B tile each.
  * Launches whose products all qualify (operands of at most two bf16 terms, M a multiple of 256,
@@ -310,6 +329,13 @@ mw_status mw_profile_end(double* total_ms, int64_t* launches, double* flops, dou
  * default) turns it back on; returns the previous setting.  Process-wide; for comparisons and
  * tests (the paper has no counterpart). */
 int32_t mw_set_pair_mode(int32_t enable);
+
+/* Pair form, operands of two bf16 terms: with enable = 1 (the default) the three kept cross
+ * products of a tile accumulate in one block of 256 accumulator columns (full-width tensor-core
+ * instructions); with 0 the leading product and the two first-order products have blocks of
+ * their own, added in the epilogue (tiles of 128 columns).  Returns the previous setting.
+ * Process-wide; for comparisons and tests (the paper has no counterpart). */
+int32_t mw_set_merge_orders(int32_t enable);
 
 #ifdef __cplusplus
 }

@@ -85,6 +85,9 @@ def lib() -> C.CDLL:
         L.mw_launch_count.restype = C.c_int64
         L.mw_set_pair_mode.argtypes = [i32]
         L.mw_set_pair_mode.restype = i32
+        L.mw_selftest_bounded_wait.argtypes = [vp, sz, C.c_uint32, C.POINTER(i32), vp]
+        L.mw_set_merge_orders.argtypes = [i32]
+        L.mw_set_merge_orders.restype = i32
         L.mw_profile_begin.argtypes = []
         L.mw_profile_begin.restype = None
         L.mw_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64),
@@ -265,6 +268,24 @@ def launch_count() -> int:
 def set_pair_mode(enable: bool) -> bool:
     """Turn the CTA-pair form of the product kernel on or off; returns the previous setting."""
     return bool(lib().mw_set_pair_mode(int(bool(enable))))
+
+
+def selftest_bounded_wait(limit_ms: int = 5, stream=None) -> int:
+    """Run the library's self-test of its bounded device-side waits; returns the status that the
+    deliberately unsatisfiable launch recorded (MW_ERR_TIMEOUT = 6 when the path works)."""
+    import torch
+    scratch = torch.empty(512 * 1024, dtype=torch.uint8, device="cuda")
+    p = (int(scratch.data_ptr()) + 255) // 256 * 256
+    out = C.c_int32(-1)
+    _check(lib().mw_selftest_bounded_wait(p, scratch.numel() - 256, int(limit_ms), C.byref(out),
+                                          _stream_handle(stream)), "mw_selftest_bounded_wait")
+    return int(out.value)
+
+
+def set_merge_orders(enable: bool) -> bool:
+    """Two-term products of the pair form: one accumulator block for all cross products (True) or
+    one per order (False); returns the previous setting."""
+    return bool(lib().mw_set_merge_orders(int(bool(enable))))
 
 
 def profile_begin():

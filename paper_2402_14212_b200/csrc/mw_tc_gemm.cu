@@ -1238,6 +1238,20 @@ int pick_bn(int pa, int pb, int M, int N, int batch, bool wide = false) {
   return bn;
 }
 
+// Pair form, two-term operands: 1 = all kept cross products of a tile accumulate in ONE block of 256
+// columns (three full-width instructions per K step, both accumulator sets in use); 0 = products of
+// order 0 and order 1 in blocks of their own, which halves the tile (instructions of 128 columns
+// run at two thirds of the tensor rate).
+int g_merge_orders = 1;
+
+// tile width in the pair form
+int pair_bn(int pa, int pb, int N) {
+  const int t = pa > pb ? pa : pb;
+  int bn = (t == 1 || g_merge_orders) ? 256 : 128;
+  while (bn > 128 && N % bn != 0) bn >>= 1;
+  return bn;
+}
+
 // 0: never use the pair form, 1: wherever a launch qualifies (default)
 int g_pair_mode = 1;
 // 1: epilogues hand plain outputs to the copy engine (0: per-lane stores everywhere)
@@ -1250,7 +1264,7 @@ bool pair_capable(const TcGemm& d) {
   if (d.conv.mode != TC_CONV_NONE || d.split_k > 1) return false;
   if (d.A.planes > 2 || d.B.planes > 2) return false;
   if (d.M % 256 != 0 || d.N % 128 != 0) return false;
-  return pick_bn(d.A.planes, d.B.planes, d.M, d.N, d.batch) >= 128;
+  return true;
 }
 
 }  // namespace
@@ -1474,6 +1488,7 @@ uint32_t make_idesc(bool a_mn, bool b_mn, int n, int m = BM) {
 double build_ops_pair(TcProblem& P) {
   const int pa = P.pa, pb = P.pb, bn = P.bn;
   const int t = pa > pb ? pa : pb;
+  const bool merge = t * bn > kSetCols;       // no room for a block per order: one block for all
   const uint32_t b0 = (uint32_t)pa * kATileBytes;
   bool init[4] = {false, false, false, false};
   int n = 0;
@@ -1481,18 +1496,19 @@ double build_ops_pair(TcProblem& P) {
   for (int i = 0; i < pa; ++i)
     for (int j = 0; j < pb; ++j) {
       if (i + j >= t) continue;
+      const int blk = merge ? 0 : i + j;
       TcOp& o = P.ops[n++];
       o.a_off16 = ((uint32_t)i * kATileBytes) >> 4;
       o.b_off16 = (b0 + (uint32_t)j * P.b_tile_bytes) >> 4;
       o.idesc = make_idesc(P.a_mn != 0, P.b_mn != 0, bn, 2 * BM);
-      o.dcol = (uint16_t)((i + j) * bn);
+      o.dcol = (uint16_t)(blk * bn);
       o.rot = 0;
-      o.first_kbs = init[i + j] ? 0u : 1u;
-      init[i + j] = true;
+      o.first_kbs = init[blk] ? 0u : 1u;
+      init[blk] = true;
       cycles += 4.0 * std::max(bn / 2.0, 88.0);
     }
   P.nops = n;
-  P.nblocks = t;
+  P.nblocks = merge ? 1 : t;
   return cycles;
 }
 
@@ -1611,7 +1627,7 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   P.b_mn = d.B.mn_major ? 1 : 0;
   P.a_batch_planes = d.A.batch_planes ? d.A.batch_planes : d.A.planes;
   P.b_batch_planes = d.B.batch_planes ? d.B.batch_planes : d.B.planes;
-  P.bn = pick_bn(P.pa, P.pb, d.M, d.N, d.batch, d.wide_tiles != 0);
+  P.bn = pair ? pair_bn(P.pa, P.pb, d.N) : pick_bn(P.pa, P.pb, d.M, d.N, d.batch, d.wide_tiles != 0);
   P.num_kb = (d.K + BK - 1) / BK;
   int split = d.split_k > 1 ? d.split_k : 1;
   if (split > P.num_kb) split = P.num_kb;
@@ -1903,6 +1919,15 @@ int tc_program_add(TcProgram* pr, TcMapCache* cache, const TcGemm& d, const int*
   return self;
 }
 
+int tc_program_add_group(TcProgram* pr);
+
+// test hook: an entry that nothing ever completes (a group without members that claims one arrival)
+int tc_program_add_unreachable(TcProgram* pr) {
+  const int q = tc_program_add_group(pr);
+  if (q >= 0) pr->target[(size_t)q] = 1u;
+  return q;
+}
+
 int tc_program_add_group(TcProgram* pr) {
   if ((int)pr->table.size() >= kMaxProgram) return -1;
   pr->table.emplace_back();
@@ -1966,14 +1991,19 @@ bool tc_pair_ok(int a_planes, int b_planes, int M, int N) {
   d.A.planes = a_planes; d.B.planes = b_planes; d.M = M; d.N = N; d.K = 64;
   return g_pair_mode != 0 && pair_capable(d);
 }
+int tc_set_merge_orders(int mode) {
+  const int old = g_merge_orders;
+  g_merge_orders = mode != 0;
+  return old;
+}
 int tc_set_pair_mode(int mode) {
   const int old = g_pair_mode;
   g_pair_mode = mode != 0;
   return old;
 }
 void tc_set_wait_limit_ns(uint64_t ns) { g_wait_limit_ns = ns ? ns : kDefaultWaitLimitNs; }
-size_t tc_sumsq_slots(int a_planes, int b_planes, int M, int N) {
-  const int bn = pick_bn(a_planes, b_planes, M, N, 1);
+size_t tc_sumsq_slots(int a_planes, int b_planes, int M, int N, bool pair) {
+  const int bn = pair ? pair_bn(a_planes, b_planes, N) : pick_bn(a_planes, b_planes, M, N, 1);
   return (size_t)((M + BM - 1) / BM) * ((N + bn - 1) / bn) * kEpiWarps;
 }
 
@@ -2066,6 +2096,56 @@ extern "C" mw_status mw_gemm_split_bf16(const float* A, int32_t a_mn, const floa
   MW_CUDA_OK(cudaMemcpyAsync(&host, st, sizeof(host), cudaMemcpyDeviceToHost, s));
   MW_CUDA_OK(cudaStreamSynchronize(s));
   return host.code == 0 ? MW_OK : (mw_status)host.code;
+}
+
+// ---------------------------------------------------------------------------------------
+// Self-test of the bounded device-side waits
+// ---------------------------------------------------------------------------------------
+extern "C" mw_status mw_selftest_bounded_wait(void* scratch, size_t scratch_bytes, uint32_t limit_ms,
+                                              int32_t* timed_out_status, void* stream) {
+  using namespace mw;
+  if (!scratch || !timed_out_status || limit_ms < 1 || limit_ms > 1000) return MW_ERR_INVALID_ARG;
+  const int M = 128, N = 64, K = 128;
+  const size_t table_off = 256, done_off = table_off + tc_program_table_bytes(4), op_off = align_up(done_off + 64, 256);
+  const size_t need = op_off + 2 * (size_t)(M * K + N * K) + 4 * (size_t)M * N + 1024;
+  if (((uintptr_t)scratch & 255u) || scratch_bytes < need) return MW_ERR_WORKSPACE;
+  cudaStream_t s = (cudaStream_t)stream;
+  char* base = static_cast<char*>(scratch);
+  DeviceStatus* st = reinterpret_cast<DeviceStatus*>(base);
+  MW_CUDA_OK(cudaMemsetAsync(base, 0, need, s));        // status, counters, zero operands
+  __nv_bfloat16* A = reinterpret_cast<__nv_bfloat16*>(base + op_off);
+  __nv_bfloat16* B = A + (size_t)M * K;
+  float* D = reinterpret_cast<float*>(B + (size_t)N * K);
+  TcProgram* pr = tc_program_create();
+  tc_program_begin(pr, base + table_off, reinterpret_cast<unsigned int*>(base + done_off), false);
+  TcGemm g;
+  g.A.base = A; g.A.rows = M; g.A.cols = K; g.A.planes = 1; g.A.plane_stride = (int64_t)M * K;
+  g.B.base = B; g.B.rows = N; g.B.cols = K; g.B.planes = 1; g.B.plane_stride = (int64_t)N * K;
+  g.M = M; g.N = N; g.K = K;
+  g.epi.mode = TC_EPI_PLAIN;
+  g.epi.out_f32 = D;
+  mw_status rc = MW_OK;
+  // a product that waits for an entry nothing will ever complete: its copy-issuing lane gives up
+  // after the limit, records the timeout and raises the CTA's abort flag; the issuing lane and the
+  // epilogue warps, waiting for data that will not come, see the flag and leave; tensor memory is
+  // released and the kernel ends
+  const int never = tc_program_add_unreachable(pr);
+  const int deps[1] = {never};
+  if (never < 0 || tc_program_add(pr, nullptr, g, deps, 1, &rc) < 0) {
+    tc_program_destroy(pr);
+    return rc != MW_OK ? rc : MW_ERR_UNSUPPORTED;
+  }
+  tc_set_wait_limit_ns((uint64_t)limit_ms * 1000000ull);
+  rc = tc_program_launch(pr, st, s);
+  tc_set_wait_limit_ns(0);
+  tc_program_destroy(pr);
+  if (rc != MW_OK) return rc;
+  DeviceStatus host;
+  MW_CUDA_OK(cudaMemcpyAsync(&host, st, sizeof(host), cudaMemcpyDeviceToHost, s));
+  MW_CUDA_OK(cudaStreamSynchronize(s));
+  *timed_out_status = (int32_t)host.code;
+  MW_CUDA_OK(cudaMemsetAsync(st, 0, 256, s));
+  return MW_OK;
 }
 
 // ---------------------------------------------------------------------------------------

@@ -194,7 +194,10 @@ int tc_set_pair_mode(int mode);           // 0: never (for comparisons), 1: wher
 // bound of the device-side waits of later launches (0 = default, 2 s)
 void tc_set_wait_limit_ns(uint64_t ns);
 // slots of TcEpilogue::sumsq for one product
-size_t tc_sumsq_slots(int a_planes, int b_planes, int M, int N);
+size_t tc_sumsq_slots(int a_planes, int b_planes, int M, int N, bool pair = false);
+// pair form, two-term operands: one accumulator block for all kept cross products (1, default) or
+// a block per order (0); returns the old setting
+int tc_set_merge_orders(int mode);
 
 // Per-launch timing of the product kernel (CUDA events around every launch while enabled).
 void tc_profile_begin();

@@ -105,19 +105,44 @@ __global__ void frob_final_kernel(const double* __restrict__ partial, int group,
   }
 }
 
-// X0 = c W^T (fp32) through a 32x32 shared tile; blockIdx.z = matrix of the group
+// X0 = c W^T through a 64 x 64 shared tile, written once as fp32 (the iteration's running sum) and
+// as its first `planes` bf16 term planes (the first step's operand); blockIdx.z = matrix of the
+// group.  Matrix g writes X + g*n*n and planes P + g*group_stride + p*n*n.
 template <typename TW>
 __global__ void __launch_bounds__(256)
-x0_kernel(PtrBatch Ws, int n, const float* __restrict__ c, float* __restrict__ X) {
-  __shared__ float tile[32][33];
+x0_kernel(PtrBatch Ws, int n, const float* __restrict__ c, float* __restrict__ X,
+          __nv_bfloat16* __restrict__ P, int planes, int64_t group_stride) {
+  __shared__ float tile[64][65];
   const TW* W = static_cast<const TW*>(Ws.p[blockIdx.z]);
-  float* Xg = X + (int64_t)blockIdx.z * n * n;
-  const int bx = blockIdx.x * 32, by = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int r = ty; r < 32; r += 8) tile[r][tx] = to_f32(W[(int64_t)(by + r) * n + bx + tx]);
+  const int64_t nn = (int64_t)n * n;
+  float* Xg = X + (int64_t)blockIdx.z * nn;
+  __nv_bfloat16* Pg = P + (int64_t)blockIdx.z * group_stride;
+  const int bx = blockIdx.x * 64, by = blockIdx.y * 64;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;      // 64 columns x 4 rows per pass
+  for (int r = ty; r < 64; r += 4) tile[r][tx] = to_f32(W[(int64_t)(by + r) * n + bx + tx]);
   __syncthreads();
   const float cc = c[blockIdx.z];
-  for (int r = ty; r < 32; r += 8) Xg[(int64_t)(bx + r) * n + by + tx] = cc * tile[tx][r];
+  // every thread: 4 consecutive columns of one row of the transposed tile
+  const int q = (threadIdx.x & 15) * 4;
+  for (int r = threadIdx.x >> 4; r < 64; r += 16) {
+    float v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = cc * tile[q + j][r];
+    const int64_t at = (int64_t)(bx + r) * n + by + q;
+    *reinterpret_cast<float4*>(Xg + at) = make_float4(v[0], v[1], v[2], v[3]);
+    for (int p = 0; p < planes; ++p) {
+      __nv_bfloat16 b[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        b[j] = __float2bfloat16_rn(v[j]);
+        v[j] -= __bfloat162float(b[j]);
+      }
+      uint2 pk;
+      pk.x = (uint32_t)__bfloat16_as_ushort(b[0]) | ((uint32_t)__bfloat16_as_ushort(b[1]) << 16);
+      pk.y = (uint32_t)__bfloat16_as_ushort(b[2]) | ((uint32_t)__bfloat16_as_ushort(b[3]) << 16);
+      *reinterpret_cast<uint2*>(Pg + (int64_t)p * nn + at) = pk;
+    }
+  }
 }
 
 // fp32 weights of the group -> 3 bf16 term planes each (dst + g*3*n2)
@@ -285,18 +310,17 @@ mw_status newton_schulz_group(const Ctx& c, int l0, int G, const void* const* pa
   NsStep sched[16];
   const int steps = ns_schedule(c.n, sched);
   if (steps < 1) return MW_ERR_INVALID_ARG;
+  const int first = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;
   if (f32) {
     frob_partial_kernel<float><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
     frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
-    x0_kernel<float><<<dim3(d / 32, d / 32, G), 256, 0, c.s>>>(wp, d, cscale, X);
+    x0_kernel<float><<<dim3(d / 64, d / 64, G), 256, 0, c.s>>>(wp, d, cscale, X, Xp[0], first, 3 * c.nn);
   } else {
     frob_partial_kernel<__nv_bfloat16><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
     frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
-    x0_kernel<__nv_bfloat16><<<dim3(d / 32, d / 32, G), 256, 0, c.s>>>(wp, d, cscale, X);
+    x0_kernel<__nv_bfloat16><<<dim3(d / 64, d / 64, G), 256, 0, c.s>>>(wp, d, cscale, X, Xp[0], first, 3 * c.nn);
   }
   MW_TRY(launch_ok(3));
-  const int first = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;
-  MW_TRY(split_planes_batched(X, c.nn, G, c.nn, Xp[0], first, c.nn, 3 * c.nn, c.s));
   int cur = 0;
   for (int it = 0; it < steps; ++it) {
     const bool last = it + 1 == steps;
@@ -315,7 +339,8 @@ mw_status newton_schulz_group(const Ctx& c, int l0, int G, const void* const* pa
       // the update squares this residual: gate on it so a diverging layer is reported
       const double limit = f32 ? 2e-3 : 2e-2;
       residual_gate_kernel<<<G, 256, 0, c.s>>>(sumsq, (int64_t)gate_slots(d),
-                                               (int64_t)tc_sumsq_slots(pw, sched[it].pr, d, d), d, limit, c.st, l0);
+                                               (int64_t)tc_sumsq_slots(pw, sched[it].pr, d, d, tc_pair_ok(pw, sched[it].pr, d, d)), d, limit,
+                                               c.st, l0);
       MW_TRY(launch_ok());
     }
     // X' = X + X R
@@ -479,15 +504,15 @@ mw_status ns_prepare_all(const Ctx& c, const void* const* params, const NsStep* 
     if (f32) {
       frob_partial_kernel<float><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
       frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
-      x0_kernel<float><<<dim3(d / 32, d / 32, G), 256, 0, c.s>>>(wp, d, cscale, X);
+      x0_kernel<float><<<dim3(d / 64, d / 64, G), 256, 0, c.s>>>(wp, d, cscale, X, nb.Xp[0] + (int64_t)l0 * 3 * c.nn,
+                                                                first, 3 * c.nn);
     } else {
       frob_partial_kernel<__nv_bfloat16><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
       frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
-      x0_kernel<__nv_bfloat16><<<dim3(d / 32, d / 32, G), 256, 0, c.s>>>(wp, d, cscale, X);
+      x0_kernel<__nv_bfloat16><<<dim3(d / 64, d / 64, G), 256, 0, c.s>>>(wp, d, cscale, X,
+                                                                         nb.Xp[0] + (int64_t)l0 * 3 * c.nn, first, 3 * c.nn);
     }
     MW_TRY(launch_ok(3));
-    MW_TRY(split_planes_batched(X, c.nn, G, c.nn, nb.Xp[0] + (int64_t)l0 * 3 * c.nn, first, c.nn,
-                                3 * c.nn, c.s));
   }
   return MW_OK;
 }
@@ -1111,7 +1136,7 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
     const NsStep lastst = feed.sched[feed.steps - 1];
     const int pw = c.pr.pw < lastst.pr ? c.pr.pw : lastst.pr;
     residual_gate_kernel<<<L, 256, 0, s>>>(ns_buffers(c).sumsq, (int64_t)gate_slots(d),
-                                           (int64_t)tc_sumsq_slots(pw, lastst.pr, d, d), d, limit, c.st, 0,
+                                           (int64_t)tc_sumsq_slots(pw, lastst.pr, d, d, net_pair(c)), d, limit, c.st, 0,
                                            warm ? 1 : 0);
     MW_TRY(launch_ok());
     n->inv_side = (feed.side0 + feed.steps) & 1;
