@@ -458,6 +458,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.no_coop:
+        mwb.set_cooperative_launch(False)
     p = workload(args.workload, depth=args.depth, block=args.frag_block)
     b = Bench(p, args, dev)
     net = b.net
@@ -786,6 +788,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--blocks", type=int, default=5,
                     help="repetitions of the timed block of --steps steps (the median block is reported)")
+    ap.add_argument("--no-coop", action="store_true",
+                    help="program launches without the cooperative attribute (for launch lists under a profiler)")
     ap.add_argument("--quick", action="store_true",
                     help="the main line only: no per_config / depth_sweep sections")
     ap.add_argument("--backend", default="auto", choices=["auto", "simt", "tensor"])

@@ -337,6 +337,13 @@ int32_t mw_set_pair_mode(int32_t enable);
  * Process-wide; for comparisons and tests (the paper has no counterpart). */
 int32_t mw_set_merge_orders(int32_t enable);
 
+/* Whole phases run as one launch whose products wait for one another, which needs every CTA
+ * resident: such launches carry the cooperative-launch attribute (enable = 1, the default).  A
+ * profiler that cannot replay a cooperative launch of clusters can have it left out (0); the grid
+ * never exceeds what the device holds at once, so on an otherwise idle GPU nothing changes.
+ * Returns the previous setting.  Process-wide (the paper has no counterpart). */
+int32_t mw_set_cooperative_launch(int32_t enable);
+
 #ifdef __cplusplus
 }
 #endif

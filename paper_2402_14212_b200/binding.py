@@ -86,6 +86,8 @@ def lib() -> C.CDLL:
         L.mw_set_pair_mode.argtypes = [i32]
         L.mw_set_pair_mode.restype = i32
         L.mw_selftest_bounded_wait.argtypes = [vp, sz, C.c_uint32, C.POINTER(i32), vp]
+        L.mw_set_cooperative_launch.argtypes = [i32]
+        L.mw_set_cooperative_launch.restype = i32
         L.mw_set_merge_orders.argtypes = [i32]
         L.mw_set_merge_orders.restype = i32
         L.mw_profile_begin.argtypes = []
@@ -280,6 +282,11 @@ def selftest_bounded_wait(limit_ms: int = 5, stream=None) -> int:
     _check(lib().mw_selftest_bounded_wait(p, scratch.numel() - 256, int(limit_ms), C.byref(out),
                                           _stream_handle(stream)), "mw_selftest_bounded_wait")
     return int(out.value)
+
+
+def set_cooperative_launch(enable: bool) -> bool:
+    """Program launches with or without the cooperative-launch attribute (profiling aid)."""
+    return bool(lib().mw_set_cooperative_launch(int(bool(enable))))
 
 
 def set_merge_orders(enable: bool) -> bool:

@@ -36,7 +36,7 @@ struct Layout {
   std::vector<Region> cw, cwhat, cwinv;      // per layer: kernel, folded kernel, centre-tap inverse (term planes)
   std::vector<Region> cfrag;                 // per layer: fragmental checkpoints of a 1-D convolution
   Region cwinv_f32, cwhat_f32, cg[2], chpf, cxf, cpart, clogits, cseed;
-  Region ns_sumsq;
+  Region ns_sumsq, ns_scale;
   Region prog_table[3], prog_done[3];        // product tables and completion counters of program launches
   Region split[3];                           // K-split meeting places of concurrently running products
 };

@@ -499,10 +499,17 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
       break;
     }
     case TC_EPI_RESID: {
+      if (e.scale_dev) {
+        // acc = W W^T: the factor T = c (2 I - c W W^T) of the first step X_1 = W^T T
+        const float cs = __ldg(e.scale_dev);
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        v[i] = ((col0 + i) == row ? 1.f : 0.f) - v[i];
-        if (valid) sumsq_local += (double)v[i] * (double)v[i];
+        for (int i = 0; i < 32; ++i) v[i] = cs * (((col0 + i) == row ? 2.f : 0.f) - cs * v[i]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          v[i] = ((col0 + i) == row ? 1.f : 0.f) - v[i];
+          if (valid) sumsq_local += (double)v[i] * (double)v[i];
+        }
       }
       if (e.out_f32) store_f32x32(v, e.out_f32 + off, valid, eo, col0);
       if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0);
@@ -1011,6 +1018,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         if (epi.planes2) epi.planes2 += z * epi.bs_planes2;
         if (epi.mask) epi.mask += z * epi.bs_mask;
         if (epi.sumsq) epi.sumsq += z * epi.bs_sumsq;
+        if (epi.scale_dev) epi.scale_dev += z;
       }
       // The row's sign words of this tile are fetched now, while the products are still running:
       // read inside the chunk loop, each would put a trip to global memory on the epilogue's
@@ -1735,6 +1743,9 @@ static mw_status ensure_kernel_attr() {
 
 // bound of the device-side waits of the launches that follow (test hook; 0 restores the default)
 static uint64_t g_wait_limit_ns = kDefaultWaitLimitNs;
+// 0: program launches go without the cooperative attribute (profilers that cannot replay a
+// cooperative launch of clusters; residency is then the caller's business).  Default 1.
+static int g_cooperative = 1;
 
 // CTA pairs that can be resident at once (cached per device); 0 when clusters cannot be launched
 static int max_pairs(size_t smem) {
@@ -1775,7 +1786,7 @@ static cudaError_t launch_kernel(bool program, bool pair, int grid, size_t smem,
   int na = 0;
   if (program) {
     attr[na].id = cudaLaunchAttributeCooperative;
-    attr[na].val.cooperative = 1;
+    attr[na].val.cooperative = g_cooperative;
   } else {
     attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[na].val.programmaticStreamSerializationAllowed = 1;
@@ -1990,6 +2001,11 @@ bool tc_pair_ok(int a_planes, int b_planes, int M, int N) {
   TcGemm d;
   d.A.planes = a_planes; d.B.planes = b_planes; d.M = M; d.N = N; d.K = 64;
   return g_pair_mode != 0 && pair_capable(d);
+}
+int tc_set_cooperative(int mode) {
+  const int old = g_cooperative;
+  g_cooperative = mode != 0;
+  return old;
 }
 int tc_set_merge_orders(int mode) {
   const int old = g_merge_orders;

@@ -38,7 +38,8 @@ struct TcOperand {
 
 enum TcEpiMode : int {
   TC_EPI_PLAIN = 0,    // v = alpha*acc (+ addend);  out_f32 and/or planes
-  TC_EPI_RESID = 1,    // v = (row == col) - acc;    planes; sum of squares -> sumsq
+  TC_EPI_RESID = 1,    // v = (row == col) - acc, or with scale_dev (c = *scale_dev) v = c (2 (row == col) - c acc);
+                       // planes; sum of squares -> sumsq
   TC_EPI_FWD = 2,      // z = acc; sign word written (write_mask) or read; x = phi(z) -> planes (+ out_f32)
   TC_EPI_BWD = 3,      // h = acc -> out_f32 / planes2 (optional), ReLU fragments (optional); g = h * phi'(mask) -> planes
   TC_EPI_VIJP = 4,     // g = alpha*acc (+ addend); activation vijp: h -> planes2 (+ out_f32); g (zero at dead
@@ -60,6 +61,9 @@ struct TcEpilogue {
   int write_mask = 0;
   int act = MW_ACT_NONE;
   float slope = 1.f;
+  // TC_EPI_RESID: a scalar in device memory (one per batch item) that turns the residual of the
+  // start X_0 = c W^T into the factor of the first Newton-Schulz step (see TC_EPI_RESID)
+  const float* scale_dev = nullptr;
   // TC_EPI_RESID: ||v||_F^2 in pieces, one slot per 128-row block, column tile and epilogue warp
   // (tc_sumsq_slots of them; each is written, none accumulated: the reader adds them in order)
   double* sumsq = nullptr;
@@ -198,6 +202,8 @@ size_t tc_sumsq_slots(int a_planes, int b_planes, int M, int N, bool pair = fals
 // pair form, two-term operands: one accumulator block for all kept cross products (1, default) or
 // a block per order (0); returns the old setting
 int tc_set_merge_orders(int mode);
+// program launches with (1, default) or without (0) the cooperative-launch attribute
+int tc_set_cooperative(int mode);
 
 // Per-launch timing of the product kernel (CUDA events around every launch while enabled).
 void tc_profile_begin();

@@ -486,33 +486,24 @@ NsBuffers ns_buffers(const Ctx& c) {
   return b;
 }
 
-// X_0 = (n / ||W||_F^2) W^T and its first term planes, all layers (weight planes exist already)
-mw_status ns_prepare_all(const Ctx& c, const void* const* params, const NsStep* sched) {
+// c_l = n / ||W_l||_F^2 of every layer: the scale of the start X_0 = c W^T.  X_0 itself is never
+// formed: the first step X_1 = X_0 (2 I - W X_0) = W^T [c (2 I - c W W^T)] is two products that
+// read W in place (ns_product).
+mw_status ns_prepare_all(const Ctx& c, const void* const* params) {
   const Layout& lay = *c.lay;
   const int L = c.n->L, d = c.dim;
   const bool f32 = c.n->opts.prec == MW_F32;
-  const NsBuffers nb = ns_buffers(c);
   char* sc = c.at<char>(lay.inv_scratch);
-  float* cscale = reinterpret_cast<float*>(sc + 8 * kMaxGroup);
   double* fpart = reinterpret_cast<double*>(sc + 12 * kMaxGroup + 64);
-  const int first = sched[0].pr > sched[0].pu ? sched[0].pr : sched[0].pu;
+  float* cscale = c.at<float>(lay.ns_scale);
   for (int l0 = 0; l0 < L; l0 += kMaxGroup) {
     const int G = (L - l0) < kMaxGroup ? (L - l0) : kMaxGroup;
     PtrBatch wp{};
     for (int g = 0; g < G; ++g) wp.p[g] = params[l0 + g];
-    float* X = nb.X + (int64_t)l0 * c.nn;
-    if (f32) {
-      frob_partial_kernel<float><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
-      frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
-      x0_kernel<float><<<dim3(d / 64, d / 64, G), 256, 0, c.s>>>(wp, d, cscale, X, nb.Xp[0] + (int64_t)l0 * 3 * c.nn,
-                                                                first, 3 * c.nn);
-    } else {
-      frob_partial_kernel<__nv_bfloat16><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
-      frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale);
-      x0_kernel<__nv_bfloat16><<<dim3(d / 64, d / 64, G), 256, 0, c.s>>>(wp, d, cscale, X,
-                                                                         nb.Xp[0] + (int64_t)l0 * 3 * c.nn, first, 3 * c.nn);
-    }
-    MW_TRY(launch_ok(3));
+    if (f32) frob_partial_kernel<float><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
+    else frob_partial_kernel<__nv_bfloat16><<<dim3(kFrobBlocks, G), 256, 0, c.s>>>(wp, c.nn, fpart);
+    frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, G, d, cscale + l0);
+    MW_TRY(launch_ok(2));
   }
   return MW_OK;
 }
@@ -520,7 +511,7 @@ mw_status ns_prepare_all(const Ctx& c, const void* const* params, const NsStep* 
 // product `stage` of layer l: even = residual R = I - W X of step stage/2, odd = its update
 // (the iterate alternates between its two homes Xp[0], Xp[1]; step `it` reads home side0 + it)
 TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, const NsStep* sched,
-                  int steps, int side0) {
+                  int steps, int side0, bool warm) {
   const Layout& lay = *c.lay;
   const int d = c.dim, it = stage >> 1, cur = (side0 + it) & 1;
   const bool last = it + 1 == steps;
@@ -532,9 +523,32 @@ TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, con
   TcGemm g;
   g.M = d; g.N = d; g.K = d;
   g.wide_tiles = 1;      // throughput work beside the latency-bound chains
+  const void* W = c.n->opts.prec == MW_F32 ? (const void*)c.at<__nv_bfloat16>(lay.w_planes[l]) : params[l];
+  if (it == 0 && !warm) {
+    // from scratch: X_0 = c W^T stays implicit.  Stage 0: T = c (2 I - c W W^T) (W against itself,
+    // both K-major); stage 1: X_1 = W^T T (W read through its transpose), no addend.
+    const int pw = c.pr.pw < sched[0].pu ? c.pr.pw : sched[0].pu;
+    if (!(stage & 1)) {
+      g.A = operand(W, d, d, pw, false);
+      g.B = operand(W, d, d, pw, false);
+      g.epi.mode = TC_EPI_RESID;
+      g.epi.scale_dev = c.at<float>(lay.ns_scale) + l;
+      g.epi.planes = Rp; g.epi.n_planes = sched[0].pu; g.epi.plane_stride = c.nn;
+    } else {
+      int next_terms = c.pr.ph;
+      if (!last) next_terms = sched[1].pr > sched[1].pu ? sched[1].pr : sched[1].pu;
+      g.A = operand(W, d, d, pw, true);
+      g.B = operand(Rp, d, d, sched[0].pu, true);
+      g.epi.mode = TC_EPI_PLAIN;
+      g.epi.out_f32 = (last && !c.n->opts.warm_inverse) ? nullptr : X;
+      g.epi.planes = Xn;
+      g.epi.n_planes = next_terms;
+      g.epi.plane_stride = c.nn;
+    }
+    return g;
+  }
   if (!(stage & 1)) {
     const int pw = c.pr.pw < sched[it].pr ? c.pr.pw : sched[it].pr;
-    const void* W = c.n->opts.prec == MW_F32 ? (const void*)c.at<__nv_bfloat16>(lay.w_planes[l]) : params[l];
     g.A = operand(W, d, d, pw, false);
     g.B = operand(Xc, d, d, sched[it].pr, true);
     g.epi.mode = TC_EPI_RESID;
@@ -630,7 +644,8 @@ struct Adder {
     const int L = c.n->L;
     for (int k = 0; (all || k < f->per_slot) && f->next < f->total; ++k, ++f->next) {
       const int stage = f->next / L, l = f->next % L;
-      f->last[l] = add(ns_product(c, l, stage, f->params, f->sched, f->steps, f->side0), f->last[l]);
+      f->last[l] = add(ns_product(c, l, stage, f->params, f->sched, f->steps, f->side0, (f->variant & 2) != 0),
+                       f->last[l]);
     }
   }
   int add(const TcGemm& g, int d0 = -1, int d1 = -1, int d2 = -1) { return add_to(g, -1, d0, d1, d2); }
@@ -1080,6 +1095,7 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     // program path: every layer keeps its own Newton-Schulz iterate
     const size_t G = use_programs(n) ? (size_t)L : (size_t)ns_group(n);
     lay.ns_sumsq = b.take(sizeof(double) * gate_slots((int)d) * G);
+    lay.ns_scale = b.take(sizeof(float) * (size_t)L);
     lay.ns_x = b.take(4 * nn * G);
     lay.ns_r = b.take(2 * 9 * nn * G);  // per group member: R planes [3] + two iterate plane sets
     if (n->opts.prec != MW_F32 && G > 1 && !use_programs(n)) lay.ns_w = b.take(2 * nn * G);
@@ -1124,7 +1140,7 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
     NsFeed feed = make_feed(c, params, warm, warm ? n->inv_side : 0);
     if (feed.steps < 1) return MW_ERR_INVALID_ARG;
     MW_TRY(split_all_weights(c, params));
-    if (!warm) MW_TRY(ns_prepare_all(c, params, feed.sched));
+    if (!warm) MW_TRY(ns_prepare_all(c, params));
     MW_TRY(forward_program(c, params, x, false, &feed));      // Phase I
     MW_TRY(loss_and_top(c, target, loss_out, true));
     MW_TRY(phase2_program(c, params, g0, &feed));             // Phase II

@@ -5,6 +5,7 @@
   python -m paper_2402_14212_b200.profile_cases fragments --rows 65536 --cols 2048
   python -m paper_2402_14212_b200.profile_cases conv --images 512 --op 1 --terms 2
   python -m paper_2402_14212_b200.profile_cases sconv --images 16 --op 0 --terms 3
+  python -m paper_2402_14212_b200.profile_cases step --workload sweep_mlp --depth 4 --no-coop
 
 Each case allocates its seeded inputs, runs the kernel `--reps` times and exits.
 """
@@ -19,7 +20,12 @@ def main():
     import torch
     from . import binding as mwb
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["gemm", "pack", "fragments", "vijp", "conv", "sconv"])
+    ap.add_argument("case", choices=["gemm", "pack", "fragments", "vijp", "conv", "sconv", "step"])
+    ap.add_argument("--workload", default="sweep_mlp", help="step: a workload of paper_2402_14212_b200.synth")
+    ap.add_argument("--depth", type=int, default=4)
+    ap.add_argument("--no-coop", action="store_true",
+                    help="step: program launches without the cooperative attribute (for profilers)")
+    ap.add_argument("--no-pair", action="store_true", help="one CTA per tile everywhere")
     ap.add_argument("--M", type=int, default=256)
     ap.add_argument("--N", type=int, default=1024)
     ap.add_argument("--K", type=int, default=1024)
@@ -33,7 +39,29 @@ def main():
     ap.add_argument("--op", type=int, default=0, help="0 conv, 1 TransposeConv, 2 weight vjp")
     a = ap.parse_args()
     g = torch.Generator(device="cuda").manual_seed(0)
-    if a.case == "gemm":
+    if a.no_pair:
+        mwb.set_pair_mode(False)
+    if a.case == "step":
+        # warm steps, then `reps` whole Moonwalk steps of a synthetic workload (launch lists)
+        from . import synth as S
+        make = {"sweep_mlp": lambda: S.sweep_mlp(seed=0, depth=a.depth, pool=4),
+                "mixed_mlp": lambda: S.mixed_mlp(seed=0, depth=a.depth),
+                "deep_mlp": lambda: S.deep_mlp(seed=0, depth=a.depth)}[a.workload]
+        p = make()
+        if a.no_coop:
+            mwb.set_cooperative_launch(False)
+        net = mwb.net_for(p, backend="tensor")
+        params, x, target = mwb.to_device(p)
+        ws = net.alloc_workspace("moonwalk")
+        g0 = torch.empty(x.shape, dtype=torch.float32, device="cuda")
+        dW = [torch.empty(w.shape, dtype=torch.float32, device="cuda") for w in params]
+        for _ in range(2 + a.reps):
+            net.input_cotangent(params, x, target, ws, g0_out=g0)
+            net.forward_sweep(params, x, g0, ws, dW_out=dW)
+        torch.cuda.synchronize()
+        code, detail = net.last_device_status(ws)
+        assert code == 0, (code, detail)
+    elif a.case == "gemm":
         A = torch.randn((a.K, a.M) if a.a_mn else (a.M, a.K), device="cuda", generator=g)
         B = torch.randn((a.K, a.N) if a.b_mn else (a.N, a.K), device="cuda", generator=g)
         for _ in range(a.reps):
