@@ -344,6 +344,12 @@ int32_t mw_set_merge_orders(int32_t enable);
  * Returns the previous setting.  Process-wide (the paper has no counterpart). */
 int32_t mw_set_cooperative_launch(int32_t enable);
 
+/* Epilogues of the product kernel hand outputs that are plain [M][N] arrays to the copy engine
+ * (staged in shared memory, cp.async.bulk.tensor stores; enable = 1, the default) or write them
+ * with per-lane 16-byte stores (0), as scattered outputs always are.  Returns the previous
+ * setting.  Process-wide; for comparisons and tests (the paper has no counterpart). */
+int32_t mw_set_bulk_epilogue(int32_t enable);
+
 #ifdef __cplusplus
 }
 #endif

@@ -86,6 +86,8 @@ def lib() -> C.CDLL:
         L.mw_set_pair_mode.argtypes = [i32]
         L.mw_set_pair_mode.restype = i32
         L.mw_selftest_bounded_wait.argtypes = [vp, sz, C.c_uint32, C.POINTER(i32), vp]
+        L.mw_set_bulk_epilogue.argtypes = [i32]
+        L.mw_set_bulk_epilogue.restype = i32
         L.mw_set_cooperative_launch.argtypes = [i32]
         L.mw_set_cooperative_launch.restype = i32
         L.mw_set_merge_orders.argtypes = [i32]
@@ -282,6 +284,11 @@ def selftest_bounded_wait(limit_ms: int = 5, stream=None) -> int:
     _check(lib().mw_selftest_bounded_wait(p, scratch.numel() - 256, int(limit_ms), C.byref(out),
                                           _stream_handle(stream)), "mw_selftest_bounded_wait")
     return int(out.value)
+
+
+def set_bulk_epilogue(enable: bool) -> bool:
+    """Epilogue outputs through the copy engine (True) or per-lane stores (False)."""
+    return bool(lib().mw_set_bulk_epilogue(int(bool(enable))))
 
 
 def set_cooperative_launch(enable: bool) -> bool:

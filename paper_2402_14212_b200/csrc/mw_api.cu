@@ -694,6 +694,7 @@ extern "C" int64_t mw_launch_count(void) { return (int64_t)g_launch_count; }
 extern "C" int32_t mw_set_pair_mode(int32_t enable) { return tc_set_pair_mode(enable); }
 extern "C" int32_t mw_set_merge_orders(int32_t enable) { return tc_set_merge_orders(enable); }
 extern "C" int32_t mw_set_cooperative_launch(int32_t enable) { return tc_set_cooperative(enable); }
+extern "C" int32_t mw_set_bulk_epilogue(int32_t enable) { return tc_set_bulk_epilogue(enable); }
 
 extern "C" void mw_profile_begin(void) { tc_profile_begin(); }
 

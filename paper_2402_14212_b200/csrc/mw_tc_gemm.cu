@@ -983,7 +983,9 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
     const int quarter = warp & 3;                 // tensor-memory lane quarter this warp may read
     const int half = 0;
     // this warp's buffer for bulk stores (0: none, direct stores)
-    const uint32_t epi_sbuf = p.epi_stage_off ? tiles + p.epi_stage_off + (uint32_t)quarter * kEpiStageBytes : 0u;
+    // (pair form only: the one-CTA form serves the small fp32-accurate tiles and the convolution
+    // windows, whose epilogues are at the register limit without it)
+    const uint32_t epi_sbuf = (kPair && p.epi_stage_off) ? tiles + p.epi_stage_off + (uint32_t)quarter * kEpiStageBytes : 0u;
     bool bulk_used = false;
     int j = 0, q = 0, rr = 0;
     bool ok = true;
@@ -1026,7 +1028,8 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       uint32_t mw[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) mw[i] = 0xffffffffu;
-      if (epi.mask && epi.act != MW_ACT_NONE && row < P.M &&
+      const bool early_words = kPair;
+      if (early_words && epi.mask && epi.act != MW_ACT_NONE && row < P.M &&
           ((epi.mode == TC_EPI_FWD && !epi.write_mask) || epi.mode == TC_EPI_BWD || epi.mode == TC_EPI_VIJP)) {
         const uint32_t* mrow = epi.mask + (int64_t)orow * (N >> 5) + (w.n0 >> 5);
 #pragma unroll
@@ -1141,7 +1144,11 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
             const int ci = c >> 5;      // the chunk's sign word, by selection (no indexed registers)
             const uint32_t lo = ci & 2 ? (ci & 1 ? mw[3] : mw[2]) : (ci & 1 ? mw[1] : mw[0]);
             const uint32_t hi = ci & 2 ? (ci & 1 ? mw[7] : mw[6]) : (ci & 1 ? mw[5] : mw[4]);
-            epilogue_chunk(epi, N, row, orow, w.n0 + c, v, sumsq_local, row < P.M, eo, ci & 4 ? hi : lo);
+            uint32_t mword = ci & 4 ? hi : lo;
+            if (!early_words && epi.mask && epi.act != MW_ACT_NONE && row < P.M &&
+                ((epi.mode == TC_EPI_FWD && !epi.write_mask) || epi.mode == TC_EPI_BWD || epi.mode == TC_EPI_VIJP))
+              mword = epi.mask[(int64_t)orow * (N >> 5) + ((w.n0 + c) >> 5)];
+            epilogue_chunk(epi, N, row, orow, w.n0 + c, v, sumsq_local, row < P.M, eo, mword);
           }
         }
       }
@@ -2001,6 +2008,11 @@ bool tc_pair_ok(int a_planes, int b_planes, int M, int N) {
   TcGemm d;
   d.A.planes = a_planes; d.B.planes = b_planes; d.M = M; d.N = N; d.K = 64;
   return g_pair_mode != 0 && pair_capable(d);
+}
+int tc_set_bulk_epilogue(int mode) {
+  const int old = g_bulk_epilogue;
+  g_bulk_epilogue = mode != 0;
+  return old;
 }
 int tc_set_cooperative(int mode) {
   const int old = g_cooperative;

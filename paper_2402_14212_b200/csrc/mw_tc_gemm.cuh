@@ -202,6 +202,8 @@ size_t tc_sumsq_slots(int a_planes, int b_planes, int M, int N, bool pair = fals
 // pair form, two-term operands: one accumulator block for all kept cross products (1, default) or
 // a block per order (0); returns the old setting
 int tc_set_merge_orders(int mode);
+// epilogue outputs through the copy engine (1, default) or per-lane stores only (0)
+int tc_set_bulk_epilogue(int mode);
 // program launches with (1, default) or without (0) the cooperative-launch attribute
 int tc_set_cooperative(int mode);
 
