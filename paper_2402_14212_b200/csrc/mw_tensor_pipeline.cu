@@ -13,6 +13,8 @@
 //              (Eq. "h_i"), and the weight vjp of the layer before, dW = g_z^T x (Eq. "g_i").
 // Products with too few output tiles for the machine are cut along K (deterministic meeting in
 // the workspace).
+#include <cstring>
+
 #include "mw_tc_gemm.cuh"
 #include "mw_tensor.cuh"
 
@@ -618,11 +620,10 @@ bool net_pair(const Ctx& c) {
   return c.n->opts.prec != MW_F32 && tc_pair_ok(2, 2, c.B, c.dim) && tc_pair_ok(2, 2, c.dim, c.dim);
 }
 
-// sizes at which the sweep may run as chains (the workspace then holds the longer rings)
+// sizes at which the sweep may run as chains (the workspace then holds the longer rings): row
+// blocks of 256 for the pair form, of 128 otherwise
 bool chain_sizes(const mw_net* n) {
-  const int d = n->layers[0].n_in;
-  return n->opts.prec != MW_F32 && n->opts.resident_inverse != 0 && n->B % 256 == 0 && d % 256 == 0 &&
-         5 * (n->L + 1) <= kTcMaxProgram;
+  return n->opts.resident_inverse != 0 && n->B % 128 == 0 && n->B / 128 <= 16 && 5 * (n->L + 1) <= kTcMaxProgram;
 }
 
 TcProgram* program_begin(const Ctx& c, int idx, int slot, int variant = 0) {
@@ -895,7 +896,9 @@ mw_status sweep_chain_program(const Ctx& c0, TcProgram* pr, int l0, int l1, cons
   auto at_or = [&](const std::vector<int>& v, int l) { return l >= l0 && l < l1 ? v[(size_t)(l - l0)] : -1; };
   auto weight_vjp = [&](int k) {
     if (!dW[k]) return;
-    const TcGemm g = weight_vjp_product(c, c.at<__nv_bfloat16>(lay.gzp[k % c.ngz]), xbuf(k), (float*)dW[k], k);
+    TcGemm g = weight_vjp_product(c, c.at<__nv_bfloat16>(lay.gzp[k % c.ngz]), xbuf(k), (float*)dW[k], k);
+    g.split_k = 1;
+    g.split_scratch = nullptr;
     // g_z of layer k (all of V_k) and x_k (all of R_{k-1}); a K-split product shares its meeting
     // place with the previous weight vjp
     D[(size_t)(k - l0)] = a.add(g, at_or(GV, k), at_or(GR, k - 1), g.split_k > 1 ? at_or(D, k - 1) : -1);
@@ -911,6 +914,8 @@ mw_status sweep_chain_program(const Ctx& c0, TcProgram* pr, int l0, int l1, cons
       for (int m = 0; m < mt; ++m) {
         TcGemm g = full;
         g.M = rb;
+        g.split_k = 1;         // (the chains run side by side: no shared meeting place)
+        g.split_scratch = nullptr;
         g.A.base = static_cast<const __nv_bfloat16*>(full.A.base) + m * blk;
         g.A.rows = rb;
         TcEpilogue& e = g.epi;
@@ -931,6 +936,8 @@ mw_status sweep_chain_program(const Ctx& c0, TcProgram* pr, int l0, int l1, cons
       for (int m = 0; m < mt; ++m) {
         TcGemm g = full;
         g.M = rb;
+        g.split_k = 1;
+        g.split_scratch = nullptr;
         g.A.base = static_cast<const __nv_bfloat16*>(full.A.base) + m * blk;
         g.A.rows = rb;
         g.epi.mask += (int64_t)m * rb * (d / 32);
@@ -951,6 +958,12 @@ mw_status sweep_chain_program(const Ctx& c0, TcProgram* pr, int l0, int l1, cons
 
 // 1: nets that qualify run the sweep as chained programs (0: one launch per layer, for comparisons)
 int g_sweep_chains = 1;
+
+inline uint32_t __float_as_uint_host(float f) {
+  uint32_t u;
+  memcpy(&u, &f, sizeof(u));
+  return u;
+}
 
 // entries of the product table per layer of a chained sweep
 int chain_entries_per_layer(const Ctx& c, bool pair) { return 2 * (c.B / (pair ? 256 : 128)) + 3; }
@@ -1218,13 +1231,17 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
   MW_TRY(split_planes((const float*)g0, c.bn, c.at<__nv_bfloat16>(lay.hp[0]), c.pr.ph, c.bn, s));
   // Nets whose products all run in the pair form (bf16 storage, sizes multiples of 256): the sweep
   // as chains of products inside program launches, as many layers per launch as the table holds.
-  if (use_programs(n) && chain_sizes(n) && !n->apply_params && net_pair(c) && g_sweep_chains) {
+  if (use_programs(n) && chain_sizes(n) && g_sweep_chains) {
     TensorState* t = state_of(c);
-    const int per_layer = chain_entries_per_layer(c, true);
+    const bool pair = net_pair(c);
+    const int per_layer = chain_entries_per_layer(c, pair);
     const int chunk = (kTcMaxProgram - 4) / per_layer;
     if (chunk >= 1) {
       const int nchunks = (L + chunk - 1) / chunk;
-      const std::vector<const void*> key = key_of(c, params, x, nullptr, dW);
+      std::vector<const void*> key = key_of(c, params, x, nullptr, dW);
+      // the fused update (mw_forward_sweep_apply) changes the weight vjp's epilogue
+      key.push_back(n->apply_params);
+      key.push_back(reinterpret_cast<const void*>((uintptr_t)__float_as_uint_host(n->apply_lr)));
       const int v = n->inv_side & 1;       // the programs name the inverses' current home
       std::vector<TcProgram*>& progs = t->sweep[v];
       if (t->sweep_key[v] != key || (int)progs.size() != nchunks) {
@@ -1233,7 +1250,7 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
         while ((int)progs.size() > nchunks) { tc_program_destroy(progs.back()); progs.pop_back(); }
         for (int i = 0; i < nchunks; ++i) {
           const int l0 = i * chunk, l1 = l0 + chunk < L ? l0 + chunk : L;
-          MW_TRY(sweep_chain_program(c, progs[(size_t)i], l0, l1, params, dW, x0p, true));
+          MW_TRY(sweep_chain_program(c, progs[(size_t)i], l0, l1, params, dW, x0p, pair));
         }
         t->sweep_key[v] = key;
       }
