@@ -178,6 +178,17 @@ mw_status mw_forward_sweep(mw_net* net, const void* const* params, const void* x
                            void* const* dW_out, void* workspace, size_t workspace_bytes,
                            void* stream);
 
+/* Gradient buckets for data-parallel training (Algorithm 1 produces the gradients front to back, so
+ * the all-reduce of the first layers can run while the sweep works on the later ones).  After this
+ * call every mw_forward_sweep on `net` records events[b] (CUDA events of the caller, n_events =
+ * ceil(n_layers / layers_per_bucket)) on its stream as soon as the work that completes dW of the
+ * layers [b * layers_per_bucket, (b + 1) * layers_per_bucket) is enqueued; a consumer stream that
+ * waits for events[b] may then reduce those gradients.  Dense nets on the tensor cores signal the
+ * buckets as they go (one launch per bucket); other nets record all events at the end of the
+ * call.  layers_per_bucket = 0 turns the feature off.  The events stay the caller's. */
+mw_status mw_sweep_bucket_events(mw_net* net, int32_t layers_per_bucket, void* const* events,
+                                 int32_t n_events);
+
 /* Plain reverse mode ("Backprop", Appendix "Complexity Analysis" item 1): forward storing every
  * layer input, backward with both vjps.  Same kernels, for the memory and runtime comparison. */
 mw_status mw_backprop_reference(mw_net* net, const void* const* params, const void* x,

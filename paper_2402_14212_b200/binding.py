@@ -66,6 +66,7 @@ def lib() -> C.CDLL:
         L.mw_input_cotangent.argtypes = [vp, C.POINTER(vp), vp, vp, vp, vp, vp, sz, vp]
         L.mw_forward_sweep.argtypes = [vp, C.POINTER(vp), vp, vp, C.POINTER(vp), vp, sz, vp]
         L.mw_forward_sweep_apply.argtypes = [vp, C.POINTER(vp), vp, vp, C.c_double, C.POINTER(vp), vp, sz, vp]
+        L.mw_sweep_bucket_events.argtypes = [vp, i32, C.POINTER(vp), i32]
         L.mw_backprop_reference.argtypes = [vp, C.POINTER(vp), vp, vp, C.POINTER(vp), vp, vp, sz, vp]
         L.mw_export_masks.argtypes = [vp, vp, i32, vp, sz, C.POINTER(i32), C.POINTER(i32), vp]
         L.mw_last_device_status.argtypes = [vp, vp, vp, C.POINTER(C.c_uint32)]
@@ -219,6 +220,18 @@ class Net:
                                             _ptr_array(params_out), wp, wb, _stream_handle(stream)),
                "mw_forward_sweep_apply")
         return params_out
+
+    def set_bucket_events(self, layers_per_bucket: int, events=None):
+        """events: torch.cuda.Event objects (already recorded once, so that their handles exist), one
+        per bucket of `layers_per_bucket` layers; the forward sweep records them as the buckets'
+        gradients are enqueued.  layers_per_bucket = 0 turns the feature off."""
+        events = list(events or [])
+        arr = (C.c_void_p * max(1, len(events)))()
+        for i, e in enumerate(events):
+            arr[i] = int(e.cuda_event)
+        _check(lib().mw_sweep_bucket_events(self._h, int(layers_per_bucket), arr, len(events)),
+               "mw_sweep_bucket_events")
+        self._bucket_events = events          # keep them alive
 
     def backprop_reference(self, params, x, target, workspace, dW_out=None, loss_out=None,
                            stream=None):

@@ -549,13 +549,32 @@ extern "C" mw_status mw_forward_sweep(mw_net* net, const void* const* params, co
   MW_TRY(check_ws(workspace, workspace_bytes, net->mwl.total));
   if (net->ws_done != workspace || net->x_done != x) return MW_ERR_STATE;
   cudaStream_t s = (cudaStream_t)stream;
+  net->buckets_recorded = 0;
+  mw_status r;
   if (net->backend == MW_BACKEND_TENSOR)
-    return tensor_forward_sweep(net, params, x, g0, dW_out, workspace, s);
-  if (net->opts.prec == MW_F64)
-    return simt_forward_sweep<double>(net, params, (const double*)x, (const double*)g0, dW_out,
-                                      workspace, s);
-  return simt_forward_sweep<float>(net, params, (const float*)x, (const float*)g0, dW_out,
-                                   workspace, s);
+    r = tensor_forward_sweep(net, params, x, g0, dW_out, workspace, s);
+  else if (net->opts.prec == MW_F64)
+    r = simt_forward_sweep<double>(net, params, (const double*)x, (const double*)g0, dW_out, workspace, s);
+  else
+    r = simt_forward_sweep<float>(net, params, (const float*)x, (const float*)g0, dW_out, workspace, s);
+  // buckets that the pipeline did not signal on its way are complete now at the latest
+  if (r == MW_OK) record_buckets(net, net->L, s);
+  return r;
+}
+
+extern "C" mw_status mw_sweep_bucket_events(mw_net* net, int32_t layers_per_bucket, void* const* events,
+                                            int32_t n_events) {
+  if (!net || layers_per_bucket < 0 || n_events < 0) return MW_ERR_INVALID_ARG;
+  net->bucket_events.clear();
+  net->bucket_layers = 0;
+  if (layers_per_bucket == 0 || n_events == 0) return MW_OK;
+  if (!events || n_events != (net->L + layers_per_bucket - 1) / layers_per_bucket) return MW_ERR_INVALID_ARG;
+  for (int i = 0; i < n_events; ++i) {
+    if (!events[i]) { net->bucket_events.clear(); return MW_ERR_INVALID_ARG; }
+    net->bucket_events.push_back((cudaEvent_t)events[i]);
+  }
+  net->bucket_layers = layers_per_bucket;
+  return MW_OK;
 }
 
 extern "C" mw_status mw_forward_sweep_apply(mw_net* net, const void* const* params, const void* x,

@@ -65,9 +65,25 @@ struct mw_net {
   // (theta = apply_params[l]) instead of g
   const void* const* apply_params = nullptr;
   float apply_lr = 0.f;
+  // mw_sweep_bucket_events: the forward sweep records bucket_events[b] on its stream once the
+  // gradients of layers [b * bucket_layers, (b + 1) * bucket_layers) are enqueued
+  std::vector<cudaEvent_t> bucket_events;
+  int bucket_layers = 0;
+  int buckets_recorded = 0;     // during a sweep: events already recorded
 };
 
 namespace mw {
+// called by a sweep after the launch that completes the gradients of all layers < done_layers
+inline void record_buckets(mw_net* n, int done_layers, cudaStream_t s) {
+  if (n->bucket_layers <= 0) return;
+  const int nb = (int)n->bucket_events.size();
+  while (n->buckets_recorded < nb) {
+    const int last = (n->buckets_recorded + 1) * n->bucket_layers;      // one past the bucket's last layer
+    if ((last < n->L ? last : n->L) > done_layers) break;
+    cudaEventRecord(n->bucket_events[(size_t)n->buckets_recorded], s);
+    ++n->buckets_recorded;
+  }
+}
 inline bool is_reseed(const mw_net* n, int l_out) {   // l_out = index of x_l / h_l, 1..L-1
   const int K = n->opts.reseed_every;
   return K > 0 && l_out > 0 && l_out < n->L && (l_out % K) == 0;

@@ -1235,7 +1235,10 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
     TensorState* t = state_of(c);
     const bool pair = net_pair(c);
     const int per_layer = chain_entries_per_layer(c, pair);
-    const int chunk = (kTcMaxProgram - 4) / per_layer;
+    int chunk = (kTcMaxProgram - 4) / per_layer;
+    // gradient buckets (mw_sweep_bucket_events): a launch per bucket, so that each bucket's event
+    // can be recorded while the later layers still run
+    if (n->bucket_layers > 0 && n->bucket_layers < chunk) chunk = n->bucket_layers;
     if (chunk >= 1) {
       const int nchunks = (L + chunk - 1) / chunk;
       std::vector<const void*> key = key_of(c, params, x, nullptr, dW);
@@ -1254,7 +1257,10 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
         }
         t->sweep_key[v] = key;
       }
-      for (TcProgram* pr : progs) MW_TRY(tc_program_launch(pr, c.st, c.s));
+      for (int i = 0; i < nchunks; ++i) {
+        MW_TRY(tc_program_launch(progs[(size_t)i], c.st, c.s));
+        record_buckets(n, (i + 1) * chunk < L ? (i + 1) * chunk : L, c.s);
+      }
       return MW_OK;
     }
   }
@@ -1282,6 +1288,7 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
       g[cnt++] = weight_vjp_product(c, c.at<__nv_bfloat16>(lay.gzp[(l - 1) & 1]), xbuf(l - 1),
                                     (float*)dW[l - 1], l - 1);
     if (cnt) MW_TRY(run(c, g, cnt));
+    record_buckets(n, l, c.s);      // launch l carries the weight vjp of layer l - 1
   }
   return MW_OK;
 }

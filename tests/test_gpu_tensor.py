@@ -97,3 +97,35 @@ def test_bf16_pair_sizes_gradients_skipped():
     ref = O.backprop(p.layers, p.params, p.x, p.target, p.loss, masks=masks)
     for l in keep:
         assert O.normwise_error(dW[l].double().cpu().numpy(), ref["dW"][l]) <= 2e-2, l
+
+
+@pytest.mark.parametrize("kind", ["pair", "fp32_small"])
+def test_bucket_events_and_single_rank_data_parallel_step(kind):
+    """mw_sweep_bucket_events: the sweep records one event per bucket of layers (a launch per bucket
+    where the sweep runs as chains); the data-parallel step built on it, with one rank, returns the
+    gradients of the plain step bit for bit."""
+    import torch
+    from paper_2402_14212_b200 import binding as mwb
+    from paper_2402_14212_b200 import data_parallel as dp
+    if kind == "pair":
+        p = S.sweep_mlp(seed=6, depth=7, n=256, batch=256, reseed_every=3, prec=S.BF16)
+    else:
+        p = S.deep_mlp(seed=6, depth=5, n=128, batch=40, reseed_every=2, prec=S.F32)
+    net = mwb.net_for(p, backend="tensor")
+    params, x, target = mwb.to_device(p)
+    ws = net.alloc_workspace("moonwalk")
+    g0 = net.input_cotangent(params, x, target, ws)
+    plain = [d.clone() for d in net.forward_sweep(params, x, g0, ws)]
+    step = dp.DataParallelStep(net, p.loss, world=1, layers_per_bucket=3)
+    assert len(step.events) == (len(p.layers) + 2) // 3
+    dW = [torch.zeros_like(d) for d in plain]
+    step.step(params, x, target, ws, g0, dW)
+    torch.cuda.synchronize()
+    assert net.last_device_status(ws)[0] == 0
+    assert all(e.query() for e in step.events)
+    for a, b in zip(plain, dW):
+        assert torch.equal(a, b)
+    net.set_bucket_events(0)
+    again = net.forward_sweep(params, x, g0, ws)
+    for a, b in zip(plain, again):
+        assert torch.equal(a, b)
