@@ -314,6 +314,7 @@ class Bench:
         self.dW = [torch.empty(w.shape, dtype=self.net.grad_dtype(), device=dev) for w in self.params]
         self.loss = torch.zeros(1, dtype=torch.float64, device=dev)
         self.stream = torch.cuda.current_stream()
+        self.dp = None
 
     def cotangent(self):
         self.net.input_cotangent(self.params, self.x, self.target, self.ws, g0_out=self.g0,
@@ -323,8 +324,17 @@ class Bench:
         self.net.forward_sweep(self.params, self.x, self.g0, self.ws, dW_out=self.dW)
 
     def step(self):
+        if self.dp is not None:
+            self.dp.step(self.params, self.x, self.target, self.ws, self.g0, self.dW, loss_out=self.loss)
+            return
         self.cotangent()
         self.sweep()
+
+    def enable_data_parallel(self, world, layers_per_bucket=8):
+        """--parallel dp: this rank's net holds one shard of the batch; the step all-reduces the
+        gradients bucket by bucket on a side stream while the sweep runs (data_parallel.py)."""
+        from paper_2402_14212_b200 import data_parallel
+        self.dp = data_parallel.DataParallelStep(self.net, self.p.loss, world, layers_per_bucket, device=self.dev)
 
     def warm(self, n):
         for _ in range(n):
@@ -461,7 +471,15 @@ def run_ours(args):
     if args.no_coop:
         mwb.set_cooperative_launch(False)
     p = workload(args.workload, depth=args.depth, block=args.frag_block)
+    global_batch = p.batch
+    if args.parallel == "dp":
+        # the batch of the workload is the GLOBAL batch: this rank keeps its shard (strong scaling)
+        from paper_2402_14212_b200 import data_parallel
+        lo, hi = data_parallel.shard_bounds(p.batch, rank, world)
+        p.x, p.target, p.batch = p.x[lo:hi], p.target[lo:hi], hi - lo
     b = Bench(p, args, dev)
+    if args.parallel == "dp":
+        b.enable_data_parallel(world)
     net = b.net
     mw_bytes, bp_bytes, (mw_res, bp_res) = net.workspace_bytes()
     warm = max(args.warmup, 3)
@@ -482,7 +500,7 @@ def run_ours(args):
     launches = (mwb.launch_count() - launches0) // max(1, args.blocks)
     clocks = sampler.stop()
     ms = statistics.median(blocks)
-    value, ms_max = aggregate_replicas(ms, p.batch, args.steps, world, dev)
+    value, ms_max = aggregate_replicas(ms, p.batch, args.steps, world, dev)   # shards or replicas: all samples
     step_ms = ms_max / args.steps
 
     reps = min(args.steps, 5)
@@ -554,12 +572,14 @@ def run_ours(args):
         sm = clocks.get("sm_mhz")
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": warm, "ms_per_step": step_ms,
-                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "higher_is_better": True, "scaling": "strong" if args.parallel == "dp" else "weak",
+                "vs_baseline": None,
                 "dtype": {"f64": "f64", "f32": "f32 (bf16x3 split on tensor cores, fp32 accumulate)",
                           "bf16_f32acc": "bf16 (fp32 accumulate)"}[p.prec]
                 if net_backend_is_tensor(net) else ("f64" if p.prec == "f64" else "f32"),
                 "data": "synthetic", "config": describe(p),
-                "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                "parallelism": (f"data parallel x{world}: global batch {global_batch} in equal shards, bucketed all-reduce of dW"
+                                if args.parallel == "dp" else (f"replicas x{world}" if world > 1 else "single GPU")),
                 "l2_policy": "working set (weights, inverses, gradients: GBs) far above the 126 MB L2; no flush between steps",
                 "timed_blocks": {"count": len(blocks), "steps_each": args.steps, "ms": blocks, "reported": "median"},
                 "clocks": clocks, "ms_per_step_x_sm_mhz": (step_ms * sm) if sm else None,
@@ -788,6 +808,9 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--blocks", type=int, default=5,
                     help="repetitions of the timed block of --steps steps (the median block is reported)")
+    ap.add_argument("--parallel", default="replicas", choices=["replicas", "dp"],
+                    help="N > 1: independent replicas (default), or dp = the batch sharded over the ranks with a "
+                         "bucketed all-reduce of the gradients overlapped with the sweep (not measured on hardware here)")
     ap.add_argument("--no-coop", action="store_true",
                     help="program launches without the cooperative attribute (for launch lists under a profiler)")
     ap.add_argument("--quick", action="store_true",
