@@ -361,6 +361,15 @@ int32_t mw_set_cooperative_launch(int32_t enable);
  * setting.  Process-wide; for comparisons and tests (the paper has no counterpart). */
 int32_t mw_set_bulk_epilogue(int32_t enable);
 
+/* Dense nets with resident inverses run the forward sweep (Algorithm 1) as chains: per block of
+ * batch rows, layer l's recompute and vijp wait only for the same rows of layer l - 1, all inside
+ * one launch (enable = 1, the default): on CTA pairs with row blocks of 256 when a layer has at
+ * least 32 such tiles per product, else on single CTAs with row blocks of 128.  2: CTA pairs
+ * whenever the sizes allow.  0: one launch per layer instead.  Returns the previous setting.
+ * Process-wide; read when a net's sweep is first built (a net keeps the form it
+ * started with); for comparisons and tests (the paper has no counterpart). */
+int32_t mw_set_sweep_chains(int32_t enable);
+
 #ifdef __cplusplus
 }
 #endif

@@ -87,6 +87,8 @@ def lib() -> C.CDLL:
         L.mw_set_pair_mode.argtypes = [i32]
         L.mw_set_pair_mode.restype = i32
         L.mw_selftest_bounded_wait.argtypes = [vp, sz, C.c_uint32, C.POINTER(i32), vp]
+        L.mw_set_sweep_chains.argtypes = [i32]
+        L.mw_set_sweep_chains.restype = i32
         L.mw_set_bulk_epilogue.argtypes = [i32]
         L.mw_set_bulk_epilogue.restype = i32
         L.mw_set_cooperative_launch.argtypes = [i32]
@@ -297,6 +299,12 @@ def selftest_bounded_wait(limit_ms: int = 5, stream=None) -> int:
     _check(lib().mw_selftest_bounded_wait(p, scratch.numel() - 256, int(limit_ms), C.byref(out),
                                           _stream_handle(stream)), "mw_selftest_bounded_wait")
     return int(out.value)
+
+
+def set_sweep_chains(mode: int) -> int:
+    """Forward sweep of dense nets as per-row-block chains in one launch (1: form chosen by tile
+    count, 2: CTA pairs whenever possible) or as a launch per layer (0).  Returns the old mode."""
+    return int(lib().mw_set_sweep_chains(int(mode)))
 
 
 def set_bulk_epilogue(enable: bool) -> bool:

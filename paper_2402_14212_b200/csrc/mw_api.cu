@@ -714,6 +714,14 @@ extern "C" int32_t mw_set_pair_mode(int32_t enable) { return tc_set_pair_mode(en
 extern "C" int32_t mw_set_merge_orders(int32_t enable) { return tc_set_merge_orders(enable); }
 extern "C" int32_t mw_set_cooperative_launch(int32_t enable) { return tc_set_cooperative(enable); }
 extern "C" int32_t mw_set_bulk_epilogue(int32_t enable) { return tc_set_bulk_epilogue(enable); }
+namespace mw {
+int g_sweep_chains = 1;
+}
+extern "C" int32_t mw_set_sweep_chains(int32_t enable) {
+  const int32_t old = mw::g_sweep_chains;
+  mw::g_sweep_chains = enable < 0 ? 0 : enable > 2 ? 2 : enable;
+  return old;
+}
 
 extern "C" void mw_profile_begin(void) { tc_profile_begin(); }
 

@@ -12,6 +12,8 @@ enum { MW_PROG_PHASE1 = 0, MW_PROG_PHASE2, MW_PROG_BP_FWD, MW_PROG_BP_BWD, MW_PR
 // variants of a program: which home of the Newton-Schulz iterate it starts from (0, 1), cold or
 // refreshing (+2).  A training loop alternates between two of them; each is built once.
 constexpr int kProgVariants = 4;
+// 1: dense nets that qualify run the forward sweep as chained programs (mw_set_sweep_chains)
+extern int g_sweep_chains;
 struct TensorState {
   TcMapCache* cache = nullptr;
   TcProgram* prog[MW_PROG_COUNT][kProgVariants] = {};

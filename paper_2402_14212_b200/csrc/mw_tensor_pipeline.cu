@@ -956,9 +956,6 @@ mw_status sweep_chain_program(const Ctx& c0, TcProgram* pr, int l0, int l1, cons
   return a.status;
 }
 
-// 1: nets that qualify run the sweep as chained programs (0: one launch per layer, for comparisons)
-int g_sweep_chains = 1;
-
 inline uint32_t __float_as_uint_host(float f) {
   uint32_t u;
   memcpy(&u, &f, sizeof(u));
@@ -1233,7 +1230,10 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
   // as chains of products inside program launches, as many layers per launch as the table holds.
   if (use_programs(n) && chain_sizes(n) && g_sweep_chains) {
     TensorState* t = state_of(c);
-    const bool pair = net_pair(c);
+    // The chains of one layer are (B / 256) x (d / 256) pair tiles per product; with few of them
+    // most pairs wait on the chain's critical path, and tiles of 128 rows on single CTAs (four
+    // times as many, each half as long) finish the sweep sooner.
+    const bool pair = net_pair(c) && (g_sweep_chains == 2 || (c.B / 256) * (c.dim / 256) >= 32);
     const int per_layer = chain_entries_per_layer(c, pair);
     int chunk = (kTcMaxProgram - 4) / per_layer;
     // gradient buckets (mw_sweep_bucket_events): a launch per bucket, so that each bucket's event

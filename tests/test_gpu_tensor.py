@@ -60,29 +60,35 @@ def test_config5_full_width(depth, resident):
     assert len(errs) == depth
 
 
-@pytest.mark.parametrize("pair", [True, False])
+@pytest.mark.parametrize("form", ["pair_chains", "default", "single", "launch_per_layer"])
 @pytest.mark.parametrize("n,depth,batch,K", [(256, 8, 256, 4), (512, 10, 512, 4), (256, 9, 768, 3)])
-def test_bf16_mixed_pair_sizes(n, depth, batch, K, pair):
+def test_bf16_mixed_pair_sizes(n, depth, batch, K, form):
     """Sizes at which every product qualifies for the CTA-pair form (batch and width multiples of
-    256): the sweep then runs as chains of row blocks inside program launches.  The same nets with
-    the pair form switched off take the one-launch-per-layer path; both against the oracle."""
+    256).  The sweep runs as chains of row blocks inside program launches: on CTA pairs
+    (forced here, since so few tiles would choose single CTAs), in the form the tile count
+    chooses (Phases I-II on pairs, the sweep on single CTAs), with the pair form switched off
+    everywhere, and as one launch per layer; each against the oracle."""
     from paper_2402_14212_b200 import binding as mwb
-    old = mwb.set_pair_mode(pair)
+    old_pair = mwb.set_pair_mode(form != "single")
+    old_chains = mwb.set_sweep_chains({"pair_chains": 2, "launch_per_layer": 0}.get(form, 1))
     try:
         p = S.mixed_mlp(seed=4, depth=depth, n=n, batch=batch, reseed_every=K, prec=S.BF16)
         check_problem(p, 2e-2, backend="tensor", exact_masks=False, tau=2e-2)
     finally:
-        mwb.set_pair_mode(old)
+        mwb.set_pair_mode(old_pair)
+        mwb.set_sweep_chains(old_chains)
 
 
-def test_bf16_pair_sizes_gradients_skipped():
-    """dW_out entries left out (gradients need not coexist): the chained sweep drops the weight vjp
-    of those layers and still carries the cotangent through them."""
+@pytest.mark.parametrize("chains", [1, 2])
+def test_bf16_pair_sizes_gradients_skipped(chains):
+    """dW_out entries left out (gradients need not coexist): the chained sweep (on single CTAs and
+    on CTA pairs) drops the weight vjp of those layers and still carries the cotangent through."""
     import torch
     from paper_2402_14212_b200 import binding as mwb
     from oracle import moonwalk_oracle as O
     from parity_util import oracle_masks_from_words
     p = S.sweep_mlp(seed=5, depth=7, n=256, batch=256, reseed_every=3, prec=S.BF16)
+    old_chains = mwb.set_sweep_chains(chains)
     net = mwb.net_for(p, backend="tensor")
     params, x, target = mwb.to_device(p)
     ws = net.alloc_workspace("moonwalk")
@@ -90,7 +96,10 @@ def test_bf16_pair_sizes_gradients_skipped():
     keep = [0, 2, 3, 6]
     dW = [torch.zeros(w.shape, dtype=torch.float32, device="cuda") if l in keep else None
           for l, w in enumerate(params)]
-    net.forward_sweep(params, x, g0, ws, dW_out=dW)
+    try:
+        net.forward_sweep(params, x, g0, ws, dW_out=dW)
+    finally:
+        mwb.set_sweep_chains(old_chains)
     code, detail = net.last_device_status(ws)
     assert code == 0, detail
     masks = oracle_masks_from_words(p, [net.export_masks(ws, l) for l in range(len(p.layers))])
