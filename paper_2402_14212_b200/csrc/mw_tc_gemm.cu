@@ -102,7 +102,8 @@ struct alignas(64) TcProblem {
 constexpr int kMaxProgram = 768;   // products of one program launch
 
 struct alignas(64) TcGroupParams {
-  int nprob, total_units, stages, pad0;
+  int nprob, total_units, stages;
+  int sched_len;              // program launch with a unit schedule: entries per CTA (pair)
   uint32_t stage_bytes, pad1;
   uint64_t wait_limit_ns;     // bound of every device-side wait
   uint32_t epi_stage_off;     // byte offset (from the first stage) of the epilogue's transposition
@@ -110,6 +111,7 @@ struct alignas(64) TcGroupParams {
   DeviceStatus* st;
   const TcProblem* table;     // program launch: the products live in global memory ...
   unsigned int* done;         // ... and count their finished tiles here (zero at launch)
+  const int* sched;           // [CTAs or pairs][sched_len] units of each, in list order, -1 ends; or null
   TcProblem prob[kTcMaxGroup];
 };
 
@@ -702,15 +704,21 @@ __device__ __forceinline__ void decode_unit(const TcProblem* probs, const int* u
   w.kb1 = e < P.num_kb ? e : P.num_kb;
 }
 
-// Units of this CTA (pair form: of this pair of CTAs): round r takes index r*G + c (even r) or
-// r*G + G-1-c (odd r); a program launch takes r*G + c throughout, so that one CTA never holds two
-// units of one short product (they would run one after the other and hold up everything that
-// waits for that product).
-// (Handing units out dynamically in list order was tried and is slower: CTAs pile up behind the
-// one product that is not complete yet.)
+// Units of this CTA (pair form: of this pair of CTAs).  Grouped launch: round r takes index
+// r*G + c (even r) or r*G + G-1-c (odd r).  Program launch: the host's schedule (balance_units)
+// when there is one, else r*G + c throughout, so that one CTA never holds two units of one short
+// product (they would run one after the other and hold up everything that waits for it).
+// (Handing units out at run time from a counter, in list order, was tried twice and is not
+// faster: CTAs pile up behind the one product that is not complete yet.)
 template <bool kProgram, bool kPair>
 __device__ __forceinline__ int next_unit(const TcGroupParams& p, int& r) {
   const int G = (int)(gridDim.x >> (kPair ? 1 : 0)), c = (int)(blockIdx.x >> (kPair ? 1 : 0));
+  if (kProgram && p.sched) {
+    if (r >= p.sched_len) return -1;
+    const int u = __ldg(p.sched + (size_t)c * p.sched_len + r);
+    ++r;
+    return u;
+  }
   while (r * G < p.total_units) {
     const int u = r * G + (((r & 1) && !kProgram) ? G - 1 - c : c);
     ++r;
@@ -1888,6 +1896,9 @@ struct TcProgram {
   bool uploaded = false;
   bool pair = false;          // every product in the pair form (clusters of two CTAs)
   std::vector<unsigned> target;   // arrivals that complete each table entry (product or group)
+  std::vector<int> sched;         // units of every CTA (pair), see balance_units
+  int sched_slots = 0, sched_len = 0;
+  bool balance = false;           // hand the units out by the schedule instead of round-robin
 };
 
 TcProgram* tc_program_create() { return new TcProgram(); }
@@ -1903,7 +1914,12 @@ void tc_program_begin(TcProgram* pr, void* table_dev, unsigned int* done_dev, bo
   pr->table_dev = table_dev;
   pr->done_dev = done_dev;
   pr->uploaded = false;
+  pr->sched.clear();
+  pr->sched_slots = pr->sched_len = 0;
+  pr->balance = false;
 }
+
+void tc_program_balance(TcProgram* pr, bool on) { pr->balance = on; }
 
 int tc_program_add(TcProgram* pr, TcMapCache* cache, const TcGemm& d, const int* deps, int ndep,
                    mw_status* status, int group) {
@@ -1961,7 +1977,50 @@ int tc_program_add_group(TcProgram* pr) {
   return (int)pr->table.size() - 1;
 }
 
-size_t tc_program_table_bytes(int products) { return (size_t)products * sizeof(TcProblem); }
+// room for the unit schedule behind the table
+constexpr size_t kSchedBytes = 256 * 1024;
+size_t tc_program_table_bytes(int products) { return (size_t)products * sizeof(TcProblem) + kSchedBytes + 256; }
+
+// Rough length of one unit in SM cycles: its tcgen05 instructions (128 cycles each at 256
+// accumulator columns, a floor of 88 below) or its epilogue (fp32 tiles cost about twice the
+// bf16 planes), whichever is longer.
+static double unit_cycles(const TcProblem& P) {
+  const int nkb = P.split > 1 ? P.kb_per_split : P.num_kb;
+  const double main_loop = (double)nkb * P.nops * (BK / 16) * (P.bn >= 256 ? 128.0 : 88.0);
+  const double per_elem = P.epi.out_f32 ? 0.25 : 0.12;
+  const double epilogue = 3000.0 + per_elem * 128.0 * P.bn;
+  return (main_loop > epilogue ? main_loop : epilogue) + 1000.0;
+}
+
+// Units of a program launch differ in length (a vijp tile of three-term operands against a
+// weight vjp tile), and whatever waits for a product waits for its slowest tile.  For programs
+// that ask for it (tc_program_balance: the chained sweep on single CTAs, where it measured 15 %
+// faster; on CTA pairs and in the Newton-Schulz programs it measured slower than round-robin)
+// the schedule gives each unit, in list order, to the CTA (pair) with the least work so far; every
+// CTA still meets its units in list order, which is all the waiting needs (a unit's operands come
+// from earlier units, each of which is the oldest unfinished one of some CTA or already done).
+static void balance_units(TcProgram* pr, int slots) {
+  std::vector<double> load((size_t)slots, 0.0);
+  std::vector<std::vector<int>> mine((size_t)slots);
+  for (const TcProblem& P : pr->table) {
+    if (P.unit_count <= 0) continue;
+    const double cyc = unit_cycles(P);
+    for (int i = 0; i < P.unit_count; ++i) {
+      int best = 0;
+      for (int g = 1; g < slots; ++g)
+        if (load[(size_t)g] < load[(size_t)best]) best = g;
+      load[(size_t)best] += cyc;
+      mine[(size_t)best].push_back(P.unit_begin + i);
+    }
+  }
+  size_t len = 0;
+  for (const auto& m : mine) len = m.size() > len ? m.size() : len;
+  pr->sched_len = (int)len + 1;
+  pr->sched_slots = slots;
+  pr->sched.assign((size_t)slots * pr->sched_len, -1);
+  for (int g = 0; g < slots; ++g)
+    for (size_t k = 0; k < mine[(size_t)g].size(); ++k) pr->sched[(size_t)g * pr->sched_len + k] = mine[(size_t)g][k];
+}
 
 mw_status tc_program_launch(TcProgram* pr, DeviceStatus* st, cudaStream_t s) {
   const int nprob = (int)pr->table.size();
@@ -1997,7 +2056,20 @@ mw_status tc_program_launch(TcProgram* pr, DeviceStatus* st, cudaStream_t s) {
   // products wait for one another inside the launch: every CTA must be resident (cooperative launch)
   const int slots = pr->pair ? max_pairs(smem) : sm_count();
   if (slots < 1) return MW_ERR_CUDA;
-  const int grid = (pr->total_units < slots ? pr->total_units : slots) * (pr->pair ? 2 : 1);
+  const int used = pr->total_units < slots ? pr->total_units : slots;
+  const int grid = used * (pr->pair ? 2 : 1);
+  prm.sched = nullptr;
+  prm.sched_len = 0;
+  if (pr->balance && pr->total_units > used) {
+    if (pr->sched_slots != used) balance_units(pr, used);
+    const size_t bytes = pr->sched.size() * sizeof(int);
+    if (bytes <= kSchedBytes) {
+      char* dst = static_cast<char*>(pr->table_dev) + (((size_t)nprob * sizeof(TcProblem) + 255) & ~(size_t)255);
+      MW_CUDA_OK(cudaMemcpyAsync(dst, pr->sched.data(), bytes, cudaMemcpyHostToDevice, s));
+      prm.sched = reinterpret_cast<const int*>(dst);
+      prm.sched_len = pr->sched_len;
+    }
+  }
   const cudaError_t e = launch_kernel(true, pr->pair, grid, smem, s, prm);
   ++g_launch_count;
   if (prof) cudaEventRecord(prof_event(), s);

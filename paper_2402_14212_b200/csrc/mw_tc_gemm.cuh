@@ -181,6 +181,8 @@ int tc_program_add(TcProgram*, TcMapCache* cache, const TcGemm& g, const int* de
                    mw_status* status, int group = -1);
 // an entry without work that stands for "all products added to it"; add it before its members
 int tc_program_add_group(TcProgram*);
+// units handed to the CTAs by a load-balanced schedule (call after tc_program_begin; default off)
+void tc_program_balance(TcProgram*, bool on);
 size_t tc_program_table_bytes(int products);
 mw_status tc_program_launch(TcProgram*, DeviceStatus* st, cudaStream_t s);
 constexpr int kTcMaxProgram = 768;

@@ -882,6 +882,7 @@ mw_status sweep_chain_program(const Ctx& c0, TcProgram* pr, int l0, int l1, cons
   const int L = n->L, d = c.dim;
   const int rb = pair ? 256 : 128, mt = c.B / rb;
   tc_program_begin(pr, c.at<char>(lay.prog_table[0]), c.at<unsigned int>(lay.prog_done[0]), pair);
+  tc_program_balance(pr, !pair);
   Adder a{c, pr};
   auto xbuf = [&](int l) -> const __nv_bfloat16* {
     return l == 0 ? x0p : c.at<__nv_bfloat16>(lay.xp[l % c.nx]);
