@@ -27,7 +27,10 @@ Eq. "conv-vjp" for h', computed with the paper's relation
 w_centre h'_{i'} = h_{i'} - TransposeConv(h', w~)_{i'} used as a fixed-point
 iteration with the whole C x C centre tap as the pivot block; a convolution
 that meets Lemma 1 (stride above padding, triangular anchor tap) takes the
-lemma's elimination itself, which is exact.
+lemma's elimination itself, which is exact; a dense layer may be parameterised
+by the triangular factors of its weight (W = L U, one array holding both), the
+paper's constrained-layer idea carried to dense layers: its vijp is two
+substitutions, its parameter cotangent the chain rule through the product.
 
 Pinned by tests/test_oracle_*.py: finite differences, Moonwalk == Backprop,
 vjp(vijp(h)) == h, closed-form leaky-ReLU inverse, explicit-Jacobian brute
@@ -169,13 +172,37 @@ def conv1d_weight_vjp(x, gz, k, stride, pad):
     return dw
 
 
+def is_lu(layer):
+    """A dense layer whose parameter array holds the factors of its weight (see lu_factors)."""
+    return layer.kind == DENSE and bool(getattr(layer, "lu", False))
+
+
+def lu_factors(p):
+    """LU-parameterised dense layer: the paper constrains its convolutions so that the vijp is
+    cheap by construction (Section "Constrained Convolutions"); the same idea for a square dense
+    layer is to learn the triangular factors of W instead of W.  One n x n array p holds both:
+    L = I + strictly lower part of p (unit diagonal, not a parameter), U = upper part of p with
+    its diagonal.  The layer's weight is W = L U, invertible whenever diag(U) has no zero."""
+    p = np.asarray(p, dtype=np.float64)
+    return np.tril(p, -1) + np.eye(p.shape[0]), np.triu(p)
+
+
+def lu_weight(p):
+    L, U = lu_factors(p)
+    return L @ U
+
+
+def dense_weight(layer, w):
+    return lu_weight(w) if is_lu(layer) else w
+
+
 def linear_forward(layer, w, x):
     if layer.kind == CONV1D:
         return conv1d_forward(x, w, layer.stride, layer.pad)
     if layer.kind == CONV2D:
         return conv_forward(x, w, layer.stride, layer.pad)
     x2 = x.reshape(x.shape[0], -1)
-    return x2 @ w.T
+    return x2 @ dense_weight(layer, w).T
 
 
 def linear_vjp_input(layer, w, g, in_shape):
@@ -184,16 +211,22 @@ def linear_vjp_input(layer, w, g, in_shape):
         return transpose_conv1d(g, w, layer.W, layer.stride, layer.pad)
     if layer.kind == CONV2D:
         return transpose_conv(g, w, (layer.H, layer.W), layer.stride, layer.pad)
-    return (g @ w).reshape(in_shape)
+    return (g @ dense_weight(layer, w)).reshape(in_shape)
 
 
-def linear_vjp_param(layer, x, g):
-    """vjp(f, theta, g) of the linear part: Eq. "g_i"."""
+def linear_vjp_param(layer, x, g, w=None):
+    """vjp(f, theta, g) of the linear part: Eq. "g_i".  An LU-parameterised layer needs its
+    parameters `w`: with G = g^T x the cotangent of W = L U, the chain rule through the product
+    gives dJ/dL = G U^T on the strictly lower entries and dJ/dU = L^T G on the upper ones."""
     if layer.kind == CONV1D:
         return conv1d_weight_vjp(x, g, layer.k, layer.stride, layer.pad)
     if layer.kind == CONV2D:
         return conv_weight_vjp(x, g, layer.k, layer.stride, layer.pad)
-    return g.T @ x.reshape(x.shape[0], -1)
+    G = g.T @ x.reshape(x.shape[0], -1)
+    if is_lu(layer):
+        L, U = lu_factors(w)
+        return np.tril(G @ U.T, -1) + np.triu(L.T @ G)
+    return G
 
 
 # ----------------------------------------------------------------------------
@@ -202,6 +235,22 @@ def linear_vjp_param(layer, x, g):
 def vijp_dense(w, h):
     """The g with g W = h, by an LU solve with partial pivoting (never forms W^-1)."""
     return np.linalg.solve(w.T, h.reshape(h.shape[0], -1).T).T
+
+
+def vijp_dense_lu(p, h):
+    """The g with g L U = h for the factors held in p, by two substitutions and no inverse:
+    first y U = h column by column from the left (U upper triangular), then g L = y column by
+    column from the right (L unit lower triangular)."""
+    L, U = lu_factors(p)
+    h2 = h.reshape(h.shape[0], -1)
+    n = h2.shape[1]
+    y = np.zeros_like(h2, dtype=np.float64)
+    for j in range(n):
+        y[:, j] = (h2[:, j] - y[:, :j] @ U[:j, j]) / U[j, j]
+    g = np.zeros_like(y)
+    for j in range(n - 1, -1, -1):
+        g[:, j] = y[:, j] - g[:, j + 1:] @ L[j + 1:, j]
+    return g
 
 
 def vijp_conv_fixed_point(layer, w, h, tol=1e-14, max_iters=400, iters=None, trace=None):
@@ -340,6 +389,8 @@ def vijp_linear(layer, w, h, conv_iters=None):
         if layer.stride > layer.pad:
             return vijp_conv_submersive(layer, w, h)
         return vijp_conv_fixed_point(layer, w, h, iters=conv_iters)
+    if is_lu(layer):
+        return vijp_dense_lu(w, h)
     return vijp_dense(w, h)
 
 
@@ -400,7 +451,7 @@ def backprop(layers, params, x0, target, loss, masks=None):
     dW = [None] * L
     for l in range(L - 1, -1, -1):
         gz = hs[l + 1] * act_derivative(layers[l], ms[l])
-        dW[l] = linear_vjp_param(layers[l], xs[l], gz)
+        dW[l] = linear_vjp_param(layers[l], xs[l], gz, params[l])
         hs[l] = linear_vjp_input(layers[l], params[l], gz, xs[l].shape)
     return dict(loss=J, dW=dW, h=hs, g0=hs[0], masks=ms, x=xs, z=zs)
 
@@ -521,7 +572,7 @@ def forward_sweep(layers, params, x0, g0, store, conv_iters=None, apply=None):
             hn = vijp_leaky(layer, m, gz)
         else:
             hn = gz
-        dW[l] = linear_vjp_param(layer, x, gz)
+        dW[l] = linear_vjp_param(layer, x, gz, w)
         if apply is not None:
             apply(l, dW[l])
         x = act_forward(z, layer, m)

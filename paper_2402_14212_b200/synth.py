@@ -44,6 +44,7 @@ class Layer:
     k: int = 0
     stride: int = 1
     pad: int = 0
+    lu: bool = False    # dense: the parameter array holds the factors of W = L U (L unit lower, U upper)
 
     def out_hw(self):
         wo = (self.W + 2 * self.pad - self.k) // self.stride + 1
@@ -134,6 +135,26 @@ def deep_mlp(seed=0, depth=64, n=1024, batch=256, reseed_every=4, prec=F32) -> P
     w = lambda rng, n, l: orthogonal(rng, n) + 0.05 * rng.standard_normal((n, n)) / np.sqrt(n)
     return dense_chain("deep_mlp", n, depth, batch, prec, LOSS_MSE_MEAN, [ACT_LEAKY], 0.1, w,
                        seed, reseed_every)
+
+
+def lu_mlp(seed=0, depth=64, n=1024, batch=256, reseed_every=4, prec=F32) -> Problem:
+    """Dense leaky-ReLU MLP whose layers are parameterised by triangular factors (`Layer.lu`):
+    the array of layer l holds L below its diagonal (unit diagonal implied) and U on and above it,
+    L = I + 0.3*N(0,1)/sqrt(n) strictly below, U = diag(+-(1 + 0.1*u)) + 0.3*N(0,1)/sqrt(n) strictly
+    above, u uniform in [-1, 1] (W = L U has singular values in about [0.6, 1.5]).  Sizes of
+    config 2."""
+    rng = np.random.default_rng(seed)
+    layers, params = [], []
+    for l in range(depth):
+        lo = np.tril(rng.standard_normal((n, n)), -1) * (0.3 / np.sqrt(n))
+        up = np.triu(rng.standard_normal((n, n)), 1) * (0.3 / np.sqrt(n))
+        d = np.where(rng.random(n) < 0.5, -1.0, 1.0) * (1.0 + 0.1 * (2.0 * rng.random(n) - 1.0))
+        layers.append(Layer(DENSE, ACT_LEAKY, 0.1, n, n, lu=True))
+        params.append(round_storage(lo + up + np.diag(d), prec))
+    x = round_storage(rng.standard_normal((batch, n)), prec)
+    t = round_storage(rng.standard_normal((batch, n)), F32 if prec == BF16 else prec)
+    return Problem("lu_mlp", layers, params, x, t, LOSS_MSE_MEAN, prec, batch,
+                   reseed_every=reseed_every, seed=seed)
 
 
 def mixed_mlp(seed=0, depth=128, n=2048, batch=512, reseed_every=4, prec=BF16) -> Problem:

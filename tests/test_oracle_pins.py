@@ -479,3 +479,82 @@ def test_generators_recipes():
     assert not np.array_equal(S.tiny_mlp(seed=1).x, p1.x)
     c = S.submersive_cnn(seed=0, depth=1, C=8, H=4, W=4, batch=1)
     assert c.params[0].shape == (3, 3, 8, 8) and abs(c.params[0][1, 1, 0, 0] - 1.0) < 0.1
+
+
+# ----------------------------------------------------------------------------
+# LU-parameterised dense layers (the constrained-layer idea carried to dense layers)
+# ----------------------------------------------------------------------------
+def _lu_chain(n, depth, batch, seed, acts=(S.ACT_LEAKY, S.ACT_RELU), K=0):
+    p = S.lu_mlp(seed=seed, depth=depth, n=n, batch=batch, reseed_every=K, prec=S.F64)
+    for l, layer in enumerate(p.layers):
+        layer.act = acts[l % len(acts)]
+        layer.slope = 0.1 if layer.act == S.ACT_LEAKY else 0.0
+    return p
+
+
+def test_lu_factors_hand_made_example():
+    p = np.array([[2.0, 3.0, 4.0], [5.0, 6.0, 7.0], [8.0, 9.0, 10.0]])
+    L, U = O.lu_factors(p)
+    assert np.array_equal(L, [[1, 0, 0], [5, 1, 0], [8, 9, 1]])
+    assert np.array_equal(U, [[2, 3, 4], [0, 6, 7], [0, 0, 10]])
+    # W = L U multiplied out by hand
+    assert np.array_equal(O.lu_weight(p), [[2, 3, 4], [10, 21, 27], [16, 78, 105]])
+
+
+def test_lu_net_is_the_dense_net_of_its_products():
+    p = _lu_chain(10, 4, 6, seed=3)
+    dense_layers = [S.Layer(S.DENSE, l.act, l.slope, l.n_in, l.n_out) for l in p.layers]
+    W = []
+    for a in p.params:                      # W_ij = sum_k L_ik U_kj, element by element
+        n = a.shape[0]
+        w = np.zeros((n, n))
+        for i in range(n):
+            for j in range(n):
+                for k in range(min(i, j) + 1):
+                    w[i, j] += (1.0 if k == i else a[i, k]) * a[k, j]
+        W.append(w)
+    lu = O.backprop(p.layers, p.params, p.x, p.target, p.loss)
+    de = O.backprop(dense_layers, W, p.x, p.target, p.loss)
+    assert abs(lu["loss"] - de["loss"]) <= 1e-14 * abs(de["loss"])
+    assert np.allclose(lu["g0"], de["g0"], rtol=1e-12, atol=1e-15)
+    for l, a in enumerate(p.params):
+        L, U = O.lu_factors(a)
+        G = de["dW"][l]                     # cotangent of W: the chain rule through W = L U
+        assert np.allclose(np.tril(lu["dW"][l], -1), np.tril(G @ U.T, -1), rtol=1e-11, atol=1e-14)
+        assert np.allclose(np.triu(lu["dW"][l]), np.triu(L.T @ G), rtol=1e-11, atol=1e-14)
+
+
+def test_lu_param_vjp_matches_finite_differences():
+    p = _lu_chain(6, 3, 4, seed=1)
+    check_off_kinks(p.layers, p.params, p.x)
+    ref = O.backprop(p.layers, p.params, p.x, p.target, p.loss)
+    for l in range(3):
+        for idx in [(4, 1), (5, 0), (2, 2), (0, 0), (1, 4), (0, 5), (3, 2), (2, 3)]:   # below, on, above the diagonal
+            fd = fd_grad(p.layers, p.params, p.x, p.target, p.loss, l, idx)
+            assert abs(fd - ref["dW"][l][idx]) <= 1e-7 * max(1.0, abs(fd)), (l, idx)
+
+
+def test_lu_vijp_is_right_inverse_without_forming_it():
+    rng = np.random.default_rng(5)
+    p = _lu_chain(14, 1, 5, seed=2)
+    a = p.params[0]
+    h = rng.standard_normal((5, 14))
+    g = O.vijp_dense_lu(a, h)
+    W = O.lu_weight(a)
+    assert np.allclose(g @ W, h, atol=1e-12)
+    assert np.allclose(g, O.vijp_dense(W, h), atol=1e-12)
+    assert np.allclose(O.vijp_linear(p.layers[0], a, h), g, atol=0)
+
+
+@pytest.mark.parametrize("K", [0, 2])
+def test_lu_moonwalk_equals_backprop_and_sgd_step(K):
+    p = _lu_chain(24, 6, 8, seed=4, K=K)
+    ref = O.backprop(p.layers, p.params, p.x, p.target, p.loss)
+    mw = O.moonwalk(p.layers, p.params, p.x, p.target, p.loss, reseed_every=K)
+    assert np.array_equal(np.asarray(ref["g0"]), np.asarray(mw["g0"]))
+    for l in range(6):
+        assert O.normwise_error(mw["dW"][l], ref["dW"][l]) < 1e-9
+    new = O.moonwalk_sgd_step(p.layers, p.params, p.x, p.target, p.loss, 0.05, reseed_every=K)
+    for l in range(6):
+        assert np.allclose(new[l], p.params[l] - 0.05 * ref["dW"][l], rtol=1e-9, atol=1e-12)
+        assert np.all(O.trainable_entries(p.layers[l], p.params[l]) == 1.0)
