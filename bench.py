@@ -11,7 +11,7 @@ over depth (`depth_sweep`); --quick leaves them out.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
 
-Workloads: sweep_mlp --depth D (default, config 5), deep_mlp (config 2), deep_mlp_small, mixed_mlp
+Workloads: sweep_mlp --depth D (default, config 5), deep_mlp (config 2), lu_mlp (config 2's sizes, LU-parameterised layers), deep_mlp_small, mixed_mlp
 (config 4), submersive_cnn (config 3), tiny_mlp (config 1); the paper's own convolutional experiments
 strided_cnn [--depth D] (stride-2 submersive layers) and fragmental_cnn1d [--depth D --frag-block B]
 (1-D, fragmental checkpoints), their bf16 forms strided_cnn_bf16 / fragmental_cnn1d_bf16, and
@@ -56,6 +56,9 @@ def workload(name: str, seed: int = 0, depth: int = 0, block: int = 0):
         return S.deep_mlp(seed=seed, depth=8, n=256, batch=128)
     if name == "mixed_mlp":
         return S.mixed_mlp(seed=seed)
+    if name == "lu_mlp":
+        # config 2's sizes with every layer parameterised by the triangular factors of its weight
+        return S.lu_mlp(seed=seed, depth=depth or 64)
     if name == "sweep_mlp":
         return S.sweep_mlp(seed=seed, depth=depth or 32, pool=4)
     if name == "submersive_cnn":
@@ -164,7 +167,7 @@ class ClockSampler:
 # sample of the workload -- the first `batch` samples through the first `layers` layers -- and
 # scale the result to the full depth (cost is linear in depth); (0, 0) = the whole workload.
 ORACLE_SAMPLE = {
-    "sweep_mlp": (32, 1), "mixed_mlp": (32, 4), "deep_mlp": (32, 0), "submersive_cnn": (2, 8),
+    "sweep_mlp": (32, 1), "mixed_mlp": (32, 4), "deep_mlp": (32, 0), "lu_mlp": (32, 0), "submersive_cnn": (2, 8),
     "strided_cnn": (1, 0), "strided_cnn_bf16": (1, 0), "fragmental_cnn1d": (1, 0),
     "fragmental_cnn1d_bf16": (1, 0),
 }
@@ -600,7 +603,7 @@ def run_ours(args):
 
 
 # the other baseline configurations and the paper's two experiments, reported beside the main line
-PER_CONFIG = ["deep_mlp", "submersive_cnn", "mixed_mlp", "strided_cnn", "fragmental_cnn1d"]
+PER_CONFIG = ["deep_mlp", "lu_mlp", "submersive_cnn", "mixed_mlp", "strided_cnn", "fragmental_cnn1d"]
 
 
 def measure_config(name, args, dev):

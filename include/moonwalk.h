@@ -105,6 +105,18 @@ typedef struct {
   int32_t frag_block;      /* MW_CONV1D nets: Phase II keeps the output cotangent of every
                               convolution at the first k - 1 positions of each block of this
                               many positions (2..64, dividing W); Phase III rebuilds the rest  */
+  int32_t lu_param;        /* 1: every dense layer is parameterised by the triangular factors of
+                              its weight, the paper's constrained-layer idea (Section "Constrained
+                              Convolutions") carried to dense layers: params[l] ([n][n]) holds L
+                              strictly below the diagonal (unit diagonal implied) and U on and
+                              above it, the layer's weight is W = L U, and gradients come back in
+                              the same layout (dJ/dL below, dJ/dU on and above the diagonal).
+                              W^-1 = U^-1 L^-1 is then built from the factors by block
+                              substitution, exactly: no Newton-Schulz iteration, no convergence
+                              domain; a zero on the diagonal of U is the only failure
+                              (MW_ERR_NOT_SUBMERSIVE).  Tensor-core backend, MW_F32, widths that
+                              are multiples of 128, resident_inverse = 1, warm_inverse = 0;
+                              mw_forward_sweep_apply is not available.  0: params[l] is W.      */
 } mw_net_opts;
 
 /* Build a host-side description.  `batch` is fixed per net.

@@ -44,7 +44,7 @@ class NetOpts(C.Structure):
     _fields_ = [("prec", C.c_int32), ("loss", C.c_int32), ("reseed_every", C.c_int32),
                 ("conv_vijp_iters", C.c_int32), ("backend", C.c_int32),
                 ("inverse_iters", C.c_int32), ("resident_inverse", C.c_int32),
-                ("warm_inverse", C.c_int32), ("frag_block", C.c_int32)]
+                ("warm_inverse", C.c_int32), ("frag_block", C.c_int32), ("lu_param", C.c_int32)]
 
 
 _lib = None
@@ -141,12 +141,16 @@ class Net:
                  conv_vijp_iters: int = 10, backend: str = "auto", inverse_iters: int = 0,
                  resident_inverse: bool = True, frag_block: int = 0, warm_inverse: bool = False):
         self.layers = list(layers)
+        # LU-parameterised dense layers (Layer.lu): all layers of a net or none
+        lu = [bool(getattr(l, "lu", False)) for l in self.layers]
+        if any(lu) and not all(lu):
+            raise ValueError("a net is LU-parameterised in every layer or in none")
         self.batch = int(batch)
         self.prec, self.loss = prec, loss
         self._h = C.c_void_p()
         opts = NetOpts(PREC[prec], LOSS[loss], int(reseed_every), int(conv_vijp_iters),
                        BACKEND[backend], int(inverse_iters), int(bool(resident_inverse)),
-                       int(bool(warm_inverse)), int(frag_block))
+                       int(bool(warm_inverse)), int(frag_block), int(any(lu)))
         descs = make_layer_descs(self.layers)
         _check(lib().mw_net_create(descs, len(self.layers), self.batch, C.byref(opts),
                                    C.byref(self._h)), "mw_net_create")

@@ -160,6 +160,14 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
     return MW_ERR_INVALID_ARG;
   if (opts->backend < MW_BACKEND_AUTO || opts->backend > MW_BACKEND_TENSOR) return MW_ERR_INVALID_ARG;
   if (opts->warm_inverse != 0 && opts->warm_inverse != 1) return MW_ERR_INVALID_ARG;
+  if (opts->lu_param != 0 && opts->lu_param != 1) return MW_ERR_INVALID_ARG;
+  if (opts->lu_param) {
+    // triangular factors as parameters: dense nets on the tensor cores in MW_F32, inverses resident
+    if (opts->prec != MW_F32 || opts->backend == MW_BACKEND_SIMT || !opts->resident_inverse || opts->warm_inverse)
+      return MW_ERR_UNSUPPORTED;
+    for (int l = 0; l < n_layers; ++l)
+      if (layers[l].kind != MW_DENSE || layers[l].n_in % 128 != 0) return MW_ERR_UNSUPPORTED;
+  }
   for (int l = 0; l < n_layers; ++l) {
     if (layers[l].kind < MW_DENSE || layers[l].kind > MW_CONV1D) return MW_ERR_INVALID_ARG;
     if (!valid_layer(layers[l], l, n_layers)) return MW_ERR_UNSUPPORTED;
@@ -219,6 +227,10 @@ extern "C" mw_status mw_net_create(const mw_layer_desc* layers, int32_t n_layers
   }
   if (opts->backend == MW_BACKEND_AUTO) n->backend = tensor_ok ? MW_BACKEND_TENSOR : MW_BACKEND_SIMT;
   else n->backend = opts->backend;
+  if (opts->lu_param && n->backend != MW_BACKEND_TENSOR) {
+    delete n;
+    return MW_ERR_UNSUPPORTED;
+  }
   if (n->backend == MW_BACKEND_SIMT && opts->prec == MW_BF16_F32ACC) {
     delete n;
     return MW_ERR_UNSUPPORTED;
@@ -581,7 +593,7 @@ extern "C" mw_status mw_forward_sweep_apply(mw_net* net, const void* const* para
                                             const void* g0, double lr, void* const* params_out,
                                             void* workspace, size_t workspace_bytes, void* stream) {
   if (!net || !params || !params_out) return MW_ERR_INVALID_ARG;
-  if (net->backend != MW_BACKEND_TENSOR || net->opts.prec != MW_F32) return MW_ERR_UNSUPPORTED;
+  if (net->backend != MW_BACKEND_TENSOR || net->opts.prec != MW_F32 || net->opts.lu_param) return MW_ERR_UNSUPPORTED;
   net->apply_params = params;
   net->apply_lr = (float)lr;
   const mw_status r = mw_forward_sweep(net, params, x, g0, params_out, workspace, workspace_bytes, stream);

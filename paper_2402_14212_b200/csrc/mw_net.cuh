@@ -39,6 +39,10 @@ struct Layout {
   Region ns_sumsq, ns_scale;
   Region prog_table[3], prog_done[3];        // product tables and completion counters of program launches
   Region split[3];                           // K-split meeting places of concurrently running products
+  // LU-parameterised dense nets: term planes of one layer's L, U, L^-1, U^-1, two block-substitution
+  // temporaries, the planes of one gradient, two fp32 products of the gradient's chain rule, and
+  // the inverted diagonal blocks of every layer (fp32)
+  Region lu_l, lu_u, lu_t, lu_s, lu_y[2], lu_g, lu_a, lu_b, lu_diag;
 };
 
 }  // namespace mw

@@ -257,6 +257,11 @@ Ctx make_ctx(mw_net* n, const Layout& lay, void* ws, cudaStream_t s) {
 // weight operand of layer l (MW_F32: split planes in the workspace, made here when `make`;
 // bf16: the caller's array itself)
 mw_status weight_planes(const Ctx& c, int l, const void* W, bool make, const __nv_bfloat16** out) {
+  if (c.n->opts.lu_param) {
+    // the parameters are the factors: the planes of W = L U were made by lu_prepare
+    *out = c.at<__nv_bfloat16>(c.lay->w_planes[l]);
+    return MW_OK;
+  }
   if (c.n->opts.prec == MW_F32) {
     __nv_bfloat16* p = c.at<__nv_bfloat16>(c.lay->w_planes[l]);
     if (make) MW_TRY(split_planes((const float*)W, c.nn, p, 3, c.nn, c.s));
@@ -400,6 +405,228 @@ mw_status clear_split_counters(const Ctx& c) {
       MW_CUDA_OK(cudaMemsetAsync(c.at<char>(c.lay->split[i]), 0, kTcSplitCounterBytes, c.s));
   return MW_OK;
 }
+
+// ---- LU-parameterised dense layers -------------------------------------------------------------
+// params[l] holds L strictly below the diagonal (unit diagonal implied) and U on and above it;
+// W = L U.  What Newton-Schulz does for a free W is done here exactly, from the structure:
+// L^-1 and U^-1 by block substitution (diagonal blocks of 128 inverted on the CUDA cores in
+// fp64, then [[A, 0], [C, D]]^-1 = [[A^-1, 0], [-D^-1 C A^-1, D^-1]] level by level on the
+// tensor cores), W^-1 = U^-1 L^-1 and W = L U as two more products, everything as three bf16
+// term planes (fp32-accurate).  The gradient of W that the sweep forms is mapped to the factors
+// by the chain rule: dJ/dL = G U^T below the diagonal, dJ/dU = L^T G on and above it.
+constexpr int kLuBlock = 128;
+
+__device__ __forceinline__ void split3(float v, __nv_bfloat16* p, int64_t stride) {
+  const __nv_bfloat16 a = __float2bfloat16_rn(v);
+  const float r1 = v - __bfloat162float(a);
+  const __nv_bfloat16 b = __float2bfloat16_rn(r1);
+  const __nv_bfloat16 d = __float2bfloat16_rn(r1 - __bfloat162float(b));
+  p[0] = a; p[stride] = b; p[2 * stride] = d;
+}
+
+// Inverses of the diagonal blocks of L (which = 0) and U (which = 1) of up to kMaxGroup layers:
+// one CTA per block, thread j owns column j of the inverse (forward substitution; an upper block
+// is handled as the lower block it becomes when rows and columns are reversed).
+// out: [layer][which][n / 128][128][128] fp32, row-major blocks.
+__global__ void __launch_bounds__(kLuBlock)
+lu_diag_inverse_kernel(PtrBatch Ps, int n, float* __restrict__ out, DeviceStatus* st, int layer0) {
+  const int blk = blockIdx.x, which = blockIdx.y, lay = blockIdx.z;
+  const float* P = static_cast<const float*>(Ps.p[lay]);
+  const int o = blk * kLuBlock, j = threadIdx.x, r = kLuBlock - 1;
+  // the block as a lower triangular matrix M: L's block itself (unit diagonal), or U's block with
+  // rows and columns reversed, M[i][k] = U[r-i][r-k], whose inverse is U^-1 reversed the same way
+  double x[kLuBlock];
+  bool bad = false;
+  for (int i = 0; i < j; ++i) x[i] = 0.0;
+  for (int i = j; i < kLuBlock; ++i) {
+    double s = i == j ? 1.0 : 0.0;
+    for (int k = j; k < i; ++k) {
+      const double m = which == 0 ? (double)P[(int64_t)(o + i) * n + o + k]
+                                  : (double)P[(int64_t)(o + r - i) * n + o + r - k];
+      s -= m * x[k];
+    }
+    const double d = which == 0 ? 1.0 : (double)P[(int64_t)(o + r - i) * n + o + r - i];
+    if (!(d != 0.0) || !(d - d == 0.0)) { bad = true; x[i] = 0.0; }
+    else x[i] = s / d;
+  }
+  if (bad) record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)(layer0 + lay), (unsigned)blk, 5u, 0u);
+  float* dst = out + (((int64_t)lay * 2 + which) * (n / kLuBlock) + blk) * kLuBlock * kLuBlock;
+  for (int i = 0; i < kLuBlock; ++i) {
+    if (which == 0) dst[i * kLuBlock + j] = (float)x[i];
+    else dst[(r - i) * kLuBlock + (r - j)] = (float)x[i];
+  }
+}
+
+// term planes of L (unit lower) and U (upper) of one layer; with `diag` also the planes of L^-1
+// and U^-1 holding their inverted diagonal blocks and zeros elsewhere
+__global__ void __launch_bounds__(256)
+lu_split_kernel(const float* __restrict__ P, int n, __nv_bfloat16* __restrict__ Lp,
+                __nv_bfloat16* __restrict__ Up, const float* __restrict__ diag,
+                __nv_bfloat16* __restrict__ Tp, __nv_bfloat16* __restrict__ Sp) {
+  const int64_t nn = (int64_t)n * n;
+  for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < nn; e += (int64_t)gridDim.x * 256) {
+    const int i = (int)(e / n), j = (int)(e - (int64_t)i * n);
+    const float v = P[e];
+    split3(i > j ? v : (i == j ? 1.f : 0.f), Lp + e, nn);
+    split3(i <= j ? v : 0.f, Up + e, nn);
+    if (diag) {
+      const int bi = i / kLuBlock, bj = j / kLuBlock;
+      float t = 0.f, u = 0.f;
+      if (bi == bj) {
+        const int64_t off = (int64_t)bi * kLuBlock * kLuBlock + (i - bi * kLuBlock) * kLuBlock + (j - bj * kLuBlock);
+        t = diag[off];
+        u = diag[(int64_t)(n / kLuBlock) * kLuBlock * kLuBlock + off];
+      }
+      split3(t, Tp + e, nn);
+      split3(u, Sp + e, nn);
+    }
+  }
+}
+
+// dP = (a below the diagonal, b on and above it)
+__global__ void __launch_bounds__(256)
+lu_combine_kernel(const float* __restrict__ a, const float* __restrict__ b, int n, float* __restrict__ out) {
+  const int64_t nn = (int64_t)n * n;
+  for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < nn; e += (int64_t)gridDim.x * 256) {
+    const int i = (int)(e / n), j = (int)(e - (int64_t)i * n);
+    out[e] = i > j ? a[e] : b[e];
+  }
+}
+
+// a block of an n x n matrix kept as three term planes, as an operand / as an output
+TcOperand lu_block(const Ctx& c, const __nv_bfloat16* planes, int r0, int c0, int rows, int cols, bool mn) {
+  TcOperand o = operand(planes + (int64_t)r0 * c.dim + c0, rows, cols, 3, mn);
+  o.plane_stride = c.nn;
+  o.ld = c.dim;
+  return o;
+}
+TcEpilogue lu_block_out(const Ctx& c, __nv_bfloat16* planes, int r0, int c0, float alpha) {
+  TcEpilogue e;
+  e.mode = TC_EPI_PLAIN;
+  e.alpha = alpha;
+  e.planes = planes + (int64_t)r0 * c.dim + c0;
+  e.n_planes = 3;
+  e.plane_stride = c.nn;
+  e.ld = c.dim;
+  return e;
+}
+TcGemm lu_product(const TcOperand& A, const TcOperand& B, int M, int N, int K, const TcEpilogue& e) {
+  TcGemm g;
+  g.A = A; g.B = B; g.M = M; g.N = N; g.K = K; g.epi = e;
+  g.split_k = 1;
+  return g;
+}
+mw_status lu_run(const Ctx& c, const std::vector<TcGemm>& g) {
+  for (size_t i = 0; i < g.size(); i += kTcMaxGroup) {
+    const size_t k = g.size() - i < (size_t)kTcMaxGroup ? g.size() - i : (size_t)kTcMaxGroup;
+    MW_TRY(run(c, g.data() + i, (int)k));
+  }
+  return MW_OK;
+}
+
+// Fills w_planes[l] (W = L U) of every layer and, with `inverses`, inv[l] (W^-1 = U^-1 L^-1).
+mw_status lu_prepare(const Ctx& c, const void* const* params, bool inverses) {
+  const Layout& lay = *c.lay;
+  const int L = c.n->L, d = c.dim, nb = d / kLuBlock;
+  __nv_bfloat16* Lp = c.at<__nv_bfloat16>(lay.lu_l);
+  __nv_bfloat16* Up = c.at<__nv_bfloat16>(lay.lu_u);
+  __nv_bfloat16* Tp = inverses ? c.at<__nv_bfloat16>(lay.lu_t) : nullptr;
+  __nv_bfloat16* Sp = inverses ? c.at<__nv_bfloat16>(lay.lu_s) : nullptr;
+  float* diag = inverses ? c.at<float>(lay.lu_diag) : nullptr;
+  const int64_t diag_layer = 2 * (int64_t)nb * kLuBlock * kLuBlock;
+  if (inverses) {
+    for (int l0 = 0; l0 < L; l0 += kMaxGroup) {
+      const int G = (L - l0) < kMaxGroup ? (L - l0) : kMaxGroup;
+      PtrBatch ps{};
+      for (int g = 0; g < G; ++g) ps.p[g] = params[l0 + g];
+      lu_diag_inverse_kernel<<<dim3((unsigned)nb, 2u, (unsigned)G), kLuBlock, 0, c.s>>>(
+          ps, d, diag + (int64_t)l0 * diag_layer, c.st, l0);
+      MW_TRY(launch_ok());
+    }
+  }
+  int64_t bx = (c.nn + 255) / 256;
+  if (bx > 1184) bx = 1184;
+  for (int l = 0; l < L; ++l) {
+    lu_split_kernel<<<(unsigned)bx, 256, 0, c.s>>>((const float*)params[l], d, Lp, Up,
+                                                   inverses ? diag + (int64_t)l * diag_layer : nullptr, Tp, Sp);
+    MW_TRY(launch_ok());
+    if (inverses) {
+      __nv_bfloat16* Yl = c.at<__nv_bfloat16>(lay.lu_y[0]);
+      __nv_bfloat16* Yu = c.at<__nv_bfloat16>(lay.lu_y[1]);
+      // segments [seg[i], seg[i+1]) whose diagonal blocks of L^-1 and U^-1 are complete
+      std::vector<int> seg;
+      for (int b = 0; b <= nb; ++b) seg.push_back(b * kLuBlock);
+      while (seg.size() > 2) {
+        std::vector<TcGemm> first, second;
+        std::vector<int> merged;
+        merged.push_back(seg[0]);
+        for (size_t i = 0; i + 2 < seg.size(); i += 2) {
+          const int a0 = seg[i], a1 = seg[i + 1], a2 = seg[i + 2], m1 = a1 - a0, m2 = a2 - a1;
+          // L^-1[a1:a2, a0:a1] = -D^-1 C A^-1
+          first.push_back(lu_product(lu_block(c, Lp, a1, a0, m2, m1, false), lu_block(c, Tp, a0, a0, m1, m1, true),
+                                     m2, m1, m1, lu_block_out(c, Yl, a1, a0, 1.f)));
+          second.push_back(lu_product(lu_block(c, Tp, a1, a1, m2, m2, false), lu_block(c, Yl, a1, a0, m2, m1, true),
+                                      m2, m1, m2, lu_block_out(c, Tp, a1, a0, -1.f)));
+          // U^-1[a0:a1, a1:a2] = -A^-1 B D^-1
+          first.push_back(lu_product(lu_block(c, Up, a0, a1, m1, m2, false), lu_block(c, Sp, a1, a1, m2, m2, true),
+                                     m1, m2, m2, lu_block_out(c, Yu, a0, a1, 1.f)));
+          second.push_back(lu_product(lu_block(c, Sp, a0, a0, m1, m1, false), lu_block(c, Yu, a0, a1, m1, m2, true),
+                                      m1, m2, m1, lu_block_out(c, Sp, a0, a1, -1.f)));
+          merged.push_back(a2);
+        }
+        if (merged.back() != seg.back()) merged.push_back(seg.back());   // an odd segment waits a level
+        MW_TRY(lu_run(c, first));
+        MW_TRY(lu_run(c, second));
+        seg.swap(merged);
+      }
+    }
+    std::vector<TcGemm> last;
+    {
+      TcEpilogue e;
+      e.mode = TC_EPI_PLAIN;
+      e.planes = c.at<__nv_bfloat16>(lay.w_planes[l]);
+      e.n_planes = 3;
+      e.plane_stride = c.nn;
+      last.push_back(lu_product(operand(Lp, d, d, 3, false), operand(Up, d, d, 3, true), d, d, d, e));
+    }
+    if (inverses) {
+      TcEpilogue e;
+      e.mode = TC_EPI_PLAIN;
+      e.planes = c.at<__nv_bfloat16>(lay.inv[l]);
+      e.n_planes = c.pr.ph;
+      e.plane_stride = c.nn;
+      last.push_back(lu_product(operand(Sp, d, d, 3, false), operand(Tp, d, d, 3, true), d, d, d, e));
+    }
+    MW_TRY(lu_run(c, last));
+  }
+  return MW_OK;
+}
+
+// dW[l] holds G = dJ/dW of layer l; replaces it by the gradient of the factors
+mw_status lu_map_gradient(const Ctx& c, const void* P, float* dW) {
+  const Layout& lay = *c.lay;
+  const int d = c.dim;
+  __nv_bfloat16* Lp = c.at<__nv_bfloat16>(lay.lu_l);
+  __nv_bfloat16* Up = c.at<__nv_bfloat16>(lay.lu_u);
+  __nv_bfloat16* Gp = c.at<__nv_bfloat16>(lay.lu_g);
+  int64_t bx = (c.nn + 255) / 256;
+  if (bx > 1184) bx = 1184;
+  lu_split_kernel<<<(unsigned)bx, 256, 0, c.s>>>((const float*)P, d, Lp, Up, nullptr, nullptr, nullptr);
+  MW_TRY(launch_ok());
+  MW_TRY(split_planes(dW, c.nn, Gp, 3, c.nn, c.s));
+  std::vector<TcGemm> g;
+  TcEpilogue ea, eb;
+  ea.mode = eb.mode = TC_EPI_PLAIN;
+  ea.out_f32 = c.at<float>(lay.lu_a);
+  eb.out_f32 = c.at<float>(lay.lu_b);
+  // G U^T: B operand [N][K] = U itself;  L^T G: A operand MN-major = L as [K][M], B = G as [K][N]
+  g.push_back(lu_product(operand(Gp, d, d, 3, false), operand(Up, d, d, 3, false), d, d, d, ea));
+  g.push_back(lu_product(operand(Lp, d, d, 3, true), operand(Gp, d, d, 3, true), d, d, d, eb));
+  MW_TRY(lu_run(c, g));
+  lu_combine_kernel<<<(unsigned)bx, 256, 0, c.s>>>(c.at<float>(lay.lu_a), c.at<float>(lay.lu_b), d, dW);
+  return launch_ok();
+}
+
 
 // forward pass shared by Phase I and backprop's forward; y (fp32 network output) lands in lay.z
 mw_status forward_pass(const Ctx& c, const void* const* params, const void* x, bool store_acts) {
@@ -604,6 +831,7 @@ NsFeed make_feed(const Ctx& c, const void* const* params, bool warm, int side0) 
 // ---- whole phases as one launch ("programs") -------------------------------------------------
 // needs every layer's weight and inverse planes resident, and room in the product table
 bool use_programs(const mw_net* n) {
+  if (n->opts.lu_param) return false;      // LU-parameterised nets: one launch per layer
   return n->opts.resident_inverse != 0 && 5 * (n->L + 1) <= kTcMaxProgram;
 }
 
@@ -1094,6 +1322,22 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
       for (int l = 0; l < L; ++l) lay.w_planes[l] = slot;
     }
   }
+  if (n->opts.lu_param) {
+    lay.lu_l = b.take(6 * nn);
+    lay.lu_u = b.take(6 * nn);
+    lay.lu_g = b.take(6 * nn);
+    lay.lu_a = b.take(4 * nn);
+    lay.lu_b = b.take(4 * nn);
+    if (!backprop) {
+      lay.lu_t = b.take(6 * nn);
+      lay.lu_s = b.take(6 * nn);
+      for (int i = 0; i < 2; ++i) lay.lu_y[i] = b.take(6 * nn);
+      lay.lu_diag = b.take(sizeof(float) * 2 * (size_t)L * d * kLuBlock);
+      for (int l = 0; l < L; ++l) lay.inv[l] = b.take(2 * (size_t)pr.ph * nn);
+    }
+    lay.total = b.cur;
+    return;
+  }
   if (!backprop) {
     if (use_programs(n)) {
       // the inverses stay where the last Newton-Schulz step wrote them (ns_r)
@@ -1170,7 +1414,9 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
     if (n->opts.warm_inverse) n->warm_ws = ws;
     return MW_OK;
   }
-  if (resident) {
+  if (n->opts.lu_param) {
+    MW_TRY(lu_prepare(c, params, true));      // W and W^-1 of every layer from its factors
+  } else if (resident) {
     const int G = ns_group(n);
     for (int l = 0; l < L; l += G) MW_TRY(newton_schulz_group(c, l, (L - l) < G ? (L - l) : G, params));
   }
@@ -1289,6 +1535,8 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
       g[cnt++] = weight_vjp_product(c, c.at<__nv_bfloat16>(lay.gzp[(l - 1) & 1]), xbuf(l - 1),
                                     (float*)dW[l - 1], l - 1);
     if (cnt) MW_TRY(run(c, g, cnt));
+    // LU-parameterised layer: the gradient of W just formed becomes the gradient of the factors
+    if (n->opts.lu_param && l >= 1 && dW[l - 1]) MW_TRY(lu_map_gradient(c, params[l - 1], (float*)dW[l - 1]));
     record_buckets(n, l, c.s);      // launch l carries the weight vjp of layer l - 1
   }
   return MW_OK;
@@ -1311,6 +1559,7 @@ mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, c
     MW_TRY(split_all_weights(c, params));
     MW_TRY(forward_program(c, params, x, true));
   } else {
+    if (n->opts.lu_param) MW_TRY(lu_prepare(c, params, false));
     MW_TRY(forward_pass(c, params, x, true));
   }
   MW_TRY(loss_and_top(c, target, loss_out, false));
@@ -1349,6 +1598,7 @@ mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, c
                          d, d, c.B, e, 2);
     }
     if (cnt) MW_TRY(run(c, g, cnt));
+    if (n->opts.lu_param && dW[l]) MW_TRY(lu_map_gradient(c, params[l], (float*)dW[l]));
     cur ^= 1;
   }
   return MW_OK;
