@@ -457,46 +457,73 @@ lu_diag_inverse_kernel(PtrBatch Ps, int n, float* __restrict__ out, DeviceStatus
   }
 }
 
-// term planes of L (unit lower) and U (upper) of one layer; with `diag` also the planes of L^-1
-// and U^-1 holding their inverted diagonal blocks and zeros elsewhere
+// term planes of L (unit lower) and U (upper) of the layers of a chunk (blockIdx.y), laid out
+// [layer][plane][n][n]; with `diag` also the planes of L^-1 and U^-1 holding their inverted
+// diagonal blocks and zeros elsewhere
 __global__ void __launch_bounds__(256)
-lu_split_kernel(const float* __restrict__ P, int n, __nv_bfloat16* __restrict__ Lp,
-                __nv_bfloat16* __restrict__ Up, const float* __restrict__ diag,
-                __nv_bfloat16* __restrict__ Tp, __nv_bfloat16* __restrict__ Sp) {
-  const int64_t nn = (int64_t)n * n;
+lu_split_kernel(PtrBatch Ps, int n, __nv_bfloat16* __restrict__ Lp, __nv_bfloat16* __restrict__ Up,
+                const float* __restrict__ diag, __nv_bfloat16* __restrict__ Tp,
+                __nv_bfloat16* __restrict__ Sp) {
+  const int64_t nn = (int64_t)n * n, base = (int64_t)blockIdx.y * 3 * nn;
+  const float* P = static_cast<const float*>(Ps.p[blockIdx.y]);
+  const int nb = n / kLuBlock;
+  if (diag) diag += (int64_t)blockIdx.y * 2 * nb * kLuBlock * kLuBlock;
   for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < nn; e += (int64_t)gridDim.x * 256) {
     const int i = (int)(e / n), j = (int)(e - (int64_t)i * n);
     const float v = P[e];
-    split3(i > j ? v : (i == j ? 1.f : 0.f), Lp + e, nn);
-    split3(i <= j ? v : 0.f, Up + e, nn);
+    split3(i > j ? v : (i == j ? 1.f : 0.f), Lp + base + e, nn);
+    split3(i <= j ? v : 0.f, Up + base + e, nn);
     if (diag) {
       const int bi = i / kLuBlock, bj = j / kLuBlock;
       float t = 0.f, u = 0.f;
       if (bi == bj) {
         const int64_t off = (int64_t)bi * kLuBlock * kLuBlock + (i - bi * kLuBlock) * kLuBlock + (j - bj * kLuBlock);
         t = diag[off];
-        u = diag[(int64_t)(n / kLuBlock) * kLuBlock * kLuBlock + off];
+        u = diag[(int64_t)nb * kLuBlock * kLuBlock + off];
       }
-      split3(t, Tp + e, nn);
-      split3(u, Sp + e, nn);
+      split3(t, Tp + base + e, nn);
+      split3(u, Sp + base + e, nn);
     }
   }
 }
 
-// dP = (a below the diagonal, b on and above it)
+// term planes of the gradients of W of a chunk of layers
 __global__ void __launch_bounds__(256)
-lu_combine_kernel(const float* __restrict__ a, const float* __restrict__ b, int n, float* __restrict__ out) {
-  const int64_t nn = (int64_t)n * n;
+lu_gsplit_kernel(PtrBatch Gs, int64_t nn, __nv_bfloat16* __restrict__ Gp) {
+  const float* G = static_cast<const float*>(Gs.p[blockIdx.y]);
+  const int64_t base = (int64_t)blockIdx.y * 3 * nn;
+  for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < nn; e += (int64_t)gridDim.x * 256)
+    split3(G[e], Gp + base + e, nn);
+}
+
+// dP = (a below the diagonal, b on and above it), per layer of the chunk
+struct OutBatch { void* p[kMaxGroup]; };
+__global__ void __launch_bounds__(256)
+lu_combine_kernel(const float* __restrict__ a, const float* __restrict__ b, int n, OutBatch outs) {
+  const int64_t nn = (int64_t)n * n, base = (int64_t)blockIdx.y * nn;
+  float* out = static_cast<float*>(outs.p[blockIdx.y]);
   for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < nn; e += (int64_t)gridDim.x * 256) {
     const int i = (int)(e / n), j = (int)(e - (int64_t)i * n);
-    out[e] = i > j ? a[e] : b[e];
+    out[e] = i > j ? a[base + e] : b[base + e];
   }
 }
 
-// a block of an n x n matrix kept as three term planes, as an operand / as an output
+// layers whose factors are worked on together (their planes and temporaries: 36 n^2 bytes each)
+int lu_chunk(const mw_net* n) {
+  const size_t d = (size_t)n->layers[0].n_in;
+  size_t g = ((size_t)768 << 20) / (36 * d * d);
+  if (g < 1) g = 1;
+  if (g > 16) g = 16;
+  if (g > (size_t)n->L) g = (size_t)n->L;
+  return (int)g;
+}
+
+// a block of the n x n matrices of G layers kept as [layer][plane][n][n], as an operand / output
+// of a product batched over the layers
 TcOperand lu_block(const Ctx& c, const __nv_bfloat16* planes, int r0, int c0, int rows, int cols, bool mn) {
   TcOperand o = operand(planes + (int64_t)r0 * c.dim + c0, rows, cols, 3, mn);
   o.plane_stride = c.nn;
+  o.batch_planes = 3;
   o.ld = c.dim;
   return o;
 }
@@ -507,12 +534,14 @@ TcEpilogue lu_block_out(const Ctx& c, __nv_bfloat16* planes, int r0, int c0, flo
   e.planes = planes + (int64_t)r0 * c.dim + c0;
   e.n_planes = 3;
   e.plane_stride = c.nn;
+  e.bs_planes = 3 * c.nn;
   e.ld = c.dim;
   return e;
 }
-TcGemm lu_product(const TcOperand& A, const TcOperand& B, int M, int N, int K, const TcEpilogue& e) {
+TcGemm lu_product(const TcOperand& A, const TcOperand& B, int M, int N, int K, const TcEpilogue& e, int batch) {
   TcGemm g;
   g.A = A; g.B = B; g.M = M; g.N = N; g.K = K; g.epi = e;
+  g.batch = batch;
   g.split_k = 1;
   return g;
 }
@@ -524,35 +553,38 @@ mw_status lu_run(const Ctx& c, const std::vector<TcGemm>& g) {
   return MW_OK;
 }
 
-// Fills w_planes[l] (W = L U) of every layer and, with `inverses`, inv[l] (W^-1 = U^-1 L^-1).
+// Fills w_planes[l] (W = L U) of every layer and, with `inverses`, inv[l] (W^-1 = U^-1 L^-1),
+// a chunk of layers at a time: every product below is one entry batched over the chunk.
 mw_status lu_prepare(const Ctx& c, const void* const* params, bool inverses) {
   const Layout& lay = *c.lay;
-  const int L = c.n->L, d = c.dim, nb = d / kLuBlock;
+  const int L = c.n->L, d = c.dim, nb = d / kLuBlock, chunk = lu_chunk(c.n);
   __nv_bfloat16* Lp = c.at<__nv_bfloat16>(lay.lu_l);
   __nv_bfloat16* Up = c.at<__nv_bfloat16>(lay.lu_u);
   __nv_bfloat16* Tp = inverses ? c.at<__nv_bfloat16>(lay.lu_t) : nullptr;
   __nv_bfloat16* Sp = inverses ? c.at<__nv_bfloat16>(lay.lu_s) : nullptr;
+  __nv_bfloat16* Yl = inverses ? c.at<__nv_bfloat16>(lay.lu_y[0]) : nullptr;
+  __nv_bfloat16* Yu = inverses ? c.at<__nv_bfloat16>(lay.lu_y[1]) : nullptr;
   float* diag = inverses ? c.at<float>(lay.lu_diag) : nullptr;
   const int64_t diag_layer = 2 * (int64_t)nb * kLuBlock * kLuBlock;
-  if (inverses) {
-    for (int l0 = 0; l0 < L; l0 += kMaxGroup) {
-      const int G = (L - l0) < kMaxGroup ? (L - l0) : kMaxGroup;
-      PtrBatch ps{};
-      for (int g = 0; g < G; ++g) ps.p[g] = params[l0 + g];
-      lu_diag_inverse_kernel<<<dim3((unsigned)nb, 2u, (unsigned)G), kLuBlock, 0, c.s>>>(
-          ps, d, diag + (int64_t)l0 * diag_layer, c.st, l0);
+  int64_t bx = (c.nn + 255) / 256;
+  if (bx > 296) bx = 296;
+  for (int l0 = 0; l0 < L; l0 += chunk) {
+    const int G = (L - l0) < chunk ? (L - l0) : chunk;
+    PtrBatch ps{};
+    for (int g = 0; g < G; ++g) ps.p[g] = params[l0 + g];
+    // the regions of consecutive layers must lie 3 planes apart for the batched outputs
+    for (int g = 1; g < G; ++g) {
+      if (lay.w_planes[l0 + g].off - lay.w_planes[l0 + g - 1].off != (size_t)(6 * c.nn)) return MW_ERR_WORKSPACE;
+      if (inverses && lay.inv[l0 + g].off - lay.inv[l0 + g - 1].off != (size_t)(6 * c.nn)) return MW_ERR_WORKSPACE;
+    }
+    if (inverses) {
+      lu_diag_inverse_kernel<<<dim3((unsigned)nb, 2u, (unsigned)G), kLuBlock, 0, c.s>>>(ps, d, diag, c.st, l0);
       MW_TRY(launch_ok());
     }
-  }
-  int64_t bx = (c.nn + 255) / 256;
-  if (bx > 1184) bx = 1184;
-  for (int l = 0; l < L; ++l) {
-    lu_split_kernel<<<(unsigned)bx, 256, 0, c.s>>>((const float*)params[l], d, Lp, Up,
-                                                   inverses ? diag + (int64_t)l * diag_layer : nullptr, Tp, Sp);
+    lu_split_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(ps, d, Lp, Up, diag, Tp, Sp);
     MW_TRY(launch_ok());
+    (void)diag_layer;
     if (inverses) {
-      __nv_bfloat16* Yl = c.at<__nv_bfloat16>(lay.lu_y[0]);
-      __nv_bfloat16* Yu = c.at<__nv_bfloat16>(lay.lu_y[1]);
       // segments [seg[i], seg[i+1]) whose diagonal blocks of L^-1 and U^-1 are complete
       std::vector<int> seg;
       for (int b = 0; b <= nb; ++b) seg.push_back(b * kLuBlock);
@@ -564,14 +596,14 @@ mw_status lu_prepare(const Ctx& c, const void* const* params, bool inverses) {
           const int a0 = seg[i], a1 = seg[i + 1], a2 = seg[i + 2], m1 = a1 - a0, m2 = a2 - a1;
           // L^-1[a1:a2, a0:a1] = -D^-1 C A^-1
           first.push_back(lu_product(lu_block(c, Lp, a1, a0, m2, m1, false), lu_block(c, Tp, a0, a0, m1, m1, true),
-                                     m2, m1, m1, lu_block_out(c, Yl, a1, a0, 1.f)));
+                                     m2, m1, m1, lu_block_out(c, Yl, a1, a0, 1.f), G));
           second.push_back(lu_product(lu_block(c, Tp, a1, a1, m2, m2, false), lu_block(c, Yl, a1, a0, m2, m1, true),
-                                      m2, m1, m2, lu_block_out(c, Tp, a1, a0, -1.f)));
+                                      m2, m1, m2, lu_block_out(c, Tp, a1, a0, -1.f), G));
           // U^-1[a0:a1, a1:a2] = -A^-1 B D^-1
           first.push_back(lu_product(lu_block(c, Up, a0, a1, m1, m2, false), lu_block(c, Sp, a1, a1, m2, m2, true),
-                                     m1, m2, m2, lu_block_out(c, Yu, a0, a1, 1.f)));
+                                     m1, m2, m2, lu_block_out(c, Yu, a0, a1, 1.f), G));
           second.push_back(lu_product(lu_block(c, Sp, a0, a0, m1, m1, false), lu_block(c, Yu, a0, a1, m1, m2, true),
-                                      m1, m2, m1, lu_block_out(c, Sp, a0, a1, -1.f)));
+                                      m1, m2, m1, lu_block_out(c, Sp, a0, a1, -1.f), G));
           merged.push_back(a2);
         }
         if (merged.back() != seg.back()) merged.push_back(seg.back());   // an odd segment waits a level
@@ -581,54 +613,57 @@ mw_status lu_prepare(const Ctx& c, const void* const* params, bool inverses) {
       }
     }
     std::vector<TcGemm> last;
-    {
-      TcEpilogue e;
-      e.mode = TC_EPI_PLAIN;
-      e.planes = c.at<__nv_bfloat16>(lay.w_planes[l]);
-      e.n_planes = 3;
-      e.plane_stride = c.nn;
-      last.push_back(lu_product(operand(Lp, d, d, 3, false), operand(Up, d, d, 3, true), d, d, d, e));
-    }
-    if (inverses) {
-      TcEpilogue e;
-      e.mode = TC_EPI_PLAIN;
-      e.planes = c.at<__nv_bfloat16>(lay.inv[l]);
-      e.n_planes = c.pr.ph;
-      e.plane_stride = c.nn;
-      last.push_back(lu_product(operand(Sp, d, d, 3, false), operand(Tp, d, d, 3, true), d, d, d, e));
-    }
+    last.push_back(lu_product(lu_block(c, Lp, 0, 0, d, d, false), lu_block(c, Up, 0, 0, d, d, true), d, d, d,
+                              lu_block_out(c, c.at<__nv_bfloat16>(lay.w_planes[l0]), 0, 0, 1.f), G));
+    if (inverses)
+      last.push_back(lu_product(lu_block(c, Sp, 0, 0, d, d, false), lu_block(c, Tp, 0, 0, d, d, true), d, d, d,
+                                lu_block_out(c, c.at<__nv_bfloat16>(lay.inv[l0]), 0, 0, 1.f), G));
     MW_TRY(lu_run(c, last));
   }
   return MW_OK;
 }
 
-// dW[l] holds G = dJ/dW of layer l; replaces it by the gradient of the factors
-mw_status lu_map_gradient(const Ctx& c, const void* P, float* dW) {
+// dW[l] of layers [l0, l1) hold G = dJ/dW; replaces each by the gradient of the layer's factors
+mw_status lu_map_gradients(const Ctx& c, const void* const* params, void* const* dW, int l0, int l1) {
   const Layout& lay = *c.lay;
-  const int d = c.dim;
+  const int d = c.dim, chunk = lu_chunk(c.n);
   __nv_bfloat16* Lp = c.at<__nv_bfloat16>(lay.lu_l);
   __nv_bfloat16* Up = c.at<__nv_bfloat16>(lay.lu_u);
   __nv_bfloat16* Gp = c.at<__nv_bfloat16>(lay.lu_g);
   int64_t bx = (c.nn + 255) / 256;
-  if (bx > 1184) bx = 1184;
-  lu_split_kernel<<<(unsigned)bx, 256, 0, c.s>>>((const float*)P, d, Lp, Up, nullptr, nullptr, nullptr);
-  MW_TRY(launch_ok());
-  MW_TRY(split_planes(dW, c.nn, Gp, 3, c.nn, c.s));
-  std::vector<TcGemm> g;
-  TcEpilogue ea, eb;
-  ea.mode = eb.mode = TC_EPI_PLAIN;
-  ea.out_f32 = c.at<float>(lay.lu_a);
-  eb.out_f32 = c.at<float>(lay.lu_b);
-  // G U^T: B operand [N][K] = U itself;  L^T G: A operand MN-major = L as [K][M], B = G as [K][N]
-  g.push_back(lu_product(operand(Gp, d, d, 3, false), operand(Up, d, d, 3, false), d, d, d, ea));
-  g.push_back(lu_product(operand(Lp, d, d, 3, true), operand(Gp, d, d, 3, true), d, d, d, eb));
-  MW_TRY(lu_run(c, g));
-  lu_combine_kernel<<<(unsigned)bx, 256, 0, c.s>>>(c.at<float>(lay.lu_a), c.at<float>(lay.lu_b), d, dW);
-  return launch_ok();
+  if (bx > 296) bx = 296;
+  std::vector<int> todo;
+  for (int l = l0; l < l1; ++l)
+    if (dW[l]) todo.push_back(l);
+  for (size_t t0 = 0; t0 < todo.size(); t0 += (size_t)chunk) {
+    const int G = (int)(todo.size() - t0 < (size_t)chunk ? todo.size() - t0 : (size_t)chunk);
+    PtrBatch ps{}, gs{};
+    OutBatch outs{};
+    for (int g = 0; g < G; ++g) {
+      ps.p[g] = params[todo[t0 + g]];
+      gs.p[g] = dW[todo[t0 + g]];
+      outs.p[g] = dW[todo[t0 + g]];
+    }
+    lu_split_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(ps, d, Lp, Up, nullptr, nullptr, nullptr);
+    MW_TRY(launch_ok());
+    lu_gsplit_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(gs, c.nn, Gp);
+    MW_TRY(launch_ok());
+    TcEpilogue ea, eb;
+    ea.mode = eb.mode = TC_EPI_PLAIN;
+    ea.out_f32 = c.at<float>(lay.lu_a);
+    eb.out_f32 = c.at<float>(lay.lu_b);
+    ea.bs_f32 = eb.bs_f32 = c.nn;
+    std::vector<TcGemm> g;
+    // G U^T: B operand [N][K] = U itself;  L^T G: A operand MN-major = L as [K][M], B = G as [K][N]
+    g.push_back(lu_product(lu_block(c, Gp, 0, 0, d, d, false), lu_block(c, Up, 0, 0, d, d, false), d, d, d, ea, G));
+    g.push_back(lu_product(lu_block(c, Lp, 0, 0, d, d, true), lu_block(c, Gp, 0, 0, d, d, true), d, d, d, eb, G));
+    MW_TRY(lu_run(c, g));
+    lu_combine_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(c.at<float>(lay.lu_a), c.at<float>(lay.lu_b), d, outs);
+    MW_TRY(launch_ok());
+  }
+  return MW_OK;
 }
 
-
-// forward pass shared by Phase I and backprop's forward; y (fp32 network output) lands in lay.z
 mw_status forward_pass(const Ctx& c, const void* const* params, const void* x, bool store_acts) {
   const Layout& lay = *c.lay;
   const int L = c.n->L, d = c.dim;
@@ -831,7 +866,6 @@ NsFeed make_feed(const Ctx& c, const void* const* params, bool warm, int side0) 
 // ---- whole phases as one launch ("programs") -------------------------------------------------
 // needs every layer's weight and inverse planes resident, and room in the product table
 bool use_programs(const mw_net* n) {
-  if (n->opts.lu_param) return false;      // LU-parameterised nets: one launch per layer
   return n->opts.resident_inverse != 0 && 5 * (n->L + 1) <= kTcMaxProgram;
 }
 
@@ -1029,7 +1063,7 @@ const __nv_bfloat16* h_planes(const Ctx& c, int l) {
 
 // W^-1 of layer l as term planes: where the prep left it
 const __nv_bfloat16* inverse_planes(const Ctx& c, int l) {
-  if (use_programs(c.n)) return ns_buffers(c).Xp[c.n->inv_side & 1] + (int64_t)l * 3 * c.nn;
+  if (use_programs(c.n) && !c.n->opts.lu_param) return ns_buffers(c).Xp[c.n->inv_side & 1] + (int64_t)l * 3 * c.nn;
   return c.at<__nv_bfloat16>(c.lay->inv[l]);
 }
 
@@ -1323,16 +1357,17 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     }
   }
   if (n->opts.lu_param) {
-    lay.lu_l = b.take(6 * nn);
-    lay.lu_u = b.take(6 * nn);
-    lay.lu_g = b.take(6 * nn);
-    lay.lu_a = b.take(4 * nn);
-    lay.lu_b = b.take(4 * nn);
+    const size_t G = (size_t)lu_chunk(n);
+    lay.lu_l = b.take(6 * nn * G);
+    lay.lu_u = b.take(6 * nn * G);
+    lay.lu_g = b.take(6 * nn * G);
+    lay.lu_a = b.take(4 * nn * G);
+    lay.lu_b = b.take(4 * nn * G);
     if (!backprop) {
-      lay.lu_t = b.take(6 * nn);
-      lay.lu_s = b.take(6 * nn);
-      for (int i = 0; i < 2; ++i) lay.lu_y[i] = b.take(6 * nn);
-      lay.lu_diag = b.take(sizeof(float) * 2 * (size_t)L * d * kLuBlock);
+      lay.lu_t = b.take(6 * nn * G);
+      lay.lu_s = b.take(6 * nn * G);
+      for (int i = 0; i < 2; ++i) lay.lu_y[i] = b.take(6 * nn * G);
+      lay.lu_diag = b.take(sizeof(float) * 2 * G * d * kLuBlock);
       for (int l = 0; l < L; ++l) lay.inv[l] = b.take(2 * (size_t)pr.ph * nn);
     }
     lay.total = b.cur;
@@ -1387,6 +1422,13 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
   MW_CUDA_OK(cudaMemsetAsync(at<char>(ws, lay.status), 0, 256, s));
   MW_TRY(clear_split_counters(c));
   const bool resident = n->opts.resident_inverse != 0;
+  if (use_programs(n) && n->opts.lu_param) {
+    // LU-parameterised layers: W and W^-1 come from the factors; each phase is then one launch
+    MW_TRY(lu_prepare(c, params, true));
+    MW_TRY(forward_program(c, params, x, false));             // Phase I
+    MW_TRY(loss_and_top(c, target, loss_out, true));
+    return phase2_program(c, params, g0, nullptr);            // Phase II
+  }
   if (use_programs(n)) {
     // each phase is one launch, and the inverse steps of all layers ride along in both
     // a workspace that kept its inverses: refresh them (one step) instead of starting over
@@ -1506,7 +1548,10 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
       }
       for (int i = 0; i < nchunks; ++i) {
         MW_TRY(tc_program_launch(progs[(size_t)i], c.st, c.s));
-        record_buckets(n, (i + 1) * chunk < L ? (i + 1) * chunk : L, c.s);
+        const int l1 = (i + 1) * chunk < L ? (i + 1) * chunk : L;
+        // LU-parameterised layers: the gradients of W just formed become those of the factors
+        if (n->opts.lu_param) MW_TRY(lu_map_gradients(c, params, dW, i * chunk, l1));
+        record_buckets(n, l1, c.s);
       }
       return MW_OK;
     }
@@ -1536,7 +1581,7 @@ mw_status tensor_forward_sweep(mw_net* n, const void* const* params, const void*
                                     (float*)dW[l - 1], l - 1);
     if (cnt) MW_TRY(run(c, g, cnt));
     // LU-parameterised layer: the gradient of W just formed becomes the gradient of the factors
-    if (n->opts.lu_param && l >= 1 && dW[l - 1]) MW_TRY(lu_map_gradient(c, params[l - 1], (float*)dW[l - 1]));
+    if (n->opts.lu_param && l >= 1) MW_TRY(lu_map_gradients(c, params, dW, l - 1, l));
     record_buckets(n, l, c.s);      // launch l carries the weight vjp of layer l - 1
   }
   return MW_OK;
@@ -1556,7 +1601,8 @@ mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, c
   MW_TRY(clear_split_counters(c));
   const bool programs = use_programs(n);
   if (programs) {
-    MW_TRY(split_all_weights(c, params));
+    if (n->opts.lu_param) MW_TRY(lu_prepare(c, params, false));
+    else MW_TRY(split_all_weights(c, params));
     MW_TRY(forward_program(c, params, x, true));
   } else {
     if (n->opts.lu_param) MW_TRY(lu_prepare(c, params, false));
@@ -1566,7 +1612,11 @@ mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, c
   const __nv_bfloat16* x0p = nullptr;
   if (n->opts.prec == MW_F32) x0p = c.at<__nv_bfloat16>(lay.xp[0]);   // split by the forward pass
   else x0p = (const __nv_bfloat16*)x;
-  if (programs) return backprop_program(c, params, x, dW, x0p);
+  if (programs) {
+    MW_TRY(backprop_program(c, params, x, dW, x0p));
+    if (n->opts.lu_param) MW_TRY(lu_map_gradients(c, params, dW, 0, L));
+    return MW_OK;
+  }
   int cur = 0;
   // one launch per layer: both vjps of layer l read the same g_z
   for (int l = L - 1; l >= 0; --l) {
@@ -1598,7 +1648,7 @@ mw_status tensor_backprop(mw_net* n, const void* const* params, const void* x, c
                          d, d, c.B, e, 2);
     }
     if (cnt) MW_TRY(run(c, g, cnt));
-    if (n->opts.lu_param && dW[l]) MW_TRY(lu_map_gradient(c, params[l], (float*)dW[l]));
+    if (n->opts.lu_param) MW_TRY(lu_map_gradients(c, params, dW, l, l + 1));
     cur ^= 1;
   }
   return MW_OK;
