@@ -43,6 +43,7 @@ struct Layout {
   // temporaries, the planes of one gradient, two fp32 products of the gradient's chain rule, and
   // the inverted diagonal blocks of every layer (fp32)
   Region lu_l, lu_u, lu_t, lu_s, lu_y[2], lu_g, lu_a, lu_b, lu_diag;
+  Region lu_table, lu_done;                  // product table and counters of the factor-preparation program
 };
 
 }  // namespace mw

@@ -22,6 +22,10 @@ struct TensorState {
   // (two variants: the inverses' current home)
   std::vector<TcProgram*> sweep[2];
   std::vector<const void*> sweep_key[2];
+  // LU-parameterised nets: the products that turn a chunk of layers' factors into W and W^-1
+  // ([0]: W only, for the backprop reference; [1]: both), one program per chunk of layers
+  std::vector<TcProgram*> lu_prog[2];
+  std::vector<std::vector<const void*>> lu_key[2];
 };
 
 // convolutional nets on the tensor cores (mw_conv_pipeline.cu): stride-1 same-size convolutions

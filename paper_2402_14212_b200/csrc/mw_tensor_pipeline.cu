@@ -415,6 +415,7 @@ mw_status clear_split_counters(const Ctx& c) {
 // term planes (fp32-accurate).  The gradient of W that the sweep forms is mapped to the factors
 // by the chain rule: dJ/dL = G U^T below the diagonal, dJ/dU = L^T G on and above it.
 constexpr int kLuBlock = 128;
+constexpr int kLuProgEntries = 256;   // products of one factor-preparation program
 
 __device__ __forceinline__ void split3(float v, __nv_bfloat16* p, int64_t stride) {
   const __nv_bfloat16 a = __float2bfloat16_rn(v);
@@ -433,27 +434,42 @@ lu_diag_inverse_kernel(PtrBatch Ps, int n, float* __restrict__ out, DeviceStatus
   const int blk = blockIdx.x, which = blockIdx.y, lay = blockIdx.z;
   const float* P = static_cast<const float*>(Ps.p[lay]);
   const int o = blk * kLuBlock, j = threadIdx.x, r = kLuBlock - 1;
-  // the block as a lower triangular matrix M: L's block itself (unit diagonal), or U's block with
-  // rows and columns reversed, M[i][k] = U[r-i][r-k], whose inverse is U^-1 reversed the same way
-  double x[kLuBlock];
+  // the block as a lower triangular matrix M in shared memory: L's block itself (unit diagonal),
+  // or U's block with rows and columns reversed, M[i][k] = U[r-i][r-k], whose inverse is U^-1
+  // reversed the same way
+  extern __shared__ float Msh[];                      // [kLuBlock][kLuBlock + 1]
+  for (int e = threadIdx.x; e < kLuBlock * kLuBlock; e += kLuBlock) {
+    const int i = e / kLuBlock, k = e - i * kLuBlock;
+    float v;
+    if (which == 0) v = k < i ? P[(int64_t)(o + i) * n + o + k] : (k == i ? 1.f : 0.f);
+    else v = k <= i ? P[(int64_t)(o + r - i) * n + o + r - k] : 0.f;
+    Msh[i * (kLuBlock + 1) + k] = v;
+  }
+  __syncthreads();
+  // thread j owns column j of the inverse: x_i = (delta_ij - sum_{k<i} M_ik x_k) / M_ii, with the
+  // sum carried as an fp32 pair (error-free product and sum) so the result is fp32-accurate
+  float x[kLuBlock];
   bool bad = false;
-  for (int i = 0; i < j; ++i) x[i] = 0.0;
-  for (int i = j; i < kLuBlock; ++i) {
-    double s = i == j ? 1.0 : 0.0;
+  for (int i = 0; i < kLuBlock; ++i) {
+    float hi = i == j ? 1.f : 0.f, lo = 0.f;
+    const float* row = Msh + i * (kLuBlock + 1);
     for (int k = j; k < i; ++k) {
-      const double m = which == 0 ? (double)P[(int64_t)(o + i) * n + o + k]
-                                  : (double)P[(int64_t)(o + r - i) * n + o + r - k];
-      s -= m * x[k];
+      const float m = row[k], p = -m * x[k];
+      const float pe = fmaf(-m, x[k], -p);            // exact product = p + pe
+      const float t = hi + p;
+      const float z = t - hi;
+      lo += (hi - (t - z)) + (p - z) + pe;            // two-sum remainder
+      hi = t;
     }
-    const double d = which == 0 ? 1.0 : (double)P[(int64_t)(o + r - i) * n + o + r - i];
-    if (!(d != 0.0) || !(d - d == 0.0)) { bad = true; x[i] = 0.0; }
-    else x[i] = s / d;
+    const float d = row[i];
+    if (!(d != 0.f) || !(d - d == 0.f)) { bad = true; x[i] = 0.f; }
+    else x[i] = i < j ? 0.f : (hi + lo) / d;
   }
   if (bad) record_error(st, MW_ERR_NOT_SUBMERSIVE, (unsigned)(layer0 + lay), (unsigned)blk, 5u, 0u);
   float* dst = out + (((int64_t)lay * 2 + which) * (n / kLuBlock) + blk) * kLuBlock * kLuBlock;
   for (int i = 0; i < kLuBlock; ++i) {
-    if (which == 0) dst[i * kLuBlock + j] = (float)x[i];
-    else dst[(r - i) * kLuBlock + (r - j)] = (float)x[i];
+    if (which == 0) dst[i * kLuBlock + j] = x[i];
+    else dst[(r - i) * kLuBlock + (r - j)] = x[i];
   }
 }
 
@@ -578,47 +594,114 @@ mw_status lu_prepare(const Ctx& c, const void* const* params, bool inverses) {
       if (inverses && lay.inv[l0 + g].off - lay.inv[l0 + g - 1].off != (size_t)(6 * c.nn)) return MW_ERR_WORKSPACE;
     }
     if (inverses) {
-      lu_diag_inverse_kernel<<<dim3((unsigned)nb, 2u, (unsigned)G), kLuBlock, 0, c.s>>>(ps, d, diag, c.st, l0);
+      constexpr size_t kDiagSmem = sizeof(float) * kLuBlock * (kLuBlock + 1);
+      static bool attr[16] = {};
+      int dev = 0;
+      MW_CUDA_OK(cudaGetDevice(&dev));
+      if (dev >= 0 && dev < 16 && !attr[dev]) {
+        MW_CUDA_OK(cudaFuncSetAttribute(lu_diag_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDiagSmem));
+        attr[dev] = true;
+      }
+      lu_diag_inverse_kernel<<<dim3((unsigned)nb, 2u, (unsigned)G), kLuBlock, kDiagSmem, c.s>>>(ps, d, diag, c.st, l0);
       MW_TRY(launch_ok());
     }
     lu_split_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(ps, d, Lp, Up, diag, Tp, Sp);
     MW_TRY(launch_ok());
     (void)diag_layer;
+    // the products of this chunk, in an order in which each comes after what it reads: `phase`
+    // numbers the sets of mutually independent ones, d0 / d1 name the products it waits for
+    struct Item { TcGemm g; int phase, d0, d1; };
+    std::vector<Item> items;
+    int phase = 0, top_l = -1, top_u = -1;
     if (inverses) {
-      // segments [seg[i], seg[i+1]) whose diagonal blocks of L^-1 and U^-1 are complete
-      std::vector<int> seg;
+      // segments [seg[i], seg[i+1]) whose diagonal blocks of L^-1 and U^-1 are complete, and the
+      // product that completed each (-1: a single block, inverted by lu_diag_inverse_kernel)
+      std::vector<int> seg, zl((size_t)nb, -1), zu((size_t)nb, -1);
       for (int b = 0; b <= nb; ++b) seg.push_back(b * kLuBlock);
       while (seg.size() > 2) {
-        std::vector<TcGemm> first, second;
-        std::vector<int> merged;
+        std::vector<int> merged, mzl, mzu;
+        std::vector<Item> second;
         merged.push_back(seg[0]);
+        const int first_index = (int)items.size();
+        int pairs = 0;
+        for (size_t i = 0; i + 2 < seg.size(); i += 2) ++pairs;
         for (size_t i = 0; i + 2 < seg.size(); i += 2) {
           const int a0 = seg[i], a1 = seg[i + 1], a2 = seg[i + 2], m1 = a1 - a0, m2 = a2 - a1;
+          const int yl = first_index + 2 * (int)(i / 2), yu = yl + 1;
           // L^-1[a1:a2, a0:a1] = -D^-1 C A^-1
-          first.push_back(lu_product(lu_block(c, Lp, a1, a0, m2, m1, false), lu_block(c, Tp, a0, a0, m1, m1, true),
-                                     m2, m1, m1, lu_block_out(c, Yl, a1, a0, 1.f), G));
-          second.push_back(lu_product(lu_block(c, Tp, a1, a1, m2, m2, false), lu_block(c, Yl, a1, a0, m2, m1, true),
-                                      m2, m1, m2, lu_block_out(c, Tp, a1, a0, -1.f), G));
+          items.push_back({lu_product(lu_block(c, Lp, a1, a0, m2, m1, false), lu_block(c, Tp, a0, a0, m1, m1, true),
+                                      m2, m1, m1, lu_block_out(c, Yl, a1, a0, 1.f), G), phase, zl[i], -1});
+          second.push_back({lu_product(lu_block(c, Tp, a1, a1, m2, m2, false), lu_block(c, Yl, a1, a0, m2, m1, true),
+                                       m2, m1, m2, lu_block_out(c, Tp, a1, a0, -1.f), G), phase + 1, yl, zl[i + 1]});
           // U^-1[a0:a1, a1:a2] = -A^-1 B D^-1
-          first.push_back(lu_product(lu_block(c, Up, a0, a1, m1, m2, false), lu_block(c, Sp, a1, a1, m2, m2, true),
-                                     m1, m2, m2, lu_block_out(c, Yu, a0, a1, 1.f), G));
-          second.push_back(lu_product(lu_block(c, Sp, a0, a0, m1, m1, false), lu_block(c, Yu, a0, a1, m1, m2, true),
-                                      m1, m2, m1, lu_block_out(c, Sp, a0, a1, -1.f), G));
+          items.push_back({lu_product(lu_block(c, Up, a0, a1, m1, m2, false), lu_block(c, Sp, a1, a1, m2, m2, true),
+                                      m1, m2, m2, lu_block_out(c, Yu, a0, a1, 1.f), G), phase, zu[i + 1], -1});
+          second.push_back({lu_product(lu_block(c, Sp, a0, a0, m1, m1, false), lu_block(c, Yu, a0, a1, m1, m2, true),
+                                       m1, m2, m1, lu_block_out(c, Sp, a0, a1, -1.f), G), phase + 1, yu, zu[i]});
           merged.push_back(a2);
+          // the merged segment is complete once its two second-stage products are
+          mzl.push_back(first_index + 2 * pairs + 2 * (int)(i / 2));
+          mzu.push_back(first_index + 2 * pairs + 2 * (int)(i / 2) + 1);
         }
-        if (merged.back() != seg.back()) merged.push_back(seg.back());   // an odd segment waits a level
-        MW_TRY(lu_run(c, first));
-        MW_TRY(lu_run(c, second));
+        if (merged.back() != seg.back()) {       // an odd segment waits a level
+          merged.push_back(seg.back());
+          mzl.push_back(zl[seg.size() - 2]);
+          mzu.push_back(zu[seg.size() - 2]);
+        }
+        for (const Item& it : second) items.push_back(it);
+        phase += 2;
         seg.swap(merged);
+        zl.swap(mzl);
+        zu.swap(mzu);
+      }
+      top_l = zl[0];
+      top_u = zu[0];
+    }
+    // W = L U and W^-1 = U^-1 L^-1 by blocks of rows: a block of rows of L ends at its diagonal
+    // block, one of U^-1 starts there, so each product runs over the K range that is not zero
+    const int bs = d % 256 == 0 ? 256 : kLuBlock;
+    for (int r0 = 0; r0 < d; r0 += bs) {
+      const int k1 = r0 + bs;
+      items.push_back({lu_product(lu_block(c, Lp, r0, 0, bs, k1, false), lu_block(c, Up, 0, 0, k1, d, true), bs, d, k1,
+                                  lu_block_out(c, c.at<__nv_bfloat16>(lay.w_planes[l0]), r0, 0, 1.f), G), phase, -1, -1});
+      if (inverses)
+        items.push_back({lu_product(lu_block(c, Sp, r0, r0, bs, d - r0, false), lu_block(c, Tp, r0, 0, d - r0, d, true),
+                                    bs, d, d - r0, lu_block_out(c, c.at<__nv_bfloat16>(lay.inv[l0]), r0, 0, 1.f), G),
+                         phase, top_l, top_u});
+    }
+    if ((int)items.size() <= kLuProgEntries) {
+      // one launch for the whole chunk: every product starts when the ones it reads are complete
+      TensorState* t = static_cast<TensorState*>(c.n->tc);
+      const int which = inverses ? 1 : 0;
+      const size_t ci = (size_t)(l0 / chunk);
+      if (t->lu_prog[which].size() <= ci) {
+        t->lu_prog[which].resize(ci + 1, nullptr);
+        t->lu_key[which].resize(ci + 1);
+      }
+      const std::vector<const void*> key = {c.ws, reinterpret_cast<const void*>((uintptr_t)G)};
+      if (!t->lu_prog[which][ci] || t->lu_key[which][ci] != key) {
+        if (!t->lu_prog[which][ci]) t->lu_prog[which][ci] = tc_program_create();
+        t->lu_key[which][ci].clear();
+        TcProgram* pr = t->lu_prog[which][ci];
+        tc_program_begin(pr, c.at<char>(lay.lu_table), c.at<unsigned int>(lay.lu_done), false);
+        for (const Item& it : items) {
+          const int deps[2] = {it.d0, it.d1};
+          mw_status st;
+          if (tc_program_add(pr, c.cache, it.g, deps, 2, &st, -1) < 0) return st;
+        }
+        t->lu_key[which][ci] = key;
+      }
+      MW_TRY(tc_program_launch(t->lu_prog[which][ci], c.st, c.s));
+    } else {
+      std::vector<TcGemm> same;
+      for (size_t i = 0; i < items.size(); ++i) {
+        same.push_back(items[i].g);
+        if (i + 1 == items.size() || items[i + 1].phase != items[i].phase) {
+          MW_TRY(lu_run(c, same));
+          same.clear();
+        }
       }
     }
-    std::vector<TcGemm> last;
-    last.push_back(lu_product(lu_block(c, Lp, 0, 0, d, d, false), lu_block(c, Up, 0, 0, d, d, true), d, d, d,
-                              lu_block_out(c, c.at<__nv_bfloat16>(lay.w_planes[l0]), 0, 0, 1.f), G));
-    if (inverses)
-      last.push_back(lu_product(lu_block(c, Sp, 0, 0, d, d, false), lu_block(c, Tp, 0, 0, d, d, true), d, d, d,
-                                lu_block_out(c, c.at<__nv_bfloat16>(lay.inv[l0]), 0, 0, 1.f), G));
-    MW_TRY(lu_run(c, last));
   }
   return MW_OK;
 }
@@ -648,15 +731,26 @@ mw_status lu_map_gradients(const Ctx& c, const void* const* params, void* const*
     MW_TRY(launch_ok());
     lu_gsplit_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(gs, c.nn, Gp);
     MW_TRY(launch_ok());
-    TcEpilogue ea, eb;
-    ea.mode = eb.mode = TC_EPI_PLAIN;
-    ea.out_f32 = c.at<float>(lay.lu_a);
-    eb.out_f32 = c.at<float>(lay.lu_b);
-    ea.bs_f32 = eb.bs_f32 = c.nn;
+    // Only the strictly lower part of G U^T and the upper part of L^T G are wanted, and U^T, L^T
+    // are triangular: by blocks of columns (rows), each product covers the wanted tiles and the K
+    // range that is not zero.
+    const int bs = d % 256 == 0 ? 256 : kLuBlock;
     std::vector<TcGemm> g;
-    // G U^T: B operand [N][K] = U itself;  L^T G: A operand MN-major = L as [K][M], B = G as [K][N]
-    g.push_back(lu_product(lu_block(c, Gp, 0, 0, d, d, false), lu_block(c, Up, 0, 0, d, d, false), d, d, d, ea, G));
-    g.push_back(lu_product(lu_block(c, Lp, 0, 0, d, d, true), lu_block(c, Gp, 0, 0, d, d, true), d, d, d, eb, G));
+    for (int o = 0; o < d; o += bs) {
+      const int rest = d - o;
+      TcEpilogue ea, eb;
+      ea.mode = eb.mode = TC_EPI_PLAIN;
+      ea.out_f32 = c.at<float>(lay.lu_a) + (int64_t)o * d + o;
+      eb.out_f32 = c.at<float>(lay.lu_b) + (int64_t)o * d + o;
+      ea.bs_f32 = eb.bs_f32 = c.nn;
+      ea.ld = eb.ld = d;
+      // (G U^T)[o:, o:o+bs]: B operand [N][K] = rows o.. of U from column o on
+      g.push_back(lu_product(lu_block(c, Gp, o, o, rest, rest, false), lu_block(c, Up, o, o, bs, rest, false),
+                             rest, bs, rest, ea, G));
+      // (L^T G)[o:o+bs, o:]: A operand MN-major = L[o:, o:o+bs] as [K][M], B = G[o:, o:] as [K][N]
+      g.push_back(lu_product(lu_block(c, Lp, o, o, rest, bs, true), lu_block(c, Gp, o, o, rest, rest, true),
+                             bs, rest, rest, eb, G));
+    }
     MW_TRY(lu_run(c, g));
     lu_combine_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(c.at<float>(lay.lu_a), c.at<float>(lay.lu_b), d, outs);
     MW_TRY(launch_ok());
@@ -1363,6 +1457,8 @@ void tensor_layout(mw_net* n, bool backprop, Layout& lay, size_t start) {
     lay.lu_g = b.take(6 * nn * G);
     lay.lu_a = b.take(4 * nn * G);
     lay.lu_b = b.take(4 * nn * G);
+    lay.lu_table = b.take(tc_program_table_bytes(kLuProgEntries));
+    lay.lu_done = b.take(sizeof(unsigned int) * (kLuProgEntries + 1));
     if (!backprop) {
       lay.lu_t = b.take(6 * nn * G);
       lay.lu_s = b.take(6 * nn * G);
@@ -1402,6 +1498,9 @@ void tensor_destroy(mw_net* n) {
         if (t->prog[i][v]) tc_program_destroy(t->prog[i][v]);
     for (int v = 0; v < 2; ++v)
       for (TcProgram* pr : t->sweep[v]) tc_program_destroy(pr);
+    for (int v = 0; v < 2; ++v)
+      for (TcProgram* pr : t->lu_prog[v])
+        if (pr) tc_program_destroy(pr);
     tc_cache_destroy(t->cache);
     delete t;
     n->tc = nullptr;

@@ -145,3 +145,22 @@ def test_calls_reject_null_and_small_workspace_without_touching_a_gpu():
     assert L.mw_pack_sign_bits(None, 1, 0, 4, None, None) == 0
     assert L.mw_pack_sign_bits(1, 7, 2, 4, 1, None) == 1
     assert L.mw_activation_vijp(1, 1, 2, 4, 1, 0.0, None, None, 1, None, None) == 1   # slope 0
+
+
+def test_net_create_lu_parameterised_layers():
+    lu = lambda n: S.Layer(S.DENSE, S.ACT_LEAKY, 0.1, n, n, lu=True)
+    net = mwb.Net([lu(256), lu(256)], 64, S.F32, S.LOSS_MSE_MEAN, backend="tensor")
+    mw_b, bp_b, _ = net.workspace_bytes()
+    assert mw_b > bp_b > 0
+    for bad in [dict(prec=S.BF16), dict(prec=S.F64), dict(backend="simt"), dict(resident_inverse=False),
+                dict(warm_inverse=True)]:
+        kw = dict(prec=S.F32, backend="tensor")
+        kw.update(bad)
+        prec = kw.pop("prec")
+        with pytest.raises(mwb.MwError) as e:
+            mwb.Net([lu(256)], 64, prec, S.LOSS_MSE_MEAN, **kw)
+        assert e.value.code == 2, bad
+    with pytest.raises(mwb.MwError):      # widths must be multiples of the 128-wide diagonal blocks
+        mwb.Net([lu(192)], 64, S.F32, S.LOSS_MSE_MEAN, backend="tensor")
+    with pytest.raises(ValueError):       # all layers or none
+        mwb.Net([lu(256), S.Layer(S.DENSE, S.ACT_LEAKY, 0.1, 256, 256)], 64, S.F32, S.LOSS_MSE_MEAN)
