@@ -126,7 +126,8 @@ typedef struct {
  * number of steps: it converges while sigma_max(W)^2 < 2 mean(sigma_i^2) and reaches working
  * precision in its default schedule when ||I - W X_0|| is about 0.15 or less, i.e. for weights
  * near a multiple of an orthogonal matrix (mw_net_opts.inverse_iters adds steps).  Outside that
- * domain the layer is reported per step as MW_ERR_NOT_SUBMERSIVE, never answered silently.
+ * domain the layer is reported per step as MW_ERR_NOT_SUBMERSIVE, never answered silently
+ * (mw_net_opts.lu_param parameterises the layers so that the inverse is exact instead).
  * Returns MW_ERR_UNSUPPORTED for
  * shapes outside: dense layers square; convolutions with C_in = C_out, either stride 1 with
  * k = 2*pad+1 (same size), or every layer of the net meeting Lemma 1 (i) with stride 2 (the

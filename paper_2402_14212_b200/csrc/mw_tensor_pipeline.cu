@@ -581,7 +581,6 @@ mw_status lu_prepare(const Ctx& c, const void* const* params, bool inverses) {
   __nv_bfloat16* Yl = inverses ? c.at<__nv_bfloat16>(lay.lu_y[0]) : nullptr;
   __nv_bfloat16* Yu = inverses ? c.at<__nv_bfloat16>(lay.lu_y[1]) : nullptr;
   float* diag = inverses ? c.at<float>(lay.lu_diag) : nullptr;
-  const int64_t diag_layer = 2 * (int64_t)nb * kLuBlock * kLuBlock;
   int64_t bx = (c.nn + 255) / 256;
   if (bx > 296) bx = 296;
   for (int l0 = 0; l0 < L; l0 += chunk) {
@@ -598,16 +597,16 @@ mw_status lu_prepare(const Ctx& c, const void* const* params, bool inverses) {
       static bool attr[16] = {};
       int dev = 0;
       MW_CUDA_OK(cudaGetDevice(&dev));
-      if (dev >= 0 && dev < 16 && !attr[dev]) {
+      const bool known = dev >= 0 && dev < 16;
+      if (!known || !attr[dev]) {     // the opt-in belongs to the device
         MW_CUDA_OK(cudaFuncSetAttribute(lu_diag_inverse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDiagSmem));
-        attr[dev] = true;
+        if (known) attr[dev] = true;
       }
       lu_diag_inverse_kernel<<<dim3((unsigned)nb, 2u, (unsigned)G), kLuBlock, kDiagSmem, c.s>>>(ps, d, diag, c.st, l0);
       MW_TRY(launch_ok());
     }
     lu_split_kernel<<<dim3((unsigned)bx, (unsigned)G), 256, 0, c.s>>>(ps, d, Lp, Up, diag, Tp, Sp);
     MW_TRY(launch_ok());
-    (void)diag_layer;
     // the products of this chunk, in an order in which each comes after what it reads: `phase`
     // numbers the sets of mutually independent ones, d0 / d1 name the products it waits for
     struct Item { TcGemm g; int phase, d0, d1; };

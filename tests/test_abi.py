@@ -52,6 +52,11 @@ def test_net_create_rejects_bad_descriptions():
     with pytest.raises(mwb.MwError):
         mwb.Net([S.Layer(S.CONV2D, S.ACT_LEAKY, 0.1, H=8, W=8, C_in=4, C_out=4, k=3, stride=2, pad=1)],
                 2, S.F32, S.LOSS_MSE_MEAN)
+    # a leaky-ReLU of slope 0 (or a non-finite slope) is not submersive: its vijp would divide by zero
+    for slope in (0.0, float("nan"), float("inf")):
+        with pytest.raises(mwb.MwError) as e:
+            mwb.Net([S.Layer(S.DENSE, S.ACT_LEAKY, slope, 8, 8)], 4, S.F64, S.LOSS_MSE_MEAN)
+        assert e.value.code == 2, slope
 
 
 def test_net_create_convolution_families():
