@@ -77,6 +77,7 @@ struct alignas(64) TcProblem {
   int M, N, K, num_kb, kb_per_split, split;
   int bn, tiles_n, tiles_mn, unit_begin, unit_count;
   int bm;                      // rows of one tile: 128, or 256 in the pair form
+  int sym;                     // 1: square symmetric result, tiles (mt, nt >= mt) only (see TcEpilogue::symmetric)
   int pa, pb, a_mn, b_mn, a_batch_planes, b_batch_planes;
   uint32_t b_tile_bytes, tx_bytes;   // per CTA: in the pair form a CTA stages half of the B tile
   // Layout of a stage (operands without a convolution window): every operand arrives with ONE
@@ -359,6 +360,7 @@ struct EpiOut {
   int row0 = 0;                      // first row of the warp's block
   int z = 0;                         // batch item
   uint32_t half = 0;                 // which 2 KB half the next block takes
+  bool mirror = false;               // symmetric product, off-diagonal tile: blocks are stored transposed too
 };
 
 __device__ __forceinline__ void bulk_wait_read_all() {
@@ -393,7 +395,7 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 // lanes of the warp take part; block (col0, eo.row0) of every plane).
 __device__ __forceinline__ void store_planes32(float (&v)[32], __nv_bfloat16* base, int planes,
                                                int64_t plane_stride, int64_t off, bool valid,
-                                               const CUtensorMap* map, EpiOut& eo, int col0) {
+                                               const CUtensorMap* map, EpiOut& eo, int col0, bool mirror = false) {
   const int lane = threadIdx.x & 31;
   for (int p = 0; p < planes; ++p) {
     uint32_t pk[16];
@@ -426,6 +428,26 @@ __device__ __forceinline__ void store_planes32(float (&v)[32], __nv_bfloat16* ba
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
     if (lane == 0) bulk_store_4d(map, tile, col0, eo.row0, p, eo.z);
+    if (mirror) {
+      // the same block transposed: value i of lane r is element (i, r); two-byte stores of a warp
+      // fill one 64-byte row, piece (r >> 3) of row i at (r >> 3) ^ ((i >> 1) & 3)
+      if (lane == 0) bulk_wait_read_but_one();
+      __syncwarp();
+      const uint32_t tt = eo.sbuf + eo.half * 2048u;
+      eo.half ^= 1u;
+      const uint32_t piece = (uint32_t)lane >> 3, inside = ((uint32_t)lane & 7u) * 2u;
+#pragma unroll
+      for (uint32_t i = 0; i < 16; ++i) {
+        const uint32_t r0 = 2u * i, r1 = 2u * i + 1u;
+        const uint32_t a0 = tt + r0 * 64u + ((piece ^ ((r0 >> 1) & 3u)) << 4) + inside;
+        const uint32_t a1 = tt + r1 * 64u + ((piece ^ ((r1 >> 1) & 3u)) << 4) + inside;
+        asm volatile("st.shared.b16 [%0], %1;" ::"r"(a0), "h"((unsigned short)(pk[i] & 0xffffu)) : "memory");
+        asm volatile("st.shared.b16 [%0], %1;" ::"r"(a1), "h"((unsigned short)(pk[i] >> 16)) : "memory");
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) bulk_store_4d(map, tt, eo.row0, col0, p, eo.z);
+    }
   }
 }
 
@@ -514,7 +536,9 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
         }
       }
       if (e.out_f32) store_f32x32(v, e.out_f32 + off, valid, eo, col0);
-      if (e.n_planes) store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0);
+      if (e.n_planes)
+        store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0,
+                       eo.mirror && eo.m_pl != nullptr);
       break;
     }
     case TC_EPI_FWD: {
@@ -692,13 +716,20 @@ __device__ __forceinline__ void decode_unit(const TcProblem* probs, const int* u
   const int ks = local - tl * P.split;
   const int z = tl / P.tiles_mn;
   const int r = tl - z * P.tiles_mn;
-  const int mt = r / P.tiles_n;
+  int mt = r / P.tiles_n, nt = r - mt * P.tiles_n;
+  if (P.sym) {
+    // tiles on and above the diagonal, row by row: row m has tiles_n - m of them
+    int t = r, len = P.tiles_n;
+    mt = 0;
+    while (t >= len) { t -= len; --len; ++mt; }
+    nt = mt + t;
+  }
   w.q = q;
   w.tl = tl;
   w.ks = ks;
   w.z = z;
   w.m0 = mt * P.bm;
-  w.n0 = (r - mt * P.tiles_n) * P.bn;
+  w.n0 = nt * P.bn;
   w.kb0 = ks * P.kb_per_split;
   const int e = w.kb0 + P.kb_per_split;
   w.kb1 = e < P.num_kb ? e : P.num_kb;
@@ -1064,6 +1095,7 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         eo.m_pl2 = (P.out_tma & 4) ? &P.tmP2 : nullptr;
         eo.row0 = row - lane;
         eo.z = w.z;
+        eo.mirror = kPair && P.sym && w.n0 != w.m0;
       }
       const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + set * (uint32_t)kSetCols;
       // sum of the column blocks of 32 accumulator columns starting at c
@@ -1661,6 +1693,13 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   const int tiles_m = (d.M + P.bm - 1) / P.bm;
   P.tiles_n = (d.N + P.bn - 1) / P.bn;
   P.tiles_mn = tiles_m * P.tiles_n;
+  // symmetric result (TcEpilogue::symmetric): square tiles of a square product, term planes only,
+  // stored by the copy engine (checked below, once the output maps are known)
+  P.sym = (pair && d.epi.symmetric && d.epi.mode == TC_EPI_RESID && d.epi.scale_dev && d.M == d.N && P.bn == P.bm &&
+           d.M % P.bm == 0 && split == 1 && d.batch == 1 && !d.epi.out_f32 && !d.epi.sumsq && d.epi.n_planes > 0 &&
+           d.A.base == d.B.base && g_bulk_epilogue && d.epi.remap_s == 0 && !d.epi.ld)
+              ? 1 : 0;
+  if (P.sym) P.tiles_mn = tiles_m * (tiles_m + 1) / 2;
   const int64_t units = (int64_t)P.tiles_mn * d.batch * split;
   if (units > (1 << 30)) return MW_ERR_UNSUPPORTED;
   P.unit_count = (int)units;
@@ -1691,6 +1730,12 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
                     &P.tmP2))
       P.out_tma |= 4;
   }
+  if (P.sym && !(P.out_tma & 2)) {     // no copy-engine path for the planes: the full product
+    P.sym = 0;
+    P.tiles_mn = tiles_m * P.tiles_n;
+    P.unit_count = P.tiles_mn * d.batch * split;
+  }
+  P.epi.symmetric = P.sym;
   P.split_partials = nullptr;
   P.split_counters = nullptr;
   if (split > 1) {
@@ -1720,7 +1765,9 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
     for (int b = 0; b < P.pb; ++b)
       if (a + b < t) ++np;
   *flops += 2.0 * d.M * d.N * d.K * d.batch;
-  *mma_flops += 2.0 * d.M * d.N * d.K * np * d.batch;
+  // (a symmetric product executes only its tiles on and above the diagonal)
+  const double done_share = P.sym ? (double)P.tiles_mn / ((double)P.tiles_n * P.tiles_n) : 1.0;
+  *mma_flops += 2.0 * d.M * d.N * d.K * np * d.batch * done_share;
   return MW_OK;
 }
 
@@ -1869,6 +1916,9 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
   prm.stages = stages;
   size_t smem = (size_t)stages * stage_bytes + 1024;
   prm.epi_stage_off = epi_stage_offset(stages, stage_bytes, &smem);
+  // a symmetric product mirrors its tiles through the epilogue's staging buffers
+  for (int i = 0; i < prm.nprob; ++i)
+    if (prm.prob[i].sym && !prm.epi_stage_off) return MW_ERR_UNSUPPORTED;
   const bool prof = g_prof.on;
   if (prof) {
     cudaEventRecord(prof_event(), s);
@@ -2046,6 +2096,9 @@ mw_status tc_program_launch(TcProgram* pr, DeviceStatus* st, cudaStream_t s) {
   prm.stages = stages;
   size_t smem = (size_t)stages * pr->stage_bytes + 1024;
   prm.epi_stage_off = epi_stage_offset(stages, pr->stage_bytes, &smem);
+  if (!prm.epi_stage_off)
+    for (const TcProblem& P : pr->table)
+      if (P.sym) return MW_ERR_UNSUPPORTED;   // (mirrors its tiles through the staging buffers)
   MW_TRY(ensure_kernel_attr());
   const bool prof = g_prof.on;
   if (prof) {

@@ -890,6 +890,7 @@ TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, con
       g.B = operand(W, d, d, pw, false);
       g.epi.mode = TC_EPI_RESID;
       g.epi.scale_dev = c.at<float>(lay.ns_scale) + l;
+      g.epi.symmetric = 1;    // W W^T: tiles on and above the diagonal, mirrored (where the kernel form allows)
       g.epi.planes = Rp; g.epi.n_planes = sched[0].pu; g.epi.plane_stride = c.nn;
     } else {
       int next_terms = c.pr.ph;
