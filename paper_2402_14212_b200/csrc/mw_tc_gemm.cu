@@ -1203,8 +1203,13 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
       if (epi.mode == TC_EPI_RESID && epi.sumsq && fused_step) {
         // this warp's share of ||v||_F^2 goes to a slot of its own (fixed-order sum by the reader)
         for (int o = 16; o; o >>= 1) sumsq_local += __shfl_xor_sync(0xffffffffu, sumsq_local, o);
-        if (lane == 0)
+        if (lane == 0) {
           epi.sumsq[((int64_t)(row >> 7) * P.tiles_n + w.n0 / bn) * kEpiWarps + quarter] = sumsq_local;
+          // symmetric product: the tile below the diagonal that this one stands for has the same sum
+          if (eo.mirror)
+            epi.sumsq[((int64_t)(2 * (w.n0 / bn) + (int)rank) * P.tiles_n + w.m0 / P.bm) * kEpiWarps + quarter] =
+                sumsq_local;
+        }
       }
       if (kProgram && fused_step) {
         // program launch: publish this warp's part of the tile to the products that wait for it
@@ -1695,9 +1700,9 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   P.tiles_mn = tiles_m * P.tiles_n;
   // symmetric result (TcEpilogue::symmetric): square tiles of a square product, term planes only,
   // stored by the copy engine (checked below, once the output maps are known)
-  P.sym = (pair && d.epi.symmetric && d.epi.mode == TC_EPI_RESID && d.epi.scale_dev && d.M == d.N && P.bn == P.bm &&
-           d.M % P.bm == 0 && split == 1 && d.batch == 1 && !d.epi.out_f32 && !d.epi.sumsq && d.epi.n_planes > 0 &&
-           d.A.base == d.B.base && g_bulk_epilogue && d.epi.remap_s == 0 && !d.epi.ld)
+  P.sym = (pair && d.epi.symmetric && d.epi.mode == TC_EPI_RESID && d.M == d.N && P.bn == P.bm &&
+           d.M % P.bm == 0 && split == 1 && d.batch == 1 && !d.epi.out_f32 && d.epi.n_planes > 0 &&
+           g_bulk_epilogue && d.epi.remap_s == 0 && !d.epi.ld)
               ? 1 : 0;
   if (P.sym) P.tiles_mn = tiles_m * (tiles_m + 1) / 2;
   const int64_t units = (int64_t)P.tiles_mn * d.batch * split;

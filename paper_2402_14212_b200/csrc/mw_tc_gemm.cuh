@@ -64,9 +64,10 @@ struct TcEpilogue {
   // TC_EPI_RESID: a scalar in device memory (one per batch item) that turns the residual of the
   // start X_0 = c W^T into the factor of the first Newton-Schulz step (see TC_EPI_RESID)
   const float* scale_dev = nullptr;
-  // TC_EPI_RESID with scale_dev, A and B the same square matrix: the result is symmetric.  With 1
-  // (pair form, term planes through the copy engine) only the tiles on and above the diagonal are
-  // computed and every off-diagonal tile is also stored transposed below it.
+  // TC_EPI_RESID of a square product whose result the caller knows to be symmetric (W W^T; W X for an
+  // iterate X = W^T p(W W^T)).  With 1 (pair form, term planes through the copy engine) only the
+  // tiles on and above the diagonal are computed and every off-diagonal tile is also stored
+  // transposed below it (its sum-of-squares pieces are written for both).
   int symmetric = 0;
   // TC_EPI_RESID: ||v||_F^2 in pieces, one slot per 128-row block, column tile and epilogue warp
   // (tc_sumsq_slots of them; each is written, none accumulated: the reader adds them in order)

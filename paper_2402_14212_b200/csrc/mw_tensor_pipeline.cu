@@ -911,6 +911,10 @@ TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, con
     g.B = operand(Xc, d, d, sched[it].pr, true);
     g.epi.mode = TC_EPI_RESID;
     g.epi.planes = Rp; g.epi.n_planes = sched[it].pu; g.epi.plane_stride = c.nn;
+    // Every iterate is X = W^T p(W W^T), so W X is symmetric up to the rounding of X's term planes:
+    // the residual is computed on and above the diagonal and mirrored.  (Not for a kept inverse
+    // that is being refreshed: it belongs to the previous W.)
+    g.epi.symmetric = warm ? 0 : 1;
     // only the last residual is gated (the update that follows squares it)
     if (last) g.epi.sumsq = nb.sumsq + (int64_t)l * (int64_t)gate_slots(d);
   } else {
