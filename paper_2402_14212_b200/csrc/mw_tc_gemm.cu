@@ -395,7 +395,8 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 // lanes of the warp take part; block (col0, eo.row0) of every plane).
 __device__ __forceinline__ void store_planes32(float (&v)[32], __nv_bfloat16* base, int planes,
                                                int64_t plane_stride, int64_t off, bool valid,
-                                               const CUtensorMap* map, EpiOut& eo, int col0, bool mirror = false) {
+                                               const CUtensorMap* map, EpiOut& eo, int col0, bool mirror = false,
+                                               int64_t off_t = 0, int64_t ld_t = 0) {
   const int lane = threadIdx.x & 31;
   for (int p = 0; p < planes; ++p) {
     uint32_t pk[16];
@@ -412,6 +413,16 @@ __device__ __forceinline__ void store_planes32(float (&v)[32], __nv_bfloat16* ba
         uint4* dst = reinterpret_cast<uint4*>(base + (int64_t)p * plane_stride + off);
 #pragma unroll
         for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+        if (mirror) {
+          // the same values transposed: value i of this lane's row is element (col0 + i, row); the
+          // lanes of a warp write consecutive two-byte elements of one row
+          unsigned short* dt = reinterpret_cast<unsigned short*>(base + (int64_t)p * plane_stride + off_t);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            dt[(int64_t)(2 * i) * ld_t] = (unsigned short)(pk[i] & 0xffffu);
+            dt[(int64_t)(2 * i + 1) * ld_t] = (unsigned short)(pk[i] >> 16);
+          }
+        }
       }
       continue;
     }
@@ -537,8 +548,8 @@ __device__ __forceinline__ void epilogue_chunk(const TcEpilogue& e, int N, int p
       }
       if (e.out_f32) store_f32x32(v, e.out_f32 + off, valid, eo, col0);
       if (e.n_planes)
-        store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0,
-                       eo.mirror && eo.m_pl != nullptr);
+        store_planes32(v, e.planes, e.n_planes, e.plane_stride, off, valid, eo.m_pl, eo, col0, eo.mirror,
+                       (int64_t)col0 * ldo + row, ldo);
       break;
     }
     case TC_EPI_FWD: {
@@ -718,11 +729,16 @@ __device__ __forceinline__ void decode_unit(const TcProblem* probs, const int* u
   const int r = tl - z * P.tiles_mn;
   int mt = r / P.tiles_n, nt = r - mt * P.tiles_n;
   if (P.sym) {
-    // tiles on and above the diagonal, row by row: row m has tiles_n - m of them
-    int t = r, len = P.tiles_n;
+    // tiles that reach the diagonal or lie above it, row by row: row m starts at the tile that
+    // holds column m * bm
+    int t = r;
     mt = 0;
-    while (t >= len) { t -= len; --len; ++mt; }
-    nt = mt + t;
+    for (;;) {
+      const int start = (mt * P.bm) / P.bn, len = P.tiles_n - start;
+      if (t < len) { nt = start + t; break; }
+      t -= len;
+      ++mt;
+    }
   }
   w.q = q;
   w.tl = tl;
@@ -1095,8 +1111,9 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         eo.m_pl2 = (P.out_tma & 4) ? &P.tmP2 : nullptr;
         eo.row0 = row - lane;
         eo.z = w.z;
-        eo.mirror = kPair && P.sym && w.n0 != w.m0;
       }
+      // symmetric product: a tile that lies wholly above the diagonal stands for its mirror image too
+      eo.mirror = P.sym && w.n0 >= w.m0 + P.bm;
       const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + set * (uint32_t)kSetCols;
       // sum of the column blocks of 32 accumulator columns starting at c
       auto load_chunk = [&](int c, float (&v)[32]) {
@@ -1206,9 +1223,15 @@ tc_group_kernel(const __grid_constant__ TcGroupParams p) {
         if (lane == 0) {
           epi.sumsq[((int64_t)(row >> 7) * P.tiles_n + w.n0 / bn) * kEpiWarps + quarter] = sumsq_local;
           // symmetric product: the tile below the diagonal that this one stands for has the same sum
-          if (eo.mirror)
-            epi.sumsq[((int64_t)(2 * (w.n0 / bn) + (int)rank) * P.tiles_n + w.m0 / P.bm) * kEpiWarps + quarter] =
-                sumsq_local;
+          // (pair form: written to that tile's slots; one-CTA form: counted twice here, the slots of
+          // the tiles that are left out stay as the caller zeroed them)
+          if (eo.mirror) {
+            if (kPair)
+              epi.sumsq[((int64_t)(2 * (w.n0 / bn) + (int)rank) * P.tiles_n + w.m0 / P.bm) * kEpiWarps + quarter] =
+                  sumsq_local;
+            else
+              epi.sumsq[((int64_t)(row >> 7) * P.tiles_n + w.n0 / bn) * kEpiWarps + quarter] = 2.0 * sumsq_local;
+          }
         }
       }
       if (kProgram && fused_step) {
@@ -1700,11 +1723,14 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
   P.tiles_mn = tiles_m * P.tiles_n;
   // symmetric result (TcEpilogue::symmetric): square tiles of a square product, term planes only,
   // stored by the copy engine (checked below, once the output maps are known)
-  P.sym = (pair && d.epi.symmetric && d.epi.mode == TC_EPI_RESID && d.M == d.N && P.bn == P.bm &&
-           d.M % P.bm == 0 && split == 1 && d.batch == 1 && !d.epi.out_f32 && d.epi.n_planes > 0 &&
-           g_bulk_epilogue && d.epi.remap_s == 0 && !d.epi.ld)
+  P.sym = (d.epi.symmetric && d.epi.mode == TC_EPI_RESID && d.M == d.N && d.M % P.bm == 0 && d.N % P.bn == 0 &&
+           (!pair || (P.bn == P.bm && g_bulk_epilogue)) && cv.mode == TC_CONV_NONE && split == 1 && d.batch == 1 &&
+           !d.epi.out_f32 && d.epi.n_planes > 0 && d.epi.remap_s == 0 && !d.epi.ld)
               ? 1 : 0;
-  if (P.sym) P.tiles_mn = tiles_m * (tiles_m + 1) / 2;
+  if (P.sym) {
+    P.tiles_mn = 0;
+    for (int m = 0; m < tiles_m; ++m) P.tiles_mn += P.tiles_n - (m * P.bm) / P.bn;
+  }
   const int64_t units = (int64_t)P.tiles_mn * d.batch * split;
   if (units > (1 << 30)) return MW_ERR_UNSUPPORTED;
   P.unit_count = (int)units;
@@ -1735,7 +1761,7 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
                     &P.tmP2))
       P.out_tma |= 4;
   }
-  if (P.sym && !(P.out_tma & 2)) {     // no copy-engine path for the planes: the full product
+  if (P.sym && pair && !(P.out_tma & 2)) {     // pair form without a copy-engine path for the planes: the full product
     P.sym = 0;
     P.tiles_mn = tiles_m * P.tiles_n;
     P.unit_count = P.tiles_mn * d.batch * split;
@@ -1771,7 +1797,7 @@ static mw_status setup_problem(TcMapCache* cache, const TcGemm& d, TcProblem& P,
       if (a + b < t) ++np;
   *flops += 2.0 * d.M * d.N * d.K * d.batch;
   // (a symmetric product executes only its tiles on and above the diagonal)
-  const double done_share = P.sym ? (double)P.tiles_mn / ((double)P.tiles_n * P.tiles_n) : 1.0;
+  const double done_share = P.sym ? (double)P.tiles_mn / ((double)tiles_m * P.tiles_n) : 1.0;
   *mma_flops += 2.0 * d.M * d.N * d.K * np * d.batch * done_share;
   return MW_OK;
 }
@@ -1923,7 +1949,7 @@ mw_status tc_gemm_group(TcMapCache* cache, const TcGemm* g, int count, DeviceSta
   prm.epi_stage_off = epi_stage_offset(stages, stage_bytes, &smem);
   // a symmetric product mirrors its tiles through the epilogue's staging buffers
   for (int i = 0; i < prm.nprob; ++i)
-    if (prm.prob[i].sym && !prm.epi_stage_off) return MW_ERR_UNSUPPORTED;
+    if (pair && prm.prob[i].sym && !prm.epi_stage_off) return MW_ERR_UNSUPPORTED;
   const bool prof = g_prof.on;
   if (prof) {
     cudaEventRecord(prof_event(), s);
@@ -2101,7 +2127,7 @@ mw_status tc_program_launch(TcProgram* pr, DeviceStatus* st, cudaStream_t s) {
   prm.stages = stages;
   size_t smem = (size_t)stages * pr->stage_bytes + 1024;
   prm.epi_stage_off = epi_stage_offset(stages, pr->stage_bytes, &smem);
-  if (!prm.epi_stage_off)
+  if (pr->pair && !prm.epi_stage_off)
     for (const TcProblem& P : pr->table)
       if (P.sym) return MW_ERR_UNSUPPORTED;   // (mirrors its tiles through the staging buffers)
   MW_TRY(ensure_kernel_attr());

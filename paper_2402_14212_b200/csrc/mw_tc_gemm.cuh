@@ -65,9 +65,10 @@ struct TcEpilogue {
   // start X_0 = c W^T into the factor of the first Newton-Schulz step (see TC_EPI_RESID)
   const float* scale_dev = nullptr;
   // TC_EPI_RESID of a square product whose result the caller knows to be symmetric (W W^T; W X for an
-  // iterate X = W^T p(W W^T)).  With 1 (pair form, term planes through the copy engine) only the
-  // tiles on and above the diagonal are computed and every off-diagonal tile is also stored
-  // transposed below it (its sum-of-squares pieces are written for both).
+  // iterate X = W^T p(W W^T)).  With 1 only the tiles that reach the diagonal or lie above it are
+  // computed, and every tile wholly above it is also stored transposed below it (pair form: through
+  // the copy engine).  Its sum-of-squares pieces count for both; in the one-CTA form the pieces of
+  // the tiles that are left out are never written: the caller zeroes `sumsq` first.
   int symmetric = 0;
   // TC_EPI_RESID: ||v||_F^2 in pieces, one slot per 128-row block, column tile and epilogue warp
   // (tc_sumsq_slots of them; each is written, none accumulated: the reader adds them in order)

@@ -911,10 +911,14 @@ TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, con
     g.B = operand(Xc, d, d, sched[it].pr, true);
     g.epi.mode = TC_EPI_RESID;
     g.epi.planes = Rp; g.epi.n_planes = sched[it].pu; g.epi.plane_stride = c.nn;
-    // Every iterate is X = W^T p(W W^T), so W X is symmetric up to the rounding of X's term planes:
-    // the residual is computed on and above the diagonal and mirrored.  (Not for a kept inverse
-    // that is being refreshed: it belongs to the previous W.)
-    g.epi.symmetric = warm ? 0 : 1;
+    // bf16 nets: X_1 = W^T T is W^T times a polynomial of W W^T, so W X_1 is symmetric up to the
+    // rounding of X_1's term planes (2^-17): the residual of the second step is computed on and
+    // above the diagonal and mirrored.  Not where that form is broken (measured: gradient errors
+    // of 2e-4 to 5e-3 in fp32 when the asymmetric part is dropped): fp32 nets, whose first step
+    // reads W rounded to one term (W round(W)^T is not symmetric); later iterates, which went
+    // through an update with fewer terms, X + round(X) round(R); a kept inverse that is being
+    // refreshed for a new W.
+    g.epi.symmetric = (!warm && it == 1 && c.n->opts.prec != MW_F32) ? 1 : 0;
     // only the last residual is gated (the update that follows squares it)
     if (last) g.epi.sumsq = nb.sumsq + (int64_t)l * (int64_t)gate_slots(d);
   } else {
@@ -1541,6 +1545,8 @@ mw_status tensor_input_cotangent(mw_net* n, const void* const* params, const voi
     if (feed.steps < 1) return MW_ERR_INVALID_ARG;
     MW_TRY(split_all_weights(c, params));
     if (!warm) MW_TRY(ns_prepare_all(c, params));
+    // (a symmetric residual product on single CTAs leaves the pieces of its left-out tiles unwritten)
+    MW_CUDA_OK(cudaMemsetAsync(c.at<char>(lay.ns_sumsq), 0, lay.ns_sumsq.bytes, s));
     MW_TRY(forward_program(c, params, x, false, &feed));      // Phase I
     MW_TRY(loss_and_top(c, target, loss_out, true));
     MW_TRY(phase2_program(c, params, g0, &feed));             // Phase II
