@@ -138,3 +138,13 @@ def test_bucket_events_and_single_rank_data_parallel_step(kind):
     again = net.forward_sweep(params, x, g0, ws)
     for a, b in zip(plain, again):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("prec,n,batch,iters,tol", [(S.BF16, 512, 256, 3, 2e-2), (S.F32, 256, 64, 4, 1e-4),
+                                                   (S.BF16, 512, 256, 1, 6e-2)])
+def test_inverse_iters_changes_the_newton_schulz_schedule(prec, n, batch, iters, tol):
+    """More steps than the default repeat the most accurate one (their residuals are computed in
+    full: only the second step's is symmetric); a single step leaves the start's squared residual
+    (about 4e-3 for these weights), which the looser bar allows for."""
+    p = S.sweep_mlp(seed=8, depth=4, n=n, batch=batch, reseed_every=2, prec=prec)
+    check_problem(p, tol, backend="tensor", inverse_iters=iters, exact_masks=False, tau=tol)
