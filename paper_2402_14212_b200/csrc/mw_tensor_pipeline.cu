@@ -275,10 +275,18 @@ mw_status weight_planes(const Ctx& c, int l, const void* W, bool make, const __n
 // W^-1 of layers [l0, l0+G) into their inverse regions as `ph` term planes (row-major
 // X = W^-1), all G layers advancing together in batched launches.  Also leaves the split weight
 // planes of those layers in w_planes (MW_F32).
+mw_status newton_schulz_single(const Ctx& c, int l, const void* const* params);
+
 mw_status newton_schulz_group(const Ctx& c, int l0, int G, const void* const* params) {
   const Layout& lay = *c.lay;
   const int d = c.dim;
   const bool f32 = c.n->opts.prec == MW_F32;
+  // bf16 layers whose products fill the GPU on their own gain nothing from batching: one at a time,
+  // with the cheaper product list of newton_schulz_single
+  if (!f32 && (G == 1 || d >= 2048)) {
+    for (int g = 0; g < G; ++g) MW_TRY(newton_schulz_single(c, l0 + g, params));
+    return MW_OK;
+  }
   float* X = c.at<float>(lay.ns_x);                             // [G][n*n]
   __nv_bfloat16* Rp = c.at<__nv_bfloat16>(lay.ns_r);            // [G][3][n*n]
   __nv_bfloat16* Xp[2] = {Rp + (int64_t)3 * G * c.nn, Rp + (int64_t)6 * G * c.nn};
@@ -867,16 +875,17 @@ mw_status ns_prepare_all(const Ctx& c, const void* const* params) {
 
 // product `stage` of layer l: even = residual R = I - W X of step stage/2, odd = its update
 // (the iterate alternates between its two homes Xp[0], Xp[1]; step `it` reads home side0 + it)
-TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, const NsStep* sched,
-                  int steps, int side0, bool warm) {
+// (`nb`, `lb`, `scale`: the iterate's buffers, the layer's index inside them and its start scale;
+// the program path keeps them per layer, the one-layer-at-a-time path has one set)
+TcGemm ns_product_at(const Ctx& c, int l, const NsBuffers& nb, int lb, const float* scale, int stage,
+                     const void* const* params, const NsStep* sched, int steps, int side0, bool warm) {
   const Layout& lay = *c.lay;
   const int d = c.dim, it = stage >> 1, cur = (side0 + it) & 1;
   const bool last = it + 1 == steps;
-  const NsBuffers nb = ns_buffers(c);
-  float* X = nb.X + (int64_t)l * c.nn;
-  __nv_bfloat16* Rp = nb.Rp + (int64_t)l * 3 * c.nn;
-  __nv_bfloat16* Xc = nb.Xp[cur] + (int64_t)l * 3 * c.nn;
-  __nv_bfloat16* Xn = nb.Xp[cur ^ 1] + (int64_t)l * 3 * c.nn;
+  float* X = nb.X + (int64_t)lb * c.nn;
+  __nv_bfloat16* Rp = nb.Rp + (int64_t)lb * 3 * c.nn;
+  __nv_bfloat16* Xc = nb.Xp[cur] + (int64_t)lb * 3 * c.nn;
+  __nv_bfloat16* Xn = nb.Xp[cur ^ 1] + (int64_t)lb * 3 * c.nn;
   TcGemm g;
   g.M = d; g.N = d; g.K = d;
   g.wide_tiles = 1;      // throughput work beside the latency-bound chains
@@ -889,7 +898,7 @@ TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, con
       g.A = operand(W, d, d, pw, false);
       g.B = operand(W, d, d, pw, false);
       g.epi.mode = TC_EPI_RESID;
-      g.epi.scale_dev = c.at<float>(lay.ns_scale) + l;
+      g.epi.scale_dev = scale;
       g.epi.symmetric = 1;    // W W^T: tiles on and above the diagonal, mirrored (where the kernel form allows)
       g.epi.planes = Rp; g.epi.n_planes = sched[0].pu; g.epi.plane_stride = c.nn;
     } else {
@@ -920,7 +929,7 @@ TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, con
     // refreshed for a new W.
     g.epi.symmetric = (!warm && it == 1 && c.n->opts.prec != MW_F32) ? 1 : 0;
     // only the last residual is gated (the update that follows squares it)
-    if (last) g.epi.sumsq = nb.sumsq + (int64_t)l * (int64_t)gate_slots(d);
+    if (last) g.epi.sumsq = nb.sumsq + (int64_t)lb * (int64_t)gate_slots(d);
   } else {
     int next_terms = c.pr.ph;
     if (!last) next_terms = sched[it + 1].pr > sched[it + 1].pu ? sched[it + 1].pr : sched[it + 1].pu;
@@ -935,6 +944,54 @@ TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, con
     g.epi.plane_stride = c.nn;
   }
   return g;
+}
+
+TcGemm ns_product(const Ctx& c, int l, int stage, const void* const* params, const NsStep* sched,
+                  int steps, int side0, bool warm) {
+  return ns_product_at(c, l, ns_buffers(c), l, c.at<float>(c.lay->ns_scale) + l, stage, params, sched, steps,
+                       side0, warm);
+}
+
+// One bf16 layer at a time (transient inverse slot, or a net too deep for the product tables): the
+// same products as the program path -- implicit start, symmetric W W^T and second residual --
+// as single launches, the last update writing the term planes the sweep reads.
+mw_status newton_schulz_single(const Ctx& c, int l, const void* const* params) {
+  const Layout& lay = *c.lay;
+  const int d = c.dim;
+  NsStep sched[16];
+  const int steps = ns_schedule(c.n, sched);
+  if (steps < 1) return MW_ERR_INVALID_ARG;
+  char* sc = c.at<char>(lay.inv_scratch);
+  float* cscale = reinterpret_cast<float*>(sc + 8 * kMaxGroup);
+  double* fpart = reinterpret_cast<double*>(sc + 12 * kMaxGroup + 64);
+  NsBuffers nb;
+  nb.X = c.at<float>(lay.ns_x);
+  nb.Rp = c.at<__nv_bfloat16>(lay.ns_r);
+  nb.Xp[0] = nb.Rp + 3 * c.nn;
+  nb.Xp[1] = nb.Rp + 6 * c.nn;
+  nb.sumsq = c.at<double>(lay.ns_sumsq);
+  PtrBatch wp{};
+  wp.p[0] = params[l];
+  frob_partial_kernel<__nv_bfloat16><<<dim3(kFrobBlocks, 1), 256, 0, c.s>>>(wp, c.nn, fpart);
+  frob_final_kernel<<<1, kMaxGroup, 0, c.s>>>(fpart, 1, d, cscale);
+  MW_TRY(launch_ok(2));
+  MW_CUDA_OK(cudaMemsetAsync(nb.sumsq, 0, sizeof(double) * gate_slots(d), c.s));
+  for (int stage = 0; stage < 2 * steps; ++stage) {
+    TcGemm g = ns_product_at(c, l, nb, 0, cscale, stage, params, sched, steps, 0, false);
+    const bool last_update = stage == 2 * steps - 1;
+    if (last_update) g.epi.planes = c.at<__nv_bfloat16>(lay.inv[l]);
+    MW_TRY(run(c, &g, 1));
+    if (stage == 2 * (steps - 1) && steps > 1) {
+      // the update squares this residual: gate on it so a diverging layer is reported
+      const NsStep lastst = sched[steps - 1];
+      const int pw = c.pr.pw < lastst.pr ? c.pr.pw : lastst.pr;
+      residual_gate_kernel<<<1, 256, 0, c.s>>>(nb.sumsq, (int64_t)gate_slots(d),
+                                               (int64_t)tc_sumsq_slots(pw, lastst.pr, d, d, tc_pair_ok(pw, lastst.pr, d, d)),
+                                               d, 2e-2, c.st, l);
+      MW_TRY(launch_ok());
+    }
+  }
+  return MW_OK;
 }
 
 // the inverse steps handed out to the chain steps of Phase I and Phase II, in step-major order

@@ -148,3 +148,12 @@ def test_inverse_iters_changes_the_newton_schulz_schedule(prec, n, batch, iters,
     (about 4e-3 for these weights), which the looser bar allows for."""
     p = S.sweep_mlp(seed=8, depth=4, n=n, batch=batch, reseed_every=2, prec=prec)
     check_problem(p, tol, backend="tensor", inverse_iters=iters, exact_masks=False, tau=tol)
+
+
+@pytest.mark.parametrize("n,batch", [(256, 256), (512, 96), (768, 512)])
+def test_bf16_transient_inverse_slot(n, batch):
+    """resident_inverse = 0 on bf16 nets: one inverse slot, each layer's W^-1 rebuilt in the sweep by
+    single launches of the same products the program path uses (implicit start, symmetric W W^T
+    and second residual), on CTA pairs or single CTAs as the sizes allow."""
+    p = S.mixed_mlp(seed=9, depth=6, n=n, batch=batch, reseed_every=3, prec=S.BF16)
+    check_problem(p, 2e-2, backend="tensor", resident=False, exact_masks=False, tau=2e-2)
