@@ -157,3 +157,11 @@ def test_bf16_transient_inverse_slot(n, batch):
     and second residual), on CTA pairs or single CTAs as the sizes allow."""
     p = S.mixed_mlp(seed=9, depth=6, n=n, batch=batch, reseed_every=3, prec=S.BF16)
     check_problem(p, 2e-2, backend="tensor", resident=False, exact_masks=False, tau=2e-2)
+
+
+def test_bf16_net_deeper_than_the_product_tables():
+    """154 layers of width 2048 do not fit the tables of the program launches: every phase runs as a
+    launch per layer, and the resident inverses are built one layer at a time."""
+    p = S.mixed_mlp(seed=10, depth=154, n=2048, batch=256, reseed_every=4, prec=S.BF16)
+    out, ref, errs = check_problem(p, 2e-2, backend="tensor", exact_masks=False, tau=2e-2)
+    assert len(errs) == 154
